@@ -1,0 +1,332 @@
+"""fp64 CPU oracle for Hadamard Linear Attention (HLA).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain reference the CUDA
+library is checked against.  Only the tests, the smoke check and the CPU-baseline
+leg of the benchmark may import it; the product path never does.  It shares no
+code, tables or helpers with the CUDA sources and imports nothing from the
+package.
+
+Everything is numpy float64 and works on ONE head at a time:
+
+    q      [N, d_phi]      query features  phi_q(q_i)            (>= 0 for the normaliser)
+    ks     list of F arrays [N, d_phi]     key features phi_{k_f}(k_j)
+    v      [N, d]          values
+    o      [N, d]          attention output
+
+Two independent forms of the same operator are implemented:
+
+  * the literal quadratic definition (paper Eq. "hla", Section 4.1): the F
+    similarity matrices are multiplied elementwise, rows are normalised, and the
+    result multiplies V;
+  * the factored linear-time scheme (Lemma 4.1, Theorem 4.2, the normaliser
+    paragraph after it, and the 2-/3-factor einsum listings of the appendix):
+    per-token outer-product tensors T_k, T_q, the context tensor C = T_k (x)_1 V,
+    the key-side sum z, eta = T_q . z, and the readout T_q (x) C;
+
+plus the sequential-update recurrence (Eq. "seq.updates") for the state, analytic
+gradients in both forms, and the feature networks phi of the appendix
+("Defining phi": Linear - GELU - Linear - optional ReLU).
+
+Readings of points the paper leaves open (the same readings the CUDA library
+takes):
+  * eps is added to the normaliser before dividing: o = num / (eta + eps)
+    (the listings write `eta + eps`; the value of eps is not given - it is an argument here).
+  * The division is applied to the contracted numerator; the listings divide the
+    query outer products first, which is the same up to rounding.
+  * eta_i = sum_j A_ij = T_q[i] . sum_j T_k[j]  (the listings' `sum_over_k`); the
+    displayed formula for eta in the text is garbled.
+  * In the theorem's proof the summed token index is the key/value index j.
+  * The P = d_phi**F features of a token are flattened with the FIRST factor's
+    index slowest (the listings' `bhsdef -> view(dp**3)`).
+  * phi: exact (erf) GELU, both Linear layers have a bias, hidden width = d,
+    ReLU applied at the end for phi_q and phi_k.  The figure defining phi is
+    missing from the text, so the phi functions here are PARITY UNPINNED by the
+    paper beyond that verbal description; they are pinned only against
+    math.erf, a pure-Python loop version and finite differences.
+"""
+from __future__ import annotations
+
+import numpy as np
+from scipy.special import erf as _erf
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------- #
+# Feature networks phi (appendix "Defining phi"; Algorithm 1 step 4)
+# --------------------------------------------------------------------------- #
+def gelu_erf(x):
+    """GELU(x) = x * Phi(x) with the exact normal CDF Phi(x) = (1 + erf(x / sqrt 2)) / 2."""
+    x = np.asarray(x, dtype=F64)
+    return 0.5 * x * (1.0 + _erf(x / np.sqrt(2.0)))
+
+
+def gelu_erf_grad(x):
+    """d/dx GELU(x) = Phi(x) + x * pdf(x)."""
+    x = np.asarray(x, dtype=F64)
+    cdf = 0.5 * (1.0 + _erf(x / np.sqrt(2.0)))
+    pdf = np.exp(-0.5 * x * x) / np.sqrt(2.0 * np.pi)
+    return cdf + x * pdf
+
+
+def phi_mlp(x, W1, b1, W2, b2, relu=True):
+    """Feature map of the appendix: two Linear layers with a GELU in between and
+    a final ReLU (which the normaliser's non-negativity requirement needs).
+
+    x [N, d];  W1 [d, d_hidden] (input index first), b1 [d_hidden];
+    W2 [d_hidden, d_phi], b2 [d_phi].  Returns features [N, d_phi].
+    """
+    x = np.asarray(x, F64)
+    h = x @ np.asarray(W1, F64) + np.asarray(b1, F64)       # first Linear
+    g = gelu_erf(h)                                          # GELU
+    p = g @ np.asarray(W2, F64) + np.asarray(b2, F64)       # second Linear
+    return np.maximum(p, 0.0) if relu else p
+
+
+def phi_mlp_backward(x, W1, b1, W2, b2, dfeat, relu=True):
+    """Gradient of sum(dfeat * phi_mlp(x)) with respect to x (weights held fixed)."""
+    x = np.asarray(x, F64)
+    W1 = np.asarray(W1, F64)
+    W2 = np.asarray(W2, F64)
+    h = x @ W1 + np.asarray(b1, F64)
+    g = gelu_erf(h)
+    p = g @ W2 + np.asarray(b2, F64)
+    dp = np.asarray(dfeat, F64) * (p > 0.0) if relu else np.asarray(dfeat, F64)
+    dg = dp @ W2.T
+    dh = dg * gelu_erf_grad(h)
+    return dh @ W1.T
+
+
+# --------------------------------------------------------------------------- #
+# Outer-product tensors T_q, T_k (paragraph before Theorem 4.2)
+# --------------------------------------------------------------------------- #
+def outer_features(vectors):
+    """[T]_j = vectors[0][j] (x) vectors[1][j] (x) ... flattened to [N, d_phi**F],
+    first factor's index slowest."""
+    t = np.asarray(vectors[0], F64)
+    n = t.shape[0]
+    for r in vectors[1:]:
+        r = np.asarray(r, F64)
+        t = np.einsum("np,ne->npe", t, r).reshape(n, -1)
+    return t
+
+
+# --------------------------------------------------------------------------- #
+# Form 1: the literal quadratic definition (Eq. "hla")
+# --------------------------------------------------------------------------- #
+def similarity_matrices(q, ks):
+    """s^f = phi_q(Q) phi_{k_f}(K)^T, one N x N matrix per factor."""
+    q = np.asarray(q, F64)
+    return [q @ np.asarray(k, F64).T for k in ks]
+
+
+def attention_matrix(q, ks):
+    """A = s^1 (.) s^2 (.) ... : the Hadamard product of the F similarity matrices."""
+    s = similarity_matrices(q, ks)
+    A = s[0].copy()
+    for sf in s[1:]:
+        A = A * sf
+    return A
+
+
+def hla_quadratic(q, ks, v, eps):
+    """o_i = (sum_j A_ij v_j) / (sum_j A_ij + eps).  Returns (o, eta)."""
+    A = attention_matrix(q, ks)
+    eta = A.sum(axis=1)
+    num = A @ np.asarray(v, F64)
+    return num / (eta + eps)[:, None], eta
+
+
+def hla_quadratic_rows(q_rows, ks, v, eps):
+    """The definition evaluated for a subset of query rows only (the definition is
+    separable over query rows).  q_rows [m, d_phi]."""
+    return hla_quadratic(q_rows, ks, v, eps)
+
+
+# --------------------------------------------------------------------------- #
+# Form 2: the factored linear-time scheme (Theorem 4.2 + listings)
+# --------------------------------------------------------------------------- #
+def context_state(ks, v):
+    """C = T_k (x)_1 V  in  R^{P x d}  and  z = sum_j [T_k]_j  in R^P."""
+    Tk = outer_features(ks)
+    C = np.einsum("jp,jg->pg", Tk, np.asarray(v, F64))
+    z = Tk.sum(axis=0)
+    return C, z
+
+
+def context_state_streaming(ks, v):
+    """The same state by the sequential update C^i = C^{i-1} + T_{k_i} (x) v_i."""
+    Tk = outer_features(ks)
+    v = np.asarray(v, F64)
+    C = np.zeros((Tk.shape[1], v.shape[1]), F64)
+    z = np.zeros(Tk.shape[1], F64)
+    for i in range(Tk.shape[0]):
+        C = C + np.multiply.outer(Tk[i], v[i])
+        z = z + Tk[i]
+    return C, z
+
+
+def readout(q, F, C, z, eps):
+    """o = (T_q (x) C) / (T_q . z + eps).  Returns (o, eta)."""
+    Tq = outer_features([q] * F)
+    eta = Tq @ z
+    num = Tq @ C
+    return num / (eta + eps)[:, None], eta
+
+
+def hla_factored(q, ks, v, eps):
+    """Linear-time HLA: state build then query readout.  Returns (o, eta, C, z)."""
+    C, z = context_state(ks, v)
+    o, eta = readout(q, len(ks), C, z, eps)
+    return o, eta, C, z
+
+
+# --------------------------------------------------------------------------- #
+# Gradients (the paper trains through the operator; the formulas below are the
+# derivatives of the two forms above)
+# --------------------------------------------------------------------------- #
+def hla_quadratic_backward(q, ks, v, do, eps):
+    """Gradients of L = sum(do * o) through the quadratic form.
+    Returns (dq [N,d_phi], dks list of [N,d_phi], dv [N,d])."""
+    q = np.asarray(q, F64)
+    ks = [np.asarray(k, F64) for k in ks]
+    v = np.asarray(v, F64)
+    do = np.asarray(do, F64)
+    s = similarity_matrices(q, ks)
+    A = attention_matrix(q, ks)
+    eta = A.sum(axis=1)
+    r = 1.0 / (eta + eps)
+    o = (A @ v) * r[:, None]
+    # dL/dA_ij = r_i * do_i . (v_j - o_i)
+    dA = r[:, None] * (do @ v.T - np.sum(do * o, axis=1)[:, None])
+    dv = (A * r[:, None]).T @ do
+    dq = np.zeros_like(q)
+    dks = []
+    for f in range(len(ks)):
+        others = np.ones_like(A)
+        for f2 in range(len(ks)):
+            if f2 != f:
+                others = others * s[f2]
+        ds = dA * others                      # dL/ds^f_ij
+        dq += ds @ ks[f]
+        dks.append(ds.T @ q)
+    return dq, dks, dv
+
+
+def _slot_contract(dT, vectors, slot):
+    """sum over all tensor indices except `slot` of dT[j, i_1..i_F] * prod_{f != slot} vectors[f][j, i_f].
+    dT is [N, d_phi**F] (first factor slowest); returns [N, d_phi]."""
+    Fn = len(vectors)
+    n, dphi = vectors[0].shape
+    letters = "abcdefgh"[:Fn]
+    t = dT.reshape((n,) + (dphi,) * Fn)
+    operands = [t]
+    subs = ["n" + letters]
+    for f in range(Fn):
+        if f != slot:
+            operands.append(np.asarray(vectors[f], F64))
+            subs.append("n" + letters[f])
+    return np.einsum(",".join(subs) + "->n" + letters[slot], *operands)
+
+
+def hla_factored_backward(q, ks, v, do, eps):
+    """Gradients of L = sum(do * o) through the factored form (two passes:
+    one over the queries that also reduces dC, dz; one over the keys).
+    Returns (dq, dks, dv)."""
+    q = np.asarray(q, F64)
+    ks = [np.asarray(k, F64) for k in ks]
+    v = np.asarray(v, F64)
+    do = np.asarray(do, F64)
+    Fn = len(ks)
+    Tk = outer_features(ks)
+    Tq = outer_features([q] * Fn)
+    C = Tk.T @ v
+    z = Tk.sum(axis=0)
+    eta = Tq @ z
+    r = 1.0 / (eta + eps)
+    o = (Tq @ C) * r[:, None]
+    dnum = do * r[:, None]
+    deta = -r * np.sum(do * o, axis=1)
+    # pass over the queries
+    dC = Tq.T @ dnum
+    dz = Tq.T @ deta
+    dTq = dnum @ C.T + np.multiply.outer(deta, z)
+    dq = np.zeros_like(q)
+    for slot in range(Fn):                    # the same vector sits in every slot of T_q
+        dq += _slot_contract(dTq, [q] * Fn, slot)
+    # pass over the keys
+    dv = Tk @ dC
+    dTk = v @ dC.T + dz[None, :]
+    dks = [_slot_contract(dTk, ks, f) for f in range(Fn)]
+    return dq, dks, dv
+
+
+# --------------------------------------------------------------------------- #
+# Whole-operator wrappers over [B, H, N, *] tensors (Algorithm 1 steps 4-5)
+# --------------------------------------------------------------------------- #
+def hla_core_forward(qf, kf, V, eps, form="factored"):
+    """qf [B,H,N,d_phi], kf [B,H,F,N,d_phi], V [B,H,N,d] -> (O [B,H,N,d], eta [B,H,N])."""
+    B, H, N, _ = qf.shape
+    Fn = kf.shape[2]
+    O = np.empty(V.shape, F64)
+    ETA = np.empty((B, H, N), F64)
+    for b in range(B):
+        for h in range(H):
+            ks = [kf[b, h, f] for f in range(Fn)]
+            if form == "quadratic":
+                o, eta = hla_quadratic(qf[b, h], ks, V[b, h], eps)
+            else:
+                o, eta, _, _ = hla_factored(qf[b, h], ks, V[b, h], eps)
+            O[b, h] = o
+            ETA[b, h] = eta
+    return O, ETA
+
+
+def hla_core_backward(qf, kf, V, dO, eps, form="factored"):
+    """Gradients of sum(dO * O) w.r.t. qf, kf, V (same shapes as the inputs)."""
+    B, H, N, _ = qf.shape
+    Fn = kf.shape[2]
+    dqf = np.empty(qf.shape, F64)
+    dkf = np.empty(kf.shape, F64)
+    dV = np.empty(V.shape, F64)
+    fn = hla_quadratic_backward if form == "quadratic" else hla_factored_backward
+    for b in range(B):
+        for h in range(H):
+            ks = [kf[b, h, f] for f in range(Fn)]
+            dq, dks, dv = fn(qf[b, h], ks, V[b, h], dO[b, h], eps)
+            dqf[b, h] = dq
+            for f in range(Fn):
+                dkf[b, h, f] = dks[f]
+            dV[b, h] = dv
+    return dqf, dkf, dV
+
+
+def phi_features(Q, K, phi_q, phi_k):
+    """Algorithm 1 step 4: q <- hla_to_q(q); k_f <- hla_to_k_f(k), one weight set
+    per map shared by all batches and heads.  phi_q = (W1,b1,W2,b2); phi_k = list of F such tuples.
+    Q, K [B,H,N,d] -> qf [B,H,N,d_phi], kf [B,H,F,N,d_phi]."""
+    B, H, N, d = Q.shape
+    qf = phi_mlp(Q.reshape(-1, d), *phi_q).reshape(B, H, N, -1)
+    kfs = [phi_mlp(K.reshape(-1, d), *w).reshape(B, H, N, -1) for w in phi_k]
+    return qf, np.stack(kfs, axis=2)
+
+
+def hla_forward(Q, K, V, phi_q, phi_k, eps, form="factored"):
+    """Steps 4-5 of Algorithm 1 on raw per-head Q, K, V [B,H,N,d].
+    Returns (O, eta, qf, kf)."""
+    qf, kf = phi_features(Q, K, phi_q, phi_k)
+    O, eta = hla_core_forward(qf, kf, V, eps, form)
+    return O, eta, qf, kf
+
+
+def hla_backward(Q, K, V, dO, phi_q, phi_k, eps, form="factored"):
+    """Gradients of sum(dO * O) w.r.t. raw Q, K, V through phi and the core.
+    Returns (dQ, dK, dV, dqf, dkf)."""
+    B, H, N, d = Q.shape
+    qf, kf = phi_features(Q, K, phi_q, phi_k)
+    dqf, dkf, dV = hla_core_backward(qf, kf, V, dO, eps, form)
+    dQ = phi_mlp_backward(Q.reshape(-1, d), *phi_q, dqf.reshape(-1, dqf.shape[-1])).reshape(Q.shape)
+    dK = np.zeros(K.shape, F64)
+    for f, w in enumerate(phi_k):             # the same K feeds every key map
+        dK += phi_mlp_backward(K.reshape(-1, d), *w, dkf[:, :, f].reshape(-1, dkf.shape[-1])).reshape(K.shape)
+    return dQ, dK, dV, dqf, dkf

@@ -1,0 +1,312 @@
+"""Pins for the fp64 oracle: every check compares it with something other than
+itself - the paper's identities, closed forms, brute force in pure Python,
+textbook special cases, finite differences, and the FLOP counts the paper prints."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import hla_oracle as orc
+from paper_2602_12128_b200 import flops
+
+RNG = np.random.default_rng(1234)
+
+
+def feats(n, dphi, F, rng=RNG):
+    q = np.abs(rng.standard_normal((n, dphi)))
+    ks = [np.abs(rng.standard_normal((n, dphi))) for _ in range(F)]
+    return q, ks
+
+
+# ---- Lemma 4.1 --------------------------------------------------------------
+@pytest.mark.parametrize("F", [1, 2, 3, 4])
+def test_lemma_4_1_outer_products(F):
+    """prod_f (q . r^f) == sum over all entries of (q x..x q) (.) (r^1 x..x r^F)."""
+    dphi = 5
+    q = RNG.standard_normal((7, dphi))
+    rs = [RNG.standard_normal((7, dphi)) for _ in range(F)]
+    lhs = np.ones(7)
+    for r in rs:
+        lhs *= np.sum(q * r, axis=1)
+    rhs = np.sum(orc.outer_features([q] * F) * orc.outer_features(rs), axis=1)
+    np.testing.assert_allclose(rhs, lhs, rtol=1e-12, atol=1e-13)
+
+
+def test_outer_features_index_order():
+    """First factor's index is the slowest one in the flattened feature axis."""
+    a = np.array([[1.0, 10.0]])
+    b = np.array([[2.0, 3.0]])
+    c = np.array([[5.0, 7.0]])
+    t = orc.outer_features([a, b, c])[0]
+    want = [a[0, i] * b[0, j] * c[0, k] for i in range(2) for j in range(2) for k in range(2)]
+    np.testing.assert_allclose(t, want)
+
+
+# ---- equality of the forms (Theorem 4.2, sequential updates) ------------------
+@pytest.mark.parametrize("F,dphi", [(1, 8), (2, 12), (3, 6), (2, 3)])
+def test_quadratic_equals_factored_equals_streaming(F, dphi):
+    n, d = 37, 9
+    q, ks = feats(n, dphi, F)
+    v = RNG.standard_normal((n, d))
+    eps = 1e-6
+    o1, eta1 = orc.hla_quadratic(q, ks, v, eps)
+    o2, eta2, C, z = orc.hla_factored(q, ks, v, eps)
+    Cs, zs = orc.context_state_streaming(ks, v)
+    np.testing.assert_allclose(o2, o1, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(eta2, eta1, rtol=1e-12)
+    np.testing.assert_allclose(Cs, C, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(zs, z, rtol=1e-12)
+    assert C.shape == (dphi ** F, d)
+
+
+# ---- brute force in pure Python -----------------------------------------------
+def brute_force(q, ks, v, eps):
+    n, d = len(v), len(v[0])
+    out = [[0.0] * d for _ in range(n)]
+    for i in range(n):
+        w = []
+        for j in range(n):
+            a = 1.0
+            for k in ks:
+                a *= sum(q[i][t] * k[j][t] for t in range(len(q[i])))
+            w.append(a)
+        eta = sum(w)
+        for g in range(d):
+            out[i][g] = sum(w[j] * v[j][g] for j in range(n)) / (eta + eps)
+    return np.array(out)
+
+
+@pytest.mark.parametrize("F", [2, 3])
+def test_brute_force_tiny(F):
+    n, dphi, d = 6, 3, 4
+    q, ks = feats(n, dphi, F)
+    v = RNG.standard_normal((n, d))
+    want = brute_force(q.tolist(), [k.tolist() for k in ks], v.tolist(), 1e-3)
+    np.testing.assert_allclose(orc.hla_quadratic(q, ks, v, 1e-3)[0], want, rtol=1e-12)
+    np.testing.assert_allclose(orc.hla_factored(q, ks, v, 1e-3)[0], want, rtol=1e-11)
+
+
+def test_brute_force_state_entries():
+    """C[(a,b,c), g] = sum_j k1_j[a] k2_j[b] k3_j[c] v_j[g] by explicit loops."""
+    n, dphi, d = 5, 3, 2
+    _, ks = feats(n, dphi, 3)
+    v = RNG.standard_normal((n, d))
+    C, z = orc.context_state(ks, v)
+    for a, b, c in itertools.product(range(dphi), repeat=3):
+        p = (a * dphi + b) * dphi + c
+        zz = sum(ks[0][j, a] * ks[1][j, b] * ks[2][j, c] for j in range(n))
+        assert abs(z[p] - zz) < 1e-12
+        for g in range(d):
+            cc = sum(ks[0][j, a] * ks[1][j, b] * ks[2][j, c] * v[j, g] for j in range(n))
+            assert abs(C[p, g] - cc) < 1e-12
+
+
+def test_one_hot_features_group_mean():
+    """With one-hot features A is a 0/1 matrix and o_i is the mean of V over the
+    keys that share the query's class in every factor."""
+    n, dphi, d = 12, 3, 5
+    cls_q = RNG.integers(0, dphi, n)
+    cls_k = [RNG.integers(0, dphi, n) for _ in range(3)]
+    eye = np.eye(dphi)
+    q = eye[cls_q]
+    ks = [eye[c] for c in cls_k]
+    v = RNG.standard_normal((n, d))
+    o, eta = orc.hla_factored(q, ks, v, 0.0 + 1e-300)[:2]
+    for i in range(n):
+        members = [j for j in range(n) if all(c[j] == cls_q[i] for c in cls_k)]
+        assert eta[i] == len(members)
+        if members:
+            np.testing.assert_allclose(o[i], v[members].mean(axis=0), rtol=1e-12, atol=1e-14)
+
+
+# ---- special cases ---------------------------------------------------------------
+def test_F1_is_normalised_linear_attention():
+    n, dphi, d = 50, 8, 6
+    q, ks = feats(n, dphi, 1)
+    v = RNG.standard_normal((n, d))
+    want = (q @ (ks[0].T @ v)) / (q @ ks[0].sum(axis=0))[:, None]       # phi(Q)(phi(K)^T V) / (phi(Q) . sum phi(K))
+    np.testing.assert_allclose(orc.hla_factored(q, ks, v, 0.0)[0], want, rtol=1e-12)
+    np.testing.assert_allclose(orc.hla_quadratic(q, ks, v, 0.0)[0], want, rtol=1e-12)
+
+
+@pytest.mark.parametrize("F", [2, 3])
+def test_equal_key_maps_give_elementwise_power(F):
+    n, dphi = 20, 4
+    q, ks = feats(n, dphi, 1)
+    A = orc.attention_matrix(q, ks * F)
+    np.testing.assert_allclose(A, (q @ ks[0].T) ** F, rtol=1e-12)
+
+
+def test_rank_bound():
+    """rank(A) <= min(N, d_phi^F) (rank relaxation paragraph)."""
+    n, dphi, F = 40, 2, 3
+    q, ks = feats(n, dphi, F)
+    A = orc.attention_matrix(q, ks)
+    assert np.linalg.matrix_rank(A, tol=1e-9) <= dphi ** F
+
+
+# ---- normaliser invariants ----------------------------------------------------------
+def test_rows_sum_to_one_and_convexity():
+    n, dphi, d, F = 33, 6, 7, 3
+    q, ks = feats(n, dphi, F)
+    eps = 1e-6
+    ones = np.ones((n, d))
+    o, eta = orc.hla_factored(q, ks, ones, eps)[:2]
+    np.testing.assert_allclose(o, np.repeat((eta / (eta + eps))[:, None], d, 1), rtol=1e-12)
+    v = RNG.standard_normal((n, d))
+    o = orc.hla_factored(q, ks, v, 0.0)[0]
+    assert np.all(o <= v.max(axis=0) + 1e-12) and np.all(o >= v.min(axis=0) - 1e-12)
+    W = orc.attention_matrix(q, ks)
+    W = W / W.sum(axis=1, keepdims=True)
+    np.testing.assert_allclose(W.sum(axis=1), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(W @ v, o, rtol=1e-10, atol=1e-13)
+
+
+def test_symmetries():
+    n, dphi, d, F = 21, 4, 5, 3
+    q, ks = feats(n, dphi, F)
+    v = RNG.standard_normal((n, d))
+    o = orc.hla_factored(q, ks, v, 0.0)[0]
+    perm = RNG.permutation(n)
+    np.testing.assert_allclose(orc.hla_factored(q, [k[perm] for k in ks], v[perm], 0.0)[0], o, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(orc.hla_factored(q[perm], ks, v, 0.0)[0], o[perm], rtol=1e-12)
+    scale = np.abs(RNG.standard_normal((n, 1))) + 0.5
+    np.testing.assert_allclose(orc.hla_factored(q * scale, ks, v, 0.0)[0], o, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(orc.hla_factored(q, [ks[0], 3.0 * ks[1], ks[2]], v, 0.0)[0], o, rtol=1e-11, atol=1e-13)
+
+
+# ---- gradients -------------------------------------------------------------------------
+def fd_grad(fun, x, h=1e-6):
+    g = np.zeros_like(x)
+    it = np.nditer(x, flags=["multi_index"])
+    for _ in it:
+        idx = it.multi_index
+        xp = x.copy(); xp[idx] += h
+        xm = x.copy(); xm[idx] -= h
+        g[idx] = (fun(xp) - fun(xm)) / (2 * h)
+    return g
+
+
+@pytest.mark.parametrize("F,dphi", [(2, 3), (3, 3), (3, 2)])
+@pytest.mark.parametrize("form", ["quadratic", "factored"])
+def test_core_gradients_finite_differences(F, dphi, form):
+    n, d = 9, 4
+    rng = np.random.default_rng(7)
+    q = np.abs(rng.standard_normal((n, dphi))) + 0.1
+    ks = [np.abs(rng.standard_normal((n, dphi))) + 0.1 for _ in range(F)]
+    v = rng.standard_normal((n, d))
+    do = rng.standard_normal((n, d))
+    eps = 1e-2
+    bw = orc.hla_quadratic_backward if form == "quadratic" else orc.hla_factored_backward
+    dq, dks, dv = bw(q, ks, v, do, eps)
+
+    def loss(q_=q, ks_=ks, v_=v):
+        return float(np.sum(do * orc.hla_quadratic(q_, ks_, v_, eps)[0]))
+
+    np.testing.assert_allclose(dq, fd_grad(lambda x: loss(q_=x), q), rtol=1e-6, atol=1e-8)
+    np.testing.assert_allclose(dv, fd_grad(lambda x: loss(v_=x), v), rtol=1e-6, atol=1e-8)
+    for f in range(F):
+        def lf(x, f=f):
+            kk = list(ks); kk[f] = x
+            return loss(ks_=kk)
+        np.testing.assert_allclose(dks[f], fd_grad(lf, ks[f]), rtol=1e-6, atol=1e-8)
+
+
+def test_backward_forms_agree_and_scale_identities():
+    n, dphi, d, F = 40, 6, 8, 3
+    q, ks = feats(n, dphi, F)
+    v = RNG.standard_normal((n, d))
+    do = RNG.standard_normal((n, d))
+    g1 = orc.hla_quadratic_backward(q, ks, v, do, 0.0)
+    g2 = orc.hla_factored_backward(q, ks, v, do, 0.0)
+    np.testing.assert_allclose(g2[0], g1[0], rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(g2[2], g1[2], rtol=1e-9, atol=1e-12)
+    for f in range(F):
+        np.testing.assert_allclose(g2[1][f], g1[1][f], rtol=1e-9, atol=1e-12)
+    # o is invariant to rescaling a query or a whole key map (eps = 0) -> Euler identities
+    np.testing.assert_allclose(np.sum(q * g1[0], axis=1), 0.0, atol=1e-10)
+    for f in range(F):
+        assert abs(np.sum(ks[f] * g1[1][f])) < 1e-9
+    # rows of the normalised weights sum to one -> sum_j dV_j = sum_i dO_i
+    np.testing.assert_allclose(g1[2].sum(axis=0), do.sum(axis=0), rtol=1e-10)
+
+
+# ---- phi networks ------------------------------------------------------------------------
+def test_gelu_against_math_erf_and_known_values():
+    xs = np.linspace(-6, 6, 97)
+    want = [0.5 * x * (1.0 + math.erf(x / math.sqrt(2.0))) for x in xs]
+    np.testing.assert_allclose(orc.gelu_erf(xs), want, rtol=1e-14, atol=1e-16)
+    assert orc.gelu_erf(0.0) == 0.0
+    assert abs(orc.gelu_erf(1.0) - 0.8413447460685429) < 1e-15      # Phi(1)
+    assert abs(orc.gelu_erf(-1.0) + 0.15865525393145707) < 1e-15    # -Phi(-1)
+    assert abs(orc.gelu_erf(10.0) - 10.0) < 1e-12
+
+
+def test_phi_mlp_against_python_loops_and_fd():
+    rng = np.random.default_rng(3)
+    n, d, dphi = 4, 5, 3
+    x = rng.standard_normal((n, d))
+    W1 = rng.standard_normal((d, d)); b1 = rng.standard_normal(d)
+    W2 = rng.standard_normal((d, dphi)); b2 = rng.standard_normal(dphi)
+    got = orc.phi_mlp(x, W1, b1, W2, b2)
+    for t in range(n):
+        h = [sum(x[t, i] * W1[i, j] for i in range(d)) + b1[j] for j in range(d)]
+        g = [0.5 * a * (1.0 + math.erf(a / math.sqrt(2.0))) for a in h]
+        p = [sum(g[j] * W2[j, o] for j in range(d)) + b2[o] for o in range(dphi)]
+        np.testing.assert_allclose(got[t], [max(a, 0.0) for a in p], rtol=1e-13, atol=1e-15)
+    assert np.all(got >= 0) and np.any(got == 0) and np.any(got > 0)
+    dfeat = rng.standard_normal((n, dphi))
+    dx = orc.phi_mlp_backward(x, W1, b1, W2, b2, dfeat)
+    fd = fd_grad(lambda xx: float(np.sum(dfeat * orc.phi_mlp(xx, W1, b1, W2, b2))), x)
+    np.testing.assert_allclose(dx, fd, rtol=1e-6, atol=1e-8)
+
+
+def test_full_operator_gradients_fd():
+    """dQ, dK, dV through phi and the core against central differences (tiny sizes;
+    the seed keeps every ReLU pre-activation away from its kink)."""
+    rng = np.random.default_rng(11)
+    B, H, N, d, dphi, F = 1, 2, 6, 4, 2, 3
+    Q = rng.standard_normal((B, H, N, d)); K = rng.standard_normal((B, H, N, d))
+    V = rng.standard_normal((B, H, N, d)); dO = rng.standard_normal((B, H, N, d))
+    mk = lambda: (rng.standard_normal((d, d)), rng.standard_normal(d), rng.standard_normal((d, dphi)), rng.standard_normal(dphi) + 0.5)
+    phi_q, phi_k = mk(), [mk() for _ in range(F)]
+    eps = 1e-3
+    dQ, dK, dV, _, _ = orc.hla_backward(Q, K, V, dO, phi_q, phi_k, eps)
+    loss = lambda Q_=Q, K_=K, V_=V: float(np.sum(dO * orc.hla_forward(Q_, K_, V_, phi_q, phi_k, eps, "quadratic")[0]))
+    np.testing.assert_allclose(dQ, fd_grad(lambda x: loss(Q_=x), Q, 1e-6), rtol=2e-5, atol=1e-8)
+    np.testing.assert_allclose(dK, fd_grad(lambda x: loss(K_=x), K, 1e-6), rtol=2e-5, atol=1e-8)
+    np.testing.assert_allclose(dV, fd_grad(lambda x: loss(V_=x), V, 1e-6), rtol=2e-5, atol=1e-8)
+
+
+# ---- FLOP model against the paper's tables ---------------------------------------------------
+def load_golden():
+    path = os.path.join(os.path.dirname(__file__), "golden", "paper_flop_tables.txt")
+    out = {}
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            k, val = line.split()[:2]
+            out[k] = float(val)
+    return out
+
+
+def test_flop_model_matches_paper_tables():
+    gold = load_golden()
+    T = 1e12
+    H, d = 12, 128
+    l3 = {n: flops.paper_layer_flops(n, H, d, 3, 6)["total"] / T for n in (12600, 32760)}
+    l2 = flops.paper_layer_flops(32760, H, d, 2, 12)["total"] / T
+    qd = {n: flops.quadratic_layer_flops(n, H, d) / T for n in (12600, 32760)}
+    assert abs(qd[12600] - gold["quadratic_layer_12600"]) < 0.006
+    assert abs(qd[32760] - gold["quadratic_layer_32760"]) < 0.006
+    assert abs(l3[12600] - gold["hla3f_layer_12600"]) < 0.006
+    assert abs(l3[32760] - gold["hla3f_layer_32760"]) < 0.006
+    # whole model = quadratic model - (#HLA blocks) * (quadratic layer - HLA layer)
+    assert abs(gold["wan_model_32760"] - 21 * (qd[32760] - l3[32760]) - gold["hla3f_r1_21_model"]) < 0.05
+    assert abs(gold["wan_model_32760"] - 10 * (qd[32760] - l3[32760]) - gold["hla3f_r1_10_model"]) < 0.05
+    assert abs(gold["wan_model_12600"] - 15 * (qd[12600] - l3[12600]) - gold["hla3f_r2_15_model"]) < 0.05
+    assert abs(gold["wan_model_32760"] - 21 * (qd[32760] - l2) - gold["hla2f_r1_21_model"]) < 0.05
+    # the operator core is d_phi^F features against d channels
+    assert flops.n_features(3, 6) == 216 and flops.n_features(2, 12) == 144
+    assert flops.core_fwd_flops_per_token(128, 3, 6) == 111456
