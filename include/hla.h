@@ -1,0 +1,150 @@
+/*
+ * hla.h - C ABI of the B200 (sm_100a) Hadamard Linear Attention operator.
+ *
+ * The operator is the linear-time form of HLA (paper Section 4.2, Lemma 4.1 and
+ * Theorem 4.2, the normaliser paragraph after it, Algorithm 1 steps 4-5 and the
+ * 2-/3-factor einsum listings of the appendix):
+ *
+ *     q_i   = phi_q(Q_i),   k^f_j = phi_{k_f}(K_j),  f = 1..F      (Algorithm 1 step 4)
+ *     T_k[j] = k^1_j (x) ... (x) k^F_j,   T_q[i] = q_i (x) ... (x) q_i     in R^P, P = d_phi^F
+ *     C = sum_j T_k[j] v_j^T  (P x d),    z = sum_j T_k[j]               (state build)
+ *     eta_i = T_q[i] . z,    o_i = (T_q[i]^T C) / (eta_i + eps)          (readout + normaliser)
+ *
+ * which equals row-normalising A = (.)_f phi_q(Q) phi_{k_f}(K)^T (Eq. "hla") and
+ * multiplying by V.  The backward entry point returns the gradients of
+ * sum(dO * O) with respect to the inputs.
+ *
+ * General rules
+ *   - All tensor pointers are DEVICE pointers, contiguous, innermost dimension
+ *     last, 16-byte aligned.  The caller owns every buffer, including the
+ *     workspace and the phi weights; the library allocates no device memory and
+ *     borrows pointers only for the work it enqueues.
+ *   - hla_ctx is host memory owned by the library (hla_create / hla_destroy).
+ *   - hla_forward / hla_backward only enqueue work on `cuda_stream` (a
+ *     cudaStream_t passed as void*; NULL = default stream) and return without
+ *     synchronising.  They never throw, abort or print: every failure is a
+ *     return code, and arguments are validated before anything is launched.
+ *   - Device-side waits are bounded; a wait that runs out makes the kernel
+ *     record a code in the workspace and return.  hla_last_device_status reads it.
+ *   - One ctx must not be used from two host threads at once.
+ */
+#ifndef HLA_H_
+#define HLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hla_ctx hla_ctx;
+
+typedef enum {
+    HLA_OK = 0,
+    HLA_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, non-positive size, bad enum   */
+    HLA_ERR_UNSUPPORTED = 2,   /* valid request outside the supported set (see hla_config)  */
+    HLA_ERR_WORKSPACE = 3,     /* workspace smaller than hla_workspace_bytes()              */
+    HLA_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                        */
+    HLA_ERR_DEVICE_TIMEOUT = 5 /* a bounded device-side wait expired (results are invalid)  */
+} hla_status;
+
+typedef enum { HLA_BF16 = 0, HLA_F32 = 1 } hla_dtype;
+
+typedef enum {
+    HLA_PHI_MLP = 0, /* Q, K are raw per-head tensors [B,H,N,d]; the library applies phi_q, phi_k1..F  */
+    HLA_PHI_NONE = 1 /* Q is q_phi [B,H,N,d_phi] fp32, K is k_phi [B,H,F,N,d_phi] fp32 (the listings'
+                        signature: features are given, must be >= 0 for the normaliser to make sense) */
+} hla_phi_mode;
+
+/*
+ * Problem statement.  V, O, dO, dV (and Q, K, dQ, dK in HLA_PHI_MLP mode) are
+ * [B,H,N,d] in `dtype`.  Features (HLA_PHI_NONE inputs and their gradients) are
+ * always fp32.  Supported set: F in {1,2,3,4}, d_phi^F <= 256, d <= 128 and
+ * d % 4 == 0, causal == 0.  dtype bf16 with d in {64,128} and (F,d_phi) in
+ * {(3,6),(2,12)} runs on the tensor-core kernels; everything else in the
+ * supported set runs on the fp32 SIMT kernels.
+ */
+typedef struct {
+    int32_t B, H, N, d;
+    int32_t F;        /* number of Hadamard factors; 0 -> 3 (the paper's main model)          */
+    int32_t d_phi;    /* feature width; 0 -> 6 if F == 3, 12 if F == 2 (appendix "Defining phi") */
+    int32_t phi;      /* hla_phi_mode                                                          */
+    int32_t dtype;    /* hla_dtype                                                             */
+    float eps;        /* added to the normaliser, o = num / (eta + eps); <= 0 -> 1e-6          */
+    int32_t n_splits; /* token splits of the state build per head; 0 -> chosen from the SM count */
+    int32_t causal;   /* must be 0: the causal / decayed variant (Section 4.4) is not built    */
+} hla_config;
+
+/*
+ * One feature network (appendix "Defining phi"): feat = ReLU(W2^T GELU(W1^T x + b1) + b2),
+ * exact (erf) GELU.  Device pointers in the ctx dtype: W1 [d][d] (input index
+ * first), b1 [d], W2 [d][d_phi], b2 [d_phi].  One set per map, shared by all
+ * batches and heads.
+ */
+typedef struct {
+    const void *W1, *b1, *W2, *b2;
+} hla_mlp;
+
+/* Byte offsets of the regions of the workspace that outlive a call (for
+ * checking and for callers that want the state).  A region that the
+ * configuration does not use has offset (size_t)-1. */
+typedef struct {
+    size_t status;   /* int32[16]  device status words                                   */
+    size_t qf;       /* fp32 [B,H,N,d_phi]     features phi_q(Q)        (HLA_PHI_MLP)   */
+    size_t kf;       /* fp32 [B,H,F,N,d_phi]   features phi_kf(K)       (HLA_PHI_MLP)   */
+    size_t state;    /* fp32 [B,H,P,state_ld]  columns 0..d-1 = C, column d = z         */
+    size_t eta;      /* fp32 [B,H,N]           normaliser before eps                    */
+    size_t dstate;   /* fp32 [B,H,P,state_ld]  dC | dz   (after hla_backward)           */
+    size_t dqf;      /* fp32 [B,H,N,d_phi]     feature gradients        (HLA_PHI_MLP)   */
+    size_t dkf;      /* fp32 [B,H,F,N,d_phi]                            (HLA_PHI_MLP)   */
+    int32_t state_ld; /* row stride of state / dstate in floats (>= d+1)                */
+    int32_t n_splits; /* the split count in use                                          */
+    int32_t tensor_core; /* 1 if this configuration runs the tcgen05 kernels              */
+} hla_ws_layout;
+
+/* Validates the configuration and creates a context.  *out is NULL on failure. */
+hla_status hla_create(const hla_config *cfg, hla_ctx **out);
+
+/* HLA_PHI_MLP only: remembers the weight pointers (phi_k points to F entries).
+ * The weights must stay valid and unchanged while the ctx is used. */
+hla_status hla_set_phi(hla_ctx *ctx, const hla_mlp *phi_q, const hla_mlp *phi_k);
+
+/* Bytes of caller-provided device scratch that forward and backward need. */
+size_t hla_workspace_bytes(const hla_ctx *ctx);
+
+hla_status hla_workspace_layout(const hla_ctx *ctx, hla_ws_layout *out);
+
+/*
+ * Forward: O = HLA(Q, K, V).  Leaves the features, the state (C, z) and eta in
+ * the workspace for a later hla_backward.  The workspace must be 256-byte
+ * aligned and at least hla_workspace_bytes() long.
+ */
+hla_status hla_forward(hla_ctx *ctx, const void *Q, const void *K, const void *V, void *O,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Backward of the forward that last wrote `workspace` (same Q, K, V, O; the
+ * workspace untouched in between): dQ, dK, dV = d sum(dO * O) / d(Q, K, V).
+ * In HLA_PHI_NONE mode dQ, dK are fp32 feature gradients with the shapes of Q, K.
+ * Gradients with respect to the phi weights are not computed.
+ */
+hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *V, const void *O,
+                        const void *dO, void *dQ, void *dK, void *dV,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the device status words of `workspace`
+ * and returns HLA_OK, HLA_ERR_DEVICE_TIMEOUT or HLA_ERR_CUDA. */
+hla_status hla_last_device_status(hla_ctx *ctx, const void *workspace, void *cuda_stream);
+
+/* Number of kernels the last hla_forward / hla_backward on this ctx launched. */
+int32_t hla_last_launch_count(const hla_ctx *ctx);
+
+hla_status hla_destroy(hla_ctx *ctx);
+
+const char *hla_status_string(hla_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HLA_H_ */

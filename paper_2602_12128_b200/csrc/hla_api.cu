@@ -1,0 +1,353 @@
+// C ABI of the HLA library: context, validation, workspace layout and the
+// launch sequences of forward and backward.  See include/hla.h for the contract.
+#include "../../include/hla.h"
+
+#include <new>
+
+#include "hla_common.cuh"
+#include "hla_simt.cuh"
+#include "hla_tc.cuh"
+
+using namespace hla;
+
+struct hla_ctx {
+    hla_config cfg;
+    Dims D;
+    int BH;
+    bool tc;            // tensor-core kernels in use
+    bool phi_set;
+    hla_mlp phi_q;
+    hla_mlp phi_k[kMaxF];
+    hla_ws_layout L;
+    size_t off_part;    // split partials (scratch)
+    tc::Plan tcp;       // tensor-core operand buffers inside the workspace
+    size_t ws_bytes;
+    int sm_count;
+    int launches;
+};
+
+namespace {
+
+constexpr size_t kNone = (size_t)-1;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        const size_t o = off;
+        off = align_up(off + bytes, 256);
+        return o;
+    }
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int ipow(int b, int e) {
+    long long r = 1;
+    for (int i = 0; i < e; ++i) {
+        r *= b;
+        if (r > (1 << 20)) return 1 << 20;
+    }
+    return (int)r;
+}
+
+#define HLA_LAUNCH_CHECK(ctx)                                   \
+    do {                                                        \
+        (ctx)->launches++;                                      \
+        if (cudaPeekAtLastError() != cudaSuccess) return HLA_ERR_CUDA; \
+    } while (0)
+
+template <typename T>
+simt::PhiWeights<T> pack_weights(const hla_mlp* m, int n) {
+    simt::PhiWeights<T> w{};
+    w.nmaps = n;
+    for (int i = 0; i < n; ++i) {
+        w.W1[i] = static_cast<const T*>(m[i].W1);
+        w.b1[i] = static_cast<const T*>(m[i].b1);
+        w.W2[i] = static_cast<const T*>(m[i].W2);
+        w.b2[i] = static_cast<const T*>(m[i].b2);
+    }
+    return w;
+}
+
+int reduce_blocks(size_t total) {
+    size_t b = (total + 255) / 256;
+    return (int)(b > 4096 ? 4096 : (b < 1 ? 1 : b));
+}
+
+// ---- fp32 SIMT path --------------------------------------------------------
+template <typename T>
+hla_status simt_phi_forward(hla_ctx* c, const void* Q, const void* K, char* ws, cudaStream_t st) {
+    const Dims& D = c->D;
+    const size_t rows = (size_t)c->BH * D.N;
+    const int blocks = (int)((rows + simt::kTok - 1) / simt::kTok);
+    simt::phi_forward_kernel<T, false><<<blocks, simt::kPhiThreads, 0, st>>>(
+        static_cast<const T*>(Q), pack_weights<T>(&c->phi_q, 1), reinterpret_cast<float*>(ws + c->L.qf), rows, D.N, D.d, D.dphi);
+    HLA_LAUNCH_CHECK(c);
+    simt::phi_forward_kernel<T, true><<<blocks, simt::kPhiThreads, 0, st>>>(
+        static_cast<const T*>(K), pack_weights<T>(c->phi_k, D.F), reinterpret_cast<float*>(ws + c->L.kf), rows, D.N, D.d, D.dphi);
+    HLA_LAUNCH_CHECK(c);
+    return HLA_OK;
+}
+
+template <typename T>
+hla_status simt_core_forward(hla_ctx* c, const float* qf, const float* kf, const void* V, void* O, char* ws, cudaStream_t st) {
+    const Dims& D = c->D;
+    float* part = reinterpret_cast<float*>(ws + c->off_part);
+    float* state = reinterpret_cast<float*>(ws + c->L.state);
+    float* eta = reinterpret_cast<float*>(ws + c->L.eta);
+    simt::state_build_kernel<T, false><<<dim3(D.S, c->BH), simt::kThreads, 0, st>>>(D, kf, static_cast<const T*>(V), nullptr, nullptr, part);
+    HLA_LAUNCH_CHECK(c);
+    const size_t n_per = (size_t)D.P * D.ld;
+    simt::reduce_partials_kernel<<<reduce_blocks(n_per * c->BH), 256, 0, st>>>(state, part, c->BH, D.S, n_per);
+    HLA_LAUNCH_CHECK(c);
+    const int tiles = (D.N + simt::kTok - 1) / simt::kTok;
+    simt::readout_kernel<T, true><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, qf, state, static_cast<T*>(O), eta);
+    HLA_LAUNCH_CHECK(c);
+    return HLA_OK;
+}
+
+template <typename T>
+hla_status simt_core_backward(hla_ctx* c, const float* qf, const float* kf, const void* V, const void* O, const void* dO,
+                              float* dqf, float* dkf, void* dV, char* ws, cudaStream_t st) {
+    const Dims& D = c->D;
+    float* part = reinterpret_cast<float*>(ws + c->off_part);
+    const float* state = reinterpret_cast<const float*>(ws + c->L.state);
+    float* dstate = reinterpret_cast<float*>(ws + c->L.dstate);
+    const float* eta = reinterpret_cast<const float*>(ws + c->L.eta);
+    const int tiles = (D.N + simt::kTok - 1) / simt::kTok;
+    const size_t n_per = (size_t)D.P * D.ld;
+    // pass over the queries: dC, dz, then dq
+    simt::state_build_kernel<T, true><<<dim3(D.S, c->BH), simt::kThreads, 0, st>>>(D, qf, static_cast<const T*>(dO), static_cast<const T*>(O), eta, part);
+    HLA_LAUNCH_CHECK(c);
+    simt::reduce_partials_kernel<<<reduce_blocks(n_per * c->BH), 256, 0, st>>>(dstate, part, c->BH, D.S, n_per);
+    HLA_LAUNCH_CHECK(c);
+    simt::feature_grad_kernel<T, true><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, qf, static_cast<const T*>(dO), static_cast<const T*>(O), eta, state, dqf);
+    HLA_LAUNCH_CHECK(c);
+    // pass over the keys: dV, dk^f
+    simt::readout_kernel<T, false><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, kf, dstate, static_cast<T*>(dV), nullptr);
+    HLA_LAUNCH_CHECK(c);
+    simt::feature_grad_kernel<T, false><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, kf, static_cast<const T*>(V), nullptr, nullptr, dstate, dkf);
+    HLA_LAUNCH_CHECK(c);
+    return HLA_OK;
+}
+
+template <typename T>
+hla_status simt_phi_backward(hla_ctx* c, const void* Q, const void* K, void* dQ, void* dK, char* ws, cudaStream_t st) {
+    const Dims& D = c->D;
+    const size_t rows = (size_t)c->BH * D.N;
+    const int blocks = (int)((rows + simt::kTok - 1) / simt::kTok);
+    simt::phi_backward_kernel<T, false><<<blocks, simt::kPhiThreads, 0, st>>>(
+        static_cast<const T*>(Q), pack_weights<T>(&c->phi_q, 1), reinterpret_cast<const float*>(ws + c->L.dqf), static_cast<T*>(dQ), rows, D.N, D.d, D.dphi);
+    HLA_LAUNCH_CHECK(c);
+    simt::phi_backward_kernel<T, true><<<blocks, simt::kPhiThreads, 0, st>>>(
+        static_cast<const T*>(K), pack_weights<T>(c->phi_k, D.F), reinterpret_cast<const float*>(ws + c->L.dkf), static_cast<T*>(dK), rows, D.N, D.d, D.dphi);
+    HLA_LAUNCH_CHECK(c);
+    return HLA_OK;
+}
+
+template <typename T>
+hla_status forward_simt(hla_ctx* c, const void* Q, const void* K, const void* V, void* O, char* ws, cudaStream_t st) {
+    const float *qf, *kf;
+    if (c->cfg.phi == HLA_PHI_MLP) {
+        hla_status s = simt_phi_forward<T>(c, Q, K, ws, st);
+        if (s != HLA_OK) return s;
+        qf = reinterpret_cast<const float*>(ws + c->L.qf);
+        kf = reinterpret_cast<const float*>(ws + c->L.kf);
+    } else {
+        qf = static_cast<const float*>(Q);
+        kf = static_cast<const float*>(K);
+    }
+    return simt_core_forward<T>(c, qf, kf, V, O, ws, st);
+}
+
+template <typename T>
+hla_status backward_simt(hla_ctx* c, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ,
+                         void* dK, void* dV, char* ws, cudaStream_t st) {
+    const bool mlp = c->cfg.phi == HLA_PHI_MLP;
+    const float* qf = mlp ? reinterpret_cast<const float*>(ws + c->L.qf) : static_cast<const float*>(Q);
+    const float* kf = mlp ? reinterpret_cast<const float*>(ws + c->L.kf) : static_cast<const float*>(K);
+    float* dqf = mlp ? reinterpret_cast<float*>(ws + c->L.dqf) : static_cast<float*>(dQ);
+    float* dkf = mlp ? reinterpret_cast<float*>(ws + c->L.dkf) : static_cast<float*>(dK);
+    hla_status s = simt_core_backward<T>(c, qf, kf, V, O, dO, dqf, dkf, dV, ws, st);
+    if (s != HLA_OK || !mlp) return s;
+    return simt_phi_backward<T>(c, Q, K, dQ, dK, ws, st);
+}
+
+hla_status check_call(const hla_ctx* c, const void* const* ptrs, int n, const void* ws, size_t ws_bytes) {
+    if (!c) return HLA_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i)
+        if (!ptrs[i] || !aligned16(ptrs[i])) return HLA_ERR_INVALID_ARG;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return HLA_ERR_INVALID_ARG;
+    if (ws_bytes < c->ws_bytes) return HLA_ERR_WORKSPACE;
+    if (c->cfg.phi == HLA_PHI_MLP && !c->phi_set) return HLA_ERR_INVALID_ARG;
+    return HLA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
+    if (out) *out = nullptr;
+    if (!cfg || !out) return HLA_ERR_INVALID_ARG;
+    hla_config c = *cfg;
+    if (c.B <= 0 || c.H <= 0 || c.N <= 0 || c.d <= 0) return HLA_ERR_INVALID_ARG;
+    if (c.F < 0 || c.d_phi < 0 || c.n_splits < 0) return HLA_ERR_INVALID_ARG;
+    if (c.phi != HLA_PHI_MLP && c.phi != HLA_PHI_NONE) return HLA_ERR_INVALID_ARG;
+    if (c.dtype != HLA_BF16 && c.dtype != HLA_F32) return HLA_ERR_INVALID_ARG;
+    if (c.F == 0) c.F = 3;
+    if (c.d_phi == 0) {
+        if (c.F == 3) c.d_phi = 6;
+        else if (c.F == 2) c.d_phi = 12;
+        else return HLA_ERR_INVALID_ARG;
+    }
+    if (!(c.eps > 0.f)) c.eps = 1e-6f;
+    if (c.causal != 0) return HLA_ERR_UNSUPPORTED;
+    if (c.F > kMaxF) return HLA_ERR_UNSUPPORTED;
+    const int P = ipow(c.d_phi, c.F);
+    if (P > kMaxP) return HLA_ERR_UNSUPPORTED;
+    if (c.d > kMaxD || (c.d % 4) != 0) return HLA_ERR_UNSUPPORTED;
+    if ((long long)c.B * c.H > 65535) return HLA_ERR_UNSUPPORTED;
+    if (c.dtype == HLA_BF16 && (c.d % 8) != 0) return HLA_ERR_UNSUPPORTED;   // 16-byte rows
+
+    hla_ctx* x = new (std::nothrow) hla_ctx();
+    if (!x) return HLA_ERR_INVALID_ARG;
+    x->cfg = c;
+    x->BH = c.B * c.H;
+    x->phi_set = false;
+    x->launches = 0;
+    x->sm_count = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) x->sm_count = n;
+    }
+    (void)cudaGetLastError();
+    Dims& D = x->D;
+    D.B = c.B; D.H = c.H; D.N = c.N; D.d = c.d; D.F = c.F; D.dphi = c.d_phi; D.P = P;
+    D.ld = c.d + 4;
+    D.eps = c.eps;
+    x->tc = tc::supported(c.dtype == HLA_BF16, c.d, c.F, c.d_phi);
+    const int tile = x->tc ? tc::kTileTokens : simt::kTok;
+    const int tiles = (c.N + tile - 1) / tile;
+    int S = c.n_splits;
+    if (S == 0) {
+        const int target = x->tc ? x->sm_count : 2 * x->sm_count;
+        S = (target + x->BH - 1) / x->BH;
+    }
+    if (S > tiles) S = tiles;
+    if (S < 1) S = 1;
+    D.S = S;
+
+    const bool mlp = c.phi == HLA_PHI_MLP;
+    const size_t tok = (size_t)x->BH * c.N;
+    Carver cv;
+    hla_ws_layout& L = x->L;
+    L.status = cv.take(64);
+    L.qf = mlp ? cv.take(tok * c.d_phi * 4) : kNone;
+    L.kf = mlp ? cv.take(tok * c.F * c.d_phi * 4) : kNone;
+    L.state = cv.take((size_t)x->BH * P * D.ld * 4);
+    L.eta = cv.take(tok * 4);
+    L.dstate = cv.take((size_t)x->BH * P * D.ld * 4);
+    L.dqf = mlp ? cv.take(tok * c.d_phi * 4) : kNone;
+    L.dkf = mlp ? cv.take(tok * c.F * c.d_phi * 4) : kNone;
+    L.state_ld = D.ld;
+    L.n_splits = S;
+    L.tensor_core = x->tc ? 1 : 0;
+    x->off_part = cv.take((size_t)x->BH * S * P * D.ld * 4);
+    if (x->tc) cv.off = tc::plan(x->tcp, D, x->BH, cv.off);
+    x->ws_bytes = cv.off;
+    *out = x;
+    return HLA_OK;
+}
+
+hla_status hla_set_phi(hla_ctx* ctx, const hla_mlp* phi_q, const hla_mlp* phi_k) {
+    if (!ctx || !phi_q || !phi_k) return HLA_ERR_INVALID_ARG;
+    if (ctx->cfg.phi != HLA_PHI_MLP) return HLA_ERR_INVALID_ARG;
+    const hla_mlp* all[1 + kMaxF];
+    all[0] = phi_q;
+    for (int f = 0; f < ctx->D.F; ++f) all[1 + f] = phi_k + f;
+    for (int i = 0; i < 1 + ctx->D.F; ++i) {
+        const void* p[4] = {all[i]->W1, all[i]->b1, all[i]->W2, all[i]->b2};
+        for (int j = 0; j < 4; ++j)
+            if (!p[j]) return HLA_ERR_INVALID_ARG;
+        if (!aligned16(all[i]->W1) || !aligned16(all[i]->W2)) return HLA_ERR_INVALID_ARG;
+    }
+    ctx->phi_q = *phi_q;
+    for (int f = 0; f < ctx->D.F; ++f) ctx->phi_k[f] = phi_k[f];
+    ctx->phi_set = true;
+    return HLA_OK;
+}
+
+size_t hla_workspace_bytes(const hla_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
+
+hla_status hla_workspace_layout(const hla_ctx* ctx, hla_ws_layout* out) {
+    if (!ctx || !out) return HLA_ERR_INVALID_ARG;
+    *out = ctx->L;
+    return HLA_OK;
+}
+
+hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V, void* O, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+    const void* ptrs[4] = {Q, K, V, O};
+    hla_status s = check_call(ctx, ptrs, 4, workspace, workspace_bytes);
+    if (s != HLA_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    ctx->launches = 0;
+    (void)cudaGetLastError();
+    if (cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
+    if (ctx->tc) return tc::forward(ctx->tcp, ctx->D, ctx->BH, ctx->cfg.phi == HLA_PHI_MLP, &ctx->phi_q, ctx->phi_k, Q, K, V, O, ws,
+                                    ctx->L, ctx->off_part, ctx->sm_count, st, &ctx->launches);
+    if (ctx->cfg.dtype == HLA_F32) return forward_simt<float>(ctx, Q, K, V, O, ws, st);
+    return forward_simt<__nv_bfloat16>(ctx, Q, K, V, O, ws, st);
+}
+
+hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ,
+                        void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const void* ptrs[8] = {Q, K, V, O, dO, dQ, dK, dV};
+    hla_status s = check_call(ctx, ptrs, 8, workspace, workspace_bytes);
+    if (s != HLA_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    ctx->launches = 0;
+    (void)cudaGetLastError();
+    if (ctx->tc) return tc::backward(ctx->tcp, ctx->D, ctx->BH, ctx->cfg.phi == HLA_PHI_MLP, &ctx->phi_q, ctx->phi_k, Q, K, V, O, dO, dQ,
+                                     dK, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, st, &ctx->launches);
+    if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
+    return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
+}
+
+hla_status hla_last_device_status(hla_ctx* ctx, const void* workspace, void* cuda_stream) {
+    if (!ctx || !workspace) return HLA_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t words[16] = {0};
+    if (cudaMemcpyAsync(words, static_cast<const char*>(workspace) + ctx->L.status, sizeof(words), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return HLA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return HLA_ERR_CUDA;
+    return words[kStatusTimeout] != 0 ? HLA_ERR_DEVICE_TIMEOUT : HLA_OK;
+}
+
+int32_t hla_last_launch_count(const hla_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+hla_status hla_destroy(hla_ctx* ctx) {
+    if (!ctx) return HLA_ERR_INVALID_ARG;
+    delete ctx;
+    return HLA_OK;
+}
+
+const char* hla_status_string(hla_status s) {
+    switch (s) {
+        case HLA_OK: return "ok";
+        case HLA_ERR_INVALID_ARG: return "invalid argument";
+        case HLA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case HLA_ERR_WORKSPACE: return "workspace too small";
+        case HLA_ERR_CUDA: return "CUDA error";
+        case HLA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"
