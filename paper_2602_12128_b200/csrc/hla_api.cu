@@ -299,8 +299,19 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
     ctx->launches = 0;
     (void)cudaGetLastError();
     if (cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
-    if (ctx->tc) return tc::forward(ctx->tcp, ctx->D, ctx->BH, ctx->cfg.phi == HLA_PHI_MLP, &ctx->phi_q, ctx->phi_k, Q, K, V, O, ws,
-                                    ctx->L, ctx->off_part, ctx->sm_count, st, &ctx->launches);
+    if (ctx->tc) {
+        const float *qf, *kf;
+        if (ctx->cfg.phi == HLA_PHI_MLP) {
+            s = simt_phi_forward<__nv_bfloat16>(ctx, Q, K, ws, st);
+            if (s != HLA_OK) return s;
+            qf = reinterpret_cast<const float*>(ws + ctx->L.qf);
+            kf = reinterpret_cast<const float*>(ws + ctx->L.kf);
+        } else {
+            qf = static_cast<const float*>(Q);
+            kf = static_cast<const float*>(K);
+        }
+        return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, st, &ctx->launches);
+    }
     if (ctx->cfg.dtype == HLA_F32) return forward_simt<float>(ctx, Q, K, V, O, ws, st);
     return forward_simt<__nv_bfloat16>(ctx, Q, K, V, O, ws, st);
 }
@@ -314,8 +325,6 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     char* ws = static_cast<char*>(workspace);
     ctx->launches = 0;
     (void)cudaGetLastError();
-    if (ctx->tc) return tc::backward(ctx->tcp, ctx->D, ctx->BH, ctx->cfg.phi == HLA_PHI_MLP, &ctx->phi_q, ctx->phi_k, Q, K, V, O, dO, dQ,
-                                     dK, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, st, &ctx->launches);
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
 }

@@ -1,0 +1,69 @@
+"""GPU parity of the bf16 tensor-core kernels (tcgen05 state build, reduce/emit,
+readout) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hla_oracle as orc
+from paper_2602_12128_b200 import binding, synth
+from hla_testlib import GpuRun, TOL, oracle_state, relerr, l2err
+
+pytestmark = pytest.mark.gpu
+EPS = 1e-6
+
+
+@pytest.mark.parametrize("d,N,B,H,splits", [(128, 1000, 1, 2, 0), (128, 128, 1, 1, 1), (128, 77, 1, 3, 0), (64, 1500, 2, 2, 5),
+                                            (128, 4096 + 40, 1, 2, 7), (64, 129, 1, 1, 4)])
+def test_core_forward_bf16_features(d, N, B, H, splits):
+    """Feature-level entry point: the features are fp32 inputs, V is bf16; spans several
+    128-token tiles, ragged tails, more splits than tiles, and both head widths."""
+    s = synth.HlaShape("t", B, H, N, d, "bf16", "inv_sqrt_d")
+    _, _, V = synth.make_qkv(s)
+    V = synth.bf16_round(V * np.float32(np.sqrt(d)))          # V ~ N(0,1)
+    qf, kf = synth.make_features(s)
+    run = GpuRun(s, "none", EPS, splits)
+    assert run.op.layout.tensor_core == 1
+    O = run.forward(qf, kf, V)
+    f64 = lambda a: a.astype(np.float64)
+    Oq, eta = orc.hla_core_forward(f64(qf), f64(kf), f64(V), EPS, "factored")
+    C, z = run.state()
+    Co, zo = oracle_state(f64(kf), f64(V))
+    assert relerr(z, zo) < 1e-5                      # fp32 accumulation of unrounded products
+    assert relerr(C, Co) < TOL["bf16"] / 4           # T_k rounded to bf16 once
+    assert relerr(run.eta(), eta) < TOL["bf16"] / 4
+    assert relerr(O, Oq) < TOL["bf16"], (relerr(O, Oq), l2err(O, Oq))
+    assert run.op.launches() == 3
+
+
+def test_config2_small_bf16_forward_stagewise():
+    """B=2,H=12,N=4096,d=64 bf16 with the phi maps: features against the oracle's,
+    then the core against the oracle core run on the features the GPU produced,
+    then end to end on rows whose normaliser is not tiny."""
+    s = synth.CONFIGS["small_bf16"]
+    Q, K, V = synth.make_qkv(s)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    run = GpuRun(s, "mlp", EPS)
+    run.set_weights(pq, pk)
+    O = run.forward(Q, K, V)
+    f64 = lambda a: a.astype(np.float64)
+    Oq, eta, qf, kf = orc.hla_forward(f64(Q), f64(K), f64(V), pq, pk, EPS, "factored")
+    gq, gk = run.features()
+    assert relerr(gq, qf) < TOL["bf16"] and relerr(gk, kf) < TOL["bf16"]
+    Oc, _ = orc.hla_core_forward(gq, gk, f64(V), EPS, "factored")
+    assert relerr(O, Oc) < TOL["bf16"]
+    keep = eta >= 1e-3 * np.median(eta)
+    assert keep.mean() > 0.5
+    assert relerr(O[keep], Oq[keep]) < TOL["bf16"], relerr(O[keep], Oq[keep])
+    # the quadratic definition on one head
+    o_def, _ = orc.hla_quadratic(qf[1, 5], [kf[1, 5, f] for f in range(3)], f64(V)[1, 5], EPS)
+    np.testing.assert_allclose(o_def, Oq[1, 5], rtol=1e-8, atol=1e-12)
+
+
+def test_tc_bitwise_reproducible():
+    s = synth.HlaShape("t", 1, 3, 2000, 128, "bf16", "inv_sqrt_d")
+    _, _, V = synth.make_qkv(s)
+    qf, kf = synth.make_features(s)
+    run = GpuRun(s, "none", EPS, 4)
+    a = run.forward(qf, kf, V)
+    b = run.forward(qf, kf, V)
+    assert np.array_equal(a, b)
