@@ -140,6 +140,19 @@ hla_status hla_last_device_status(hla_ctx *ctx, const void *workspace, void *cud
 /* Number of kernels the last hla_forward / hla_backward on this ctx launched. */
 int32_t hla_last_launch_count(const hla_ctx *ctx);
 
+/*
+ * Optional per-kernel timing (no counterpart in the paper: a measurement aid).
+ * While enabled, every kernel launch of hla_forward / hla_backward is bracketed
+ * by CUDA events on the launching stream.  After the caller has synchronised
+ * the stream, hla_timing_collect folds the recorded launches into per-kernel
+ * totals (replacing earlier totals) and returns how many distinct kernels
+ * there are; hla_timing_get returns entry i: a static name, the summed device
+ * time in milliseconds and the number of launches.
+ */
+hla_status hla_timing_enable(hla_ctx *ctx, int32_t on);
+int32_t hla_timing_collect(hla_ctx *ctx);
+hla_status hla_timing_get(const hla_ctx *ctx, int32_t i, const char **name, double *total_ms, int64_t *launches);
+
 hla_status hla_destroy(hla_ctx *ctx);
 
 const char *hla_status_string(hla_status s);

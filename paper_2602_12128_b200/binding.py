@@ -18,7 +18,8 @@ HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
     "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward",
-    "hla_last_device_status", "hla_last_launch_count", "hla_destroy", "hla_status_string",
+    "hla_last_device_status", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
+    "hla_destroy", "hla_status_string",
 ]
 
 
@@ -75,6 +76,12 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_last_device_status.restype = c_int32
     lib.hla_last_launch_count.argtypes = [c_void_p]
     lib.hla_last_launch_count.restype = c_int32
+    lib.hla_timing_enable.argtypes = [c_void_p, c_int32]
+    lib.hla_timing_enable.restype = c_int32
+    lib.hla_timing_collect.argtypes = [c_void_p]
+    lib.hla_timing_collect.restype = c_int32
+    lib.hla_timing_get.argtypes = [c_void_p, c_int32, POINTER(c_char_p), POINTER(ctypes.c_double), POINTER(ctypes.c_int64)]
+    lib.hla_timing_get.restype = c_int32
     lib.hla_destroy.argtypes = [c_void_p]
     lib.hla_destroy.restype = c_int32
     lib.hla_status_string.argtypes = [c_int32]
@@ -154,6 +161,28 @@ def hla_last_device_status(ctx: int, workspace, stream=None) -> int:
 
 def hla_last_launch_count(ctx: int) -> int:
     return int(load_library().hla_last_launch_count(ctx))
+
+
+def hla_timing_enable(ctx: int, on: bool) -> None:
+    st = load_library().hla_timing_enable(ctx, 1 if on else 0)
+    if st != HLA_OK:
+        raise HlaError(st, "hla_timing_enable")
+
+
+def hla_timing_collect(ctx: int) -> dict:
+    """After a stream synchronise: {kernel name: (total_ms, launches)} of the launches recorded since the last collect."""
+    lib = load_library()
+    n = lib.hla_timing_collect(ctx)
+    out = {}
+    for i in range(n):
+        name = c_char_p()
+        ms = ctypes.c_double()
+        cnt = ctypes.c_int64()
+        st = lib.hla_timing_get(ctx, i, byref(name), byref(ms), byref(cnt))
+        if st != HLA_OK:
+            raise HlaError(st, "hla_timing_get")
+        out[name.value.decode()] = (ms.value, cnt.value)
+    return out
 
 
 def hla_destroy(ctx: int) -> None:

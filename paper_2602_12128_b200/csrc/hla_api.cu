@@ -3,6 +3,7 @@
 #include "../../include/hla.h"
 
 #include <new>
+#include <string.h>
 
 #include "hla_common.cuh"
 #include "hla_simt.cuh"
@@ -23,7 +24,7 @@ struct hla_ctx {
     tc::Plan tcp;       // tensor-core operand buffers inside the workspace
     size_t ws_bytes;
     int sm_count;
-    int launches;
+    LaunchRec rec;      // launch counter and optional per-kernel event timing
 };
 
 namespace {
@@ -52,12 +53,6 @@ int ipow(int b, int e) {
     return (int)r;
 }
 
-#define HLA_LAUNCH_CHECK(ctx)                                   \
-    do {                                                        \
-        (ctx)->launches++;                                      \
-        if (cudaPeekAtLastError() != cudaSuccess) return HLA_ERR_CUDA; \
-    } while (0)
-
 template <typename T>
 simt::PhiWeights<T> pack_weights(const hla_mlp* m, int n) {
     simt::PhiWeights<T> w{};
@@ -82,12 +77,14 @@ hla_status simt_phi_forward(hla_ctx* c, const void* Q, const void* K, char* ws, 
     const Dims& D = c->D;
     const size_t rows = (size_t)c->BH * D.N;
     const int blocks = (int)((rows + simt::kTok - 1) / simt::kTok);
+    c->rec.begin("simt_phi_forward");
     simt::phi_forward_kernel<T, false><<<blocks, simt::kPhiThreads, 0, st>>>(
         static_cast<const T*>(Q), pack_weights<T>(&c->phi_q, 1), reinterpret_cast<float*>(ws + c->L.qf), rows, D.N, D.d, D.dphi);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
+    c->rec.begin("simt_phi_forward");
     simt::phi_forward_kernel<T, true><<<blocks, simt::kPhiThreads, 0, st>>>(
         static_cast<const T*>(K), pack_weights<T>(c->phi_k, D.F), reinterpret_cast<float*>(ws + c->L.kf), rows, D.N, D.d, D.dphi);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     return HLA_OK;
 }
 
@@ -97,14 +94,17 @@ hla_status simt_core_forward(hla_ctx* c, const float* qf, const float* kf, const
     float* part = reinterpret_cast<float*>(ws + c->off_part);
     float* state = reinterpret_cast<float*>(ws + c->L.state);
     float* eta = reinterpret_cast<float*>(ws + c->L.eta);
+    c->rec.begin("simt_state_build");
     simt::state_build_kernel<T, false><<<dim3(D.S, c->BH), simt::kThreads, 0, st>>>(D, kf, static_cast<const T*>(V), nullptr, nullptr, part);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     const size_t n_per = (size_t)D.P * D.ld;
+    c->rec.begin("simt_reduce_partials");
     simt::reduce_partials_kernel<<<reduce_blocks(n_per * c->BH), 256, 0, st>>>(state, part, c->BH, D.S, n_per);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + simt::kTok - 1) / simt::kTok;
+    c->rec.begin("simt_readout");
     simt::readout_kernel<T, true><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, qf, state, static_cast<T*>(O), eta);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     return HLA_OK;
 }
 
@@ -119,17 +119,22 @@ hla_status simt_core_backward(hla_ctx* c, const float* qf, const float* kf, cons
     const int tiles = (D.N + simt::kTok - 1) / simt::kTok;
     const size_t n_per = (size_t)D.P * D.ld;
     // pass over the queries: dC, dz, then dq
+    c->rec.begin("simt_state_build");
     simt::state_build_kernel<T, true><<<dim3(D.S, c->BH), simt::kThreads, 0, st>>>(D, qf, static_cast<const T*>(dO), static_cast<const T*>(O), eta, part);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
+    c->rec.begin("simt_reduce_partials");
     simt::reduce_partials_kernel<<<reduce_blocks(n_per * c->BH), 256, 0, st>>>(dstate, part, c->BH, D.S, n_per);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
+    c->rec.begin("simt_feature_grad");
     simt::feature_grad_kernel<T, true><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, qf, static_cast<const T*>(dO), static_cast<const T*>(O), eta, state, dqf);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     // pass over the keys: dV, dk^f
+    c->rec.begin("simt_readout");
     simt::readout_kernel<T, false><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, kf, dstate, static_cast<T*>(dV), nullptr);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
+    c->rec.begin("simt_feature_grad");
     simt::feature_grad_kernel<T, false><<<dim3(tiles, c->BH), simt::kThreads, 0, st>>>(D, kf, static_cast<const T*>(V), nullptr, nullptr, dstate, dkf);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     return HLA_OK;
 }
 
@@ -138,12 +143,14 @@ hla_status simt_phi_backward(hla_ctx* c, const void* Q, const void* K, void* dQ,
     const Dims& D = c->D;
     const size_t rows = (size_t)c->BH * D.N;
     const int blocks = (int)((rows + simt::kTok - 1) / simt::kTok);
+    c->rec.begin("simt_phi_backward");
     simt::phi_backward_kernel<T, false><<<blocks, simt::kPhiThreads, 0, st>>>(
         static_cast<const T*>(Q), pack_weights<T>(&c->phi_q, 1), reinterpret_cast<const float*>(ws + c->L.dqf), static_cast<T*>(dQ), rows, D.N, D.d, D.dphi);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
+    c->rec.begin("simt_phi_backward");
     simt::phi_backward_kernel<T, true><<<blocks, simt::kPhiThreads, 0, st>>>(
         static_cast<const T*>(K), pack_weights<T>(c->phi_k, D.F), reinterpret_cast<const float*>(ws + c->L.dkf), static_cast<T*>(dK), rows, D.N, D.d, D.dphi);
-    HLA_LAUNCH_CHECK(c);
+    if (!c->rec.end()) return HLA_ERR_CUDA;
     return HLA_OK;
 }
 
@@ -217,7 +224,6 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     x->cfg = c;
     x->BH = c.B * c.H;
     x->phi_set = false;
-    x->launches = 0;
     x->sm_count = 148;
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) {
@@ -296,7 +302,7 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
     if (s != HLA_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
-    ctx->launches = 0;
+    ctx->rec.start_call(st);
     (void)cudaGetLastError();
     if (cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
     if (ctx->tc) {
@@ -310,7 +316,7 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
             qf = static_cast<const float*>(Q);
             kf = static_cast<const float*>(K);
         }
-        return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, st, &ctx->launches);
+        return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
     }
     if (ctx->cfg.dtype == HLA_F32) return forward_simt<float>(ctx, Q, K, V, O, ws, st);
     return forward_simt<__nv_bfloat16>(ctx, Q, K, V, O, ws, st);
@@ -323,7 +329,7 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     if (s != HLA_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
-    ctx->launches = 0;
+    ctx->rec.start_call(st);
     (void)cudaGetLastError();
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
@@ -339,7 +345,23 @@ hla_status hla_last_device_status(hla_ctx* ctx, const void* workspace, void* cud
     return words[kStatusTimeout] != 0 ? HLA_ERR_DEVICE_TIMEOUT : HLA_OK;
 }
 
-int32_t hla_last_launch_count(const hla_ctx* ctx) { return ctx ? ctx->launches : 0; }
+int32_t hla_last_launch_count(const hla_ctx* ctx) { return ctx ? ctx->rec.launches : 0; }
+
+hla_status hla_timing_enable(hla_ctx* ctx, int32_t on) {
+    if (!ctx) return HLA_ERR_INVALID_ARG;
+    ctx->rec.timing = on != 0;
+    return HLA_OK;
+}
+
+int32_t hla_timing_collect(hla_ctx* ctx) { return ctx ? ctx->rec.collect() : 0; }
+
+hla_status hla_timing_get(const hla_ctx* ctx, int32_t i, const char** name, double* total_ms, int64_t* launches) {
+    if (!ctx || i < 0 || i >= (int32_t)ctx->rec.acc.size() || !name || !total_ms || !launches) return HLA_ERR_INVALID_ARG;
+    *name = ctx->rec.acc[i].name;
+    *total_ms = ctx->rec.acc[i].ms;
+    *launches = ctx->rec.acc[i].n;
+    return HLA_OK;
+}
 
 hla_status hla_destroy(hla_ctx* ctx) {
     if (!ctx) return HLA_ERR_INVALID_ARG;

@@ -7,6 +7,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
+
+#include <vector>
 
 namespace hla {
 
@@ -46,5 +49,51 @@ __device__ __forceinline__ float warp_sum(float v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
+
+// Host side: counts the kernels a call launches and, when enabled, brackets each
+// launch with CUDA events on the launching stream so a caller can read per-kernel device time.
+struct LaunchRec {
+    struct Ev { cudaEvent_t a, b; const char* name; };
+    struct Acc { const char* name; double ms; long long n; };
+    cudaStream_t st = nullptr;
+    int launches = 0;
+    bool timing = false;
+    std::vector<Ev> pool;
+    size_t used = 0;
+    std::vector<Acc> acc;
+
+    void start_call(cudaStream_t s) { st = s; launches = 0; }
+    void begin(const char* name) {
+        ++launches;
+        if (!timing) return;
+        if (used == pool.size()) {
+            Ev e{nullptr, nullptr, name};
+            if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) { timing = false; return; }
+            pool.push_back(e);
+        }
+        pool[used].name = name;
+        cudaEventRecord(pool[used].a, st);
+    }
+    bool end() {
+        if (timing && used < pool.size()) cudaEventRecord(pool[used++].b, st);
+        return cudaPeekAtLastError() == cudaSuccess;
+    }
+    // Caller has synchronised the stream.  Folds the recorded pairs into per-name totals (replacing earlier totals).
+    int collect() {
+        acc.clear();
+        for (size_t i = 0; i < used; ++i) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, pool[i].a, pool[i].b) != cudaSuccess) continue;
+            size_t j = 0;
+            for (; j < acc.size(); ++j) if (strcmp(acc[j].name, pool[i].name) == 0) break;
+            if (j == acc.size()) acc.push_back(Acc{pool[i].name, 0.0, 0});
+            acc[j].ms += ms;
+            acc[j].n += 1;
+        }
+        used = 0;
+        return (int)acc.size();
+    }
+    ~LaunchRec() { for (auto& e : pool) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); } }
+};
 
 }  // namespace hla

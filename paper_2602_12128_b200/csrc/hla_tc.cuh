@@ -531,7 +531,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
 // ---- host launch helpers ---------------------------------------------------------------
 template <int DV>
 inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
-                                      const hla_ws_layout& L, size_t off_part, int sm_count, cudaStream_t st, int* launches) {
+                                      const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
     CUtensorMap mapV, mapO, mapB3;
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
     if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens) ||
@@ -548,22 +548,25 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
         if (cudaFuncSetAttribute(tc_readout_kernel<DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, RoCfg<DV>::kSmem) != cudaSuccess) return HLA_ERR_CUDA;
         attr_done = true;
     }
+    cudaStream_t st = rec.st;
+    rec.begin("tc_state_build");
     tc_state_build_kernel<DV><<<dim3(D.S, BH), kSbThreads, kSbSmem, st>>>(mapV, kf, part, D.N, D.S, D.ld, status);
-    ++*launches;
+    if (!rec.end()) return HLA_ERR_CUDA;
+    rec.begin("tc_reduce_emit");
     tc_reduce_emit_kernel<DV><<<BH, 256, 0, st>>>(part, state, b3, D.S, D.ld);
-    ++*launches;
+    if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
+    rec.begin("tc_readout");
     tc_readout_kernel<DV><<<grid, kRoThreads, RoCfg<DV>::kSmem, st>>>(mapB3, mapO, qf, eta, D.N, BH, D.eps, status);
-    ++*launches;
-    return cudaPeekAtLastError() == cudaSuccess ? HLA_OK : HLA_ERR_CUDA;
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
 inline hla_status core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
-                               const hla_ws_layout& L, size_t off_part, int sm_count, cudaStream_t st, int* launches) {
-    if (D.d == 128) return launch_core_forward<128>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, st, launches);
-    return launch_core_forward<64>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, st, launches);
+                               const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
+    if (D.d == 128) return launch_core_forward<128>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec);
+    return launch_core_forward<64>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec);
 }
 
 }  // namespace tc
