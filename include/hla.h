@@ -93,12 +93,16 @@ typedef struct {
     size_t status;   /* int32[16]  device status words                                   */
     size_t qf;       /* fp32 [B,H,N,d_phi]     features phi_q(Q)        (HLA_PHI_MLP)   */
     size_t kf;       /* fp32 [B,H,F,N,d_phi]   features phi_kf(K)       (HLA_PHI_MLP)   */
-    size_t state;    /* fp32 [B,H,P,state_ld]  columns 0..d-1 = C, column d = z         */
+    size_t state;    /* fp32 [B,H,state_rows,state_ld]  columns 0..d-1 = C, column d = z.  state_rows = P = d_phi^F
+                        on the SIMT path.  The tensor-core path keeps the state folded over the permutation
+                        symmetry of the query tensor q (x) q (x) q: row m = (a <= b <= c) in lexicographic order
+                        holds the sum of C over the distinct permutations of (a,b,c); 56 rows for F = 3, d_phi = 6 */
     size_t eta;      /* fp32 [B,H,N]           normaliser before eps                    */
-    size_t dstate;   /* fp32 [B,H,P,state_ld]  dC | dz   (after hla_backward)           */
+    size_t dstate;   /* fp32 [B,H,state_rows,state_ld]  gradient of the loss w.r.t. that state (after hla_backward) */
     size_t dqf;      /* fp32 [B,H,N,d_phi]     feature gradients        (HLA_PHI_MLP)   */
     size_t dkf;      /* fp32 [B,H,F,N,d_phi]                            (HLA_PHI_MLP)   */
     int32_t state_ld; /* row stride of state / dstate in floats (>= d+1)                */
+    int32_t state_rows;
     int32_t n_splits; /* the split count in use                                          */
     int32_t tensor_core; /* 1 if this configuration runs the tcgen05 kernels              */
 } hla_ws_layout;

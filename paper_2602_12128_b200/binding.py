@@ -34,7 +34,7 @@ class HlaMlp(ctypes.Structure):
 
 class HlaWsLayout(ctypes.Structure):
     _fields_ = [("status", c_size_t), ("qf", c_size_t), ("kf", c_size_t), ("state", c_size_t), ("eta", c_size_t),
-                ("dstate", c_size_t), ("dqf", c_size_t), ("dkf", c_size_t), ("state_ld", c_int32), ("n_splits", c_int32),
+                ("dstate", c_size_t), ("dqf", c_size_t), ("dkf", c_size_t), ("state_ld", c_int32), ("state_rows", c_int32), ("n_splits", c_int32),
                 ("tensor_core", c_int32)]
 
 

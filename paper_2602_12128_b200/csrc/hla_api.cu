@@ -260,6 +260,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     L.dqf = mlp ? cv.take(tok * c.d_phi * 4) : kNone;
     L.dkf = mlp ? cv.take(tok * c.F * c.d_phi * 4) : kNone;
     L.state_ld = D.ld;
+    L.state_rows = x->tc ? tc::kMono : P;
     L.n_splits = S;
     L.tensor_core = x->tc ? 1 : 0;
     x->off_part = cv.take((size_t)x->BH * S * P * D.ld * 4);
@@ -331,6 +332,16 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     char* ws = static_cast<char*>(workspace);
     ctx->rec.start_call(st);
     (void)cudaGetLastError();
+    if (ctx->tc) {
+        const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
+        const float* qf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.qf) : static_cast<const float*>(Q);
+        const float* kf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.kf) : static_cast<const float*>(K);
+        float* dqf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dqf) : static_cast<float*>(dQ);
+        float* dkf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dkf) : static_cast<float*>(dK);
+        s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
+        if (s != HLA_OK || !mlp) return s;
+        return simt_phi_backward<__nv_bfloat16>(ctx, Q, K, dQ, dK, ws, st);
+    }
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
 }

@@ -1,15 +1,23 @@
-// Tensor-core (tcgen05 / TMEM / TMA) kernels of the HLA path for bf16,
-// F = 3 factors with d_phi = 6 (P = 216 features), d in {64, 128}.
+// Tensor-core (tcgen05 / TMEM / TMA) kernels of the HLA core for bf16, F = 3
+// factors with d_phi = 6 (P = 216 features), d in {64, 128}.
 //
-//   state build  : C^T[d x P] += V_tile^T[d x 128 tok] * T_k tile[128 tok x P]   (Theorem 4.2, C = T_k (x)_1 V)
-//                  T_k rows are formed in registers from the 3 x 6 key features of each token, rounded once to
-//                  bf16 and written straight into the swizzled shared-memory operand tile; z = sum_j T_k[j] is
-//                  accumulated in fp32 registers on the way.
-//   reduce/emit  : sums the split partials in a fixed order, keeps the fp32 state, and emits the readout operand.
-//   readout      : T_q[i] = q_i (x) q_i (x) q_i is symmetric, so only its 56 distinct monomials q_a q_b q_c
-//                  (a <= b <= c) are formed, against the state folded over index permutations
-//                  (Csym[m] = sum over distinct permutations of C[abc]).  One MMA per tile gives
-//                  num (d columns) and eta (the extra column holding zsym); o = num / (eta + eps).
+// Symmetry folding.  The query tensor T_q[i] = q_i (x) q_i (x) q_i is symmetric, so the
+// readout sum_p T_q[i][p] C[p] only sees C summed over index permutations:
+//     sum_p T_q[i][p] C[p][g] = sum_m mono_i[m] Csym[m][g],   m = (a <= b <= c), 56 monomials,
+//     mono_i[m] = q_a q_b q_c,   Csym[m] = sum over the distinct permutations (x,y,z) of (a,b,c) of C[xyz].
+// Because C = sum_j T_k[j] v_j^T (Theorem 4.2), Csym = sum_j Tsym_k[j] v_j^T with the folded key
+// feature Tsym_k[j][m] = sum over distinct permutations of k1_j[x] k2_j[y] k3_j[z].  So every
+// contraction of the path runs over 56 (padded to 64) features instead of 216, with identical
+// results up to rounding order; the kept state is the folded one, [56][d] (+ the folded z).
+//
+//   state build : Csym^T[d x 64] += V_tile^T[d x 128 tok] * Tsym_k tile[128 tok x 64]; zsym in fp32 registers
+//   reduce/emit : fixed-order sum of the split partials; emits the bf16 MMA operands of the state
+//   readout     : [num | eta][128 tok x (d+16)] = mono tile[128 x 64] * [Csym | zsym]; o = num / (eta + eps)
+//   bwd (query) : D2 = dO * Csym^T -> delta, dmono, dq on the ALUs;  dCsym^T += dO^T * (r mono);  dzsym on the ALUs
+//   bwd (key)   : dV = Tsym_k * dCsym;  G = V * dCsym^T + dzsym -> dk1, dk2, dk3 on the ALUs
+//
+// Operand tiles are formed in registers, rounded once to bf16 and written straight into the
+// 128-byte-swizzled shared-memory layout the MMA descriptors describe; T_q / T_k never exist in global memory.
 #pragma once
 #include "../../include/hla.h"
 #include "hla_common.cuh"
@@ -19,14 +27,23 @@ namespace hla {
 namespace tc {
 
 constexpr int kTileTokens = 128;
-constexpr int kP = 216;          // d_phi^F
-constexpr int kNP = 224;         // P rounded up to the MMA's N granularity
 constexpr int kMono = 56;        // distinct monomials of degree 3 in 6 variables
 constexpr int kMonoPad = 64;
 constexpr int kBlk = 16384;      // one 128-row x 128-byte swizzled block
 
+// index of the monomial (a <= b <= c) in lexicographic order
+__host__ __device__ constexpr int mono_idx(int a, int b, int c) { return a * (a * a - 21 * a + 146) / 6 + (b - a) * (13 - a - b) / 2 + (c - b); }
+__host__ __device__ constexpr int imin(int a, int b) { return a < b ? a : b; }
+__host__ __device__ constexpr int imax(int a, int b) { return a > b ? a : b; }
+__host__ __device__ constexpr int mono_of(int x, int y, int z) {
+    return mono_idx(imin(imin(x, y), z), x + y + z - imin(imin(x, y), z) - imax(imax(x, y), z), imax(imax(x, y), z));
+}
+
 struct Plan {
-    size_t b3;     // bf16 [BH][d+16][64]  readout operand: rows g < d: Csym[.][g]; row d: zsym; rest 0
+    size_t b3;    // bf16 [BH][d+16][64]  rows g < d: Csym[.][g] (K-major over m); row d: zsym; rest 0
+    size_t bq;    // bf16 [BH][64][d]     Csym[m][.]
+    size_t bd3;   // the same two operands of the gradient state (dCsym | dzsym)
+    size_t bdq;
     size_t end;
 };
 
@@ -34,8 +51,11 @@ inline bool supported(bool bf16, int d, int F, int dphi) { return bf16 && (d == 
 
 inline size_t plan(Plan& p, const Dims& D, int BH, size_t off) {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-    p.b3 = off;
-    off = up(off + (size_t)BH * (D.d + 16) * kMonoPad * 2);
+    const size_t n3 = (size_t)BH * (D.d + 16) * kMonoPad * 2, nq = (size_t)BH * kMonoPad * D.d * 2;
+    p.b3 = off; off = up(off + n3);
+    p.bq = off; off = up(off + nq);
+    p.bd3 = off; off = up(off + n3);
+    p.bdq = off; off = up(off + nq);
     p.end = off;
     return off;
 }
@@ -68,85 +88,156 @@ inline bool make_map_bhnd(CUtensorMap* m, const void* ptr, int BH, int N, int d,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// bf16 matrix [rows][64], box = 64 x box_rows, 128-byte swizzle.
-inline bool make_map_rows64(CUtensorMap* m, const void* ptr, size_t rows, int box_rows) {
+// bf16 matrix [rows][cols], box = 64 columns x box_rows, 128-byte swizzle.
+inline bool make_map_2d(CUtensorMap* m, const void* ptr, size_t rows, int cols, int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {64, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {128};
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t es[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// ---- small device helpers ----------------------------------------------------------------
 __device__ __forceinline__ void report_timeout(int* status, int where) {
     atomicExch(status + kStatusTimeout, 1);
     atomicExch(status + kStatusWhere, where);
 }
-
 __device__ __forceinline__ void named_barrier(int id, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
-
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void load6(float* dst, const float* __restrict__ src) {
+    const float2* s = reinterpret_cast<const float2*>(src);
+    const float2 a = __ldg(s), b = __ldg(s + 1), c = __ldg(s + 2);
+    dst[0] = a.x; dst[1] = a.y; dst[2] = b.x; dst[3] = b.y; dst[4] = c.x; dst[5] = c.y;
+}
+__device__ __forceinline__ void store6(float* dst, const float* v) {
+    float2* d = reinterpret_cast<float2*>(dst);
+    d[0] = make_float2(v[0], v[1]); d[1] = make_float2(v[2], v[3]); d[2] = make_float2(v[4], v[5]);
+}
+
+// One operand row of 64 bf16 (56 values * scale, 8 zeros) into row `row` of a swizzled 128-row block.
+__device__ __forceinline__ void store_mono_row(uint32_t blk, uint32_t row, const float (&m)[kMono], float scale) {
+#pragma unroll
+    for (int c = 0; c < 7; ++c)
+        st_shared_v4(blk + sw128_off(row, c), pack_bf16(m[8 * c] * scale, m[8 * c + 1] * scale), pack_bf16(m[8 * c + 2] * scale, m[8 * c + 3] * scale),
+                     pack_bf16(m[8 * c + 4] * scale, m[8 * c + 5] * scale), pack_bf16(m[8 * c + 6] * scale, m[8 * c + 7] * scale));
+    st_shared_v4(blk + sw128_off(row, 7), 0u, 0u, 0u, 0u);
+}
+
+// mono[m] = q_a q_b q_c for a <= b <= c.
+__device__ __forceinline__ void query_monomials(const float (&q)[6], float (&mono)[kMono]) {
+#pragma unroll
+    for (int a = 0; a < 6; ++a)
+#pragma unroll
+        for (int b = a; b < 6; ++b) {
+            const float qab = q[a] * q[b];
+#pragma unroll
+            for (int c = b; c < 6; ++c) mono[mono_idx(a, b, c)] = qab * q[c];
+        }
+}
+
+// dq[x] = sum_m dmono[m] * d(q_a q_b q_c)/dq_x.
+__device__ __forceinline__ void query_monomials_grad(const float (&q)[6], const float (&dm)[kMono], float (&dq)[6]) {
+    float qq[6][6];
+#pragma unroll
+    for (int a = 0; a < 6; ++a)
+#pragma unroll
+        for (int b = a; b < 6; ++b) qq[a][b] = q[a] * q[b];
+#pragma unroll
+    for (int a = 0; a < 6; ++a) dq[a] = 0.f;
+#pragma unroll
+    for (int a = 0; a < 6; ++a)
+#pragma unroll
+        for (int b = a; b < 6; ++b)
+#pragma unroll
+            for (int c = b; c < 6; ++c) {
+                const float g = dm[mono_idx(a, b, c)];
+                dq[a] = fmaf(g, qq[b][c], dq[a]);
+                dq[b] = fmaf(g, qq[a][c], dq[b]);
+                dq[c] = fmaf(g, qq[a][b], dq[c]);
+            }
+}
+
+// Folded key features: ts[m] = sum over the distinct permutations (x,y,z) of m = (a,b,c) of k1[x] k2[y] k3[z].
+// k = (k1[0..5], k2[0..5], k3[0..5]).
+__device__ __forceinline__ void key_folded(const float (&k)[18], float (&ts)[kMono]) {
+    float s12[6][6];   // [x][y], x < y: k1[x]k2[y] + k1[y]k2[x];  [x][x]: k1[x]k2[x]
+#pragma unroll
+    for (int x = 0; x < 6; ++x)
+#pragma unroll
+        for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k[x] * k[6 + x] : fmaf(k[x], k[6 + y], k[y] * k[6 + x]);
+#pragma unroll
+    for (int a = 0; a < 6; ++a)
+#pragma unroll
+        for (int b = a; b < 6; ++b)
+#pragma unroll
+            for (int c = b; c < 6; ++c) {
+                float v;
+                if (a == b && b == c) v = s12[a][a] * k[12 + a];
+                else if (a == b) v = fmaf(s12[a][a], k[12 + c], s12[a][c] * k[12 + a]);
+                else if (b == c) v = fmaf(s12[a][c], k[12 + c], s12[c][c] * k[12 + a]);
+                else v = fmaf(s12[a][b], k[12 + c], fmaf(s12[a][c], k[12 + b], s12[b][c] * k[12 + a]));
+                ts[mono_idx(a, b, c)] = v;
+            }
+}
+
+// Gradients of L = sum_{x,y,z} G[sort(x,y,z)] k1[x] k2[y] k3[z] with respect to k1, k2, k3.
+__device__ __forceinline__ void key_folded_grad(const float (&k)[18], const float (&G)[kMono], float (&dk)[18]) {
+    float s12[6][6];
+#pragma unroll
+    for (int x = 0; x < 6; ++x)
+#pragma unroll
+        for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k[x] * k[6 + x] : fmaf(k[x], k[6 + y], k[y] * k[6 + x]);
+#pragma unroll
+    for (int i = 0; i < 18; ++i) dk[i] = 0.f;
+#pragma unroll
+    for (int z = 0; z < 6; ++z)
+#pragma unroll
+        for (int x = 0; x < 6; ++x)
+#pragma unroll
+            for (int y = x; y < 6; ++y) dk[12 + z] = fmaf(G[mono_of(x, y, z)], s12[x][y], dk[12 + z]);
+#pragma unroll
+    for (int x = 0; x < 6; ++x)
+#pragma unroll
+        for (int y = x; y < 6; ++y) {
+            float h = 0.f;   // H[x][y] = sum_z G[sort(x,y,z)] k3[z], symmetric in (x, y)
+#pragma unroll
+            for (int z = 0; z < 6; ++z) h = fmaf(G[mono_of(x, y, z)], k[12 + z], h);
+            dk[x] = fmaf(h, k[6 + y], dk[x]);
+            dk[6 + y] = fmaf(h, k[x], dk[6 + y]);
+            if (x != y) {
+                dk[y] = fmaf(h, k[6 + x], dk[y]);
+                dk[6 + x] = fmaf(h, k[y], dk[6 + x]);
+            }
+        }
 }
 
 // =======================================================================================
 // State build
 // =======================================================================================
-constexpr int kSbThreads = 320;            // warp 0: TMA, warp 1: MMA, warps 2..9: T_k generators
-constexpr int kSbStages = 2;
-constexpr int kSbStageBytes = 2 * kBlk + 4 * kBlk;   // V (two 64-column blocks) + T_k (four 64-feature blocks)
-constexpr int kSbZHalf0 = 14 * 8;          // features 0..111 belong to the first generator half, 112..215 to the second
-constexpr int kSbSmem = 1024 + kSbStages * kSbStageBytes + 8 * kSbZHalf0 * 4 + 256;
-
-// One generator thread: half of the 216 products of one token -> bf16 operand row + fp32 z accumulators.
-template <int HALF>
-__device__ __forceinline__ void sb_generate(const float (&k)[18], float (&zacc)[kSbZHalf0], uint32_t t_tile, uint32_t row) {
-    constexpr int C0 = HALF ? 14 : 0, C1 = HALF ? 27 : 14;
-    float k12[36];
-#pragma unroll
-    for (int ab = 0; ab < 36; ++ab) k12[ab] = k[ab / 6] * k[6 + ab % 6];
-#pragma unroll
-    for (int c = C0; c < C1; ++c) {
-        float t[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int p = 8 * c + e;
-            t[e] = k12[p / 6] * k[12 + p % 6];
-            zacc[p - 8 * C0] += t[e];
-        }
-        st_shared_v4(t_tile + (c >> 3) * kBlk + sw128_off(row, c & 7), pack_bf16(t[0], t[1]), pack_bf16(t[2], t[3]),
-                     pack_bf16(t[4], t[5]), pack_bf16(t[6], t[7]));
-    }
-}
-
-__device__ __forceinline__ void sb_load_features(float (&k)[18], const float* __restrict__ kf, int bh, int N, int tok) {
-    if (tok < N) {
-#pragma unroll
-        for (int f = 0; f < 3; ++f) {
-            const float2* src = reinterpret_cast<const float2*>(kf + (((size_t)bh * 3 + f) * N + tok) * 6);
-            const float2 a = __ldg(src), b = __ldg(src + 1), c = __ldg(src + 2);
-            k[6 * f + 0] = a.x; k[6 * f + 1] = a.y; k[6 * f + 2] = b.x; k[6 * f + 3] = b.y; k[6 * f + 4] = c.x; k[6 * f + 5] = c.y;
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 18; ++i) k[i] = 0.f;
-    }
-}
+constexpr int kSbThreads = 320;            // warp 0: TMA, warp 1: MMA, warps 2..9: two generator groups of 128 threads
+constexpr int kSbStages = 4;
+constexpr int kSbStageBytes = 2 * kBlk + kBlk;   // V (two 64-column blocks) + folded key tile (one block)
+constexpr int kSbOffZ = kSbStages * kSbStageBytes;              // zred [8 warps][64] floats
+constexpr int kSbOffBars = kSbOffZ + 8 * 64 * 4;
+constexpr int kSbSmem = 1024 + kSbOffBars + 256;
 
 template <int DV>
 __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __grid_constant__ CUtensorMap mapV, const float* __restrict__ kf,
                                                                        float* __restrict__ part, int N, int S, int ld, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    float* zred = reinterpret_cast<float*>(smem + kSbStages * kSbStageBytes);          // [8 warps][112]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSbStages * kSbStageBytes + 8 * kSbZHalf0 * 4);
-    uint64_t* full_v = bars;            // [2]
-    uint64_t* full_t = bars + 2;        // [2]
-    uint64_t* empty = bars + 4;         // [2]
-    uint64_t* acc_done = bars + 6;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7);
+    float* zred = reinterpret_cast<float*>(smem + kSbOffZ);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSbOffBars);
+    uint64_t* full_v = bars;                    // [4]
+    uint64_t* full_t = bars + kSbStages;        // [4]
+    uint64_t* empty = bars + 2 * kSbStages;     // [4]
+    uint64_t* acc_done = bars + 3 * kSbStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSbStages + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int s = blockIdx.x, bh = blockIdx.y;
@@ -154,28 +245,23 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     const int tiles_per = (tiles + S - 1) / S;
     const int tile0 = s * tiles_per;
     const int ntiles = max(0, min(tiles, tile0 + tiles_per) - tile0);
-    float* out = part + ((size_t)bh * S + s) * kP * ld;
+    float* out = part + ((size_t)bh * S + s) * kMono * ld;
 
     if (ntiles == 0) {   // an empty split contributes zeros
-        for (int i = tid; i < kP * ld; i += kSbThreads) out[i] = 0.f;
+        for (int i = tid; i < kMono * ld; i += kSbThreads) out[i] = 0.f;
         return;
     }
-
-    // zero what the generators never write: feature columns 216..223 of each T_k tile, and for d = 64 the
-    // second V block (rows 64..127 of the MMA's M dimension read it)
-    for (int st = 0; st < kSbStages; ++st) {
-        uint8_t* tt = smem + st * kSbStageBytes + 2 * kBlk;
-        for (int r = tid; r < kTileTokens; r += kSbThreads) *reinterpret_cast<uint4*>(tt + 3 * kBlk + sw128_off(r, 3)) = make_uint4(0, 0, 0, 0);
-        if (DV == 64) {
+    if (DV == 64) {      // rows 64..127 of the MMA's M dimension read a second V block: keep it zero
+        for (int st = 0; st < kSbStages; ++st) {
             uint4* vz = reinterpret_cast<uint4*>(smem + st * kSbStageBytes + kBlk);
             for (int i = tid; i < kBlk / 16; i += kSbThreads) vz[i] = make_uint4(0, 0, 0, 0);
         }
+        fence_proxy_async();
     }
-    fence_proxy_async();
     if (tid == 0) {
         for (int i = 0; i < kSbStages; ++i) {
             mbar_init(&full_v[i], 1);
-            mbar_init(&full_t[i], 256);
+            mbar_init(&full_t[i], 128);
             mbar_init(&empty[i], 1);
         }
         mbar_init(acc_done, 1);
@@ -183,7 +269,7 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
         prefetch_tmap(&mapV);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, 256);
+        tmem_alloc(tmem_slot, 64);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -194,10 +280,9 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int it = 0; it < ntiles && ok; ++it) {
-                const int st = it & 1, u = it >> 1;
-                ok = mbar_wait(&empty[st], (u & 1) ^ 1);
-                if (!ok) { report_timeout(status, 101); break; }
+            for (int it = 0; it < ntiles; ++it) {
+                const int st = it % kSbStages, u = it / kSbStages;
+                if (!mbar_wait(&empty[st], (u & 1) ^ 1)) { report_timeout(status, 101); break; }
                 uint8_t* vs = smem + st * kSbStageBytes;
                 mbar_arrive_expect_tx(&full_v[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b) tma_load_3d(vs + b * kBlk, &mapV, &full_v[st], b * 64, (tile0 + it) * kTileTokens, bh);
@@ -205,11 +290,10 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = idesc_bf16(128, kNP, true, true);
-            for (int it = 0; it < ntiles && ok; ++it) {
-                const int st = it & 1, u = it >> 1;
-                ok = mbar_wait(&full_v[st], u & 1) && mbar_wait(&full_t[st], u & 1);
-                if (!ok) { report_timeout(status, 102); break; }
+            const uint32_t idesc = idesc_bf16(128, kMonoPad, true, true);
+            for (int it = 0; it < ntiles; ++it) {
+                const int st = it % kSbStages, u = it / kSbStages;
+                if (!(mbar_wait(&full_v[st], u & 1) && mbar_wait(&full_t[st], u & 1))) { report_timeout(status, 102); break; }
                 tc_fence_after();
                 const uint32_t va = smem_u32(smem + st * kSbStageBytes), ta = va + 2 * kBlk;
 #pragma unroll
@@ -221,57 +305,57 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
             umma_commit(acc_done);
         }
     } else {
-        const int gi = tid - 64;
-        const int row = gi & 127, half = gi >> 7;
-        float zacc[kSbZHalf0];
+        const int grp = (warp - 2) >> 2;
+        const int row = ((warp - 2) & 3) * 32 + lane;
+        float zacc[kMono];
 #pragma unroll
-        for (int i = 0; i < kSbZHalf0; ++i) zacc[i] = 0.f;
-        float kcur[18], knext[18];
-        sb_load_features(knext, kf, bh, N, tile0 * kTileTokens + row);
-        for (int it = 0; it < ntiles; ++it) {
-            const int st = it & 1, u = it >> 1;
+        for (int i = 0; i < kMono; ++i) zacc[i] = 0.f;
+        float k[18];
+        for (int it = grp; it < ntiles; it += 2) {
+            const int st = it % kSbStages, u = it / kSbStages;
+            const int tok = (tile0 + it) * kTileTokens + row;
+            if (tok < N) {
 #pragma unroll
-            for (int i = 0; i < 18; ++i) kcur[i] = knext[i];
-            if (it + 1 < ntiles) sb_load_features(knext, kf, bh, N, (tile0 + it + 1) * kTileTokens + row);
-            if (ok) {
-                ok = mbar_wait(&empty[st], (u & 1) ^ 1);
-                if (!ok) report_timeout(status, 103);
+                for (int f = 0; f < 3; ++f) load6(k + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 18; ++i) k[i] = 0.f;
             }
+            float ts[kMono];
+            key_folded(k, ts);
+#pragma unroll
+            for (int i = 0; i < kMono; ++i) zacc[i] += ts[i];
+            if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 103); }
             if (ok) {
-                const uint32_t ta = smem_u32(smem + st * kSbStageBytes + 2 * kBlk);
-                if (half == 0) sb_generate<0>(kcur, zacc, ta, row);
-                else sb_generate<1>(kcur, zacc, ta, row);
+                store_mono_row(smem_u32(smem + st * kSbStageBytes + 2 * kBlk), row, ts, 1.f);
                 fence_proxy_async();
                 mbar_arrive(&full_t[st]);
             }
         }
-        // z: sum the per-token-slot accumulators over the 128 slots of this half
+        // zsym: sum the per-token-slot accumulators over the 256 generator threads
 #pragma unroll
-        for (int i = 0; i < kSbZHalf0; ++i) {
+        for (int i = 0; i < kMono; ++i) {
             const float v = warp_sum(zacc[i]);
-            if (lane == 0) zred[(warp - 2) * kSbZHalf0 + i] = v;
+            if (lane == 0) zred[(warp - 2) * 64 + i] = v;
         }
         named_barrier(1, 256);
-        if (gi < kP) {
-            const int h = gi >= kSbZHalf0 ? 1 : 0, i = gi - h * kSbZHalf0;
+        const int gi = tid - 64;
+        if (gi < kMono) {
             float z = 0.f;
 #pragma unroll
-            for (int w = 0; w < 4; ++w) z += zred[(h * 4 + w) * kSbZHalf0 + i];
+            for (int w = 0; w < 8; ++w) z += zred[w * 64 + gi];
             out[(size_t)gi * ld + DV] = z;
             for (int c = DV + 1; c < ld; ++c) out[(size_t)gi * ld + c] = 0.f;
         }
-        if (warp < 6) {   // warps 2..5 cover the four TMEM lane quarters
+        if (warp < 6) {   // warps 2..5 cover the four TMEM lane quarters (lane = value channel g)
             const int quarter = warp & 3;
-            if (ok) {
-                ok = mbar_wait(acc_done, 0);
-                if (!ok && lane == 0) report_timeout(status, 104);
-            }
+            if (ok && !mbar_wait(acc_done, 0)) { ok = false; report_timeout(status, 104); }
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
             const int g = quarter * 32 + lane;
             if (ok && quarter * 32 < DV) {
-#pragma unroll 1
-                for (int c = 0; c < kP / 8; ++c) {
+#pragma unroll
+                for (int c = 0; c < kMono / 8; ++c) {
                     uint32_t r[8];
                     tmem_ld8(tmem + ((uint32_t)(quarter * 32) << 16) + 8 * c, r);
                     tmem_ld_wait();
@@ -283,53 +367,34 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 256);
+    if (warp == 1) tmem_dealloc(tmem, 64);
 }
 
 // =======================================================================================
-// Reduce the split partials, keep the fp32 state, emit the readout operand
+// Reduce the split partials [BH][S][56][ld] in a fixed order -> fp32 folded state [BH][56][ld]
+// (column d = folded z) and the two bf16 MMA operands of that state.
 // =======================================================================================
 template <int DV>
 __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __restrict__ part, float* __restrict__ state,
-                                                             __nv_bfloat16* __restrict__ b3, int S, int ld) {
-    __shared__ uint8_t perm[kMono][6];
-    __shared__ uint8_t nperm[kMono];
+                                                             __nv_bfloat16* __restrict__ b3, __nv_bfloat16* __restrict__ bq, int S, int ld) {
     const int bh = blockIdx.x, tid = threadIdx.x;
-    const size_t n_per = (size_t)kP * ld;
+    const size_t n_per = (size_t)kMono * ld;
     float* st = state + (size_t)bh * n_per;
     for (size_t i = tid; i < n_per; i += 256) {
         float a = 0.f;
         for (int s = 0; s < S; ++s) a += part[((size_t)bh * S + s) * n_per + i];
         st[i] = a;
     }
-    if (tid < kMono) {
-        int m = 0, A = 0, Bq = 0, C = 0;
-        for (int a = 0; a < 6; ++a)
-            for (int b = a; b < 6; ++b)
-                for (int c = b; c < 6; ++c) {
-                    if (m == tid) { A = a; Bq = b; C = c; }
-                    ++m;
-                }
-        const int idx[3] = {A, Bq, C};
-        const int order[6][3] = {{0, 1, 2}, {0, 2, 1}, {1, 0, 2}, {1, 2, 0}, {2, 0, 1}, {2, 1, 0}};
-        int n = 0;
-        for (int o = 0; o < 6; ++o) {
-            const int p = (idx[order[o][0]] * 6 + idx[order[o][1]]) * 6 + idx[order[o][2]];
-            bool seen = false;
-            for (int j = 0; j < n; ++j) seen |= (perm[tid][j] == p);
-            if (!seen) perm[tid][n++] = (uint8_t)p;
-        }
-        nperm[tid] = (uint8_t)n;
-    }
     __syncthreads();
-    __nv_bfloat16* o = b3 + (size_t)bh * (DV + 16) * kMonoPad;
+    __nv_bfloat16* o3 = b3 + (size_t)bh * (DV + 16) * kMonoPad;
     for (int i = tid; i < (DV + 16) * kMonoPad; i += 256) {
         const int row = i / kMonoPad, m = i % kMonoPad;
-        float v = 0.f;
-        if (m < kMono && row <= DV) {
-            for (int j = 0; j < nperm[m]; ++j) v += st[(size_t)perm[m][j] * ld + row];   // row == DV reads the z column
-        }
-        o[i] = __float2bfloat16_rn(v);
+        o3[i] = __float2bfloat16_rn((m < kMono && row <= DV) ? st[(size_t)m * ld + row] : 0.f);   // row == DV is the z column
+    }
+    __nv_bfloat16* oq = bq + (size_t)bh * kMonoPad * DV;
+    for (int i = tid; i < kMonoPad * DV; i += 256) {
+        const int m = i / DV, g = i % DV;
+        oq[i] = __float2bfloat16_rn(m < kMono ? st[(size_t)m * ld + g] : 0.f);
     }
 }
 
@@ -401,24 +466,21 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
             const uint32_t idesc = idesc_bf16(128, Cfg::kNmma, false, false);
             const uint32_t b3a = smem_u32(smem + Cfg::kOffB3);
             int cur_bh = -1, nload = 0;
-            for (int it = 0; it < nwork && ok; ++it) {
+            for (int it = 0; it < nwork; ++it) {
                 const int work = w0 + it, bh = work / tiles_per_head;
                 const int ab = it & 1, u = it >> 1;
                 if (bh != cur_bh) {
                     if (cur_bh >= 0) {   // every MMA that reads the old state operand must have finished
                         umma_commit(b3_free);
-                        ok = mbar_wait(b3_free, (nload - 1) & 1);
-                        if (!ok) { report_timeout(status, 201); break; }
+                        if (!mbar_wait(b3_free, (nload - 1) & 1)) { report_timeout(status, 201); break; }
                     }
                     mbar_arrive_expect_tx(b3_full, Cfg::kB3Bytes);
                     tma_load_2d(smem + Cfg::kOffB3, &mapB3, b3_full, 0, bh * Cfg::kNmma);
-                    ok = mbar_wait(b3_full, nload & 1);
-                    if (!ok) { report_timeout(status, 202); break; }
+                    if (!mbar_wait(b3_full, nload & 1)) { report_timeout(status, 202); break; }
                     ++nload;
                     cur_bh = bh;
                 }
-                ok = mbar_wait(&a_full[ab], u & 1) && mbar_wait(&acc_empty[ab], (u & 1) ^ 1);
-                if (!ok) { report_timeout(status, 203); break; }
+                if (!(mbar_wait(&a_full[ab], u & 1) && mbar_wait(&acc_empty[ab], (u & 1) ^ 1))) { report_timeout(status, 203); break; }
                 tc_fence_after();
                 const uint32_t aa = smem_u32(smem + Cfg::kOffA + ab * kBlk);
 #pragma unroll
@@ -431,49 +493,20 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
         }
     } else if (warp >= 4) {
         const int row = tid - 128;
-        float q[6], qn[6];
-        auto load_q = [&](float (&dst)[6], int work) {
-            const int bh = work / tiles_per_head, tok = (work % tiles_per_head) * kTileTokens + row;
-            if (tok < N) {
-                const float2* src = reinterpret_cast<const float2*>(qf + ((size_t)bh * N + tok) * 6);
-                const float2 a = __ldg(src), b = __ldg(src + 1), c = __ldg(src + 2);
-                dst[0] = a.x; dst[1] = a.y; dst[2] = b.x; dst[3] = b.y; dst[4] = c.x; dst[5] = c.y;
-            } else {
-#pragma unroll
-                for (int i = 0; i < 6; ++i) dst[i] = 0.f;
-            }
-        };
-        if (nwork > 0) load_q(qn, w0);
         for (int it = 0; it < nwork; ++it) {
+            const int work = w0 + it, bh = work / tiles_per_head, tok = (work % tiles_per_head) * kTileTokens + row;
             const int ab = it & 1, u = it >> 1;
+            float q[6];
+            if (tok < N) load6(q, qf + ((size_t)bh * N + tok) * 6);
+            else {
 #pragma unroll
-            for (int i = 0; i < 6; ++i) q[i] = qn[i];
-            if (it + 1 < nwork) load_q(qn, w0 + it + 1);
-            if (ok) {
-                ok = mbar_wait(&a_empty[ab], (u & 1) ^ 1);
-                if (!ok) report_timeout(status, 204);
+                for (int i = 0; i < 6; ++i) q[i] = 0.f;
             }
+            float mono[kMono];
+            query_monomials(q, mono);
+            if (ok && !mbar_wait(&a_empty[ab], (u & 1) ^ 1)) { ok = false; report_timeout(status, 204); }
             if (!ok) continue;
-            // the 56 monomials q_a q_b q_c, a <= b <= c, in lexicographic order of (a, b, c)
-            float mono[kMonoPad];
-            {
-                int m = 0;
-#pragma unroll
-                for (int a = 0; a < 6; ++a)
-#pragma unroll
-                    for (int b = a; b < 6; ++b) {
-                        const float qab = q[a] * q[b];
-#pragma unroll
-                        for (int c = b; c < 6; ++c) mono[m++] = qab * q[c];
-                    }
-#pragma unroll
-                for (; m < kMonoPad; ++m) mono[m] = 0.f;
-            }
-            const uint32_t aa = smem_u32(smem + Cfg::kOffA + ab * kBlk);
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                st_shared_v4(aa + sw128_off(row, c), pack_bf16(mono[8 * c], mono[8 * c + 1]), pack_bf16(mono[8 * c + 2], mono[8 * c + 3]),
-                             pack_bf16(mono[8 * c + 4], mono[8 * c + 5]), pack_bf16(mono[8 * c + 6], mono[8 * c + 7]));
+            store_mono_row(smem_u32(smem + Cfg::kOffA + ab * kBlk), row, mono, 1.f);
             fence_proxy_async();
             mbar_arrive(&a_full[ab]);
         }
@@ -486,6 +519,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
                 report_timeout(status, 205);
                 *abort_flag = 1;
             }
+            if (tid == 0) tma_store_wait_read1();      // the staging tile of two tiles ago has been read by its store
             named_barrier(3, 128);                     // every epilogue thread arrives, timed out or not
             if (*abort_flag) break;                    // uniform across the four warps
             tc_fence_after();
@@ -495,9 +529,6 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
             tmem_ld_wait();
             const float eta = __uint_as_float(r[0]);
             const float rinv = 1.f / (eta + eps);
-            // the staging tile of two tiles ago must have been read by its TMA store
-            if (tid == 0) tma_store_wait_read1();
-            named_barrier(2, 128);
             const uint32_t os = smem_u32(smem + Cfg::kOffO + ab * Cfg::kOBytes);
 #pragma unroll
             for (int c = 0; c < DV / 16; ++c) {
@@ -528,32 +559,449 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
     if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
+// =======================================================================================
+// Backward, pass over the queries (split over tokens like the state build):
+//   D2[i][m]  = sum_g dO_i[g] Csym[m][g]                                   (MMA, K = d)
+//   s_i       = sum_m mono_i[m] D2[i][m] ;  delta_i = dO_i . o_i = r_i s_i ;  deta_i = -r_i delta_i
+//   dmono_i[m]= r_i D2[i][m] + deta_i zsym[m]  ->  dq_i                     (ALUs)
+//   dCsym^T  += dO_tile^T * (r_i mono_i)                                    (MMA, K = tokens)
+//   dzsym[m] += mono_i[m] deta_i                                            (ALUs)
+// O itself is not read: dO . o is recovered from D2.
+// =======================================================================================
+constexpr int kBqThreads = 320;
+constexpr int kBqStages = 3;
+constexpr int kBqStageBytes = 2 * kBlk + kBlk;          // dO tile (two 64-column blocks) + r*mono tile
+constexpr int kBqOffOp = kBqStages * kBqStageBytes;     // Csym operand [64][d] bf16 (two 8 KB blocks)
+constexpr int kBqOffZ = kBqOffOp + kBlk;                // zsym (64 floats) then zred [8][64]
+constexpr int kBqOffBars = kBqOffZ + 64 * 4 + 8 * 64 * 4;
+constexpr int kBqSmem = 1024 + kBqOffBars + 256;
+
+template <int DV>
+__global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __grid_constant__ CUtensorMap mapdO, const __grid_constant__ CUtensorMap mapBq,
+                                                                     const float* __restrict__ qf, const float* __restrict__ eta,
+                                                                     const float* __restrict__ state, float* __restrict__ dqf,
+                                                                     float* __restrict__ part, int N, int S, int ld, float eps, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    float* zsym = reinterpret_cast<float*>(smem + kBqOffZ);
+    float* zred = zsym + 64;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBqOffBars);
+    uint64_t* full_do = bars;             // [3]
+    uint64_t* full_rm = bars + 3;         // [3] 128 arrivals
+    uint64_t* empty = bars + 6;           // [3] MMA commit
+    uint64_t* d2_full = bars + 9;         // [2] MMA commit
+    uint64_t* d2_empty = bars + 11;       // [2] 128 arrivals
+    uint64_t* op_full = bars + 13;
+    uint64_t* acc_done = bars + 14;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int s = blockIdx.x, bh = blockIdx.y;
+    const int tiles = (N + kTileTokens - 1) / kTileTokens;
+    const int tiles_per = (tiles + S - 1) / S;
+    const int tile0 = s * tiles_per;
+    const int ntiles = max(0, min(tiles, tile0 + tiles_per) - tile0);
+    float* out = part + ((size_t)bh * S + s) * kMono * ld;
+    if (ntiles == 0) {
+        for (int i = tid; i < kMono * ld; i += kBqThreads) out[i] = 0.f;
+        return;
+    }
+    if (DV == 64) {
+        for (int st = 0; st < kBqStages; ++st) {
+            uint4* vz = reinterpret_cast<uint4*>(smem + st * kBqStageBytes + kBlk);
+            for (int i = tid; i < kBlk / 16; i += kBqThreads) vz[i] = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async();
+    }
+    if (tid < 64) zsym[tid] = tid < kMono ? state[((size_t)bh * kMono + tid) * ld + DV] : 0.f;
+    if (tid == 0) {
+        for (int i = 0; i < kBqStages; ++i) {
+            mbar_init(&full_do[i], 1);
+            mbar_init(&full_rm[i], 128);
+            mbar_init(&empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&d2_full[i], 1);
+            mbar_init(&d2_empty[i], 128);
+        }
+        mbar_init(op_full, 1);
+        mbar_init(acc_done, 1);
+        fence_mbar_init();
+        prefetch_tmap(&mapdO);
+        prefetch_tmap(&mapBq);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    bool ok = true;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(op_full, kMonoPad * DV * 2);
+            for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + kBqOffOp + b * (kBlk / 2), &mapBq, op_full, b * 64, bh * kMonoPad);
+            for (int it = 0; it < ntiles; ++it) {
+                const int st = it % kBqStages, u = it / kBqStages;
+                if (!mbar_wait(&empty[st], (u & 1) ^ 1)) { report_timeout(status, 301); break; }
+                uint8_t* ds = smem + st * kBqStageBytes;
+                mbar_arrive_expect_tx(&full_do[st], DV * kTileTokens * 2);
+                for (int b = 0; b < DV / 64; ++b) tma_load_3d(ds + b * kBlk, &mapdO, &full_do[st], b * 64, (tile0 + it) * kTileTokens, bh);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc2 = idesc_bf16(128, kMonoPad, false, false);   // D2 = dO (K-major over g) * Csym (K-major over g)
+            const uint32_t idesc1 = idesc_bf16(128, kMonoPad, true, true);     // dCsym^T += dO^T (MN-major) * r mono (MN-major)
+            const uint32_t opa = smem_u32(smem + kBqOffOp);
+            bool good = mbar_wait(op_full, 0);
+            if (!good) report_timeout(status, 302);
+            for (int it = 0; it < ntiles && good; ++it) {
+                const int st = it % kBqStages, u = it / kBqStages, buf = it & 1, ub = it >> 1;
+                if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&d2_empty[buf], (ub & 1) ^ 1))) { report_timeout(status, 303); break; }
+                tc_fence_after();
+                const uint32_t da = smem_u32(smem + st * kBqStageBytes), ra = da + 2 * kBlk;
+#pragma unroll
+                for (int ks = 0; ks < DV / 16; ++ks)
+                    umma_bf16(tmem + 64 + 64 * buf, smem_desc_sw128(da + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                              smem_desc_sw128(opa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
+                umma_commit(&d2_full[buf]);
+                if (!mbar_wait(&full_rm[st], u & 1)) { report_timeout(status, 304); break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kTileTokens / 16; ++ks)
+                    umma_bf16(tmem, smem_desc_sw128(da + ks * 2048, kBlk, 1024), smem_desc_sw128(ra + ks * 2048, kBlk, 1024), idesc1,
+                              (it > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(&empty[st]);
+            }
+            umma_commit(acc_done);
+        }
+    } else {
+        const int grp = (warp - 2) >> 2, quarter = warp & 3;
+        const int row = quarter * 32 + lane;    // token row of the tile == TMEM lane this thread can read
+        float dzacc[kMono];
+#pragma unroll
+        for (int i = 0; i < kMono; ++i) dzacc[i] = 0.f;
+        for (int it = grp; it < ntiles; it += 2) {
+            const int st = it % kBqStages, u = it / kBqStages, buf = it & 1, ub = it >> 1;
+            const int tok = (tile0 + it) * kTileTokens + row;
+            float q[6], r = 0.f;
+            if (tok < N) {
+                load6(q, qf + ((size_t)bh * N + tok) * 6);
+                r = 1.f / (__ldg(eta + (size_t)bh * N + tok) + eps);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 6; ++i) q[i] = 0.f;
+            }
+            float mono[kMono];
+            query_monomials(q, mono);
+            if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
+            if (ok) {
+                store_mono_row(smem_u32(smem + st * kBqStageBytes + 2 * kBlk), row, mono, r);
+                fence_proxy_async();
+                mbar_arrive(&full_rm[st]);
+            }
+            if (ok && !mbar_wait(&d2_full[buf], ub & 1)) { ok = false; report_timeout(status, 306); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) continue;
+            tc_fence_after();
+            float d2[kMono];
+            const uint32_t ta = tmem + 64 + 64 * buf + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll
+            for (int c = 0; c < kMono / 8; ++c) {
+                uint32_t rr[8];
+                tmem_ld8(ta + 8 * c, rr);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 8; ++e) d2[8 * c + e] = __uint_as_float(rr[e]);
+            }
+            tc_fence_before();
+            mbar_arrive(&d2_empty[buf]);
+            float sdot = 0.f;
+#pragma unroll
+            for (int m = 0; m < kMono; ++m) sdot = fmaf(mono[m], d2[m], sdot);
+            const float deta = -r * r * sdot;
+            float dm[kMono];
+#pragma unroll
+            for (int m = 0; m < kMono; ++m) {
+                dm[m] = fmaf(r, d2[m], deta * zsym[m]);
+                dzacc[m] = fmaf(mono[m], deta, dzacc[m]);
+            }
+            float dq[6];
+            query_monomials_grad(q, dm, dq);
+            if (tok < N) store6(dqf + ((size_t)bh * N + tok) * 6, dq);
+        }
+#pragma unroll
+        for (int i = 0; i < kMono; ++i) {
+            const float v = warp_sum(dzacc[i]);
+            if (lane == 0) zred[(warp - 2) * 64 + i] = v;
+        }
+        named_barrier(1, 256);
+        const int gi = tid - 64;
+        if (gi < kMono) {
+            float z = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) z += zred[w * 64 + gi];
+            out[(size_t)gi * ld + DV] = z;
+            for (int c = DV + 1; c < ld; ++c) out[(size_t)gi * ld + c] = 0.f;
+        }
+        if (warp < 6) {
+            if (ok && !mbar_wait(acc_done, 0)) { ok = false; report_timeout(status, 307); }
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after();
+            if (ok && quarter * 32 < DV) {
+#pragma unroll
+                for (int c = 0; c < kMono / 8; ++c) {
+                    uint32_t rr[8];
+                    tmem_ld8(tmem + ((uint32_t)(quarter * 32) << 16) + 8 * c, rr);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) out[(size_t)(8 * c + e) * ld + row] = __uint_as_float(rr[e]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 256);
+}
+
+// =======================================================================================
+// Backward, pass over the keys (persistent over (head, tile) like the readout):
+//   dV_j      = sum_m Tsym_k[j][m] dCsym[m][:]                               (MMA, K = 64)
+//   G_j[m]    = sum_g v_j[g] dCsym[m][g] + dzsym[m]                          (MMA, K = d; + on the ALUs)
+//   dk1, dk2, dk3 from G_j and the key features                              (ALUs)
+// =======================================================================================
+constexpr int kBkThreads = 320;   // warp 0: TMA loads, warp 1: MMA, warps 2..9: two worker groups of 128 threads
+template <int DV> struct BkCfg {
+    static constexpr int kVBytes = 2 * kBlk;                              // V stage (two 64-column blocks; d = 64 uses one)
+    static constexpr int kOffV = 0;                                       // 2 stages
+    static constexpr int kOffA = 2 * kVBytes;                             // 2 folded key tiles (one per group)
+    static constexpr int kOffB3 = kOffA + 2 * kBlk;                       // dCsym operand [d+16][64]
+    static constexpr int kB3Bytes = (DV + 16) * 128;
+    static constexpr int kOffBq = kOffB3 + ((kB3Bytes + 1023) / 1024) * 1024;   // dCsym operand [64][d]
+    static constexpr int kOffO = kOffBq + kBlk;                           // 2 dV staging tiles (one per group)
+    static constexpr int kOBytes = kTileTokens * DV * 2;
+    static constexpr int kOffBars = kOffO + 2 * kOBytes;
+    static constexpr int kSmemUsed = 1024 + kOffBars + 256;
+    static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
+};
+
+template <int DV>
+__global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapB3,
+                                                                   const __grid_constant__ CUtensorMap mapBq, const __grid_constant__ CUtensorMap mapdV,
+                                                                   const float* __restrict__ kf, const float* __restrict__ dstate,
+                                                                   float* __restrict__ dkf, int N, int BH, int ld, int* status) {
+    using Cfg = BkCfg<DV>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
+    uint64_t* full_v = bars;            // [2]
+    uint64_t* empty_v = bars + 2;       // [2] MMA commit
+    uint64_t* a_full = bars + 4;        // [2] 128 arrivals (per group)
+    uint64_t* d4_full = bars + 6;       // [2] MMA commit
+    uint64_t* d3_full = bars + 8;       // [2] MMA commit
+    uint64_t* acc_empty = bars + 10;    // [2] 128 arrivals
+    uint64_t* op_full = bars + 12;
+    uint64_t* op_free = bars + 13;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tiles_per_head = (N + kTileTokens - 1) / kTileTokens;
+    const long long total = (long long)BH * tiles_per_head;
+    const int w0 = (int)(total * blockIdx.x / gridDim.x), w1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    const int nwork = w1 - w0;
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&full_v[i], 1);
+            mbar_init(&empty_v[i], 1);
+            mbar_init(&a_full[i], 128);
+            mbar_init(&d4_full[i], 1);
+            mbar_init(&d3_full[i], 1);
+            mbar_init(&acc_empty[i], 128);
+        }
+        mbar_init(op_full, 1);
+        mbar_init(op_free, 1);
+        fence_mbar_init();
+        prefetch_tmap(&mapV);
+        prefetch_tmap(&mapB3);
+        prefetch_tmap(&mapBq);
+        prefetch_tmap(&mapdV);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;     // D3[grp] at columns 128*grp, D4[grp] at columns 256 + 64*grp
+    bool ok = true;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int it = 0; it < nwork; ++it) {
+                const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
+                const int st = it & 1, u = it >> 1;
+                if (!mbar_wait(&empty_v[st], (u & 1) ^ 1)) { report_timeout(status, 401); break; }
+                uint8_t* vs = smem + Cfg::kOffV + st * Cfg::kVBytes;
+                mbar_arrive_expect_tx(&full_v[st], DV * kTileTokens * 2);
+                for (int b = 0; b < DV / 64; ++b) tma_load_3d(vs + b * kBlk, &mapV, &full_v[st], b * 64, tile * kTileTokens, bh);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc4 = idesc_bf16(128, kMonoPad, false, false);   // G  = V (K-major over g) * dCsym (K-major over g)
+            const uint32_t idesc3 = idesc_bf16(128, DV, false, false);         // dV = Tsym_k (K-major over m) * dCsym^T (K-major over m)
+            const uint32_t b3a = smem_u32(smem + Cfg::kOffB3), bqa = smem_u32(smem + Cfg::kOffBq);
+            int cur_bh = -1, nload = 0;
+            for (int it = 0; it < nwork; ++it) {
+                const int work = w0 + it, bh = work / tiles_per_head;
+                const int st = it & 1, u = it >> 1, grp = it & 1;
+                if (bh != cur_bh) {
+                    if (cur_bh >= 0) {
+                        umma_commit(op_free);
+                        if (!mbar_wait(op_free, (nload - 1) & 1)) { report_timeout(status, 402); break; }
+                    }
+                    mbar_arrive_expect_tx(op_full, Cfg::kB3Bytes + kMonoPad * DV * 2);
+                    tma_load_2d(smem + Cfg::kOffB3, &mapB3, op_full, 0, bh * (DV + 16));
+                    for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + Cfg::kOffBq + b * (kBlk / 2), &mapBq, op_full, b * 64, bh * kMonoPad);
+                    if (!mbar_wait(op_full, nload & 1)) { report_timeout(status, 403); break; }
+                    ++nload;
+                    cur_bh = bh;
+                }
+                if (!(mbar_wait(&full_v[st], u & 1) && mbar_wait(&acc_empty[grp], (u & 1) ^ 1))) { report_timeout(status, 404); break; }
+                tc_fence_after();
+                const uint32_t va = smem_u32(smem + Cfg::kOffV + st * Cfg::kVBytes);
+#pragma unroll
+                for (int ks = 0; ks < DV / 16; ++ks)
+                    umma_bf16(tmem + 256 + 64 * grp, smem_desc_sw128(va + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                              smem_desc_sw128(bqa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc4, ks > 0 ? 1u : 0u);
+                umma_commit(&d4_full[grp]);
+                umma_commit(&empty_v[st]);
+                if (!mbar_wait(&a_full[grp], u & 1)) { report_timeout(status, 405); break; }
+                tc_fence_after();
+                const uint32_t aa = smem_u32(smem + Cfg::kOffA + grp * kBlk);
+#pragma unroll
+                for (int ks = 0; ks < kMonoPad / 16; ++ks)
+                    umma_bf16(tmem + 128 * grp, smem_desc_sw128(aa + ks * 32, 16, 1024), smem_desc_sw128(b3a + ks * 32, 16, 1024), idesc3,
+                              ks > 0 ? 1u : 0u);
+                umma_commit(&d3_full[grp]);
+            }
+        }
+    } else {
+        const int grp = (warp - 2) >> 2, quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const bool leader = (warp - 2) == 4 * grp && lane == 0;
+        for (int it = grp; it < nwork; it += 2) {
+            const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
+            const int u = it >> 1;
+            const int tok = tile * kTileTokens + row;
+            float k[18];
+            if (tok < N) {
+#pragma unroll
+                for (int f = 0; f < 3; ++f) load6(k + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 18; ++i) k[i] = 0.f;
+            }
+            {
+                float ts[kMono];
+                key_folded(k, ts);
+                // the folded key tile of this group is free: its last reader (the dV MMA two tiles ago) was waited for below
+                store_mono_row(smem_u32(smem + Cfg::kOffA + grp * kBlk), row, ts, 1.f);
+                fence_proxy_async();
+                mbar_arrive(&a_full[grp]);
+            }
+            // ---- G -> dk
+            if (ok && !mbar_wait(&d4_full[grp], u & 1)) { ok = false; report_timeout(status, 406); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                float G[kMono];
+                const uint32_t ta = tmem + 256 + 64 * grp + ((uint32_t)(quarter * 32) << 16);
+                const float* dz = dstate + (size_t)bh * kMono * ld + DV;
+#pragma unroll
+                for (int c = 0; c < kMono / 8; ++c) {
+                    uint32_t rr[8];
+                    tmem_ld8(ta + 8 * c, rr);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) G[8 * c + e] = __uint_as_float(rr[e]) + __ldg(dz + (size_t)(8 * c + e) * ld);
+                }
+                float dk[18];
+                key_folded_grad(k, G, dk);
+                if (tok < N) {
+#pragma unroll
+                    for (int f = 0; f < 3; ++f) store6(dkf + (((size_t)bh * 3 + f) * N + tok) * 6, dk + 6 * f);
+                }
+            }
+            // ---- dV
+            if (ok && !mbar_wait(&d3_full[grp], u & 1)) { ok = false; report_timeout(status, 407); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (leader) tma_store_wait_read0();          // this group's staging tile has been read by its previous store
+            named_barrier(1 + grp, 128);
+            if (ok) {
+                tc_fence_after();
+                const uint32_t ta = tmem + 128 * grp + ((uint32_t)(quarter * 32) << 16);
+                const uint32_t os = smem_u32(smem + Cfg::kOffO + grp * Cfg::kOBytes);
+#pragma unroll
+                for (int c = 0; c < DV / 16; ++c) {
+                    uint32_t r[16];
+                    tmem_ld16(ta + 16 * c, r);
+                    tmem_ld_wait();
+                    uint32_t w[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                    const uint32_t blk = os + (c >> 2) * kBlk;
+                    st_shared_v4(blk + sw128_off(row, (2 * c) & 7), w[0], w[1], w[2], w[3]);
+                    st_shared_v4(blk + sw128_off(row, (2 * c + 1) & 7), w[4], w[5], w[6], w[7]);
+                }
+                tc_fence_before();
+                mbar_arrive(&acc_empty[grp]);
+                fence_proxy_async();
+            }
+            named_barrier(1 + grp, 128);
+            if (ok && leader) {
+                for (int b = 0; b < DV / 64; ++b) tma_store_3d(&mapdV, smem + Cfg::kOffO + grp * Cfg::kOBytes + b * kBlk, b * 64, tile * kTileTokens, bh);
+                tma_store_commit();
+            }
+        }
+        if (leader) tma_store_wait_all0();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
 // ---- host launch helpers ---------------------------------------------------------------
+template <typename K>
+inline bool set_smem(K kernel, int bytes) { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess; }
+
 template <int DV>
 inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
                                       const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
     CUtensorMap mapV, mapO, mapB3;
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
+    __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
     if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens) ||
-        !make_map_rows64(&mapB3, b3, (size_t)BH * (DV + 16), DV + 16))
+        !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), kMonoPad, DV + 16))
         return HLA_ERR_CUDA;
     int* status = reinterpret_cast<int*>(ws + L.status);
     float* part = reinterpret_cast<float*>(ws + off_part);
     float* state = reinterpret_cast<float*>(ws + L.state);
     float* eta = reinterpret_cast<float*>(ws + L.eta);
-
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(tc_state_build_kernel<DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSbSmem) != cudaSuccess) return HLA_ERR_CUDA;
-        if (cudaFuncSetAttribute(tc_readout_kernel<DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, RoCfg<DV>::kSmem) != cudaSuccess) return HLA_ERR_CUDA;
-        attr_done = true;
-    }
+    if (!set_smem(tc_state_build_kernel<DV>, kSbSmem) || !set_smem(tc_readout_kernel<DV>, RoCfg<DV>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
     rec.begin("tc_state_build");
     tc_state_build_kernel<DV><<<dim3(D.S, BH), kSbThreads, kSbSmem, st>>>(mapV, kf, part, D.N, D.S, D.ld, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    tc_reduce_emit_kernel<DV><<<BH, 256, 0, st>>>(part, state, b3, D.S, D.ld);
+    tc_reduce_emit_kernel<DV><<<BH, 256, 0, st>>>(part, state, b3, bq, D.S, D.ld);
     if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
@@ -567,6 +1015,45 @@ inline hla_status core_forward(const Plan& P, const Dims& D, int BH, const float
                                const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
     if (D.d == 128) return launch_core_forward<128>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec);
     return launch_core_forward<64>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec);
+}
+
+template <int DV>
+inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, const void* dO,
+                                       float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count,
+                                       LaunchRec& rec) {
+    CUtensorMap mapV, mapdO, mapdV, mapBq, mapBd3, mapBdq;
+    __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
+    __nv_bfloat16* bd3 = reinterpret_cast<__nv_bfloat16*>(ws + P.bd3);
+    __nv_bfloat16* bdq = reinterpret_cast<__nv_bfloat16*>(ws + P.bdq);
+    if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapdO, dO, BH, D.N, DV, kTileTokens) ||
+        !make_map_bhnd(&mapdV, dV, BH, D.N, DV, kTileTokens) || !make_map_2d(&mapBq, bq, (size_t)BH * kMonoPad, DV, kMonoPad) ||
+        !make_map_2d(&mapBd3, bd3, (size_t)BH * (DV + 16), kMonoPad, DV + 16) || !make_map_2d(&mapBdq, bdq, (size_t)BH * kMonoPad, DV, kMonoPad))
+        return HLA_ERR_CUDA;
+    int* status = reinterpret_cast<int*>(ws + L.status);
+    float* part = reinterpret_cast<float*>(ws + off_part);
+    const float* state = reinterpret_cast<const float*>(ws + L.state);
+    float* dstate = reinterpret_cast<float*>(ws + L.dstate);
+    const float* eta = reinterpret_cast<const float*>(ws + L.eta);
+    if (!set_smem(tc_bwd_query_kernel<DV>, kBqSmem) || !set_smem(tc_bwd_key_kernel<DV>, BkCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    cudaStream_t st = rec.st;
+    rec.begin("tc_bwd_query");
+    tc_bwd_query_kernel<DV><<<dim3(D.S, BH), kBqThreads, kBqSmem, st>>>(mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps, status);
+    if (!rec.end()) return HLA_ERR_CUDA;
+    rec.begin("tc_reduce_emit");
+    tc_reduce_emit_kernel<DV><<<BH, 256, 0, st>>>(part, dstate, bd3, bdq, D.S, D.ld);
+    if (!rec.end()) return HLA_ERR_CUDA;
+    const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
+    const long long total = (long long)BH * tiles;
+    const int grid = (int)(total < sm_count ? total : sm_count);
+    rec.begin("tc_bwd_key");
+    tc_bwd_key_kernel<DV><<<grid, kBkThreads, BkCfg<DV>::kSmem, st>>>(mapV, mapBd3, mapBdq, mapdV, kf, dstate, dkf, D.N, BH, D.ld, status);
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+
+inline hla_status core_backward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, const void* dO,
+                                float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
+    if (D.d == 128) return launch_core_backward<128>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+    return launch_core_backward<64>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
 }
 
 }  // namespace tc

@@ -79,10 +79,11 @@ class GpuRun:
                 self.region("kf", nq * s.F, (s.B, s.H, s.F, s.N, s.d_phi)))
 
     def state(self, name="state"):
+        """(C, z) as the library keeps them: [B,H,state_rows,d] and [B,H,state_rows]."""
         s = self.shape
-        P = s.d_phi ** s.F
+        R = self.op.layout.state_rows
         ld = self.op.layout.state_ld
-        st = self.region(name, s.B * s.H * P * ld, (s.B, s.H, P, ld))
+        st = self.region(name, s.B * s.H * R * ld, (s.B, s.H, R, ld))
         return st[..., : s.d], st[..., s.d]
 
     def eta(self):
@@ -98,3 +99,19 @@ def oracle_state(kf, V):
         for h in range(H):
             C[b, h], z[b, h] = orc.context_state([kf[b, h, f] for f in range(F)], V[b, h])
     return C, z
+
+
+def fold_symmetric(T, dphi=6, F=3):
+    """Sum a tensor whose axis -2 (or last axis for a vector field) indexes the P = dphi^F outer-product
+    entries over the distinct permutations of each sorted index tuple: [.., P, d] -> [.., n_mono, d].
+    This is what the readout of the symmetric query tensor q (x) q (x) q can see of the state."""
+    import itertools
+    monos = [t for t in itertools.combinations_with_replacement(range(dphi), F)]
+    out = np.zeros(T.shape[:-2] + (len(monos), T.shape[-1]))
+    for m, t in enumerate(monos):
+        for perm in set(itertools.permutations(t)):
+            p = 0
+            for i in perm:
+                p = p * dphi + i
+            out[..., m, :] += T[..., p, :]
+    return out

@@ -6,7 +6,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import GpuRun, TOL, oracle_state, relerr, l2err
+from hla_testlib import GpuRun, TOL, fold_symmetric, oracle_state, relerr, l2err
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -26,10 +26,12 @@ def test_core_forward_bf16_features(d, N, B, H, splits):
     O = run.forward(qf, kf, V)
     f64 = lambda a: a.astype(np.float64)
     Oq, eta = orc.hla_core_forward(f64(qf), f64(kf), f64(V), EPS, "factored")
-    C, z = run.state()
+    C, z = run.state()                               # folded over the permutation symmetry: 56 rows
     Co, zo = oracle_state(f64(kf), f64(V))
+    Co, zo = fold_symmetric(Co), fold_symmetric(zo[..., None])[..., 0]
+    assert C.shape[2] == 56
     assert relerr(z, zo) < 1e-5                      # fp32 accumulation of unrounded products
-    assert relerr(C, Co) < TOL["bf16"] / 4           # T_k rounded to bf16 once
+    assert relerr(C, Co) < TOL["bf16"] / 4           # folded key features rounded to bf16 once
     assert relerr(run.eta(), eta) < TOL["bf16"] / 4
     assert relerr(O, Oq) < TOL["bf16"], (relerr(O, Oq), l2err(O, Oq))
     assert run.op.launches() == 3
@@ -67,3 +69,57 @@ def test_tc_bitwise_reproducible():
     a = run.forward(qf, kf, V)
     b = run.forward(qf, kf, V)
     assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("d,N,B,H,splits", [(128, 1000, 1, 2, 0), (64, 700, 2, 2, 3), (128, 130, 1, 1, 0), (128, 2500, 1, 3, 5)])
+def test_core_backward_bf16_features(d, N, B, H, splits):
+    """dq, dk^f (fp32 feature gradients) and dV (bf16) of the tensor-core backward against the quadratic-form oracle."""
+    s = synth.HlaShape("t", B, H, N, d, "bf16", "inv_sqrt_d")
+    _, _, V = synth.make_qkv(s)
+    V = synth.bf16_round(V * np.float32(np.sqrt(d)))
+    qf, kf = synth.make_features(s)
+    dO = synth.make_dO(s)
+    run = GpuRun(s, "none", EPS, splits)
+    O = run.forward(qf, kf, V)
+    dq, dk, dv = run.backward(dO)
+    f64 = lambda a: a.astype(np.float64)
+    form = "quadratic" if N <= 1000 else "factored"
+    rq, rk, rv = orc.hla_core_backward(f64(qf), f64(kf), f64(V), f64(dO), EPS, form)
+    assert relerr(dv, rv) < TOL["bf16"], relerr(dv, rv)
+    assert relerr(dq, rq) < TOL["bf16"], relerr(dq, rq)
+    assert relerr(dk, rk) < TOL["bf16"], relerr(dk, rk)
+    assert run.op.launches() == 3
+
+
+def test_full_backward_bf16_mlp_stagewise():
+    """Training-step shape at reduced size (d=128, ragged N) with the phi maps: every stage against the oracle
+    run on that stage's actual inputs, then end to end."""
+    s = synth.HlaShape("t", 2, 3, 1500, 128, "bf16", "rms_qk", backward=True)
+    Q, K, V = synth.make_qkv(s)
+    dO = synth.make_dO(s)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    run = GpuRun(s, "mlp", EPS)
+    run.set_weights(pq, pk)
+    O = run.forward(Q, K, V)
+    dQ, dK, dV = run.backward(dO)
+    f64 = lambda a: a.astype(np.float64)
+    gq, gk = run.features()
+    nq = s.B * s.H * s.N * s.d_phi
+    dqf = run.region("dqf", nq, (s.B, s.H, s.N, s.d_phi))
+    dkf = run.region("dkf", nq * s.F, (s.B, s.H, s.F, s.N, s.d_phi))
+    # core gradients at the features the GPU used
+    rq, rk, rv = orc.hla_core_backward(gq, gk, f64(V), f64(dO), EPS, "factored")
+    assert relerr(dV, rv) < TOL["bf16"]
+    assert relerr(dqf, rq) < TOL["bf16"]
+    assert relerr(dkf, rk) < TOL["bf16"]
+    # phi backward at the feature gradients the GPU produced
+    d = s.d
+    rQ = orc.phi_mlp_backward(f64(Q).reshape(-1, d), *pq, dqf.reshape(-1, s.d_phi)).reshape(Q.shape)
+    rK = sum(orc.phi_mlp_backward(f64(K).reshape(-1, d), *pk[f], dkf[:, :, f].reshape(-1, s.d_phi)).reshape(K.shape) for f in range(s.F))
+    assert relerr(dQ, rQ) < TOL["bf16"]
+    assert relerr(dK, rK) < TOL["bf16"]
+    # end to end
+    eQ, eK, eV, _, _ = orc.hla_backward(f64(Q), f64(K), f64(V), f64(dO), pq, pk, EPS, "factored")
+    assert relerr(dV, eV) < TOL["bf16"], relerr(dV, eV)
+    assert l2err(dQ, eQ) < TOL["bf16"], l2err(dQ, eQ)
+    assert l2err(dK, eK) < TOL["bf16"], l2err(dK, eK)
