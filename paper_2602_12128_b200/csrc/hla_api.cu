@@ -8,6 +8,7 @@
 #include "hla_common.cuh"
 #include "hla_simt.cuh"
 #include "hla_tc.cuh"
+#include "hla_tc_phi.cuh"
 
 using namespace hla;
 
@@ -309,7 +310,7 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
     if (ctx->tc) {
         const float *qf, *kf;
         if (ctx->cfg.phi == HLA_PHI_MLP) {
-            s = simt_phi_forward<__nv_bfloat16>(ctx, Q, K, ws, st);
+            s = tc::phi_forward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, ws, ctx->L, ctx->sm_count, ctx->rec);
             if (s != HLA_OK) return s;
             qf = reinterpret_cast<const float*>(ws + ctx->L.qf);
             kf = reinterpret_cast<const float*>(ws + ctx->L.kf);
