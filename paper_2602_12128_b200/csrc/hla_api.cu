@@ -341,7 +341,7 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
         float* dkf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dkf) : static_cast<float*>(dK);
         s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
         if (s != HLA_OK || !mlp) return s;
-        return simt_phi_backward<__nv_bfloat16>(ctx, Q, K, dQ, dK, ws, st);
+        return tc::phi_backward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, dQ, dK, ws, ctx->L, ctx->sm_count, ctx->rec);
     }
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
