@@ -185,11 +185,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="train_bf16", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
+    ap.add_argument("--H", type=int, default=0, help="override the workload's head count")
+    ap.add_argument("--N", type=int, default=0, help="override the workload's token count")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     shape = synth.CONFIGS[args.workload]
+    if args.B or args.H or args.N:
+        import dataclasses
+        shape = dataclasses.replace(shape, name=shape.name + "_resized", B=args.B or shape.B, H=args.H or shape.H, N=args.N or shape.N)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
