@@ -25,7 +25,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2602_12128_b200 import flops as F_, synth  # noqa: E402
+from paper_2602_12128_b200 import flops as F_, multi, synth  # noqa: E402
 
 METRIC = "hla_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
@@ -219,7 +219,7 @@ def main():
 
     # ---- synthetic inputs (seeded per rank), resident in HBM -----------------------------------------------------
     g = torch.Generator(device=dev)
-    g.manual_seed(1000 + rank)
+    g.manual_seed(multi.rank_seed(1000, rank))
     dims = (shape.B, shape.H, shape.N, shape.d)
 
     def draw():
@@ -281,12 +281,9 @@ def main():
     clocks = sampler.stop()
     kt = binding.hla_timing_collect(op.ctx)
     binding.hla_timing_enable(op.ctx, False)
-    t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = multi.max_over_ranks(ms_total, dist, dev) / args.steps
     fl_step, by_step = work_model(shape)
-    value = world * fl_step / (ms_step * 1e-3) / 1e12
+    value = multi.whole_job_rate(fl_step, world, ms_step) / 1e12
 
     # ---- end to end through the C ABI from pinned host buffers -----------------------------------------------------
     e2e = None
@@ -311,11 +308,8 @@ def main():
             e2e_step()
         e1.record()
         barrier()
-        t2 = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
-        if dist is not None:
-            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t2.item()) / nsteps
-        e2e = {"value": world * fl_step / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e, "steps": nsteps,
+        ms_e2e = multi.max_over_ranks(e0.elapsed_time(e1), dist, dev) / nsteps
+        e2e = {"value": multi.whole_job_rate(fl_step, world, ms_e2e) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e, "steps": nsteps,
                "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in ins)),
                "d2h_bytes_per_step": int(sum(x.numel() * x.element_size() for x in outs))}
 
@@ -362,7 +356,7 @@ def main():
             "config": {"workload": shape.name, "B": shape.B, "H": shape.H, "N": shape.N, "d": shape.d, "F": shape.F, "d_phi": shape.d_phi,
                        "phi": "mlp", "pass": "fwd+bwd" if shape.backward else "fwd", "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (each tensor %.0f MB)" % (Q.numel() * Q.element_size() / 1e6)},
-            "tokens_per_s": world * shape.B * shape.N / (ms_step * 1e-3),
+            "tokens_per_s": multi.whole_job_rate(shape.B * shape.N, world, ms_step),
             "step_roofline": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_step, "flops": fl_step, "bytes": by_step,
                               "peaks": peaks},
             "roofline": roof, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
