@@ -62,10 +62,12 @@ def kernel_models(shape):
     m = {
         "tc_state_build": (contr, d * e + Fn * dp * 4, "tensor"),
         "tc_readout": (contr, d * e + dp * 4 + 4, "tensor"),
-        "tc_phi_forward": ((1 + Fn) * phi1, 2 * d * e + (1 + Fn) * dp * 4, "tensor"),
+        "tc_phi_forward_q": (phi1, d * e + dp * 4, "tensor"),
+        "tc_phi_forward_k": (Fn * phi1, d * e + Fn * dp * 4, "tensor"),
         "tc_bwd_query": (2 * contr, 2 * d * e + 3 * dp * 4, "tensor"),
         "tc_bwd_key": (2 * contr, 2 * d * e + 2 * Fn * dp * 4, "tensor"),
-        "tc_phi_backward": ((1 + Fn) * (4 * d * d + 2 * d * dp), 4 * d * e + (1 + Fn) * dp * 4, "tensor"),
+        "tc_phi_backward_q": (4 * d * d + 2 * d * dp, 2 * d * e + 2 * dp * 4, "tensor"),
+        "tc_phi_backward_k": (Fn * (4 * d * d + 2 * d * dp), 2 * d * e + 2 * Fn * dp * 4, "tensor"),
         "simt_phi_forward": ((1 + Fn) * phi1 / 2, d * e + (1 + Fn) * dp * 2, "alu"),          # two launches: Q side, K side
         "simt_state_build": (contr, 2 * d * e + Fn * dp * 4, "alu"),
         "simt_readout": (contr, d * e + Fn * dp * 4, "alu"),

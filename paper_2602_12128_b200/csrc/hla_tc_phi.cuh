@@ -3,32 +3,49 @@
 //
 // Per 128-token tile of X (Q or K, TMA-loaded once) and per map m:
 //   D1 = X * W1[m]            tcgen05, fp32 in TMEM        [128 tok x d hidden]
-//   G  = bf16(GELU(D1 + b1))  8 warps, thread = (token, half of the hidden units); written as the next MMA's A operand
+//   G  = bf16(GELU(D1 + b1))  16 warps, thread = (token, quarter of the hidden units); written as the next MMA's A operand
 //   D2 = G * W2[m]            tcgen05, N padded to 16
 //   feat = ReLU(D2 + b2)      fp32 features to global memory
 // The key side runs its F maps on the same X tile, so K is read once.
 // GELU is the exact erf form evaluated with an odd polynomial for erf (fit_gelu_poly.py: |error| < 7e-5,
-// far below the bf16 rounding of G) - no special-function unit on the hot loop.
+// far below the bf16 rounding of G) on packed fp32 pairs - no special-function unit on the forward's hot loop.
 #pragma once
 #include "hla_tc.cuh"
 
 namespace hla {
 namespace tc {
 
-__device__ __forceinline__ float gelu_poly(float x) {
-    const float u = fminf(fmaxf(x * 0.70710678f, -3.0f), 3.0f);
-    const float t = u * u;
-    float p = 4.074210630e-08f;
-    p = fmaf(p, t, -1.944822741e-06f);
-    p = fmaf(p, t, 4.106052437e-05f);
-    p = fmaf(p, t, -5.110368664e-04f);
-    p = fmaf(p, t, 4.235427410e-03f);
-    p = fmaf(p, t, -2.510286119e-02f);
-    p = fmaf(p, t, 1.110793351e-01f);
-    p = fmaf(p, t, -3.753148748e-01f);
-    p = fmaf(p, t, 1.128268423e+00f);
-    const float hx = 0.5f * x;
-    return fmaf(hx, u * p, hx);
+// Phi(x) = 1/2 + erf(x / sqrt 2) / 2 as 1/2 + xc * P(xc^2) with xc = x clamped to +-3 sqrt 2 (fit_gelu_poly.py; the
+// coefficients are those of erf(u) ~ u P(u^2) rescaled to the variable x).  Evaluated on pairs with the packed
+// fp32 instructions (fma.rn.f32x2), which halve the number of issue slots.
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float2 normal_cdf2(float2 x) {
+    constexpr float kClamp = 4.2426405f;
+    const float2 xc = make_float2(fminf(fmaxf(x.x, -kClamp), kClamp), fminf(fmaxf(x.y, -kClamp), kClamp));
+    const float2 t = __fmul2_rn(xc, xc);
+    float2 p = splat2(5.626761649e-11f);
+    p = __ffma2_rn(p, t, splat2(-5.371864642e-09f));
+    p = __ffma2_rn(p, t, splat2(2.268294939e-07f));
+    p = __ffma2_rn(p, t, splat2(-5.646213026e-06f));
+    p = __ffma2_rn(p, t, splat2(9.359060759e-05f));
+    p = __ffma2_rn(p, t, splat2(-1.109400211e-03f));
+    p = __ffma2_rn(p, t, splat2(9.818118887e-03f));
+    p = __ffma2_rn(p, t, splat2(-6.634692326e-02f));
+    p = __ffma2_rn(p, t, splat2(3.989031265e-01f));
+    return __ffma2_rn(xc, p, splat2(0.5f));
+}
+// GELU(x) = x Phi(x)
+__device__ __forceinline__ float2 gelu2(float2 x) { return __fmul2_rn(x, normal_cdf2(x)); }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// GELU'(x) = Phi(x) + x pdf(x),  pdf(x) = exp(-x^2 / 2) / sqrt(2 pi)
+__device__ __forceinline__ float2 gelu_grad2(float2 x) {
+    const float2 a = __fmul2_rn(__fmul2_rn(x, x), splat2(-0.72134752f));     // -x^2 / 2 * log2(e)
+    const float2 e = make_float2(ex2_approx(a.x), ex2_approx(a.y));
+    return __ffma2_rn(__fmul2_rn(x, e), splat2(0.39894228f), normal_cdf2(x));
 }
 
 struct PhiPtrs {
@@ -40,15 +57,16 @@ struct PhiMaps {
     CUtensorMap w1[3];
 };
 
-constexpr int kPfThreads = 320;   // warp 0: TMA, warp 1: MMA, warps 2..9: epilogue (thread = token row x half of the hidden units)
+constexpr int kPfThreads = 576;   // warp 0: TMA, warp 1: MMA, warps 2..17: epilogue (thread = token row x quarter of the hidden units)
 
 template <int DV, int NMAPS> struct PfCfg {
+    static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;   // one stage is enough when a tile has three units
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
     static constexpr int kW2Bytes = (DV / 64) * 2048;            // [16 rows][DV] bf16, K-major, per map
-    static constexpr int kOffX = 0;                              // 2 stages
-    static constexpr int kOffG = 2 * kXBytes;                    // GELU output tile
-    static constexpr int kOffW1 = kOffG + kXBytes;
+    static constexpr int kOffX = 0;
+    static constexpr int kOffG = kXStages * kXBytes;             // 2 GELU output tiles
+    static constexpr int kOffW1 = kOffG + 2 * kXBytes;
     static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;
     static constexpr int kOffBias = kOffW2 + NMAPS * kW2Bytes;   // per map: b1[DV], b2[8] floats
     static constexpr int kOffBars = kOffBias + NMAPS * (DV + 8) * 4;
@@ -57,11 +75,14 @@ template <int DV, int NMAPS> struct PfCfg {
 };
 
 // X [rows][DV] bf16 (rows = B*H*N tokens).  KSIDE: features to kf[bh][f][n][6], else qf[row][6].
+// A "unit" is one map of one tile.  h and the GELU tile are double-buffered, and the feature epilogue of a unit
+// runs one unit late, so the GELU warps never wait for a tensor-core round trip.
 template <int DV, int NMAPS, bool KSIDE>
 __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
                                                                        PhiPtrs P, float* __restrict__ feat, long long rows, int N, int* status) {
     using Cfg = PfCfg<DV, NMAPS>;
-    constexpr int HC = DV / 2;          // hidden units per epilogue thread
+    constexpr int HC = DV / 4;          // hidden units per epilogue thread
+    constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     float* bias = reinterpret_cast<float*>(smem + Cfg::kOffBias);
@@ -69,13 +90,13 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     uint64_t* x_full = bars;           // [2]
     uint64_t* x_empty = bars + 2;      // [2] MMA commit
     uint64_t* d1_full = bars + 4;      // [2] MMA commit
-    uint64_t* d1_empty = bars + 6;     // [2] 256 arrivals
-    uint64_t* g_full = bars + 8;       // 256 arrivals
-    uint64_t* g_free = bars + 9;       // MMA commit
-    uint64_t* d2_full = bars + 10;     // [2] MMA commit
-    uint64_t* d2_empty = bars + 12;    // [2] 128 arrivals
-    uint64_t* w_full = bars + 14;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+    uint64_t* d1_empty = bars + 6;     // [2] 512 arrivals
+    uint64_t* g_full = bars + 8;       // [2] 512 arrivals
+    uint64_t* g_free = bars + 10;      // [2] MMA commit
+    uint64_t* d2_full = bars + 12;     // [2] MMA commit
+    uint64_t* d2_empty = bars + 14;    // [2] 128 arrivals
+    uint64_t* w_full = bars + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -101,12 +122,12 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             mbar_init(&x_full[i], 1);
             mbar_init(&x_empty[i], 1);
             mbar_init(&d1_full[i], 1);
-            mbar_init(&d1_empty[i], 256);
+            mbar_init(&d1_empty[i], 512);
+            mbar_init(&g_full[i], 512);
+            mbar_init(&g_free[i], 1);
             mbar_init(&d2_full[i], 1);
             mbar_init(&d2_empty[i], 128);
         }
-        mbar_init(g_full, 256);
-        mbar_init(g_free, 1);
         mbar_init(w_full, 1);
         fence_mbar_init();
         prefetch_tmap(&mapX);
@@ -128,7 +149,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
                 for (int b = 0; b < DV / 64; ++b)
                     tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
             for (int it = 0; it < ntiles; ++it) {
-                const int st = it & 1, u = it >> 1;
+                const int st = it % XST, u = it / XST;
                 if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 501); break; }
                 mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
                 for (int b = 0; b < DV / 64; ++b)
@@ -139,12 +160,11 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
         if (lane == 0 && ntiles > 0) {
             const uint32_t idesc1 = idesc_bf16(128, DV, false, true);   // X K-major, W1 [in][hidden] MN-major
             const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G K-major, W2 operand K-major
-            const uint32_t ga = smem_u32(smem + Cfg::kOffG);
             bool good = mbar_wait(w_full, 0);
             if (!good) report_timeout(status, 502);
             auto issue_mma1 = [&](int unit) -> bool {
-                const int it = unit / NMAPS, m = unit % NMAPS, st = it & 1, b = unit & 1;
-                if (m == 0 && !mbar_wait(&x_full[st], (it >> 1) & 1)) return false;
+                const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
+                if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) return false;
                 if (!mbar_wait(&d1_empty[b], ((unit >> 1) & 1) ^ 1)) return false;
                 tc_fence_after();
                 const uint32_t xa = smem_u32(smem + Cfg::kOffX + st * Cfg::kXBytes);
@@ -160,43 +180,73 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             if (good && nunits > 0) good = issue_mma1(0);
             if (good && nunits > 1) good = issue_mma1(1);
             for (int unit = 0; unit < nunits && good; ++unit) {
-                const int m = unit % NMAPS, b = unit & 1;
-                if (!(mbar_wait(g_full, unit & 1) && mbar_wait(&d2_empty[b], ((unit >> 1) & 1) ^ 1))) { good = false; break; }
+                const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
+                if (!(mbar_wait(&g_full[b], par) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
                 tc_fence_after();
+                const uint32_t ga = smem_u32(smem + Cfg::kOffG + b * Cfg::kXBytes);
                 const uint32_t w2a = smem_u32(smem + Cfg::kOffW2 + m * Cfg::kW2Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 256 + 32 * b, smem_desc_sw128(ga + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
                               smem_desc_sw128(w2a + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
-                umma_commit(g_free);
+                umma_commit(&g_free[b]);
                 umma_commit(&d2_full[b]);
                 if (unit + 2 < nunits) good = issue_mma1(unit + 2);
             }
             if (!good) report_timeout(status, 503);
         }
     } else {
-        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int quarter = warp & 3, part = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
-        for (int unit = 0; unit < nunits; ++unit) {
+        // feature epilogue of one unit (the part-0 warps only): ReLU(D2 + b2) -> global memory
+        auto emit_features = [&](int unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1;
+            if (ok && !mbar_wait(&d2_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 506); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            tc_fence_after();
+            uint32_t r[8];
+            tmem_ld8(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), r);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(&d2_empty[b]);
+            const long long grow = (t0 + it) * kTileTokens + row;
+            if (grow < rows) {
+                const float* b2s = bias + m * (DV + 8) + DV;
+                float f[6];
+#pragma unroll
+                for (int o = 0; o < 6; ++o) f[o] = fmaxf(__uint_as_float(r[o]) + b2s[o], 0.f);
+                if (KSIDE) {
+                    const long long bh = grow / N, n = grow - bh * N;
+                    store6(feat + ((bh * NMAPS + m) * N + n) * 6, f);
+                } else {
+                    store6(feat + grow * 6, f);
+                }
+            }
+        };
+        for (int unit = 0; unit < nunits && ok; ++unit) {
+            const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
             const float* b1s = bias + m * (DV + 8);
-            if (ok && !mbar_wait(&d1_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 504); }
-            if (ok && unit > 0 && !mbar_wait(g_free, (unit - 1) & 1)) { ok = false; report_timeout(status, 505); }
+            if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 504); }
+            if (ok && !mbar_wait(&g_free[b], par ^ 1)) { ok = false; report_timeout(status, 505); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + half * HC;
-            const uint32_t gblk = smem_u32(smem + Cfg::kOffG);
+            const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
+            const uint32_t gblk = smem_u32(smem + Cfg::kOffG + b * Cfg::kXBytes);
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
                 uint32_t r[16];
                 tmem_ld16(ta + 16 * c, r);
                 tmem_ld_wait();
-                const int col = half * HC + 16 * c;
+                const int col = part * HC + 16 * c;
+                const float2* bb = reinterpret_cast<const float2*>(b1s + col);
                 uint32_t w[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    w[e] = pack_bf16(gelu_poly(__uint_as_float(r[2 * e]) + b1s[col + 2 * e]), gelu_poly(__uint_as_float(r[2 * e + 1]) + b1s[col + 2 * e + 1]));
+                for (int e = 0; e < 8; ++e) {
+                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), bb[e]));
+                    w[e] = pack_bf16(g.x, g.y);
+                }
                 const uint32_t blk = gblk + (col >> 6) * kBlk;
                 st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
                 st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
@@ -204,31 +254,10 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             tc_fence_before();
             mbar_arrive(&d1_empty[b]);
             fence_proxy_async();
-            mbar_arrive(g_full);
-            if (half == 0) {
-                if (!mbar_wait(&d2_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 506); }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t r[8];
-                tmem_ld8(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), r);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(&d2_empty[b]);
-                const long long grow = (t0 + it) * kTileTokens + row;
-                if (grow < rows) {
-                    float f[6];
-#pragma unroll
-                    for (int o = 0; o < 6; ++o) f[o] = fmaxf(__uint_as_float(r[o]) + b1s[DV + o], 0.f);
-                    if (KSIDE) {
-                        const long long bh = grow / N, n = grow - bh * N;
-                        store6(feat + ((bh * NMAPS + m) * N + n) * 6, f);
-                    } else {
-                        store6(feat + grow * 6, f);
-                    }
-                }
-            }
+            mbar_arrive(&g_full[b]);
+            if (part == 0 && unit > 0) emit_features(unit - 1);
         }
+        if (part == 0 && ok && nunits > 0) emit_features(nunits - 1);
     }
     tc_fence_before();
     __syncthreads();
@@ -261,10 +290,10 @@ inline hla_status launch_phi_forward(const Dims& D, int BH, const hla_mlp* phi_q
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     cudaStream_t st = rec.st;
-    rec.begin("tc_phi_forward");
+    rec.begin("tc_phi_forward_q");
     tc_phi_forward_kernel<DV, 1, false><<<grid, kPfThreads, PfCfg<DV, 1>::kSmem, st>>>(mapQ, mq, pq, reinterpret_cast<float*>(ws + L.qf), rows, D.N, status);
     if (!rec.end()) return HLA_ERR_CUDA;
-    rec.begin("tc_phi_forward");
+    rec.begin("tc_phi_forward_k");
     tc_phi_forward_kernel<DV, 3, true><<<grid, kPfThreads, PfCfg<DV, 3>::kSmem, st>>>(mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
@@ -285,54 +314,36 @@ inline hla_status phi_forward(const Dims& D, int BH, const hla_mlp* phi_q, const
 // written as the second MMA's A operand, and the W1 image in shared memory serves both MMAs
 // (MN-major B for X W1, K-major B for dh W1^T).
 // =======================================================================================
-// GELU'(x) = Phi(x) + x pdf(x) = 1/2 + u (P(u^2)/2 + exp(-u^2)/sqrt(pi)),  u = x / sqrt 2, erf(u) = u P(u^2).
-__device__ __forceinline__ float gelu_grad_poly(float x) {
-    const float uu = x * 0.70710678f;
-    const float u = fminf(fmaxf(uu, -3.0f), 3.0f);
-    const float t = u * u;
-    float p = 4.074210630e-08f;
-    p = fmaf(p, t, -1.944822741e-06f);
-    p = fmaf(p, t, 4.106052437e-05f);
-    p = fmaf(p, t, -5.110368664e-04f);
-    p = fmaf(p, t, 4.235427410e-03f);
-    p = fmaf(p, t, -2.510286119e-02f);
-    p = fmaf(p, t, 1.110793351e-01f);
-    p = fmaf(p, t, -3.753148748e-01f);
-    p = fmaf(p, t, 1.128268423e+00f);
-    const float e = exp2f(uu * uu * -1.44269504f);
-    return fmaf(uu, 0.564189584f * e, fmaf(0.5f * u, p, 0.5f));
-}
-
 struct PhiBwdPtrs {
     const __nv_bfloat16* b1[3];
     const __nv_bfloat16* W2[3];
 };
 
-constexpr int kPbThreads = 320;   // warp 0: TMA loads, warp 1: MMA, warps 2..9: epilogue (thread = token row x half of the columns)
+constexpr int kPbThreads = 576;   // warp 0: TMA loads, warp 1: MMA, warps 2..17: epilogue (thread = token row x quarter of the columns)
 
 template <int DV, int NMAPS> struct PbCfg {
     static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
     static constexpr int kOffX = 0;
-    static constexpr int kOffDh = kXStages * kXBytes;            // dh tile (A operand of the second MMA)
-    static constexpr int kOffOut = kOffDh + kXBytes;             // dX staging tile for the TMA store
-    static constexpr int kOffW1 = kOffOut + kXBytes;
-    static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;     // fp32 [NMAPS][DV][8]  (6 used)
-    static constexpr int kOffB1 = kOffW2 + NMAPS * DV * 8 * 4;   // fp32 [NMAPS][DV]
+    static constexpr int kOffDh = kXStages * kXBytes;            // 2 dh tiles (A operand of the second MMA)
+    static constexpr int kOffW1 = kOffDh + 2 * kXBytes;
+    static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;     // fp32 [NMAPS][6][DV]: W2 transposed, hidden index innermost
+    static constexpr int kOffB1 = kOffW2 + NMAPS * 6 * DV * 4;   // fp32 [NMAPS][DV]
     static constexpr int kOffBars = kOffB1 + NMAPS * DV * 4;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
 
 // X, dX [rows][DV] bf16.  KSIDE: feat / dfeat are [bh][NMAPS][N][6], else [rows][6].
+// h and the dh tile are double-buffered; the dX accumulator (double-buffered in TMEM) of a tile is drained
+// one unit late, straight from registers to global memory.
 template <int DV, int NMAPS, bool KSIDE>
-__global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapdX,
-                                                                        const __grid_constant__ PhiMaps maps, PhiBwdPtrs P,
-                                                                        const float* __restrict__ feat, const float* __restrict__ dfeat,
-                                                                        long long rows, int N, int* status) {
+__global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
+                                                                        PhiBwdPtrs P, const float* __restrict__ feat, const float* __restrict__ dfeat,
+                                                                        __nv_bfloat16* __restrict__ dX, long long rows, int N, int* status) {
     using Cfg = PbCfg<DV, NMAPS>;
-    constexpr int HC = DV / 2;
+    constexpr int HC = DV / 4;
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -342,13 +353,13 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* x_full = bars;           // [2]
     uint64_t* x_empty = bars + 2;      // [2] MMA commit
     uint64_t* h_full = bars + 4;       // [2] MMA commit
-    uint64_t* h_empty = bars + 6;      // [2] 256 arrivals
-    uint64_t* dh_full = bars + 8;      // 256 arrivals
-    uint64_t* dh_free = bars + 9;      // MMA commit
-    uint64_t* dx_full = bars + 10;     // [2] MMA commit
-    uint64_t* dx_empty = bars + 12;    // [2] 256 arrivals
-    uint64_t* w_full = bars + 14;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+    uint64_t* h_empty = bars + 6;      // [2] 512 arrivals
+    uint64_t* dh_full = bars + 8;      // [2] 512 arrivals
+    uint64_t* dh_free = bars + 10;     // [2] MMA commit
+    uint64_t* dx_full = bars + 12;     // [2] MMA commit
+    uint64_t* dx_empty = bars + 14;    // [2] 512 arrivals
+    uint64_t* w_full = bars + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -356,9 +367,9 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     const int ntiles = (int)(t1 - t0);
     const int nunits = ntiles * NMAPS;
 
-    for (int i = tid; i < NMAPS * DV * 8; i += kPbThreads) {
-        const int m = i / (DV * 8), j = (i >> 3) % DV, o = i & 7;
-        w2s[i] = o < 6 ? __bfloat162float(P.W2[m][j * 6 + o]) : 0.f;
+    for (int i = tid; i < NMAPS * 6 * DV; i += kPbThreads) {
+        const int m = i / (6 * DV), o = (i / DV) % 6, j = i % DV;
+        w2s[i] = __bfloat162float(P.W2[m][j * 6 + o]);
     }
     for (int i = tid; i < NMAPS * DV; i += kPbThreads) b1s[i] = __bfloat162float(P.b1[i / DV][i % DV]);
     if (tid == 0) {
@@ -366,16 +377,15 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             mbar_init(&x_full[i], 1);
             mbar_init(&x_empty[i], 1);
             mbar_init(&h_full[i], 1);
-            mbar_init(&h_empty[i], 256);
+            mbar_init(&h_empty[i], 512);
+            mbar_init(&dh_full[i], 512);
+            mbar_init(&dh_free[i], 1);
             mbar_init(&dx_full[i], 1);
-            mbar_init(&dx_empty[i], 256);
+            mbar_init(&dx_empty[i], 512);
         }
-        mbar_init(dh_full, 256);
-        mbar_init(dh_free, 1);
         mbar_init(w_full, 1);
         fence_mbar_init();
         prefetch_tmap(&mapX);
-        prefetch_tmap(&mapdX);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, 512);
@@ -405,7 +415,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         if (lane == 0 && ntiles > 0) {
             const uint32_t idesc1 = idesc_bf16(128, DV, false, true);    // h  = X (K-major) * W1 [in][hidden] (MN-major)
             const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (K-major over hidden) * W1 as [in][hidden] (K-major)
-            const uint32_t dha = smem_u32(smem + Cfg::kOffDh);
             bool good = mbar_wait(w_full, 0);
             if (!good) report_timeout(status, 602);
             auto issue_mma1 = [&](int unit) -> bool {
@@ -426,32 +435,56 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             if (good && nunits > 0) good = issue_mma1(0);
             if (good && nunits > 1) good = issue_mma1(1);
             for (int unit = 0; unit < nunits && good; ++unit) {
-                const int it = unit / NMAPS, m = unit % NMAPS, tb = it & 1;
-                if (!mbar_wait(dh_full, unit & 1)) { good = false; break; }
+                const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, tb = it & 1;
+                if (!mbar_wait(&dh_full[b], (unit >> 1) & 1)) { good = false; break; }
                 if (m == 0 && !mbar_wait(&dx_empty[tb], ((it >> 1) & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
+                const uint32_t dha = smem_u32(smem + Cfg::kOffDh + b * Cfg::kXBytes);
                 const uint32_t wa = smem_u32(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 256 + 128 * tb, smem_desc_sw128(dha + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
                               smem_desc_sw128(wa + (ks >> 2) * (DV * 128) + (ks & 3) * 32, 16, 1024), idesc2, (m > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(dh_free);
+                umma_commit(&dh_free[b]);
                 if (m == NMAPS - 1) umma_commit(&dx_full[tb]);
                 if (unit + 2 < nunits) good = issue_mma1(unit + 2);
             }
             if (!good) report_timeout(status, 603);
         }
     } else {
-        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int quarter = warp & 3, part = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
-        const bool leader = tid == 64;
-        // After a wait has run out (ok == false) the loop keeps going without waiting or touching TMEM / shared
-        // memory, so that every thread still reaches the named barriers.
-        for (int unit = 0; unit < nunits; ++unit) {
-            const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, tb = it & 1;
+        // dX of tile `it`: TMEM -> bf16 -> global memory (each thread: HC contiguous columns of its row)
+        auto drain_dx = [&](int it) {
+            const int tb = it & 1;
+            if (ok && !mbar_wait(&dx_full[tb], (it >> 1) & 1)) { ok = false; report_timeout(status, 606); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) return;
+            tc_fence_after();
+            const uint32_t tx = tmem + 256 + 128 * tb + ((uint32_t)(quarter * 32) << 16) + part * HC;
             const long long grow = (t0 + it) * kTileTokens + row;
-            float dp[6];
-            if (ok && grow < rows) {
+            uint4* dst = reinterpret_cast<uint4*>(dX + (size_t)grow * DV + part * HC);
+#pragma unroll
+            for (int c = 0; c < HC / 16; ++c) {
+                uint32_t r[16];
+                tmem_ld16(tx + 16 * c, r);
+                tmem_ld_wait();
+                uint32_t w[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                if (grow < rows) {
+                    dst[2 * c] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[2 * c + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&dx_empty[tb]);
+        };
+        for (int unit = 0; unit < nunits && ok; ++unit) {
+            const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
+            const long long grow = (t0 + it) * kTileTokens + row;
+            float2 dp[6];
+            if (grow < rows) {
                 size_t off;
                 if (KSIDE) {
                     const long long bh = grow / N, n = grow - bh * N;
@@ -459,96 +492,63 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 } else {
                     off = (size_t)grow * 6;
                 }
-                float f[6];
+                float f[6], g[6];
                 load6(f, feat + off);
-                load6(dp, dfeat + off);
+                load6(g, dfeat + off);
 #pragma unroll
-                for (int o = 0; o < 6; ++o) dp[o] = f[o] > 0.f ? dp[o] : 0.f;
+                for (int o = 0; o < 6; ++o) dp[o] = splat2(f[o] > 0.f ? g[o] : 0.f);
             } else {
 #pragma unroll
-                for (int o = 0; o < 6; ++o) dp[o] = 0.f;
+                for (int o = 0; o < 6; ++o) dp[o] = splat2(0.f);
             }
-            if (ok && !mbar_wait(&h_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 604); }
+            if (!mbar_wait(&h_full[b], par)) { ok = false; report_timeout(status, 604); }
+            if (ok && !mbar_wait(&dh_free[b], par ^ 1)) { ok = false; report_timeout(status, 605); }
             ok = __all_sync(0xffffffffu, ok);
-            if (ok) {
-                tc_fence_after();
-                const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + half * HC;
-                const uint32_t dblk = smem_u32(smem + Cfg::kOffDh);
-                const float* bm = b1s + m * DV;
-                const float4* wm = reinterpret_cast<const float4*>(w2s + m * DV * 8);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
+            const uint32_t dblk = smem_u32(smem + Cfg::kOffDh + b * Cfg::kXBytes);
+            const float* bm = b1s + m * DV;
+            const float* wm = w2s + m * 6 * DV;
 #pragma unroll
-                for (int c = 0; c < HC / 16; ++c) {
-                    uint32_t r[16];
-                    tmem_ld16(ta + 16 * c, r);
-                    tmem_ld_wait();
-                    const int col = half * HC + 16 * c;
-                    float dh[16];
+            for (int c = 0; c < HC / 16; ++c) {
+                uint32_t r[16];
+                tmem_ld16(ta + 16 * c, r);
+                tmem_ld_wait();
+                const int col = part * HC + 16 * c;
+                uint32_t w[8];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float4 wa = wm[2 * (col + e)], wb = wm[2 * (col + e) + 1];
-                        float dg = dp[0] * wa.x;
-                        dg = fmaf(dp[1], wa.y, dg);
-                        dg = fmaf(dp[2], wa.z, dg);
-                        dg = fmaf(dp[3], wa.w, dg);
-                        dg = fmaf(dp[4], wb.x, dg);
-                        dg = fmaf(dp[5], wb.y, dg);
-                        dh[e] = dg * gelu_grad_poly(__uint_as_float(r[e]) + bm[col + e]);
-                    }
-                    if (c == 0 && unit > 0) {   // the dh tile is free once the previous unit's second MMA has read it
-                        if (!mbar_wait(dh_free, (unit - 1) & 1)) { ok = false; report_timeout(status, 605); }
-                        ok = __all_sync(0xffffffffu, ok);
-                    }
-                    if (ok) {
-                        uint32_t w[8];
+                for (int q4 = 0; q4 < 4; ++q4) {      // four hidden units at a time: dg = dp . W2[j][:], dh = dg GELU'(h + b1)
+                    float2 dga, dgb;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(dh[2 * e], dh[2 * e + 1]);
-                        const uint32_t blk = dblk + (col >> 6) * kBlk;
-                        st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
-                        st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
+                    for (int o = 0; o < 6; ++o) {
+                        const float4 wv = *reinterpret_cast<const float4*>(wm + o * DV + col + 4 * q4);
+                        if (o == 0) {
+                            dga = __fmul2_rn(dp[0], make_float2(wv.x, wv.y));
+                            dgb = __fmul2_rn(dp[0], make_float2(wv.z, wv.w));
+                        } else {
+                            dga = __ffma2_rn(dp[o], make_float2(wv.x, wv.y), dga);
+                            dgb = __ffma2_rn(dp[o], make_float2(wv.z, wv.w), dgb);
+                        }
                     }
+                    const float4 bv = *reinterpret_cast<const float4*>(bm + col + 4 * q4);
+                    const float2 ha = __fadd2_rn(make_float2(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1])), make_float2(bv.x, bv.y));
+                    const float2 hb = __fadd2_rn(make_float2(__uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3])), make_float2(bv.z, bv.w));
+                    const float2 da = __fmul2_rn(dga, gelu_grad2(ha)), db = __fmul2_rn(dgb, gelu_grad2(hb));
+                    w[2 * q4] = pack_bf16(da.x, da.y);
+                    w[2 * q4 + 1] = pack_bf16(db.x, db.y);
                 }
+                const uint32_t blk = dblk + (col >> 6) * kBlk;
+                st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
+                st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
             }
-            if (ok) {
-                tc_fence_before();
-                mbar_arrive(&h_empty[b]);
-                fence_proxy_async();
-                mbar_arrive(dh_full);
-            }
-            if (m == NMAPS - 1) {   // the tile's dX is complete after this unit's second MMA
-                if (ok && !mbar_wait(&dx_full[tb], (it >> 1) & 1)) { ok = false; report_timeout(status, 606); }
-                ok = __all_sync(0xffffffffu, ok);
-                if (leader) tma_store_wait_read0();     // the staging tile has been read by the previous store
-                named_barrier(1, 256);
-                if (ok) {
-                    tc_fence_after();
-                    const uint32_t tx = tmem + 256 + 128 * tb + ((uint32_t)(quarter * 32) << 16) + half * HC;
-                    const uint32_t os = smem_u32(smem + Cfg::kOffOut);
-#pragma unroll
-                    for (int c = 0; c < HC / 16; ++c) {
-                        uint32_t r[16];
-                        tmem_ld16(tx + 16 * c, r);
-                        tmem_ld_wait();
-                        const int col = half * HC + 16 * c;
-                        uint32_t w[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                        const uint32_t blk = os + (col >> 6) * kBlk;
-                        st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
-                        st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
-                    }
-                    tc_fence_before();
-                    mbar_arrive(&dx_empty[tb]);
-                    fence_proxy_async();
-                }
-                named_barrier(1, 256);
-                if (ok && leader) {
-                    for (int bb = 0; bb < DV / 64; ++bb)
-                        tma_store_2d(&mapdX, smem + Cfg::kOffOut + bb * kBlk, bb * 64, (int)((t0 + it) * kTileTokens));
-                    tma_store_commit();
-                }
-            }
+            tc_fence_before();
+            mbar_arrive(&h_empty[b]);
+            fence_proxy_async();
+            mbar_arrive(&dh_full[b]);
+            if (m == 0 && it > 0) drain_dx(it - 1);
         }
-        if (leader) tma_store_wait_all0();
+        if (ok && ntiles > 0) drain_dx(ntiles - 1);
     }
     tc_fence_before();
     __syncthreads();
@@ -559,12 +559,10 @@ template <int DV>
 inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, void* dQ,
                                       void* dK, char* ws, const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
     const long long rows = (long long)BH * D.N;
-    CUtensorMap mapQ, mapK, mapdQ, mapdK;
+    CUtensorMap mapQ, mapK;
     PhiMaps mq, mk;
     PhiBwdPtrs pq{}, pk{};
-    if (!make_map_2d(&mapQ, Q, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens) ||
-        !make_map_2d(&mapdQ, dQ, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapdK, dK, (size_t)rows, DV, kTileTokens))
-        return HLA_ERR_CUDA;
+    if (!make_map_2d(&mapQ, Q, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
     if (!make_map_2d(&mq.w1[0], phi_q->W1, DV, DV, DV)) return HLA_ERR_CUDA;
     mq.w1[1] = mq.w1[0];
     mq.w1[2] = mq.w1[0];
@@ -581,13 +579,13 @@ inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     cudaStream_t st = rec.st;
-    rec.begin("tc_phi_backward");
+    rec.begin("tc_phi_backward_q");
     tc_phi_backward_kernel<DV, 1, false><<<grid, kPbThreads, PbCfg<DV, 1>::kSmem, st>>>(
-        mapQ, mapdQ, mq, pq, reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), rows, D.N, status);
+        mapQ, mq, pq, reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), static_cast<__nv_bfloat16*>(dQ), rows, D.N, status);
     if (!rec.end()) return HLA_ERR_CUDA;
-    rec.begin("tc_phi_backward");
+    rec.begin("tc_phi_backward_k");
     tc_phi_backward_kernel<DV, 3, true><<<grid, kPbThreads, PbCfg<DV, 3>::kSmem, st>>>(
-        mapK, mapdK, mk, pk, reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), rows, D.N, status);
+        mapK, mk, pk, reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), static_cast<__nv_bfloat16*>(dK), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
