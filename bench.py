@@ -88,7 +88,7 @@ class ClockSampler:
         q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
-            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100"],
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -280,9 +280,16 @@ def main():
     e1.record()
     barrier()
     ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop()
     kt = binding.hla_timing_collect(op.ctx)
     binding.hla_timing_enable(op.ctx, False)
+    # The timed region can be shorter than one nvidia-smi sample: keep the same steps running (untimed) until the
+    # sampler has had about a second under the same load, then stop it.
+    t_tail = time.perf_counter()
+    while time.perf_counter() - t_tail < 1.0:
+        step()
+        torch.cuda.synchronize()
+    clocks = sampler.stop()
+    clocks["note"] = "sampled over the timed steps and an untimed 1 s tail of the same steps"
     ms_step = multi.max_over_ranks(ms_total, dist, dev) / args.steps
     fl_step, by_step = work_model(shape)
     value = multi.whole_job_rate(fl_step, world, ms_step) / 1e12

@@ -374,27 +374,35 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
 // Reduce the split partials [BH][S][56][ld] in a fixed order -> fp32 folded state [BH][56][ld]
 // (column d = folded z) and the two bf16 MMA operands of that state.
 // =======================================================================================
+// grid = (8, heads): block c of a head owns the monomials 8c .. 8c+7 (block 7 owns only the zero padding 56..63).
 template <int DV>
 __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __restrict__ part, float* __restrict__ state,
                                                              __nv_bfloat16* __restrict__ b3, __nv_bfloat16* __restrict__ bq, int S, int ld) {
-    const int bh = blockIdx.x, tid = threadIdx.x;
+    __shared__ float sm[8][kMaxD + 8];
+    const int m0 = 8 * blockIdx.x, bh = blockIdx.y, tid = threadIdx.x;
     const size_t n_per = (size_t)kMono * ld;
-    float* st = state + (size_t)bh * n_per;
-    for (size_t i = tid; i < n_per; i += 256) {
+    for (int i = tid; i < 8 * ld; i += 256) {
+        const int mm = i / ld, col = i - mm * ld, m = m0 + mm;
         float a = 0.f;
-        for (int s = 0; s < S; ++s) a += part[((size_t)bh * S + s) * n_per + i];
-        st[i] = a;
+        if (m < kMono) {
+            const float* src = part + (size_t)bh * S * n_per + (size_t)m * ld + col;
+            for (int s = 0; s < S; ++s) a += src[(size_t)s * n_per];      // fixed order: bit-reproducible
+            state[(size_t)bh * n_per + (size_t)m * ld + col] = a;
+        }
+        sm[mm][col] = a;
     }
     __syncthreads();
     __nv_bfloat16* o3 = b3 + (size_t)bh * (DV + 16) * kMonoPad;
-    for (int i = tid; i < (DV + 16) * kMonoPad; i += 256) {
-        const int row = i / kMonoPad, m = i % kMonoPad;
-        o3[i] = __float2bfloat16_rn((m < kMono && row <= DV) ? st[(size_t)m * ld + row] : 0.f);   // row == DV is the z column
+    for (int row = tid; row < DV + 16; row += 256) {       // row <= DV: column `row` of the state (row == DV is z); rest zero
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) w[e] = row <= DV ? pack_bf16(sm[2 * e][row], sm[2 * e + 1][row]) : 0u;
+        *reinterpret_cast<uint4*>(o3 + (size_t)row * kMonoPad + m0) = make_uint4(w[0], w[1], w[2], w[3]);
     }
     __nv_bfloat16* oq = bq + (size_t)bh * kMonoPad * DV;
-    for (int i = tid; i < kMonoPad * DV; i += 256) {
-        const int m = i / DV, g = i % DV;
-        oq[i] = __float2bfloat16_rn(m < kMono ? st[(size_t)m * ld + g] : 0.f);
+    for (int i = tid; i < 8 * DV; i += 256) {
+        const int mm = i / DV, g = i - mm * DV;
+        oq[(size_t)(m0 + mm) * DV + g] = __float2bfloat16_rn(sm[mm][g]);
     }
 }
 
@@ -1001,7 +1009,7 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     tc_state_build_kernel<DV><<<dim3(D.S, BH), kSbThreads, kSbSmem, st>>>(mapV, kf, part, D.N, D.S, D.ld, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    tc_reduce_emit_kernel<DV><<<BH, 256, 0, st>>>(part, state, b3, bq, D.S, D.ld);
+    tc_reduce_emit_kernel<DV><<<dim3(8, BH), 256, 0, st>>>(part, state, b3, bq, D.S, D.ld);
     if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
@@ -1040,7 +1048,7 @@ inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, con
     tc_bwd_query_kernel<DV><<<dim3(D.S, BH), kBqThreads, kBqSmem, st>>>(mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    tc_reduce_emit_kernel<DV><<<BH, 256, 0, st>>>(part, dstate, bd3, bdq, D.S, D.ld);
+    tc_reduce_emit_kernel<DV><<<dim3(8, BH), 256, 0, st>>>(part, dstate, bd3, bdq, D.S, D.ld);
     if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;

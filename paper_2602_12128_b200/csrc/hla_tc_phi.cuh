@@ -325,19 +325,26 @@ template <int DV, int NMAPS> struct PbCfg {
     static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
+    static constexpr int kW2tBytes = (DV / 64) * 2048;           // per map: [16 K rows][DV] bf16, MN-major B operand of the dg product
     static constexpr int kOffX = 0;
     static constexpr int kOffDh = kXStages * kXBytes;            // 2 dh tiles (A operand of the second MMA)
     static constexpr int kOffW1 = kOffDh + 2 * kXBytes;
-    static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;     // fp32 [NMAPS][6][DV]: W2 transposed, hidden index innermost
-    static constexpr int kOffB1 = kOffW2 + NMAPS * 6 * DV * 4;   // fp32 [NMAPS][DV]
+    static constexpr int kOffDp = kOffW1 + NMAPS * kW1Bytes;     // one swizzled block = 4 dp tiles [128 tok][16] (K slices 0..3)
+    static constexpr int kOffW2t = kOffDp + kBlk;
+    static constexpr int kOffB1 = kOffW2t + NMAPS * kW2tBytes;   // fp32 [NMAPS][DV]
     static constexpr int kOffBars = kOffB1 + NMAPS * DV * 4;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
 
 // X, dX [rows][DV] bf16.  KSIDE: feat / dfeat are [bh][NMAPS][N][6], else [rows][6].
-// h and the dh tile are double-buffered; the dX accumulator (double-buffered in TMEM) of a tile is drained
-// one unit late, straight from registers to global memory.
+// Per unit (one map of one 128-token tile) three products run on the tensor cores:
+//   h  = X * W1                         [128 x DV], K = DV
+//   dg = [dp_hi | dp_lo] * [W2^T; W2^T]  [128 x DV], K = 16: dp = dfeat (.) 1[feat > 0] split into two bf16 halves, so dg is exact to ~2^-17
+//   dX += dh * W1^T                     [128 x DV], K = DV,  dh = dg (.) GELU'(h + b1) formed by the 16 epilogue warps
+// h and the dh tile are double-buffered; dg is taken into registers at the start of a unit so that the next unit's dg
+// product overlaps this unit's arithmetic; the dX accumulator of a tile is drained one unit late, straight from
+// registers to global memory.  Warp 0 issues the TMA loads and writes the dp tiles up to four units ahead.
 template <int DV, int NMAPS, bool KSIDE>
 __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
                                                                         PhiBwdPtrs P, const float* __restrict__ feat, const float* __restrict__ dfeat,
@@ -347,7 +354,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    float* w2s = reinterpret_cast<float*>(smem + Cfg::kOffW2);
     float* b1s = reinterpret_cast<float*>(smem + Cfg::kOffB1);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* x_full = bars;           // [2]
@@ -356,10 +362,14 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* h_empty = bars + 6;      // [2] 512 arrivals
     uint64_t* dh_full = bars + 8;      // [2] 512 arrivals
     uint64_t* dh_free = bars + 10;     // [2] MMA commit
-    uint64_t* dx_full = bars + 12;     // [2] MMA commit
-    uint64_t* dx_empty = bars + 14;    // [2] 512 arrivals
-    uint64_t* w_full = bars + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+    uint64_t* dp_full = bars + 12;     // [4] 32 arrivals (warp 0)
+    uint64_t* dp_free = bars + 16;     // [4] MMA commit
+    uint64_t* dg_full = bars + 20;     // MMA commit
+    uint64_t* dg_empty = bars + 21;    // 512 arrivals
+    uint64_t* dx_full = bars + 22;     // MMA commit
+    uint64_t* dx_empty = bars + 23;    // 512 arrivals
+    uint64_t* w_full = bars + 24;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -367,11 +377,15 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     const int ntiles = (int)(t1 - t0);
     const int nunits = ntiles * NMAPS;
 
-    for (int i = tid; i < NMAPS * 6 * DV; i += kPbThreads) {
-        const int m = i / (6 * DV), o = (i / DV) % 6, j = i % DV;
-        w2s[i] = __bfloat162float(P.W2[m][j * 6 + o]);
+    // W2^T stacked twice (rows 0..5 meet dp_hi, rows 6..11 meet dp_lo, rows 12..15 are zero), as an MN-major operand
+    for (int i = tid; i < NMAPS * 16 * DV; i += kPbThreads) {
+        const int m = i / (16 * DV), k = (i / DV) & 15, j = i % DV;
+        uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * 2048;
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? P.W2[m][j * 6 + (k % 6)] : __float2bfloat16_rn(0.f);
     }
     for (int i = tid; i < NMAPS * DV; i += kPbThreads) b1s[i] = __bfloat162float(P.b1[i / DV][i % DV]);
+    for (int i = tid; i < kBlk / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(&x_full[i], 1);
@@ -380,9 +394,15 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             mbar_init(&h_empty[i], 512);
             mbar_init(&dh_full[i], 512);
             mbar_init(&dh_free[i], 1);
-            mbar_init(&dx_full[i], 1);
-            mbar_init(&dx_empty[i], 512);
         }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(&dp_full[i], 32);
+            mbar_init(&dp_free[i], 1);
+        }
+        mbar_init(dg_full, 1);
+        mbar_init(dg_empty, 512);
+        mbar_init(dx_full, 1);
+        mbar_init(dx_empty, 512);
         mbar_init(w_full, 1);
         fence_mbar_init();
         prefetch_tmap(&mapX);
@@ -394,27 +414,92 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;     // h[b] at columns 128*b, dX[b] at columns 256 + 128*b
+    const uint32_t tmem = *tmem_slot;     // h[b] at columns 128*b, dg at 256, dX at 384
     bool ok = true;
 
     if (warp == 0) {
-        if (lane == 0 && ntiles > 0) {
-            mbar_arrive_expect_tx(w_full, NMAPS * Cfg::kW1Bytes);
-            for (int m = 0; m < NMAPS; ++m)
-                for (int b = 0; b < DV / 64; ++b)
-                    tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
-            for (int it = 0; it < ntiles; ++it) {
-                const int st = it % XST, u = it / XST;
-                if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 601); break; }
-                mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
-                for (int b = 0; b < DV / 64; ++b)
-                    tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
+        if (ntiles > 0) {
+            if (lane == 0) {
+                mbar_arrive_expect_tx(w_full, NMAPS * Cfg::kW1Bytes);
+                for (int m = 0; m < NMAPS; ++m)
+                    for (int b = 0; b < DV / 64; ++b)
+                        tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
+            }
+            const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
+            // Features and feature gradients of rows lane, lane + 32, lane + 64, lane + 96 of a unit.  The loads are
+            // unconditional (row index clamped) and issued one unit ahead, so their latency never sits on the unit's path.
+            float fr[4][6], gr[4][6];
+            auto load_rows = [&](int unit) {
+                const int it = unit / NMAPS, m = unit % NMAPS;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    long long grow = (t0 + it) * kTileTokens + lane + 32 * i;
+                    grow = grow < rows ? grow : rows - 1;
+                    size_t off;
+                    if (KSIDE) {
+                        const long long bh = grow / N, n = grow - bh * N;
+                        off = (size_t)((bh * NMAPS + m) * N + n) * 6;
+                    } else {
+                        off = (size_t)grow * 6;
+                    }
+                    load6(fr[i], feat + off);
+                    load6(gr[i], dfeat + off);
+                }
+            };
+            load_rows(0);
+            for (int unit = 0; unit < nunits; ++unit) {
+                const int it = unit / NMAPS, m = unit % NMAPS, slot = unit & 3;
+                if (m == 0) {      // this tile's X
+                    if (lane == 0) {
+                        const int st = it % XST, u = it / XST;
+                        ok = mbar_wait(&x_empty[st], (u & 1) ^ 1);
+                        if (ok) {
+                            mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
+                            for (int b = 0; b < DV / 64; ++b)
+                                tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
+                        } else {
+                            report_timeout(status, 601);
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                }
+                uint32_t w[4][6];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const bool live = (t0 + it) * kTileTokens + lane + 32 * i < rows;
+                    float dp[6], lo[6];
+#pragma unroll
+                    for (int o = 0; o < 6; ++o) {
+                        dp[o] = (live && fr[i][o] > 0.f) ? gr[i][o] : 0.f;
+                        lo[o] = dp[o] - __bfloat162float(__float2bfloat16_rn(dp[o]));
+                    }
+                    w[i][0] = pack_bf16(dp[0], dp[1]);
+                    w[i][1] = pack_bf16(dp[2], dp[3]);
+                    w[i][2] = pack_bf16(dp[4], dp[5]);
+                    w[i][3] = pack_bf16(lo[0], lo[1]);
+                    w[i][4] = pack_bf16(lo[2], lo[3]);
+                    w[i][5] = pack_bf16(lo[4], lo[5]);
+                }
+                if (unit + 1 < nunits) load_rows(unit + 1);
+                if (!mbar_wait(&dp_free[slot], ((unit >> 2) & 1) ^ 1)) { ok = false; report_timeout(status, 607); }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t r = lane + 32 * i;
+                    st_shared_v4(dpblk + sw128_off(r, 2 * slot), w[i][0], w[i][1], w[i][2], w[i][3]);
+                    st_shared_v4(dpblk + sw128_off(r, 2 * slot + 1), w[i][4], w[i][5], 0u, 0u);
+                }
+                fence_proxy_async();
+                mbar_arrive(&dp_full[slot]);
             }
         }
     } else if (warp == 1) {
         if (lane == 0 && ntiles > 0) {
-            const uint32_t idesc1 = idesc_bf16(128, DV, false, true);    // h  = X (K-major) * W1 [in][hidden] (MN-major)
+            const uint32_t idesc1 = idesc_bf16(128, DV, false, true);    // h = X (K-major) * W1 [in][hidden] (MN-major); dg = dp (K-major) * W2^T (MN-major)
             const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (K-major over hidden) * W1 as [in][hidden] (K-major)
+            const uint32_t dpa = smem_u32(smem + Cfg::kOffDp);
             bool good = mbar_wait(w_full, 0);
             if (!good) report_timeout(status, 602);
             auto issue_mma1 = [&](int unit) -> bool {
@@ -432,21 +517,35 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 if (m == NMAPS - 1) umma_commit(&x_empty[st]);
                 return true;
             };
+            // dg of `unit`; the epilogue of unit - 1 must have taken its dg into registers
+            auto issue_dg = [&](int unit) -> bool {
+                const int m = unit % NMAPS, slot = unit & 3;
+                if (unit > 0 && !mbar_wait(dg_empty, (unit - 1) & 1)) return false;
+                if (!mbar_wait(&dp_full[slot], (unit >> 2) & 1)) return false;
+                tc_fence_after();
+                umma_bf16(tmem + 256, smem_desc_sw128(dpa + slot * 32, 16, 1024),
+                          smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t + m * Cfg::kW2tBytes), 2048, 1024), idesc1, 0u);
+                umma_commit(dg_full);
+                umma_commit(&dp_free[slot]);
+                return true;
+            };
             if (good && nunits > 0) good = issue_mma1(0);
             if (good && nunits > 1) good = issue_mma1(1);
+            if (good && nunits > 0) good = issue_dg(0);
             for (int unit = 0; unit < nunits && good; ++unit) {
-                const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, tb = it & 1;
+                const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1;
+                if (unit + 1 < nunits && !issue_dg(unit + 1)) { good = false; break; }
                 if (!mbar_wait(&dh_full[b], (unit >> 1) & 1)) { good = false; break; }
-                if (m == 0 && !mbar_wait(&dx_empty[tb], ((it >> 1) & 1) ^ 1)) { good = false; break; }
+                if (m == 0 && !mbar_wait(dx_empty, (it & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
                 const uint32_t dha = smem_u32(smem + Cfg::kOffDh + b * Cfg::kXBytes);
                 const uint32_t wa = smem_u32(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 256 + 128 * tb, smem_desc_sw128(dha + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                    umma_bf16(tmem + 384, smem_desc_sw128(dha + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
                               smem_desc_sw128(wa + (ks >> 2) * (DV * 128) + (ks & 3) * 32, 16, 1024), idesc2, (m > 0 || ks > 0) ? 1u : 0u);
                 umma_commit(&dh_free[b]);
-                if (m == NMAPS - 1) umma_commit(&dx_full[tb]);
+                if (m == NMAPS - 1) umma_commit(dx_full);
                 if (unit + 2 < nunits) good = issue_mma1(unit + 2);
             }
             if (!good) report_timeout(status, 603);
@@ -454,14 +553,14 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     } else {
         const int quarter = warp & 3, part = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         // dX of tile `it`: TMEM -> bf16 -> global memory (each thread: HC contiguous columns of its row)
         auto drain_dx = [&](int it) {
-            const int tb = it & 1;
-            if (ok && !mbar_wait(&dx_full[tb], (it >> 1) & 1)) { ok = false; report_timeout(status, 606); }
+            if (ok && !mbar_wait(dx_full, it & 1)) { ok = false; report_timeout(status, 606); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return;
             tc_fence_after();
-            const uint32_t tx = tmem + 256 + 128 * tb + ((uint32_t)(quarter * 32) << 16) + part * HC;
+            const uint32_t tx = tmem + 384 + lane_base + part * HC;
             const long long grow = (t0 + it) * kTileTokens + row;
             uint4* dst = reinterpret_cast<uint4*>(dX + (size_t)grow * DV + part * HC);
 #pragma unroll
@@ -478,65 +577,42 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 }
             }
             tc_fence_before();
-            mbar_arrive(&dx_empty[tb]);
+            mbar_arrive(dx_empty);
         };
         for (int unit = 0; unit < nunits && ok; ++unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
-            const long long grow = (t0 + it) * kTileTokens + row;
-            float2 dp[6];
-            if (grow < rows) {
-                size_t off;
-                if (KSIDE) {
-                    const long long bh = grow / N, n = grow - bh * N;
-                    off = (size_t)((bh * NMAPS + m) * N + n) * 6;
-                } else {
-                    off = (size_t)grow * 6;
-                }
-                float f[6], g[6];
-                load6(f, feat + off);
-                load6(g, dfeat + off);
+            if (!mbar_wait(dg_full, unit & 1)) { ok = false; report_timeout(status, 608); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t dgr[HC];
 #pragma unroll
-                for (int o = 0; o < 6; ++o) dp[o] = splat2(f[o] > 0.f ? g[o] : 0.f);
-            } else {
-#pragma unroll
-                for (int o = 0; o < 6; ++o) dp[o] = splat2(0.f);
-            }
+            for (int c = 0; c < HC / 16; ++c) tmem_ld16(tmem + 256 + lane_base + part * HC + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(dgr + 16 * c));
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(dg_empty);
             if (!mbar_wait(&h_full[b], par)) { ok = false; report_timeout(status, 604); }
             if (ok && !mbar_wait(&dh_free[b], par ^ 1)) { ok = false; report_timeout(status, 605); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
+            const uint32_t ta = tmem + 128 * b + lane_base + part * HC;
             const uint32_t dblk = smem_u32(smem + Cfg::kOffDh + b * Cfg::kXBytes);
             const float* bm = b1s + m * DV;
-            const float* wm = w2s + m * 6 * DV;
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
                 uint32_t r[16];
                 tmem_ld16(ta + 16 * c, r);
                 tmem_ld_wait();
                 const int col = part * HC + 16 * c;
+                const float2* bb = reinterpret_cast<const float2*>(bm + col);
                 uint32_t w[8];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {      // four hidden units at a time: dg = dp . W2[j][:], dh = dg GELU'(h + b1)
-                    float2 dga, dgb;
-#pragma unroll
-                    for (int o = 0; o < 6; ++o) {
-                        const float4 wv = *reinterpret_cast<const float4*>(wm + o * DV + col + 4 * q4);
-                        if (o == 0) {
-                            dga = __fmul2_rn(dp[0], make_float2(wv.x, wv.y));
-                            dgb = __fmul2_rn(dp[0], make_float2(wv.z, wv.w));
-                        } else {
-                            dga = __ffma2_rn(dp[o], make_float2(wv.x, wv.y), dga);
-                            dgb = __ffma2_rn(dp[o], make_float2(wv.z, wv.w), dgb);
-                        }
-                    }
-                    const float4 bv = *reinterpret_cast<const float4*>(bm + col + 4 * q4);
-                    const float2 ha = __fadd2_rn(make_float2(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1])), make_float2(bv.x, bv.y));
-                    const float2 hb = __fadd2_rn(make_float2(__uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3])), make_float2(bv.z, bv.w));
-                    const float2 da = __fmul2_rn(dga, gelu_grad2(ha)), db = __fmul2_rn(dgb, gelu_grad2(hb));
-                    w[2 * q4] = pack_bf16(da.x, da.y);
-                    w[2 * q4 + 1] = pack_bf16(db.x, db.y);
+                for (int e = 0; e < 8; ++e) {
+                    const float2 h = __fadd2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), bb[e]);
+                    const float2 dg = make_float2(__uint_as_float(dgr[16 * c + 2 * e]), __uint_as_float(dgr[16 * c + 2 * e + 1]));
+                    const float2 dh = __fmul2_rn(dg, gelu_grad2(h));
+                    w[e] = pack_bf16(dh.x, dh.y);
                 }
                 const uint32_t blk = dblk + (col >> 6) * kBlk;
                 st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
