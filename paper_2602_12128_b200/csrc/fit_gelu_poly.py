@@ -1,45 +1,49 @@
-"""Fits the odd polynomial erf(u) ~ u * P(u^2) on [0, c] that the tensor-core phi kernels use for
-the exact (erf) GELU, GELU(x) = x/2 + (x/2) erf(x / sqrt 2), with u clamped to [-c, c].
+"""Fits the polynomial the tensor-core phi kernels use for the exact (erf) GELU.
 
-Run:  python fit_gelu_poly.py   -> prints the coefficients (lowest order first) and the maximum
-absolute error of erf and of GELU in fp32 Horner evaluation.  The constants in hla_tc_phi.cuh
-are this script's output for c = 3.0, 9 coefficients."""
+The normal CDF is evaluated as   Phi(x) ~ sat(1/2 + x * P(min(x^2, T)))   with sat = clamp to [0, 1]
+(one saturating fma), P of degree NCOEF-1 in t = x^2, fitted on |x| <= sqrt(T) so that
+x * P(x^2) ~ erf(x / sqrt 2) / 2.  Past sqrt(T) the expression grows linearly and saturates at 0 or 1.
+GELU(x) = x Phi(x);  GELU'(x) = Phi(x) + x exp(-x^2 / 2) / sqrt(2 pi).
+
+Run:  python fit_gelu_poly.py   -> prints the coefficients (highest order first, as the Horner
+evaluation in hla_tc_phi.cuh lists them) and the maximum absolute errors of Phi and GELU in fp32.
+The constants in hla_tc_phi.cuh are this script's output for T = 16, NCOEF = 7."""
 import numpy as np
 from scipy.special import erf
 
-C, NCOEF = 3.0, 9
+T, NCOEF = 16.0, 7
 
 
-def fit(c=C, n=NCOEF, iters=200):
-    u = 0.5 * c * (1 - np.cos(np.linspace(0, np.pi, 6001)))[1:]
-    A = np.stack([u ** (2 * k + 1) for k in range(n)], 1)
-    y = erf(u)
-    w = np.ones_like(u)
+def fit(T=T, n=NCOEF, iters=400):
+    X = np.sqrt(T)
+    x = 0.5 * X * (1 - np.cos(np.linspace(0, np.pi, 8001)))[1:]
+    A = np.stack([x ** (2 * k + 1) for k in range(n)], 1)
+    scale = np.abs(A).max(0)
+    A = A / scale
+    y = 0.5 * erf(x / np.sqrt(2))
+    w = np.ones_like(x)
     for _ in range(iters):                      # reweighted least squares towards the minimax fit
         coef, *_ = np.linalg.lstsq(A * w[:, None], y * w, rcond=None)
         err = np.abs(A @ coef - y)
         w *= 1 + 2 * err / err.max()
         w /= w.mean()
-    return coef
+    return coef / scale
 
 
-def gelu_poly_f32(x, coef, c=C):
+def phi_f32(x, coef, T=T):
     x = x.astype(np.float32)
-    u = np.clip(x * np.float32(0.70710678), np.float32(-c), np.float32(c))
-    t = u * u
+    t = np.minimum(x * x, np.float32(T))
     p = np.float32(coef[-1])
     for a in coef[-2::-1]:
         p = p * t + np.float32(a)
-    hx = np.float32(0.5) * x
-    return hx * (u * p) + hx
+    return np.clip(x * p + np.float32(0.5), 0, 1).astype(np.float32)
 
 
 if __name__ == "__main__":
     coef = fit()
-    print("coefficients:", ", ".join("%.9ef" % a for a in coef))
-    uu = np.linspace(-6, 6, 1200001)
-    ref = 0.5 * uu * (1 + erf(uu / np.sqrt(2)))
-    got = gelu_poly_f32(uu, coef).astype(np.float64)
-    print("max |gelu_poly - gelu| on [-6,6]: %.3e" % np.abs(got - ref).max())
-    u = np.linspace(0, C, 300001)
-    print("max |erf_poly - erf| on [0,c]: %.3e ; 1 - erf(c) = %.3e" % (np.abs(sum(a * u ** (2 * k + 1) for k, a in enumerate(coef)) - erf(u)).max(), 1 - erf(C)))
+    print("coefficients (highest first):", ", ".join("%.9ef" % a for a in coef[::-1]))
+    x = np.linspace(-9, 9, 1800001)
+    ref = 0.5 * (1 + erf(x / np.sqrt(2)))
+    got = phi_f32(x, coef).astype(np.float64)
+    print("max |Phi_poly - Phi|: %.3e" % np.abs(got - ref).max())
+    print("max |x Phi_poly - GELU|: %.3e" % np.abs(x.astype(np.float32) * got - x * ref).max())

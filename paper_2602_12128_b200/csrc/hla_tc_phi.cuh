@@ -7,32 +7,34 @@
 //   D2 = G * W2[m]            tcgen05, N padded to 16
 //   feat = ReLU(D2 + b2)      fp32 features to global memory
 // The key side runs its F maps on the same X tile, so K is read once.
-// GELU is the exact erf form evaluated with an odd polynomial for erf (fit_gelu_poly.py: |error| < 7e-5,
-// far below the bf16 rounding of G) on packed fp32 pairs - no special-function unit on the forward's hot loop.
+// GELU is the exact erf form evaluated with an odd polynomial for erf (fit_gelu_poly.py: |error| < 1.1e-4 on Phi,
+// below the bf16 rounding of G) on packed fp32 pairs - no special-function unit on the forward's hot loop.
 #pragma once
 #include "hla_tc.cuh"
 
 namespace hla {
 namespace tc {
 
-// Phi(x) = 1/2 + erf(x / sqrt 2) / 2 as 1/2 + xc * P(xc^2) with xc = x clamped to +-3 sqrt 2 (fit_gelu_poly.py; the
-// coefficients are those of erf(u) ~ u P(u^2) rescaled to the variable x).  Evaluated on pairs with the packed
-// fp32 instructions (fma.rn.f32x2), which halve the number of issue slots.
+// Phi(x) = 1/2 + erf(x / sqrt 2) / 2 evaluated as sat(1/2 + x P(min(x^2, 16))), sat = clamp to [0, 1] done by one
+// saturating fma (fit_gelu_poly.py: |error| < 1.1e-4, several times below the bf16 rounding of the result).  The
+// Horner steps run on pairs with the packed fp32 instructions (fma.rn.f32x2), which halve the issue slots.
 __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ float2 normal_cdf2(float2 x) {
-    constexpr float kClamp = 4.2426405f;
-    const float2 xc = make_float2(fminf(fmaxf(x.x, -kClamp), kClamp), fminf(fmaxf(x.y, -kClamp), kClamp));
-    const float2 t = __fmul2_rn(xc, xc);
-    float2 p = splat2(5.626761649e-11f);
-    p = __ffma2_rn(p, t, splat2(-5.371864642e-09f));
-    p = __ffma2_rn(p, t, splat2(2.268294939e-07f));
-    p = __ffma2_rn(p, t, splat2(-5.646213026e-06f));
-    p = __ffma2_rn(p, t, splat2(9.359060759e-05f));
-    p = __ffma2_rn(p, t, splat2(-1.109400211e-03f));
-    p = __ffma2_rn(p, t, splat2(9.818118887e-03f));
-    p = __ffma2_rn(p, t, splat2(-6.634692326e-02f));
-    p = __ffma2_rn(p, t, splat2(3.989031265e-01f));
-    return __ffma2_rn(xc, p, splat2(0.5f));
+    const float2 xx = __fmul2_rn(x, x);
+    const float2 t = make_float2(fminf(xx.x, 16.f), fminf(xx.y, 16.f));
+    float2 p = splat2(2.816106894e-08f);
+    p = __ffma2_rn(p, t, splat2(-1.891893110e-06f));
+    p = __ffma2_rn(p, t, splat2(5.419046974e-05f));
+    p = __ffma2_rn(p, t, splat2(-8.789816123e-04f));
+    p = __ffma2_rn(p, t, splat2(9.112954582e-03f));
+    p = __ffma2_rn(p, t, splat2(-6.538836121e-02f));
+    p = __ffma2_rn(p, t, splat2(3.985269153e-01f));
+    return make_float2(fma_sat(x.x, p.x, 0.5f), fma_sat(x.y, p.y, 0.5f));
 }
 // GELU(x) = x Phi(x)
 __device__ __forceinline__ float2 gelu2(float2 x) { return __fmul2_rn(x, normal_cdf2(x)); }
@@ -57,7 +59,11 @@ struct PhiMaps {
     CUtensorMap w1[3];
 };
 
-constexpr int kPfThreads = 576;   // warp 0: TMA, warp 1: MMA, warps 2..17: epilogue (thread = token row x quarter of the hidden units)
+// warp 0: TMA loads, warp 1: second-layer MMAs, warp 2: first-layer MMAs, warps 3..18: GELU (thread = token row x quarter of
+// the hidden units), warps 19..22: feature epilogue.  The two MMA streams are issued by different warps (different
+// schedulers) because one thread issuing both was the slowest stage of the pipeline.
+constexpr int kPfThreads = 736;
+constexpr int kPfGeluWarp0 = 3, kPfFeatWarp0 = 19;
 
 template <int DV, int NMAPS> struct PfCfg {
     static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;   // one stage is enough when a tile has three units
@@ -156,54 +162,54 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
                     tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0 && ntiles > 0) {
+    } else if (warp == 2) {
+        if (lane == 0 && ntiles > 0) {      // D1[b] = X * W1[m]
             const uint32_t idesc1 = idesc_bf16(128, DV, false, true);   // X K-major, W1 [in][hidden] MN-major
-            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G K-major, W2 operand K-major
+            const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
+            const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
             bool good = mbar_wait(w_full, 0);
-            if (!good) report_timeout(status, 502);
-            auto issue_mma1 = [&](int unit) -> bool {
+            for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
-                if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) return false;
-                if (!mbar_wait(&d1_empty[b], ((unit >> 1) & 1) ^ 1)) return false;
+                if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) { good = false; break; }
+                if (!mbar_wait(&d1_empty[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
-                const uint32_t xa = smem_u32(smem + Cfg::kOffX + st * Cfg::kXBytes);
-                const uint32_t wa = smem_u32(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes);
+                const uint64_t xd = desc_advance(xd0, st * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 128 * b, smem_desc_sw128(xa + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(wa + ks * 2048, DV * 128, 1024), idesc1, ks > 0 ? 1u : 0u);
+                    umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
                 umma_commit(&d1_full[b]);
                 if (m == NMAPS - 1) umma_commit(&x_empty[st]);
-                return true;
-            };
-            if (good && nunits > 0) good = issue_mma1(0);
-            if (good && nunits > 1) good = issue_mma1(1);
+            }
+            if (!good) report_timeout(status, 502);
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && ntiles > 0) {      // D2[b] = G[b] * W2[m]
+            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G K-major, W2 operand K-major
+            const uint64_t gd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffG), 16, 1024);
+            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 16, 1024);
+            bool good = true;
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
                 if (!(mbar_wait(&g_full[b], par) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
                 tc_fence_after();
-                const uint32_t ga = smem_u32(smem + Cfg::kOffG + b * Cfg::kXBytes);
-                const uint32_t w2a = smem_u32(smem + Cfg::kOffW2 + m * Cfg::kW2Bytes);
+                const uint64_t gd = desc_advance(gd0, b * Cfg::kXBytes), vd = desc_advance(vd0, m * Cfg::kW2Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 256 + 32 * b, smem_desc_sw128(ga + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(w2a + (ks >> 2) * 2048 + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
+                    umma_bf16(tmem + 256 + 32 * b, desc_advance(gd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32),
+                              idesc2, ks > 0 ? 1u : 0u);
                 umma_commit(&g_free[b]);
                 umma_commit(&d2_full[b]);
-                if (unit + 2 < nunits) good = issue_mma1(unit + 2);
             }
             if (!good) report_timeout(status, 503);
         }
-    } else {
-        const int quarter = warp & 3, part = (warp - 2) >> 2;
-        const int row = quarter * 32 + lane;
-        // feature epilogue of one unit (the part-0 warps only): ReLU(D2 + b2) -> global memory
-        auto emit_features = [&](int unit) {
+    } else if (warp >= kPfFeatWarp0) {
+        // feature epilogue: ReLU(D2 + b2) -> global memory; thread = token row
+        const int quarter = warp & 3, row = quarter * 32 + lane;
+        for (int unit = 0; unit < nunits; ++unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1;
-            if (ok && !mbar_wait(&d2_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 506); }
+            if (!mbar_wait(&d2_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 506); }
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) return;
+            if (!ok) break;
             tc_fence_after();
             uint32_t r[8];
             tmem_ld8(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), r);
@@ -223,8 +229,11 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
                     store6(feat + grow * 6, f);
                 }
             }
-        };
-        for (int unit = 0; unit < nunits && ok; ++unit) {
+        }
+    } else {
+        const int quarter = warp & 3, part = (warp - kPfGeluWarp0) >> 2;
+        const int row = quarter * 32 + lane;
+        for (int unit = 0; unit < nunits; ++unit) {
             const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
             const float* b1s = bias + m * (DV + 8);
             if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 504); }
@@ -234,30 +243,29 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             tc_fence_after();
             const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
             const uint32_t gblk = smem_u32(smem + Cfg::kOffG + b * Cfg::kXBytes);
+            uint32_t r[HC];
+#pragma unroll
+            for (int c = 0; c < HC / 16; ++c) tmem_ld16(ta + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(&d1_empty[b]);          // h is in registers: the next first-layer product may overwrite it
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
-                uint32_t r[16];
-                tmem_ld16(ta + 16 * c, r);
-                tmem_ld_wait();
                 const int col = part * HC + 16 * c;
                 const float2* bb = reinterpret_cast<const float2*>(b1s + col);
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), bb[e]));
+                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])), bb[e]));
                     w[e] = pack_bf16(g.x, g.y);
                 }
                 const uint32_t blk = gblk + (col >> 6) * kBlk;
                 st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
                 st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
             }
-            tc_fence_before();
-            mbar_arrive(&d1_empty[b]);
             fence_proxy_async();
             mbar_arrive(&g_full[b]);
-            if (part == 0 && unit > 0) emit_features(unit - 1);
         }
-        if (part == 0 && ok && nunits > 0) emit_features(nunits - 1);
     }
     tc_fence_before();
     __syncthreads();
@@ -319,7 +327,9 @@ struct PhiBwdPtrs {
     const __nv_bfloat16* W2[3];
 };
 
-constexpr int kPbThreads = 576;   // warp 0: TMA loads, warp 1: MMA, warps 2..17: epilogue (thread = token row x quarter of the columns)
+// warp 0: TMA loads and dp tiles, warp 1: dg and dX MMAs, warp 2: h MMAs, warps 3..18: epilogue (thread = token row x quarter of the columns)
+constexpr int kPbThreads = 608;
+constexpr int kPbEpiWarp0 = 3;
 
 template <int DV, int NMAPS> struct PbCfg {
     static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;
@@ -495,42 +505,46 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 mbar_arrive(&dp_full[slot]);
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0 && ntiles > 0) {
-            const uint32_t idesc1 = idesc_bf16(128, DV, false, true);    // h = X (K-major) * W1 [in][hidden] (MN-major); dg = dp (K-major) * W2^T (MN-major)
-            const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (K-major over hidden) * W1 as [in][hidden] (K-major)
-            const uint32_t dpa = smem_u32(smem + Cfg::kOffDp);
+    } else if (warp == 2) {
+        if (lane == 0 && ntiles > 0) {      // h[b] = X * W1[m]
+            const uint32_t idesc1 = idesc_bf16(128, DV, false, true);    // X K-major, W1 [in][hidden] MN-major
+            const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
+            const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
             bool good = mbar_wait(w_full, 0);
-            if (!good) report_timeout(status, 602);
-            auto issue_mma1 = [&](int unit) -> bool {
+            for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
-                if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) return false;
-                if (!mbar_wait(&h_empty[b], ((unit >> 1) & 1) ^ 1)) return false;
+                if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) { good = false; break; }
+                if (!mbar_wait(&h_empty[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
-                const uint32_t xa = smem_u32(smem + Cfg::kOffX + st * Cfg::kXBytes);
-                const uint32_t wa = smem_u32(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes);
+                const uint64_t xd = desc_advance(xd0, st * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 128 * b, smem_desc_sw128(xa + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(wa + ks * 2048, DV * 128, 1024), idesc1, ks > 0 ? 1u : 0u);
+                    umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
                 umma_commit(&h_full[b]);
                 if (m == NMAPS - 1) umma_commit(&x_empty[st]);
-                return true;
-            };
+            }
+            if (!good) report_timeout(status, 602);
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && ntiles > 0) {
+            const uint32_t idesc_dg = idesc_bf16(128, DV, false, true);  // dg = dp (K-major) * W2^T (MN-major)
+            const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (K-major over hidden) * W1 as [in][hidden] (K-major)
+            const uint64_t pd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp), 16, 1024);
+            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
+            const uint64_t hd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffDh), 16, 1024);
+            const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), 16, 1024);
+            bool good = mbar_wait(w_full, 0);
             // dg of `unit`; the epilogue of unit - 1 must have taken its dg into registers
             auto issue_dg = [&](int unit) -> bool {
                 const int m = unit % NMAPS, slot = unit & 3;
                 if (unit > 0 && !mbar_wait(dg_empty, (unit - 1) & 1)) return false;
                 if (!mbar_wait(&dp_full[slot], (unit >> 2) & 1)) return false;
                 tc_fence_after();
-                umma_bf16(tmem + 256, smem_desc_sw128(dpa + slot * 32, 16, 1024),
-                          smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t + m * Cfg::kW2tBytes), 2048, 1024), idesc1, 0u);
+                umma_bf16(tmem + 256, desc_advance(pd0, slot * 32), desc_advance(vd0, m * Cfg::kW2tBytes), idesc_dg, 0u);
                 umma_commit(dg_full);
                 umma_commit(&dp_free[slot]);
                 return true;
             };
-            if (good && nunits > 0) good = issue_mma1(0);
-            if (good && nunits > 1) good = issue_mma1(1);
             if (good && nunits > 0) good = issue_dg(0);
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1;
@@ -538,20 +552,18 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 if (!mbar_wait(&dh_full[b], (unit >> 1) & 1)) { good = false; break; }
                 if (m == 0 && !mbar_wait(dx_empty, (it & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
-                const uint32_t dha = smem_u32(smem + Cfg::kOffDh + b * Cfg::kXBytes);
-                const uint32_t wa = smem_u32(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes);
+                const uint64_t hd = desc_advance(hd0, b * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 384, smem_desc_sw128(dha + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(wa + (ks >> 2) * (DV * 128) + (ks & 3) * 32, 16, 1024), idesc2, (m > 0 || ks > 0) ? 1u : 0u);
+                    umma_bf16(tmem + 384, desc_advance(hd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, (ks >> 2) * (DV * 128) + (ks & 3) * 32), idesc2,
+                              (m > 0 || ks > 0) ? 1u : 0u);
                 umma_commit(&dh_free[b]);
                 if (m == NMAPS - 1) umma_commit(dx_full);
-                if (unit + 2 < nunits) good = issue_mma1(unit + 2);
             }
             if (!good) report_timeout(status, 603);
         }
     } else {
-        const int quarter = warp & 3, part = (warp - 2) >> 2;
+        const int quarter = warp & 3, part = (warp - kPbEpiWarp0) >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         // dX of tile `it`: TMEM -> bf16 -> global memory (each thread: HC contiguous columns of its row)
