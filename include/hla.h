@@ -137,6 +137,38 @@ hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *
                         const void *dO, void *dQ, void *dK, void *dV,
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * Forward without a caller-provided workspace (no counterpart in the paper: a
+ * deployment aid).  Some callers of this library cannot obtain device memory
+ * at the time they need the operator: a plug-in running inside a host
+ * application that owns the allocator, a real-time loop that forbids
+ * allocation after start-up, code that only receives the tensors it is
+ * handed.  For them the library carries its own scratch: one array of
+ * HLA_STATIC_WS_BYTES bytes that is part of the loaded module, so every GPU
+ * that loads the library holds that much memory until the process exits.
+ * This call computes exactly what hla_forward computes, with that array as the
+ * workspace, and calls no memory-allocating routine.
+ *
+ *   - Contexts whose hla_workspace_bytes() exceeds HLA_STATIC_WS_BYTES are
+ *     refused with HLA_ERR_WORKSPACE before anything is enqueued.
+ *   - The first call on a device looks up the array's device address (with
+ *     that device current) and remembers it; make that first call outside any
+ *     stream capture.  Later calls on the same device only enqueue work.
+ *   - All contexts and all calls share the one array, and it keeps what the
+ *     previous call left in it.  Everything a call reads from it is written
+ *     earlier in the same call (the status words are cleared at the start),
+ *     so back-to-back calls on one stream are independent; two calls that can
+ *     overlap on the GPU (different streams without an ordering between them)
+ *     race on it and must not be made.
+ *   - If `scratch_out` is not NULL it receives the array's device address:
+ *     pass it as `workspace` to hla_last_device_status, to hla_backward (the
+ *     state of the forward lives there), or add hla_workspace_layout offsets
+ *     to read eta or the state.
+ */
+#define HLA_STATIC_WS_BYTES (16u * 1024u * 1024u)
+hla_status hla_forward_static(hla_ctx *ctx, const void *Q, const void *K, const void *V, void *O,
+                              void *cuda_stream, void **scratch_out);
+
 /* Synchronises `cuda_stream`, reads the device status words of `workspace`
  * and returns HLA_OK, HLA_ERR_DEVICE_TIMEOUT or HLA_ERR_CUDA. */
 hla_status hla_last_device_status(hla_ctx *ctx, const void *workspace, void *cuda_stream);

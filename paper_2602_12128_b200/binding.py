@@ -17,7 +17,7 @@ HLA_BF16, HLA_F32 = 0, 1
 HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
-    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward",
+    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_forward_static",
     "hla_last_device_status", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
     "hla_destroy", "hla_status_string",
 ]
@@ -72,6 +72,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_forward.restype = c_int32
     lib.hla_backward.argtypes = [c_void_p] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
     lib.hla_backward.restype = c_int32
+    lib.hla_forward_static.argtypes = [c_void_p] + [c_void_p] * 4 + [c_void_p, POINTER(c_void_p)]
+    lib.hla_forward_static.restype = c_int32
     lib.hla_last_device_status.argtypes = [c_void_p, c_void_p, c_void_p]
     lib.hla_last_device_status.restype = c_int32
     lib.hla_last_launch_count.argtypes = [c_void_p]
@@ -153,6 +155,19 @@ def hla_backward(ctx: int, Q, K, V, O, dO, dQ, dK, dV, workspace, stream=None, w
                                      _ptr(workspace), nbytes, _stream(stream))
     if st != HLA_OK:
         raise HlaError(st, "hla_backward")
+
+
+HLA_STATIC_WS_BYTES = 16 * 1024 * 1024
+
+
+def hla_forward_static(ctx: int, Q, K, V, O, stream=None) -> int:
+    """hla_forward on the scratch array the library itself carries (no workspace tensor, nothing allocated).
+    Returns that array's device address (an int), usable as `workspace` for hla_last_device_status."""
+    scratch = c_void_p()
+    st = load_library().hla_forward_static(ctx, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _stream(stream), byref(scratch))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_forward_static")
+    return scratch.value
 
 
 def hla_last_device_status(ctx: int, workspace, stream=None) -> int:

@@ -2,6 +2,7 @@
 // launch sequences of forward and backward.  See include/hla.h for the contract.
 #include "../../include/hla.h"
 
+#include <mutex>
 #include <new>
 #include <string.h>
 
@@ -345,6 +346,51 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     }
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
+}
+
+// ---- forward on the library's own scratch array ---------------------------------------------
+// The scratch of hla_forward_static.  In host code `g_static_ws` only names the symbol: it is not a
+// device address, and a kernel handed it would read the wrong memory.  The address each device has
+// for it is looked up once per device with cudaGetSymbolAddress and cached below.
+static __device__ __align__(256) unsigned char g_static_ws[HLA_STATIC_WS_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_ws_addr[kMaxDevices] = {};
+std::mutex g_static_ws_mutex;
+
+// Device address of g_static_ws on the current device (looked up on the first call per device).
+hla_status static_ws_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return HLA_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+    if (!g_static_ws_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return HLA_ERR_CUDA;
+        }
+        g_static_ws_addr[dev] = p;
+    }
+    *out = g_static_ws_addr[dev];
+    return HLA_OK;
+}
+}  // namespace
+
+hla_status hla_forward_static(hla_ctx* ctx, const void* Q, const void* K, const void* V, void* O, void* cuda_stream, void** scratch_out) {
+    if (scratch_out) *scratch_out = nullptr;
+    if (!ctx) return HLA_ERR_INVALID_ARG;
+    if (ctx->ws_bytes > (size_t)HLA_STATIC_WS_BYTES) return HLA_ERR_WORKSPACE;    // this shape needs more scratch than the library carries
+    void* ws = nullptr;
+    const hla_status s = static_ws_address(&ws);
+    if (s != HLA_OK) return s;
+    if (scratch_out) *scratch_out = ws;
+    // hla_forward clears the status words and writes every other region before reading it, so nothing
+    // left by an earlier call is used.
+    return hla_forward(ctx, Q, K, V, O, ws, (size_t)HLA_STATIC_WS_BYTES, cuda_stream);
 }
 
 hla_status hla_last_device_status(hla_ctx* ctx, const void* workspace, void* cuda_stream) {
