@@ -237,7 +237,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     D.B = c.B; D.H = c.H; D.N = c.N; D.d = c.d; D.F = c.F; D.dphi = c.d_phi; D.P = P;
     D.ld = c.d + 4;
     D.eps = c.eps;
-    x->tc = tc::supported(c.dtype == HLA_BF16, c.d, c.F, c.d_phi);
+    x->tc = tc::supported(c.dtype == HLA_BF16, c.d, c.F, c.d_phi) && (long long)c.B * c.H * c.N < (1ll << 31);   // the tensor-core kernels index tokens in 32 bits
     const int tile = x->tc ? tc::kTileTokens : simt::kTok;
     const int tiles = (c.N + tile - 1) / tile;
     int S = c.n_splits;

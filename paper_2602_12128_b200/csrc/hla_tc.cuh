@@ -310,17 +310,21 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
         float zacc[kMono];
 #pragma unroll
         for (int i = 0; i < kMono; ++i) zacc[i] = 0.f;
-        float k[18];
+        // The key features of the group's next tile are loaded while the current one is processed (row index clamped:
+        // the loads are unconditional, out-of-range rows are zeroed when used).
+        float k[18], kn[18];
+        auto prefetch = [&](int it) {
+            const int tok = min((tile0 + it) * kTileTokens + row, N - 1);
+#pragma unroll
+            for (int f = 0; f < 3; ++f) load6(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+        };
+        if (grp < ntiles) prefetch(grp);
         for (int it = grp; it < ntiles; it += 2) {
             const int st = it % kSbStages, u = it / kSbStages;
             const int tok = (tile0 + it) * kTileTokens + row;
-            if (tok < N) {
 #pragma unroll
-                for (int f = 0; f < 3; ++f) load6(k + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 18; ++i) k[i] = 0.f;
-            }
+            for (int i = 0; i < 18; ++i) k[i] = tok < N ? kn[i] : 0.f;
+            if (it + 2 < ntiles) prefetch(it + 2);
             float ts[kMono];
             key_folded(k, ts);
 #pragma unroll
@@ -501,15 +505,19 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
         }
     } else if (warp >= 4) {
         const int row = tid - 128;
+        float qn[6];      // query features of the next tile, loaded one tile ahead (row index clamped)
+        auto prefetch = [&](int it) {
+            const int work = w0 + it, bh = work / tiles_per_head, tok = min((work % tiles_per_head) * kTileTokens + row, N - 1);
+            load6(qn, qf + ((size_t)bh * N + tok) * 6);
+        };
+        if (nwork > 0) prefetch(0);
         for (int it = 0; it < nwork; ++it) {
-            const int work = w0 + it, bh = work / tiles_per_head, tok = (work % tiles_per_head) * kTileTokens + row;
+            const int work = w0 + it, tok = (work % tiles_per_head) * kTileTokens + row;
             const int ab = it & 1, u = it >> 1;
             float q[6];
-            if (tok < N) load6(q, qf + ((size_t)bh * N + tok) * 6);
-            else {
 #pragma unroll
-                for (int i = 0; i < 6; ++i) q[i] = 0.f;
-            }
+            for (int i = 0; i < 6; ++i) q[i] = tok < N ? qn[i] : 0.f;
+            if (it + 1 < nwork) prefetch(it + 1);
             float mono[kMono];
             query_monomials(q, mono);
             if (ok && !mbar_wait(&a_empty[ab], (u & 1) ^ 1)) { ok = false; report_timeout(status, 204); }
@@ -667,18 +675,26 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             const uint32_t opa = smem_u32(smem + kBqOffOp);
             bool good = mbar_wait(op_full, 0);
             if (!good) report_timeout(status, 302);
-            for (int it = 0; it < ntiles && good; ++it) {
+            // D2 of tile `it`; issued one tile ahead of the tile's dC product so that the generators never wait for it
+            auto issue_d2 = [&](int it) -> bool {
                 const int st = it % kBqStages, u = it / kBqStages, buf = it & 1, ub = it >> 1;
-                if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&d2_empty[buf], (ub & 1) ^ 1))) { report_timeout(status, 303); break; }
+                if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&d2_empty[buf], (ub & 1) ^ 1))) return false;
                 tc_fence_after();
-                const uint32_t da = smem_u32(smem + st * kBqStageBytes), ra = da + 2 * kBlk;
+                const uint32_t da = smem_u32(smem + st * kBqStageBytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 64 + 64 * buf, smem_desc_sw128(da + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
                               smem_desc_sw128(opa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
                 umma_commit(&d2_full[buf]);
+                return true;
+            };
+            if (good && !issue_d2(0)) { good = false; report_timeout(status, 303); }
+            for (int it = 0; it < ntiles && good; ++it) {
+                const int st = it % kBqStages, u = it / kBqStages;
+                if (it + 1 < ntiles && !issue_d2(it + 1)) { report_timeout(status, 303); break; }
                 if (!mbar_wait(&full_rm[st], u & 1)) { report_timeout(status, 304); break; }
                 tc_fence_after();
+                const uint32_t da = smem_u32(smem + st * kBqStageBytes), ra = da + 2 * kBlk;
 #pragma unroll
                 for (int ks = 0; ks < kTileTokens / 16; ++ks)
                     umma_bf16(tmem, smem_desc_sw128(da + ks * 2048, kBlk, 1024), smem_desc_sw128(ra + ks * 2048, kBlk, 1024), idesc1,
@@ -693,17 +709,23 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
         float dzacc[kMono];
 #pragma unroll
         for (int i = 0; i < kMono; ++i) dzacc[i] = 0.f;
+        // The features and the normaliser of the group's next tile are loaded while the current one is processed
+        // (row index clamped: the loads are unconditional, out-of-range rows are zeroed when used).
+        float qn[6], etan;
+        auto prefetch = [&](int it) {
+            const int tok = min((tile0 + it) * kTileTokens + row, N - 1);
+            load6(qn, qf + ((size_t)bh * N + tok) * 6);
+            etan = __ldg(eta + (size_t)bh * N + tok);
+        };
+        if (grp < ntiles) prefetch(grp);
         for (int it = grp; it < ntiles; it += 2) {
             const int st = it % kBqStages, u = it / kBqStages, buf = it & 1, ub = it >> 1;
             const int tok = (tile0 + it) * kTileTokens + row;
             float q[6], r = 0.f;
-            if (tok < N) {
-                load6(q, qf + ((size_t)bh * N + tok) * 6);
-                r = 1.f / (__ldg(eta + (size_t)bh * N + tok) + eps);
-            } else {
 #pragma unroll
-                for (int i = 0; i < 6; ++i) q[i] = 0.f;
-            }
+            for (int i = 0; i < 6; ++i) q[i] = tok < N ? qn[i] : 0.f;
+            if (tok < N) r = 1.f / (etan + eps);
+            if (it + 2 < ntiles) prefetch(it + 2);
             float mono[kMono];
             query_monomials(q, mono);
             if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
@@ -716,26 +738,21 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) continue;
             tc_fence_after();
-            float d2[kMono];
+            uint32_t d2[kMono];
             const uint32_t ta = tmem + 64 + 64 * buf + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
-            for (int c = 0; c < kMono / 8; ++c) {
-                uint32_t rr[8];
-                tmem_ld8(ta + 8 * c, rr);
-                tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 8; ++e) d2[8 * c + e] = __uint_as_float(rr[e]);
-            }
+            for (int c = 0; c < kMono / 8; ++c) tmem_ld8(ta + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(d2 + 8 * c));
+            tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(&d2_empty[buf]);
             float sdot = 0.f;
 #pragma unroll
-            for (int m = 0; m < kMono; ++m) sdot = fmaf(mono[m], d2[m], sdot);
+            for (int m = 0; m < kMono; ++m) sdot = fmaf(mono[m], __uint_as_float(d2[m]), sdot);
             const float deta = -r * r * sdot;
             float dm[kMono];
 #pragma unroll
             for (int m = 0; m < kMono; ++m) {
-                dm[m] = fmaf(r, d2[m], deta * zsym[m]);
+                dm[m] = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);
                 dzacc[m] = fmaf(mono[m], deta, dzacc[m]);
             }
             float dq[6];
@@ -905,18 +922,21 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const bool leader = (warp - 2) == 4 * grp && lane == 0;
+        float kn[18];     // key features of the group's next tile, loaded one tile ahead (row index clamped)
+        auto prefetch = [&](int it) {
+            const int work = w0 + it, bh = work / tiles_per_head, tok = min((work % tiles_per_head) * kTileTokens + row, N - 1);
+#pragma unroll
+            for (int f = 0; f < 3; ++f) load6(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+        };
+        if (grp < nwork) prefetch(grp);
         for (int it = grp; it < nwork; it += 2) {
             const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
             const int u = it >> 1;
             const int tok = tile * kTileTokens + row;
             float k[18];
-            if (tok < N) {
 #pragma unroll
-                for (int f = 0; f < 3; ++f) load6(k + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 18; ++i) k[i] = 0.f;
-            }
+            for (int i = 0; i < 18; ++i) k[i] = tok < N ? kn[i] : 0.f;
+            if (it + 2 < nwork) prefetch(it + 2);
             {
                 float ts[kMono];
                 key_folded(k, ts);
@@ -933,14 +953,12 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                 float G[kMono];
                 const uint32_t ta = tmem + 256 + 64 * grp + ((uint32_t)(quarter * 32) << 16);
                 const float* dz = dstate + (size_t)bh * kMono * ld + DV;
+                uint32_t gr[kMono];
 #pragma unroll
-                for (int c = 0; c < kMono / 8; ++c) {
-                    uint32_t rr[8];
-                    tmem_ld8(ta + 8 * c, rr);
-                    tmem_ld_wait();
+                for (int c = 0; c < kMono / 8; ++c) tmem_ld8(ta + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(gr + 8 * c));
+                tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) G[8 * c + e] = __uint_as_float(rr[e]) + __ldg(dz + (size_t)(8 * c + e) * ld);
-                }
+                for (int m = 0; m < kMono; ++m) G[m] = __uint_as_float(gr[m]) + __ldg(dz + (size_t)m * ld);
                 float dk[18];
                 key_folded_grad(k, G, dk);
                 if (tok < N) {

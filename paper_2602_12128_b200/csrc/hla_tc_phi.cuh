@@ -223,8 +223,8 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
 #pragma unroll
                 for (int o = 0; o < 6; ++o) f[o] = fmaxf(__uint_as_float(r[o]) + b2s[o], 0.f);
                 if (KSIDE) {
-                    const long long bh = grow / N, n = grow - bh * N;
-                    store6(feat + ((bh * NMAPS + m) * N + n) * 6, f);
+                    const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
+                    store6(feat + ((size_t)(bh * NMAPS + m) * N + n) * 6, f);
                 } else {
                     store6(feat + grow * 6, f);
                 }
@@ -447,8 +447,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                     grow = grow < rows ? grow : rows - 1;
                     size_t off;
                     if (KSIDE) {
-                        const long long bh = grow / N, n = grow - bh * N;
-                        off = (size_t)((bh * NMAPS + m) * N + n) * 6;
+                        const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
+                        off = ((size_t)(bh * NMAPS + m) * N + n) * 6;
                     } else {
                         off = (size_t)grow * 6;
                     }
