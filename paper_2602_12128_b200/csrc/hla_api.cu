@@ -242,8 +242,20 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     const int tiles = (c.N + tile - 1) / tile;
     int S = c.n_splits;
     if (S == 0) {
-        const int target = x->tc ? x->sm_count : 2 * x->sm_count;
-        S = (target + x->BH - 1) / x->BH;
+        if (x->tc) {
+            // One CTA per SM: S * heads CTAs run in ceil(S * heads / SMs) waves.  Take the split count that fills its
+            // waves best (each extra wave is charged 2 % for its start-up and drain), with at least 8 tiles per CTA.
+            const int smax = tiles / 8 > 1 ? (tiles / 8 < 64 ? tiles / 8 : 64) : 1;
+            double best = -1.0;
+            for (int cand = 1; cand <= smax; ++cand) {
+                const long long ctas = (long long)cand * x->BH;
+                const long long waves = (ctas + x->sm_count - 1) / x->sm_count;
+                const double score = (double)ctas / (double)(waves * x->sm_count) - 0.02 * (double)(waves - 1);
+                if (score > best + 1e-9) { best = score; S = cand; }
+            }
+        } else {
+            S = (2 * x->sm_count + x->BH - 1) / x->BH;
+        }
     }
     if (S > tiles) S = tiles;
     if (S < 1) S = 1;

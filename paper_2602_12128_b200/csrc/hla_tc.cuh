@@ -726,13 +726,24 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             for (int i = 0; i < 6; ++i) q[i] = tok < N ? qn[i] : 0.f;
             if (tok < N) r = 1.f / (etan + eps);
             if (it + 2 < ntiles) prefetch(it + 2);
-            float mono[kMono];
-            query_monomials(q, mono);
-            if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
-            if (ok) {
-                store_mono_row(smem_u32(smem + st * kBqStageBytes + 2 * kBlk), row, mono, r);
-                fence_proxy_async();
-                mbar_arrive(&full_rm[st]);
+            {   // operand row r_i * mono_i; formed from (r q_a) q_b q_c so that no monomial stays live across the wait below
+                float qs[6], rmono[kMono];
+#pragma unroll
+                for (int i = 0; i < 6; ++i) qs[i] = r * q[i];
+#pragma unroll
+                for (int a = 0; a < 6; ++a)
+#pragma unroll
+                    for (int b = a; b < 6; ++b) {
+                        const float qab = qs[a] * q[b];
+#pragma unroll
+                        for (int c = b; c < 6; ++c) rmono[mono_idx(a, b, c)] = qab * q[c];
+                    }
+                if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
+                if (ok) {
+                    store_mono_row(smem_u32(smem + st * kBqStageBytes + 2 * kBlk), row, rmono, 1.f);
+                    fence_proxy_async();
+                    mbar_arrive(&full_rm[st]);
+                }
             }
             if (ok && !mbar_wait(&d2_full[buf], ub & 1)) { ok = false; report_timeout(status, 306); }
             ok = __all_sync(0xffffffffu, ok);
@@ -745,18 +756,38 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(&d2_empty[buf]);
-            float sdot = 0.f;
+            // The monomials are recomputed where they are used (two multiplies each) instead of being kept in 56 registers.
+            float qq[6][6];
 #pragma unroll
-            for (int m = 0; m < kMono; ++m) sdot = fmaf(mono[m], __uint_as_float(d2[m]), sdot);
+            for (int a = 0; a < 6; ++a)
+#pragma unroll
+                for (int b = a; b < 6; ++b) qq[a][b] = q[a] * q[b];
+            float sd[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int a = 0; a < 6; ++a)
+#pragma unroll
+                for (int b = a; b < 6; ++b)
+#pragma unroll
+                    for (int c = b; c < 6; ++c) {
+                        const int m = mono_idx(a, b, c);
+                        sd[m & 3] = fmaf(qq[a][b] * q[c], __uint_as_float(d2[m]), sd[m & 3]);
+                    }
+            const float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
             const float deta = -r * r * sdot;
-            float dm[kMono];
+            float dq[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int m = 0; m < kMono; ++m) {
-                dm[m] = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);
-                dzacc[m] = fmaf(mono[m], deta, dzacc[m]);
-            }
-            float dq[6];
-            query_monomials_grad(q, dm, dq);
+            for (int a = 0; a < 6; ++a)
+#pragma unroll
+                for (int b = a; b < 6; ++b)
+#pragma unroll
+                    for (int c = b; c < 6; ++c) {
+                        const int m = mono_idx(a, b, c);
+                        const float g = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);      // dmono_i[m]
+                        dzacc[m] = fmaf(q[a] * qq[b][c], deta, dzacc[m]);
+                        dq[a] = fmaf(g, qq[b][c], dq[a]);
+                        dq[b] = fmaf(g, qq[a][c], dq[b]);
+                        dq[c] = fmaf(g, qq[a][b], dq[c]);
+                    }
             if (tok < N) store6(dqf + ((size_t)bh * N + tok) * 6, dq);
         }
 #pragma unroll
@@ -953,12 +984,14 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                 float G[kMono];
                 const uint32_t ta = tmem + 256 + 64 * grp + ((uint32_t)(quarter * 32) << 16);
                 const float* dz = dstate + (size_t)bh * kMono * ld + DV;
-                uint32_t gr[kMono];
 #pragma unroll
-                for (int c = 0; c < kMono / 8; ++c) tmem_ld8(ta + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(gr + 8 * c));
-                tmem_ld_wait();
+                for (int c = 0; c < kMono / 8; ++c) {
+                    uint32_t rr[8];
+                    tmem_ld8(ta + 8 * c, rr);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int m = 0; m < kMono; ++m) G[m] = __uint_as_float(gr[m]) + __ldg(dz + (size_t)m * ld);
+                    for (int e = 0; e < 8; ++e) G[8 * c + e] = __uint_as_float(rr[e]) + __ldg(dz + (size_t)(8 * c + e) * ld);
+                }
                 float dk[18];
                 key_folded_grad(k, G, dk);
                 if (tok < N) {
