@@ -413,7 +413,10 @@ __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __rest
 // =======================================================================================
 // Readout + normaliser
 // =======================================================================================
-constexpr int kRoThreads = 288;   // warps 0..3: epilogue, warps 4..7: monomial generators, warp 8: TMA + MMA
+// warps 0..7: epilogue (thread = token row x half of the value channels; one warp per scheduler could not keep up with
+// the tile rate), warps 8..11: monomial generators, warp 12: TMA + MMA
+constexpr int kRoThreads = 416;
+constexpr int kRoGenWarp0 = 8, kRoMmaWarp = 12;
 template <int DV> struct RoCfg {
     static constexpr int kNmma = DV + 16;
     static constexpr int kB3Bytes = kNmma * 128;
@@ -437,7 +440,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
     uint64_t* a_full = bars;          // [2] 128 generator arrivals
     uint64_t* a_empty = bars + 2;     // [2] MMA commit
     uint64_t* acc_full = bars + 4;    // [2] MMA commit
-    uint64_t* acc_empty = bars + 6;   // [2] 128 epilogue arrivals
+    uint64_t* acc_empty = bars + 6;   // [2] 256 epilogue arrivals
     uint64_t* b3_full = bars + 8;
     uint64_t* b3_free = bars + 9;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
@@ -454,7 +457,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
             mbar_init(&a_full[i], 128);
             mbar_init(&a_empty[i], 1);
             mbar_init(&acc_full[i], 1);
-            mbar_init(&acc_empty[i], 128);
+            mbar_init(&acc_empty[i], 256);
         }
         mbar_init(b3_full, 1);
         mbar_init(b3_free, 1);
@@ -463,7 +466,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
         prefetch_tmap(&mapB3);
         prefetch_tmap(&mapO);
     }
-    if (warp == 8) {
+    if (warp == kRoMmaWarp) {
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
@@ -473,7 +476,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
     const uint32_t tmem = *tmem_slot;
     bool ok = true;
 
-    if (warp == 8) {
+    if (warp == kRoMmaWarp) {
         if (lane == 0) {
             const uint32_t idesc = idesc_bf16(128, Cfg::kNmma, false, false);
             const uint32_t b3a = smem_u32(smem + Cfg::kOffB3);
@@ -503,8 +506,8 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
                 umma_commit(&acc_full[ab]);
             }
         }
-    } else if (warp >= 4) {
-        const int row = tid - 128;
+    } else if (warp >= kRoGenWarp0) {
+        const int row = tid - kRoGenWarp0 * 32;
         float qn[6];      // query features of the next tile, loaded one tile ahead (row index clamped)
         auto prefetch = [&](int it) {
             const int work = w0 + it, bh = work / tiles_per_head, tok = min((work % tiles_per_head) * kTileTokens + row, N - 1);
@@ -527,7 +530,8 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
             mbar_arrive(&a_full[ab]);
         }
     } else {
-        const int row = tid;   // TMEM lane = token row of the tile
+        const int row = tid & 127, half = tid >> 7;   // TMEM lane = token row of the tile; columns half * DV/2 ...
+        constexpr int HC = DV / 2;
         for (int it = 0; it < nwork; ++it) {
             const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
             const int ab = it & 1, u = it >> 1;
@@ -536,43 +540,45 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
                 *abort_flag = 1;
             }
             if (tid == 0) tma_store_wait_read1();      // the staging tile of two tiles ago has been read by its store
-            named_barrier(3, 128);                     // every epilogue thread arrives, timed out or not
-            if (*abort_flag) break;                    // uniform across the four warps
+            named_barrier(3, 256);                     // every epilogue thread arrives, timed out or not
+            if (*abort_flag) break;                    // uniform across the eight warps
             tc_fence_after();
-            const uint32_t ta = tmem + ab * 256 + ((uint32_t)(warp * 32) << 16);
-            uint32_t r[16];
-            tmem_ld16(ta + DV, r);
+            const uint32_t ta = tmem + ab * 256 + ((uint32_t)((warp & 3) * 32) << 16);
+            // the whole accumulator row (numerator and normaliser) in one batch of TMEM loads, then the buffer is released
+            uint32_t re[8], r[HC];
+            tmem_ld8(ta + DV, re);
+#pragma unroll
+            for (int c = 0; c < HC / 16; ++c) tmem_ld16(ta + half * HC + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
             tmem_ld_wait();
-            const float eta = __uint_as_float(r[0]);
+            tc_fence_before();
+            mbar_arrive(&acc_empty[ab]);
+            const float eta = __uint_as_float(re[0]);
             const float rinv = 1.f / (eta + eps);
             const uint32_t os = smem_u32(smem + Cfg::kOffO + ab * Cfg::kOBytes);
 #pragma unroll
-            for (int c = 0; c < DV / 16; ++c) {
-                tmem_ld16(ta + 16 * c, r);
-                tmem_ld_wait();
+            for (int c = 0; c < HC / 16; ++c) {
                 uint32_t w[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]) * rinv, __uint_as_float(r[2 * e + 1]) * rinv);
-                const uint32_t blk = os + (c >> 2) * kBlk;
-                st_shared_v4(blk + sw128_off(row, (2 * c) & 7), w[0], w[1], w[2], w[3]);
-                st_shared_v4(blk + sw128_off(row, (2 * c + 1) & 7), w[4], w[5], w[6], w[7]);
+                for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[16 * c + 2 * e]) * rinv, __uint_as_float(r[16 * c + 2 * e + 1]) * rinv);
+                const int cc = half * (HC / 16) + c;      // 16-column chunk of the row
+                const uint32_t blk = os + (cc >> 2) * kBlk;
+                st_shared_v4(blk + sw128_off(row, (2 * cc) & 7), w[0], w[1], w[2], w[3]);
+                st_shared_v4(blk + sw128_off(row, (2 * cc + 1) & 7), w[4], w[5], w[6], w[7]);
             }
-            tc_fence_before();
-            mbar_arrive(&acc_empty[ab]);
             fence_proxy_async();
-            named_barrier(2, 128);
+            named_barrier(2, 256);
             if (tid == 0) {
                 for (int b = 0; b < DV / 64; ++b) tma_store_3d(&mapO, smem + Cfg::kOffO + ab * Cfg::kOBytes + b * kBlk, b * 64, tile * kTileTokens, bh);
                 tma_store_commit();
             }
             const int tok = tile * kTileTokens + row;
-            if (tok < N) eta_out[(size_t)bh * N + tok] = eta;
+            if (half == 0 && tok < N) eta_out[(size_t)bh * N + tok] = eta;
         }
         if (tid == 0) tma_store_wait_all0();
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) tmem_dealloc(tmem, 512);
+    if (warp == kRoMmaWarp) tmem_dealloc(tmem, 512);
 }
 
 // =======================================================================================
@@ -1009,16 +1015,20 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                 const uint32_t ta = tmem + 128 * grp + ((uint32_t)(quarter * 32) << 16);
                 const uint32_t os = smem_u32(smem + Cfg::kOffO + grp * Cfg::kOBytes);
 #pragma unroll
-                for (int c = 0; c < DV / 16; ++c) {
-                    uint32_t r[16];
-                    tmem_ld16(ta + 16 * c, r);
-                    tmem_ld_wait();
-                    uint32_t w[8];
+                for (int h = 0; h < DV / 64; ++h) {      // 64 columns per batch of TMEM loads
+                    uint32_t r[64];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                    const uint32_t blk = os + (c >> 2) * kBlk;
-                    st_shared_v4(blk + sw128_off(row, (2 * c) & 7), w[0], w[1], w[2], w[3]);
-                    st_shared_v4(blk + sw128_off(row, (2 * c + 1) & 7), w[4], w[5], w[6], w[7]);
+                    for (int c = 0; c < 4; ++c) tmem_ld16(ta + 64 * h + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1]));
+                        const uint32_t blk = os + h * kBlk;
+                        st_shared_v4(blk + sw128_off(row, 2 * c), w[0], w[1], w[2], w[3]);
+                        st_shared_v4(blk + sw128_off(row, 2 * c + 1), w[4], w[5], w[6], w[7]);
+                    }
                 }
                 tc_fence_before();
                 mbar_arrive(&acc_empty[grp]);
