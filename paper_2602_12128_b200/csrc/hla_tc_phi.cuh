@@ -583,10 +583,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                if (grow < rows) {
-                    dst[2 * c] = make_uint4(w[0], w[1], w[2], w[3]);
-                    dst[2 * c + 1] = make_uint4(w[4], w[5], w[6], w[7]);
-                }
+                if (grow < rows) st_global_v8(dst + 2 * c, w);      // one full 32-byte sector per store
             }
             tc_fence_before();
             mbar_arrive(dx_empty);
