@@ -327,7 +327,7 @@ struct PhiBwdPtrs {
     const __nv_bfloat16* W2[3];
 };
 
-// warp 0: TMA loads and dp tiles, warp 1: dg and dX MMAs, warp 2: h MMAs, warps 3..18: epilogue (thread = token row x quarter of the columns)
+// warp 0: TMA loads, warp 1: dg and dX MMAs, warp 2: h MMAs, warps 3..18: epilogue (thread = token row x quarter of the columns)
 constexpr int kPbThreads = 608;
 constexpr int kPbEpiWarp0 = 3;
 
@@ -354,7 +354,7 @@ template <int DV, int NMAPS> struct PbCfg {
 //   dX += dh * W1^T                     [128 x DV], K = DV,  dh = dg (.) GELU'(h + b1) formed by the 16 epilogue warps
 // h and the dh tile are double-buffered; dg is taken into registers at the start of a unit so that the next unit's dg
 // product overlaps this unit's arithmetic; the dX accumulator of a tile is drained one unit late, straight from
-// registers to global memory.  Warp 0 issues the TMA loads and writes the dp tiles up to four units ahead.
+// registers to global memory.  The epilogue threads also write the dp tiles (one feature pair each, one unit ahead).
 template <int DV, int NMAPS, bool KSIDE>
 __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
                                                                         PhiBwdPtrs P, const float* __restrict__ feat, const float* __restrict__ dfeat,
@@ -372,8 +372,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* h_empty = bars + 6;      // [2] 512 arrivals
     uint64_t* dh_full = bars + 8;      // [2] 512 arrivals
     uint64_t* dh_free = bars + 10;     // [2] MMA commit
-    uint64_t* dp_full = bars + 12;     // [4] 32 arrivals (warp 0)
-    uint64_t* dp_free = bars + 16;     // [4] MMA commit
+    uint64_t* dp_full = bars + 12;     // [2] 512 arrivals
     uint64_t* dg_full = bars + 20;     // MMA commit
     uint64_t* dg_empty = bars + 21;    // 512 arrivals
     uint64_t* dx_full = bars + 22;     // MMA commit
@@ -405,10 +404,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             mbar_init(&dh_full[i], 512);
             mbar_init(&dh_free[i], 1);
         }
-        for (int i = 0; i < 4; ++i) {
-            mbar_init(&dp_full[i], 32);
-            mbar_init(&dp_free[i], 1);
-        }
+        for (int i = 0; i < 2; ++i) mbar_init(&dp_full[i], 512);
         mbar_init(dg_full, 1);
         mbar_init(dg_empty, 512);
         mbar_init(dx_full, 1);
@@ -428,81 +424,17 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     bool ok = true;
 
     if (warp == 0) {
-        if (ntiles > 0) {
-            if (lane == 0) {
-                mbar_arrive_expect_tx(w_full, NMAPS * Cfg::kW1Bytes);
-                for (int m = 0; m < NMAPS; ++m)
-                    for (int b = 0; b < DV / 64; ++b)
-                        tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
-            }
-            const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
-            // Features and feature gradients of rows lane, lane + 32, lane + 64, lane + 96 of a unit.  The loads are
-            // unconditional (row index clamped) and issued one unit ahead, so their latency never sits on the unit's path.
-            float fr[4][6], gr[4][6];
-            auto load_rows = [&](int unit) {
-                const int it = unit / NMAPS, m = unit % NMAPS;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    long long grow = (t0 + it) * kTileTokens + lane + 32 * i;
-                    grow = grow < rows ? grow : rows - 1;
-                    size_t off;
-                    if (KSIDE) {
-                        const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
-                        off = ((size_t)(bh * NMAPS + m) * N + n) * 6;
-                    } else {
-                        off = (size_t)grow * 6;
-                    }
-                    load6(fr[i], feat + off);
-                    load6(gr[i], dfeat + off);
-                }
-            };
-            load_rows(0);
-            for (int unit = 0; unit < nunits; ++unit) {
-                const int it = unit / NMAPS, m = unit % NMAPS, slot = unit & 3;
-                if (m == 0) {      // this tile's X
-                    if (lane == 0) {
-                        const int st = it % XST, u = it / XST;
-                        ok = mbar_wait(&x_empty[st], (u & 1) ^ 1);
-                        if (ok) {
-                            mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
-                            for (int b = 0; b < DV / 64; ++b)
-                                tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
-                        } else {
-                            report_timeout(status, 601);
-                        }
-                    }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) break;
-                }
-                uint32_t w[4][6];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const bool live = (t0 + it) * kTileTokens + lane + 32 * i < rows;
-                    float dp[6], lo[6];
-#pragma unroll
-                    for (int o = 0; o < 6; ++o) {
-                        dp[o] = (live && fr[i][o] > 0.f) ? gr[i][o] : 0.f;
-                        lo[o] = dp[o] - __bfloat162float(__float2bfloat16_rn(dp[o]));
-                    }
-                    w[i][0] = pack_bf16(dp[0], dp[1]);
-                    w[i][1] = pack_bf16(dp[2], dp[3]);
-                    w[i][2] = pack_bf16(dp[4], dp[5]);
-                    w[i][3] = pack_bf16(lo[0], lo[1]);
-                    w[i][4] = pack_bf16(lo[2], lo[3]);
-                    w[i][5] = pack_bf16(lo[4], lo[5]);
-                }
-                if (unit + 1 < nunits) load_rows(unit + 1);
-                if (!mbar_wait(&dp_free[slot], ((unit >> 2) & 1) ^ 1)) { ok = false; report_timeout(status, 607); }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t r = lane + 32 * i;
-                    st_shared_v4(dpblk + sw128_off(r, 2 * slot), w[i][0], w[i][1], w[i][2], w[i][3]);
-                    st_shared_v4(dpblk + sw128_off(r, 2 * slot + 1), w[i][4], w[i][5], 0u, 0u);
-                }
-                fence_proxy_async();
-                mbar_arrive(&dp_full[slot]);
+        if (lane == 0 && ntiles > 0) {
+            mbar_arrive_expect_tx(w_full, NMAPS * Cfg::kW1Bytes);
+            for (int m = 0; m < NMAPS; ++m)
+                for (int b = 0; b < DV / 64; ++b)
+                    tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
+            for (int it = 0; it < ntiles; ++it) {
+                const int st = it % XST, u = it / XST;
+                if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 601); break; }
+                mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
+                for (int b = 0; b < DV / 64; ++b)
+                    tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
             }
         }
     } else if (warp == 2) {
@@ -536,13 +468,12 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             bool good = mbar_wait(w_full, 0);
             // dg of `unit`; the epilogue of unit - 1 must have taken its dg into registers
             auto issue_dg = [&](int unit) -> bool {
-                const int m = unit % NMAPS, slot = unit & 3;
+                const int m = unit % NMAPS, slot = unit & 1;
                 if (unit > 0 && !mbar_wait(dg_empty, (unit - 1) & 1)) return false;
-                if (!mbar_wait(&dp_full[slot], (unit >> 2) & 1)) return false;
+                if (!mbar_wait(&dp_full[slot], (unit >> 1) & 1)) return false;
                 tc_fence_after();
                 umma_bf16(tmem + 256, desc_advance(pd0, slot * 32), desc_advance(vd0, m * Cfg::kW2tBytes), idesc_dg, 0u);
                 umma_commit(dg_full);
-                umma_commit(&dp_free[slot]);
                 return true;
             };
             if (good && nunits > 0) good = issue_dg(0);
@@ -588,8 +519,54 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             tc_fence_before();
             mbar_arrive(dx_empty);
         };
+        // dp = dfeat (.) 1[feat > 0] as the A operand [dp_hi | dp_lo] of the dg product.  Every epilogue thread of parts
+        // 0..2 owns one pair of features of its row: it loads them two units ahead (row index clamped, the loads are
+        // unconditional) and writes the tile of unit u + 1 at the start of unit u, so no single warp carries this work.
+        // Slot (u + 1) & 1 is free then: its last reader, the dg product of unit u - 1, completed before unit u - 1's
+        // dg was read.
+        const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
+        float2 fpre = make_float2(0.f, 0.f), gpre = make_float2(0.f, 0.f);
+        bool live_pre = false;
+        int off_it = -1;          // tile whose row offset is cached in off_tile (the offset of map 0)
+        size_t off_tile = 0;
+        auto dp_load = [&](int unit) {
+            if (part == 3 || unit >= nunits) return;
+            const int it = unit / NMAPS, m = unit % NMAPS;
+            if (it != off_it) {
+                long long grow = (t0 + it) * kTileTokens + row;
+                live_pre = grow < rows;
+                grow = live_pre ? grow : rows - 1;
+                if (KSIDE) {
+                    const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
+                    off_tile = ((size_t)bh * NMAPS * N + n) * 6;
+                } else {
+                    off_tile = (size_t)grow * 6;
+                }
+                off_it = it;
+            }
+            const size_t off = off_tile + (KSIDE ? (size_t)m * N * 6 : 0);
+            fpre = __ldg(reinterpret_cast<const float2*>(feat + off) + part);
+            gpre = __ldg(reinterpret_cast<const float2*>(dfeat + off) + part);
+        };
+        auto dp_store = [&](int unit) {      // the pair loaded by the last dp_load goes into the tile of `unit`
+            if (unit >= nunits) return;
+            if (part < 3) {
+                const float d0 = (live_pre && fpre.x > 0.f) ? gpre.x : 0.f, d1 = (live_pre && fpre.y > 0.f) ? gpre.y : 0.f;
+                const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
+                const uint32_t slot = unit & 1, khi = 2 * part, klo = 6 + 2 * part;      // K indices of the pair: hi half, lo half
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(dpblk + sw128_off(row, 2 * slot + (khi >> 3)) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(dpblk + sw128_off(row, 2 * slot + (klo >> 3)) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
+            }
+            fence_proxy_async();
+            mbar_arrive(&dp_full[unit & 1]);
+        };
+        dp_load(0);
+        dp_store(0);
+        dp_load(1);
         for (int unit = 0; unit < nunits && ok; ++unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
+            dp_store(unit + 1);
+            dp_load(unit + 2);
             if (!mbar_wait(dg_full, unit & 1)) { ok = false; report_timeout(status, 608); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
