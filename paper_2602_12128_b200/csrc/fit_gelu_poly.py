@@ -7,7 +7,11 @@ GELU(x) = x Phi(x);  GELU'(x) = Phi(x) + x exp(-x^2 / 2) / sqrt(2 pi).
 
 Run:  python fit_gelu_poly.py   -> prints the coefficients (highest order first, as the Horner
 evaluation in hla_tc_phi.cuh lists them) and the maximum absolute errors of Phi and GELU in fp32.
-The constants in hla_tc_phi.cuh are this script's output for T = 16, NCOEF = 7."""
+The constants in hla_tc_phi.cuh are this script's output for T = 16, NCOEF = 7 (used by the backward's GELU').
+
+The forward evaluates Phi(x) ~ 1/2 + tanh(x (a + b x^2)) / 2 instead (one tanh.approx on the special-function
+unit); fit_tanh() gives a, b (fitted against erf(x / sqrt 2) on |x| <= 6) and the error before the hardware
+approximation's own 2^-11 relative error."""
 import numpy as np
 from scipy.special import erf
 
@@ -39,7 +43,23 @@ def phi_f32(x, coef, T=T):
     return np.clip(x * p + np.float32(0.5), 0, 1).astype(np.float32)
 
 
+def fit_tanh(iters=60):
+    from scipy.optimize import least_squares
+    x = np.linspace(0, 6, 6001)[1:]
+    ref = erf(x / np.sqrt(2))
+    res = lambda c: np.tanh(x * (c[0] + c[1] * x * x)) - ref
+    c, w = np.array([0.7978845608, 0.0356774]), np.ones_like(x)
+    for _ in range(iters):                      # reweighted least squares towards the minimax fit
+        c = least_squares(lambda c: res(c) * w, c).x
+        e = np.abs(res(c))
+        w *= 1 + 2 * e / e.max()
+        w /= w.mean()
+    return c, np.abs(res(c)).max() / 2
+
+
 if __name__ == "__main__":
+    (a, b), err = fit_tanh()
+    print("tanh form: a = %.8ff, b = %.8ff, max |Phi error| = %.3e" % (a, b, err))
     coef = fit()
     print("coefficients (highest first):", ", ".join("%.9ef" % a for a in coef[::-1]))
     x = np.linspace(-9, 9, 1800001)
