@@ -63,6 +63,7 @@ def kernel_models(shape):
         "tc_state_build": (contr, d * e + Fn * dp * 4, "tensor"),
         "tc_readout": (contr, d * e + dp * 4 + 4, "tensor"),
         "tc_phi_forward_q": (phi1, d * e + dp * 4, "tensor"),
+        "tc_phiq_readout": (phi1 + contr, 2 * d * e + dp * 4 + 4, "tensor"),      # phi_q + readout + normaliser in one kernel
         "tc_phi_forward_k": (Fn * phi1, d * e + Fn * dp * 4, "tensor"),
         "tc_bwd_query": (2 * contr, 2 * d * e + 3 * dp * 4, "tensor"),
         "tc_bwd_key": (2 * contr, 2 * d * e + 2 * Fn * dp * 4, "tensor"),

@@ -10,6 +10,7 @@
 #include "hla_simt.cuh"
 #include "hla_tc.cuh"
 #include "hla_tc_phi.cuh"
+#include "hla_tc_fused.cuh"
 
 using namespace hla;
 
@@ -323,10 +324,13 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
     if (ctx->tc) {
         const float *qf, *kf;
         if (ctx->cfg.phi == HLA_PHI_MLP) {
-            s = tc::phi_forward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, ws, ctx->L, ctx->sm_count, ctx->rec);
+            // key maps -> state build -> reduction -> one kernel for phi_q, readout and normaliser
+            s = tc::phi_forward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, ws, ctx->L, ctx->sm_count, ctx->rec, false);
             if (s != HLA_OK) return s;
-            qf = reinterpret_cast<const float*>(ws + ctx->L.qf);
             kf = reinterpret_cast<const float*>(ws + ctx->L.kf);
+            s = tc::core_forward(ctx->tcp, ctx->D, ctx->BH, nullptr, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec, false);
+            if (s != HLA_OK) return s;
+            return tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
         } else {
             qf = static_cast<const float*>(Q);
             kf = static_cast<const float*>(K);

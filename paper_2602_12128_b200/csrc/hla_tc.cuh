@@ -1053,7 +1053,7 @@ inline bool set_smem(K kernel, int bytes) { return cudaFuncSetAttribute(kernel, 
 
 template <int DV>
 inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
-                                      const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
+                                      const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec, bool readout) {
     CUtensorMap mapV, mapO, mapB3;
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
     __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
@@ -1072,6 +1072,7 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     rec.begin("tc_reduce_emit");
     tc_reduce_emit_kernel<DV><<<dim3(8, BH), 256, 0, st>>>(part, state, b3, bq, D.S, D.ld);
     if (!rec.end()) return HLA_ERR_CUDA;
+    if (!readout) return HLA_OK;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
@@ -1080,10 +1081,11 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
+// readout = false stops after the state has been built and reduced (the fused query-side kernel reads it out).
 inline hla_status core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
-                               const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
-    if (D.d == 128) return launch_core_forward<128>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec);
-    return launch_core_forward<64>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec);
+                               const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec, bool readout = true) {
+    if (D.d == 128) return launch_core_forward<128>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
+    return launch_core_forward<64>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
 }
 
 template <int DV>

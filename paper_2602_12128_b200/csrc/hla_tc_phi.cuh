@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
 
 template <int DV>
 inline hla_status launch_phi_forward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, char* ws,
-                                     const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
+                                     const hla_ws_layout& L, int sm_count, LaunchRec& rec, bool q_side = true) {
     const long long rows = (long long)BH * D.N;
     CUtensorMap mapQ, mapK;
     PhiMaps mq, mk;
@@ -312,18 +312,21 @@ inline hla_status launch_phi_forward(const Dims& D, int BH, const hla_mlp* phi_q
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     cudaStream_t st = rec.st;
-    rec.begin("tc_phi_forward_q");
-    tc_phi_forward_kernel<DV, 1, false><<<grid, kPfThreads, PfCfg<DV, 1>::kSmem, st>>>(mapQ, mq, pq, reinterpret_cast<float*>(ws + L.qf), rows, D.N, status);
-    if (!rec.end()) return HLA_ERR_CUDA;
+    if (q_side) {
+        rec.begin("tc_phi_forward_q");
+        tc_phi_forward_kernel<DV, 1, false><<<grid, kPfThreads, PfCfg<DV, 1>::kSmem, st>>>(mapQ, mq, pq, reinterpret_cast<float*>(ws + L.qf), rows, D.N, status);
+        if (!rec.end()) return HLA_ERR_CUDA;
+    }
     rec.begin("tc_phi_forward_k");
     tc_phi_forward_kernel<DV, 3, true><<<grid, kPfThreads, PfCfg<DV, 3>::kSmem, st>>>(mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
+// q_side = false leaves phi_q to the fused query-side kernel (hla_tc_fused.cuh).
 inline hla_status phi_forward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, char* ws,
-                              const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
-    if (D.d == 128) return launch_phi_forward<128>(D, BH, phi_q, phi_k, Q, K, ws, L, sm_count, rec);
-    return launch_phi_forward<64>(D, BH, phi_q, phi_k, Q, K, ws, L, sm_count, rec);
+                              const hla_ws_layout& L, int sm_count, LaunchRec& rec, bool q_side = true) {
+    if (D.d == 128) return launch_phi_forward<128>(D, BH, phi_q, phi_k, Q, K, ws, L, sm_count, rec, q_side);
+    return launch_phi_forward<64>(D, BH, phi_q, phi_k, Q, K, ws, L, sm_count, rec, q_side);
 }
 
 // =======================================================================================
