@@ -299,22 +299,27 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(&d1_empty[b]);          // h is in registers: the next first-layer product may overwrite it
-            if (!mbar_wait(g_free, (it & 1) ^ 1)) { ok = false; report_timeout(status, 708); }      // the previous tile's second layer has read G
+            // All of the thread's GELU outputs are formed in registers first; the wait for the previous tile's second layer
+            // (the reader of the single G tile) then comes after the arithmetic instead of in front of it.
+            uint32_t w[HC / 2];
+#pragma unroll
+            for (int c = 0; c < HC / 16; ++c) {
+                const float2* bb = reinterpret_cast<const float2*>(bias + part * HC + 16 * c);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])), bb[e]));
+                    w[8 * c + e] = pack_bf16(g.x, g.y);
+                }
+            }
+            if (!mbar_wait(g_free, (it & 1) ^ 1)) { ok = false; report_timeout(status, 708); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
                 const int col = part * HC + 16 * c;
-                const float2* bb = reinterpret_cast<const float2*>(bias + col);
-                uint32_t w[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])), bb[e]));
-                    w[e] = pack_bf16(g.x, g.y);
-                }
                 const uint32_t blk = gblk + (col >> 6) * kBlk;
-                st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
-                st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
+                st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[8 * c], w[8 * c + 1], w[8 * c + 2], w[8 * c + 3]);
+                st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[8 * c + 4], w[8 * c + 5], w[8 * c + 6], w[8 * c + 7]);
             }
             fence_proxy_async();
             mbar_arrive(g_full);
