@@ -81,8 +81,8 @@ def kernel_models(shape):
 # DRAM traffic per token-head of a launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # scaled by token-heads; see profiles/).  None = not captured yet.
 NCU_TRAFFIC_PER_TOKEN_HEAD = {
-    "tc_phi_forward_q": 272.3, "tc_phi_forward_k": 315.6, "tc_state_build": 333.0, "tc_readout": 208.8,
-    "tc_bwd_query": 305.3, "tc_bwd_key": 595.2, "tc_phi_backward_q": 501.8, "tc_phi_backward_k": 615.3,
+    "tc_phi_forward_k": 314.9, "tc_state_build": 332.9, "tc_phiq_readout": 474.7, "tc_bwd_query": 305.2, "tc_bwd_key": 594.9,
+    "tc_phi_backward_q": 504.7, "tc_phi_backward_k": 619.3,
 }
 
 
