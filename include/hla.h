@@ -61,9 +61,9 @@ typedef enum {
  * Problem statement.  V, O, dO, dV (and Q, K, dQ, dK in HLA_PHI_MLP mode) are
  * [B,H,N,d] in `dtype`.  Features (HLA_PHI_NONE inputs and their gradients) are
  * always fp32.  Supported set: F in {1,2,3,4}, d_phi^F <= 256, d <= 128 and
- * d % 4 == 0, causal == 0.  dtype bf16 with d in {64,128} and (F,d_phi) in
- * {(3,6),(2,12)} runs on the tensor-core kernels; everything else in the
- * supported set runs on the fp32 SIMT kernels.
+ * d % 4 == 0, causal == 0.  dtype bf16 with d in {64,128}, F = 3, d_phi = 6 and
+ * B*H*N < 2^31 runs on the tensor-core kernels; everything else in the
+ * supported set (F = 2 with d_phi = 12 included) runs on the fp32 SIMT kernels.
  */
 typedef struct {
     int32_t B, H, N, d;
@@ -78,7 +78,8 @@ typedef struct {
 
 /*
  * One feature network (appendix "Defining phi"): feat = ReLU(W2^T GELU(W1^T x + b1) + b2),
- * exact (erf) GELU.  Device pointers in the ctx dtype: W1 [d][d] (input index
+ * the erf form of GELU (the tensor-core kernels evaluate its normal CDF with an
+ * error below 4e-4, under the bf16 rounding of the hidden layer).  Device pointers in the ctx dtype: W1 [d][d] (input index
  * first), b1 [d], W2 [d][d_phi], b2 [d_phi].  One set per map, shared by all
  * batches and heads.
  */
@@ -172,6 +173,14 @@ hla_status hla_forward_static(hla_ctx *ctx, const void *Q, const void *K, const 
 /* Synchronises `cuda_stream`, reads the device status words of `workspace`
  * and returns HLA_OK, HLA_ERR_DEVICE_TIMEOUT or HLA_ERR_CUDA. */
 hla_status hla_last_device_status(hla_ctx *ctx, const void *workspace, void *cuda_stream);
+
+/*
+ * Self-test of the failure path (no counterpart in the paper).  Every wait inside the kernels is bounded; this
+ * call enqueues a one-block kernel that waits, with a 1 ms limit, on a barrier that nothing arrives at.  The wait
+ * must run out, the kernel must return normally, and a following hla_last_device_status(ctx, workspace, stream)
+ * must report HLA_ERR_DEVICE_TIMEOUT.  The status words are cleared by the next hla_forward.
+ */
+hla_status hla_selftest_bounded_wait(hla_ctx *ctx, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /* Number of kernels the last hla_forward / hla_backward on this ctx launched. */
 int32_t hla_last_launch_count(const hla_ctx *ctx);

@@ -18,7 +18,7 @@ HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
     "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_forward_static",
-    "hla_last_device_status", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
+    "hla_last_device_status", "hla_selftest_bounded_wait", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
     "hla_destroy", "hla_status_string",
 ]
 
@@ -76,6 +76,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_forward_static.restype = c_int32
     lib.hla_last_device_status.argtypes = [c_void_p, c_void_p, c_void_p]
     lib.hla_last_device_status.restype = c_int32
+    lib.hla_selftest_bounded_wait.argtypes = [c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.hla_selftest_bounded_wait.restype = c_int32
     lib.hla_last_launch_count.argtypes = [c_void_p]
     lib.hla_last_launch_count.restype = c_int32
     lib.hla_timing_enable.argtypes = [c_void_p, c_int32]
@@ -172,6 +174,13 @@ def hla_forward_static(ctx: int, Q, K, V, O, stream=None) -> int:
 
 def hla_last_device_status(ctx: int, workspace, stream=None) -> int:
     return int(load_library().hla_last_device_status(ctx, _ptr(workspace), _stream(stream)))
+
+
+def hla_selftest_bounded_wait(ctx: int, workspace, stream=None) -> None:
+    nbytes = workspace.numel() * workspace.element_size()
+    st = load_library().hla_selftest_bounded_wait(ctx, _ptr(workspace), nbytes, _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_selftest_bounded_wait")
 
 
 def hla_last_launch_count(ctx: int) -> int:

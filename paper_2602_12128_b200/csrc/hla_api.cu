@@ -419,6 +419,17 @@ hla_status hla_last_device_status(hla_ctx* ctx, const void* workspace, void* cud
     return words[kStatusTimeout] != 0 ? HLA_ERR_DEVICE_TIMEOUT : HLA_OK;
 }
 
+hla_status hla_selftest_bounded_wait(hla_ctx* ctx, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HLA_ERR_INVALID_ARG;
+    if (workspace_bytes < ctx->ws_bytes) return HLA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    (void)cudaGetLastError();
+    if (cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
+    tc::tc_wait_selftest_kernel<<<1, 32, 0, st>>>(reinterpret_cast<int*>(ws + ctx->L.status), 1000000ull);   // gives up after 1 ms
+    return cudaPeekAtLastError() == cudaSuccess ? HLA_OK : HLA_ERR_CUDA;
+}
+
 int32_t hla_last_launch_count(const hla_ctx* ctx) { return ctx ? ctx->rec.launches : 0; }
 
 hla_status hla_timing_enable(hla_ctx* ctx, int32_t on) {

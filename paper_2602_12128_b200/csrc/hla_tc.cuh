@@ -1047,6 +1047,18 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
+// Self-test of the bounded waits: one CTA waits on a barrier that nothing ever arrives at, with a limit of
+// `limit_ns`; the wait must run out, record the time-out in the status words and let the kernel return normally.
+__global__ void tc_wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait(&bar, 0, limit_ns)) report_timeout(status, 901);
+}
+
 // ---- host launch helpers ---------------------------------------------------------------
 template <typename K>
 inline bool set_smem(K kernel, int bytes) { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess; }

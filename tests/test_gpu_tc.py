@@ -147,3 +147,17 @@ def test_full_backward_bf16_mlp_stagewise():
     assert l2err(dQ[keep_q], eQ[keep_q]) < TOL["bf16"], l2err(dQ[keep_q], eQ[keep_q])
     assert l2err(dK[keep_k], eK[keep_k]) < TOL["bf16"], l2err(dK[keep_k], eK[keep_k])
     assert run.op.launches() == 5
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    """Failure detection without a fault: a wait that nothing satisfies runs out after its limit, the kernel returns,
+    the host reads HLA_ERR_DEVICE_TIMEOUT, and the same context computes a correct forward afterwards."""
+    s = synth.HlaShape("t", 1, 2, 300, 128, "bf16", "inv_sqrt_d")
+    _, _, V = synth.make_qkv(s)
+    qf, kf = synth.make_features(s)
+    run = GpuRun(s, "none", EPS)
+    binding.hla_selftest_bounded_wait(run.op.ctx, run.op.workspace)
+    assert run.op.device_status() == binding.HLA_ERR_DEVICE_TIMEOUT
+    O = run.forward(qf, kf, V)                                    # clears the status words; asserts HLA_OK inside
+    Oq, _ = orc.hla_core_forward(qf.astype(np.float64), kf.astype(np.float64), V.astype(np.float64), EPS, "quadratic")
+    assert relerr(O, Oq) < TOL["bf16"]
