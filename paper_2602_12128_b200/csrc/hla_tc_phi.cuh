@@ -594,8 +594,9 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(dg_empty);
+            // (dg(u) complete also means the dX product of unit u - 2 has completed - same issuing thread, issued earlier,
+            // and a commit covers everything before it - so the dh tile of this parity is free without a wait of its own.)
             if (!mbar_wait(&h_full[b], par)) { ok = false; report_timeout(status, 604); }
-            if (ok && !mbar_wait(&dh_free[b], par ^ 1)) { ok = false; report_timeout(status, 605); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
