@@ -53,7 +53,8 @@ def work_model(shape):
 
 def kernel_models(shape):
     """Per launch: (algorithmic flops, algorithmic HBM bytes, compute unit) of each kernel; the per-token-head
-    figures are listed in the design doc.  Tiny kernels (reductions) are left out."""
+    figures are FLOPs = 2 x multiply-adds of the paper's factored scheme and the tensors each kernel must stream once.
+    Tiny kernels (reductions) are left out."""
     d, P, dp, Fn = shape.d, shape.d_phi ** shape.F, shape.d_phi, shape.F
     th = shape.B * shape.H * shape.N
     e = 2
@@ -62,7 +63,6 @@ def kernel_models(shape):
     m = {
         "tc_state_build": (contr, d * e + Fn * dp * 4, "tensor"),
         "tc_readout": (contr, d * e + dp * 4 + 4, "tensor"),
-        "tc_phi_forward_q": (phi1, d * e + dp * 4, "tensor"),
         "tc_phiq_readout": (phi1 + contr, 2 * d * e + dp * 4 + 4, "tensor"),      # phi_q + readout + normaliser in one kernel
         "tc_phi_forward_k": (Fn * phi1, d * e + Fn * dp * 4, "tensor"),
         "tc_bwd_query": (2 * contr, 2 * d * e + 3 * dp * 4, "tensor"),

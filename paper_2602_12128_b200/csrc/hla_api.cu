@@ -325,7 +325,7 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
         const float *qf, *kf;
         if (ctx->cfg.phi == HLA_PHI_MLP) {
             // key maps -> state build -> reduction -> one kernel for phi_q, readout and normaliser
-            s = tc::phi_forward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, ws, ctx->L, ctx->sm_count, ctx->rec, false);
+            s = tc::phi_forward_k(ctx->D, ctx->BH, ctx->phi_k, K, ws, ctx->L, ctx->sm_count, ctx->rec);
             if (s != HLA_OK) return s;
             kf = reinterpret_cast<const float*>(ws + ctx->L.kf);
             s = tc::core_forward(ctx->tcp, ctx->D, ctx->BH, nullptr, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec, false);

@@ -286,20 +286,15 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
+// Key-side feature maps phi_k1..3 on K (phi_q runs inside the fused query-side kernel, hla_tc_fused.cuh).
 template <int DV>
-inline hla_status launch_phi_forward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, char* ws,
-                                     const hla_ws_layout& L, int sm_count, LaunchRec& rec, bool q_side = true) {
+inline hla_status launch_phi_forward_k(const Dims& D, int BH, const hla_mlp* phi_k, const void* K, char* ws, const hla_ws_layout& L, int sm_count,
+                                       LaunchRec& rec) {
     const long long rows = (long long)BH * D.N;
-    CUtensorMap mapQ, mapK;
-    PhiMaps mq, mk;
-    PhiPtrs pq{}, pk{};
-    if (!make_map_2d(&mapQ, Q, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
-    if (!make_map_2d(&mq.w1[0], phi_q->W1, DV, DV, DV)) return HLA_ERR_CUDA;
-    mq.w1[1] = mq.w1[0];
-    mq.w1[2] = mq.w1[0];
-    pq.b1[0] = static_cast<const __nv_bfloat16*>(phi_q->b1);
-    pq.W2[0] = static_cast<const __nv_bfloat16*>(phi_q->W2);
-    pq.b2[0] = static_cast<const __nv_bfloat16*>(phi_q->b2);
+    CUtensorMap mapK;
+    PhiMaps mk;
+    PhiPtrs pk{};
+    if (!make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
     for (int f = 0; f < 3; ++f) {
         if (!make_map_2d(&mk.w1[f], phi_k[f].W1, DV, DV, DV)) return HLA_ERR_CUDA;
         pk.b1[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b1);
@@ -307,26 +302,18 @@ inline hla_status launch_phi_forward(const Dims& D, int BH, const hla_mlp* phi_q
         pk.b2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b2);
     }
     int* status = reinterpret_cast<int*>(ws + L.status);
-    if (!set_smem(tc_phi_forward_kernel<DV, 1, false>, PfCfg<DV, 1>::kSmem) || !set_smem(tc_phi_forward_kernel<DV, 3, true>, PfCfg<DV, 3>::kSmem))
-        return HLA_ERR_CUDA;
+    if (!set_smem(tc_phi_forward_kernel<DV, 3, true>, PfCfg<DV, 3>::kSmem)) return HLA_ERR_CUDA;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    cudaStream_t st = rec.st;
-    if (q_side) {
-        rec.begin("tc_phi_forward_q");
-        tc_phi_forward_kernel<DV, 1, false><<<grid, kPfThreads, PfCfg<DV, 1>::kSmem, st>>>(mapQ, mq, pq, reinterpret_cast<float*>(ws + L.qf), rows, D.N, status);
-        if (!rec.end()) return HLA_ERR_CUDA;
-    }
     rec.begin("tc_phi_forward_k");
-    tc_phi_forward_kernel<DV, 3, true><<<grid, kPfThreads, PfCfg<DV, 3>::kSmem, st>>>(mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
+    tc_phi_forward_kernel<DV, 3, true><<<grid, kPfThreads, PfCfg<DV, 3>::kSmem, rec.st>>>(mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
-// q_side = false leaves phi_q to the fused query-side kernel (hla_tc_fused.cuh).
-inline hla_status phi_forward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, char* ws,
-                              const hla_ws_layout& L, int sm_count, LaunchRec& rec, bool q_side = true) {
-    if (D.d == 128) return launch_phi_forward<128>(D, BH, phi_q, phi_k, Q, K, ws, L, sm_count, rec, q_side);
-    return launch_phi_forward<64>(D, BH, phi_q, phi_k, Q, K, ws, L, sm_count, rec, q_side);
+inline hla_status phi_forward_k(const Dims& D, int BH, const hla_mlp* phi_k, const void* K, char* ws, const hla_ws_layout& L, int sm_count,
+                                LaunchRec& rec) {
+    if (D.d == 128) return launch_phi_forward_k<128>(D, BH, phi_k, K, ws, L, sm_count, rec);
+    return launch_phi_forward_k<64>(D, BH, phi_k, K, ws, L, sm_count, rec);
 }
 
 // =======================================================================================
