@@ -50,50 +50,63 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// Host side: counts the kernels a call launches and, when enabled, brackets each
-// launch with CUDA events on the launching stream so a caller can read per-kernel device time.
+// Host side: counts the kernels a call launches and, when enabled, marks each launch with CUDA events on the
+// launching stream so a caller can read per-kernel device time.  Kernels of one call run back to back on the stream,
+// so one event between two launches serves as the end of the first and the start of the second: n launches of a call
+// cost n + 1 event records.
 struct LaunchRec {
-    struct Ev { cudaEvent_t a, b; const char* name; };
+    struct Rec { const char* name; int a, b; };            // indices into `events`
     struct Acc { const char* name; double ms; long long n; };
     cudaStream_t st = nullptr;
     int launches = 0;
     bool timing = false;
-    std::vector<Ev> pool;
+    std::vector<cudaEvent_t> events;      // pool, reused after every collect()
     size_t used = 0;
+    std::vector<Rec> recs;
+    int last_end = -1;                    // event that ended the previous launch of this call
     std::vector<Acc> acc;
 
-    void start_call(cudaStream_t s) { st = s; launches = 0; }
+    void start_call(cudaStream_t s) { st = s; launches = 0; last_end = -1; }
+    int mark() {
+        if (used == events.size()) {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreate(&e) != cudaSuccess) { timing = false; return -1; }
+            events.push_back(e);
+        }
+        cudaEventRecord(events[used], st);
+        return (int)used++;
+    }
     void begin(const char* name) {
         ++launches;
         if (!timing) return;
-        if (used == pool.size()) {
-            Ev e{nullptr, nullptr, name};
-            if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) { timing = false; return; }
-            pool.push_back(e);
-        }
-        pool[used].name = name;
-        cudaEventRecord(pool[used].a, st);
+        const int a = last_end >= 0 ? last_end : mark();
+        if (a >= 0) recs.push_back(Rec{name, a, -1});
     }
     bool end() {
-        if (timing && used < pool.size()) cudaEventRecord(pool[used++].b, st);
+        if (timing && !recs.empty() && recs.back().b < 0) {
+            recs.back().b = mark();
+            last_end = recs.back().b;
+        }
         return cudaPeekAtLastError() == cudaSuccess;
     }
-    // Caller has synchronised the stream.  Folds the recorded pairs into per-name totals (replacing earlier totals).
+    // Caller has synchronised the stream.  Folds the recorded launches into per-name totals (replacing earlier totals).
     int collect() {
         acc.clear();
-        for (size_t i = 0; i < used; ++i) {
+        for (const Rec& r : recs) {
             float ms = 0.f;
-            if (cudaEventElapsedTime(&ms, pool[i].a, pool[i].b) != cudaSuccess) continue;
+            if (r.a < 0 || r.b < 0 || cudaEventElapsedTime(&ms, events[r.a], events[r.b]) != cudaSuccess) continue;
             size_t j = 0;
-            for (; j < acc.size(); ++j) if (strcmp(acc[j].name, pool[i].name) == 0) break;
-            if (j == acc.size()) acc.push_back(Acc{pool[i].name, 0.0, 0});
+            for (; j < acc.size(); ++j) if (strcmp(acc[j].name, r.name) == 0) break;
+            if (j == acc.size()) acc.push_back(Acc{r.name, 0.0, 0});
             acc[j].ms += ms;
             acc[j].n += 1;
         }
+        recs.clear();
         used = 0;
+        last_end = -1;
         return (int)acc.size();
     }
-    ~LaunchRec() { for (auto& e : pool) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); } }
+    ~LaunchRec() { for (auto e : events) cudaEventDestroy(e); }
 };
 
 }  // namespace hla
