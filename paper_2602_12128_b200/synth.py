@@ -42,6 +42,11 @@ CONFIGS = {
     "train_bf16": HlaShape("train_bf16", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=True),
 }
 
+# The paper's own two resolutions (Section 5: Wan2.1-1.3B has 12 heads of 128 channels; 81x480x832 video -> 32760
+# tokens, 81x320x480 -> 12600 tokens), as extra workloads next to the five benchmark configurations.
+CONFIGS["paper_r1_bf16"] = HlaShape("paper_r1_bf16", 1, 12, 32760, 128, "bf16", "rms_qk", backward=True)
+CONFIGS["paper_r2_bf16"] = HlaShape("paper_r2_bf16", 1, 12, 12600, 128, "bf16", "rms_qk", backward=True)
+
 
 def bf16_round(x: np.ndarray) -> np.ndarray:
     """Round float32 values to the nearest bfloat16 (ties to even); result stays float32."""

@@ -144,8 +144,17 @@ def test_config4_long_bf16_forward():
 
 def test_config5_train_bf16_forward_backward():
     """B=2, H=24, N=32760, d=128, dO ~ N(0,1): dQ, dK, dV against the oracle's analytic gradients."""
-    rng = np.random.default_rng(13)
-    r = FullRun("train_bf16")
+    check_training_step("train_bf16", np.random.default_rng(13), whole_heads=4)
+
+
+def test_paper_resolution_r2_forward_backward():
+    """The smaller of the paper's own two resolutions: 12 heads x 128 channels, 12600 tokens (Section 5), Q and K
+    RMS-normalised; forward and backward."""
+    check_training_step("paper_r2_bf16", np.random.default_rng(14), whole_heads=2)
+
+
+def check_training_step(name, rng, whole_heads):
+    r = FullRun(name)
     s = r.s
     check_features_sampled(r, rng)
     check_core_forward_rows(r, rng, rows_per_head=16)
@@ -169,7 +178,7 @@ def test_config5_train_bf16_forward_backward():
     # a few whole heads: the factored backward at the features the GPU produced, then the phi backward at the
     # feature gradients the GPU produced (rows whose ReLU mask differs from the oracle's are counted, not compared)
     d = s.d
-    for b, h in r.some_heads(4):
+    for b, h in r.some_heads(whole_heads):
         gq, gk = f64(r.gq[b, h]), [f64(r.gk[b, h, f]) for f in range(s.F)]
         dq_ref, dks_ref, dv_ref = orc.hla_factored_backward(gq, gk, f64(r.V[b, h]), f64(r.dO[b, h]), EPS)
         assert relerr(r.dV[b, h], dv_ref) < TOL["bf16"], (b, h)
