@@ -161,3 +161,34 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable():
     O = run.forward(qf, kf, V)                                    # clears the status words; asserts HLA_OK inside
     Oq, _ = orc.hla_core_forward(qf.astype(np.float64), kf.astype(np.float64), V.astype(np.float64), EPS, "quadratic")
     assert relerr(O, Oq) < TOL["bf16"]
+
+
+def test_forward_backward_replay_in_a_cuda_graph():
+    """The library only enqueues work on the caller's stream, so a whole training step can be captured once in a CUDA
+    graph and replayed; the replays must reproduce the eager results bit for bit."""
+    s = synth.HlaShape("t", 1, 3, 1500, 128, "bf16", "rms_qk", backward=True)
+    Q, K, V = synth.make_qkv(s)
+    dO = synth.make_dO(s)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    run = GpuRun(s, "mlp", EPS)
+    run.set_weights(pq, pk)
+    O_ref = run.forward(Q, K, V)
+    ref = run.backward(dO)
+    op = run.op
+    O, dQ, dK, dV = (torch.empty_like(run.V) for _ in range(4))
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            binding.hla_forward(op.ctx, run.Q, run.K, run.V, O, op.workspace, side)
+            binding.hla_backward(op.ctx, run.Q, run.K, run.V, O, run.dO, dQ, dK, dV, op.workspace, side)
+    for _ in range(2):
+        for t in (O, dQ, dK, dV):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert op.device_status() == binding.HLA_OK
+        assert np.array_equal(O.float().cpu().numpy(), O_ref.astype(np.float32))
+        for got, want in zip((dQ, dK, dV), ref):
+            assert np.array_equal(got.float().cpu().numpy(), want.astype(np.float32))
