@@ -94,9 +94,12 @@ def test_backward_bitwise_reproducible():
         assert np.array_equal(x, y)
 
 
-def test_small_config_d64_forward_backward_with_phi():
-    """The small benchmark shape (B=2, H=12, N=4096, d=64) with the phi maps, forward and backward, stage by stage."""
-    s = synth.CONFIGS["small_bf16"]
+@pytest.mark.parametrize("shape", [synth.CONFIGS["small_bf16"], synth.HlaShape("ragged64", 1, 3, 777, 64, "bf16", "rms_qk"),
+                                   synth.HlaShape("ragged128", 2, 1, 131, 128, "bf16", "inv_sqrt_d")], ids=lambda s: s.name)
+def test_forward_backward_with_phi_stage_by_stage(shape):
+    """The small benchmark shape (B=2, H=12, N=4096, d=64) and two ragged shapes with the phi maps (fused query side,
+    key maps, both phi backward kernels), forward and backward, stage by stage."""
+    s = shape
     Q, K, V = synth.make_qkv(s)
     dO = synth.make_dO(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
