@@ -106,6 +106,7 @@ __device__ __forceinline__ void report_timeout(int* status, int where) {
     atomicExch(status + kStatusWhere, where);
 }
 __device__ __forceinline__ void named_barrier(int id, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
+__device__ __forceinline__ void st_shared_b16(uint32_t addr, unsigned short v) { asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -586,17 +587,28 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
 //   D2[i][m]  = sum_g dO_i[g] Csym[m][g]                                   (MMA, K = d)
 //   s_i       = sum_m mono_i[m] D2[i][m] ;  delta_i = dO_i . o_i = r_i s_i ;  deta_i = -r_i delta_i
 //   dmono_i[m]= r_i D2[i][m] + deta_i zsym[m]  ->  dq_i                     (ALUs)
-//   dCsym^T  += dO_tile^T * (r_i mono_i)                                    (MMA, K = tokens)
-//   dzsym[m] += mono_i[m] deta_i                                            (ALUs)
+//   [dCsym | dzsym][m][:] += (r_i mono_i[m]) * [dO_i | deta_i / r_i]         (MMA, K = tokens)
 // O itself is not read: dO . o is recovered from D2.
+//
+// The second product has the monomials on the M side (64 rows) and d + 8 columns: the operand row that a generator
+// thread writes for its token is [deta/r, 0 x 7, r mono_0..55], so the same 128-byte row serves as row of the A operand
+// (rows 8..63 = monomials) and, read as the block that follows the dO blocks, as columns d..d+7 of the B operand
+// (column d = deta/r, the rest zero).  Accumulator row 8+m then holds dCsym[m][0..d-1], dzsym[m], 0, 0, 0: one row of
+// the partial state, and dz costs no product of its own.  Rows 0..7 of the accumulator are not used.
+//
+// The tensor pipe needs ~100 cycles per MMA of this size (set by the operand bytes it reads from shared memory, not by
+// the arithmetic), so the MMAs per tile are kept at 16 and are issued by two threads (D2: warp 1, dC: warp 2).
 // =======================================================================================
-constexpr int kBqThreads = 320;
-constexpr int kBqStages = 3;
-constexpr int kBqStageBytes = 2 * kBlk + kBlk;          // dO tile (two 64-column blocks) + r*mono tile
+constexpr int kBqGroups = 3;                            // generator groups of 128 threads; tile `it` belongs to group it % 3
+constexpr int kBqThreads = 128 + 128 * kBqGroups;       // warp 0: TMA, warp 1: D2 MMAs, warp 2: dC MMAs, warp 3 idle, warps 4..: generators
+constexpr int kBqStages = 4;
+constexpr int kBqStageBytes = 3 * kBlk;                 // dO tile (d/64 blocks of 64 columns) directly followed by the operand-row tile
 constexpr int kBqOffOp = kBqStages * kBqStageBytes;     // Csym operand [64][d] bf16 (two 8 KB blocks)
-constexpr int kBqOffZ = kBqOffOp + kBlk;                // zsym (64 floats) then zred [8][64]
-constexpr int kBqOffBars = kBqOffZ + 64 * 4 + 8 * 64 * 4;
+constexpr int kBqOffZ = kBqOffOp + kBlk;                // zsym (64 floats)
+constexpr int kBqOffBars = kBqOffZ + 64 * 4;
 constexpr int kBqSmem = 1024 + kBqOffBars + 256;
+constexpr int kBqColD2 = 256;                           // TMEM columns of the D2 buffers (one per group, 64 columns each)
+constexpr int kBqRowPad = 8;                            // accumulator row of monomial 0
 
 template <int DV>
 __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __grid_constant__ CUtensorMap mapdO, const __grid_constant__ CUtensorMap mapBq,
@@ -606,16 +618,19 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     float* zsym = reinterpret_cast<float*>(smem + kBqOffZ);
-    float* zred = zsym + 64;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBqOffBars);
-    uint64_t* full_do = bars;             // [3]
-    uint64_t* full_rm = bars + 3;         // [3] 128 arrivals
-    uint64_t* empty = bars + 6;           // [3] MMA commit
-    uint64_t* d2_full = bars + 9;         // [2] MMA commit
-    uint64_t* d2_empty = bars + 11;       // [2] 128 arrivals
-    uint64_t* op_full = bars + 13;
-    uint64_t* acc_done = bars + 14;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+    uint64_t* full_do = bars;                       // [stages] TMA
+    uint64_t* full_rm = bars + kBqStages;           // [stages] 128 arrivals: the operand rows of the tile are complete
+    uint64_t* empty_rm = bars + 2 * kBqStages;      // [stages] MMA commit (dC): the operand-row tile is free
+    uint64_t* empty_do = bars + 3 * kBqStages;      // [stages] MMA commits (D2 and dC): the dO tile is free
+    uint64_t* d2_full = bars + 4 * kBqStages;       // [groups] MMA commit
+    uint64_t* d2_empty = d2_full + kBqGroups;       // [groups] 128 arrivals
+    uint64_t* op_full = d2_empty + kBqGroups;
+    uint64_t* acc_done = op_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
+    static_assert((4 * kBqStages + 2 * kBqGroups + 3) * 8 <= 256, "barrier block");
+    constexpr int kRmOff = (DV / 64) * kBlk;        // operand-row tile inside a stage
+    constexpr int kNC = DV + 8;                     // columns of the dC product
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int s = blockIdx.x, bh = blockIdx.y;
@@ -628,21 +643,15 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
         for (int i = tid; i < kMono * ld; i += kBqThreads) out[i] = 0.f;
         return;
     }
-    if (DV == 64) {
-        for (int st = 0; st < kBqStages; ++st) {
-            uint4* vz = reinterpret_cast<uint4*>(smem + st * kBqStageBytes + kBlk);
-            for (int i = tid; i < kBlk / 16; i += kBqThreads) vz[i] = make_uint4(0, 0, 0, 0);
-        }
-        fence_proxy_async();
-    }
     if (tid < 64) zsym[tid] = tid < kMono ? state[((size_t)bh * kMono + tid) * ld + DV] : 0.f;
     if (tid == 0) {
         for (int i = 0; i < kBqStages; ++i) {
             mbar_init(&full_do[i], 1);
             mbar_init(&full_rm[i], 128);
-            mbar_init(&empty[i], 1);
+            mbar_init(&empty_rm[i], 1);
+            mbar_init(&empty_do[i], 2);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kBqGroups; ++i) {
             mbar_init(&d2_full[i], 1);
             mbar_init(&d2_empty[i], 128);
         }
@@ -653,7 +662,7 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
         prefetch_tmap(&mapBq);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, 256);
+        tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -668,7 +677,7 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + kBqOffOp + b * (kBlk / 2), &mapBq, op_full, b * 64, bh * kMonoPad);
             for (int it = 0; it < ntiles; ++it) {
                 const int st = it % kBqStages, u = it / kBqStages;
-                if (!mbar_wait(&empty[st], (u & 1) ^ 1)) { report_timeout(status, 301); break; }
+                if (!mbar_wait(&empty_do[st], (u & 1) ^ 1)) { report_timeout(status, 301); break; }
                 uint8_t* ds = smem + st * kBqStageBytes;
                 mbar_arrive_expect_tx(&full_do[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b) tma_load_3d(ds + b * kBlk, &mapdO, &full_do[st], b * 64, (tile0 + it) * kTileTokens, bh);
@@ -676,45 +685,46 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc2 = idesc_bf16(128, kMonoPad, false, false);   // D2 = dO (K-major over g) * Csym (K-major over g)
-            const uint32_t idesc1 = idesc_bf16(128, kMonoPad, true, true);     // dCsym^T += dO^T (MN-major) * r mono (MN-major)
+            // D2 = dO (K-major over g) * Csym (K-major over g); tile `it` is issued as soon as its dO tile has landed
+            // and the group that owns the tile has read its previous D2, which is long before the group asks for it.
+            const uint32_t idesc2 = idesc_bf16(128, kMonoPad, false, false);
             const uint32_t opa = smem_u32(smem + kBqOffOp);
-            bool good = mbar_wait(op_full, 0);
-            if (!good) report_timeout(status, 302);
-            // D2 of tile `it`; issued one tile ahead of the tile's dC product so that the generators never wait for it
-            auto issue_d2 = [&](int it) -> bool {
-                const int st = it % kBqStages, u = it / kBqStages, buf = it & 1, ub = it >> 1;
-                if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&d2_empty[buf], (ub & 1) ^ 1))) return false;
-                tc_fence_after();
-                const uint32_t da = smem_u32(smem + st * kBqStageBytes);
+            if (!mbar_wait(op_full, 0)) report_timeout(status, 302);
+            else
+                for (int it = 0; it < ntiles; ++it) {
+                    const int st = it % kBqStages, u = it / kBqStages, buf = it % kBqGroups, ub = it / kBqGroups;
+                    if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&d2_empty[buf], (ub & 1) ^ 1))) { report_timeout(status, 303); break; }
+                    tc_fence_after();
+                    const uint32_t da = smem_u32(smem + st * kBqStageBytes);
 #pragma unroll
-                for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 64 + 64 * buf, smem_desc_sw128(da + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(opa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
-                umma_commit(&d2_full[buf]);
-                return true;
-            };
-            if (good && !issue_d2(0)) { good = false; report_timeout(status, 303); }
-            for (int it = 0; it < ntiles && good; ++it) {
+                    for (int ks = 0; ks < DV / 16; ++ks)
+                        umma_bf16(tmem + kBqColD2 + 64 * buf, smem_desc_sw128(da + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                                  smem_desc_sw128(opa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
+                    umma_commit(&d2_full[buf]);
+                    umma_commit(&empty_do[st]);
+                }
+        }
+    } else if (warp == 2) {
+        if (lane == 0) {
+            // [dCsym | dzsym] += (operand rows)^T (MN-major, M = 64) * [dO | operand rows' first 8 columns] (MN-major, N = d + 8)
+            const uint32_t idesc1 = idesc_bf16(64, kNC, true, true);
+            for (int it = 0; it < ntiles; ++it) {
                 const int st = it % kBqStages, u = it / kBqStages;
-                if (it + 1 < ntiles && !issue_d2(it + 1)) { report_timeout(status, 303); break; }
-                if (!mbar_wait(&full_rm[st], u & 1)) { report_timeout(status, 304); break; }
+                if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&full_rm[st], u & 1))) { report_timeout(status, 304); break; }
                 tc_fence_after();
-                const uint32_t da = smem_u32(smem + st * kBqStageBytes), ra = da + 2 * kBlk;
+                const uint32_t da = smem_u32(smem + st * kBqStageBytes), ra = da + kRmOff;
 #pragma unroll
                 for (int ks = 0; ks < kTileTokens / 16; ++ks)
-                    umma_bf16(tmem, smem_desc_sw128(da + ks * 2048, kBlk, 1024), smem_desc_sw128(ra + ks * 2048, kBlk, 1024), idesc1,
+                    umma_bf16(tmem, smem_desc_sw128(ra + ks * 2048, kBlk, 1024), smem_desc_sw128(da + ks * 2048, kBlk, 1024), idesc1,
                               (it > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(&empty[st]);
+                umma_commit(&empty_do[st]);
+                umma_commit(&empty_rm[st]);
             }
             umma_commit(acc_done);
         }
-    } else {
-        const int grp = (warp - 2) >> 2, quarter = warp & 3;
+    } else if (warp >= 4) {
+        const int grp = (warp - 4) >> 2, quarter = warp & 3;
         const int row = quarter * 32 + lane;    // token row of the tile == TMEM lane this thread can read
-        float dzacc[kMono];
-#pragma unroll
-        for (int i = 0; i < kMono; ++i) dzacc[i] = 0.f;
         // The features and the normaliser of the group's next tile are loaded while the current one is processed
         // (row index clamped: the loads are unconditional, out-of-range rows are zeroed when used).
         float qn[6], etan;
@@ -724,15 +734,16 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             etan = __ldg(eta + (size_t)bh * N + tok);
         };
         if (grp < ntiles) prefetch(grp);
-        for (int it = grp; it < ntiles; it += 2) {
-            const int st = it % kBqStages, u = it / kBqStages, buf = it & 1, ub = it >> 1;
+        for (int it = grp; it < ntiles; it += kBqGroups) {
+            const int st = it % kBqStages, u = it / kBqStages, buf = grp, ub = it / kBqGroups;
             const int tok = (tile0 + it) * kTileTokens + row;
+            const uint32_t rblk = smem_u32(smem + st * kBqStageBytes + kRmOff);
             float q[6], r = 0.f;
 #pragma unroll
             for (int i = 0; i < 6; ++i) q[i] = tok < N ? qn[i] : 0.f;
             if (tok < N) r = 1.f / (etan + eps);
-            if (it + 2 < ntiles) prefetch(it + 2);
-            {   // operand row r_i * mono_i; formed from (r q_a) q_b q_c so that no monomial stays live across the wait below
+            {   // columns 8..63 of the operand row: r_i * mono_i, formed from (r q_a) q_b q_c so that no monomial stays live
+                // across the wait below
                 float qs[6], rmono[kMono];
 #pragma unroll
                 for (int i = 0; i < 6; ++i) qs[i] = r * q[i];
@@ -744,11 +755,12 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
 #pragma unroll
                         for (int c = b; c < 6; ++c) rmono[mono_idx(a, b, c)] = qab * q[c];
                     }
-                if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
+                if (ok && !mbar_wait(&empty_rm[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
                 if (ok) {
-                    store_mono_row(smem_u32(smem + st * kBqStageBytes + 2 * kBlk), row, rmono, 1.f);
-                    fence_proxy_async();
-                    mbar_arrive(&full_rm[st]);
+#pragma unroll
+                    for (int c = 0; c < 7; ++c)
+                        st_shared_v4(rblk + sw128_off(row, c + 1), pack_bf16(rmono[8 * c], rmono[8 * c + 1]), pack_bf16(rmono[8 * c + 2], rmono[8 * c + 3]),
+                                     pack_bf16(rmono[8 * c + 4], rmono[8 * c + 5]), pack_bf16(rmono[8 * c + 6], rmono[8 * c + 7]));
                 }
             }
             if (ok && !mbar_wait(&d2_full[buf], ub & 1)) { ok = false; report_timeout(status, 306); }
@@ -756,7 +768,7 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             if (!ok) continue;
             tc_fence_after();
             uint32_t d2[kMono];
-            const uint32_t ta = tmem + 64 + 64 * buf + ((uint32_t)(quarter * 32) << 16);
+            const uint32_t ta = tmem + kBqColD2 + 64 * buf + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
             for (int c = 0; c < kMono / 8; ++c) tmem_ld8(ta + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(d2 + 8 * c));
             tmem_ld_wait();
@@ -780,6 +792,11 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
                     }
             const float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
             const float deta = -r * r * sdot;
+            // columns 0..7 of the operand row: deta / r, then zeros; one proxy fence covers the whole row
+            st_shared_v4(rblk + sw128_off(row, 0), pack_bf16(-r * sdot, 0.f), 0u, 0u, 0u);
+            fence_proxy_async();
+            mbar_arrive(&full_rm[st]);
+            if (it + kBqGroups < ntiles) prefetch(it + kBqGroups);
             float dq[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int a = 0; a < 6; ++a)
@@ -789,46 +806,36 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
                     for (int c = b; c < 6; ++c) {
                         const int m = mono_idx(a, b, c);
                         const float g = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);      // dmono_i[m]
-                        dzacc[m] = fmaf(q[a] * qq[b][c], deta, dzacc[m]);
                         dq[a] = fmaf(g, qq[b][c], dq[a]);
                         dq[b] = fmaf(g, qq[a][c], dq[b]);
                         dq[c] = fmaf(g, qq[a][b], dq[c]);
                     }
             if (tok < N) store6(dqf + ((size_t)bh * N + tok) * 6, dq);
         }
-#pragma unroll
-        for (int i = 0; i < kMono; ++i) {
-            const float v = warp_sum(dzacc[i]);
-            if (lane == 0) zred[(warp - 2) * 64 + i] = v;
-        }
-        named_barrier(1, 256);
-        const int gi = tid - 64;
-        if (gi < kMono) {
-            float z = 0.f;
-#pragma unroll
-            for (int w = 0; w < 8; ++w) z += zred[w * 64 + gi];
-            out[(size_t)gi * ld + DV] = z;
-            for (int c = DV + 1; c < ld; ++c) out[(size_t)gi * ld + c] = 0.f;
-        }
-        if (warp < 6) {
+        if (grp == 0) {
+            // A 64-row accumulator keeps row R in TMEM lane 32 * (R / 16) + R % 16: lanes 0..15 of each warp's quarter.
             if (ok && !mbar_wait(acc_done, 0)) { ok = false; report_timeout(status, 307); }
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
-            if (ok && quarter * 32 < DV) {
-#pragma unroll
-                for (int c = 0; c < kMono / 8; ++c) {
+            const int m = quarter * 16 + lane - kBqRowPad;
+            if (ok) {
+#pragma unroll 1
+                for (int c = 0; c < kNC / 8; ++c) {
                     uint32_t rr[8];
                     tmem_ld8(tmem + ((uint32_t)(quarter * 32) << 16) + 8 * c, rr);
                     tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) out[(size_t)(8 * c + e) * ld + row] = __uint_as_float(rr[e]);
+                    if (lane < 16 && m >= 0 && m < kMono) {
+                        float4* dst = reinterpret_cast<float4*>(out + (size_t)m * ld + 8 * c);
+                        dst[0] = make_float4(__uint_as_float(rr[0]), __uint_as_float(rr[1]), __uint_as_float(rr[2]), __uint_as_float(rr[3]));
+                        if (8 * c + 4 < ld) dst[1] = make_float4(__uint_as_float(rr[4]), __uint_as_float(rr[5]), __uint_as_float(rr[6]), __uint_as_float(rr[7]));
+                    }
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 256);
+    if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
 // =======================================================================================
