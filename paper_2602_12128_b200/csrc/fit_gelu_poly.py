@@ -1,17 +1,17 @@
-"""Fits the polynomial the tensor-core phi kernels use for the exact (erf) GELU.
+"""Fits the constants the tensor-core phi kernels use for the exact (erf) GELU and its derivative.
 
-The normal CDF is evaluated as   Phi(x) ~ sat(1/2 + x * P(min(x^2, T)))   with sat = clamp to [0, 1]
-(one saturating fma), P of degree NCOEF-1 in t = x^2, fitted on |x| <= sqrt(T) so that
-x * P(x^2) ~ erf(x / sqrt 2) / 2.  Past sqrt(T) the expression grows linearly and saturates at 0 or 1.
-GELU(x) = x Phi(x);  GELU'(x) = Phi(x) + x exp(-x^2 / 2) / sqrt(2 pi).
+Forward:  Phi(x) ~ 1/2 + tanh(x (a + b x^2)) / 2  (one tanh.approx on the special-function unit per element),
+GELU(x) = x Phi(x); fit_tanh() gives a, b (fitted against erf(x / sqrt 2) on |x| <= 6) and the error before the
+hardware approximation's own 2^-11 relative error.
 
-Run:  python fit_gelu_poly.py   -> prints the coefficients (highest order first, as the Horner
-evaluation in hla_tc_phi.cuh lists them) and the maximum absolute errors of Phi and GELU in fp32.
-The constants in hla_tc_phi.cuh are this script's output for T = 16, NCOEF = 7 (used by the backward's GELU').
+Backward: GELU'(x) = Phi(x) + x pdf(x) through the same kind of tanh:
+    th = tanh(x (a + b x^2)),  r = 1/2 + th / 2,  y = 1/2 - th / 2,   GELU'(x) ~ r (1 + x (C0 + C1 x^2) y)
+(r y = (1 - th^2) / 4: the derivative of the tanh form with its inner derivative a free polynomial); fit_tanh_grad()
+fits a, b, C0, C1 against the exact GELU' on |x| <= 8.
 
-The forward evaluates Phi(x) ~ 1/2 + tanh(x (a + b x^2)) / 2 instead (one tanh.approx on the special-function
-unit); fit_tanh() gives a, b (fitted against erf(x / sqrt 2) on |x| <= 6) and the error before the hardware
-approximation's own 2^-11 relative error."""
+Run:  python fit_gelu_poly.py   -> prints both sets of constants and their maximum absolute errors; the constants in
+hla_tc_phi.cuh are this script's output.  (fit() / phi_f32() are the polynomial form
+Phi(x) ~ sat(1/2 + x P(min(x^2, T))) that earlier versions of the kernels used; kept for comparison.)"""
 import numpy as np
 from scipy.special import erf
 
@@ -57,7 +57,28 @@ def fit_tanh(iters=60):
     return c, np.abs(res(c)).max() / 2
 
 
+def gelu_grad_tanh(x, c):
+    t = x * x
+    th = np.tanh(x * (c[0] + c[1] * t))
+    r, y = 0.5 + 0.5 * th, 0.5 - 0.5 * th
+    return r * (1 + x * (c[2] + c[3] * t) * y)
+
+
+def gelu_grad_exact(x):
+    return 0.5 * (1 + erf(x / np.sqrt(2))) + x * np.exp(-x * x / 2) / np.sqrt(2 * np.pi)
+
+
+def fit_tanh_grad():
+    from scipy.optimize import least_squares
+    x = np.linspace(-8, 8, 32001)
+    ref = gelu_grad_exact(x)
+    c = least_squares(lambda c: gelu_grad_tanh(x, c) - ref, np.array([0.7988, 0.0353, 1.5976, 0.2117])).x
+    return c, np.abs(gelu_grad_tanh(x, c) - ref).max()
+
+
 if __name__ == "__main__":
+    c, err = fit_tanh_grad()
+    print("tanh form of GELU': a = %.8ff, b = %.8ff, C0 = %.8ff, C1 = %.8ff, max |error| = %.3e" % (*c, err))
     (a, b), err = fit_tanh()
     print("tanh form: a = %.8ff, b = %.8ff, max |Phi error| = %.3e" % (a, b, err))
     coef = fit()

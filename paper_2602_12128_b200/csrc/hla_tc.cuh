@@ -672,7 +672,7 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
     bool ok = true;
 
     if (warp == 0) {
-        if (lane == 0) {
+        if (elect_one()) {
             mbar_arrive_expect_tx(op_full, kMonoPad * DV * 2);
             for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + kBqOffOp + b * (kBlk / 2), &mapBq, op_full, b * 64, bh * kMonoPad);
             for (int it = 0; it < ntiles; ++it) {
@@ -684,7 +684,7 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (elect_one()) {
             // D2 = dO (K-major over g) * Csym (K-major over g); tile `it` is issued as soon as its dO tile has landed
             // and the group that owns the tile has read its previous D2, which is long before the group asks for it.
             const uint32_t idesc2 = idesc_bf16(128, kMonoPad, false, false);
@@ -705,7 +705,7 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
                 }
         }
     } else if (warp == 2) {
-        if (lane == 0) {
+        if (elect_one()) {
             // [dCsym | dzsym] += (operand rows)^T (MN-major, M = 64) * [dO | operand rows' first 8 columns] (MN-major, N = d + 8)
             const uint32_t idesc1 = idesc_bf16(64, kNC, true, true);
             for (int it = 0; it < ntiles; ++it) {

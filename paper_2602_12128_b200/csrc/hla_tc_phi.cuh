@@ -15,35 +15,16 @@
 namespace hla {
 namespace tc {
 
-// Phi(x) = 1/2 + erf(x / sqrt 2) / 2 evaluated as sat(1/2 + x P(min(x^2, 16))), sat = clamp to [0, 1] done by one
-// saturating fma (fit_gelu_poly.py: |error| < 1.1e-4, several times below the bf16 rounding of the result).  The
-// Horner steps run on pairs with the packed fp32 instructions (fma.rn.f32x2), which halve the issue slots.
+// Arithmetic on pairs uses the packed fp32 instructions (fma.rn.f32x2 and friends), which halve the issue slots.
 __device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
-__device__ __forceinline__ float fma_sat(float a, float b, float c) {
-    float d;
-    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float2 normal_cdf2(float2 x) {
-    const float2 xx = __fmul2_rn(x, x);
-    const float2 t = make_float2(fminf(xx.x, 16.f), fminf(xx.y, 16.f));
-    float2 p = splat2(2.816106894e-08f);
-    p = __ffma2_rn(p, t, splat2(-1.891893110e-06f));
-    p = __ffma2_rn(p, t, splat2(5.419046974e-05f));
-    p = __ffma2_rn(p, t, splat2(-8.789816123e-04f));
-    p = __ffma2_rn(p, t, splat2(9.112954582e-03f));
-    p = __ffma2_rn(p, t, splat2(-6.538836121e-02f));
-    p = __ffma2_rn(p, t, splat2(3.985269153e-01f));
-    return make_float2(fma_sat(x.x, p.x, 0.5f), fma_sat(x.y, p.y, 0.5f));
-}
 __device__ __forceinline__ float tanh_approx(float x) {
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 // GELU(x) = x Phi(x) through the special-function unit: Phi(x) = 1/2 + tanh(x (a + b x^2)) / 2 with a, b fitted to the erf
-// form (|Phi error| < 1.5e-4 before the 2^-11 relative error of tanh.approx).  It moves work from the FMA pipe, which
-// bounds the polynomial form, to the otherwise idle special-function pipe.
+// form (|Phi error| < 1.5e-4 before the 2^-11 relative error of tanh.approx).  A polynomial Phi kept the FMA pipe busier
+// and was slower; the special-function pipe is otherwise idle.
 __device__ __forceinline__ float2 gelu2_tanh(float2 x) {
     const float2 t = __fmul2_rn(x, x);
     const float2 u = __fmul2_rn(x, __ffma2_rn(t, splat2(0.0352821f), splat2(0.79880136f)));
@@ -51,17 +32,20 @@ __device__ __forceinline__ float2 gelu2_tanh(float2 x) {
     return __ffma2_rn(hx, make_float2(tanh_approx(u.x), tanh_approx(u.y)), hx);
 }
 __device__ __forceinline__ float2 gelu2(float2 x) { return gelu2_tanh(x); }
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// GELU'(x) = Phi(x) + x pdf(x),  pdf(x) = exp(-x^2 / 2) / sqrt(2 pi); Phi through the polynomial (the backward is not
-// bound by the FMA pipe alone, and a tanh-based Phi made no difference there).
+// GELU'(x) = Phi(x) + x pdf(x) through one tanh.approx per element:
+//   th = tanh(x (a + b x^2)),  r = 1/2 + th/2,  y = 1/2 - th/2,   GELU'(x) ~ r (1 + x (C0 + C1 x^2) y)
+// (r y = (1 - th^2) / 4, so this is the derivative of a tanh-form GELU whose inner derivative is a free polynomial);
+// a, b, C0, C1 are fitted against the exact derivative (fit_gelu_poly.py: |error| < 1.5e-4 before the 2^-11 relative
+// error of tanh.approx, < 1.3e-3 with it).  Nine packed instructions and two special-function instructions per pair
+// of elements; the polynomial Phi plus exp form needed sixteen.
 __device__ __forceinline__ float2 gelu_grad2(float2 x) {
-    const float2 a = __fmul2_rn(__fmul2_rn(x, x), splat2(-0.72134752f));     // -x^2 / 2 * log2(e)
-    const float2 e = make_float2(ex2_approx(a.x), ex2_approx(a.y));
-    return __ffma2_rn(__fmul2_rn(x, e), splat2(0.39894228f), normal_cdf2(x));
+    const float2 t = __fmul2_rn(x, x);
+    const float2 u = __fmul2_rn(x, __ffma2_rn(t, splat2(0.02936904f), splat2(0.69631102f)));
+    const float2 th = make_float2(tanh_approx(u.x), tanh_approx(u.y));
+    const float2 r = __ffma2_rn(th, splat2(0.5f), splat2(0.5f));
+    const float2 y = __ffma2_rn(th, splat2(-0.5f), splat2(0.5f));
+    const float2 v = __fmul2_rn(x, __ffma2_rn(t, splat2(-0.02169663f), splat2(1.7980557f)));
+    return __fmul2_rn(r, __ffma2_rn(v, y, splat2(1.f)));
 }
 
 struct PhiPtrs {
