@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;     // D1[b] at columns 128*b, D2[b] at columns 256 + 32*b
+    const uint32_t tmem = *tmem_slot;     // D1[b] at columns 128*b, D2[b] at columns 256 + 32*b, G[b] (bf16 pairs) at 320 + 64*b
     bool ok = true;
 
     if (warp == 0) {
@@ -182,19 +182,17 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
         }
     } else if (warp == 1) {
         if (lane == 0 && ntiles > 0) {      // D2[b] = G[b] * W2[m]
-            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G K-major, W2 operand K-major
-            const uint64_t gd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffG), 16, 1024);
+            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G from TMEM, W2 operand K-major
             const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 16, 1024);
             bool good = true;
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
                 if (!(mbar_wait(&g_full[b], par) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
                 tc_fence_after();
-                const uint64_t gd = desc_advance(gd0, b * Cfg::kXBytes), vd = desc_advance(vd0, m * Cfg::kW2Bytes);
+                const uint64_t vd = desc_advance(vd0, m * Cfg::kW2Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 256 + 32 * b, desc_advance(gd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32),
-                              idesc2, ks > 0 ? 1u : 0u);
+                    umma_bf16_ta(tmem + 256 + 32 * b, tmem + 320 + 64 * b + 8 * ks, desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32), idesc2, ks > 0 ? 1u : 0u);
                 umma_commit(&g_free[b]);
                 umma_commit(&d2_full[b]);
             }
@@ -230,7 +228,6 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
         }
     } else {
         const int quarter = warp & 3, part = (warp - kPfGeluWarp0) >> 2;
-        const int row = quarter * 32 + lane;
         for (int unit = 0; unit < nunits; ++unit) {
             const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
             const float* b1s = bias + m * (DV + 8);
@@ -240,7 +237,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
-            const uint32_t gblk = smem_u32(smem + Cfg::kOffG + b * Cfg::kXBytes);
+            const uint32_t tg = tmem + 320 + 64 * b + ((uint32_t)(quarter * 32) << 16) + part * (HC / 2);
             uint32_t r[HC];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) tmem_ld16(ta + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
@@ -257,11 +254,10 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
                     const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])), bb[e]));
                     w[e] = pack_bf16(g.x, g.y);
                 }
-                const uint32_t blk = gblk + (col >> 6) * kBlk;
-                st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
-                st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
+                tmem_st8(tg + 8 * c, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);      // the second layer's A operand lives in TMEM: no shared-memory round trip
             }
-            fence_proxy_async();
+            tmem_st_wait();
+            tc_fence_before();
             mbar_arrive(&g_full[b]);
         }
     }
@@ -357,7 +353,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* x_full = bars;           // [2]
     uint64_t* x_empty = bars + 2;      // [2] MMA commit
     uint64_t* h_full = bars + 4;       // [2] MMA commit
-    uint64_t* h_empty = bars + 6;      // [2] 512 arrivals
     uint64_t* dh_full = bars + 8;      // [2] 512 arrivals
     uint64_t* dh_free = bars + 10;     // [2] MMA commit
     uint64_t* dp_full = bars + 12;     // [2] 512 arrivals
@@ -388,7 +383,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             mbar_init(&x_full[i], 1);
             mbar_init(&x_empty[i], 1);
             mbar_init(&h_full[i], 1);
-            mbar_init(&h_empty[i], 512);
             mbar_init(&dh_full[i], 512);
             mbar_init(&dh_free[i], 1);
         }
@@ -434,7 +428,9 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
                 if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) { good = false; break; }
-                if (!mbar_wait(&h_empty[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
+                // h[b] also holds the dh operand of unit - 2 (written over the h columns that were read): it is free when
+                // that unit's dX product has completed
+                if (!mbar_wait(&dh_free[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
                 const uint64_t xd = desc_advance(xd0, st * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
 #pragma unroll
@@ -448,10 +444,9 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     } else if (warp == 1) {
         if (lane == 0 && ntiles > 0) {
             const uint32_t idesc_dg = idesc_bf16(128, DV, false, true);  // dg = dp (K-major) * W2^T (MN-major)
-            const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (K-major over hidden) * W1 as [in][hidden] (K-major)
+            const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (TMEM) * W1 as [in][hidden] (K-major)
             const uint64_t pd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp), 16, 1024);
             const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
-            const uint64_t hd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffDh), 16, 1024);
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), 16, 1024);
             bool good = mbar_wait(w_full, 0);
             // dg of `unit`; the epilogue of unit - 1 must have taken its dg into registers
@@ -471,11 +466,13 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 if (!mbar_wait(&dh_full[b], (unit >> 1) & 1)) { good = false; break; }
                 if (m == 0 && !mbar_wait(dx_empty, (it & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
-                const uint64_t hd = desc_advance(hd0, b * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
+                const uint64_t wd = desc_advance(wd0, m * Cfg::kW1Bytes);
+                // hidden units 16 ks .. 16 ks + 15 were written by the threads of part (16 ks) / HC as 8 packed columns
+                // at the start of their own column range plus ((16 ks) % HC) / 2
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 384, desc_advance(hd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, (ks >> 2) * (DV * 128) + (ks & 3) * 32), idesc2,
-                              (m > 0 || ks > 0) ? 1u : 0u);
+                    umma_bf16_ta(tmem + 384, tmem + 128 * b + ((16 * ks) / HC) * HC + ((16 * ks) % HC) / 2,
+                                 desc_advance(wd, (ks >> 2) * (DV * 128) + (ks & 3) * 32), idesc2, (m > 0 || ks > 0) ? 1u : 0u);
                 umma_commit(&dh_free[b]);
                 if (m == NMAPS - 1) umma_commit(dx_full);
             }
@@ -572,7 +569,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tmem + 128 * b + lane_base + part * HC;
-            const uint32_t dblk = smem_u32(smem + Cfg::kOffDh + b * Cfg::kXBytes);
             const float* bm = b1s + m * DV;
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
@@ -589,13 +585,11 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                     const float2 dh = __fmul2_rn(dg, gelu_grad2(h));
                     w[e] = pack_bf16(dh.x, dh.y);
                 }
-                const uint32_t blk = dblk + (col >> 6) * kBlk;
-                st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[0], w[1], w[2], w[3]);
-                st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[4], w[5], w[6], w[7]);
+                // dh as the A operand of the dX product, packed into the h columns this thread has already read
+                tmem_st8(ta + 8 * c, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
             }
+            tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(&h_empty[b]);
-            fence_proxy_async();
             mbar_arrive(&dh_full[b]);
             if (m == 0 && it > 0) drain_dx(it - 1);
         }
