@@ -56,7 +56,6 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     uint64_t* x_full = bars;           // [2] TMA   (x_full[1], x_empty[1] live at bars + 22, + 23)
     uint64_t* x_empty = bars + 1;      // [2] MMA commit
     uint64_t* d1_full = bars + 2;      // [2] MMA commit
-    uint64_t* d1_empty = bars + 4;     // [2] 512 arrivals
     uint64_t* g_full = bars + 6;       // 512 arrivals (bars + 7 unused)
     uint64_t* g_free = bars + 8;       // MMA commit (bars + 9 unused)
     uint64_t* d2_full = bars + 10;     // [2] MMA commit
@@ -95,7 +94,6 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
         mbar_init(x_empty1, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&d1_full[i], 1);
-            mbar_init(&d1_empty[i], 512);
             mbar_init(&g_full[i], 512);
             mbar_init(&g_free[i], 1);
             mbar_init(&d2_full[i], 1);
@@ -145,7 +143,9 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             bool good = mbar_wait(w_full, 0);
             for (int it = 0; it < nwork && good; ++it) {
                 const int b = it & 1, par = (it >> 1) & 1;      // accumulator buffer and Q stage alternate together
-                if (!(mbar_wait(b ? x_full1 : x_full, par) && mbar_wait(&d1_empty[b], par ^ 1))) { good = false; break; }
+                // D1[b] also holds the GELU tile of work item it - 2 (packed over the columns that were read): free when that
+                // item's second-layer product has completed
+                if (!(mbar_wait(b ? x_full1 : x_full, par) && mbar_wait(&g_free[b], par ^ 1))) { good = false; break; }
                 tc_fence_after();
                 const uint64_t xs = desc_advance(xd, b * Cfg::kXBytes);
 #pragma unroll
@@ -158,19 +158,18 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
         }
     } else if (warp == 1) {
         if (lane == 0 && nwork > 0) {      // D2[b] = G[b] * W2
-            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);           // G K-major, W2 operand K-major
-            const uint64_t gd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffG), 16, 1024);
+            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);           // G from TMEM, W2 operand K-major
             const uint64_t vd = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 16, 1024);
             bool good = true;
             for (int it = 0; it < nwork && good; ++it) {
                 const int b = it & 1, par = (it >> 1) & 1;
-                if (!(mbar_wait(g_full, it & 1) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
+                if (!(mbar_wait(&g_full[b], par) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 256 + 32 * b, desc_advance(gd0, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32),
-                              idesc2, ks > 0 ? 1u : 0u);
-                umma_commit(g_free);
+                    umma_bf16_ta(tmem + 256 + 32 * b, tmem + 128 * b + ((16 * ks) / HC) * HC + ((16 * ks) % HC) / 2,
+                                 desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32), idesc2, ks > 0 ? 1u : 0u);
+                umma_commit(&g_free[b]);
                 umma_commit(&d2_full[b]);
             }
             if (!good) report_timeout(status, 703);
@@ -284,7 +283,6 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     } else {
         // GELU: thread = token row x quarter of the hidden units
         const int quarter = warp & 3, part = (warp - kFqGeluWarp0) >> 2;
-        const int row = quarter * 32 + lane;
         for (int it = 0; it < nwork; ++it) {
             const int b = it & 1, par = (it >> 1) & 1;
             if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 707); }
@@ -292,15 +290,12 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
-            const uint32_t gblk = smem_u32(smem + Cfg::kOffG);
             uint32_t r[HC];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) tmem_ld16(ta + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
             tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(&d1_empty[b]);          // h is in registers: the next first-layer product may overwrite it
-            // All of the thread's GELU outputs are formed in registers first; the wait for the previous tile's second layer
-            // (the reader of the single G tile) then comes after the arithmetic instead of in front of it.
+            // The GELU outputs go back into TMEM as the second layer's A operand: bf16 pairs packed over the first half of
+            // the h columns this thread has just read (hidden units 16 c .. 16 c + 15 of its range -> 8 columns).
             uint32_t w[HC / 2];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
@@ -311,18 +306,12 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
                     w[8 * c + e] = pack_bf16(g.x, g.y);
                 }
             }
-            if (!mbar_wait(g_free, (it & 1) ^ 1)) { ok = false; report_timeout(status, 708); }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
 #pragma unroll
-            for (int c = 0; c < HC / 16; ++c) {
-                const int col = part * HC + 16 * c;
-                const uint32_t blk = gblk + (col >> 6) * kBlk;
-                st_shared_v4(blk + sw128_off(row, (col & 63) >> 3), w[8 * c], w[8 * c + 1], w[8 * c + 2], w[8 * c + 3]);
-                st_shared_v4(blk + sw128_off(row, ((col & 63) >> 3) + 1), w[8 * c + 4], w[8 * c + 5], w[8 * c + 6], w[8 * c + 7]);
-            }
-            fence_proxy_async();
-            mbar_arrive(g_full);
+            for (int c = 0; c < HC / 16; ++c)
+                tmem_st8(ta + 8 * c, w[8 * c], w[8 * c + 1], w[8 * c + 2], w[8 * c + 3], w[8 * c + 4], w[8 * c + 5], w[8 * c + 6], w[8 * c + 7]);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&g_full[b]);
         }
     }
     tc_fence_before();
