@@ -28,8 +28,7 @@ template <int DV> struct FqCfg {
     static constexpr int kNmma = DV + 16;                        // readout product: d value channels, then the normaliser column
     static constexpr int kB3Bytes = kNmma * 128;
     static constexpr int kOffX = 0;                              // 2 Q tiles (the load of a tile takes longer than a tile's arithmetic)
-    static constexpr int kOffG = 2 * kXBytes;                    // GELU output tile (one: its reader, the second-layer product, is short)
-    static constexpr int kOffW1 = kOffG + kXBytes;
+    static constexpr int kOffW1 = 2 * kXBytes;                   // (the GELU tile lives in TMEM)
     static constexpr int kOffW2 = kOffW1 + kW1Bytes;
     static constexpr int kOffB3 = kOffW2 + ((kW2Bytes + 1023) / 1024) * 1024;      // state operand of the current head
     static constexpr int kOffA = kOffB3 + ((kB3Bytes + 1023) / 1024) * 1024;        // monomial tile

@@ -64,13 +64,12 @@ constexpr int kPfThreads = 736;
 constexpr int kPfGeluWarp0 = 3, kPfFeatWarp0 = 19;
 
 template <int DV, int NMAPS> struct PfCfg {
-    static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;   // one stage is enough when a tile has three units
+    static constexpr int kXStages = 2;
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
     static constexpr int kW2Bytes = (DV / 64) * 2048;            // [16 rows][DV] bf16, K-major, per map
     static constexpr int kOffX = 0;
-    static constexpr int kOffG = kXStages * kXBytes;             // 2 GELU output tiles
-    static constexpr int kOffW1 = kOffG + 2 * kXBytes;
+    static constexpr int kOffW1 = kXStages * kXBytes;            // (the GELU tiles live in TMEM)
     static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;
     static constexpr int kOffBias = kOffW2 + NMAPS * kW2Bytes;   // per map: b1[DV], b2[8] floats
     static constexpr int kOffBars = kOffBias + NMAPS * (DV + 8) * 4;
@@ -316,13 +315,12 @@ constexpr int kPbThreads = 608;
 constexpr int kPbEpiWarp0 = 3;
 
 template <int DV, int NMAPS> struct PbCfg {
-    static constexpr int kXStages = (DV == 128 && NMAPS == 3) ? 1 : 2;
+    static constexpr int kXStages = 2;
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
     static constexpr int kW2tBytes = (DV / 64) * 2048;           // per map: [16 K rows][DV] bf16, MN-major B operand of the dg product
     static constexpr int kOffX = 0;
-    static constexpr int kOffDh = kXStages * kXBytes;            // 2 dh tiles (A operand of the second MMA)
-    static constexpr int kOffW1 = kOffDh + 2 * kXBytes;
+    static constexpr int kOffW1 = kXStages * kXBytes;            // (the dh tiles live in TMEM)
     static constexpr int kOffDp = kOffW1 + NMAPS * kW1Bytes;     // one swizzled block = 4 dp tiles [128 tok][16] (K slices 0..3)
     static constexpr int kOffW2t = kOffDp + kBlk;
     static constexpr int kOffB1 = kOffW2t + NMAPS * kW2tBytes;   // fp32 [NMAPS][DV]
