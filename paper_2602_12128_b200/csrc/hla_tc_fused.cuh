@@ -33,7 +33,12 @@ template <int DV> struct FqCfg {
     static constexpr int kOffB3 = kOffW2 + ((kW2Bytes + 1023) / 1024) * 1024;      // state operand of the current head
     static constexpr int kOffA = kOffB3 + ((kB3Bytes + 1023) / 1024) * 1024;        // monomial tile
     static constexpr int kOffO = kOffA + kBlk;                   // O staging tile
-    static constexpr int kOffBias = kOffO + kXBytes;             // b1[DV], b2[8] floats
+    // b1 is added on the tensor cores by a ninth K step of the first-layer product: A = a constant tile whose K column
+    // 0 is 1, B = a tile whose K row 0 is b1 (both zero elsewhere)
+    static constexpr int kOffOnes = kOffO + kXBytes;             // [128 rows][64 K] bf16, K-major (16 K columns used)
+    static constexpr int kB1Bytes = (DV / 64) * 2048;            // [16 K rows][DV] bf16, MN-major
+    static constexpr int kOffB1 = kOffOnes + kBlk;
+    static constexpr int kOffBias = kOffB1 + kB1Bytes;           // b1[DV] (unused by the kernel), b2[8] floats
     static constexpr int kOffBars = kOffBias + (DV + 8) * 4;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
@@ -84,6 +89,12 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
         uint8_t* base = smem + Cfg::kOffW2 + (j >> 6) * 2048;
         *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = W2g[j * 6 + o];
     }
+    for (int i = tid; i < (kBlk + Cfg::kB1Bytes) / 16; i += kFqThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffOnes)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    for (int i = tid; i < kTileTokens; i += kFqThreads)
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffOnes + sw128_off(i, 0)) = __float2bfloat16_rn(1.f);
+    for (int j = tid; j < DV; j += kFqThreads)      // K row 0 of the MN-major tile: 64-column block j / 64, no swizzle in row 0
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffB1 + (j >> 6) * 2048 + (j & 63) * 2) = b1g[j];
     for (int j = tid; j < DV + 8; j += kFqThreads) bias[j] = j < DV ? __bfloat162float(b1g[j]) : (j - DV < 6 ? __bfloat162float(b2g[j - DV]) : 0.f);
     fence_proxy_async();
     if (tid == 0) {
@@ -139,6 +150,8 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             const uint32_t idesc1 = idesc_bf16(128, DV, false, true);   // Q K-major, W1 [in][hidden] MN-major
             const uint64_t xd = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
             const uint64_t wd = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
+            const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffOnes), 16, 1024);
+            const uint64_t bd = smem_desc_sw128(smem_u32(smem + Cfg::kOffB1), 2048, 1024);
             bool good = mbar_wait(w_full, 0);
             for (int it = 0; it < nwork && good; ++it) {
                 const int b = it & 1, par = (it >> 1) & 1;      // accumulator buffer and Q stage alternate together
@@ -150,6 +163,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 128 * b, desc_advance(xs, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
+                umma_bf16(tmem + 128 * b, od, bd, idesc1, 1u);      // + 1 * b1
                 umma_commit(&d1_full[b]);
                 umma_commit(b ? x_empty1 : x_empty);
             }
@@ -298,10 +312,9 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             uint32_t w[HC / 2];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
-                const float2* bb = reinterpret_cast<const float2*>(bias + part * HC + 16 * c);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])), bb[e]));
+                    const float2 g = gelu2(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
                     w[8 * c + e] = pack_bf16(g.x, g.y);
                 }
             }

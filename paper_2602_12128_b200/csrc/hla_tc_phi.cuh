@@ -71,7 +71,12 @@ template <int DV, int NMAPS> struct PfCfg {
     static constexpr int kOffX = 0;
     static constexpr int kOffW1 = kXStages * kXBytes;            // (the GELU tiles live in TMEM)
     static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;
-    static constexpr int kOffBias = kOffW2 + NMAPS * kW2Bytes;   // per map: b1[DV], b2[8] floats
+    // The first-layer bias rides on the tensor cores as a ninth K step: A = a constant tile whose K column 0 is 1,
+    // B = per map a tile whose K row 0 is b1 (both zero elsewhere), so the arithmetic warps add nothing.
+    static constexpr int kOffOnes = kOffW2 + ((NMAPS * kW2Bytes + 1023) / 1024) * 1024;   // [128 rows][64 K] bf16, K-major (16 K columns used)
+    static constexpr int kB1Bytes = (DV / 64) * 2048;            // per map: [16 K rows][DV] bf16, MN-major
+    static constexpr int kOffB1 = kOffOnes + kBlk;
+    static constexpr int kOffBias = kOffB1 + NMAPS * kB1Bytes;   // per map: b1[DV] (unused by the kernel), b2[8] floats
     static constexpr int kOffBars = kOffBias + NMAPS * (DV + 8) * 4;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
@@ -114,6 +119,14 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
         const int m = i / (DV * 6), j = (i / 6) % DV, o = i % 6;
         uint8_t* base = smem + Cfg::kOffW2 + m * Cfg::kW2Bytes + (j >> 6) * 2048;
         *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = P.W2[m][j * 6 + o];
+    }
+    for (int i = tid; i < (kBlk + NMAPS * Cfg::kB1Bytes) / 16; i += kPfThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffOnes)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    for (int i = tid; i < kTileTokens; i += kPfThreads)
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffOnes + sw128_off(i, 0)) = __float2bfloat16_rn(1.f);
+    for (int i = tid; i < NMAPS * DV; i += kPfThreads) {
+        const int m = i / DV, j = i % DV;       // K row 0 of the MN-major tile: 64-column block j / 64, no swizzle in row 0
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffB1 + m * Cfg::kB1Bytes + (j >> 6) * 2048 + (j & 63) * 2) = P.b1[m][j];
     }
     for (int i = tid; i < NMAPS * (DV + 8); i += kPfThreads) {
         const int m = i / (DV + 8), j = i % (DV + 8);
@@ -164,6 +177,8 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             const uint32_t idesc1 = idesc_bf16(128, DV, false, true);   // X K-major, W1 [in][hidden] MN-major
             const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
+            const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffOnes), 16, 1024);
+            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffB1), 2048, 1024);
             bool good = mbar_wait(w_full, 0);
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
@@ -174,6 +189,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
+                umma_bf16(tmem + 128 * b, od, desc_advance(bd0, m * Cfg::kB1Bytes), idesc1, 1u);      // + 1 * b1
                 umma_commit(&d1_full[b]);
                 if (m == NMAPS - 1) umma_commit(&x_empty[st]);
             }
@@ -228,8 +244,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     } else {
         const int quarter = warp & 3, part = (warp - kPfGeluWarp0) >> 2;
         for (int unit = 0; unit < nunits; ++unit) {
-            const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
-            const float* b1s = bias + m * (DV + 8);
+            const int b = unit & 1, par = (unit >> 1) & 1;
             if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 504); }
             if (ok && !mbar_wait(&g_free[b], par ^ 1)) { ok = false; report_timeout(status, 505); }
             ok = __all_sync(0xffffffffu, ok);
@@ -245,12 +260,10 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
             mbar_arrive(&d1_empty[b]);          // h is in registers: the next first-layer product may overwrite it
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
-                const int col = part * HC + 16 * c;
-                const float2* bb = reinterpret_cast<const float2*>(b1s + col);
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2(__fadd2_rn(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])), bb[e]));
+                    const float2 g = gelu2(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
                     w[e] = pack_bf16(g.x, g.y);
                 }
                 tmem_st8(tg + 8 * c, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);      // the second layer's A operand lives in TMEM: no shared-memory round trip
@@ -323,8 +336,10 @@ template <int DV, int NMAPS> struct PbCfg {
     static constexpr int kOffW1 = kXStages * kXBytes;            // (the dh tiles live in TMEM)
     static constexpr int kOffDp = kOffW1 + NMAPS * kW1Bytes;     // one swizzled block = 4 dp tiles [128 tok][16] (K slices 0..3)
     static constexpr int kOffW2t = kOffDp + kBlk;
-    static constexpr int kOffB1 = kOffW2t + NMAPS * kW2tBytes;   // fp32 [NMAPS][DV]
-    static constexpr int kOffBars = kOffB1 + NMAPS * DV * 4;
+    // b1 is added on the tensor cores by a ninth K step of the h product: A = K columns 32..47 of the dp block (column
+    // 32 is a constant 1, never written again; the dp tiles use columns 0..31), B = per map a tile whose K row 0 is b1
+    static constexpr int kOffB1 = kOffW2t + NMAPS * kW2tBytes;   // per map: [16 K rows][DV] bf16, MN-major
+    static constexpr int kOffBars = kOffB1 + NMAPS * kW2tBytes;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
@@ -346,7 +361,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    float* b1s = reinterpret_cast<float*>(smem + Cfg::kOffB1);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* x_full = bars;           // [2]
     uint64_t* x_empty = bars + 2;      // [2] MMA commit
@@ -373,8 +387,15 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * 2048;
         *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? P.W2[m][j * 6 + (k % 6)] : __float2bfloat16_rn(0.f);
     }
-    for (int i = tid; i < NMAPS * DV; i += kPbThreads) b1s[i] = __bfloat162float(P.b1[i / DV][i % DV]);
     for (int i = tid; i < kBlk / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < NMAPS * Cfg::kW2tBytes / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffB1)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    for (int i = tid; i < kTileTokens; i += kPbThreads)
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffDp + sw128_off(i, 4)) = __float2bfloat16_rn(1.f);
+    for (int i = tid; i < NMAPS * DV; i += kPbThreads) {
+        const int m = i / DV, j = i % DV;       // K row 0 of the MN-major tile: 64-column block j / 64, no swizzle in row 0
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffB1 + m * Cfg::kW2tBytes + (j >> 6) * 2048 + (j & 63) * 2) = P.b1[m][j];
+    }
     fence_proxy_async();
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -422,6 +443,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             const uint32_t idesc1 = idesc_bf16(128, DV, false, true);    // X K-major, W1 [in][hidden] MN-major
             const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
+            const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp) + 64, 16, 1024);
+            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffB1), 2048, 1024);
             bool good = mbar_wait(w_full, 0);
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
@@ -434,6 +457,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
+                umma_bf16(tmem + 128 * b, od, desc_advance(bd0, m * Cfg::kW2tBytes), idesc1, 1u);      // + 1 * b1
                 umma_commit(&h_full[b]);
                 if (m == NMAPS - 1) umma_commit(&x_empty[st]);
             }
@@ -567,18 +591,15 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tmem + 128 * b + lane_base + part * HC;
-            const float* bm = b1s + m * DV;
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
                 uint32_t r[16];
                 tmem_ld16(ta + 16 * c, r);
                 tmem_ld_wait();
-                const int col = part * HC + 16 * c;
-                const float2* bb = reinterpret_cast<const float2*>(bm + col);
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float2 h = __fadd2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), bb[e]);
+                    const float2 h = make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
                     const float2 dg = make_float2(__uint_as_float(dgr[16 * c + 2 * e]), __uint_as_float(dgr[16 * c + 2 * e + 1]));
                     const float2 dh = __fmul2_rn(dg, gelu_grad2(h));
                     w[e] = pack_bf16(dh.x, dh.y);
