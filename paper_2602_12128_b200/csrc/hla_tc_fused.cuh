@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     for (int i = tid; i < DV * 6; i += kFqThreads) {
         const int j = i / 6, o = i % 6;
         uint8_t* base = smem + Cfg::kOffW2 + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = W2g[j * 6 + o];
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = half_bf16(W2g[j * 6 + o]);
     }
     for (int i = tid; i < (kBlk + Cfg::kB1Bytes) / 16; i += kFqThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffOnes)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             for (int c = 0; c < HC / 16; ++c) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
+                    const float2 g = gelu2_twice(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
                     w[8 * c + e] = pack_bf16(g.x, g.y);
                 }
             }

@@ -24,28 +24,29 @@ __device__ __forceinline__ float tanh_approx(float x) {
 }
 // GELU(x) = x Phi(x) through the special-function unit: Phi(x) = 1/2 + tanh(x (a + b x^2)) / 2 with a, b fitted to the erf
 // form (|Phi error| < 1.5e-4 before the 2^-11 relative error of tanh.approx).  A polynomial Phi kept the FMA pipe busier
-// and was slower; the special-function pipe is otherwise idle.
-__device__ __forceinline__ float2 gelu2_tanh(float2 x) {
+// and was slower; the special-function pipe is otherwise idle.  The kernels form 2 GELU(x) = x + x tanh(..) and stage the
+// second-layer weights halved (exact in bf16), which saves the multiplication by 1/2.
+__device__ __forceinline__ float2 gelu2_twice(float2 x) {
     const float2 t = __fmul2_rn(x, x);
     const float2 u = __fmul2_rn(x, __ffma2_rn(t, splat2(0.0352821f), splat2(0.79880136f)));
-    const float2 hx = __fmul2_rn(x, splat2(0.5f));
-    return __ffma2_rn(hx, make_float2(tanh_approx(u.x), tanh_approx(u.y)), hx);
+    return __ffma2_rn(x, make_float2(tanh_approx(u.x), tanh_approx(u.y)), x);
 }
-__device__ __forceinline__ float2 gelu2(float2 x) { return gelu2_tanh(x); }
+__device__ __forceinline__ __nv_bfloat16 half_bf16(__nv_bfloat16 w) { return __float2bfloat16_rn(0.5f * __bfloat162float(w)); }
 // GELU'(x) = Phi(x) + x pdf(x) through one tanh.approx per element:
-//   th = tanh(x (a + b x^2)),  r = 1/2 + th/2,  y = 1/2 - th/2,   GELU'(x) ~ r (1 + x (C0 + C1 x^2) y)
-// (r y = (1 - th^2) / 4, so this is the derivative of a tanh-form GELU whose inner derivative is a free polynomial);
-// a, b, C0, C1 are fitted against the exact derivative (fit_gelu_poly.py: |error| < 1.5e-4 before the 2^-11 relative
-// error of tanh.approx, < 1.3e-3 with it).  Nine packed instructions and two special-function instructions per pair
-// of elements; the polynomial Phi plus exp form needed sixteen.
-__device__ __forceinline__ float2 gelu_grad2(float2 x) {
+//   th = tanh(x (a + b x^2)),   2 GELU'(x) ~ (1 + th) (1 + V (1 - th)) = 1 + V + th (1 - V th),   V = x (C0 + C1 x^2) / 2
+// (the derivative of a tanh-form GELU whose inner derivative is a free polynomial); a, b, C0, C1 are fitted against the
+// exact derivative (fit_gelu_poly.py: |error| < 1.5e-4 before the 2^-11 relative error of tanh.approx, < 1.3e-3 with
+// it).  The kernel evaluates it with -V (negated constants) so that every step is one packed multiply or fma, and the
+// factor 1/2 sits in the staged W2^T of the dg product (exact in bf16): 9 packed + 2 special-function instructions
+// per pair of elements; the polynomial Phi plus exp form needed sixteen.
+__device__ __forceinline__ float2 gelu_grad2_twice(float2 x) {
     const float2 t = __fmul2_rn(x, x);
     const float2 u = __fmul2_rn(x, __ffma2_rn(t, splat2(0.02936904f), splat2(0.69631102f)));
     const float2 th = make_float2(tanh_approx(u.x), tanh_approx(u.y));
-    const float2 r = __ffma2_rn(th, splat2(0.5f), splat2(0.5f));
-    const float2 y = __ffma2_rn(th, splat2(-0.5f), splat2(0.5f));
-    const float2 v = __fmul2_rn(x, __ffma2_rn(t, splat2(-0.02169663f), splat2(1.7980557f)));
-    return __fmul2_rn(r, __ffma2_rn(v, y, splat2(1.f)));
+    const float2 vn = __fmul2_rn(x, __ffma2_rn(t, splat2(0.010848315f), splat2(-0.89902785f)));   // -V
+    const float2 a1 = __ffma2_rn(vn, th, splat2(1.f));          // 1 - V th
+    const float2 b1 = __ffma2_rn(th, a1, splat2(1.f));          // 1 + th (1 - V th)
+    return __ffma2_rn(vn, splat2(-1.f), b1);                    // + V
 }
 
 struct PhiPtrs {
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     for (int i = tid; i < NMAPS * DV * 6; i += kPfThreads) {
         const int m = i / (DV * 6), j = (i / 6) % DV, o = i % 6;
         uint8_t* base = smem + Cfg::kOffW2 + m * Cfg::kW2Bytes + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = P.W2[m][j * 6 + o];
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = half_bf16(P.W2[m][j * 6 + o]);
     }
     for (int i = tid; i < (kBlk + NMAPS * Cfg::kB1Bytes) / 16; i += kPfThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffOnes)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
@@ -263,7 +264,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
+                    const float2 g = gelu2_twice(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
                     w[e] = pack_bf16(g.x, g.y);
                 }
                 tmem_st8(tg + 8 * c, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);      // the second layer's A operand lives in TMEM: no shared-memory round trip
@@ -385,7 +386,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     for (int i = tid; i < NMAPS * 16 * DV; i += kPbThreads) {
         const int m = i / (16 * DV), k = (i / DV) & 15, j = i % DV;
         uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? P.W2[m][j * 6 + (k % 6)] : __float2bfloat16_rn(0.f);
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? half_bf16(P.W2[m][j * 6 + (k % 6)]) : __float2bfloat16_rn(0.f);
     }
     for (int i = tid; i < kBlk / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
     for (int i = tid; i < NMAPS * Cfg::kW2tBytes / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffB1)[i] = make_uint4(0, 0, 0, 0);
@@ -601,7 +602,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 for (int e = 0; e < 8; ++e) {
                     const float2 h = make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
                     const float2 dg = make_float2(__uint_as_float(dgr[16 * c + 2 * e]), __uint_as_float(dgr[16 * c + 2 * e + 1]));
-                    const float2 dh = __fmul2_rn(dg, gelu_grad2(h));
+                    const float2 dh = __fmul2_rn(dg, gelu_grad2_twice(h));      // dg holds dg / 2 (halved W2^T)
                     w[e] = pack_bf16(dh.x, dh.y);
                 }
                 // dh as the A operand of the dX product, packed into the h columns this thread has already read
