@@ -125,3 +125,43 @@ def test_forward_backward_with_phi_stage_by_stage(shape):
     same_q, same_k = ~flip_q.any(axis=-1), ~flip_k.any(axis=(2, 4))
     assert relerr(dQ[same_q], rQ[same_q]) < TOL["bf16"]
     assert relerr(dK[same_k], rK[same_k]) < TOL["bf16"]
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_phi_with_large_biases(d):
+    """First-layer biases of the size of the pre-activations themselves (the kernels add b1 inside the first-layer
+    product): features against the oracle's phi, and the phi backward at the feature gradients the GPU produced."""
+    s = synth.HlaShape(f"bias{d}", 1, 2, 300, d, "bf16", "rms_qk")
+    Q, K, V = synth.make_qkv(s)
+    dO = synth.make_dO(s)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    rng = np.random.default_rng(5)
+    bf = lambda a: torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).float().numpy()
+
+    def with_bias(w):
+        W1, b1, W2, b2 = w
+        return W1, bf(rng.standard_normal(b1.shape)), W2, bf(0.5 * rng.standard_normal(b2.shape))
+
+    pq, pk = with_bias(pq), [with_bias(w) for w in pk]
+    run = GpuRun(s, "mlp", EPS)
+    run.set_weights(pq, pk)
+    run.forward(Q, K, V)
+    dQ, dK, dV = run.backward(dO)
+    gq, gk = run.features()
+    ref_q = orc.phi_mlp(f64(Q).reshape(-1, d), *pq).reshape(gq.shape)
+    assert relerr(gq, ref_q) < TOL["bf16"]
+    for f in range(s.F):
+        ref_k = orc.phi_mlp(f64(K).reshape(-1, d), *pk[f]).reshape(gq.shape)
+        assert relerr(gk[:, :, f], ref_k) < TOL["bf16"]
+    nq = s.B * s.H * s.N * s.d_phi
+    dqf = run.region("dqf", nq, (s.B, s.H, s.N, s.d_phi))
+    dkf = run.region("dkf", nq * s.F, (s.B, s.H, s.F, s.N, s.d_phi))
+    pre_q = orc.phi_mlp(f64(Q).reshape(-1, d), *pq, relu=False).reshape(gq.shape)
+    pre_k = np.stack([orc.phi_mlp(f64(K).reshape(-1, d), *w, relu=False).reshape(gq.shape) for w in pk], axis=2)
+    same_q = ~((gq > 0) != (pre_q > 0)).any(axis=-1)
+    same_k = ~((gk > 0) != (pre_k > 0)).any(axis=(2, 4))
+    assert same_q.mean() > 0.95 and same_k.mean() > 0.9
+    rQ = orc.phi_mlp_backward(f64(Q).reshape(-1, d), *pq, dqf.reshape(-1, s.d_phi)).reshape(Q.shape)
+    rK = sum(orc.phi_mlp_backward(f64(K).reshape(-1, d), *pk[f], dkf[:, :, f].reshape(-1, s.d_phi)).reshape(K.shape) for f in range(s.F))
+    assert relerr(dQ[same_q], rQ[same_q]) < TOL["bf16"]
+    assert relerr(dK[same_k], rK[same_k]) < TOL["bf16"]
