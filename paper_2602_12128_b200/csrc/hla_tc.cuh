@@ -21,6 +21,7 @@
 #pragma once
 #include "../../include/hla.h"
 #include "hla_common.cuh"
+#include <utility>
 #include "hla_tc_prim.cuh"
 
 namespace hla {
@@ -98,6 +99,24 @@ inline bool make_map_2d(CUtensorMap* m, const void* ptr, size_t rows, int cols, 
     cuuint32_t es[2] = {1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launch with programmatic stream serialization (see grid_dependency_wait): the kernel's blocks may start while the
+// previous kernel of the stream drains; every kernel launched this way waits for its predecessor before it touches
+// global memory that the library's kernels write or read.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 // ---- small device helpers ----------------------------------------------------------------
@@ -248,7 +267,9 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     const int ntiles = max(0, min(tiles, tile0 + tiles_per) - tile0);
     float* out = part + ((size_t)bh * S + s) * kMono * ld;
 
+    grid_launch_dependents();
     if (ntiles == 0) {   // an empty split contributes zeros
+        grid_dependency_wait();
         for (int i = tid; i < kMono * ld; i += kSbThreads) out[i] = 0.f;
         return;
     }
@@ -277,6 +298,7 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    grid_dependency_wait();
     bool ok = true;
 
     if (warp == 0) {
@@ -385,6 +407,8 @@ __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __rest
                                                              __nv_bfloat16* __restrict__ b3, __nv_bfloat16* __restrict__ bq, int S, int ld) {
     __shared__ float sm[8][kMaxD + 8];
     const int m0 = 8 * blockIdx.x, bh = blockIdx.y, tid = threadIdx.x;
+    grid_launch_dependents();
+    grid_dependency_wait();
     const size_t n_per = (size_t)kMono * ld;
     for (int i = tid; i < 8 * ld; i += 256) {
         const int mm = i / ld, col = i - mm * ld, m = m0 + mm;
@@ -452,6 +476,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
     const long long total = (long long)BH * tiles_per_head;
     const int w0 = (int)(total * blockIdx.x / gridDim.x), w1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
     const int nwork = w1 - w0;
+    grid_launch_dependents();
 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -475,6 +500,7 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    grid_dependency_wait();
     bool ok = true;
 
     if (warp == kRoMmaWarp) {
@@ -639,11 +665,12 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
     const int tile0 = s * tiles_per;
     const int ntiles = max(0, min(tiles, tile0 + tiles_per) - tile0);
     float* out = part + ((size_t)bh * S + s) * kMono * ld;
+    grid_launch_dependents();
     if (ntiles == 0) {
+        grid_dependency_wait();
         for (int i = tid; i < kMono * ld; i += kBqThreads) out[i] = 0.f;
         return;
     }
-    if (tid < 64) zsym[tid] = tid < kMono ? state[((size_t)bh * kMono + tid) * ld + DV] : 0.f;
     if (tid == 0) {
         for (int i = 0; i < kBqStages; ++i) {
             mbar_init(&full_do[i], 1);
@@ -669,6 +696,12 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    grid_dependency_wait();
+    // (zsym is read by the generator warps only; the named barrier keeps the other warps out of it)
+    if (warp >= 4) {
+        if (tid - 128 < 64) zsym[tid - 128] = tid - 128 < kMono ? state[((size_t)bh * kMono + tid - 128) * ld + DV] : 0.f;
+        named_barrier(1, 128 * kBqGroups);
+    }
     bool ok = true;
 
     if (warp == 0) {
@@ -883,6 +916,7 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
     const long long total = (long long)BH * tiles_per_head;
     const int w0 = (int)(total * blockIdx.x / gridDim.x), w1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
     const int nwork = w1 - w0;
+    grid_launch_dependents();
 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -909,6 +943,7 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;     // D3[grp] at columns 128*grp, D4[grp] at columns 256 + 64*grp
+    grid_dependency_wait();
     bool ok = true;
 
     if (warp == 0) {
@@ -1086,17 +1121,17 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     if (!set_smem(tc_state_build_kernel<DV>, kSbSmem) || !set_smem(tc_readout_kernel<DV>, RoCfg<DV>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
     rec.begin("tc_state_build");
-    tc_state_build_kernel<DV><<<dim3(D.S, BH), kSbThreads, kSbSmem, st>>>(mapV, kf, part, D.N, D.S, D.ld, status);
+    launch_pdl(tc_state_build_kernel<DV>, dim3(D.S, BH), dim3(kSbThreads), kSbSmem, st, mapV, kf, part, D.N, D.S, D.ld, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    tc_reduce_emit_kernel<DV><<<dim3(8, BH), 256, 0, st>>>(part, state, b3, bq, D.S, D.ld);
+    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, state, b3, bq, D.S, D.ld);
     if (!rec.end()) return HLA_ERR_CUDA;
     if (!readout) return HLA_OK;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_readout");
-    tc_readout_kernel<DV><<<grid, kRoThreads, RoCfg<DV>::kSmem, st>>>(mapB3, mapO, qf, eta, D.N, BH, D.eps, status);
+    launch_pdl(tc_readout_kernel<DV>, grid, dim3(kRoThreads), RoCfg<DV>::kSmem, st, mapB3, mapO, qf, eta, D.N, BH, D.eps, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
@@ -1127,16 +1162,16 @@ inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, con
     if (!set_smem(tc_bwd_query_kernel<DV>, kBqSmem) || !set_smem(tc_bwd_key_kernel<DV>, BkCfg<DV>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
     rec.begin("tc_bwd_query");
-    tc_bwd_query_kernel<DV><<<dim3(D.S, BH), kBqThreads, kBqSmem, st>>>(mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps, status);
+    launch_pdl(tc_bwd_query_kernel<DV>, dim3(D.S, BH), dim3(kBqThreads), kBqSmem, st, mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    tc_reduce_emit_kernel<DV><<<dim3(8, BH), 256, 0, st>>>(part, dstate, bd3, bdq, D.S, D.ld);
+    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld);
     if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_bwd_key");
-    tc_bwd_key_kernel<DV><<<grid, kBkThreads, BkCfg<DV>::kSmem, st>>>(mapV, mapBd3, mapBdq, mapdV, kf, dstate, dkf, D.N, BH, D.ld, status);
+    launch_pdl(tc_bwd_key_kernel<DV>, grid, dim3(kBkThreads), BkCfg<DV>::kSmem, st, mapV, mapBd3, mapBdq, mapdV, kf, dstate, dkf, D.N, BH, D.ld, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 

@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     using Cfg = FqCfg<DV>;
     constexpr int HC = DV / 4;          // hidden units per GELU thread
     extern __shared__ uint8_t smem_raw[];
+    grid_launch_dependents();
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     float* bias = reinterpret_cast<float*>(smem + Cfg::kOffBias);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
@@ -130,6 +131,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;     // D1[b] at columns 128*b, D2[b] at 256 + 32*b, readout accumulator at 320
+    grid_dependency_wait();
     bool ok = true;
 
     if (warp == 0) {
@@ -344,7 +346,7 @@ inline hla_status launch_phiq_readout(const Plan& P, const Dims& D, int BH, cons
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_phiq_readout");
-    tc_phiq_readout_kernel<DV><<<grid, kFqThreads, FqCfg<DV>::kSmem, rec.st>>>(
+    launch_pdl(tc_phiq_readout_kernel<DV>, grid, dim3(kFqThreads), FqCfg<DV>::kSmem, rec.st, 
         mapQ, mapW1, mapB3, mapO, static_cast<const __nv_bfloat16*>(phi_q->b1), static_cast<const __nv_bfloat16*>(phi_q->W2),
         static_cast<const __nv_bfloat16*>(phi_q->b2), reinterpret_cast<float*>(ws + L.qf), reinterpret_cast<float*>(ws + L.eta), D.N, BH, D.eps,
         reinterpret_cast<int*>(ws + L.status));

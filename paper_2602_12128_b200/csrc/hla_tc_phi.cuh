@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     constexpr int HC = DV / 4;          // hidden units per epilogue thread
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
+    grid_launch_dependents();
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     float* bias = reinterpret_cast<float*>(smem + Cfg::kOffBias);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
@@ -157,6 +158,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __g
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;     // D1[b] at columns 128*b, D2[b] at columns 256 + 32*b, G[b] (bf16 pairs) at 320 + 64*b
+    grid_dependency_wait();
     bool ok = true;
 
     if (warp == 0) {
@@ -299,7 +301,7 @@ inline hla_status launch_phi_forward_k(const Dims& D, int BH, const hla_mlp* phi
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     rec.begin("tc_phi_forward_k");
-    tc_phi_forward_kernel<DV, 3, true><<<grid, kPfThreads, PfCfg<DV, 3>::kSmem, rec.st>>>(mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
+    launch_pdl(tc_phi_forward_kernel<DV, 3, true>, grid, dim3(kPfThreads), PfCfg<DV, 3>::kSmem, rec.st, mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
@@ -361,6 +363,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     constexpr int HC = DV / 4;
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
+    grid_launch_dependents();
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* x_full = bars;           // [2]
@@ -423,6 +426,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;     // h[b] at columns 128*b, dg at 256, dX at 384
+    grid_dependency_wait();
     bool ok = true;
 
     if (warp == 0) {
@@ -645,11 +649,11 @@ inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     cudaStream_t st = rec.st;
     rec.begin("tc_phi_backward_q");
-    tc_phi_backward_kernel<DV, 1, false><<<grid, kPbThreads, PbCfg<DV, 1>::kSmem, st>>>(
+    launch_pdl(tc_phi_backward_kernel<DV, 1, false>, grid, dim3(kPbThreads), PbCfg<DV, 1>::kSmem, st, 
         mapQ, mq, pq, reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), static_cast<__nv_bfloat16*>(dQ), rows, D.N, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_phi_backward_k");
-    tc_phi_backward_kernel<DV, 3, true><<<grid, kPbThreads, PbCfg<DV, 3>::kSmem, st>>>(
+    launch_pdl(tc_phi_backward_kernel<DV, 3, true>, grid, dim3(kPbThreads), PbCfg<DV, 3>::kSmem, st, 
         mapK, mk, pk, reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), static_cast<__nv_bfloat16*>(dK), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }

@@ -24,6 +24,15 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ---- programmatic dependent launch --------------------------------------------------
+// Every tensor-core kernel is launched with the programmatic-stream-serialization attribute: its blocks may be
+// scheduled while the previous kernel of the stream is still draining, run their set-up (barriers, TMEM, weight
+// staging) and then wait here until the previous kernel has completed and its writes are visible.  No global memory
+// that another kernel of the library writes or reads is touched before this wait.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel's blocks be scheduled as soon as every block of this one has started.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier -------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
