@@ -118,6 +118,17 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
+// The same without the attribute, for a kernel that reads caller-provided memory (the phi weights) before its wait and
+// may directly follow a kernel of the caller that wrote it: it starts only after everything before it has completed.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_serial(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ---- small device helpers ----------------------------------------------------------------
 __device__ __forceinline__ void report_timeout(int* status, int where) {

@@ -301,7 +301,8 @@ inline hla_status launch_phi_forward_k(const Dims& D, int BH, const hla_mlp* phi
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     rec.begin("tc_phi_forward_k");
-    launch_pdl(tc_phi_forward_kernel<DV, 3, true>, grid, dim3(kPfThreads), PfCfg<DV, 3>::kSmem, rec.st, mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
+    // first kernel of hla_forward, and it stages the weights before its dependency wait: no overlap with what precedes it
+    launch_serial(tc_phi_forward_kernel<DV, 3, true>, grid, dim3(kPfThreads), PfCfg<DV, 3>::kSmem, rec.st, mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
