@@ -8,7 +8,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import GpuRun, TOL, relerr, l2err
+from hla_testlib import GpuRun, TOL, relerr, l2err, dev_weights, to_dev
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -165,3 +165,36 @@ def test_phi_with_large_biases(d):
     rK = sum(orc.phi_mlp_backward(f64(K).reshape(-1, d), *pk[f], dkf[:, :, f].reshape(-1, s.d_phi)).reshape(K.shape) for f in range(s.F))
     assert relerr(dQ[same_q], rQ[same_q]) < TOL["bf16"]
     assert relerr(dK[same_k], rK[same_k]) < TOL["bf16"]
+
+
+def test_back_to_back_steps_without_host_sync():
+    """Twelve training steps enqueued back to back on one stream, alternating between two sets of inputs and output
+    buffers, with no host synchronisation in between (each kernel's set-up overlaps the drain of the previous one):
+    every step's O, dQ, dK, dV must be bit-identical to the same step run alone."""
+    s = synth.HlaShape("b2b", 1, 6, 5000, 128, "bf16", "rms_qk", backward=True)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    op = binding.Hla(s.B, s.H, s.N, s.d, dtype=s.dtype, phi="mlp", F=s.F, d_phi=s.d_phi, eps=EPS)
+    op.set_phi(*dev_weights(pq, pk, s.dtype))
+    sets = []
+    for seed in (0, 7):
+        Q, K, V = synth.make_qkv(s, seed=seed)
+        dO = synth.make_dO(s)
+        sets.append(tuple(to_dev(a, s.dtype) for a in (Q, K, V, dO)))
+    ref = []
+    for Q, K, V, dO in sets:           # each set alone, synchronised
+        O = op.forward(Q, K, V)
+        dQ, dK, dV = op.backward(Q, K, V, O, dO)
+        torch.cuda.synchronize()
+        assert op.device_status() == binding.HLA_OK
+        ref.append([t.clone() for t in (O, dQ, dK, dV)])
+    outs = []
+    for step in range(12):             # enqueued back to back
+        Q, K, V, dO = sets[step & 1]
+        O = op.forward(Q, K, V)
+        dQ, dK, dV = op.backward(Q, K, V, O, dO)
+        outs.append((O, dQ, dK, dV))
+    torch.cuda.synchronize()
+    assert op.device_status() == binding.HLA_OK
+    for step, got in enumerate(outs):
+        for a, b in zip(got, ref[step & 1]):
+            assert torch.equal(a, b), step
