@@ -39,7 +39,7 @@ def dev_weights(phi_q, phi_k, dtype):
     return tuple(to_dev(a, dtype) for a in phi_q), [tuple(to_dev(a, dtype) for a in w) for w in phi_k]
 
 
-class GpuRun:
+class DeviceRun:
     """One library context fed from numpy inputs; keeps device tensors for reuse."""
 
     def __init__(self, shape: synth.HlaShape, phi="mlp", eps=0.0, n_splits=0):

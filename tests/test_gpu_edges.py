@@ -8,7 +8,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import GpuRun, TOL, relerr, l2err, dev_weights, to_dev
+from hla_testlib import DeviceRun, TOL, relerr, l2err, dev_weights, to_dev
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -28,7 +28,7 @@ def _inputs(s, vscale=True, seed=0):
 def test_degenerate_token_counts_forward_backward(d, N, B, H):
     s = synth.HlaShape("t", B, H, N, d, "bf16", "inv_sqrt_d")
     qf, kf, V, dO = _inputs(s)
-    run = GpuRun(s, "none", EPS)
+    run = DeviceRun(s, "none", EPS)
     assert run.op.layout.tensor_core == 1
     O = run.forward(qf, kf, V)
     dq, dk, dv = run.backward(dO)
@@ -49,7 +49,7 @@ def test_many_heads(d, N, B, H):
     count that does not divide the SM count."""
     s = synth.HlaShape("t", B, H, N, d, "bf16", "inv_sqrt_d")
     qf, kf, V, dO = _inputs(s)
-    run = GpuRun(s, "none", EPS)
+    run = DeviceRun(s, "none", EPS)
     O = run.forward(qf, kf, V)
     dq, dk, dv = run.backward(dO)
     Oq, eta = orc.hla_core_forward(f64(qf), f64(kf), f64(V), EPS, "quadratic")
@@ -65,7 +65,7 @@ def test_queries_with_all_zero_features_and_large_eps():
     qf, kf, V, dO = _inputs(s)
     qf[0, :, ::7, :] = 0.0
     for eps in (1e-6, 1e-2):
-        run = GpuRun(s, "none", eps)
+        run = DeviceRun(s, "none", eps)
         O = run.forward(qf, kf, V)
         dq, dk, dv = run.backward(dO)
         assert np.all(O[0, :, ::7, :] == 0.0)
@@ -84,7 +84,7 @@ def test_backward_bitwise_reproducible():
     Q, K, V = synth.make_qkv(s)
     dO = synth.make_dO(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS, n_splits=4)
+    run = DeviceRun(s, "mlp", EPS, n_splits=4)
     run.set_weights(pq, pk)
     run.forward(Q, K, V)
     a = run.backward(dO)
@@ -103,7 +103,7 @@ def test_forward_backward_with_phi_stage_by_stage(shape):
     Q, K, V = synth.make_qkv(s)
     dO = synth.make_dO(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     O = run.forward(Q, K, V)
     dQ, dK, dV = run.backward(dO)
@@ -143,7 +143,7 @@ def test_phi_with_large_biases(d):
         return W1, bf(rng.standard_normal(b1.shape)), W2, bf(0.5 * rng.standard_normal(b2.shape))
 
     pq, pk = with_bias(pq), [with_bias(w) for w in pk]
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     run.forward(Q, K, V)
     dQ, dK, dV = run.backward(dO)

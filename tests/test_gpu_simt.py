@@ -6,7 +6,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import GpuRun, TOL, oracle_state, relerr
+from hla_testlib import DeviceRun, TOL, oracle_state, relerr
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -17,7 +17,7 @@ def test_config1_tiny_f32_forward_mlp():
     s = synth.CONFIGS["tiny_f32"]
     Q, K, V = synth.make_qkv(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     O = run.forward(Q, K, V)
     Oq, eta, qf, kf = orc.hla_forward(Q, K, V, pq, pk, EPS, "quadratic")
@@ -35,7 +35,7 @@ def test_core_forward_f32_features(F, dphi, d, N, splits):
     s = synth.HlaShape("t", 2, 3, N, d, "f32", "inv_sqrt_d", F=F, d_phi=dphi)
     _, _, V = synth.make_qkv(s)
     qf, kf = synth.make_features(s)
-    run = GpuRun(s, "none", EPS, splits)
+    run = DeviceRun(s, "none", EPS, splits)
     O = run.forward(qf, kf, V)
     Oq, eta = orc.hla_core_forward(qf.astype(np.float64), kf.astype(np.float64), V.astype(np.float64), EPS, "quadratic")
     assert relerr(O, Oq) < TOL["f32"]
@@ -51,7 +51,7 @@ def test_core_backward_f32_features(F, dphi, d, N):
     _, _, V = synth.make_qkv(s)
     qf, kf = synth.make_features(s)
     dO = synth.make_dO(s)
-    run = GpuRun(s, "none", EPS)
+    run = DeviceRun(s, "none", EPS)
     run.forward(qf, kf, V)
     dq, dk, dv = run.backward(dO)
     rq, rk, rv = orc.hla_core_backward(qf.astype(np.float64), kf.astype(np.float64), V.astype(np.float64), dO.astype(np.float64), EPS, "quadratic")
@@ -67,7 +67,7 @@ def test_full_backward_f32_mlp():
     Q, K, V = synth.make_qkv(s)
     dO = synth.make_dO(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     O = run.forward(Q, K, V)
     dQ, dK, dV = run.backward(dO)
@@ -83,7 +83,7 @@ def test_bf16_shape_outside_tensor_core_set_runs_simt():
     s = synth.HlaShape("t", 1, 2, 300, 32, "bf16", "rms_qk")
     Q, K, V = synth.make_qkv(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     assert run.op.layout.tensor_core == 0
     run.set_weights(pq, pk)
     O = run.forward(Q, K, V)
@@ -98,7 +98,7 @@ def test_bitwise_reproducible():
     s = synth.HlaShape("t", 1, 2, 500, 16, "f32", "inv_sqrt_d")
     _, _, V = synth.make_qkv(s)
     qf, kf = synth.make_features(s)
-    run = GpuRun(s, "none", EPS, 5)
+    run = DeviceRun(s, "none", EPS, 5)
     a = run.forward(qf, kf, V)
     b = run.forward(qf, kf, V)
     assert np.array_equal(a, b)

@@ -6,7 +6,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import GpuRun, TOL, fold_symmetric, oracle_state, relerr, l2err
+from hla_testlib import DeviceRun, TOL, fold_symmetric, oracle_state, relerr, l2err
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -21,7 +21,7 @@ def test_core_forward_bf16_features(d, N, B, H, splits):
     _, _, V = synth.make_qkv(s)
     V = synth.bf16_round(V * np.float32(np.sqrt(d)))          # V ~ N(0,1)
     qf, kf = synth.make_features(s)
-    run = GpuRun(s, "none", EPS, splits)
+    run = DeviceRun(s, "none", EPS, splits)
     assert run.op.layout.tensor_core == 1
     O = run.forward(qf, kf, V)
     f64 = lambda a: a.astype(np.float64)
@@ -44,7 +44,7 @@ def test_config2_small_bf16_forward_stagewise():
     s = synth.CONFIGS["small_bf16"]
     Q, K, V = synth.make_qkv(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     O = run.forward(Q, K, V)
     f64 = lambda a: a.astype(np.float64)
@@ -68,7 +68,7 @@ def test_tc_bitwise_reproducible():
     s = synth.HlaShape("t", 1, 3, 2000, 128, "bf16", "inv_sqrt_d")
     _, _, V = synth.make_qkv(s)
     qf, kf = synth.make_features(s)
-    run = GpuRun(s, "none", EPS, 4)
+    run = DeviceRun(s, "none", EPS, 4)
     a = run.forward(qf, kf, V)
     b = run.forward(qf, kf, V)
     assert np.array_equal(a, b)
@@ -82,7 +82,7 @@ def test_core_backward_bf16_features(d, N, B, H, splits):
     V = synth.bf16_round(V * np.float32(np.sqrt(d)))
     qf, kf = synth.make_features(s)
     dO = synth.make_dO(s)
-    run = GpuRun(s, "none", EPS, splits)
+    run = DeviceRun(s, "none", EPS, splits)
     O = run.forward(qf, kf, V)
     dq, dk, dv = run.backward(dO)
     f64 = lambda a: a.astype(np.float64)
@@ -101,7 +101,7 @@ def test_full_backward_bf16_mlp_stagewise():
     Q, K, V = synth.make_qkv(s)
     dO = synth.make_dO(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     O = run.forward(Q, K, V)
     dQ, dK, dV = run.backward(dO)
@@ -155,7 +155,7 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable():
     s = synth.HlaShape("t", 1, 2, 300, 128, "bf16", "inv_sqrt_d")
     _, _, V = synth.make_qkv(s)
     qf, kf = synth.make_features(s)
-    run = GpuRun(s, "none", EPS)
+    run = DeviceRun(s, "none", EPS)
     binding.hla_selftest_bounded_wait(run.op.ctx, run.op.workspace)
     assert run.op.device_status() == binding.HLA_ERR_DEVICE_TIMEOUT
     O = run.forward(qf, kf, V)                                    # clears the status words; asserts HLA_OK inside
@@ -170,7 +170,7 @@ def test_forward_backward_replay_in_a_cuda_graph():
     Q, K, V = synth.make_qkv(s)
     dO = synth.make_dO(s)
     pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
-    run = GpuRun(s, "mlp", EPS)
+    run = DeviceRun(s, "mlp", EPS)
     run.set_weights(pq, pk)
     O_ref = run.forward(Q, K, V)
     ref = run.backward(dO)
