@@ -343,8 +343,14 @@ template <int DV, int NMAPS> struct PbCfg {
     // b1 is added on the tensor cores by a ninth K step of the h product: A = K columns 32..47 of the dp block (column
     // 32 is a constant 1, never written again; the dp tiles use columns 0..31), B = per map a tile whose K row 0 is b1
     static constexpr int kOffB1 = kOffW2t + NMAPS * kW2tBytes;   // per map: [16 K rows][DV] bf16, MN-major
-    static constexpr int kOffBars = kOffB1 + NMAPS * kW2tBytes;
+    // dX staging tile for a TMA store where the whole 128 x DV tile fits (one map, or d = 64); with three maps and
+    // d = 128 only half a tile would fit, and a drain in two halves (measured) is slower than direct stores
+    static constexpr bool kStagedDrain = NMAPS == 1 || DV == 64;
+    static constexpr int kStageBlocks = kStagedDrain ? DV / 64 : 0;
+    static constexpr int kOffStage = kOffB1 + NMAPS * kW2tBytes;
+    static constexpr int kOffBars = kOffStage + kStageBlocks * kBlk;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
+    static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
 
@@ -358,7 +364,8 @@ template <int DV, int NMAPS> struct PbCfg {
 // registers to global memory.  The epilogue threads also write the dp tiles (one feature pair each, one unit ahead).
 template <int DV, int NMAPS, bool KSIDE>
 __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
-                                                                        PhiBwdPtrs P, const float* __restrict__ feat, const float* __restrict__ dfeat,
+                                                                        const __grid_constant__ CUtensorMap mapdX, PhiBwdPtrs P,
+                                                                        const float* __restrict__ feat, const float* __restrict__ dfeat,
                                                                         __nv_bfloat16* __restrict__ dX, long long rows, int N, int* status) {
     using Cfg = PbCfg<DV, NMAPS>;
     constexpr int HC = DV / 4;
@@ -418,6 +425,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         mbar_init(w_full, 1);
         fence_mbar_init();
         prefetch_tmap(&mapX);
+        prefetch_tmap(&mapdX);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, 512);
@@ -510,27 +518,57 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         const int quarter = warp & 3, part = (warp - kPbEpiWarp0) >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        // dX of tile `it`: TMEM -> bf16 -> global memory (each thread: HC contiguous columns of its row)
+        // dX of tile `it`: TMEM -> bf16 -> global memory.  Staged: through a swizzled tile in shared memory and a TMA store
+        // (direct 32-byte stores put 32 separate sectors into every store instruction and hold the 16 warps for ~1000
+        // cycles per tile).  Otherwise each thread stores its HC contiguous columns directly, one sector per store.
         auto drain_dx = [&](int it) {
             if (ok && !mbar_wait(dx_full, it & 1)) { ok = false; report_timeout(status, 606); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) return;
             tc_fence_after();
             const uint32_t tx = tmem + 384 + lane_base + part * HC;
-            const long long grow = (t0 + it) * kTileTokens + row;
-            uint4* dst = reinterpret_cast<uint4*>(dX + (size_t)grow * DV + part * HC);
+            if constexpr (Cfg::kStagedDrain) {
+                uint32_t w[HC / 2];
 #pragma unroll
-            for (int c = 0; c < HC / 16; ++c) {
-                uint32_t r[16];
-                tmem_ld16(tx + 16 * c, r);
-                tmem_ld_wait();
-                uint32_t w[8];
+                for (int c = 0; c < HC / 16; ++c) {
+                    uint32_t r[16];
+                    tmem_ld16(tx + 16 * c, r);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                if (grow < rows) st_global_v8(dst + 2 * c, w);      // one full 32-byte sector per store
+                    for (int e = 0; e < 8; ++e) w[8 * c + e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                }
+                tc_fence_before();
+                mbar_arrive(dx_empty);          // the accumulator is in registers
+                const int col0 = part * HC;     // first column of this thread
+                const uint32_t sblk = smem_u32(smem + Cfg::kOffStage) + (col0 / 64) * kBlk;
+                if (tid == kPbEpiWarp0 * 32) tma_store_wait_read0();      // the previous tile's store has read the staging tile
+                named_barrier(2, 512);
+#pragma unroll
+                for (int j = 0; j < HC / 8; ++j)
+                    st_shared_v4(sblk + sw128_off(row, (col0 & 63) / 8 + j), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                fence_proxy_async();
+                named_barrier(2, 512);
+                if (tid == kPbEpiWarp0 * 32) {
+                    for (int blk = 0; blk < Cfg::kStageBlocks; ++blk)
+                        tma_store_2d(&mapdX, smem + Cfg::kOffStage + blk * kBlk, blk * 64, (int)((t0 + it) * kTileTokens));
+                    tma_store_commit();
+                }
+            } else {
+                const long long grow = (t0 + it) * kTileTokens + row;
+                uint4* dst = reinterpret_cast<uint4*>(dX + (size_t)grow * DV + part * HC);
+#pragma unroll
+                for (int c = 0; c < HC / 16; ++c) {
+                    uint32_t r[16];
+                    tmem_ld16(tx + 16 * c, r);
+                    tmem_ld_wait();
+                    uint32_t w[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                    if (grow < rows) st_global_v8(dst + 2 * c, w);      // one full 32-byte sector per store
+                }
+                tc_fence_before();
+                mbar_arrive(dx_empty);
             }
-            tc_fence_before();
-            mbar_arrive(dx_empty);
         };
         // dp = dfeat (.) 1[feat > 0] as the A operand [dp_hi | dp_lo] of the dg product.  Every epilogue thread of parts
         // 0..2 owns one pair of features of its row: it loads them two units ahead (row index clamped, the loads are
@@ -619,6 +657,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             if (m == 0 && it > 0) drain_dx(it - 1);
         }
         if (ok && ntiles > 0) drain_dx(ntiles - 1);
+        if (Cfg::kStagedDrain && tid == kPbEpiWarp0 * 32) tma_store_wait_all0();
     }
     tc_fence_before();
     __syncthreads();
@@ -629,10 +668,11 @@ template <int DV>
 inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, void* dQ,
                                       void* dK, char* ws, const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
     const long long rows = (long long)BH * D.N;
-    CUtensorMap mapQ, mapK;
+    CUtensorMap mapQ, mapK, mapdQ, mapdK;
     PhiMaps mq, mk;
     PhiBwdPtrs pq{}, pk{};
     if (!make_map_2d(&mapQ, Q, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
+    if (!make_map_2d(&mapdQ, dQ, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapdK, dK, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
     if (!make_map_2d(&mq.w1[0], phi_q->W1, DV, DV, DV)) return HLA_ERR_CUDA;
     mq.w1[1] = mq.w1[0];
     mq.w1[2] = mq.w1[0];
@@ -651,11 +691,11 @@ inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_
     cudaStream_t st = rec.st;
     rec.begin("tc_phi_backward_q");
     launch_pdl(tc_phi_backward_kernel<DV, 1, false>, grid, dim3(kPbThreads), PbCfg<DV, 1>::kSmem, st, 
-        mapQ, mq, pq, reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), static_cast<__nv_bfloat16*>(dQ), rows, D.N, status);
+        mapQ, mq, mapdQ, pq, reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), static_cast<__nv_bfloat16*>(dQ), rows, D.N, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_phi_backward_k");
     launch_pdl(tc_phi_backward_kernel<DV, 3, true>, grid, dim3(kPbThreads), PbCfg<DV, 3>::kSmem, st, 
-        mapK, mk, pk, reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), static_cast<__nv_bfloat16*>(dK), rows, D.N, status);
+        mapK, mk, mapdK, pk, reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), static_cast<__nv_bfloat16*>(dK), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
