@@ -341,13 +341,15 @@ template <int DV, int NMAPS> struct PbCfg {
     static constexpr int kOffDp = kOffW1 + NMAPS * kW1Bytes;     // one swizzled block = 4 dp tiles [128 tok][16] (K slices 0..3)
     static constexpr int kOffW2t = kOffDp + kBlk;
     // b1 is added on the tensor cores by a ninth K step of the h product: A = K columns 32..47 of the dp block (column
-    // 32 is a constant 1, never written again; the dp tiles use columns 0..31), B = per map a tile whose K row 0 is b1
-    static constexpr int kOffB1 = kOffW2t + NMAPS * kW2tBytes;   // per map: [16 K rows][DV] bf16, MN-major
-    // dX staging tile for a TMA store where the whole 128 x DV tile fits (one map, or d = 64); with three maps and
-    // d = 128 only half a tile would fit, and a drain in two halves (measured) is slower than direct stores
+    // 44 is a constant 1, never written again; the dp tiles use columns 0..31), B = the map's W2^T tile, whose K row 12
+    // holds b1 (rows 12..15 meet the zero columns 12..15 of the dp tiles in the dg product, so they are free there)
+    static constexpr int kB1Row = 12;
+    // dX staging tile (128 x DV) for a TMA store: query side and d = 64.  On the key side at d = 128 (a drain every
+    // third unit) the two block-wide barriers of the staged drain cost more than the direct stores they replace
+    // (measured, also as a drain in two halves).
     static constexpr bool kStagedDrain = NMAPS == 1 || DV == 64;
     static constexpr int kStageBlocks = kStagedDrain ? DV / 64 : 0;
-    static constexpr int kOffStage = kOffB1 + NMAPS * kW2tBytes;
+    static constexpr int kOffStage = kOffW2t + NMAPS * kW2tBytes;
     static constexpr int kOffBars = kOffStage + kStageBlocks * kBlk;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static_assert(kSmemUsed <= 227 * 1024, "shared memory");
@@ -397,17 +399,12 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     for (int i = tid; i < NMAPS * 16 * DV; i += kPbThreads) {
         const int m = i / (16 * DV), k = (i / DV) & 15, j = i % DV;
         uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? half_bf16(P.W2[m][j * 6 + (k % 6)]) : __float2bfloat16_rn(0.f);
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? half_bf16(P.W2[m][j * 6 + (k % 6)]) : (k == Cfg::kB1Row ? P.b1[m][j] : __float2bfloat16_rn(0.f));
     }
     for (int i = tid; i < kBlk / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < NMAPS * Cfg::kW2tBytes / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffB1)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
-    for (int i = tid; i < kTileTokens; i += kPbThreads)
-        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffDp + sw128_off(i, 4)) = __float2bfloat16_rn(1.f);
-    for (int i = tid; i < NMAPS * DV; i += kPbThreads) {
-        const int m = i / DV, j = i % DV;       // K row 0 of the MN-major tile: 64-column block j / 64, no swizzle in row 0
-        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffB1 + m * Cfg::kW2tBytes + (j >> 6) * 2048 + (j & 63) * 2) = P.b1[m][j];
-    }
+    for (int i = tid; i < kTileTokens; i += kPbThreads)      // K column 32 + kB1Row of the dp block
+        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffDp + sw128_off(i, 4 + Cfg::kB1Row / 8) + (Cfg::kB1Row & 7) * 2) = __float2bfloat16_rn(1.f);
     fence_proxy_async();
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -458,7 +455,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
             const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp) + 64, 16, 1024);
-            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffB1), 2048, 1024);
+            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
             bool good = mbar_wait(w_full, 0);
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
