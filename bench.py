@@ -81,8 +81,8 @@ def kernel_models(shape):
 # DRAM traffic per token-head of a launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # scaled by token-heads; see profiles/).  None = not captured yet.
 NCU_TRAFFIC_PER_TOKEN_HEAD = {
-    "tc_phi_forward_k": 313.9, "tc_state_build": 332.6, "tc_phiq_readout": 478.3, "tc_bwd_query": 303.6, "tc_bwd_key": 593.7,
-    "tc_phi_backward_q": 504.5, "tc_phi_backward_k": 616.7,
+    "tc_phi_forward_k": 313.5, "tc_state_build": 333.0, "tc_phiq_readout": 477.8, "tc_bwd_query": 305.7, "tc_bwd_key": 594.1,
+    "tc_phi_backward_q": 498.8, "tc_phi_backward_k": 619.3,
 }
 
 
