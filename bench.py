@@ -13,7 +13,9 @@ slowest rank's device time.
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
+import math
 import os
 import subprocess
 import sys
@@ -87,20 +89,28 @@ NCU_TRAFFIC_PER_TOKEN_HEAD = {
 
 
 class ClockSampler:
+    """nvidia-smi polled in the background.  Every sample carries its own time stamp, so the samples that fall inside a
+    window of the run (sustained warm-up + timed region) can be picked afterwards; of those, the ones with a GPU
+    utilisation above 50 % are the samples under load."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,utilization.gpu,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASONS = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
     def __init__(self, index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
-            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20"],
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
+        self.rows = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.rows is not None:
+            return
+        self.rows = []
         if self.p is None:
-            return out
+            return
         self.p.terminate()
         try:
             self.p.wait(timeout=5)
@@ -108,28 +118,33 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 8:
+            if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
+                t = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                self.rows.append((t, float(parts[1]), float(parts[2]), float(parts[3]), float(parts[4]),
+                                  [nm for nm, val in zip(self.REASONS, parts[5:9]) if val.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
         self.f.close()
         os.unlink(self.f.name)
-        if sm:
-            busy = sorted(sm)[len(sm) // 2:]          # the upper half are the samples under load
-            out["sm_mhz"] = float(np.median(busy))
-            out["sm_max_mhz"] = float(max(mx))
-            out["samples"] = len(sm)
-        out["reasons"] = sorted(reasons)
+
+    def window(self, t0: float, t1: float) -> dict:
+        """Summary of the samples stamped in [t0, t1] (host clock, seconds)."""
+        self.stop()
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        busy = [r for r in rows if r[4] > 50.0]
+        out = {"sm_mhz": None, "sm_min_mhz": None, "sm_max_mhz": None, "power_w": None, "reasons": [], "samples": len(rows),
+               "samples_under_load": len(busy), "note": "samples stamped inside the sustained warm-up and the timed region; under load = utilisation > 50 %"}
+        use = busy or rows
+        if use:
+            out["sm_mhz"] = float(np.median([r[1] for r in use]))
+            out["sm_min_mhz"] = float(min(r[1] for r in use))
+            out["sm_max_mhz"] = float(max(r[2] for r in use))
+            out["power_w"] = float(np.median([r[3] for r in use]))
+            out["reasons"] = sorted({nm for r in use for nm in r[5]})
         return out
 
 
@@ -184,10 +199,138 @@ def run_reference(args, shape, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def roofline_of(shape, ms_step, world, peaks):
+    """Step roofline.  `frac` uses the work the hardware has to do: the larger of the algorithmic HBM bytes at the copy
+    bandwidth and the FLOPs of the symmetry-folded scheme (what the kernels execute) at the tensor peak.
+    `frac_algorithmic` is the same with the paper's unfolded FLOP count (P = d_phi^F features per contraction), which
+    the kernels never issue; it is kept as a labelled second figure."""
+    fl_alg, by = work_model(shape)
+    th = shape.B * shape.H * shape.N
+    fl_exec = th * F_.folded_flops_per_token(shape.d, shape.F, shape.d_phi, shape.backward)
+    t_mem = by / (peaks["hbm"] * 1e9)
+    t_exec = fl_exec / (peaks["tensor"] * 1e12)
+    t_alg = fl_alg / (peaks["tensor"] * 1e12)
+    t_roof = max(t_mem, t_exec)
+    return {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_step, "bound": "hbm" if t_mem >= t_exec else "tensor",
+            "t_hbm_ms": t_mem * 1e3, "t_tensor_executed_ms": t_exec * 1e3, "t_tensor_algorithmic_ms": t_alg * 1e3,
+            "frac_algorithmic": max(t_mem, t_alg) * 1e3 / ms_step, "flops_algorithmic": fl_alg, "flops_executed": fl_exec, "bytes": by,
+            "peaks": peaks}
+
+
+class Workload:
+    """One configuration resident in HBM: synthetic inputs (seeded per rank), the operator context and its outputs."""
+
+    def __init__(self, shape, rank, dev):
+        import torch
+        from paper_2602_12128_b200 import binding
+        self.torch, self.binding, self.shape, self.dev = torch, binding, shape, dev
+        tdt = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
+        g = torch.Generator(device=dev)
+        g.manual_seed(multi.rank_seed(1000, rank))
+        dims = (shape.B, shape.H, shape.N, shape.d)
+
+        def draw():
+            return torch.randn(dims, generator=g, device=dev, dtype=torch.float32)
+
+        Q, K, V = draw(), draw(), draw()
+        if shape.scale == "inv_sqrt_d":
+            sc = 1.0 / np.sqrt(shape.d)
+            Q, K, V = Q * sc, K * sc, V * sc
+        else:
+            Q = Q / Q.pow(2).mean(-1, keepdim=True).sqrt()
+            K = K / K.pow(2).mean(-1, keepdim=True).sqrt()
+        self.Q, self.K, self.V = Q.to(tdt), K.to(tdt), V.to(tdt)
+        self.dO = draw().to(tdt) if shape.backward else None
+        del Q, K, V
+        pq, pk = synth.make_phi_weights(shape.d, shape.d_phi, shape.F, shape.dtype)
+        to_dev = lambda a: torch.from_numpy(a).to(tdt).to(dev)
+        self.op = binding.Hla(shape.B, shape.H, shape.N, shape.d, dtype=shape.dtype, phi="mlp", F=shape.F, d_phi=shape.d_phi, eps=1e-6, device=dev)
+        self.op.set_phi(tuple(to_dev(a) for a in pq), [tuple(to_dev(a) for a in w) for w in pk])
+        self.O = torch.empty_like(self.V)
+        self.dQ, self.dK, self.dV = (torch.empty_like(self.V) for _ in range(3)) if shape.backward else (None, None, None)
+        self.launches = 0
+
+    def step(self):
+        b, op = self.binding, self.op
+        b.hla_forward(op.ctx, self.Q, self.K, self.V, self.O, op.workspace)
+        n = op.launches()
+        if self.shape.backward:
+            b.hla_backward(op.ctx, self.Q, self.K, self.V, self.O, self.dO, self.dQ, self.dK, self.dV, op.workspace)
+            n += op.launches()
+        self.launches = n
+
+    def timed(self, nsteps):
+        """Device time of `nsteps` steps enqueued back to back (CUDA events on the launching stream), in ms."""
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(nsteps):
+            self.step()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def sustain(self, seconds, ms_estimate):
+        """The same steps, untimed and without host synchronisation, for about `seconds` of device time, so that the
+        clocks settle under the power cap before anything is timed."""
+        n = int(min(max(math.ceil(seconds * 1e3 / max(ms_estimate, 1e-3)), 1), 50000))
+        for _ in range(n):
+            self.step()
+        return n
+
+    def kernel_times(self, nsteps):
+        """Per-kernel device time from event records inside the library, on steps of their own (the records stall the
+        stream a few microseconds each, so they stay out of every timed region)."""
+        b, op = self.binding, self.op
+        b.hla_timing_enable(op.ctx, True)
+        self.step()
+        self.torch.cuda.synchronize()
+        b.hla_timing_collect(op.ctx)            # discard: creates the event pool
+        for _ in range(nsteps):
+            self.step()
+        self.torch.cuda.synchronize()
+        kt = b.hla_timing_collect(op.ctx)
+        b.hla_timing_enable(op.ctx, False)
+        return kt
+
+
+def extra_leg(name, rank, dev, peaks, local):
+    """One of the other configurations, timed by the same code: >= 1 s of untimed sustained steps, then >= 0.5 s timed."""
+    import torch
+    from paper_2602_12128_b200 import binding
+    shape = synth.CONFIGS[name]
+    w = Workload(shape, rank, dev)
+    for _ in range(3):
+        w.step()
+    torch.cuda.synchronize()
+    if w.op.device_status() != binding.HLA_OK:
+        raise SystemExit(f"device-side wait timed out ({name})")
+    est = w.timed(5) / 5
+    sampler = ClockSampler(local)
+    t0 = time.time()
+    w.sustain(1.0, est)
+    n = int(min(max(math.ceil(500.0 / est), 10), 50000))
+    ms = w.timed(n) / n
+    t1 = time.time()
+    clocks = sampler.window(t0, t1)
+    fl, _ = work_model(shape)
+    roof = roofline_of(shape, ms, 1, peaks)
+    roof.pop("peaks")
+    out = {"config": {"B": shape.B, "H": shape.H, "N": shape.N, "d": shape.d, "pass": "fwd+bwd" if shape.backward else "fwd"},
+           "ms_per_step": ms, "steps": n, "tflops": fl / (ms * 1e-3) / 1e12, "tokens_per_s": shape.B * shape.N / (ms * 1e-3),
+           "gpu_launches_per_step": w.launches, "step_roofline": roof,
+           "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_min_mhz", "power_w", "reasons", "samples_under_load")}}
+    if clocks["sm_mhz"]:
+        out["ms_x_mhz"] = ms * clocks["sm_mhz"]
+    del w
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="train_bf16", choices=sorted(synth.CONFIGS))
@@ -196,8 +339,12 @@ def main():
     ap.add_argument("--N", type=int, default=0, help="override the workload's token count")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations (the `extra` object of the line)")
+    ap.add_argument("--profile", action="store_true", help="only warm-up and the timed steps: no sustained phase, no extra legs (for ncu)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    if args.profile:
+        args.no_e2e = args.no_cpu_baseline = args.no_extra = True
     shape = synth.CONFIGS[args.workload]
     if args.B or args.H or args.N:
         import dataclasses
@@ -221,89 +368,53 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
-    tdt = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
-
-    # ---- synthetic inputs (seeded per rank), resident in HBM -----------------------------------------------------
-    g = torch.Generator(device=dev)
-    g.manual_seed(multi.rank_seed(1000, rank))
-    dims = (shape.B, shape.H, shape.N, shape.d)
-
-    def draw():
-        return torch.randn(dims, generator=g, device=dev, dtype=torch.float32)
-
-    Q, K, V = draw(), draw(), draw()
-    if shape.scale == "inv_sqrt_d":
-        s = 1.0 / np.sqrt(shape.d)
-        Q, K, V = Q * s, K * s, V * s
-    else:
-        Q = Q / Q.pow(2).mean(-1, keepdim=True).sqrt()
-        K = K / K.pow(2).mean(-1, keepdim=True).sqrt()
-    Q, K, V = Q.to(tdt), K.to(tdt), V.to(tdt)
-    dO = draw().to(tdt) if shape.backward else None
-    pq, pk = synth.make_phi_weights(shape.d, shape.d_phi, shape.F, shape.dtype)
-    to_dev = lambda a: torch.from_numpy(a).to(tdt).to(dev)
-    pq_d = tuple(to_dev(a) for a in pq)
-    pk_d = [tuple(to_dev(a) for a in w) for w in pk]
-
-    op = binding.Hla(shape.B, shape.H, shape.N, shape.d, dtype=shape.dtype, phi="mlp", F=shape.F, d_phi=shape.d_phi, eps=1e-6, device=dev)
-    op.set_phi(pq_d, pk_d)
-    O = torch.empty_like(V)
-    dQ, dK, dV = (torch.empty_like(V) for _ in range(3)) if shape.backward else (None, None, None)
-    launches = [0]
-
-    def step():
-        binding.hla_forward(op.ctx, Q, K, V, O, op.workspace)
-        n = op.launches()
-        if shape.backward:
-            binding.hla_backward(op.ctx, Q, K, V, O, dO, dQ, dK, dV, op.workspace)
-            n += op.launches()
-        launches[0] = n
+    peaks = measured_peaks()
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
+    w = Workload(shape, rank, dev)
+    op = w.op
     for _ in range(max(args.warmup, 1)):
-        step()
+        w.step()
     torch.cuda.synchronize()
     if op.device_status() != binding.HLA_OK:
         raise SystemExit("device-side wait timed out during warm-up")
 
-    # ---- timed region: K steps, CUDA events on the launching stream, per-kernel events inside the library -------
-    binding.hla_timing_enable(op.ctx, True)
-    step()
-    torch.cuda.synchronize()
-    binding.hla_timing_collect(op.ctx)          # discard: creates the event pool outside the timed region
+    # ---- sustained untimed steps (>= 1 s, no host synchronisation), then the timed region: exactly K steps ------------
+    est = w.timed(3) / 3
     sampler = ClockSampler(local)
+    t_win0 = time.time()
+    n_sustain = 0 if args.profile else w.sustain(1.0, est)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
-    for i in range(args.steps):
-        binding.hla_timing_enable(op.ctx, i % 4 == 0)      # per-kernel events on every fourth step: each record stalls the stream ~3 us
-        step()
+    for _ in range(args.steps):
+        w.step()
     e1.record()
     barrier()
     ms_total = e0.elapsed_time(e1)
-    kt = binding.hla_timing_collect(op.ctx)
-    binding.hla_timing_enable(op.ctx, False)
-    # The timed region can be shorter than one nvidia-smi sample: keep the same steps running (untimed) until the
-    # sampler has had about a second under the same load, then stop it.
-    t_tail = time.perf_counter()
-    while time.perf_counter() - t_tail < 1.0:
-        step()
-        torch.cuda.synchronize()
-    clocks = sampler.stop()
-    clocks["note"] = "sampled over the timed steps and an untimed 1 s tail of the same steps"
+    # a longer run of the same steps right behind it: the steady-state figure (>= 0.5 s of device time)
+    ms_steady, n_steady = None, 0
+    if not args.profile:
+        n_steady = int(min(max(math.ceil(500.0 / est), args.steps), 50000))
+        ms_steady = w.timed(n_steady) / n_steady
+    t_win1 = time.time()
+    clocks = sampler.window(t_win0, t_win1)
+    kt = {} if args.profile else w.kernel_times(8)
     ms_step = multi.max_over_ranks(ms_total, dist, dev) / args.steps
+    if ms_steady is not None:
+        ms_steady = multi.max_over_ranks(ms_steady, dist, dev)
     fl_step, by_step = work_model(shape)
     value = multi.whole_job_rate(fl_step, world, ms_step) / 1e12
 
     # ---- end to end through the C ABI from pinned host buffers -----------------------------------------------------
     e2e = None
     if not args.no_e2e:
-        ins = [Q, K, V] + ([dO] if shape.backward else [])
-        outs = [O] + ([dQ, dK, dV] if shape.backward else [])
+        ins = [w.Q, w.K, w.V] + ([w.dO] if shape.backward else [])
+        outs = [w.O] + ([w.dQ, w.dK, w.dV] if shape.backward else [])
         h_in = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True).copy_(x) for x in ins]
         h_out = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in outs]
         nsteps = max(2, min(args.steps, 6))
@@ -350,6 +461,7 @@ def main():
         e2e = {"value": multi.whole_job_rate(fl_step, world, ms_e2e) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e, "steps": nsteps,
                "h2d_bytes_per_step": int(sum(x.numel() * x.element_size() for x in ins)),
                "d2h_bytes_per_step": int(sum(x.numel() * x.element_size() for x in outs))}
+        del h_in, h_out, sets_in, sets_out
 
     if rank != 0:
         if dist is not None:
@@ -357,11 +469,9 @@ def main():
         return
 
     # ---- roofline of the dominant kernel ------------------------------------------------------------------------------
-    peaks = measured_peaks()
     models = kernel_models(shape)
-    timed_steps = len(range(0, args.steps, 4))
-    per_kernel = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / timed_steps, "share": v[0] / max(sum(x[0] for x in kt.values()), 1e-9)}
-                  for k, v in kt.items()}
+    tot_k = max(sum(x[0] for x in kt.values()), 1e-9)
+    per_kernel = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / 8, "share": v[0] / tot_k} for k, v in kt.items()}
     roof = None
     if kt:
         top = max(kt, key=lambda k: kt[k][0])
@@ -380,26 +490,41 @@ def main():
             roof["kernel"] = top
             roof["peak_source"] = peaks["src"] if roof["bound"] != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"
             roof["ms_per_launch"] = dur * 1e3
-    t_roof = max(by_step / (peaks["hbm"] * 1e9), fl_step / (peaks["tensor"] * 1e12))
+            roof["flops_per_launch"] = fl
+            roof["bytes_per_launch"] = by
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         nh = min(8, shape.B * shape.H)
         dt, fl = oracle_sample(shape, heads=nh)
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-               "sample": f"{nh} of {shape.B * shape.H} heads of {shape.name} (N={shape.N}, d={shape.d}), fp64 factored form, {dt:.1f} s"}
+               "sample": f"{nh} of {shape.B * shape.H} heads of {shape.name} (N={shape.N}, d={shape.d}), numpy fp64 factored form with BLAS threads, {dt:.1f} s"}
+
+    tensor_mb = w.Q.numel() * w.Q.element_size() / 1e6
+    launches_per_step = w.launches
+    # ---- the other configurations, timed by the same code (single-GPU runs only) ----------------------------------------
+    extra = None
+    if not args.no_extra and world == 1:
+        del w, op
+        torch.cuda.empty_cache()
+        extra = {}
+        for name in ("long_bf16", "dit_bf16", "small_bf16", "paper_r1_bf16", "paper_r2_bf16"):
+            if name != shape.name:
+                extra[name] = extra_leg(name, rank, dev, peaks, local)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype,
+            "ms_per_step": ms_step, "ms_per_step_steady": ms_steady, "steady_steps": n_steady, "sustained_untimed_steps": n_sustain,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype,
             "data": "synthetic",
             "config": {"workload": shape.name, "B": shape.B, "H": shape.H, "N": shape.N, "d": shape.d, "F": shape.F, "d_phi": shape.d_phi,
                        "phi": "mlp", "pass": "fwd+bwd" if shape.backward else "fwd", "parallelism": f"replicas x{world}",
-                       "l2": "inputs larger than L2 (each tensor %.0f MB)" % (Q.numel() * Q.element_size() / 1e6)},
+                       "l2": "inputs larger than L2 (each tensor %.0f MB)" % tensor_mb},
             "tokens_per_s": multi.whole_job_rate(shape.B * shape.N, world, ms_step),
-            "step_roofline": {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_step, "flops": fl_step, "bytes": by_step,
-                              "peaks": peaks},
-            "roofline": roof, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
-            "clocks": clocks}
+            "step_roofline": roofline_of(shape, ms_step, world, peaks),
+            "roofline": roof, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks, "extra": extra}
+    if clocks.get("sm_mhz"):
+        line["ms_x_mhz"] = ms_step * clocks["sm_mhz"]
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -26,6 +26,9 @@
  *     return code, and arguments are validated before anything is launched.
  *   - Device-side waits are bounded; a wait that runs out makes the kernel
  *     record a code in the workspace and return.  hla_last_device_status reads it.
+ *     Each wait gives up after two seconds, and the warps of a block that depend
+ *     on one another give up one after the other, so a launch that has timed out
+ *     can take several times two seconds to return.
  *   - One ctx must not be used from two host threads at once.
  */
 #ifndef HLA_H_
@@ -46,7 +49,8 @@ typedef enum {
     HLA_ERR_UNSUPPORTED = 2,   /* valid request outside the supported set (see hla_config)  */
     HLA_ERR_WORKSPACE = 3,     /* workspace smaller than hla_workspace_bytes()              */
     HLA_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed                        */
-    HLA_ERR_DEVICE_TIMEOUT = 5 /* a bounded device-side wait expired (results are invalid)  */
+    HLA_ERR_DEVICE_TIMEOUT = 5,/* a bounded device-side wait expired (results are invalid)  */
+    HLA_ERR_NO_MEMORY = 6      /* host memory for the context could not be obtained          */
 } hla_status;
 
 typedef enum { HLA_BF16 = 0, HLA_F32 = 1 } hla_dtype;
@@ -133,7 +137,10 @@ hla_status hla_forward(hla_ctx *ctx, const void *Q, const void *K, const void *V
  * Backward of the forward that last wrote `workspace` (same Q, K, V, O; the
  * workspace untouched in between): dQ, dK, dV = d sum(dO * O) / d(Q, K, V).
  * In HLA_PHI_NONE mode dQ, dK are fp32 feature gradients with the shapes of Q, K.
- * Gradients with respect to the phi weights are not computed.
+ * In HLA_PHI_MLP mode on the tensor-core kernels dQ and dK must be 32-byte aligned
+ * (their rows leave the kernel as 32-byte stores); anything else is refused with
+ * HLA_ERR_INVALID_ARG before a launch.
+ * Gradients with respect to the phi weights are not computed by this call.
  */
 hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *V, const void *O,
                         const void *dO, void *dQ, void *dK, void *dV,

@@ -97,6 +97,25 @@ def phi_mlp_backward(x, W1, b1, W2, b2, dfeat, relu=True):
     return dh @ W1.T
 
 
+def phi_mlp_backward_weights(x, W1, b1, W2, b2, dfeat, relu=True):
+    """Gradients of sum(dfeat * phi_mlp(x)) with respect to the weights of the map, summed over the
+    tokens (Section 5, "Training Details": the phi networks are trained).  Returns (dW1, db1, dW2, db2)
+    with the shapes of W1, b1, W2, b2."""
+    x = np.asarray(x, F64)
+    W1 = np.asarray(W1, F64)
+    W2 = np.asarray(W2, F64)
+    h = x @ W1 + np.asarray(b1, F64)
+    g = gelu_erf(h)
+    p = g @ W2 + np.asarray(b2, F64)
+    dp = np.asarray(dfeat, F64) * (p > 0.0) if relu else np.asarray(dfeat, F64)
+    dW2 = g.T @ dp                          # second Linear: p = g W2 + b2
+    db2 = dp.sum(axis=0)
+    dh = (dp @ W2.T) * gelu_erf_grad(h)
+    dW1 = x.T @ dh                          # first Linear: h = x W1 + b1
+    db1 = dh.sum(axis=0)
+    return dW1, db1, dW2, db2
+
+
 # --------------------------------------------------------------------------- #
 # Outer-product tensors T_q, T_k (paragraph before Theorem 4.2)
 # --------------------------------------------------------------------------- #
@@ -330,3 +349,15 @@ def hla_backward(Q, K, V, dO, phi_q, phi_k, eps, form="factored"):
     for f, w in enumerate(phi_k):             # the same K feeds every key map
         dK += phi_mlp_backward(K.reshape(-1, d), *w, dkf[:, :, f].reshape(-1, dkf.shape[-1])).reshape(K.shape)
     return dQ, dK, dV, dqf, dkf
+
+
+def hla_backward_weights(Q, K, V, dO, phi_q, phi_k, eps, form="factored"):
+    """Gradients of sum(dO * O) w.r.t. the weights of phi_q and of every phi_{k_f} (one weight set per
+    map, shared by all batches and heads, so the per-token gradients are summed over B, H and N).
+    Returns (gq, [gk_1, ...]), each a tuple (dW1, db1, dW2, db2)."""
+    B, H, N, d = Q.shape
+    qf, kf = phi_features(Q, K, phi_q, phi_k)
+    dqf, dkf, _ = hla_core_backward(qf, kf, V, dO, eps, form)
+    gq = phi_mlp_backward_weights(Q.reshape(-1, d), *phi_q, dqf.reshape(-1, dqf.shape[-1]))
+    gk = [phi_mlp_backward_weights(K.reshape(-1, d), *w, dkf[:, :, f].reshape(-1, dkf.shape[-1])) for f, w in enumerate(phi_k)]
+    return gq, gk

@@ -12,7 +12,7 @@ import torch
 
 from . import build as _build
 
-HLA_OK, HLA_ERR_INVALID_ARG, HLA_ERR_UNSUPPORTED, HLA_ERR_WORKSPACE, HLA_ERR_CUDA, HLA_ERR_DEVICE_TIMEOUT = range(6)
+HLA_OK, HLA_ERR_INVALID_ARG, HLA_ERR_UNSUPPORTED, HLA_ERR_WORKSPACE, HLA_ERR_CUDA, HLA_ERR_DEVICE_TIMEOUT, HLA_ERR_NO_MEMORY = range(7)
 HLA_BF16, HLA_F32 = 0, 1
 HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 

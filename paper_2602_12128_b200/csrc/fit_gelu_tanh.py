@@ -9,38 +9,10 @@ Backward: GELU'(x) = Phi(x) + x pdf(x) through the same kind of tanh:
 (r y = (1 - th^2) / 4: the derivative of the tanh form with its inner derivative a free polynomial); fit_tanh_grad()
 fits a, b, C0, C1 against the exact GELU' on |x| <= 8.
 
-Run:  python fit_gelu_poly.py   -> prints both sets of constants and their maximum absolute errors; the constants in
-hla_tc_phi.cuh are this script's output.  (fit() / phi_f32() are the polynomial form
-Phi(x) ~ sat(1/2 + x P(min(x^2, T))) that earlier versions of the kernels used; kept for comparison.)"""
+Run:  python fit_gelu_tanh.py   -> prints both sets of constants and their maximum absolute errors; the constants in
+hla_tc_phi.cuh are this script's output."""
 import numpy as np
 from scipy.special import erf
-
-T, NCOEF = 16.0, 7
-
-
-def fit(T=T, n=NCOEF, iters=400):
-    X = np.sqrt(T)
-    x = 0.5 * X * (1 - np.cos(np.linspace(0, np.pi, 8001)))[1:]
-    A = np.stack([x ** (2 * k + 1) for k in range(n)], 1)
-    scale = np.abs(A).max(0)
-    A = A / scale
-    y = 0.5 * erf(x / np.sqrt(2))
-    w = np.ones_like(x)
-    for _ in range(iters):                      # reweighted least squares towards the minimax fit
-        coef, *_ = np.linalg.lstsq(A * w[:, None], y * w, rcond=None)
-        err = np.abs(A @ coef - y)
-        w *= 1 + 2 * err / err.max()
-        w /= w.mean()
-    return coef / scale
-
-
-def phi_f32(x, coef, T=T):
-    x = x.astype(np.float32)
-    t = np.minimum(x * x, np.float32(T))
-    p = np.float32(coef[-1])
-    for a in coef[-2::-1]:
-        p = p * t + np.float32(a)
-    return np.clip(x * p + np.float32(0.5), 0, 1).astype(np.float32)
 
 
 def fit_tanh(iters=60):
@@ -81,10 +53,3 @@ if __name__ == "__main__":
     print("tanh form of GELU': a = %.8ff, b = %.8ff, C0 = %.8ff, C1 = %.8ff, max |error| = %.3e" % (*c, err))
     (a, b), err = fit_tanh()
     print("tanh form: a = %.8ff, b = %.8ff, max |Phi error| = %.3e" % (a, b, err))
-    coef = fit()
-    print("coefficients (highest first):", ", ".join("%.9ef" % a for a in coef[::-1]))
-    x = np.linspace(-9, 9, 1800001)
-    ref = 0.5 * (1 + erf(x / np.sqrt(2)))
-    got = phi_f32(x, coef).astype(np.float64)
-    print("max |Phi_poly - Phi|: %.3e" % np.abs(got - ref).max())
-    print("max |x Phi_poly - GELU|: %.3e" % np.abs(x.astype(np.float32) * got - x * ref).max())

@@ -223,7 +223,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     if (c.dtype == HLA_BF16 && (c.d % 8) != 0) return HLA_ERR_UNSUPPORTED;   // 16-byte rows
 
     hla_ctx* x = new (std::nothrow) hla_ctx();
-    if (!x) return HLA_ERR_INVALID_ARG;
+    if (!x) return HLA_ERR_NO_MEMORY;
     x->cfg = c;
     x->BH = c.B * c.H;
     x->phi_set = false;
@@ -352,6 +352,8 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     (void)cudaGetLastError();
     if (ctx->tc) {
         const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
+        // the phi backward writes rows of dQ, dK with 32-byte stores
+        if (mlp && ((reinterpret_cast<uintptr_t>(dQ) | reinterpret_cast<uintptr_t>(dK)) & 31u)) return HLA_ERR_INVALID_ARG;
         const float* qf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.qf) : static_cast<const float*>(Q);
         const float* kf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.kf) : static_cast<const float*>(K);
         float* dqf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dqf) : static_cast<float*>(dQ);
@@ -462,6 +464,7 @@ const char* hla_status_string(hla_status s) {
         case HLA_ERR_WORKSPACE: return "workspace too small";
         case HLA_ERR_CUDA: return "CUDA error";
         case HLA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case HLA_ERR_NO_MEMORY: return "out of host memory";
     }
     return "unknown status";
 }

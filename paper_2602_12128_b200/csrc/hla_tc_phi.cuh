@@ -35,7 +35,7 @@ __device__ __forceinline__ __nv_bfloat16 half_bf16(__nv_bfloat16 w) { return __f
 // GELU'(x) = Phi(x) + x pdf(x) through one tanh.approx per element:
 //   th = tanh(x (a + b x^2)),   2 GELU'(x) ~ (1 + th) (1 + V (1 - th)) = 1 + V + th (1 - V th),   V = x (C0 + C1 x^2) / 2
 // (the derivative of a tanh-form GELU whose inner derivative is a free polynomial); a, b, C0, C1 are fitted against the
-// exact derivative (fit_gelu_poly.py: |error| < 1.5e-4 before the 2^-11 relative error of tanh.approx, < 1.3e-3 with
+// exact derivative (fit_gelu_tanh.py: |error| < 1.5e-4 before the 2^-11 relative error of tanh.approx, < 1.3e-3 with
 // it).  The kernel evaluates it with -V (negated constants) so that every step is one packed multiply or fma, and the
 // factor 1/2 sits in the staged W2^T of the dg product (exact in bf16): 9 packed + 2 special-function instructions
 // per pair of elements; the polynomial Phi plus exp form needed sixteen.
@@ -388,6 +388,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* dx_empty = bars + 23;    // 512 arrivals
     uint64_t* w_full = bars + 24;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
+    uint64_t* stage_free = bars + 26;  // 1 arrival: the previous TMA store has read the dX staging tile
+    uint64_t* stage_full = bars + 27;  // 512 arrivals: the staging tile of this drain is written
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -420,6 +422,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         mbar_init(dx_full, 1);
         mbar_init(dx_empty, 512);
         mbar_init(w_full, 1);
+        mbar_init(stage_free, 1);
+        mbar_init(stage_full, 512);
         fence_mbar_init();
         prefetch_tmap(&mapX);
         prefetch_tmap(&mapdX);
@@ -538,17 +542,29 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 mbar_arrive(dx_empty);          // the accumulator is in registers
                 const int col0 = part * HC;     // first column of this thread
                 const uint32_t sblk = smem_u32(smem + Cfg::kOffStage) + (col0 / 64) * kBlk;
-                if (tid == kPbEpiWarp0 * 32) tma_store_wait_read0();      // the previous tile's store has read the staging tile
-                named_barrier(2, 512);
+                // The two hand-overs around the staging tile go through mbarriers with bounded waits (not bar.sync), so a
+                // warp that has given up elsewhere cannot leave the others waiting for ever.
+                const bool leader = tid == kPbEpiWarp0 * 32;
+                if (leader) {
+                    tma_store_wait_read0();      // the previous tile's store has read the staging tile
+                    mbar_arrive(stage_free);
+                }
+                if (!mbar_wait(stage_free, it & 1)) { ok = false; report_timeout(status, 609); }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) return;
 #pragma unroll
                 for (int j = 0; j < HC / 8; ++j)
                     st_shared_v4(sblk + sw128_off(row, (col0 & 63) / 8 + j), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
                 fence_proxy_async();
-                named_barrier(2, 512);
-                if (tid == kPbEpiWarp0 * 32) {
-                    for (int blk = 0; blk < Cfg::kStageBlocks; ++blk)
-                        tma_store_2d(&mapdX, smem + Cfg::kOffStage + blk * kBlk, blk * 64, (int)((t0 + it) * kTileTokens));
-                    tma_store_commit();
+                mbar_arrive(stage_full);
+                if (leader) {
+                    if (mbar_wait(stage_full, it & 1)) {
+                        for (int blk = 0; blk < Cfg::kStageBlocks; ++blk)
+                            tma_store_2d(&mapdX, smem + Cfg::kOffStage + blk * kBlk, blk * 64, (int)((t0 + it) * kTileTokens));
+                        tma_store_commit();
+                    } else {
+                        report_timeout(status, 610);
+                    }
                 }
             } else {
                 const long long grow = (t0 + it) * kTileTokens + row;

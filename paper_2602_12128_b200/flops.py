@@ -15,6 +15,13 @@ def n_features(F: int, d_phi: int) -> int:
     return d_phi ** F
 
 
+def n_monomials(F: int, d_phi: int) -> int:
+    """Distinct monomials of degree F in d_phi variables: what is left of the P features of the symmetric query
+    tensor q (x) ... (x) q once equal index permutations are merged (56 of 216 for F = 3, d_phi = 6)."""
+    from math import comb
+    return comb(d_phi + F - 1, F)
+
+
 def core_fwd_flops_per_token(d: int, F: int, d_phi: int) -> int:
     """State build + readout, each 2*P*(d+1)."""
     return 2 * 2 * n_features(F, d_phi) * (d + 1)
@@ -73,3 +80,15 @@ def quadratic_layer_flops(N: int, heads: int, d: int) -> int:
     """Softmax-attention block as Table 3 counts it: projections + QK^T + AV."""
     D = heads * d
     return 4 * 2 * N * D * D + 4 * N * N * d * heads
+
+
+def folded_flops_per_token(d: int, F: int, d_phi: int, backward: bool, with_phi: bool = True) -> int:
+    """FLOPs the symmetry-folded scheme has to execute: every core contraction runs over the n_monomials(F, d_phi)
+    merged features instead of P; the phi maps are unchanged.  Used for the roofline (what the hardware must do),
+    never for the reported throughput (which stays on the algorithmic counts above)."""
+    m = n_monomials(F, d_phi)
+    core = 2 * 2 * m * (d + 1) + (4 * 2 * m * (d + 1) if backward else 0)
+    phi = 0
+    if with_phi:
+        phi = phi_fwd_flops_per_token(d, F, d_phi) + (phi_bwd_flops_per_token(d, F, d_phi) if backward else 0)
+    return core + phi

@@ -24,6 +24,19 @@ def l2err(y, ref) -> float:
     return float(np.linalg.norm(y - ref) / max(np.linalg.norm(ref), 1e-300))
 
 
+def report(name: str, **values) -> None:
+    """Prints measured parity figures (errors, kept fractions) so that a test log shows how far inside its bound a
+    comparison is; with HLA_PARITY_REPORT set to a file path the same record is appended there as a JSON line."""
+    import json
+    import os
+    rec = {"check": name, **{k: (float(v) if np.isscalar(v) else v) for k, v in values.items()}}
+    print("parity:", json.dumps(rec))
+    path = os.environ.get("HLA_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(rec) + "\n")
+
+
 def to_dev(x: np.ndarray, dtype: str):
     t = torch.from_numpy(np.ascontiguousarray(x))
     if dtype == "bf16":

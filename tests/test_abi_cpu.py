@@ -100,7 +100,15 @@ def test_calls_validate_before_launching():
     need = binding.hla_workspace_bytes(ctx)
     assert lib.hla_forward(ctx, p, p, p, p, p, need, None) == binding.HLA_ERR_INVALID_ARG
     assert lib.hla_set_phi(ctx, None, None) == binding.HLA_ERR_INVALID_ARG
+    # dQ, dK leave the tensor-core phi backward as 32-byte stores: a 16-byte-aligned dK is refused before any launch
+    # (the phi weights only have to be set, they are not read by the validation)
+    w = binding.HlaMlp(p, p, p, p)
+    ws3 = (binding.HlaMlp * 3)(w, w, w)
+    assert lib.hla_set_phi(ctx, ctypes.byref(w), ws3) == binding.HLA_OK
+    assert lib.hla_backward(ctx, p, p, p, p, p, p, p + 16, p, p, need, None) == binding.HLA_ERR_INVALID_ARG
+    assert lib.hla_backward(ctx, p, p, p, p, p, p + 16, p, p, p, need, None) == binding.HLA_ERR_INVALID_ARG
     binding.hla_destroy(ctx)
     assert lib.hla_destroy(None) == binding.HLA_ERR_INVALID_ARG
+    assert binding.status_string(binding.HLA_ERR_NO_MEMORY) == "out of host memory"
     assert binding.status_string(binding.HLA_ERR_DEVICE_TIMEOUT) == "device-side wait timed out"
     assert binding.hla_workspace_bytes(None) == 0

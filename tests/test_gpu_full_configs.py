@@ -15,7 +15,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import TOL, relerr, l2err
+from hla_testlib import TOL, relerr, l2err, report
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -118,7 +118,9 @@ def check_core_forward_heads(r: FullRun, heads):
         kf = [orc.phi_mlp(f64(r.K[b, h]), *w) for w in r.pk]
         o_e2e, eta_e2e, _, _ = orc.hla_factored(qf, kf, V, EPS)
         keep = eta_e2e >= 1e-3 * np.median(eta_e2e)
-        assert keep.mean() > 0.5
+        report(f"{s.name} head ({b},{h}) end to end", kept_fraction=keep.mean(), excluded_rows=int((~keep).sum()),
+               l2_kept=l2err(r.O[b, h][keep], o_e2e[keep]), maxnorm_kept=relerr(r.O[b, h][keep], o_e2e[keep]))
+        assert keep.mean() > 0.99
         assert l2err(r.O[b, h][keep], o_e2e[keep]) < TOL["bf16"], (b, h, l2err(r.O[b, h][keep], o_e2e[keep]))
 
 
@@ -196,3 +198,19 @@ def check_training_step(name, rng, whole_heads):
         same_q, same_k = ~flip_q.any(axis=-1), ~flip_k.any(axis=(0, 2))
         assert relerr(r.dQ[b, h][same_q], rQ[same_q]) < TOL["bf16"], (b, h)
         assert relerr(r.dK[b, h][same_k], rK[same_k]) < TOL["bf16"], (b, h)
+        # end to end against the oracle's own backward of this head (its own features, its own ReLU masks).  dV is
+        # continuous in the inputs and is bounded in the max-norm; dQ, dK are bounded on the tokens away from a ReLU
+        # kink (and, for dQ, with query features that are not small: dq_i grows like 1 / |phi_q(q_i)|).
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        eQ, eK, eV, _, _ = orc.hla_backward(f64(r.Q[sl]), f64(r.K[sl]), f64(r.V[sl]), f64(r.dO[sl]), r.pq, r.pk, EPS, "factored")
+        eQ, eK, eV = eQ[0, 0], eK[0, 0], eV[0, 0]
+        qn = np.linalg.norm(np.maximum(pre_q, 0.0), axis=-1)
+        keep_q = (np.abs(pre_q).min(axis=-1) > 5e-3 * np.abs(pre_q).max()) & (qn >= 0.5 * np.median(qn))
+        keep_k = np.abs(pre_k).min(axis=(0, 2)) > 5e-3 * np.abs(pre_k).max()
+        report(f"{s.name} head ({b},{h}) backward end to end", dV_maxnorm=relerr(r.dV[b, h], eV), kept_q=keep_q.mean(), kept_k=keep_k.mean(),
+               dQ_l2_kept=l2err(r.dQ[b, h][keep_q], eQ[keep_q]), dK_l2_kept=l2err(r.dK[b, h][keep_k], eK[keep_k]),
+               dQ_maxnorm_kept=relerr(r.dQ[b, h][keep_q], eQ[keep_q]), dK_maxnorm_kept=relerr(r.dK[b, h][keep_k], eK[keep_k]))
+        assert relerr(r.dV[b, h], eV) < TOL["bf16"], (b, h)
+        assert keep_q.mean() > 0.7 and keep_k.mean() > 0.5
+        assert l2err(r.dQ[b, h][keep_q], eQ[keep_q]) < TOL["bf16"], (b, h)
+        assert l2err(r.dK[b, h][keep_k], eK[keep_k]) < TOL["bf16"], (b, h)

@@ -6,7 +6,7 @@ import torch
 
 from oracle import hla_oracle as orc
 from paper_2602_12128_b200 import binding, synth
-from hla_testlib import DeviceRun, TOL, fold_symmetric, oracle_state, relerr, l2err
+from hla_testlib import DeviceRun, TOL, fold_symmetric, oracle_state, relerr, l2err, report
 
 pytestmark = pytest.mark.gpu
 EPS = 1e-6
@@ -57,7 +57,9 @@ def test_config2_small_bf16_forward_stagewise():
     # bf16-level error of the features has an output that swings between class averages (and ReLU makes it
     # discontinuous).  So end to end the bound is on the relative L2 error, over rows whose normaliser is not tiny.
     keep = eta >= 1e-3 * np.median(eta)
-    assert keep.mean() > 0.5
+    report("config2 end to end", kept_fraction=keep.mean(), l2_kept=l2err(O[keep], Oq[keep]), maxnorm_kept=relerr(O[keep], Oq[keep]),
+           maxnorm_all=relerr(O, Oq))
+    assert keep.mean() > 0.99
     assert l2err(O[keep], Oq[keep]) < TOL["bf16"], l2err(O[keep], Oq[keep])
     # the quadratic definition on one head
     o_def, _ = orc.hla_quadratic(qf[1, 5], [kf[1, 5, f] for f in range(3)], f64(V)[1, 5], EPS)
@@ -143,6 +145,10 @@ def test_full_backward_bf16_mlp_stagewise():
     qn = np.linalg.norm(np.maximum(pre_q, 0.0), axis=-1)
     keep_q = (np.abs(pre_q).min(axis=-1) > 5e-3 * np.abs(pre_q).max()) & (qn >= 0.5 * np.median(qn))
     keep_k = np.abs(pre_k).min(axis=(2, 4)) > 5e-3 * np.abs(pre_k).max()
+    report("reduced training step end to end", kept_q=keep_q.mean(), kept_k=keep_k.mean(), dV_maxnorm=relerr(dV, eV),
+           dQ_l2_kept=l2err(dQ[keep_q], eQ[keep_q]), dK_l2_kept=l2err(dK[keep_k], eK[keep_k]),
+           dQ_maxnorm_kept=relerr(dQ[keep_q], eQ[keep_q]), dK_maxnorm_kept=relerr(dK[keep_k], eK[keep_k]),
+           flipped_q=flip_q.mean(), flipped_k=flip_k.mean())
     assert keep_q.mean() > 0.7 and keep_k.mean() > 0.5
     assert l2err(dQ[keep_q], eQ[keep_q]) < TOL["bf16"], l2err(dQ[keep_q], eQ[keep_q])
     assert l2err(dK[keep_k], eK[keep_k]) < TOL["bf16"], l2err(dK[keep_k], eK[keep_k])

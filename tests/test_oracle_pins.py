@@ -280,6 +280,95 @@ def test_full_operator_gradients_fd():
     np.testing.assert_allclose(dV, fd_grad(lambda x: loss(V_=x), V, 1e-6), rtol=2e-5, atol=1e-8)
 
 
+def test_phi_weight_gradients_fd():
+    """dW1, db1, dW2, db2 of one map against central differences of sum(dfeat * phi(x))."""
+    rng = np.random.default_rng(5)
+    n, d, dphi = 7, 4, 3
+    x = rng.standard_normal((n, d))
+    W = [rng.standard_normal((d, d)), rng.standard_normal(d), rng.standard_normal((d, dphi)), rng.standard_normal(dphi) + 0.3]
+    dfeat = rng.standard_normal((n, dphi))
+    got = orc.phi_mlp_backward_weights(x, *W, dfeat)
+    assert [g.shape for g in got] == [w.shape for w in W]
+    pre = orc.phi_mlp(x, *W, relu=False)
+    assert np.abs(pre).min() > 1e-3 and np.any(pre < 0) and np.any(pre > 0)      # away from the ReLU kink, both sides present
+    for i in range(4):
+        def loss(w, i=i):
+            Wv = list(W)
+            Wv[i] = w
+            return float(np.sum(dfeat * orc.phi_mlp(x, *Wv)))
+        np.testing.assert_allclose(got[i], fd_grad(loss, W[i]), rtol=1e-6, atol=1e-8)
+    # a dropped ReLU mask or a transposed product would also break these closed forms
+    mask = pre > 0
+    np.testing.assert_allclose(got[3], (dfeat * mask).sum(axis=0), rtol=1e-13)
+    g = orc.gelu_erf(x @ W[0] + W[1])
+    want_dW2 = sum(np.multiply.outer(g[t], (dfeat * mask)[t]) for t in range(n))
+    np.testing.assert_allclose(got[2], want_dW2, rtol=1e-12, atol=1e-14)
+
+
+def test_full_operator_weight_gradients_fd():
+    """Weight gradients of every map through the core, summed over batches, heads and tokens."""
+    rng = np.random.default_rng(12)
+    B, H, N, d, dphi, F = 2, 2, 5, 3, 2, 3
+    Q = rng.standard_normal((B, H, N, d)); K = rng.standard_normal((B, H, N, d))
+    V = rng.standard_normal((B, H, N, d)); dO = rng.standard_normal((B, H, N, d))
+    mk = lambda: [rng.standard_normal((d, d)), rng.standard_normal(d), rng.standard_normal((d, dphi)), rng.standard_normal(dphi) + 0.7]
+    phi_q, phi_k = mk(), [mk() for _ in range(F)]
+    eps = 1e-3
+    gq, gk = orc.hla_backward_weights(Q, K, V, dO, phi_q, phi_k, eps)
+
+    def loss(pq, pk):
+        return float(np.sum(dO * orc.hla_forward(Q, K, V, pq, pk, eps, "quadratic")[0]))
+
+    for i in range(4):
+        def lq(w, i=i):
+            pq = list(phi_q)
+            pq[i] = w
+            return loss(pq, phi_k)
+        np.testing.assert_allclose(gq[i], fd_grad(lq, phi_q[i], 1e-6), rtol=5e-5, atol=1e-8)
+        for f in range(F):
+            def lk(w, i=i, f=f):
+                pk = [list(m) for m in phi_k]
+                pk[f][i] = w
+                return loss(phi_q, pk)
+            np.testing.assert_allclose(gk[f][i], fd_grad(lk, phi_k[f][i], 1e-6), rtol=5e-5, atol=1e-8)
+
+
+def test_whole_operator_wrappers_against_per_head_per_token_loops():
+    """The [B,H,N,*] wrappers (phi_features, hla_core_forward, hla_forward, hla_core_backward) against explicit loops
+    over batches, heads and tokens that call the per-token map and the per-head definition: a wrong stack axis,
+    a reshape that mixes heads, or key maps applied in the wrong order fails here.  Every map has its own weights."""
+    rng = np.random.default_rng(21)
+    B, H, N, d, dphi, F = 2, 3, 5, 4, 2, 3
+    Q = rng.standard_normal((B, H, N, d)); K = rng.standard_normal((B, H, N, d)); V = rng.standard_normal((B, H, N, d))
+    dO = rng.standard_normal((B, H, N, d))
+    mk = lambda: (rng.standard_normal((d, d)), rng.standard_normal(d), rng.standard_normal((d, dphi)), rng.standard_normal(dphi) + 0.5)
+    phi_q, phi_k = mk(), [mk() for _ in range(F)]
+    eps = 1e-4
+    qf, kf = orc.phi_features(Q, K, phi_q, phi_k)
+    assert qf.shape == (B, H, N, dphi) and kf.shape == (B, H, F, N, dphi)
+    O, eta, qf2, kf2 = orc.hla_forward(Q, K, V, phi_q, phi_k, eps, "factored")
+    assert np.array_equal(qf, qf2) and np.array_equal(kf, kf2)
+    dqf, dkf, dV = orc.hla_core_backward(qf, kf, V, dO, eps, "factored")
+    for b in range(B):
+        for h in range(H):
+            q_loop = np.stack([orc.phi_mlp(Q[b, h, n][None, :], *phi_q)[0] for n in range(N)])
+            np.testing.assert_allclose(qf[b, h], q_loop, rtol=1e-13, atol=1e-15)
+            ks_loop = []
+            for f in range(F):
+                k_loop = np.stack([orc.phi_mlp(K[b, h, n][None, :], *phi_k[f])[0] for n in range(N)])
+                np.testing.assert_allclose(kf[b, h, f], k_loop, rtol=1e-13, atol=1e-15)
+                ks_loop.append(k_loop)
+            want = brute_force(q_loop.tolist(), [k.tolist() for k in ks_loop], V[b, h].tolist(), eps)
+            np.testing.assert_allclose(O[b, h], want, rtol=1e-10, atol=1e-13)
+            o_def, eta_def = orc.hla_quadratic(q_loop, ks_loop, V[b, h], eps)
+            np.testing.assert_allclose(eta[b, h], eta_def, rtol=1e-12)
+            dq, dks, dv = orc.hla_quadratic_backward(q_loop, ks_loop, V[b, h], dO[b, h], eps)
+            np.testing.assert_allclose(dqf[b, h], dq, rtol=1e-9, atol=1e-12)
+            np.testing.assert_allclose(dV[b, h], dv, rtol=1e-9, atol=1e-12)
+            for f in range(F):
+                np.testing.assert_allclose(dkf[b, h, f], dks[f], rtol=1e-9, atol=1e-12)
+
+
 # ---- FLOP model against the paper's tables ---------------------------------------------------
 def load_golden():
     path = os.path.join(os.path.dirname(__file__), "golden", "paper_flop_tables.txt")

@@ -45,6 +45,55 @@ def test_static_scratch_forward_matches_workspace_forward(dtype, d, N, H):
     assert np.array_equal(results[0], ref) and np.array_equal(results[1], ref)
 
 
+class _RawDeviceBytes:
+    """Zero-copy view of `nbytes` of device memory at `ptr` for torch.as_tensor."""
+
+    def __init__(self, ptr, nbytes):
+        self.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (ptr, False), "version": 2}
+
+
+@pytest.mark.gpu
+def test_static_scratch_with_phi_maps_after_another_user_and_as_backward_workspace():
+    """The array is shared by every context and keeps what the last call left.  Here another context (other shape,
+    other mode) uses it first and it is then overwritten with NaN bytes, before a forward with the phi maps runs on it;
+    hla_backward then takes the array as its workspace (the forward's features and state live there).  Everything
+    must agree bit for bit with the same calls on an ordinary workspace: nothing stale is read."""
+    s = synth.HlaShape("t", 1, 2, 1000, 128, "bf16", "rms_qk", backward=True)
+    Q, K, V = synth.make_qkv(s)
+    dO = synth.make_dO(s)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    op = binding.Hla(s.B, s.H, s.N, s.d, dtype="bf16", phi="mlp", eps=EPS)
+    op.set_phi(tuple(to_dev(a, "bf16") for a in pq), [tuple(to_dev(a, "bf16") for a in w) for w in pk])
+    assert binding.hla_workspace_bytes(op.ctx) <= binding.HLA_STATIC_WS_BYTES
+    Qd, Kd, Vd, dOd = (to_dev(a, "bf16") for a in (Q, K, V, dO))
+    O_ref = op.forward(Qd, Kd, Vd)
+    ref = [to_np(t) for t in (O_ref,) + tuple(op.backward(Qd, Kd, Vd, O_ref, dOd))]
+    torch.cuda.synchronize()
+    assert op.device_status() == binding.HLA_OK
+
+    # another user of the array: a feature-level fp32 context of a different shape
+    t = synth.HlaShape("u", 1, 3, 333, 16, "f32", "inv_sqrt_d")
+    _, _, Vt = synth.make_qkv(t)
+    qf, kf = synth.make_features(t)
+    other = binding.Hla(t.B, t.H, t.N, t.d, dtype="f32", phi="none", eps=EPS)
+    vt = to_dev(Vt, "f32")
+    scratch = binding.hla_forward_static(other.ctx, to_dev(qf, "f32"), to_dev(kf, "f32"), vt, torch.empty_like(vt))
+    assert binding.hla_last_device_status(other.ctx, scratch) == binding.HLA_OK
+    view = torch.as_tensor(_RawDeviceBytes(scratch, binding.HLA_STATIC_WS_BYTES), device="cuda")
+    assert view.data_ptr() == scratch
+
+    out, dQ, dK, dV = (torch.empty_like(Vd) for _ in range(4))
+    for call in range(2):
+        view.fill_(0xFF)                     # every fp32 / bf16 word of the array is now a NaN
+        for x in (out, dQ, dK, dV):
+            x.fill_(float("nan"))
+        assert binding.hla_forward_static(op.ctx, Qd, Kd, Vd, out) == scratch
+        binding.hla_backward(op.ctx, Qd, Kd, Vd, out, dOd, dQ, dK, dV, scratch, workspace_bytes=binding.HLA_STATIC_WS_BYTES)
+        assert binding.hla_last_device_status(op.ctx, scratch) == binding.HLA_OK
+        for got, want in zip((out, dQ, dK, dV), ref):
+            assert np.array_equal(to_np(got), want), call
+
+
 def test_static_scratch_refuses_shapes_that_need_more():
     big = binding.Hla(2, 24, 32760, 128, dtype="bf16", phi="mlp", eps=EPS, device=None)      # no workspace tensor is created
     assert binding.hla_workspace_bytes(big.ctx) > binding.HLA_STATIC_WS_BYTES
