@@ -66,7 +66,7 @@ def kernel_models(shape):
         "tc_state_build": (contr, d * e + Fn * dp * 4, "tensor"),
         "tc_readout": (contr, d * e + dp * 4 + 4, "tensor"),
         "tc_phiq_readout": (phi1 + contr, 2 * d * e + dp * 4 + 4, "tensor"),      # phi_q + readout + normaliser in one kernel
-        "tc_phi_forward_k": (Fn * phi1, d * e + Fn * dp * 4, "tensor"),
+        "tc_phik_state": (Fn * phi1 + contr, 2 * d * e + Fn * dp * 4, "tensor"),       # phi_k1..F + state build in one kernel
         "tc_bwd_query": (2 * contr, 2 * d * e + 3 * dp * 4, "tensor"),
         "tc_bwd_key": (2 * contr, 2 * d * e + 2 * Fn * dp * 4, "tensor"),
         "tc_phi_backward_q": (4 * d * d + 2 * d * dp, 2 * d * e + 2 * dp * 4, "tensor"),
@@ -83,7 +83,7 @@ def kernel_models(shape):
 # DRAM traffic per token-head of a launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # scaled by token-heads; see profiles/).  None = not captured yet.
 NCU_TRAFFIC_PER_TOKEN_HEAD = {
-    "tc_phi_forward_k": 313.5, "tc_state_build": 333.0, "tc_phiq_readout": 477.8, "tc_bwd_query": 305.7, "tc_bwd_key": 594.1,
+    "tc_phik_state": None, "tc_state_build": 333.0, "tc_phiq_readout": 477.8, "tc_bwd_query": 305.7, "tc_bwd_key": 594.1,
     "tc_phi_backward_q": 498.8, "tc_phi_backward_k": 619.3,
 }
 
@@ -403,7 +403,8 @@ def main():
         ms_steady = w.timed(n_steady) / n_steady
     t_win1 = time.time()
     clocks = sampler.window(t_win0, t_win1)
-    kt = {} if args.profile else w.kernel_times(8)
+    n_kt = max(8, n_steady)          # as long as the steady run, so the per-kernel times are taken under the same clocks
+    kt = {} if args.profile else w.kernel_times(n_kt)
     ms_step = multi.max_over_ranks(ms_total, dist, dev) / args.steps
     if ms_steady is not None:
         ms_steady = multi.max_over_ranks(ms_steady, dist, dev)
@@ -471,7 +472,7 @@ def main():
     # ---- roofline of the dominant kernel ------------------------------------------------------------------------------
     models = kernel_models(shape)
     tot_k = max(sum(x[0] for x in kt.values()), 1e-9)
-    per_kernel = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / 8, "share": v[0] / tot_k} for k, v in kt.items()}
+    per_kernel = {k: {"ms_per_launch": v[0] / v[1], "launches_per_step": v[1] / n_kt, "share": v[0] / tot_k} for k, v in kt.items()}
     roof = None
     if kt:
         top = max(kt, key=lambda k: kt[k][0])

@@ -11,6 +11,7 @@
 #include "hla_tc.cuh"
 #include "hla_tc_phi.cuh"
 #include "hla_tc_fused.cuh"
+#include "hla_tc_fused_k.cuh"
 
 using namespace hla;
 
@@ -24,6 +25,7 @@ struct hla_ctx {
     hla_mlp phi_k[kMaxF];
     hla_ws_layout L;
     size_t off_part;    // split partials (scratch)
+    int k_pieces;       // most pieces a head has in the fused key-side kernel of the forward
     tc::Plan tcp;       // tensor-core operand buffers inside the workspace
     size_t ws_bytes;
     int sm_count;
@@ -278,7 +280,15 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     L.state_rows = x->tc ? tc::kMono : P;
     L.n_splits = S;
     L.tensor_core = x->tc ? 1 : 0;
-    x->off_part = cv.take((size_t)x->BH * S * P * D.ld * 4);
+    // partial states: S per head from the split kernels, or the pieces of the fused key-side kernel (folded rows)
+    x->k_pieces = 0;
+    size_t part_bytes = (size_t)x->BH * S * P * D.ld * 4;
+    if (x->tc && mlp) {
+        x->k_pieces = tc::fused_key_max_pieces(x->BH, tiles, tc::fused_key_grid(x->BH, c.N, x->sm_count));
+        const size_t need = (size_t)x->BH * x->k_pieces * tc::kMono * D.ld * 4;
+        if (need > part_bytes) part_bytes = need;
+    }
+    x->off_part = cv.take(part_bytes);
     if (x->tc) cv.off = tc::plan(x->tcp, D, x->BH, cv.off);
     x->ws_bytes = cv.off;
     *out = x;
@@ -324,11 +334,12 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
     if (ctx->tc) {
         const float *qf, *kf;
         if (ctx->cfg.phi == HLA_PHI_MLP) {
-            // key maps -> state build -> reduction -> one kernel for phi_q, readout and normaliser
-            s = tc::phi_forward_k(ctx->D, ctx->BH, ctx->phi_k, K, ws, ctx->L, ctx->sm_count, ctx->rec);
+            // one kernel for the key maps and the state build -> reduction of its pieces -> one kernel for phi_q, readout
+            // and normaliser
+            s = tc::phik_state(ctx->D, ctx->BH, ctx->phi_k, K, V, ws, ctx->L, ctx->off_part, ctx->k_pieces, ctx->sm_count, ctx->rec);
             if (s != HLA_OK) return s;
-            kf = reinterpret_cast<const float*>(ws + ctx->L.kf);
-            s = tc::core_forward(ctx->tcp, ctx->D, ctx->BH, nullptr, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec, false);
+            s = tc::reduce_pieces(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, ctx->off_part, ctx->k_pieces,
+                                  tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec);
             if (s != HLA_OK) return s;
             return tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
         } else {

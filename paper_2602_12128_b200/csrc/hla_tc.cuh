@@ -413,20 +413,30 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
 // (column d = folded z) and the two bf16 MMA operands of that state.
 // =======================================================================================
 // grid = (8, heads): block c of a head owns the monomials 8c .. 8c+7 (block 7 owns only the zero padding 56..63).
+// The partials of head bh are the slots [bh * S, bh * S + count).  With G == 0 every head has count = S slots (kernels
+// whose grid is splits x heads); with G > 0 the producer was a persistent kernel of G CTAs over heads x T work items and
+// the head's slots are its pieces, one per CTA that touched it (see owner_of_work).
+__host__ __device__ inline int owner_of_work(long long w, long long total, int G) { return (int)(((w + 1) * G - 1) / total); }
+
 template <int DV>
 __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __restrict__ part, float* __restrict__ state,
-                                                             __nv_bfloat16* __restrict__ b3, __nv_bfloat16* __restrict__ bq, int S, int ld) {
+                                                             __nv_bfloat16* __restrict__ b3, __nv_bfloat16* __restrict__ bq, int S, int ld, int G, int T) {
     __shared__ float sm[8][kMaxD + 8];
     const int m0 = 8 * blockIdx.x, bh = blockIdx.y, tid = threadIdx.x;
     grid_launch_dependents();
     grid_dependency_wait();
     const size_t n_per = (size_t)kMono * ld;
+    int count = S;
+    if (G > 0) {
+        const long long total = (long long)gridDim.y * T;
+        count = owner_of_work((long long)bh * T + T - 1, total, G) - owner_of_work((long long)bh * T, total, G) + 1;
+    }
     for (int i = tid; i < 8 * ld; i += 256) {
         const int mm = i / ld, col = i - mm * ld, m = m0 + mm;
         float a = 0.f;
         if (m < kMono) {
             const float* src = part + (size_t)bh * S * n_per + (size_t)m * ld + col;
-            for (int s = 0; s < S; ++s) a += src[(size_t)s * n_per];      // fixed order: bit-reproducible
+            for (int s = 0; s < count; ++s) a += src[(size_t)s * n_per];      // fixed order: bit-reproducible
             state[(size_t)bh * n_per + (size_t)m * ld + col] = a;
         }
         sm[mm][col] = a;
@@ -1135,7 +1145,7 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     launch_pdl(tc_state_build_kernel<DV>, dim3(D.S, BH), dim3(kSbThreads), kSbSmem, st, mapV, kf, part, D.N, D.S, D.ld, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, state, b3, bq, D.S, D.ld);
+    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, state, b3, bq, D.S, D.ld, 0, 0);
     if (!rec.end()) return HLA_ERR_CUDA;
     if (!readout) return HLA_OK;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
@@ -1143,6 +1153,19 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_readout");
     launch_pdl(tc_readout_kernel<DV>, grid, dim3(kRoThreads), RoCfg<DV>::kSmem, st, mapB3, mapO, qf, eta, D.N, BH, D.eps, status);
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+
+// Reduction of the pieces the fused key-side kernel (G CTAs over heads x T tiles, at most `smax` pieces per head) left.
+inline hla_status reduce_pieces(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec) {
+    __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
+    __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
+    float* part = reinterpret_cast<float*>(ws + off_part);
+    float* state = reinterpret_cast<float*>(ws + L.state);
+    const int T = (D.N + kTileTokens - 1) / kTileTokens;
+    rec.begin("tc_reduce_emit");
+    if (D.d == 128) launch_pdl(tc_reduce_emit_kernel<128>, dim3(8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
+    else launch_pdl(tc_reduce_emit_kernel<64>, dim3(8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
@@ -1176,7 +1199,7 @@ inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, con
     launch_pdl(tc_bwd_query_kernel<DV>, dim3(D.S, BH), dim3(kBqThreads), kBqSmem, st, mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld);
+    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld, 0, 0);
     if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
