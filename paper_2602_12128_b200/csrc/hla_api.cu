@@ -30,6 +30,8 @@ struct hla_ctx {
     size_t ws_bytes;
     int sm_count;
     LaunchRec rec;      // launch counter and optional per-kernel event timing
+    tc::HostCache hc;   // tensor maps and kernel attributes already set up by earlier calls
+    int device;         // device the context was created on (the kernel attributes above are per device)
 };
 
 namespace {
@@ -197,6 +199,15 @@ hla_status check_call(const hla_ctx* c, const void* const* ptrs, int n, const vo
     return HLA_OK;
 }
 
+// The kernel attributes a context has set belong to the device that was current then.
+void follow_device(hla_ctx* ctx) {
+    int dev = ctx->device;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev != ctx->device) {
+        ctx->hc.nfuncs = 0;
+        ctx->device = dev;
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -236,6 +247,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) x->sm_count = n;
     }
     (void)cudaGetLastError();
+    x->device = dev;
     Dims& D = x->D;
     D.B = c.B; D.H = c.H; D.N = c.N; D.d = c.d; D.F = c.F; D.dphi = c.d_phi; D.P = P;
     D.ld = c.d + 4;
@@ -331,6 +343,8 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
     ctx->rec.start_call(st);
     (void)cudaGetLastError();
     if (cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
+    follow_device(ctx);
+    tc::HostCacheScope scope(&ctx->hc);
     if (ctx->tc) {
         const float *qf, *kf;
         if (ctx->cfg.phi == HLA_PHI_MLP) {
@@ -361,6 +375,8 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     char* ws = static_cast<char*>(workspace);
     ctx->rec.start_call(st);
     (void)cudaGetLastError();
+    follow_device(ctx);
+    tc::HostCacheScope scope(&ctx->hc);
     if (ctx->tc) {
         const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
         // the phi backward writes rows of dQ, dK with 32-byte stores

@@ -77,28 +77,67 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// Per-context memo of what a call would otherwise redo on the host every time: encoded tensor maps (keyed by base
+// pointer and geometry; a caller that passes the same buffers again pays a 128-byte copy instead of a driver call) and
+// the kernels whose dynamic shared-memory limit has already been raised.  hla_forward / hla_backward make their
+// context's memo current for the calling thread while they run.
+struct HostCache {
+    struct MapEntry { const void* ptr; uint64_t k0, k1; CUtensorMap map; };
+    static constexpr int kMaps = 32, kFuncs = 24;
+    MapEntry maps[kMaps];
+    int nmaps = 0, next = 0;
+    const void* funcs[kFuncs];
+    int nfuncs = 0;
+    const CUtensorMap* find(const void* ptr, uint64_t k0, uint64_t k1) const {
+        for (int i = 0; i < nmaps; ++i)
+            if (maps[i].ptr == ptr && maps[i].k0 == k0 && maps[i].k1 == k1) return &maps[i].map;
+        return nullptr;
+    }
+    void insert(const void* ptr, uint64_t k0, uint64_t k1, const CUtensorMap& m) {
+        MapEntry& e = maps[nmaps < kMaps ? nmaps++ : (next++ % kMaps)];
+        e.ptr = ptr; e.k0 = k0; e.k1 = k1; e.map = m;
+    }
+};
+inline thread_local HostCache* t_host_cache = nullptr;
+struct HostCacheScope {
+    explicit HostCacheScope(HostCache* c) { t_host_cache = c; }
+    ~HostCacheScope() { t_host_cache = nullptr; }
+};
+
 // bf16 tensor [BH][N][d] (d innermost), box = 64 columns x box_rows tokens of one head, 128-byte swizzle.
 inline bool make_map_bhnd(CUtensorMap* m, const void* ptr, int BH, int N, int d, int box_rows) {
+    const uint64_t k0 = (1ull << 63) | ((uint64_t)(uint32_t)BH << 32) | (uint32_t)N, k1 = ((uint64_t)(uint32_t)d << 32) | (uint32_t)box_rows;
+    if (t_host_cache)
+        if (const CUtensorMap* hit = t_host_cache->find(ptr, k0, k1)) { *m = *hit; return true; }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    if (t_host_cache) t_host_cache->insert(ptr, k0, k1, *m);
+    return true;
 }
 
 // bf16 matrix [rows][cols], box = 64 columns x box_rows, 128-byte swizzle.
 inline bool make_map_2d(CUtensorMap* m, const void* ptr, size_t rows, int cols, int box_rows) {
+    const uint64_t k0 = (uint64_t)rows, k1 = ((uint64_t)(uint32_t)cols << 32) | (uint32_t)box_rows;
+    if (t_host_cache)
+        if (const CUtensorMap* hit = t_host_cache->find(ptr, k0, k1)) { *m = *hit; return true; }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t es[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    if (t_host_cache) t_host_cache->insert(ptr, k0, k1, *m);
+    return true;
 }
 
 // Launch with programmatic stream serialization (see grid_dependency_wait): the kernel's blocks may start while the
@@ -1124,7 +1163,16 @@ __global__ void tc_wait_selftest_kernel(int* status, unsigned long long limit_ns
 
 // ---- host launch helpers ---------------------------------------------------------------
 template <typename K>
-inline bool set_smem(K kernel, int bytes) { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess; }
+inline bool set_smem(K kernel, int bytes) {
+    const void* key = reinterpret_cast<const void*>(kernel);
+    HostCache* hc = t_host_cache;
+    if (hc)
+        for (int i = 0; i < hc->nfuncs; ++i)
+            if (hc->funcs[i] == key) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (hc && hc->nfuncs < HostCache::kFuncs) hc->funcs[hc->nfuncs++] = key;
+    return true;
+}
 
 template <int DV>
 inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
