@@ -501,6 +501,37 @@ def main():
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                "sample": f"{nh} of {shape.B * shape.H} heads of {shape.name} (N={shape.N}, d={shape.d}), numpy fp64 factored form with BLAS threads, {dt:.1f} s"}
 
+    # ---- gradients of the phi weights (a separate call after the backward; not part of `value`) ------------------------
+    wgrad = None
+    if shape.backward and not args.profile and world == 1:
+        gq, gk = op.backward_weights(w.Q, w.K)        # allocates the outputs once
+        torch.cuda.synchronize()
+
+        def wstep():
+            binding.hla_backward_weights(op.ctx, w.Q, w.K, gq, gk, op.workspace)
+
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _ in range(5):
+            wstep()
+        ev1.record()
+        torch.cuda.synchronize()
+        est_w = ev0.elapsed_time(ev1) / 5
+        n_w = int(min(max(math.ceil(500.0 / est_w), 10), 20000))
+        for _ in range(n_w):                          # untimed, to settle the clocks
+            wstep()
+        ev0.record()
+        for _ in range(n_w):
+            wstep()
+        ev1.record()
+        torch.cuda.synchronize()
+        ms_w = ev0.elapsed_time(ev1) / n_w
+        fl_w = shape.B * shape.H * shape.N * (1 + shape.F) * (2 * shape.d * shape.d + 2 * shape.d * shape.d_phi)
+        wgrad = {"ms_per_call": ms_w, "calls": n_w, "tflops": fl_w / (ms_w * 1e-3) / 1e12, "gpu_launches_per_call": op.launches(),
+                 "flops": fl_w, "note": "hla_backward_weights: dW1, db1, dW2, db2 of phi_q and phi_k1..F; FLOPs = the two weight-gradient "
+                 "products per map (the recomputed hidden layer is not counted)"}
+        del gq, gk
+
     tensor_mb = w.Q.numel() * w.Q.element_size() / 1e6
     launches_per_step = w.launches
     # ---- the other configurations, timed by the same code (single-GPU runs only) ----------------------------------------
@@ -523,7 +554,7 @@ def main():
             "tokens_per_s": multi.whole_job_rate(shape.B * shape.N, world, ms_step),
             "step_roofline": roofline_of(shape, ms_step, world, peaks),
             "roofline": roof, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "clocks": clocks, "extra": extra}
+            "clocks": clocks, "weight_gradients": wgrad, "extra": extra}
     if clocks.get("sm_mhz"):
         line["ms_x_mhz"] = ms_step * clocks["sm_mhz"]
     print(json.dumps(line), flush=True)

@@ -92,6 +92,14 @@ typedef struct {
     const void *W1, *b1, *W2, *b2;
 } hla_mlp;
 
+/*
+ * Where hla_backward_weights puts the gradients of one feature network: fp32 device buffers with the shapes of the
+ * weights, dW1 [d][d], db1 [d], dW2 [d][d_phi], db2 [d_phi], 16-byte aligned.  The call overwrites them.
+ */
+typedef struct {
+    void *dW1, *db1, *dW2, *db2;
+} hla_mlp_grad;
+
 /* Byte offsets of the regions of the workspace that outlive a call (for
  * checking and for callers that want the state).  A region that the
  * configuration does not use has offset (size_t)-1. */
@@ -145,6 +153,18 @@ hla_status hla_forward(hla_ctx *ctx, const void *Q, const void *K, const void *V
 hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *V, const void *O,
                         const void *dO, void *dQ, void *dK, void *dV,
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Gradients of sum(dO * O) with respect to the weights of the feature networks (Section 5, "Training Details": the
+ * paper trains the phi maps with the rest of the model; Algorithm 1 step 4 defines where they act).  HLA_PHI_MLP
+ * contexts on the tensor-core kernels only (HLA_ERR_UNSUPPORTED otherwise).  Call it after hla_backward with the
+ * same Q, K and the same workspace: it reads the features the forward kept and the feature gradients the backward
+ * left there, recomputes the hidden layer, and sums over all batches, heads and tokens (one weight set per map is
+ * shared by all of them).  dphi_q receives the gradients of phi_q, dphi_k points to F entries for phi_k1..F; either
+ * may be NULL to skip that side.  The sums are formed in a fixed order: results are bit-reproducible.
+ */
+hla_status hla_backward_weights(hla_ctx *ctx, const void *Q, const void *K, const hla_mlp_grad *dphi_q, const hla_mlp_grad *dphi_k,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Forward without a caller-provided workspace (no counterpart in the paper: a

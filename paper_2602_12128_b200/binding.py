@@ -17,7 +17,7 @@ HLA_BF16, HLA_F32 = 0, 1
 HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
-    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_forward_static",
+    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_backward_weights", "hla_forward_static",
     "hla_last_device_status", "hla_selftest_bounded_wait", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
     "hla_destroy", "hla_status_string",
 ]
@@ -30,6 +30,10 @@ class HlaConfig(ctypes.Structure):
 
 class HlaMlp(ctypes.Structure):
     _fields_ = [("W1", c_void_p), ("b1", c_void_p), ("W2", c_void_p), ("b2", c_void_p)]
+
+
+class HlaMlpGrad(ctypes.Structure):
+    _fields_ = [("dW1", c_void_p), ("db1", c_void_p), ("dW2", c_void_p), ("db2", c_void_p)]
 
 
 class HlaWsLayout(ctypes.Structure):
@@ -72,6 +76,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_forward.restype = c_int32
     lib.hla_backward.argtypes = [c_void_p] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
     lib.hla_backward.restype = c_int32
+    lib.hla_backward_weights.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(HlaMlpGrad), POINTER(HlaMlpGrad), c_void_p, c_size_t, c_void_p]
+    lib.hla_backward_weights.restype = c_int32
     lib.hla_forward_static.argtypes = [c_void_p] + [c_void_p] * 4 + [c_void_p, POINTER(c_void_p)]
     lib.hla_forward_static.restype = c_int32
     lib.hla_last_device_status.argtypes = [c_void_p, c_void_p, c_void_p]
@@ -157,6 +163,16 @@ def hla_backward(ctx: int, Q, K, V, O, dO, dQ, dK, dV, workspace, stream=None, w
                                      _ptr(workspace), nbytes, _stream(stream))
     if st != HLA_OK:
         raise HlaError(st, "hla_backward")
+
+
+def hla_backward_weights(ctx: int, Q, K, dphi_q, dphi_k, workspace, stream=None, workspace_bytes=None) -> None:
+    """dphi_q = (dW1, db1, dW2, db2) fp32 device tensors or None; dphi_k = list of F such tuples or None."""
+    nbytes = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
+    q = byref(HlaMlpGrad(*[_ptr(t) for t in dphi_q])) if dphi_q is not None else None
+    ks = (HlaMlpGrad * len(dphi_k))(*[HlaMlpGrad(*[_ptr(t) for t in w]) for w in dphi_k]) if dphi_k is not None else None
+    st = load_library().hla_backward_weights(ctx, _ptr(Q), _ptr(K), q, ks, _ptr(workspace), nbytes, _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_backward_weights")
 
 
 HLA_STATIC_WS_BYTES = 16 * 1024 * 1024
@@ -245,6 +261,15 @@ class Hla:
         dV = torch.empty_like(V) if dV is None else dV
         hla_backward(self.ctx, Q, K, V, O, dO, dQ, dK, dV, self.workspace, stream)
         return dQ, dK, dV
+
+    def backward_weights(self, Q, K, stream=None):
+        """Weight gradients of phi_q and phi_k1..F (fp32, shapes of the weights), after backward()."""
+        F = self.cfg.F or 3
+        d, dphi = self.cfg.d, self.cfg.d_phi or (6 if F == 3 else 12)
+        mk = lambda: tuple(torch.empty(s, dtype=torch.float32, device=self.device) for s in ((d, d), (d,), (d, dphi), (dphi,)))
+        gq, gk = mk(), [mk() for _ in range(F)]
+        hla_backward_weights(self.ctx, Q, K, gq, gk, self.workspace, stream)
+        return gq, gk
 
     def region(self, name, dtype=torch.float32):
         """View of a persistent workspace region (see hla_ws_layout) as a flat tensor from its offset to the end."""

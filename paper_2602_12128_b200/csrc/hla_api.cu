@@ -12,6 +12,7 @@
 #include "hla_tc_phi.cuh"
 #include "hla_tc_fused.cuh"
 #include "hla_tc_fused_k.cuh"
+#include "hla_tc_wgrad.cuh"
 
 using namespace hla;
 
@@ -26,6 +27,7 @@ struct hla_ctx {
     hla_ws_layout L;
     size_t off_part;    // split partials (scratch)
     int k_pieces;       // most pieces a head has in the fused key-side kernel of the forward
+    size_t off_wpart;   // per-CTA partials of the weight gradients (scratch; tensor-core path with the phi maps)
     tc::Plan tcp;       // tensor-core operand buffers inside the workspace
     size_t ws_bytes;
     int sm_count;
@@ -301,6 +303,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
         if (need > part_bytes) part_bytes = need;
     }
     x->off_part = cv.take(part_bytes);
+    x->off_wpart = (x->tc && mlp) ? cv.take(tc::wgrad_part_bytes(c.d, (long long)x->BH * c.N, x->sm_count)) : kNone;
     if (x->tc) cv.off = tc::plan(x->tcp, D, x->BH, cv.off);
     x->ws_bytes = cv.off;
     *out = x;
@@ -391,6 +394,32 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     }
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
+}
+
+hla_status hla_backward_weights(hla_ctx* ctx, const void* Q, const void* K, const hla_mlp_grad* dphi_q, const hla_mlp_grad* dphi_k, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
+    const void* ptrs[2] = {Q, K};
+    hla_status s = check_call(ctx, ptrs, 2, workspace, workspace_bytes);
+    if (s != HLA_OK) return s;
+    if (ctx->cfg.phi != HLA_PHI_MLP) return HLA_ERR_INVALID_ARG;
+    if (!ctx->tc) return HLA_ERR_UNSUPPORTED;
+    const hla_mlp_grad* all[1 + kMaxF];
+    int n = 0;
+    if (dphi_q) all[n++] = dphi_q;
+    if (dphi_k)
+        for (int f = 0; f < ctx->D.F; ++f) all[n++] = dphi_k + f;
+    for (int i = 0; i < n; ++i) {
+        const void* p[4] = {all[i]->dW1, all[i]->db1, all[i]->dW2, all[i]->db2};
+        for (int j = 0; j < 4; ++j)
+            if (!p[j] || !aligned16(p[j])) return HLA_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    ctx->rec.start_call(st);
+    (void)cudaGetLastError();
+    follow_device(ctx);
+    tc::HostCacheScope scope(&ctx->hc);
+    return tc::phi_wgrad(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, dphi_q, dphi_k, static_cast<char*>(workspace), ctx->L, ctx->off_wpart,
+                         ctx->sm_count, ctx->rec);
 }
 
 // ---- forward on the library's own scratch array ---------------------------------------------

@@ -146,7 +146,7 @@ def test_config4_long_bf16_forward():
 
 def test_config5_train_bf16_forward_backward():
     """B=2, H=24, N=32760, d=128, dO ~ N(0,1): dQ, dK, dV against the oracle's analytic gradients."""
-    check_training_step("train_bf16", np.random.default_rng(13), whole_heads=4)
+    check_training_step("train_bf16", np.random.default_rng(13), whole_heads=4, weights=True)
 
 
 def test_paper_resolution_r2_forward_backward():
@@ -155,7 +155,32 @@ def test_paper_resolution_r2_forward_backward():
     check_training_step("paper_r2_bf16", np.random.default_rng(14), whole_heads=2)
 
 
-def check_training_step(name, rng, whole_heads):
+def check_weight_gradients(r: FullRun):
+    """hla_backward_weights at full size, stage-wise: the oracle's weight gradients of every map, accumulated head by
+    head at the masked feature gradients the GPU produced; and bit-reproducibility of a second call."""
+    s, op = r.s, r.op
+    gq, gk = op.backward_weights(r.dQ_, r.dK_)
+    gq2, gk2 = op.backward_weights(r.dQ_, r.dK_)
+    torch.cuda.synchronize()
+    assert op.device_status() == binding.HLA_OK
+    for a, b in zip(list(gq) + [t for g in gk for t in g], list(gq2) + [t for g in gk2 for t in g]):
+        assert torch.equal(a, b)
+    names = ("dW1", "db1", "dW2", "db2")
+    sides = [("phi_q", r.Q, r.pq, r.gq, r.gdq, gq)] + [(f"phi_k{f + 1}", r.K, r.pk[f], r.gk[:, :, f], r.gdk[:, :, f], gk[f]) for f in range(s.F)]
+    worst = {}
+    for label, X, w, feat, dfeat, got in sides:
+        acc = None
+        for b, h in r.heads():
+            dp = f64(dfeat[b, h]) * (feat[b, h] > 0)
+            g = orc.phi_mlp_backward_weights(f64(X[b, h]), *w, dp, relu=False)
+            acc = g if acc is None else tuple(a + c for a, c in zip(acc, g))
+        for name, t, ref in zip(names, got, acc):
+            worst[f"{label}_{name}"] = relerr(_host(t), ref)
+    report(f"{s.name} weight gradients, stage-wise", **worst)
+    assert max(worst.values()) < TOL["bf16"], worst
+
+
+def check_training_step(name, rng, whole_heads, weights=False):
     r = FullRun(name)
     s = r.s
     check_features_sampled(r, rng)
@@ -214,3 +239,5 @@ def check_training_step(name, rng, whole_heads):
         assert keep_q.mean() > 0.7 and keep_k.mean() > 0.5
         assert l2err(r.dQ[b, h][keep_q], eQ[keep_q]) < TOL["bf16"], (b, h)
         assert l2err(r.dK[b, h][keep_k], eK[keep_k]) < TOL["bf16"], (b, h)
+    if weights:
+        check_weight_gradients(r)
