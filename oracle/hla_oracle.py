@@ -38,6 +38,12 @@ takes):
   * In the theorem's proof the summed token index is the key/value index j.
   * The P = d_phi**F features of a token are flattened with the FIRST factor's
     index slowest (the listings' `bhsdef -> view(dp**3)`).
+  * Value modulation (Section 4.5; appendix "Defining phi"): the text fixes T + phi_v1(T) (.) phi_v2(V), two
+    Linear layers of width d with a GELU in between, no final activation, and says only that phi_v1, phi_v2 "use a
+    LayerNorm".  Reading taken here: the LayerNorm acts on the input of each map (over the d channels of a
+    token, biased variance, eps_ln = 1e-5, learnable scale and shift), i.e. phi_v(x) = W2^T GELU(W1^T LN(x) + b1) + b2.
+    Where the LayerNorm sits is PARITY UNPINNED by the paper; the functions are pinned against pure-Python loops,
+    closed forms and finite differences.
   * phi: exact (erf) GELU, both Linear layers have a bias, hidden width = d,
     ReLU applied at the end for phi_q and phi_k.  The figure defining phi is
     missing from the text, so the phi functions here are PARITY UNPINNED by the
@@ -361,3 +367,55 @@ def hla_backward_weights(Q, K, V, dO, phi_q, phi_k, eps, form="factored"):
     gq = phi_mlp_backward_weights(Q.reshape(-1, d), *phi_q, dqf.reshape(-1, dqf.shape[-1]))
     gk = [phi_mlp_backward_weights(K.reshape(-1, d), *w, dkf[:, :, f].reshape(-1, dkf.shape[-1])) for f, w in enumerate(phi_k)]
     return gq, gk
+
+
+# --------------------------------------------------------------------------- #
+# Value modulation (Section 4.5 "Value Modulation"; appendix "Defining phi")
+# --------------------------------------------------------------------------- #
+LN_EPS = 1e-5
+
+
+def layer_norm(x, gamma, beta, eps=LN_EPS):
+    """LayerNorm over the last axis: (x - mean) / sqrt(var + eps) * gamma + beta, biased variance."""
+    x = np.asarray(x, F64)
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps) * np.asarray(gamma, F64) + np.asarray(beta, F64)
+
+
+def phi_v_mlp(x, ln_g, ln_b, W1, b1, W2, b2):
+    """One value-modulation map: LayerNorm, Linear(d, d), GELU, Linear(d, d); no final activation.
+    x [N, d]; W1, W2 [d, d] (input index first)."""
+    xn = layer_norm(x, ln_g, ln_b)
+    return gelu_erf(xn @ np.asarray(W1, F64) + np.asarray(b1, F64)) @ np.asarray(W2, F64) + np.asarray(b2, F64)
+
+
+def phi_v_mlp_backward(x, ln_g, ln_b, W1, b1, W2, b2, dy):
+    """Gradient of sum(dy * phi_v_mlp(x)) with respect to x (weights held fixed)."""
+    x = np.asarray(x, F64)
+    W1 = np.asarray(W1, F64)
+    W2 = np.asarray(W2, F64)
+    g_ = np.asarray(ln_g, F64)
+    d = x.shape[-1]
+    mu = x.mean(axis=-1, keepdims=True)
+    rstd = 1.0 / np.sqrt(((x - mu) ** 2).mean(axis=-1, keepdims=True) + LN_EPS)
+    xhat = (x - mu) * rstd
+    h = (xhat * g_ + np.asarray(ln_b, F64)) @ W1 + np.asarray(b1, F64)
+    dh = (np.asarray(dy, F64) @ W2.T) * gelu_erf_grad(h)
+    dxhat = (dh @ W1.T) * g_
+    # LayerNorm: xhat depends on every channel of its token through the mean and the variance
+    return rstd * (dxhat - dxhat.mean(axis=-1, keepdims=True) - xhat * (dxhat * xhat).mean(axis=-1, keepdims=True))
+
+
+def value_modulation(T, V, v1, v2):
+    """T + phi_v1(T) (.) phi_v2(V) for one head: T (the attention result A V), V [N, d]; v1, v2 = (ln_g, ln_b, W1, b1, W2, b2)."""
+    return np.asarray(T, F64) + phi_v_mlp(T, *v1) * phi_v_mlp(V, *v2)
+
+
+def value_modulation_backward(T, V, dOut, v1, v2):
+    """Gradients of sum(dOut * value_modulation(T, V)) with respect to T and V."""
+    dOut = np.asarray(dOut, F64)
+    y1, y2 = phi_v_mlp(T, *v1), phi_v_mlp(V, *v2)
+    dT = dOut + phi_v_mlp_backward(T, *v1, dOut * y2)
+    dV = phi_v_mlp_backward(V, *v2, dOut * y1)
+    return dT, dV

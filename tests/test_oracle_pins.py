@@ -369,6 +369,71 @@ def test_whole_operator_wrappers_against_per_head_per_token_loops():
                 np.testing.assert_allclose(dkf[b, h, f], dks[f], rtol=1e-9, atol=1e-12)
 
 
+# ---- value modulation (Section 4.5) -------------------------------------------------------------
+def vm_weights(rng, d):
+    return (rng.standard_normal(d) * 0.3 + 1.0, rng.standard_normal(d) * 0.2, rng.standard_normal((d, d)) / np.sqrt(d), rng.standard_normal(d) * 0.1,
+            rng.standard_normal((d, d)) / np.sqrt(d), rng.standard_normal(d) * 0.1)
+
+
+def test_layer_norm_closed_forms_and_python_loops():
+    rng = np.random.default_rng(31)
+    x = rng.standard_normal((5, 7)) * 3.0 + 2.0
+    y = orc.layer_norm(x, np.ones(7), np.zeros(7), eps=0.0)
+    np.testing.assert_allclose(y.mean(axis=1), 0.0, atol=1e-14)
+    np.testing.assert_allclose((y ** 2).mean(axis=1), 1.0, rtol=1e-13)           # biased variance: exactly one
+    np.testing.assert_allclose(orc.layer_norm(4.0 * x + 9.0, np.ones(7), np.zeros(7), eps=0.0), y, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(orc.layer_norm(np.array([[1.0, 3.0]]), [1.0, 1.0], [0.0, 0.0], eps=0.0), [[-1.0, 1.0]], rtol=1e-15)
+    g, b = rng.standard_normal(7), rng.standard_normal(7)
+    got = orc.layer_norm(x, g, b)
+    for t in range(5):
+        mu = sum(x[t]) / 7
+        var = sum((a - mu) ** 2 for a in x[t]) / 7
+        want = [(x[t, i] - mu) / math.sqrt(var + 1e-5) * g[i] + b[i] for i in range(7)]
+        np.testing.assert_allclose(got[t], want, rtol=1e-13, atol=1e-15)
+
+
+def test_phi_v_mlp_against_python_loops():
+    rng = np.random.default_rng(32)
+    n, d = 3, 5
+    x = rng.standard_normal((n, d))
+    ln_g, ln_b, W1, b1, W2, b2 = vm_weights(rng, d)
+    got = orc.phi_v_mlp(x, ln_g, ln_b, W1, b1, W2, b2)
+    assert got.shape == (n, d) and np.any(got < 0)                 # no ReLU at the end
+    for t in range(n):
+        mu = sum(x[t]) / d
+        var = sum((a - mu) ** 2 for a in x[t]) / d
+        xn = [(x[t, i] - mu) / math.sqrt(var + 1e-5) * ln_g[i] + ln_b[i] for i in range(d)]
+        h = [sum(xn[i] * W1[i, j] for i in range(d)) + b1[j] for j in range(d)]
+        g = [0.5 * a * (1.0 + math.erf(a / math.sqrt(2.0))) for a in h]
+        y = [sum(g[j] * W2[j, o] for j in range(d)) + b2[o] for o in range(d)]
+        np.testing.assert_allclose(got[t], y, rtol=1e-12, atol=1e-14)
+
+
+def test_value_modulation_special_cases_and_gradients():
+    rng = np.random.default_rng(33)
+    n, d = 6, 4
+    T, V, dOut = rng.standard_normal((n, d)), rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    v1, v2 = vm_weights(rng, d), vm_weights(rng, d)
+    out = orc.value_modulation(T, V, v1, v2)
+    np.testing.assert_allclose(out, T + orc.phi_v_mlp(T, *v1) * orc.phi_v_mlp(V, *v2), rtol=1e-14)
+    # phi_v2 == 1 (zero second layer, unit bias): the update is phi_v1(T) itself; phi_v2 == 0: the identity
+    one = v2[:4] + (np.zeros((d, d)), np.ones(d))
+    zero = v2[:4] + (np.zeros((d, d)), np.zeros(d))
+    np.testing.assert_allclose(orc.value_modulation(T, V, v1, one), T + orc.phi_v_mlp(T, *v1), rtol=1e-14)
+    np.testing.assert_allclose(orc.value_modulation(T, V, v1, zero), T, rtol=0, atol=0)
+    # the LayerNorm makes each map blind to a shift and (up to eps) a positive rescaling of its input token
+    np.testing.assert_allclose(orc.phi_v_mlp(3.0 * V + 5.0, *v2), orc.phi_v_mlp(V, *v2), rtol=1e-4, atol=1e-6)
+    dT, dV = orc.value_modulation_backward(T, V, dOut, v1, v2)
+    loss = lambda T_=T, V_=V: float(np.sum(dOut * orc.value_modulation(T_, V_, v1, v2)))
+    np.testing.assert_allclose(dT, fd_grad(lambda x: loss(T_=x), T, 1e-6), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(dV, fd_grad(lambda x: loss(V_=x), V, 1e-6), rtol=2e-6, atol=1e-8)
+    dx = orc.phi_v_mlp_backward(V, *v2, dOut)
+    np.testing.assert_allclose(dx, fd_grad(lambda x: float(np.sum(dOut * orc.phi_v_mlp(x, *v2))), V, 1e-6), rtol=2e-6, atol=1e-8)
+    # a gradient through a LayerNorm has no component along the all-ones direction and (eps -> 0) none along the input's
+    # own centred direction: shifting or rescaling the token does not change the output
+    np.testing.assert_allclose(dx.sum(axis=1), 0.0, atol=1e-12)
+
+
 # ---- FLOP model against the paper's tables ---------------------------------------------------
 def load_golden():
     path = os.path.join(os.path.dirname(__file__), "golden", "paper_flop_tables.txt")
