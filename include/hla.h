@@ -78,6 +78,8 @@ typedef struct {
     float eps;        /* added to the normaliser, o = num / (eta + eps); <= 0 -> 1e-6          */
     int32_t n_splits; /* token splits of the state build per head; 0 -> chosen from the SM count */
     int32_t causal;   /* must be 0: the causal / decayed variant (Section 4.4) is not built    */
+    int32_t value_mod; /* 1: the workspace also holds the scratch of hla_value_mod_forward / _backward (bf16 with
+                          d in {64,128} only; HLA_ERR_UNSUPPORTED otherwise); 0: those calls are refused            */
 } hla_config;
 
 /*
@@ -91,6 +93,17 @@ typedef struct {
 typedef struct {
     const void *W1, *b1, *W2, *b2;
 } hla_mlp;
+
+/*
+ * One value-modulation network (Section 4.5 "Value Modulation"; appendix "Defining phi"):
+ *     phi_v(x) = W2^T GELU(W1^T LN(x) + b1) + b2,   LN(x) = (x - mean) / sqrt(var + 1e-5) * ln_g + ln_b  over the d channels
+ * (two Linear layers of width d, no final activation; the paper only says that these maps use a LayerNorm - it is read
+ * as acting on the input of the map).  Device pointers in the ctx dtype: ln_g [d], ln_b [d], W1 [d][d] (input index
+ * first), b1 [d], W2 [d][d], b2 [d]; W1 and W2 16-byte aligned.
+ */
+typedef struct {
+    const void *ln_g, *ln_b, *W1, *b1, *W2, *b2;
+} hla_vmlp;
 
 /*
  * Where hla_backward_weights puts the gradients of one feature network: fp32 device buffers with the shapes of the
@@ -165,6 +178,26 @@ hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *
  */
 hla_status hla_backward_weights(hla_ctx *ctx, const void *Q, const void *K, const hla_mlp_grad *dphi_q, const hla_mlp_grad *dphi_k,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Value modulation of the attention result (Section 4.5):  Out = T + phi_v1(T) (.) phi_v2(V), with T the output of
+ * hla_forward and V its value input, both [B,H,N,d]; one weight set per map, shared by all batches and heads.
+ * Contexts created with value_mod = 1 only.  hla_set_phi_v remembers the weight pointers (they must stay valid).
+ * The forward keeps nothing for the backward; the backward recomputes both maps and returns
+ *     dT = dOut + J1^T (dOut (.) phi_v2(V)),     dV = J2^T (dOut (.) phi_v1(T))      (J: Jacobian of a map w.r.t. its input)
+ * the gradients of sum(dOut * Out) with respect to T and V (weights fixed).  With accumulate_dV != 0 the V-side
+ * gradient is added to what dV already holds (the dV that hla_backward wrote for the same step), else dV is overwritten.
+ * Out, dT, dV must be 32-byte aligned.  Out may not alias T or V.  hla_value_mod_forward clears the device status words
+ * like hla_forward does (read hla_last_device_status before it if the record of hla_forward matters); the backward
+ * keeps them.  A whole step is then
+ *     hla_forward -> hla_value_mod_forward;   hla_value_mod_backward -> hla_backward(dO = dT) with accumulate_dV = 0 and
+ *     the two dV added by the caller, or hla_backward first and hla_value_mod_backward with accumulate_dV = 1.
+ */
+hla_status hla_set_phi_v(hla_ctx *ctx, const hla_vmlp *v1, const hla_vmlp *v2);
+hla_status hla_value_mod_forward(hla_ctx *ctx, const void *T, const void *V, void *Out, void *workspace, size_t workspace_bytes,
+                                 void *cuda_stream);
+hla_status hla_value_mod_backward(hla_ctx *ctx, const void *T, const void *V, const void *dOut, void *dT, void *dV,
+                                  int32_t accumulate_dV, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Forward without a caller-provided workspace (no counterpart in the paper: a

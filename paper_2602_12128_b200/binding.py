@@ -17,7 +17,7 @@ HLA_BF16, HLA_F32 = 0, 1
 HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
-    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_backward_weights", "hla_forward_static",
+    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_backward_weights", "hla_set_phi_v", "hla_value_mod_forward", "hla_value_mod_backward", "hla_forward_static",
     "hla_last_device_status", "hla_selftest_bounded_wait", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
     "hla_destroy", "hla_status_string",
 ]
@@ -25,11 +25,15 @@ EXPORTS = [
 
 class HlaConfig(ctypes.Structure):
     _fields_ = [("B", c_int32), ("H", c_int32), ("N", c_int32), ("d", c_int32), ("F", c_int32), ("d_phi", c_int32),
-                ("phi", c_int32), ("dtype", c_int32), ("eps", c_float), ("n_splits", c_int32), ("causal", c_int32)]
+                ("phi", c_int32), ("dtype", c_int32), ("eps", c_float), ("n_splits", c_int32), ("causal", c_int32), ("value_mod", c_int32)]
 
 
 class HlaMlp(ctypes.Structure):
     _fields_ = [("W1", c_void_p), ("b1", c_void_p), ("W2", c_void_p), ("b2", c_void_p)]
+
+
+class HlaVmlp(ctypes.Structure):
+    _fields_ = [("ln_g", c_void_p), ("ln_b", c_void_p), ("W1", c_void_p), ("b1", c_void_p), ("W2", c_void_p), ("b2", c_void_p)]
 
 
 class HlaMlpGrad(ctypes.Structure):
@@ -78,6 +82,12 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_backward.restype = c_int32
     lib.hla_backward_weights.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(HlaMlpGrad), POINTER(HlaMlpGrad), c_void_p, c_size_t, c_void_p]
     lib.hla_backward_weights.restype = c_int32
+    lib.hla_set_phi_v.argtypes = [c_void_p, POINTER(HlaVmlp), POINTER(HlaVmlp)]
+    lib.hla_set_phi_v.restype = c_int32
+    lib.hla_value_mod_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.hla_value_mod_forward.restype = c_int32
+    lib.hla_value_mod_backward.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_size_t, c_void_p]
+    lib.hla_value_mod_backward.restype = c_int32
     lib.hla_forward_static.argtypes = [c_void_p] + [c_void_p] * 4 + [c_void_p, POINTER(c_void_p)]
     lib.hla_forward_static.restype = c_int32
     lib.hla_last_device_status.argtypes = [c_void_p, c_void_p, c_void_p]
@@ -175,6 +185,27 @@ def hla_backward_weights(ctx: int, Q, K, dphi_q, dphi_k, workspace, stream=None,
         raise HlaError(st, "hla_backward_weights")
 
 
+def hla_set_phi_v(ctx: int, v1, v2) -> None:
+    """v1, v2 = (ln_g, ln_b, W1, b1, W2, b2) device tensors of the two value-modulation maps."""
+    a, b = HlaVmlp(*[_ptr(t) for t in v1]), HlaVmlp(*[_ptr(t) for t in v2])
+    st = load_library().hla_set_phi_v(ctx, byref(a), byref(b))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_set_phi_v")
+
+
+def hla_value_mod_forward(ctx: int, T, V, Out, workspace, stream=None) -> None:
+    st = load_library().hla_value_mod_forward(ctx, _ptr(T), _ptr(V), _ptr(Out), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_value_mod_forward")
+
+
+def hla_value_mod_backward(ctx: int, T, V, dOut, dT, dV, accumulate_dV, workspace, stream=None) -> None:
+    st = load_library().hla_value_mod_backward(ctx, _ptr(T), _ptr(V), _ptr(dOut), _ptr(dT), _ptr(dV), 1 if accumulate_dV else 0, _ptr(workspace),
+                                               workspace.numel() * workspace.element_size(), _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_value_mod_backward")
+
+
 HLA_STATIC_WS_BYTES = 16 * 1024 * 1024
 
 
@@ -235,9 +266,9 @@ def hla_destroy(ctx: int) -> None:
 class Hla:
     """Owns a context and its workspace tensor.  All compute happens in hla_forward / hla_backward."""
 
-    def __init__(self, B, H, N, d, dtype="bf16", phi="mlp", F=0, d_phi=0, eps=0.0, n_splits=0, device="cuda"):
+    def __init__(self, B, H, N, d, dtype="bf16", phi="mlp", F=0, d_phi=0, eps=0.0, n_splits=0, device="cuda", value_mod=False):
         self.cfg = HlaConfig(B, H, N, d, F, d_phi, HLA_PHI_MLP if phi == "mlp" else HLA_PHI_NONE,
-                             HLA_BF16 if dtype == "bf16" else HLA_F32, eps, n_splits, 0)
+                             HLA_BF16 if dtype == "bf16" else HLA_F32, eps, n_splits, 0, 1 if value_mod else 0)
         self.torch_dtype = torch.bfloat16 if dtype == "bf16" else torch.float32
         self.ctx = hla_create(self.cfg)
         self.layout = hla_workspace_layout(self.ctx)
@@ -261,6 +292,21 @@ class Hla:
         dV = torch.empty_like(V) if dV is None else dV
         hla_backward(self.ctx, Q, K, V, O, dO, dQ, dK, dV, self.workspace, stream)
         return dQ, dK, dV
+
+    def set_phi_v(self, v1, v2):
+        self._vweights = (v1, v2)           # keep the tensors alive: the library only borrows pointers
+        hla_set_phi_v(self.ctx, v1, v2)
+
+    def value_mod_forward(self, T, V, Out=None, stream=None):
+        Out = torch.empty_like(T) if Out is None else Out
+        hla_value_mod_forward(self.ctx, T, V, Out, self.workspace, stream)
+        return Out
+
+    def value_mod_backward(self, T, V, dOut, dT=None, dV=None, accumulate_dV=False, stream=None):
+        dT = torch.empty_like(T) if dT is None else dT
+        dV = torch.empty_like(V) if dV is None else dV
+        hla_value_mod_backward(self.ctx, T, V, dOut, dT, dV, accumulate_dV, self.workspace, stream)
+        return dT, dV
 
     def backward_weights(self, Q, K, stream=None):
         """Weight gradients of phi_q and phi_k1..F (fp32, shapes of the weights), after backward()."""

@@ -13,6 +13,7 @@
 #include "hla_tc_fused.cuh"
 #include "hla_tc_fused_k.cuh"
 #include "hla_tc_wgrad.cuh"
+#include "hla_tc_vmod.cuh"
 
 using namespace hla;
 
@@ -27,6 +28,9 @@ struct hla_ctx {
     hla_ws_layout L;
     size_t off_part;    // split partials (scratch)
     int k_pieces;       // most pieces a head has in the fused key-side kernel of the forward
+    bool vmod, phi_v_set;   // value modulation enabled at creation; its weights given
+    hla_vmlp phi_v[2];
+    tc::VmodPlan vmp;   // scratch of the value modulation inside the workspace
     size_t off_wpart;   // per-CTA partials of the weight gradients (scratch; tensor-core path with the phi maps)
     tc::Plan tcp;       // tensor-core operand buffers inside the workspace
     size_t ws_bytes;
@@ -230,6 +234,8 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     }
     if (!(c.eps > 0.f)) c.eps = 1e-6f;
     if (c.causal != 0) return HLA_ERR_UNSUPPORTED;
+    if (c.value_mod != 0 && c.value_mod != 1) return HLA_ERR_INVALID_ARG;
+    if (c.value_mod && !(c.dtype == HLA_BF16 && (c.d == 64 || c.d == 128) && (long long)c.B * c.H * c.N < (1ll << 31))) return HLA_ERR_UNSUPPORTED;
     if (c.F > kMaxF) return HLA_ERR_UNSUPPORTED;
     const int P = ipow(c.d_phi, c.F);
     if (P > kMaxP) return HLA_ERR_UNSUPPORTED;
@@ -305,6 +311,9 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     x->off_part = cv.take(part_bytes);
     x->off_wpart = (x->tc && mlp) ? cv.take(tc::wgrad_part_bytes(c.d, (long long)x->BH * c.N, x->sm_count)) : kNone;
     if (x->tc) cv.off = tc::plan(x->tcp, D, x->BH, cv.off);
+    x->vmod = c.value_mod != 0;
+    x->phi_v_set = false;
+    if (x->vmod) cv.off = tc::vmod_plan(x->vmp, c.d, (long long)x->BH * c.N, cv.off);
     x->ws_bytes = cv.off;
     *out = x;
     return HLA_OK;
@@ -420,6 +429,61 @@ hla_status hla_backward_weights(hla_ctx* ctx, const void* Q, const void* K, cons
     tc::HostCacheScope scope(&ctx->hc);
     return tc::phi_wgrad(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, dphi_q, dphi_k, static_cast<char*>(workspace), ctx->L, ctx->off_wpart,
                          ctx->sm_count, ctx->rec);
+}
+
+hla_status hla_set_phi_v(hla_ctx* ctx, const hla_vmlp* v1, const hla_vmlp* v2) {
+    if (!ctx || !v1 || !v2) return HLA_ERR_INVALID_ARG;
+    if (!ctx->vmod) return HLA_ERR_INVALID_ARG;
+    const hla_vmlp* all[2] = {v1, v2};
+    for (int i = 0; i < 2; ++i) {
+        const void* p[6] = {all[i]->ln_g, all[i]->ln_b, all[i]->W1, all[i]->b1, all[i]->W2, all[i]->b2};
+        for (int j = 0; j < 6; ++j)
+            if (!p[j]) return HLA_ERR_INVALID_ARG;
+        if (!aligned16(all[i]->W1) || !aligned16(all[i]->W2)) return HLA_ERR_INVALID_ARG;
+    }
+    ctx->phi_v[0] = *v1;
+    ctx->phi_v[1] = *v2;
+    ctx->phi_v_set = true;
+    return HLA_OK;
+}
+
+namespace {
+hla_status value_mod_call(hla_ctx* ctx, const void* T, const void* V, const void* dOut, void* Out, void* dT, void* dV, int accumulate, bool backward,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return HLA_ERR_INVALID_ARG;
+    if (!ctx->vmod || !ctx->phi_v_set) return HLA_ERR_INVALID_ARG;
+    const void* in[3] = {T, V, backward ? dOut : T};
+    for (int i = 0; i < 3; ++i)
+        if (!in[i] || !aligned16(in[i])) return HLA_ERR_INVALID_ARG;
+    const void* out[2] = {backward ? dT : Out, backward ? dV : Out};
+    for (int i = 0; i < 2; ++i)
+        if (!out[i] || (reinterpret_cast<uintptr_t>(out[i]) & 31u)) return HLA_ERR_INVALID_ARG;
+    if (!backward && (Out == T || Out == V)) return HLA_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HLA_ERR_INVALID_ARG;
+    if (workspace_bytes < ctx->ws_bytes) return HLA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    ctx->rec.start_call(st);
+    (void)cudaGetLastError();
+    follow_device(ctx);
+    tc::HostCacheScope scope(&ctx->hc);
+    const long long rows = (long long)ctx->BH * ctx->D.N;
+    int* status = reinterpret_cast<int*>(ws + ctx->L.status);
+    // like hla_forward, the forward starts a new record of device-side time-outs
+    if (!backward && cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
+    if (ctx->D.d == 128)
+        return tc::launch_vmod<128>(ctx->vmp, rows, ctx->phi_v, T, V, dOut, Out, dT, dV, accumulate, backward, ws, status, ctx->sm_count, ctx->rec);
+    return tc::launch_vmod<64>(ctx->vmp, rows, ctx->phi_v, T, V, dOut, Out, dT, dV, accumulate, backward, ws, status, ctx->sm_count, ctx->rec);
+}
+}  // namespace
+
+hla_status hla_value_mod_forward(hla_ctx* ctx, const void* T, const void* V, void* Out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return value_mod_call(ctx, T, V, nullptr, Out, nullptr, nullptr, 0, false, workspace, workspace_bytes, cuda_stream);
+}
+
+hla_status hla_value_mod_backward(hla_ctx* ctx, const void* T, const void* V, const void* dOut, void* dT, void* dV, int32_t accumulate_dV, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+    return value_mod_call(ctx, T, V, dOut, nullptr, dT, dV, accumulate_dV != 0, true, workspace, workspace_bytes, cuda_stream);
 }
 
 // ---- forward on the library's own scratch array ---------------------------------------------

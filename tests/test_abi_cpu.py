@@ -28,7 +28,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def cfg(**kw):
-    base = dict(B=1, H=2, N=300, d=128, F=0, d_phi=0, phi=binding.HLA_PHI_MLP, dtype=binding.HLA_BF16, eps=0.0, n_splits=0, causal=0)
+    base = dict(B=1, H=2, N=300, d=128, F=0, d_phi=0, phi=binding.HLA_PHI_MLP, dtype=binding.HLA_BF16, eps=0.0, n_splits=0, causal=0, value_mod=0)
     base.update(kw)
     return binding.HlaConfig(*[base[k] for k, _ in binding.HlaConfig._fields_])
 
@@ -75,6 +75,8 @@ def test_feature_level_entry_has_no_feature_regions():
     (dict(d=256), binding.HLA_ERR_UNSUPPORTED),
     (dict(d=20), binding.HLA_ERR_UNSUPPORTED),           # bf16 rows must be 16-byte multiples
     (dict(B=300, H=300), binding.HLA_ERR_UNSUPPORTED),
+    (dict(value_mod=2), binding.HLA_ERR_INVALID_ARG),
+    (dict(value_mod=1, dtype=binding.HLA_F32, d=16), binding.HLA_ERR_UNSUPPORTED),      # value modulation: bf16, d in {64, 128}
 ])
 def test_create_rejects(kw, want):
     st, ctx = create(**kw)
@@ -110,5 +112,21 @@ def test_calls_validate_before_launching():
     binding.hla_destroy(ctx)
     assert lib.hla_destroy(None) == binding.HLA_ERR_INVALID_ARG
     assert binding.status_string(binding.HLA_ERR_NO_MEMORY) == "out of host memory"
+    # value modulation: refused unless the context was created for it and its weights were given
+    st, ctx = create()
+    need = binding.hla_workspace_bytes(ctx)
+    assert lib.hla_value_mod_forward(ctx, p, p, p + 256, p, need, None) == binding.HLA_ERR_INVALID_ARG
+    binding.hla_destroy(ctx)
+    st, ctx = create(value_mod=1)
+    assert st == binding.HLA_OK and binding.hla_workspace_bytes(ctx) > need
+    need = binding.hla_workspace_bytes(ctx)
+    assert lib.hla_value_mod_forward(ctx, p, p, p + 256, p, need, None) == binding.HLA_ERR_INVALID_ARG      # weights not set
+    v = binding.HlaVmlp(p, p, p, p, p, p)
+    assert lib.hla_set_phi_v(ctx, ctypes.byref(v), ctypes.byref(v)) == binding.HLA_OK
+    assert lib.hla_value_mod_forward(ctx, p, p, p, p, need, None) == binding.HLA_ERR_INVALID_ARG            # Out aliases T
+    assert lib.hla_value_mod_forward(ctx, p, p, p + 16, p, need, None) == binding.HLA_ERR_INVALID_ARG       # Out not 32-byte aligned
+    assert lib.hla_value_mod_forward(ctx, p, p, p + 256, p, need - 1, None) == binding.HLA_ERR_WORKSPACE
+    assert lib.hla_value_mod_backward(ctx, p, p, p, p + 16, p, 0, p, need, None) == binding.HLA_ERR_INVALID_ARG
+    binding.hla_destroy(ctx)
     assert binding.status_string(binding.HLA_ERR_DEVICE_TIMEOUT) == "device-side wait timed out"
     assert binding.hla_workspace_bytes(None) == 0
