@@ -294,6 +294,61 @@ class Workload:
         return kt
 
 
+def value_mod_leg(shape, w, dev):
+    """hla_value_mod_forward (+ backward for workloads with a backward) on the workload's O and V, sustained like the rest."""
+    import torch
+    from paper_2602_12128_b200 import binding
+    tdt = torch.bfloat16
+    rng = np.random.default_rng(9)
+    d = shape.d
+
+    def vmlp():
+        r = lambda *s: torch.from_numpy(rng.standard_normal(s).astype(np.float32))
+        ws = (1.0 + 0.2 * r(d), 0.1 * r(d), r(d, d) / np.sqrt(d), 0.1 * r(d), r(d, d) / np.sqrt(d), 0.1 * r(d))
+        return tuple(x.to(tdt).to(dev) for x in ws)
+
+    op = binding.Hla(shape.B, shape.H, shape.N, d, dtype="bf16", phi="none", eps=1e-6, device=dev, value_mod=True)
+    op.set_phi_v(vmlp(), vmlp())
+    out = torch.empty_like(w.O)
+    dT, dV = (torch.empty_like(w.O), torch.empty_like(w.O)) if shape.backward else (None, None)
+
+    def step():
+        binding.hla_value_mod_forward(op.ctx, w.O, w.V, out, op.workspace)
+        n = op.launches()
+        if shape.backward:
+            binding.hla_value_mod_backward(op.ctx, w.O, w.V, w.dO, dT, dV, False, op.workspace)
+            n += op.launches()
+        return n
+
+    for _ in range(3):
+        launches = step()
+    torch.cuda.synchronize()
+    if op.device_status() != binding.HLA_OK:
+        raise SystemExit("device-side wait timed out (value modulation)")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    est = e0.elapsed_time(e1) / 5
+    n = int(min(max(math.ceil(500.0 / est), 10), 20000))
+    for _ in range(n):
+        step()
+    e0.record()
+    for _ in range(n):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    th = shape.B * shape.H * shape.N
+    fl = th * F_.value_mod_flops_per_token(d, shape.backward)
+    by = th * d * 2 * (3 + (4 if shape.backward else 0))      # T, V in, Out out (+ dOut in, dT, dV out, and T, V again)
+    return {"ms_per_step": ms, "steps": n, "tflops": fl / (ms * 1e-3) / 1e12, "gpu_launches_per_step": launches, "flops": fl, "bytes": by,
+            "pass": "fwd+bwd" if shape.backward else "fwd",
+            "note": "hla_value_mod_forward (+ _backward): FLOPs = the 4 (+ 4) d x d products per token; the backward's recomputed forward is not counted"}
+
+
 def extra_leg(name, rank, dev, peaks, local):
     """One of the other configurations, timed by the same code: >= 1 s of untimed sustained steps, then >= 0.5 s timed."""
     import torch
@@ -532,6 +587,11 @@ def main():
                  "products per map (the recomputed hidden layer is not counted)"}
         del gq, gk
 
+    # ---- value modulation of the attention result (Section 4.5; separate calls, not part of `value`) --------------------
+    vmod = None
+    if not args.profile and world == 1 and shape.dtype == "bf16" and shape.d in (64, 128):
+        vmod = value_mod_leg(shape, w, dev)
+
     tensor_mb = w.Q.numel() * w.Q.element_size() / 1e6
     launches_per_step = w.launches
     # ---- the other configurations, timed by the same code (single-GPU runs only) ----------------------------------------
@@ -554,7 +614,7 @@ def main():
             "tokens_per_s": multi.whole_job_rate(shape.B * shape.N, world, ms_step),
             "step_roofline": roofline_of(shape, ms_step, world, peaks),
             "roofline": roof, "kernels": per_kernel, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "clocks": clocks, "weight_gradients": wgrad, "extra": extra}
+            "clocks": clocks, "weight_gradients": wgrad, "value_modulation": vmod, "extra": extra}
     if clocks.get("sm_mhz"):
         line["ms_x_mhz"] = ms_step * clocks["sm_mhz"]
     print(json.dumps(line), flush=True)

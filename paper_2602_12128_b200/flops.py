@@ -92,3 +92,10 @@ def folded_flops_per_token(d: int, F: int, d_phi: int, backward: bool, with_phi:
     if with_phi:
         phi = phi_fwd_flops_per_token(d, F, d_phi) + (phi_bwd_flops_per_token(d, F, d_phi) if backward else 0)
     return core + phi
+
+
+def value_mod_flops_per_token(d: int, backward: bool) -> int:
+    """Value modulation T + phi_v1(T) (.) phi_v2(V): two maps of two d x d Linear layers each (Table 3 counts them in
+    the layer total).  The backward adds the two transposed products per map; the recomputed forward is not counted."""
+    fwd = 2 * (2 * d * d + 2 * d * d)
+    return fwd + (2 * (2 * d * d + 2 * d * d) if backward else 0)

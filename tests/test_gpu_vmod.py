@@ -121,3 +121,40 @@ def test_value_modulation_after_the_operator():
             rT, dV_mod[b, h] = orc.value_modulation_backward(Og[b, h], f64(V[b, h]), f64(dOut[b, h]), v1, v2)
             assert relerr(dTg[b, h], rT) < TOL["bf16"]
     assert relerr(to_np(dV), dV_core + dV_mod) < TOL["bf16"]
+
+
+@pytest.mark.parametrize("name", ["dit_bf16", "train_bf16"])
+def test_value_modulation_at_the_benchmark_shapes(name):
+    """Full-size shapes (video-DiT forward, training step): forward and input gradients on sampled token rows of every
+    head against the oracle (every token is independent of the others in this stage), plus finiteness of everything."""
+    c = synth.CONFIGS[name]
+    rng = np.random.default_rng(17)
+    dims = (c.B, c.H, c.N, c.d)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(5)
+    Td = (torch.randn(dims, generator=g, device="cuda") * 0.7 + 0.2).to(torch.bfloat16)
+    Vd = torch.randn(dims, generator=g, device="cuda").to(torch.bfloat16)
+    dOd = torch.randn(dims, generator=g, device="cuda").to(torch.bfloat16)
+    v1, v2 = make_vmlp(c.d, 7), make_vmlp(c.d, 8)
+    op = binding.Hla(c.B, c.H, c.N, c.d, dtype="bf16", phi="none", eps=1e-6, value_mod=True)
+    op.set_phi_v(tuple(to_dev(a, "bf16") for a in v1), tuple(to_dev(a, "bf16") for a in v2))
+    out = op.value_mod_forward(Td, Vd)
+    dT, dV = op.value_mod_backward(Td, Vd, dOd)
+    torch.cuda.synchronize()
+    assert op.device_status() == binding.HLA_OK
+    for t in (out, dT, dV):
+        assert bool(torch.isfinite(t).all())
+    worst = {"out": 0.0, "dT": 0.0, "dV": 0.0}
+    for b in range(c.B):
+        for h in range(c.H):
+            rows = np.sort(rng.choice(c.N, 64, replace=False))
+            rows[-1] = c.N - 1                                   # the ragged tail of the head
+            idx = torch.from_numpy(rows).cuda()
+            Ts, Vs, dOs = (to_np(x[b, h].index_select(0, idx)) for x in (Td, Vd, dOd))
+            ref = orc.value_modulation(Ts, Vs, v1, v2)
+            rT, rV = orc.value_modulation_backward(Ts, Vs, dOs, v1, v2)
+            worst["out"] = max(worst["out"], relerr(to_np(out[b, h].index_select(0, idx)), ref))
+            worst["dT"] = max(worst["dT"], relerr(to_np(dT[b, h].index_select(0, idx)), rT))
+            worst["dV"] = max(worst["dV"], relerr(to_np(dV[b, h].index_select(0, idx)), rV))
+    report(f"value modulation at {name}", **worst)
+    assert max(worst.values()) < TOL["bf16"], worst
