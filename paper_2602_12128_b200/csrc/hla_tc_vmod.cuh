@@ -26,18 +26,30 @@ constexpr float kLnEps = 1e-5f;
 struct VmlpPtrs {
     const __nv_bfloat16 *ln_g, *ln_b, *W1, *b1, *W2, *b2;
 };
-__global__ void vmod_fold_kernel(VmlpPtrs a, VmlpPtrs b, __nv_bfloat16* __restrict__ w1f, __nv_bfloat16* __restrict__ aux, int d) {
+// grid = (2 maps, d / 32 column groups), block = 32 columns x 8 row groups
+__global__ void __launch_bounds__(256) vmod_fold_kernel(VmlpPtrs a, VmlpPtrs b, __nv_bfloat16* __restrict__ w1f, __nv_bfloat16* __restrict__ aux, int d) {
+    __shared__ float sc[8][32], ss[8][32];
     const VmlpPtrs p = blockIdx.x == 0 ? a : b;
     __nv_bfloat16* wf = w1f + (size_t)blockIdx.x * d * d;
     __nv_bfloat16* ax = aux + (size_t)blockIdx.x * 16 * d;
-    for (int j = threadIdx.x; j < d; j += blockDim.x) {
-        float c = 0.f, s = 0.f;
-        for (int i = 0; i < d; ++i) {
-            const float w = __bfloat162float(p.W1[(size_t)i * d + j]);
-            const __nv_bfloat16 f = __float2bfloat16_rn(__bfloat162float(p.ln_g[i]) * w);
-            wf[(size_t)i * d + j] = f;
-            c += __bfloat162float(f);
-            s = fmaf(__bfloat162float(p.ln_b[i]), w, s);
+    const int jx = threadIdx.x & 31, iy = threadIdx.x >> 5, j = blockIdx.y * 32 + jx;
+    float c = 0.f, s = 0.f;
+    for (int i = iy; i < d; i += 8) {      // fixed order per thread, then a fixed-order sum over the 8 row groups
+        const float w = __bfloat162float(p.W1[(size_t)i * d + j]);
+        const __nv_bfloat16 f = __float2bfloat16_rn(__bfloat162float(p.ln_g[i]) * w);
+        wf[(size_t)i * d + j] = f;
+        c += __bfloat162float(f);
+        s = fmaf(__bfloat162float(p.ln_b[i]), w, s);
+    }
+    sc[iy][jx] = c;
+    ss[iy][jx] = s;
+    __syncthreads();
+    if (iy == 0) {
+        c = 0.f;
+        s = 0.f;
+        for (int k = 0; k < 8; ++k) {
+            c += sc[k][jx];
+            s += ss[k][jx];
         }
         const float b1f = __bfloat162float(p.b1[j]) + s;
         const __nv_bfloat16 chi = __float2bfloat16_rn(c), clo = __float2bfloat16_rn(c - __bfloat162float(chi));
@@ -54,7 +66,7 @@ __global__ void vmod_fold_kernel(VmlpPtrs a, VmlpPtrs b, __nv_bfloat16* __restri
 template <int DV>
 __device__ __forceinline__ void tile_row_stats(uint32_t tile, int row, float& mu, float& rstd) {
     float s = 0.f;
-#pragma unroll
+#pragma unroll 4
     for (int c = 0; c < DV / 8; ++c) {
         uint32_t w[4];
         asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(tile + (c >> 3) * kBlk + sw128_off(row, c & 7)) : "memory");
@@ -63,7 +75,7 @@ __device__ __forceinline__ void tile_row_stats(uint32_t tile, int row, float& mu
     }
     mu = s * (1.f / DV);
     float v = 0.f;
-#pragma unroll
+#pragma unroll 4
     for (int c = 0; c < DV / 8; ++c) {
         uint32_t w[4];
         asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(tile + (c >> 3) * kBlk + sw128_off(row, c & 7)) : "memory");
@@ -83,20 +95,37 @@ __device__ __forceinline__ void store_aug_row(uint32_t taddr, float mu, float rs
     tmem_st8(taddr, pack_bf16(mh, mh), pack_bf16(ml, sh), pack_bf16(sh, sl), 0u, 0u, 0u, 0u, 0u);
 }
 
+// 16 bf16 of one tile row (two 16-byte chunks 2 c, 2 c + 1 of a two-block swizzled tile) <-> 8 packed words
+__device__ __forceinline__ void lds_row16(uint32_t tile, int row, int c, uint32_t (&w)[8]) {
+    const uint32_t a = tile + (c >> 2) * kBlk + sw128_off(row, (2 * c) & 7), b = tile + (c >> 2) * kBlk + sw128_off(row, (2 * c + 1) & 7);
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(a) : "memory");
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(b) : "memory");
+}
+__device__ __forceinline__ void sts_row16(uint32_t tile, int row, int c, const uint32_t (&w)[8]) {
+    st_shared_v4(tile + (c >> 2) * kBlk + sw128_off(row, (2 * c) & 7), w[0], w[1], w[2], w[3]);
+    st_shared_v4(tile + (c >> 2) * kBlk + sw128_off(row, (2 * c + 1) & 7), w[4], w[5], w[6], w[7]);
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
 // ---- forward of one map --------------------------------------------------------------------------------------------
 // warp 0: TMA, warp 1: second-layer MMAs, warp 2: first-layer MMAs, warps 3..18: GELU (thread = token row x quarter of the
-// hidden units), warps 19..22: row statistics, warps 23..26: output (thread = token row)
+// hidden units), warps 19..22: row statistics, warps 23..26: output (thread = token row).  Every byte of global memory
+// moves through TMA: the output warps read the residual and the other map's output from a tile in shared memory, write
+// the result over it and store the tile.
 constexpr int kVfThreads = 27 * 32;
 constexpr int kVfGeluWarp0 = 3, kVfStatWarp0 = 19, kVfOutWarp0 = 23;
 constexpr int kVfColD2 = 256, kVfColOnes = 384, kVfColAug = 392;      // TMEM columns (D1[b] at 128 b, aug[b] at 392 + 8 b)
 
-template <int DV> struct VfCfg {
-    static constexpr int kXStages = 3;
-    static constexpr int kXBytes = kTileTokens * DV * 2;
+template <int DV, bool COMBINE> struct VfCfg {
+    static constexpr int kXStages = COMBINE ? 2 : 3;
+    static constexpr int kXBytes = 2 * kBlk;                     // a tile is always two 64-column blocks apart (d = 64 uses the first)
     static constexpr int kWBytes = DV * DV * 2;
     static constexpr int kAuxBytes = (DV / 64) * 2048;           // [16 K rows][DV] bf16
     static constexpr int kOffX = 0;
-    static constexpr int kOffW1 = kXStages * kXBytes;
+    static constexpr int kOffE = kXStages * kXBytes;             // COMBINE: [T tile | Y2 tile -> Out tile]; else the Out tile
+    static constexpr int kEBytes = (COMBINE ? 2 : 1) * kXBytes;
+    static constexpr int kOffW1 = kOffE + kEBytes;
     static constexpr int kOffW2 = kOffW1 + kWBytes;
     static constexpr int kOffAux = kOffW2 + kWBytes;
     static constexpr int kOffStat = kOffAux + kAuxBytes;         // rstd [2][128] floats
@@ -106,13 +135,13 @@ template <int DV> struct VfCfg {
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
 
-// X [rows][DV] bf16.  COMBINE: Out = X + y (.) Y2 (X is T), else Out = y.
+// X [rows][DV] bf16 (mapX).  COMBINE: Out = X + y (.) Y2 (X is T; mapY2 covers Y2), else Out = y.  mapOut covers Out.
 template <int DV, bool COMBINE>
 __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW1,
                                                                         const __grid_constant__ CUtensorMap mapW2, const __grid_constant__ CUtensorMap mapAux,
-                                                                        const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ Y2,
-                                                                        __nv_bfloat16* __restrict__ Out, long long rows, int* status) {
-    using Cfg = VfCfg<DV>;
+                                                                        const __grid_constant__ CUtensorMap mapY2, const __grid_constant__ CUtensorMap mapOut,
+                                                                        long long rows, int* status) {
+    using Cfg = VfCfg<DV, COMBINE>;
     constexpr int HC = DV / 4;
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
@@ -129,7 +158,9 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
     uint64_t* d2_full = bars + 14;     // MMA commit
     uint64_t* d2_empty = bars + 15;    // 128 arrivals
     uint64_t* w_full = bars + 16;      // TMA
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+    uint64_t* e_ready = bars + 17;     // the output tile may be used: TMA (COMBINE: its two input tiles have landed) or one arrival
+    uint64_t* o_full = bars + 18;      // 128 arrivals: the output tile is written
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -137,7 +168,7 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
     const int ntiles = (int)(t1 - t0);
 
     if (tid == 0) {
-        for (int i = 0; i < XST; ++i) {
+        for (int i = 0; i < 3; ++i) {
             mbar_init(&x_full[i], 1);
             mbar_init(&x_empty[i], 1);
         }
@@ -150,11 +181,15 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
         mbar_init(d2_full, 1);
         mbar_init(d2_empty, 128);
         mbar_init(w_full, 1);
+        mbar_init(e_ready, 1);
+        mbar_init(o_full, 128);
         fence_mbar_init();
         prefetch_tmap(&mapX);
         prefetch_tmap(&mapW1);
         prefetch_tmap(&mapW2);
         prefetch_tmap(&mapAux);
+        prefetch_tmap(&mapOut);
+        if (COMBINE) prefetch_tmap(&mapY2);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, 512);
@@ -185,7 +220,7 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
             for (int it = 0; it < ntiles; ++it) {
                 const int st = it % XST, u = it / XST;
                 if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 1101); break; }
-                mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
+                mbar_arrive_expect_tx(&x_full[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b)
                     tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
             }
@@ -232,46 +267,66 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
             if (!good) report_timeout(status, 1103);
         }
     } else if (warp >= kVfOutWarp0) {
-        // Out = y (or X + y (.) Y2), thread = token row, 16 columns at a time straight to global memory
+        // Out = y (or T + y (.) Y2): thread = token row; the result tile is formed in shared memory and stored by TMA
         const int quarter = warp & 3, row = quarter * 32 + lane;
+        const bool leader = warp == kVfOutWarp0 && lane == 0;
         const uint32_t ta = tmem + kVfColD2 + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t et = smem_u32(smem + Cfg::kOffE);                        // COMBINE: T tile
+        const uint32_t ot = et + (COMBINE ? Cfg::kXBytes : 0);                  // COMBINE: Y2 tile, overwritten by the result
+        auto open_tile = [&](int it) {      // leader only: the output tile is free; COMBINE fetches its two input tiles
+            if (COMBINE) {
+                mbar_arrive_expect_tx(e_ready, 2 * DV * kTileTokens * 2);
+                for (int b = 0; b < DV / 64; ++b) {
+                    tma_load_2d(smem + Cfg::kOffE + b * kBlk, &mapX, e_ready, b * 64, (int)((t0 + it) * kTileTokens));
+                    tma_load_2d(smem + Cfg::kOffE + Cfg::kXBytes + b * kBlk, &mapY2, e_ready, b * 64, (int)((t0 + it) * kTileTokens));
+                }
+            } else {
+                mbar_arrive(e_ready);
+            }
+        };
+        if (leader && ntiles > 0) open_tile(0);
         for (int it = 0; it < ntiles; ++it) {
             if (ok && !mbar_wait(d2_full, it & 1)) { ok = false; report_timeout(status, 1104); }
+            if (ok && !mbar_wait(e_ready, it & 1)) { ok = false; report_timeout(status, 1108); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const long long grow = (t0 + it) * kTileTokens + row;
-            const bool live = grow < rows;
-            const size_t off = (size_t)(live ? grow : 0) * DV;
 #pragma unroll 2
             for (int c = 0; c < DV / 16; ++c) {
-                uint32_t r[16];
+                uint32_t r[16], xw[8], yw[8], w[8];
                 tmem_ld16(ta + 16 * c, r);
-                uint4 tx[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)}, ty[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                if (COMBINE && live) {
-                    tx[0] = __ldg(reinterpret_cast<const uint4*>(X + off + 16 * c));
-                    tx[1] = __ldg(reinterpret_cast<const uint4*>(X + off + 16 * c) + 1);
-                    ty[0] = __ldg(reinterpret_cast<const uint4*>(Y2 + off + 16 * c));
-                    ty[1] = __ldg(reinterpret_cast<const uint4*>(Y2 + off + 16 * c) + 1);
+                if (COMBINE) {
+                    lds_row16(et, row, c, xw);
+                    lds_row16(ot, row, c, yw);
                 }
                 tmem_ld_wait();
-                uint32_t w[8];
-                const uint32_t* xw = reinterpret_cast<const uint32_t*>(tx);
-                const uint32_t* yw = reinterpret_cast<const uint32_t*>(ty);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     float a = __uint_as_float(r[2 * e]), b = __uint_as_float(r[2 * e + 1]);
                     if (COMBINE) {
-                        a = fmaf(a, __uint_as_float(yw[e] << 16), __uint_as_float(xw[e] << 16));
-                        b = fmaf(b, __uint_as_float(yw[e] & 0xffff0000u), __uint_as_float(xw[e] & 0xffff0000u));
+                        a = fmaf(a, bf_lo(yw[e]), bf_lo(xw[e]));
+                        b = fmaf(b, bf_hi(yw[e]), bf_hi(xw[e]));
                     }
                     w[e] = pack_bf16(a, b);
                 }
-                if (live) st_global_v8(Out + off + 16 * c, w);
+                sts_row16(ot, row, c, w);
             }
             tc_fence_before();
             mbar_arrive(d2_empty);
+            fence_proxy_async();
+            mbar_arrive(o_full);
+            if (leader) {
+                if (mbar_wait(o_full, it & 1)) {
+                    for (int b = 0; b < DV / 64; ++b) tma_store_2d(&mapOut, smem + Cfg::kOffE + (COMBINE ? Cfg::kXBytes : 0) + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
+                    tma_store_commit();
+                    tma_store_wait_read0();
+                    if (it + 1 < ntiles) open_tile(it + 1);
+                } else {
+                    report_timeout(status, 1109);
+                }
+            }
         }
+        if (leader) tma_store_wait_all0();
     } else if (warp >= kVfStatWarp0) {
         // row statistics of the tile -> rstd for the GELU warps, [-mu, sigma] for the extra K step
         const int quarter = warp & 3, row = quarter * 32 + lane;
@@ -326,48 +381,60 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
 }
 
 // ---- backward of one map (input gradient) ---------------------------------------------------------------------------
-// warp 0: TMA, warp 1: dg and dxhat MMAs, warp 2: h MMAs, warps 3..18: GELU' (thread = token row x quarter of the hidden units),
-// warps 19..22: dy = dOut (.) Yother tile and row statistics, warps 23..26: LayerNorm backward and output (thread = token row)
+// warp 0: TMA (weights, X tiles), warp 1: dg and dxhat MMAs, warp 2: h MMAs, warps 3..18: GELU' (thread = token row x quarter of
+// the hidden units), warps 19..22: dy = dOut (.) Yother and row statistics, warps 23..26: LayerNorm backward and output.
+// Shared-memory tiles: X (two stages, kept until the tile's output is formed: the LayerNorm backward needs xhat), dOut (one
+// stage: read by the dy warps, then overwritten by the result tile and stored - or added to dX - by TMA), Yother (one stage:
+// multiplied in place into dy, the A operand of the dg product).
+// The two row means of the LayerNorm backward come from the hidden layer, where the GELU' warps already hold the numbers:
+//     sum_i dxhat_i = sum_j dh_j c_j,     sum_i dxhat_i xhat_i = sum_j dh_j (h_j - b1'_j)       (dxhat = dh W1'^T, h = xhat W1' + b1')
 constexpr int kVbThreads = 27 * 32;
 constexpr int kVbGeluWarp0 = 3, kVbProdWarp0 = 19, kVbOutWarp0 = 23;
 constexpr int kVbColDg = 128, kVbColDx = 256, kVbColAug = 384;      // TMEM columns (h at 0, aug[b] at 384 + 8 b)
 
 template <int DV> struct VbCfg {
-    static constexpr int kXBytes = kTileTokens * DV * 2;
+    static constexpr int kXBytes = 2 * kBlk;
     static constexpr int kWBytes = DV * DV * 2;
     static constexpr int kAuxBytes = (DV / 64) * 2048;
     static constexpr int kOffX = 0;                              // 2 stages
-    static constexpr int kOffDy = 2 * kXBytes;                   // 2 stages: dy = dOut (.) Yother, the A operand of the dg product
-    static constexpr int kOffW1 = kOffDy + 2 * kXBytes;
+    static constexpr int kOffDo = 2 * kXBytes;                   // dOut tile -> result tile
+    static constexpr int kOffDy = kOffDo + kXBytes;              // Yother tile -> dy tile
+    static constexpr int kOffW1 = kOffDy + kXBytes;
     static constexpr int kOffW2 = kOffW1 + kWBytes;
     static constexpr int kOffAux = kOffW2 + kWBytes;
     static constexpr int kOffStat = kOffAux + kAuxBytes;         // [2][128] x (mu, rstd)
-    static constexpr int kOffBars = kOffStat + 2 * kTileTokens * 8;
+    static constexpr int kOffLnp = kOffStat + 2 * kTileTokens * 8;   // [2][4 parts][128] x (partial of sum dxhat, partial of sum dxhat xhat)
+    static constexpr int kOffCb = kOffLnp + 2 * 4 * kTileTokens * 8; // c [DV], b1' [DV] floats
+    static constexpr int kOffBars = kOffCb + 2 * DV * 4;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
 };
 
-// X, dOut, Yother, dX [rows][DV] bf16.  dX = J^T (dOut (.) Yother), plus dOut if RESIDUAL (the T side: Out = T + ...),
-// plus the previous content of dX if `accumulate` (dV on top of the gradient the attention backward wrote).
+// X, dOut, Yother, dX [rows][DV] bf16 behind their tensor maps.  dX = J^T (dOut (.) Yother), plus dOut if RESIDUAL (the T
+// side: Out = T + ...); with `accumulate` the tile is added to what dX holds instead of overwriting it.
 template <int DV, bool RESIDUAL>
 __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW1,
                                                                          const __grid_constant__ CUtensorMap mapW2, const __grid_constant__ CUtensorMap mapAux,
-                                                                         const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ dOut,
-                                                                         const __nv_bfloat16* __restrict__ Yother, __nv_bfloat16* dX, int accumulate,
-                                                                         long long rows, int* status) {
+                                                                         const __grid_constant__ CUtensorMap mapdO, const __grid_constant__ CUtensorMap mapY,
+                                                                         const __grid_constant__ CUtensorMap mapdX, const __nv_bfloat16* __restrict__ aux,
+                                                                         int accumulate, long long rows, int* status) {
     using Cfg = VbCfg<DV>;
     constexpr int HC = DV / 4;
     extern __shared__ uint8_t smem_raw[];
     grid_launch_dependents();
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     float2* stat = reinterpret_cast<float2*>(smem + Cfg::kOffStat);
+    float2* lnp = reinterpret_cast<float2*>(smem + Cfg::kOffLnp);
+    float* cb = reinterpret_cast<float*>(smem + Cfg::kOffCb);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* x_full = bars;           // [2] TMA
-    uint64_t* x_empty = bars + 2;      // [2] MMA commit
+    uint64_t* x_empty = bars + 2;      // [2] 128 arrivals (output warps)
     uint64_t* st_full = bars + 4;      // [2] 128 arrivals
-    uint64_t* dy_full = bars + 6;      // [2] 128 arrivals
-    uint64_t* dy_empty = bars + 8;     // [2] MMA commit
+    uint64_t* in_full = bars + 6;      // TMA: the dOut and Yother tiles have landed
+    uint64_t* dy_full = bars + 7;      // 128 arrivals
+    uint64_t* dy_empty = bars + 8;     // MMA commit
+    uint64_t* do_free = bars + 9;      // 1 arrival: the result tile has been read by its store
     uint64_t* h_full = bars + 10;      // MMA commit
     uint64_t* dh_full = bars + 11;     // 512 arrivals
     uint64_t* dh_free = bars + 12;     // MMA commit (the dxhat product has read dh: the h columns are free)
@@ -376,7 +443,8 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
     uint64_t* dx_full = bars + 15;     // MMA commit
     uint64_t* dx_empty = bars + 16;    // [2] 128 arrivals, by tile parity
     uint64_t* w_full = bars + 18;      // TMA
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
+    uint64_t* o_full = bars + 19;      // 128 arrivals: the result tile is written
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -386,12 +454,14 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(&x_full[i], 1);
-            mbar_init(&x_empty[i], 1);
+            mbar_init(&x_empty[i], 128);
             mbar_init(&st_full[i], 128);
-            mbar_init(&dy_full[i], 128);
-            mbar_init(&dy_empty[i], 1);
             mbar_init(&dx_empty[i], 128);
         }
+        mbar_init(in_full, 1);
+        mbar_init(dy_full, 128);
+        mbar_init(dy_empty, 1);
+        mbar_init(do_free, 1);
         mbar_init(h_full, 1);
         mbar_init(dh_full, 512);
         mbar_init(dh_free, 1);
@@ -399,11 +469,15 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
         mbar_init(dg_empty, 512);
         mbar_init(dx_full, 1);
         mbar_init(w_full, 1);
+        mbar_init(o_full, 128);
         fence_mbar_init();
         prefetch_tmap(&mapX);
         prefetch_tmap(&mapW1);
         prefetch_tmap(&mapW2);
         prefetch_tmap(&mapAux);
+        prefetch_tmap(&mapdO);
+        prefetch_tmap(&mapY);
+        prefetch_tmap(&mapdX);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, 512);
@@ -414,6 +488,12 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     grid_dependency_wait();
+    // c and b1' (fp32, from the two bf16 halves the folding kernel wrote) for the row means of the LayerNorm backward
+    for (int j = tid; j < DV; j += kVbThreads) {
+        cb[j] = __bfloat162float(aux[j]) + __bfloat162float(aux[DV + j]);
+        cb[DV + j] = __bfloat162float(aux[3 * DV + j]) + __bfloat162float(aux[4 * DV + j]);
+    }
+    __syncthreads();
     bool ok = true;
 
     if (warp == 0) {
@@ -427,7 +507,7 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
             for (int it = 0; it < ntiles; ++it) {
                 const int st = it & 1, u = it >> 1;
                 if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 1201); break; }
-                mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
+                mbar_arrive_expect_tx(&x_full[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b)
                     tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
             }
@@ -450,34 +530,30 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                     umma_bf16(tmem, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
                 umma_bf16_ta(tmem, tmem + kVbColAug + 8 * st, ad, idesc1, 1u);
                 umma_commit(h_full);
-                umma_commit(&x_empty[st]);
             }
             if (!good) report_timeout(status, 1202);
         }
     } else if (warp == 1) {
         if (lane == 0 && ntiles > 0) {
             const uint32_t idesc_k = idesc_bf16(128, DV, false, false);
-            const uint64_t yd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffDy), 16, 1024);      // dy tile, K-major over the output channels
+            const uint64_t yd = smem_desc_sw128(smem_u32(smem + Cfg::kOffDy), 16, 1024);       // dy tile, K-major over the output channels
             const uint64_t w2d = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 16, 1024);      // W2 [hidden][out] read K-major: N = hidden, K = out
             const uint64_t w1d = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), 16, 1024);      // W1' [in][hidden] read K-major: N = in, K = hidden
             bool good = mbar_wait(w_full, 0);
             auto issue_dg = [&](int it) -> bool {      // dg = dy W2^T; the GELU' warps of tile it - 1 must have taken their dg
-                const int st = it & 1;
                 if (it > 0 && !mbar_wait(dg_empty, (it - 1) & 1)) return false;
-                if (!mbar_wait(&dy_full[st], (it >> 1) & 1)) return false;
+                if (!mbar_wait(dy_full, it & 1)) return false;
                 tc_fence_after();
-                const uint64_t yd = desc_advance(yd0, st * Cfg::kXBytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + kVbColDg, desc_advance(yd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(w2d, (ks >> 2) * (DV * 128) + (ks & 3) * 32),
                               idesc_k, ks > 0 ? 1u : 0u);
                 umma_commit(dg_full);
-                umma_commit(&dy_empty[st]);
+                umma_commit(dy_empty);
                 return true;
             };
-            if (good && ntiles > 0) good = issue_dg(0);
             for (int it = 0; it < ntiles && good; ++it) {
-                if (it + 1 < ntiles && !issue_dg(it + 1)) { good = false; break; }
+                if (!issue_dg(it)) { good = false; break; }
                 // dxhat = dh W1'^T; the output warps must have read the previous tile's dxhat
                 if (!mbar_wait(dh_full, it & 1)) { good = false; break; }
                 if (it > 0 && !mbar_wait(&dx_empty[(it - 1) & 1], ((it - 1) >> 1) & 1)) { good = false; break; }
@@ -492,102 +568,106 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
             if (!good) report_timeout(status, 1203);
         }
     } else if (warp >= kVbOutWarp0) {
-        // LayerNorm backward: dx = rstd (dxhat - mean(dxhat) - xhat mean(dxhat xhat)); thread = token row, two passes over the row
+        // LayerNorm backward: dx = rstd (dxhat - mean(dxhat) - xhat mean(dxhat xhat)) (+ dOut); thread = token row.  The result
+        // replaces the dOut tile and leaves through TMA.
         const int quarter = warp & 3, row = quarter * 32 + lane;
+        const bool leader = warp == kVbOutWarp0 && lane == 0;
         const uint32_t ta = tmem + kVbColDx + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t dot = smem_u32(smem + Cfg::kOffDo);
         for (int it = 0; it < ntiles; ++it) {
+            const int st = it & 1;
             if (ok && !mbar_wait(dx_full, it & 1)) { ok = false; report_timeout(status, 1204); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const long long grow = (t0 + it) * kTileTokens + row;
-            const bool live = grow < rows;
-            const size_t off = (size_t)(live ? grow : 0) * DV;
-            const float2 ms = stat[(it & 1) * kTileTokens + row];
+            const float2 ms = stat[st * kTileTokens + row];
             const float mu = ms.x, rstd = ms.y;
             float s1 = 0.f, s2 = 0.f;
-#pragma unroll 2
-            for (int c = 0; c < DV / 16; ++c) {
-                uint32_t r[16];
-                tmem_ld16(ta + 16 * c, r);
-                uint4 tx[2];
-                tx[0] = __ldg(reinterpret_cast<const uint4*>(X + off + 16 * c));
-                tx[1] = __ldg(reinterpret_cast<const uint4*>(X + off + 16 * c) + 1);
-                tmem_ld_wait();
-                const uint32_t* xw = reinterpret_cast<const uint32_t*>(tx);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float a = __uint_as_float(r[2 * e]), b = __uint_as_float(r[2 * e + 1]);
-                    const float xa = (__uint_as_float(xw[e] << 16) - mu) * rstd, xb = (__uint_as_float(xw[e] & 0xffff0000u) - mu) * rstd;
-                    s1 += a + b;
-                    s2 = fmaf(a, xa, fmaf(b, xb, s2));
-                }
+            for (int p = 0; p < 4; ++p) {
+                const float2 v = lnp[(st * 4 + p) * kTileTokens + row];
+                s1 += v.x;
+                s2 += v.y;
             }
             const float m1 = s1 * (1.f / DV), m2 = s2 * (1.f / DV);
+            const uint32_t xt = smem_u32(smem + Cfg::kOffX + st * Cfg::kXBytes);
 #pragma unroll 2
             for (int c = 0; c < DV / 16; ++c) {
-                uint32_t r[16];
+                uint32_t r[16], xw[8], dw[8], w[8];
                 tmem_ld16(ta + 16 * c, r);
-                uint4 tx[2], td[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)}, tp[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                tx[0] = __ldg(reinterpret_cast<const uint4*>(X + off + 16 * c));
-                tx[1] = __ldg(reinterpret_cast<const uint4*>(X + off + 16 * c) + 1);
-                if (RESIDUAL) {
-                    td[0] = __ldg(reinterpret_cast<const uint4*>(dOut + off + 16 * c));
-                    td[1] = __ldg(reinterpret_cast<const uint4*>(dOut + off + 16 * c) + 1);
-                }
-                if (accumulate && live) {
-                    tp[0] = *reinterpret_cast<const uint4*>(dX + off + 16 * c);
-                    tp[1] = *(reinterpret_cast<const uint4*>(dX + off + 16 * c) + 1);
-                }
+                lds_row16(xt, row, c, xw);
+                if (RESIDUAL) lds_row16(dot, row, c, dw);
                 tmem_ld_wait();
-                const uint32_t* xw = reinterpret_cast<const uint32_t*>(tx);
-                const uint32_t* dw = reinterpret_cast<const uint32_t*>(td);
-                const uint32_t* pw = reinterpret_cast<const uint32_t*>(tp);
-                uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float xa = (__uint_as_float(xw[e] << 16) - mu) * rstd, xb = (__uint_as_float(xw[e] & 0xffff0000u) - mu) * rstd;
+                    const float xa = (bf_lo(xw[e]) - mu) * rstd, xb = (bf_hi(xw[e]) - mu) * rstd;
                     float a = rstd * (__uint_as_float(r[2 * e]) - m1 - xa * m2), b = rstd * (__uint_as_float(r[2 * e + 1]) - m1 - xb * m2);
-                    a += __uint_as_float(dw[e] << 16) + __uint_as_float(pw[e] << 16);
-                    b += __uint_as_float(dw[e] & 0xffff0000u) + __uint_as_float(pw[e] & 0xffff0000u);
+                    if (RESIDUAL) {
+                        a += bf_lo(dw[e]);
+                        b += bf_hi(dw[e]);
+                    }
                     w[e] = pack_bf16(a, b);
                 }
-                if (live) st_global_v8(dX + off + 16 * c, w);
+                sts_row16(dot, row, c, w);
             }
             tc_fence_before();
-            mbar_arrive(&dx_empty[it & 1]);
+            mbar_arrive(&dx_empty[st]);
+            mbar_arrive(&x_empty[st]);
+            fence_proxy_async();
+            mbar_arrive(o_full);
+            if (leader) {
+                if (mbar_wait(o_full, it & 1)) {
+                    for (int b = 0; b < DV / 64; ++b) {
+                        if (accumulate) tma_reduce_add_2d(&mapdX, smem + Cfg::kOffDo + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
+                        else tma_store_2d(&mapdX, smem + Cfg::kOffDo + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
+                    }
+                    tma_store_commit();
+                    tma_store_wait_read0();
+                    mbar_arrive(do_free);
+                } else {
+                    report_timeout(status, 1210);
+                }
+            }
         }
+        if (leader) tma_store_wait_all0();
     } else if (warp >= kVbProdWarp0) {
-        // dy = dOut (.) Yother -> A operand of the dg product; then the row statistics of the X tile
+        // dy = dOut (.) Yother in place over the Yother tile -> A operand of the dg product; then the row statistics of the X tile
         const int t = tid - kVbProdWarp0 * 32;      // 0..127
         const int quarter = warp & 3, row = quarter * 32 + lane;
         constexpr int CPR = DV / 8;                 // 16-byte chunks per row
+        const uint32_t dot = smem_u32(smem + Cfg::kOffDo), dyt = smem_u32(smem + Cfg::kOffDy);
         for (int it = 0; it < ntiles; ++it) {
             const int st = it & 1, par = (it >> 1) & 1;
-            if (ok && !mbar_wait(&dy_empty[st], par ^ 1)) { ok = false; report_timeout(status, 1205); }
+            if (t == 0) {
+                // both tiles are free: the dg product of the previous tile has read dy, its result tile has been stored
+                bool free_ = it == 0 || (mbar_wait(dy_empty, (it - 1) & 1) && mbar_wait(do_free, (it - 1) & 1));
+                if (free_) {
+                    mbar_arrive_expect_tx(in_full, 2 * DV * kTileTokens * 2);
+                    for (int b = 0; b < DV / 64; ++b) {
+                        tma_load_2d(smem + Cfg::kOffDo + b * kBlk, &mapdO, in_full, b * 64, (int)((t0 + it) * kTileTokens));
+                        tma_load_2d(smem + Cfg::kOffDy + b * kBlk, &mapY, in_full, b * 64, (int)((t0 + it) * kTileTokens));
+                    }
+                } else {
+                    report_timeout(status, 1205);
+                }
+            }
+            if (ok && !mbar_wait(in_full, it & 1)) { ok = false; report_timeout(status, 1211); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const uint32_t dyt = smem_u32(smem + Cfg::kOffDy + st * Cfg::kXBytes);
 #pragma unroll 4
             for (int k = 0; k < CPR; ++k) {
                 const int idx = k * 128 + t, r = idx / CPR, ch = idx % CPR;
-                const long long grow = (t0 + it) * kTileTokens + r;
-                uint4 a = make_uint4(0, 0, 0, 0), b = make_uint4(0, 0, 0, 0);
-                if (grow < rows) {
-                    a = __ldg(reinterpret_cast<const uint4*>(dOut + (size_t)grow * DV) + ch);
-                    b = __ldg(reinterpret_cast<const uint4*>(Yother + (size_t)grow * DV) + ch);
-                }
-                const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
-                const uint32_t* bw = reinterpret_cast<const uint32_t*>(&b);
+                const uint32_t off = (ch >> 3) * kBlk + sw128_off(r, ch & 7);
+                uint32_t a[4], b[4];
+                asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(dot + off) : "memory");
+                asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]) : "r"(dyt + off) : "memory");
                 uint32_t w[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    w[e] = pack_bf16(__uint_as_float(aw[e] << 16) * __uint_as_float(bw[e] << 16),
-                                     __uint_as_float(aw[e] & 0xffff0000u) * __uint_as_float(bw[e] & 0xffff0000u));
-                st_shared_v4(dyt + (ch >> 3) * kBlk + sw128_off(r, ch & 7), w[0], w[1], w[2], w[3]);
+                for (int e = 0; e < 4; ++e) w[e] = pack_bf16(bf_lo(a[e]) * bf_lo(b[e]), bf_hi(a[e]) * bf_hi(b[e]));
+                st_shared_v4(dyt + off, w[0], w[1], w[2], w[3]);
             }
             fence_proxy_async();
-            mbar_arrive(&dy_full[st]);
+            mbar_arrive(dy_full);
             // statistics: buffer st was last read by the output warps of tile it - 2
             if (ok && !mbar_wait(&x_full[st], par)) { ok = false; report_timeout(status, 1206); }
             if (ok && it >= 2 && !mbar_wait(&dx_empty[st], par ^ 1)) { ok = false; report_timeout(status, 1207); }
@@ -606,6 +686,7 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
         const int quarter = warp & 3, part = (warp - kVbGeluWarp0) >> 2, row = quarter * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         for (int it = 0; it < ntiles; ++it) {
+            const int st = it & 1;
             if (!mbar_wait(dg_full, it & 1)) { ok = false; report_timeout(status, 1208); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -620,8 +701,9 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const float rstd = stat[(it & 1) * kTileTokens + row].y;
+            const float rstd = stat[st * kTileTokens + row].y;
             const uint32_t ta = tmem + lane_base + part * HC;
+            float2 p1 = make_float2(0.f, 0.f), p2 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
                 uint32_t r[16];
@@ -630,13 +712,19 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
+                    const int j = part * HC + 16 * c + 2 * e;
                     const float2 h = __fmul2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), splat2(rstd));
                     const float2 dg = make_float2(__uint_as_float(dgr[16 * c + 2 * e]), __uint_as_float(dgr[16 * c + 2 * e + 1]));
                     const float2 dh = __fmul2_rn(__fmul2_rn(dg, splat2(0.5f)), gelu_grad2_twice(h));
                     w[e] = pack_bf16(dh.x, dh.y);
+                    const float2 dr = make_float2(bf_lo(w[e]), bf_hi(w[e]));      // dh as the dxhat product sees it
+                    const float2 cj = *reinterpret_cast<const float2*>(cb + j), bj = *reinterpret_cast<const float2*>(cb + DV + j);
+                    p1 = __ffma2_rn(dr, cj, p1);
+                    p2 = __ffma2_rn(dr, make_float2(h.x - bj.x, h.y - bj.y), p2);
                 }
                 tmem_st8(ta + 8 * c, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
             }
+            lnp[(st * 4 + part) * kTileTokens + row] = make_float2(p1.x + p1.y, p2.x + p2.y);
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(dh_full);
@@ -677,44 +765,46 @@ inline hla_status launch_vmod(const VmodPlan& P, long long rows, const hla_vmlp*
         a[i] = VmlpPtrs{static_cast<const bf*>(v[i].ln_g), static_cast<const bf*>(v[i].ln_b), static_cast<const bf*>(v[i].W1), static_cast<const bf*>(v[i].b1),
                         static_cast<const bf*>(v[i].W2), static_cast<const bf*>(v[i].b2)};
     rec.begin("vmod_fold");
-    vmod_fold_kernel<<<2, 128, 0, st>>>(a[0], a[1], w1f, aux, DV);
+    vmod_fold_kernel<<<dim3(2, DV / 32), 256, 0, st>>>(a[0], a[1], w1f, aux, DV);
     if (!rec.end()) return HLA_ERR_CUDA;
-    CUtensorMap mapT, mapV, mapW1[2], mapW2[2], mapAux[2];
-    if (!make_map_2d(&mapT, T, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapV, V, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
+    CUtensorMap mapT, mapV, mapY1, mapY2, mapW1[2], mapW2[2], mapAux[2];
+    if (!make_map_2d(&mapT, T, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapV, V, (size_t)rows, DV, kTileTokens) ||
+        !make_map_2d(&mapY1, y1, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapY2, y2, (size_t)rows, DV, kTileTokens))
+        return HLA_ERR_CUDA;
     for (int i = 0; i < 2; ++i)
         if (!make_map_2d(&mapW1[i], w1f + (size_t)i * DV * DV, DV, DV, DV) || !make_map_2d(&mapW2[i], v[i].W2, DV, DV, DV) ||
             !make_map_2d(&mapAux[i], aux + (size_t)i * 16 * DV, 16, DV, 16))
             return HLA_ERR_CUDA;
-    if (!set_smem(tc_vmlp_forward_kernel<DV, false>, VfCfg<DV>::kSmem) || !set_smem(tc_vmlp_forward_kernel<DV, true>, VfCfg<DV>::kSmem) ||
+    if (!set_smem(tc_vmlp_forward_kernel<DV, false>, VfCfg<DV, false>::kSmem) || !set_smem(tc_vmlp_forward_kernel<DV, true>, VfCfg<DV, true>::kSmem) ||
         !set_smem(tc_vmlp_backward_kernel<DV, false>, VbCfg<DV>::kSmem) || !set_smem(tc_vmlp_backward_kernel<DV, true>, VbCfg<DV>::kSmem))
         return HLA_ERR_CUDA;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    const bf* Tb = static_cast<const bf*>(T);
-    const bf* Vb = static_cast<const bf*>(V);
     // Y2 = phi_v2(V)
     rec.begin("tc_vmlp_forward");
-    launch_pdl(tc_vmlp_forward_kernel<DV, false>, grid, dim3(kVfThreads), VfCfg<DV>::kSmem, st, mapV, mapW1[1], mapW2[1], mapAux[1], Vb, (const bf*)nullptr, y2, rows,
-               status);
+    launch_pdl(tc_vmlp_forward_kernel<DV, false>, grid, dim3(kVfThreads), VfCfg<DV, false>::kSmem, st, mapV, mapW1[1], mapW2[1], mapAux[1], mapY2, mapY2, rows, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     if (!backward) {      // Out = T + phi_v1(T) (.) Y2
+        CUtensorMap mapOut;
+        if (!make_map_2d(&mapOut, Out, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
         rec.begin("tc_vmlp_forward_combine");
-        launch_pdl(tc_vmlp_forward_kernel<DV, true>, grid, dim3(kVfThreads), VfCfg<DV>::kSmem, st, mapT, mapW1[0], mapW2[0], mapAux[0], Tb, (const bf*)y2,
-                   static_cast<bf*>(Out), rows, status);
+        launch_pdl(tc_vmlp_forward_kernel<DV, true>, grid, dim3(kVfThreads), VfCfg<DV, true>::kSmem, st, mapT, mapW1[0], mapW2[0], mapAux[0], mapY2, mapOut, rows, status);
         return rec.end() ? HLA_OK : HLA_ERR_CUDA;
     }
     rec.begin("tc_vmlp_forward");      // Y1 = phi_v1(T)
-    launch_pdl(tc_vmlp_forward_kernel<DV, false>, grid, dim3(kVfThreads), VfCfg<DV>::kSmem, st, mapT, mapW1[0], mapW2[0], mapAux[0], Tb, (const bf*)nullptr, y1, rows,
-               status);
+    launch_pdl(tc_vmlp_forward_kernel<DV, false>, grid, dim3(kVfThreads), VfCfg<DV, false>::kSmem, st, mapT, mapW1[0], mapW2[0], mapAux[0], mapY1, mapY1, rows, status);
     if (!rec.end()) return HLA_ERR_CUDA;
-    const bf* dOb = static_cast<const bf*>(dOut);
+    CUtensorMap mapdO, mapdT, mapdV;
+    if (!make_map_2d(&mapdO, dOut, (size_t)rows, DV, kTileTokens) || !make_map_2d(&mapdT, dT, (size_t)rows, DV, kTileTokens) ||
+        !make_map_2d(&mapdV, dV, (size_t)rows, DV, kTileTokens))
+        return HLA_ERR_CUDA;
     rec.begin("tc_vmlp_backward_t");   // dT = dOut + J1^T (dOut (.) Y2)
-    launch_pdl(tc_vmlp_backward_kernel<DV, true>, grid, dim3(kVbThreads), VbCfg<DV>::kSmem, st, mapT, mapW1[0], mapW2[0], mapAux[0], Tb, dOb, (const bf*)y2,
-               static_cast<bf*>(dT), 0, rows, status);
+    launch_pdl(tc_vmlp_backward_kernel<DV, true>, grid, dim3(kVbThreads), VbCfg<DV>::kSmem, st, mapT, mapW1[0], mapW2[0], mapAux[0], mapdO, mapY2, mapdT,
+               (const bf*)aux, 0, rows, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_vmlp_backward_v");   // dV (+)= J2^T (dOut (.) Y1)
-    launch_pdl(tc_vmlp_backward_kernel<DV, false>, grid, dim3(kVbThreads), VbCfg<DV>::kSmem, st, mapV, mapW1[1], mapW2[1], mapAux[1], Vb, dOb, (const bf*)y1,
-               static_cast<bf*>(dV), accumulate_dV, rows, status);
+    launch_pdl(tc_vmlp_backward_kernel<DV, false>, grid, dim3(kVbThreads), VbCfg<DV>::kSmem, st, mapV, mapW1[1], mapW2[1], mapAux[1], mapdO, mapY1, mapdV,
+               (const bf*)(aux + (size_t)16 * DV), accumulate_dV, rows, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
