@@ -1,12 +1,14 @@
-// Tensor-core kernels of the feature networks phi (appendix "Defining phi";
-// Algorithm 1 step 4) for bf16:  feat = ReLU(W2^T GELU(W1^T x + b1) + b2).
+// Tensor-core building blocks of the feature networks phi (appendix "Defining phi";
+// Algorithm 1 step 4) for bf16:  feat = ReLU(W2^T GELU(W1^T x + b1) + b2), and their backward.
 //
-// Per 128-token tile of X (Q or K, TMA-loaded once) and per map m:
-//   D1 = X * W1[m]            tcgen05, fp32 in TMEM        [128 tok x d hidden]
-//   G  = bf16(GELU(D1 + b1))  16 warps, thread = (token, quarter of the hidden units); written as the next MMA's A operand
+// Forward, per 128-token tile of X (Q or K, TMA-loaded once) and per map m - the pipeline the fused key-side and
+// query-side kernels of the forward (hla_tc_fused_k.cuh, hla_tc_fused.cuh) run:
+//   D1 = X * W1[m] + b1       tcgen05, fp32 in TMEM        [128 tok x d hidden]; the bias is a ninth K step
+//   G  = bf16(GELU(D1))       16 warps, thread = (token, quarter of the hidden units); written as the next MMA's A operand
 //   D2 = G * W2[m]            tcgen05, N padded to 16
-//   feat = ReLU(D2 + b2)      fp32 features to global memory
-// The key side runs its F maps on the same X tile, so K is read once.
+//   feat = ReLU(D2 + b2)      fp32 features
+// The key side runs its F maps on the same X tile, so K is read once.  This file holds the GELU / GELU' arithmetic and
+// the backward kernel.
 // GELU is the exact erf form, x Phi(x), with Phi evaluated as 1/2 + tanh(x (a + b x^2)) / 2 (a, b fitted to erf; one
 // tanh.approx per hidden unit) - total error of Phi below 4e-4, several times below the bf16 rounding of G.
 #pragma once
@@ -57,260 +59,6 @@ struct PhiPtrs {
 struct PhiMaps {
     CUtensorMap w1[3];
 };
-
-// warp 0: TMA loads, warp 1: second-layer MMAs, warp 2: first-layer MMAs, warps 3..18: GELU (thread = token row x quarter of
-// the hidden units), warps 19..22: feature epilogue.  The two MMA streams are issued by different warps (different
-// schedulers) because one thread issuing both was the slowest stage of the pipeline.
-constexpr int kPfThreads = 736;
-constexpr int kPfGeluWarp0 = 3, kPfFeatWarp0 = 19;
-
-template <int DV, int NMAPS> struct PfCfg {
-    static constexpr int kXStages = 2;
-    static constexpr int kXBytes = kTileTokens * DV * 2;
-    static constexpr int kW1Bytes = DV * DV * 2;
-    static constexpr int kW2Bytes = (DV / 64) * 2048;            // [16 rows][DV] bf16, K-major, per map
-    static constexpr int kOffX = 0;
-    static constexpr int kOffW1 = kXStages * kXBytes;            // (the GELU tiles live in TMEM)
-    static constexpr int kOffW2 = kOffW1 + NMAPS * kW1Bytes;
-    // The first-layer bias rides on the tensor cores as a ninth K step: A = a constant tile whose K column 0 is 1,
-    // B = per map a tile whose K row 0 is b1 (both zero elsewhere), so the arithmetic warps add nothing.
-    static constexpr int kOffOnes = kOffW2 + ((NMAPS * kW2Bytes + 1023) / 1024) * 1024;   // [128 rows][64 K] bf16, K-major (16 K columns used)
-    static constexpr int kB1Bytes = (DV / 64) * 2048;            // per map: [16 K rows][DV] bf16, MN-major
-    static constexpr int kOffB1 = kOffOnes + kBlk;
-    static constexpr int kOffBias = kOffB1 + NMAPS * kB1Bytes;   // per map: b1[DV] (unused by the kernel), b2[8] floats
-    static constexpr int kOffBars = kOffBias + NMAPS * (DV + 8) * 4;
-    static constexpr int kSmemUsed = 1024 + kOffBars + 256;
-    static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
-};
-
-// X [rows][DV] bf16 (rows = B*H*N tokens).  KSIDE: features to kf[bh][f][n][6], else qf[row][6].
-// A "unit" is one map of one tile.  h and the GELU tile are double-buffered, and the feature epilogue of a unit
-// runs one unit late, so the GELU warps never wait for a tensor-core round trip.
-template <int DV, int NMAPS, bool KSIDE>
-__global__ void __launch_bounds__(kPfThreads, 1) tc_phi_forward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
-                                                                       PhiPtrs P, float* __restrict__ feat, long long rows, int N, int* status) {
-    using Cfg = PfCfg<DV, NMAPS>;
-    constexpr int HC = DV / 4;          // hidden units per epilogue thread
-    constexpr int XST = Cfg::kXStages;
-    extern __shared__ uint8_t smem_raw[];
-    grid_launch_dependents();
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    float* bias = reinterpret_cast<float*>(smem + Cfg::kOffBias);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
-    uint64_t* x_full = bars;           // [2]
-    uint64_t* x_empty = bars + 2;      // [2] MMA commit
-    uint64_t* d1_full = bars + 4;      // [2] MMA commit
-    uint64_t* d1_empty = bars + 6;     // [2] 512 arrivals
-    uint64_t* g_full = bars + 8;       // [2] 512 arrivals
-    uint64_t* g_free = bars + 10;      // [2] MMA commit
-    uint64_t* d2_full = bars + 12;     // [2] MMA commit
-    uint64_t* d2_empty = bars + 14;    // [2] 128 arrivals
-    uint64_t* w_full = bars + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
-    const long long t0 = tiles * blockIdx.x / gridDim.x, t1 = tiles * (blockIdx.x + 1) / gridDim.x;
-    const int ntiles = (int)(t1 - t0);
-    const int nunits = ntiles * NMAPS;
-
-    // second-layer weights as a K-major MMA operand [16 rows (outputs, 6 used)][DV], and the biases
-    for (int i = tid; i < NMAPS * Cfg::kW2Bytes / 16; i += kPfThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffW2)[i] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
-    for (int i = tid; i < NMAPS * DV * 6; i += kPfThreads) {
-        const int m = i / (DV * 6), j = (i / 6) % DV, o = i % 6;
-        uint8_t* base = smem + Cfg::kOffW2 + m * Cfg::kW2Bytes + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = half_bf16(P.W2[m][j * 6 + o]);
-    }
-    for (int i = tid; i < (kBlk + NMAPS * Cfg::kB1Bytes) / 16; i += kPfThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffOnes)[i] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
-    for (int i = tid; i < kTileTokens; i += kPfThreads)
-        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffOnes + sw128_off(i, 0)) = __float2bfloat16_rn(1.f);
-    for (int i = tid; i < NMAPS * DV; i += kPfThreads) {
-        const int m = i / DV, j = i % DV;       // K row 0 of the MN-major tile: 64-column block j / 64, no swizzle in row 0
-        *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffB1 + m * Cfg::kB1Bytes + (j >> 6) * 2048 + (j & 63) * 2) = P.b1[m][j];
-    }
-    for (int i = tid; i < NMAPS * (DV + 8); i += kPfThreads) {
-        const int m = i / (DV + 8), j = i % (DV + 8);
-        bias[i] = j < DV ? __bfloat162float(P.b1[m][j]) : (j - DV < 6 ? __bfloat162float(P.b2[m][j - DV]) : 0.f);
-    }
-    fence_proxy_async();
-    if (tid == 0) {
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&x_full[i], 1);
-            mbar_init(&x_empty[i], 1);
-            mbar_init(&d1_full[i], 1);
-            mbar_init(&d1_empty[i], 512);
-            mbar_init(&g_full[i], 512);
-            mbar_init(&g_free[i], 1);
-            mbar_init(&d2_full[i], 1);
-            mbar_init(&d2_empty[i], 128);
-        }
-        mbar_init(w_full, 1);
-        fence_mbar_init();
-        prefetch_tmap(&mapX);
-    }
-    if (warp == 1) {
-        tmem_alloc(tmem_slot, 512);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;     // D1[b] at columns 128*b, D2[b] at columns 256 + 32*b, G[b] (bf16 pairs) at 320 + 64*b
-    grid_dependency_wait();
-    bool ok = true;
-
-    if (warp == 0) {
-        if (lane == 0 && ntiles > 0) {
-            mbar_arrive_expect_tx(w_full, NMAPS * Cfg::kW1Bytes);
-            for (int m = 0; m < NMAPS; ++m)
-                for (int b = 0; b < DV / 64; ++b)
-                    tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
-            for (int it = 0; it < ntiles; ++it) {
-                const int st = it % XST, u = it / XST;
-                if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 501); break; }
-                mbar_arrive_expect_tx(&x_full[st], Cfg::kXBytes);
-                for (int b = 0; b < DV / 64; ++b)
-                    tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
-            }
-        }
-    } else if (warp == 2) {
-        if (lane == 0 && ntiles > 0) {      // D1[b] = X * W1[m]
-            const uint32_t idesc1 = idesc_bf16(128, DV, false, true);   // X K-major, W1 [in][hidden] MN-major
-            const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
-            const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
-            const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffOnes), 16, 1024);
-            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffB1), 2048, 1024);
-            bool good = mbar_wait(w_full, 0);
-            for (int unit = 0; unit < nunits && good; ++unit) {
-                const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
-                if (m == 0 && !mbar_wait(&x_full[st], (it / XST) & 1)) { good = false; break; }
-                if (!mbar_wait(&d1_empty[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
-                tc_fence_after();
-                const uint64_t xd = desc_advance(xd0, st * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
-#pragma unroll
-                for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
-                umma_bf16(tmem + 128 * b, od, desc_advance(bd0, m * Cfg::kB1Bytes), idesc1, 1u);      // + 1 * b1
-                umma_commit(&d1_full[b]);
-                if (m == NMAPS - 1) umma_commit(&x_empty[st]);
-            }
-            if (!good) report_timeout(status, 502);
-        }
-    } else if (warp == 1) {
-        if (lane == 0 && ntiles > 0) {      // D2[b] = G[b] * W2[m]
-            const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G from TMEM, W2 operand K-major
-            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 16, 1024);
-            bool good = true;
-            for (int unit = 0; unit < nunits && good; ++unit) {
-                const int m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
-                if (!(mbar_wait(&g_full[b], par) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
-                tc_fence_after();
-                const uint64_t vd = desc_advance(vd0, m * Cfg::kW2Bytes);
-#pragma unroll
-                for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16_ta(tmem + 256 + 32 * b, tmem + 320 + 64 * b + 8 * ks, desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32), idesc2, ks > 0 ? 1u : 0u);
-                umma_commit(&g_free[b]);
-                umma_commit(&d2_full[b]);
-            }
-            if (!good) report_timeout(status, 503);
-        }
-    } else if (warp >= kPfFeatWarp0) {
-        // feature epilogue: ReLU(D2 + b2) -> global memory; thread = token row
-        const int quarter = warp & 3, row = quarter * 32 + lane;
-        for (int unit = 0; unit < nunits; ++unit) {
-            const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1;
-            if (!mbar_wait(&d2_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 506); }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t r[8];
-            tmem_ld8(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), r);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(&d2_empty[b]);
-            const long long grow = (t0 + it) * kTileTokens + row;
-            if (grow < rows) {
-                const float* b2s = bias + m * (DV + 8) + DV;
-                float f[6];
-#pragma unroll
-                for (int o = 0; o < 6; ++o) f[o] = fmaxf(__uint_as_float(r[o]) + b2s[o], 0.f);
-                if (KSIDE) {
-                    const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
-                    store6(feat + ((size_t)(bh * NMAPS + m) * N + n) * 6, f);
-                } else {
-                    store6(feat + grow * 6, f);
-                }
-            }
-        }
-    } else {
-        const int quarter = warp & 3, part = (warp - kPfGeluWarp0) >> 2;
-        for (int unit = 0; unit < nunits; ++unit) {
-            const int b = unit & 1, par = (unit >> 1) & 1;
-            if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 504); }
-            if (ok && !mbar_wait(&g_free[b], par ^ 1)) { ok = false; report_timeout(status, 505); }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + part * HC;
-            const uint32_t tg = tmem + 320 + 64 * b + ((uint32_t)(quarter * 32) << 16) + part * (HC / 2);
-            uint32_t r[HC];
-#pragma unroll
-            for (int c = 0; c < HC / 16; ++c) tmem_ld16(ta + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(&d1_empty[b]);          // h is in registers: the next first-layer product may overwrite it
-#pragma unroll
-            for (int c = 0; c < HC / 16; ++c) {
-                uint32_t w[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float2 g = gelu2_twice(make_float2(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1])));
-                    w[e] = pack_bf16(g.x, g.y);
-                }
-                tmem_st8(tg + 8 * c, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);      // the second layer's A operand lives in TMEM: no shared-memory round trip
-            }
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(&g_full[b]);
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 512);
-}
-
-// Key-side feature maps phi_k1..3 on K (phi_q runs inside the fused query-side kernel, hla_tc_fused.cuh).
-template <int DV>
-inline hla_status launch_phi_forward_k(const Dims& D, int BH, const hla_mlp* phi_k, const void* K, char* ws, const hla_ws_layout& L, int sm_count,
-                                       LaunchRec& rec) {
-    const long long rows = (long long)BH * D.N;
-    CUtensorMap mapK;
-    PhiMaps mk;
-    PhiPtrs pk{};
-    if (!make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
-    for (int f = 0; f < 3; ++f) {
-        if (!make_map_2d(&mk.w1[f], phi_k[f].W1, DV, DV, DV)) return HLA_ERR_CUDA;
-        pk.b1[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b1);
-        pk.W2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].W2);
-        pk.b2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b2);
-    }
-    int* status = reinterpret_cast<int*>(ws + L.status);
-    if (!set_smem(tc_phi_forward_kernel<DV, 3, true>, PfCfg<DV, 3>::kSmem)) return HLA_ERR_CUDA;
-    const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
-    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    rec.begin("tc_phi_forward_k");
-    // first kernel of hla_forward, and it stages the weights before its dependency wait: no overlap with what precedes it
-    launch_serial(tc_phi_forward_kernel<DV, 3, true>, grid, dim3(kPfThreads), PfCfg<DV, 3>::kSmem, rec.st, mapK, mk, pk, reinterpret_cast<float*>(ws + L.kf), rows, D.N, status);
-    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
-}
-
-inline hla_status phi_forward_k(const Dims& D, int BH, const hla_mlp* phi_k, const void* K, char* ws, const hla_ws_layout& L, int sm_count,
-                                LaunchRec& rec) {
-    if (D.d == 128) return launch_phi_forward_k<128>(D, BH, phi_k, K, ws, L, sm_count, rec);
-    return launch_phi_forward_k<64>(D, BH, phi_k, K, ws, L, sm_count, rec);
-}
 
 // =======================================================================================
 // Backward of the feature networks with respect to their input (weights fixed):
