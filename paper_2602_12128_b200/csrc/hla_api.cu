@@ -261,6 +261,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     D.ld = c.d + 4;
     D.eps = c.eps;
     x->tc = tc::supported(c.dtype == HLA_BF16, c.d, c.F, c.d_phi) && (long long)c.B * c.H * c.N < (1ll << 31);   // the tensor-core kernels index tokens in 32 bits
+    if (c.F == 2 && c.phi == HLA_PHI_MLP) x->tc = false;      // the 2-factor geometry runs on the tensor cores at the feature level only
     const int tile = x->tc ? tc::kTileTokens : simt::kTok;
     const int tiles = (c.N + tile - 1) / tile;
     int S = c.n_splits;
@@ -297,7 +298,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     L.dqf = mlp ? cv.take(tok * c.d_phi * 4) : kNone;
     L.dkf = mlp ? cv.take(tok * c.F * c.d_phi * 4) : kNone;
     L.state_ld = D.ld;
-    L.state_rows = x->tc ? tc::kMono : P;
+    L.state_rows = x->tc ? tc::n_mono(c.F) : P;
     L.n_splits = S;
     L.tensor_core = x->tc ? 1 : 0;
     // partial states: S per head from the split kernels, or the pieces of the fused key-side kernel (folded rows)
@@ -305,7 +306,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     size_t part_bytes = (size_t)x->BH * S * P * D.ld * 4;
     if (x->tc && mlp) {
         x->k_pieces = tc::fused_key_max_pieces(x->BH, tiles, tc::fused_key_grid(x->BH, c.N, x->sm_count));
-        const size_t need = (size_t)x->BH * x->k_pieces * tc::kMono * D.ld * 4;
+        const size_t need = (size_t)x->BH * x->k_pieces * tc::n_mono(c.F) * D.ld * 4;
         if (need > part_bytes) part_bytes = need;
     }
     x->off_part = cv.take(part_bytes);
@@ -391,8 +392,9 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     tc::HostCacheScope scope(&ctx->hc);
     if (ctx->tc) {
         const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
-        // the phi backward writes rows of dQ, dK with 32-byte stores
+        // the phi backward writes rows of dQ, dK with 32-byte stores; so does the 2-factor key pass with dV
         if (mlp && ((reinterpret_cast<uintptr_t>(dQ) | reinterpret_cast<uintptr_t>(dK)) & 31u)) return HLA_ERR_INVALID_ARG;
+        if (ctx->D.F == 2 && (reinterpret_cast<uintptr_t>(dV) & 31u)) return HLA_ERR_INVALID_ARG;
         const float* qf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.qf) : static_cast<const float*>(Q);
         const float* kf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.kf) : static_cast<const float*>(K);
         float* dqf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dqf) : static_cast<float*>(dQ);

@@ -40,19 +40,32 @@ __host__ __device__ constexpr int mono_of(int x, int y, int z) {
     return mono_idx(imin(imin(x, y), z), x + y + z - imin(imin(x, y), z) - imax(imax(x, y), z), imax(imax(x, y), z));
 }
 
+// The two monomial geometries of the tensor-core path.  F factors of d_phi features each: the query tensor q (x) ... (x) q
+// has kN distinct monomials; every operand tile over the monomials is kPad columns wide, in kBlocks swizzled blocks of 64.
+//   F = 3, d_phi = 6  (the paper's main model): 56 monomials q_a q_b q_c, a <= b <= c
+//   F = 2, d_phi = 12 (its 2-factor variant):   78 monomials q_a q_b,     a <= b
+template <int F> struct MT;
+template <> struct MT<3> { static constexpr int kDphi = 6, kN = 56, kPad = 64, kBlocks = 1, kKf = 18, kMaps = 3; };
+template <> struct MT<2> { static constexpr int kDphi = 12, kN = 78, kPad = 80, kBlocks = 2, kKf = 24, kMaps = 2; };
+// index of the monomial (a <= b) of the 2-factor geometry in lexicographic order
+__host__ __device__ constexpr int mono_idx2(int a, int b) { return a * (25 - a) / 2 + (b - a); }
+
 struct Plan {
-    size_t b3;    // bf16 [BH][d+16][64]  rows g < d: Csym[.][g] (K-major over m); row d: zsym; rest 0
-    size_t bq;    // bf16 [BH][64][d]     Csym[m][.]
+    size_t b3;    // bf16 [BH][d+16][kPad]  rows g < d: Csym[.][g] (K-major over m); row d: zsym; rest 0
+    size_t bq;    // bf16 [BH][kPad][d]     Csym[m][.]
     size_t bd3;   // the same two operands of the gradient state (dCsym | dzsym)
     size_t bdq;
     size_t end;
 };
 
-inline bool supported(bool bf16, int d, int F, int dphi) { return bf16 && (d == 64 || d == 128) && F == 3 && dphi == 6; }
+inline bool supported(bool bf16, int d, int F, int dphi) { return bf16 && (d == 64 || d == 128) && ((F == 3 && dphi == 6) || (F == 2 && dphi == 12)); }
+inline int n_mono(int F) { return F == 3 ? MT<3>::kN : MT<2>::kN; }
+inline int mono_pad(int F) { return F == 3 ? MT<3>::kPad : MT<2>::kPad; }
 
 inline size_t plan(Plan& p, const Dims& D, int BH, size_t off) {
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-    const size_t n3 = (size_t)BH * (D.d + 16) * kMonoPad * 2, nq = (size_t)BH * kMonoPad * D.d * 2;
+    const int pad = mono_pad(D.F);
+    const size_t n3 = (size_t)BH * (D.d + 16) * pad * 2, nq = (size_t)BH * pad * D.d * 2;
     p.b3 = off; off = up(off + n3);
     p.bq = off; off = up(off + nq);
     p.bd3 = off; off = up(off + n3);
@@ -189,6 +202,34 @@ __device__ __forceinline__ void store6(float* dst, const float* v) {
     d[0] = make_float2(v[0], v[1]); d[1] = make_float2(v[2], v[3]); d[2] = make_float2(v[4], v[5]);
 }
 
+// d_phi consecutive fp32 features of one token
+template <int DP> __device__ __forceinline__ void load_feat(float* dst, const float* __restrict__ src) {
+    const float2* s = reinterpret_cast<const float2*>(src);
+#pragma unroll
+    for (int i = 0; i < DP / 2; ++i) {
+        const float2 a = __ldg(s + i);
+        dst[2 * i] = a.x;
+        dst[2 * i + 1] = a.y;
+    }
+}
+template <int DP> __device__ __forceinline__ void store_feat(float* dst, const float* v) {
+    float2* d = reinterpret_cast<float2*>(dst);
+#pragma unroll
+    for (int i = 0; i < DP / 2; ++i) d[i] = make_float2(v[2 * i], v[2 * i + 1]);
+}
+
+// One operand row of kPad bf16 (kN values * scale, then zeros) into row `row` of a tile of kBlocks swizzled 128-row blocks.
+template <int F> __device__ __forceinline__ void store_mono_row_t(uint32_t tile, uint32_t row, const float (&m)[MT<F>::kN], float scale) {
+    constexpr int N = MT<F>::kN;
+#pragma unroll
+    for (int c = 0; c < MT<F>::kPad / 8; ++c) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = 8 * c + e < N ? m[8 * c + e < N ? 8 * c + e : 0] * scale : 0.f;
+        st_shared_v4(tile + (c >> 3) * kBlk + sw128_off(row, c & 7), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+    }
+}
+
 // One operand row of 64 bf16 (56 values * scale, 8 zeros) into row `row` of a swizzled 128-row block.
 __device__ __forceinline__ void store_mono_row(uint32_t blk, uint32_t row, const float (&m)[kMono], float scale) {
 #pragma unroll
@@ -286,28 +327,91 @@ __device__ __forceinline__ void key_folded_grad(const float (&k)[18], const floa
         }
 }
 
+// ---- the same generators for either geometry -----------------------------------------------------------------------------
+template <int F> __device__ __forceinline__ void query_monomials_t(const float (&q)[MT<F>::kDphi], float (&mono)[MT<F>::kN]) {
+    if constexpr (F == 3) {
+        query_monomials(q, mono);
+    } else {
+#pragma unroll
+        for (int a = 0; a < 12; ++a)
+#pragma unroll
+            for (int b = a; b < 12; ++b) mono[mono_idx2(a, b)] = q[a] * q[b];
+    }
+}
+// dq[x] = sum_m dmono[m] d(monomial m) / dq_x
+template <int F> __device__ __forceinline__ void query_monomials_grad_t(const float (&q)[MT<F>::kDphi], const float (&dm)[MT<F>::kN], float (&dq)[MT<F>::kDphi]) {
+    if constexpr (F == 3) {
+        query_monomials_grad(q, dm, dq);
+    } else {
+#pragma unroll
+        for (int a = 0; a < 12; ++a) dq[a] = 0.f;
+#pragma unroll
+        for (int a = 0; a < 12; ++a)
+#pragma unroll
+            for (int b = a; b < 12; ++b) {
+                const float g = dm[mono_idx2(a, b)];
+                dq[a] = fmaf(g, q[b], dq[a]);
+                dq[b] = fmaf(g, q[a], dq[b]);
+            }
+    }
+}
+// Folded key features.  F = 2: k = (k1[0..11], k2[0..11]), ts[(a <= b)] = k1[a] k2[b] + k1[b] k2[a]  (a < b),  k1[a] k2[a]  (a == b).
+template <int F> __device__ __forceinline__ void key_folded_t(const float (&k)[MT<F>::kKf], float (&ts)[MT<F>::kN]) {
+    if constexpr (F == 3) {
+        key_folded(k, ts);
+    } else {
+#pragma unroll
+        for (int a = 0; a < 12; ++a)
+#pragma unroll
+            for (int b = a; b < 12; ++b) ts[mono_idx2(a, b)] = a == b ? k[a] * k[12 + a] : fmaf(k[a], k[12 + b], k[b] * k[12 + a]);
+    }
+}
+// Gradients of L = sum_{x,y} G[sort(x,y)] k1[x] k2[y] (F = 2) with respect to k1, k2.
+template <int F> __device__ __forceinline__ void key_folded_grad_t(const float (&k)[MT<F>::kKf], const float (&G)[MT<F>::kN], float (&dk)[MT<F>::kKf]) {
+    if constexpr (F == 3) {
+        key_folded_grad(k, G, dk);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 24; ++i) dk[i] = 0.f;
+#pragma unroll
+        for (int x = 0; x < 12; ++x)
+#pragma unroll
+            for (int y = 0; y < 12; ++y) {
+                const float g = G[mono_idx2(x < y ? x : y, x < y ? y : x)];
+                dk[x] = fmaf(g, k[12 + y], dk[x]);
+                dk[12 + y] = fmaf(g, k[x], dk[12 + y]);
+            }
+    }
+}
+
 // =======================================================================================
 // State build
 // =======================================================================================
 constexpr int kSbThreads = 320;            // warp 0: TMA, warp 1: MMA, warps 2..9: two generator groups of 128 threads
-constexpr int kSbStages = 4;
-constexpr int kSbStageBytes = 2 * kBlk + kBlk;   // V (two 64-column blocks) + folded key tile (one block)
-constexpr int kSbOffZ = kSbStages * kSbStageBytes;              // zred [8 warps][64] floats
-constexpr int kSbOffBars = kSbOffZ + 8 * 64 * 4;
-constexpr int kSbSmem = 1024 + kSbOffBars + 256;
+template <int F> struct SbCfg {
+    static constexpr int kStages = F == 3 ? 4 : 3;
+    static constexpr int kStageBytes = 2 * kBlk + MT<F>::kBlocks * kBlk;   // V (two 64-column blocks) + folded key tile
+    static constexpr int kOffZ = kStages * kStageBytes;                    // zred [8 warps][kPad] floats
+    static constexpr int kOffBars = kOffZ + 8 * MT<F>::kPad * 4;
+    static constexpr int kSmem = 1024 + kOffBars + 256;
+    static constexpr int kTmemCols = F == 3 ? 64 : 128;
+};
 
-template <int DV>
+template <int DV, int F>
 __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __grid_constant__ CUtensorMap mapV, const float* __restrict__ kf,
                                                                        float* __restrict__ part, int N, int S, int ld, int* status) {
+    using M = MT<F>;
+    using Cfg = SbCfg<F>;
+    constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    float* zred = reinterpret_cast<float*>(smem + kSbOffZ);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSbOffBars);
-    uint64_t* full_v = bars;                    // [4]
-    uint64_t* full_t = bars + kSbStages;        // [4]
-    uint64_t* empty = bars + 2 * kSbStages;     // [4]
-    uint64_t* acc_done = bars + 3 * kSbStages;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSbStages + 1);
+    float* zred = reinterpret_cast<float*>(smem + Cfg::kOffZ);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
+    uint64_t* full_v = bars;                  // [stages]
+    uint64_t* full_t = bars + kStages;        // [stages]
+    uint64_t* empty = bars + 2 * kStages;     // [stages]
+    uint64_t* acc_done = bars + 3 * kStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kStages + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int s = blockIdx.x, bh = blockIdx.y;
@@ -315,23 +419,23 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     const int tiles_per = (tiles + S - 1) / S;
     const int tile0 = s * tiles_per;
     const int ntiles = max(0, min(tiles, tile0 + tiles_per) - tile0);
-    float* out = part + ((size_t)bh * S + s) * kMono * ld;
+    float* out = part + ((size_t)bh * S + s) * M::kN * ld;
 
     grid_launch_dependents();
     if (ntiles == 0) {   // an empty split contributes zeros
         grid_dependency_wait();
-        for (int i = tid; i < kMono * ld; i += kSbThreads) out[i] = 0.f;
+        for (int i = tid; i < M::kN * ld; i += kSbThreads) out[i] = 0.f;
         return;
     }
     if (DV == 64) {      // rows 64..127 of the MMA's M dimension read a second V block: keep it zero
-        for (int st = 0; st < kSbStages; ++st) {
-            uint4* vz = reinterpret_cast<uint4*>(smem + st * kSbStageBytes + kBlk);
+        for (int st = 0; st < kStages; ++st) {
+            uint4* vz = reinterpret_cast<uint4*>(smem + st * kStageBytes + kBlk);
             for (int i = tid; i < kBlk / 16; i += kSbThreads) vz[i] = make_uint4(0, 0, 0, 0);
         }
         fence_proxy_async();
     }
     if (tid == 0) {
-        for (int i = 0; i < kSbStages; ++i) {
+        for (int i = 0; i < kStages; ++i) {
             mbar_init(&full_v[i], 1);
             mbar_init(&full_t[i], 128);
             mbar_init(&empty[i], 1);
@@ -341,7 +445,7 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
         prefetch_tmap(&mapV);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, 64);
+        tmem_alloc(tmem_slot, Cfg::kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -354,21 +458,21 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     if (warp == 0) {
         if (lane == 0) {
             for (int it = 0; it < ntiles; ++it) {
-                const int st = it % kSbStages, u = it / kSbStages;
+                const int st = it % kStages, u = it / kStages;
                 if (!mbar_wait(&empty[st], (u & 1) ^ 1)) { report_timeout(status, 101); break; }
-                uint8_t* vs = smem + st * kSbStageBytes;
+                uint8_t* vs = smem + st * kStageBytes;
                 mbar_arrive_expect_tx(&full_v[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b) tma_load_3d(vs + b * kBlk, &mapV, &full_v[st], b * 64, (tile0 + it) * kTileTokens, bh);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = idesc_bf16(128, kMonoPad, true, true);
+            const uint32_t idesc = idesc_bf16(128, M::kPad, true, true);
             for (int it = 0; it < ntiles; ++it) {
-                const int st = it % kSbStages, u = it / kSbStages;
+                const int st = it % kStages, u = it / kStages;
                 if (!(mbar_wait(&full_v[st], u & 1) && mbar_wait(&full_t[st], u & 1))) { report_timeout(status, 102); break; }
                 tc_fence_after();
-                const uint32_t va = smem_u32(smem + st * kSbStageBytes), ta = va + 2 * kBlk;
+                const uint32_t va = smem_u32(smem + st * kStageBytes), ta = va + 2 * kBlk;
 #pragma unroll
                 for (int ks = 0; ks < kTileTokens / 16; ++ks)
                     umma_bf16(tmem, smem_desc_sw128(va + ks * 2048, kBlk, 1024), smem_desc_sw128(ta + ks * 2048, kBlk, 1024), idesc,
@@ -380,47 +484,47 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
     } else {
         const int grp = (warp - 2) >> 2;
         const int row = ((warp - 2) & 3) * 32 + lane;
-        float zacc[kMono];
+        float zacc[M::kN];
 #pragma unroll
-        for (int i = 0; i < kMono; ++i) zacc[i] = 0.f;
+        for (int i = 0; i < M::kN; ++i) zacc[i] = 0.f;
         // The key features of the group's next tile are loaded while the current one is processed (row index clamped:
         // the loads are unconditional, out-of-range rows are zeroed when used).
-        float k[18], kn[18];
+        float k[M::kKf], kn[M::kKf];
         auto prefetch = [&](int it) {
             const int tok = min((tile0 + it) * kTileTokens + row, N - 1);
 #pragma unroll
-            for (int f = 0; f < 3; ++f) load6(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+            for (int f = 0; f < F; ++f) load_feat<M::kDphi>(kn + M::kDphi * f, kf + (((size_t)bh * F + f) * N + tok) * M::kDphi);
         };
         if (grp < ntiles) prefetch(grp);
         for (int it = grp; it < ntiles; it += 2) {
-            const int st = it % kSbStages, u = it / kSbStages;
+            const int st = it % kStages, u = it / kStages;
             const int tok = (tile0 + it) * kTileTokens + row;
 #pragma unroll
-            for (int i = 0; i < 18; ++i) k[i] = tok < N ? kn[i] : 0.f;
+            for (int i = 0; i < M::kKf; ++i) k[i] = tok < N ? kn[i] : 0.f;
             if (it + 2 < ntiles) prefetch(it + 2);
-            float ts[kMono];
-            key_folded(k, ts);
+            float ts[M::kN];
+            key_folded_t<F>(k, ts);
 #pragma unroll
-            for (int i = 0; i < kMono; ++i) zacc[i] += ts[i];
+            for (int i = 0; i < M::kN; ++i) zacc[i] += ts[i];
             if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 103); }
             if (ok) {
-                store_mono_row(smem_u32(smem + st * kSbStageBytes + 2 * kBlk), row, ts, 1.f);
+                store_mono_row_t<F>(smem_u32(smem + st * kStageBytes + 2 * kBlk), row, ts, 1.f);
                 fence_proxy_async();
                 mbar_arrive(&full_t[st]);
             }
         }
         // zsym: sum the per-token-slot accumulators over the 256 generator threads
 #pragma unroll
-        for (int i = 0; i < kMono; ++i) {
+        for (int i = 0; i < M::kN; ++i) {
             const float v = warp_sum(zacc[i]);
-            if (lane == 0) zred[(warp - 2) * 64 + i] = v;
+            if (lane == 0) zred[(warp - 2) * M::kPad + i] = v;
         }
         named_barrier(1, 256);
         const int gi = tid - 64;
-        if (gi < kMono) {
+        if (gi < M::kN) {
             float z = 0.f;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) z += zred[w * 64 + gi];
+            for (int w = 0; w < 8; ++w) z += zred[w * M::kPad + gi];
             out[(size_t)gi * ld + DV] = z;
             for (int c = DV + 1; c < ld; ++c) out[(size_t)gi * ld + c] = 0.f;
         }
@@ -432,19 +536,20 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
             const int g = quarter * 32 + lane;
             if (ok && quarter * 32 < DV) {
 #pragma unroll
-                for (int c = 0; c < kMono / 8; ++c) {
+                for (int c = 0; c < M::kPad / 8; ++c) {
                     uint32_t r[8];
                     tmem_ld8(tmem + ((uint32_t)(quarter * 32) << 16) + 8 * c, r);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) out[(size_t)(8 * c + e) * ld + g] = __uint_as_float(r[e]);
+                    for (int e = 0; e < 8; ++e)
+                        if (8 * c + e < M::kN) out[(size_t)(8 * c + e) * ld + g] = __uint_as_float(r[e]);
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, 64);
+    if (warp == 1) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
 // =======================================================================================
@@ -457,14 +562,15 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
 // the head's slots are its pieces, one per CTA that touched it (see owner_of_work).
 __host__ __device__ inline int owner_of_work(long long w, long long total, int G) { return (int)(((w + 1) * G - 1) / total); }
 
-template <int DV>
+template <int DV, int F>
 __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __restrict__ part, float* __restrict__ state,
                                                              __nv_bfloat16* __restrict__ b3, __nv_bfloat16* __restrict__ bq, int S, int ld, int G, int T) {
+    constexpr int kN = MT<F>::kN, kPad = MT<F>::kPad;
     __shared__ float sm[8][kMaxD + 8];
-    const int m0 = 8 * blockIdx.x, bh = blockIdx.y, tid = threadIdx.x;
+    const int m0 = 8 * blockIdx.x, bh = blockIdx.y, tid = threadIdx.x;      // gridDim.x = kPad / 8
     grid_launch_dependents();
     grid_dependency_wait();
-    const size_t n_per = (size_t)kMono * ld;
+    const size_t n_per = (size_t)kN * ld;
     int count = S;
     if (G > 0) {
         const long long total = (long long)gridDim.y * T;
@@ -473,7 +579,7 @@ __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __rest
     for (int i = tid; i < 8 * ld; i += 256) {
         const int mm = i / ld, col = i - mm * ld, m = m0 + mm;
         float a = 0.f;
-        if (m < kMono) {
+        if (m < kN) {
             const float* src = part + (size_t)bh * S * n_per + (size_t)m * ld + col;
             for (int s = 0; s < count; ++s) a += src[(size_t)s * n_per];      // fixed order: bit-reproducible
             state[(size_t)bh * n_per + (size_t)m * ld + col] = a;
@@ -481,14 +587,14 @@ __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __rest
         sm[mm][col] = a;
     }
     __syncthreads();
-    __nv_bfloat16* o3 = b3 + (size_t)bh * (DV + 16) * kMonoPad;
+    __nv_bfloat16* o3 = b3 + (size_t)bh * (DV + 16) * kPad;
     for (int row = tid; row < DV + 16; row += 256) {       // row <= DV: column `row` of the state (row == DV is z); rest zero
         uint32_t w[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) w[e] = row <= DV ? pack_bf16(sm[2 * e][row], sm[2 * e + 1][row]) : 0u;
-        *reinterpret_cast<uint4*>(o3 + (size_t)row * kMonoPad + m0) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(o3 + (size_t)row * kPad + m0) = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    __nv_bfloat16* oq = bq + (size_t)bh * kMonoPad * DV;
+    __nv_bfloat16* oq = bq + (size_t)bh * kPad * DV;
     for (int i = tid; i < 8 * DV; i += 256) {
         const int mm = i / DV, g = i - mm * DV;
         oq[(size_t)(m0 + mm) * DV + g] = __float2bfloat16_rn(sm[mm][g]);
@@ -502,23 +608,26 @@ __global__ void __launch_bounds__(256) tc_reduce_emit_kernel(const float* __rest
 // the tile rate), warps 8..11: monomial generators, warp 12: TMA + MMA
 constexpr int kRoThreads = 416;
 constexpr int kRoGenWarp0 = 8, kRoMmaWarp = 12;
-template <int DV> struct RoCfg {
+template <int DV, int F> struct RoCfg {
     static constexpr int kNmma = DV + 16;
-    static constexpr int kB3Bytes = kNmma * 128;
+    static constexpr int kABytes = MT<F>::kBlocks * kBlk;                       // one monomial tile
+    static constexpr int kB3Block = ((kNmma * 128 + 1023) / 1024) * 1024;       // one 64-monomial block of the state operand: [kNmma rows][128 B]
+    static constexpr int kB3Bytes = MT<F>::kBlocks * kNmma * 128;               // bytes the TMA loads deliver
     static constexpr int kOBytes = kTileTokens * DV * 2;
-    static constexpr int kOffA = 0;                       // 2 x 16 KB monomial tiles
-    static constexpr int kOffB3 = 2 * kBlk;
-    static constexpr int kOffO = kOffB3 + ((kB3Bytes + 1023) / 1024) * 1024;   // 2 staging tiles
+    static constexpr int kOffA = 0;                       // 2 monomial tiles
+    static constexpr int kOffB3 = 2 * kABytes;
+    static constexpr int kOffO = kOffB3 + MT<F>::kBlocks * kB3Block;   // 2 staging tiles
     static constexpr int kOffBars = kOffO + 2 * kOBytes;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (it owns all of TMEM)
 };
 
-template <int DV>
+template <int DV, int F>
 __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_constant__ CUtensorMap mapB3, const __grid_constant__ CUtensorMap mapO,
                                                                    const float* __restrict__ qf, float* __restrict__ eta_out, int N, int BH,
                                                                    float eps, int* status) {
-    using Cfg = RoCfg<DV>;
+    using Cfg = RoCfg<DV, F>;
+    using M = MT<F>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
@@ -577,42 +686,42 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
                         if (!mbar_wait(b3_free, (nload - 1) & 1)) { report_timeout(status, 201); break; }
                     }
                     mbar_arrive_expect_tx(b3_full, Cfg::kB3Bytes);
-                    tma_load_2d(smem + Cfg::kOffB3, &mapB3, b3_full, 0, bh * Cfg::kNmma);
+                    for (int b = 0; b < M::kBlocks; ++b) tma_load_2d(smem + Cfg::kOffB3 + b * Cfg::kB3Block, &mapB3, b3_full, b * 64, bh * Cfg::kNmma);
                     if (!mbar_wait(b3_full, nload & 1)) { report_timeout(status, 202); break; }
                     ++nload;
                     cur_bh = bh;
                 }
                 if (!(mbar_wait(&a_full[ab], u & 1) && mbar_wait(&acc_empty[ab], (u & 1) ^ 1))) { report_timeout(status, 203); break; }
                 tc_fence_after();
-                const uint32_t aa = smem_u32(smem + Cfg::kOffA + ab * kBlk);
+                const uint32_t aa = smem_u32(smem + Cfg::kOffA + ab * Cfg::kABytes);
 #pragma unroll
-                for (int ks = 0; ks < kMonoPad / 16; ++ks)
-                    umma_bf16(tmem + ab * 256, smem_desc_sw128(aa + ks * 32, 16, 1024), smem_desc_sw128(b3a + ks * 32, 16, 1024), idesc,
-                              ks > 0 ? 1u : 0u);
+                for (int ks = 0; ks < M::kPad / 16; ++ks)
+                    umma_bf16(tmem + ab * 256, smem_desc_sw128(aa + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                              smem_desc_sw128(b3a + (ks >> 2) * Cfg::kB3Block + (ks & 3) * 32, 16, 1024), idesc, ks > 0 ? 1u : 0u);
                 umma_commit(&a_empty[ab]);
                 umma_commit(&acc_full[ab]);
             }
         }
     } else if (warp >= kRoGenWarp0) {
         const int row = tid - kRoGenWarp0 * 32;
-        float qn[6];      // query features of the next tile, loaded one tile ahead (row index clamped)
+        float qn[M::kDphi];      // query features of the next tile, loaded one tile ahead (row index clamped)
         auto prefetch = [&](int it) {
             const int work = w0 + it, bh = work / tiles_per_head, tok = min((work % tiles_per_head) * kTileTokens + row, N - 1);
-            load6(qn, qf + ((size_t)bh * N + tok) * 6);
+            load_feat<M::kDphi>(qn, qf + ((size_t)bh * N + tok) * M::kDphi);
         };
         if (nwork > 0) prefetch(0);
         for (int it = 0; it < nwork; ++it) {
             const int work = w0 + it, tok = (work % tiles_per_head) * kTileTokens + row;
             const int ab = it & 1, u = it >> 1;
-            float q[6];
+            float q[M::kDphi];
 #pragma unroll
-            for (int i = 0; i < 6; ++i) q[i] = tok < N ? qn[i] : 0.f;
+            for (int i = 0; i < M::kDphi; ++i) q[i] = tok < N ? qn[i] : 0.f;
             if (it + 1 < nwork) prefetch(it + 1);
-            float mono[kMono];
-            query_monomials(q, mono);
+            float mono[M::kN];
+            query_monomials_t<F>(q, mono);
             if (ok && !mbar_wait(&a_empty[ab], (u & 1) ^ 1)) { ok = false; report_timeout(status, 204); }
             if (!ok) continue;
-            store_mono_row(smem_u32(smem + Cfg::kOffA + ab * kBlk), row, mono, 1.f);
+            store_mono_row_t<F>(smem_u32(smem + Cfg::kOffA + ab * Cfg::kABytes), row, mono, 1.f);
             fence_proxy_async();
             mbar_arrive(&a_full[ab]);
         }
@@ -687,34 +796,44 @@ __global__ void __launch_bounds__(kRoThreads, 1) tc_readout_kernel(const __grid_
 // =======================================================================================
 constexpr int kBqGroups = 3;                            // generator groups of 128 threads; tile `it` belongs to group it % 3
 constexpr int kBqThreads = 128 + 128 * kBqGroups;       // warp 0: TMA, warp 1: D2 MMAs, warp 2: dC MMAs, warp 3 idle, warps 4..: generators
-constexpr int kBqStages = 4;
-constexpr int kBqStageBytes = 3 * kBlk;                 // dO tile (d/64 blocks of 64 columns) directly followed by the operand-row tile
-constexpr int kBqOffOp = kBqStages * kBqStageBytes;     // Csym operand [64][d] bf16 (two 8 KB blocks)
-constexpr int kBqOffZ = kBqOffOp + kBlk;                // zsym (64 floats)
-constexpr int kBqOffBars = kBqOffZ + 64 * 4;
-constexpr int kBqSmem = 1024 + kBqOffBars + 256;
-constexpr int kBqColD2 = 256;                           // TMEM columns of the D2 buffers (one per group, 64 columns each)
 constexpr int kBqRowPad = 8;                            // accumulator row of monomial 0
+// F = 2: the operand row is [deta/r, 0 x 7, r mono_0..77, 0 x 42] = 128 columns in two blocks, the dC product has M = 128
+// (accumulator lane = row) and three stages fit; F = 3: 64 columns, M = 64 (row R in lane 32 (R / 16) + R % 16), four stages.
+template <int F> struct BqCfg {
+    static constexpr int kStages = F == 3 ? 4 : 3;
+    static constexpr int kStageBytes = (2 + MT<F>::kBlocks) * kBlk;      // dO tile (d/64 blocks of 64 columns) directly followed by the operand-row tile
+    static constexpr int kOpBlock = MT<F>::kPad * 128;                   // Csym operand [kPad][d] bf16: one block per 64 value channels
+    static constexpr int kOffOp = kStages * kStageBytes;
+    static constexpr int kOffZ = kOffOp + ((2 * kOpBlock + 1023) / 1024) * 1024;      // zsym (kPad floats)
+    static constexpr int kOffBars = kOffZ + MT<F>::kPad * 4;
+    static constexpr int kSmem = 1024 + kOffBars + 256;
+    static constexpr int kColD2 = F == 3 ? 256 : 160;                    // TMEM columns of the D2 buffers (one per group)
+    static constexpr int kD2Stride = F == 3 ? 64 : 96;
+    static constexpr int kM = F == 3 ? 64 : 128;                         // rows of the dC product
+    static_assert((4 * kStages + 2 * kBqGroups + 3) * 8 <= 256, "barrier block");
+};
 
-template <int DV>
+template <int DV, int F>
 __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __grid_constant__ CUtensorMap mapdO, const __grid_constant__ CUtensorMap mapBq,
                                                                      const float* __restrict__ qf, const float* __restrict__ eta,
                                                                      const float* __restrict__ state, float* __restrict__ dqf,
                                                                      float* __restrict__ part, int N, int S, int ld, float eps, int* status) {
+    using M = MT<F>;
+    using Cfg = BqCfg<F>;
+    constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    float* zsym = reinterpret_cast<float*>(smem + kBqOffZ);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBqOffBars);
-    uint64_t* full_do = bars;                       // [stages] TMA
-    uint64_t* full_rm = bars + kBqStages;           // [stages] 128 arrivals: the operand rows of the tile are complete
-    uint64_t* empty_rm = bars + 2 * kBqStages;      // [stages] MMA commit (dC): the operand-row tile is free
-    uint64_t* empty_do = bars + 3 * kBqStages;      // [stages] MMA commits (D2 and dC): the dO tile is free
-    uint64_t* d2_full = bars + 4 * kBqStages;       // [groups] MMA commit
-    uint64_t* d2_empty = d2_full + kBqGroups;       // [groups] 128 arrivals
+    float* zsym = reinterpret_cast<float*>(smem + Cfg::kOffZ);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
+    uint64_t* full_do = bars;                     // [stages] TMA
+    uint64_t* full_rm = bars + kStages;           // [stages] 128 arrivals: the operand rows of the tile are complete
+    uint64_t* empty_rm = bars + 2 * kStages;      // [stages] MMA commit (dC): the operand-row tile is free
+    uint64_t* empty_do = bars + 3 * kStages;      // [stages] MMA commits (D2 and dC): the dO tile is free
+    uint64_t* d2_full = bars + 4 * kStages;       // [groups] MMA commit
+    uint64_t* d2_empty = d2_full + kBqGroups;     // [groups] 128 arrivals
     uint64_t* op_full = d2_empty + kBqGroups;
     uint64_t* acc_done = op_full + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
-    static_assert((4 * kBqStages + 2 * kBqGroups + 3) * 8 <= 256, "barrier block");
     constexpr int kRmOff = (DV / 64) * kBlk;        // operand-row tile inside a stage
     constexpr int kNC = DV + 8;                     // columns of the dC product
 
@@ -724,15 +843,22 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
     const int tiles_per = (tiles + S - 1) / S;
     const int tile0 = s * tiles_per;
     const int ntiles = max(0, min(tiles, tile0 + tiles_per) - tile0);
-    float* out = part + ((size_t)bh * S + s) * kMono * ld;
+    float* out = part + ((size_t)bh * S + s) * M::kN * ld;
     grid_launch_dependents();
     if (ntiles == 0) {
         grid_dependency_wait();
-        for (int i = tid; i < kMono * ld; i += kBqThreads) out[i] = 0.f;
+        for (int i = tid; i < M::kN * ld; i += kBqThreads) out[i] = 0.f;
         return;
     }
+    if (F == 2) {      // operand-row columns 86..127 are read by the M = 128 product and never written: keep them zero
+        for (int st = 0; st < kStages; ++st) {
+            uint4* z = reinterpret_cast<uint4*>(smem + st * kStageBytes + kRmOff + kBlk);
+            for (int i = tid; i < kBlk / 16; i += kBqThreads) z[i] = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async();
+    }
     if (tid == 0) {
-        for (int i = 0; i < kBqStages; ++i) {
+        for (int i = 0; i < kStages; ++i) {
             mbar_init(&full_do[i], 1);
             mbar_init(&full_rm[i], 128);
             mbar_init(&empty_rm[i], 1);
@@ -759,19 +885,19 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
     grid_dependency_wait();
     // (zsym is read by the generator warps only; the named barrier keeps the other warps out of it)
     if (warp >= 4) {
-        if (tid - 128 < 64) zsym[tid - 128] = tid - 128 < kMono ? state[((size_t)bh * kMono + tid - 128) * ld + DV] : 0.f;
+        if (tid - 128 < M::kPad) zsym[tid - 128] = tid - 128 < M::kN ? state[((size_t)bh * M::kN + tid - 128) * ld + DV] : 0.f;
         named_barrier(1, 128 * kBqGroups);
     }
     bool ok = true;
 
     if (warp == 0) {
         if (elect_one()) {
-            mbar_arrive_expect_tx(op_full, kMonoPad * DV * 2);
-            for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + kBqOffOp + b * (kBlk / 2), &mapBq, op_full, b * 64, bh * kMonoPad);
+            mbar_arrive_expect_tx(op_full, M::kPad * DV * 2);
+            for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + Cfg::kOffOp + b * Cfg::kOpBlock, &mapBq, op_full, b * 64, bh * M::kPad);
             for (int it = 0; it < ntiles; ++it) {
-                const int st = it % kBqStages, u = it / kBqStages;
+                const int st = it % kStages, u = it / kStages;
                 if (!mbar_wait(&empty_do[st], (u & 1) ^ 1)) { report_timeout(status, 301); break; }
-                uint8_t* ds = smem + st * kBqStageBytes;
+                uint8_t* ds = smem + st * kStageBytes;
                 mbar_arrive_expect_tx(&full_do[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b) tma_load_3d(ds + b * kBlk, &mapdO, &full_do[st], b * 64, (tile0 + it) * kTileTokens, bh);
             }
@@ -780,32 +906,32 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
         if (elect_one()) {
             // D2 = dO (K-major over g) * Csym (K-major over g); tile `it` is issued as soon as its dO tile has landed
             // and the group that owns the tile has read its previous D2, which is long before the group asks for it.
-            const uint32_t idesc2 = idesc_bf16(128, kMonoPad, false, false);
-            const uint32_t opa = smem_u32(smem + kBqOffOp);
+            const uint32_t idesc2 = idesc_bf16(128, M::kPad, false, false);
+            const uint32_t opa = smem_u32(smem + Cfg::kOffOp);
             if (!mbar_wait(op_full, 0)) report_timeout(status, 302);
             else
                 for (int it = 0; it < ntiles; ++it) {
-                    const int st = it % kBqStages, u = it / kBqStages, buf = it % kBqGroups, ub = it / kBqGroups;
+                    const int st = it % kStages, u = it / kStages, buf = it % kBqGroups, ub = it / kBqGroups;
                     if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&d2_empty[buf], (ub & 1) ^ 1))) { report_timeout(status, 303); break; }
                     tc_fence_after();
-                    const uint32_t da = smem_u32(smem + st * kBqStageBytes);
+                    const uint32_t da = smem_u32(smem + st * kStageBytes);
 #pragma unroll
                     for (int ks = 0; ks < DV / 16; ++ks)
-                        umma_bf16(tmem + kBqColD2 + 64 * buf, smem_desc_sw128(da + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                                  smem_desc_sw128(opa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
+                        umma_bf16(tmem + Cfg::kColD2 + Cfg::kD2Stride * buf, smem_desc_sw128(da + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                                  smem_desc_sw128(opa + (ks >> 2) * Cfg::kOpBlock + (ks & 3) * 32, 16, 1024), idesc2, ks > 0 ? 1u : 0u);
                     umma_commit(&d2_full[buf]);
                     umma_commit(&empty_do[st]);
                 }
         }
     } else if (warp == 2) {
         if (elect_one()) {
-            // [dCsym | dzsym] += (operand rows)^T (MN-major, M = 64) * [dO | operand rows' first 8 columns] (MN-major, N = d + 8)
-            const uint32_t idesc1 = idesc_bf16(64, kNC, true, true);
+            // [dCsym | dzsym] += (operand rows)^T (MN-major, M rows) * [dO | operand rows' first 8 columns] (MN-major, N = d + 8)
+            const uint32_t idesc1 = idesc_bf16(Cfg::kM, kNC, true, true);
             for (int it = 0; it < ntiles; ++it) {
-                const int st = it % kBqStages, u = it / kBqStages;
+                const int st = it % kStages, u = it / kStages;
                 if (!(mbar_wait(&full_do[st], u & 1) && mbar_wait(&full_rm[st], u & 1))) { report_timeout(status, 304); break; }
                 tc_fence_after();
-                const uint32_t da = smem_u32(smem + st * kBqStageBytes), ra = da + kRmOff;
+                const uint32_t da = smem_u32(smem + st * kStageBytes), ra = da + kRmOff;
 #pragma unroll
                 for (int ks = 0; ks < kTileTokens / 16; ++ks)
                     umma_bf16(tmem, smem_desc_sw128(ra + ks * 2048, kBlk, 1024), smem_desc_sw128(da + ks * 2048, kBlk, 1024), idesc1,
@@ -820,104 +946,149 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
         const int row = quarter * 32 + lane;    // token row of the tile == TMEM lane this thread can read
         // The features and the normaliser of the group's next tile are loaded while the current one is processed
         // (row index clamped: the loads are unconditional, out-of-range rows are zeroed when used).
-        float qn[6], etan;
+        float qn[M::kDphi], etan;
         auto prefetch = [&](int it) {
             const int tok = min((tile0 + it) * kTileTokens + row, N - 1);
-            load6(qn, qf + ((size_t)bh * N + tok) * 6);
+            load_feat<M::kDphi>(qn, qf + ((size_t)bh * N + tok) * M::kDphi);
             etan = __ldg(eta + (size_t)bh * N + tok);
         };
         if (grp < ntiles) prefetch(grp);
         for (int it = grp; it < ntiles; it += kBqGroups) {
-            const int st = it % kBqStages, u = it / kBqStages, buf = grp, ub = it / kBqGroups;
+            const int st = it % kStages, u = it / kStages, buf = grp, ub = it / kBqGroups;
             const int tok = (tile0 + it) * kTileTokens + row;
-            const uint32_t rblk = smem_u32(smem + st * kBqStageBytes + kRmOff);
-            float q[6], r = 0.f;
+            const uint32_t rblk = smem_u32(smem + st * kStageBytes + kRmOff);
+            float q[M::kDphi], r = 0.f;
 #pragma unroll
-            for (int i = 0; i < 6; ++i) q[i] = tok < N ? qn[i] : 0.f;
+            for (int i = 0; i < M::kDphi; ++i) q[i] = tok < N ? qn[i] : 0.f;
             if (tok < N) r = 1.f / (etan + eps);
-            {   // columns 8..63 of the operand row: r_i * mono_i, formed from (r q_a) q_b q_c so that no monomial stays live
+            {   // columns 8.. of the operand row: r_i * mono_i, formed from the scaled features so that no monomial stays live
                 // across the wait below
-                float qs[6], rmono[kMono];
+                float qs[M::kDphi], rmono[M::kN];
 #pragma unroll
-                for (int i = 0; i < 6; ++i) qs[i] = r * q[i];
+                for (int i = 0; i < M::kDphi; ++i) qs[i] = r * q[i];
+                if constexpr (F == 3) {
 #pragma unroll
-                for (int a = 0; a < 6; ++a)
+                    for (int a = 0; a < 6; ++a)
 #pragma unroll
-                    for (int b = a; b < 6; ++b) {
-                        const float qab = qs[a] * q[b];
+                        for (int b = a; b < 6; ++b) {
+                            const float qab = qs[a] * q[b];
 #pragma unroll
-                        for (int c = b; c < 6; ++c) rmono[mono_idx(a, b, c)] = qab * q[c];
-                    }
+                            for (int c = b; c < 6; ++c) rmono[mono_idx(a, b, c)] = qab * q[c];
+                        }
+                } else {
+#pragma unroll
+                    for (int a = 0; a < 12; ++a)
+#pragma unroll
+                        for (int b = a; b < 12; ++b) rmono[mono_idx2(a, b)] = qs[a] * q[b];
+                }
                 if (ok && !mbar_wait(&empty_rm[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 305); }
                 if (ok) {
 #pragma unroll
-                    for (int c = 0; c < 7; ++c)
-                        st_shared_v4(rblk + sw128_off(row, c + 1), pack_bf16(rmono[8 * c], rmono[8 * c + 1]), pack_bf16(rmono[8 * c + 2], rmono[8 * c + 3]),
-                                     pack_bf16(rmono[8 * c + 4], rmono[8 * c + 5]), pack_bf16(rmono[8 * c + 6], rmono[8 * c + 7]));
+                    for (int c = 1; c < (kBqRowPad + M::kN + 7) / 8; ++c) {      // 16-byte chunk c holds the monomials 8 c - 8 .. 8 c - 1
+                        float v[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) v[e] = 8 * c - 8 + e < M::kN ? rmono[8 * c - 8 + e < M::kN ? 8 * c - 8 + e : 0] : 0.f;
+                        st_shared_v4(rblk + (c >> 3) * kBlk + sw128_off(row, c & 7), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
+                                     pack_bf16(v[6], v[7]));
+                    }
                 }
             }
             if (ok && !mbar_wait(&d2_full[buf], ub & 1)) { ok = false; report_timeout(status, 306); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) continue;
             tc_fence_after();
-            uint32_t d2[kMono];
-            const uint32_t ta = tmem + kBqColD2 + 64 * buf + ((uint32_t)(quarter * 32) << 16);
+            constexpr int kD2Chunks = (M::kN + 7) / 8;
+            uint32_t d2[8 * kD2Chunks];
+            const uint32_t ta = tmem + Cfg::kColD2 + Cfg::kD2Stride * buf + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
-            for (int c = 0; c < kMono / 8; ++c) tmem_ld8(ta + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(d2 + 8 * c));
+            for (int c = 0; c < kD2Chunks; ++c) tmem_ld8(ta + 8 * c, *reinterpret_cast<uint32_t(*)[8]>(d2 + 8 * c));
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(&d2_empty[buf]);
-            // The monomials are recomputed where they are used (two multiplies each) instead of being kept in 56 registers.
-            float qq[6][6];
+            float dq[M::kDphi];
+            float sdot, deta;
+            if constexpr (F == 3) {
+                // The monomials are recomputed where they are used (two multiplies each) instead of being kept in 56 registers.
+                float qq[6][6];
 #pragma unroll
-            for (int a = 0; a < 6; ++a)
+                for (int a = 0; a < 6; ++a)
 #pragma unroll
-                for (int b = a; b < 6; ++b) qq[a][b] = q[a] * q[b];
-            float sd[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int b = a; b < 6; ++b) qq[a][b] = q[a] * q[b];
+                float sd[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int a = 0; a < 6; ++a)
+                for (int a = 0; a < 6; ++a)
 #pragma unroll
-                for (int b = a; b < 6; ++b)
+                    for (int b = a; b < 6; ++b)
 #pragma unroll
-                    for (int c = b; c < 6; ++c) {
-                        const int m = mono_idx(a, b, c);
-                        sd[m & 3] = fmaf(qq[a][b] * q[c], __uint_as_float(d2[m]), sd[m & 3]);
+                        for (int c = b; c < 6; ++c) {
+                            const int m = mono_idx(a, b, c);
+                            sd[m & 3] = fmaf(qq[a][b] * q[c], __uint_as_float(d2[m]), sd[m & 3]);
+                        }
+                sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
+                deta = -r * r * sdot;
+                // columns 0..7 of the operand row: deta / r, then zeros; one proxy fence covers the whole row
+                st_shared_v4(rblk + sw128_off(row, 0), pack_bf16(-r * sdot, 0.f), 0u, 0u, 0u);
+                fence_proxy_async();
+                mbar_arrive(&full_rm[st]);
+                if (it + kBqGroups < ntiles) prefetch(it + kBqGroups);
+#pragma unroll
+                for (int a = 0; a < 6; ++a) dq[a] = 0.f;
+#pragma unroll
+                for (int a = 0; a < 6; ++a)
+#pragma unroll
+                    for (int b = a; b < 6; ++b)
+#pragma unroll
+                        for (int c = b; c < 6; ++c) {
+                            const int m = mono_idx(a, b, c);
+                            const float g = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);      // dmono_i[m]
+                            dq[a] = fmaf(g, qq[b][c], dq[a]);
+                            dq[b] = fmaf(g, qq[a][c], dq[b]);
+                            dq[c] = fmaf(g, qq[a][b], dq[c]);
+                        }
+            } else {
+                float sd[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int a = 0; a < 12; ++a)
+#pragma unroll
+                    for (int b = a; b < 12; ++b) {
+                        const int m = mono_idx2(a, b);
+                        sd[m & 3] = fmaf(q[a] * q[b], __uint_as_float(d2[m]), sd[m & 3]);
                     }
-            const float sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
-            const float deta = -r * r * sdot;
-            // columns 0..7 of the operand row: deta / r, then zeros; one proxy fence covers the whole row
-            st_shared_v4(rblk + sw128_off(row, 0), pack_bf16(-r * sdot, 0.f), 0u, 0u, 0u);
-            fence_proxy_async();
-            mbar_arrive(&full_rm[st]);
-            if (it + kBqGroups < ntiles) prefetch(it + kBqGroups);
-            float dq[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                sdot = (sd[0] + sd[1]) + (sd[2] + sd[3]);
+                deta = -r * r * sdot;
+                st_shared_v4(rblk + sw128_off(row, 0), pack_bf16(-r * sdot, 0.f), 0u, 0u, 0u);
+                fence_proxy_async();
+                mbar_arrive(&full_rm[st]);
+                if (it + kBqGroups < ntiles) prefetch(it + kBqGroups);
 #pragma unroll
-            for (int a = 0; a < 6; ++a)
+                for (int a = 0; a < 12; ++a) dq[a] = 0.f;
 #pragma unroll
-                for (int b = a; b < 6; ++b)
+                for (int a = 0; a < 12; ++a)
 #pragma unroll
-                    for (int c = b; c < 6; ++c) {
-                        const int m = mono_idx(a, b, c);
-                        const float g = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);      // dmono_i[m]
-                        dq[a] = fmaf(g, qq[b][c], dq[a]);
-                        dq[b] = fmaf(g, qq[a][c], dq[b]);
-                        dq[c] = fmaf(g, qq[a][b], dq[c]);
+                    for (int b = a; b < 12; ++b) {
+                        const int m = mono_idx2(a, b);
+                        const float g = fmaf(r, __uint_as_float(d2[m]), deta * zsym[m]);          // dmono_i[m]
+                        dq[a] = fmaf(g, q[b], dq[a]);
+                        dq[b] = fmaf(g, q[a], dq[b]);
                     }
-            if (tok < N) store6(dqf + ((size_t)bh * N + tok) * 6, dq);
+            }
+            if (tok < N) store_feat<M::kDphi>(dqf + ((size_t)bh * N + tok) * M::kDphi, dq);
         }
         if (grp == 0) {
-            // A 64-row accumulator keeps row R in TMEM lane 32 * (R / 16) + R % 16: lanes 0..15 of each warp's quarter.
             if (ok && !mbar_wait(acc_done, 0)) { ok = false; report_timeout(status, 307); }
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
-            const int m = quarter * 16 + lane - kBqRowPad;
+            // F = 3: a 64-row accumulator keeps row R in TMEM lane 32 * (R / 16) + R % 16 (lanes 0..15 of each warp's quarter);
+            // F = 2: a 128-row accumulator keeps row R in lane R
+            const int m = (F == 3 ? quarter * 16 + lane : quarter * 32 + lane) - kBqRowPad;
+            const bool mine = (F == 3 ? lane < 16 : true) && m >= 0 && m < M::kN;
             if (ok) {
 #pragma unroll 1
                 for (int c = 0; c < kNC / 8; ++c) {
                     uint32_t rr[8];
                     tmem_ld8(tmem + ((uint32_t)(quarter * 32) << 16) + 8 * c, rr);
                     tmem_ld_wait();
-                    if (lane < 16 && m >= 0 && m < kMono) {
+                    if (mine) {
                         float4* dst = reinterpret_cast<float4*>(out + (size_t)m * ld + 8 * c);
                         dst[0] = make_float4(__uint_as_float(rr[0]), __uint_as_float(rr[1]), __uint_as_float(rr[2]), __uint_as_float(rr[3]));
                         if (8 * c + 4 < ld) dst[1] = make_float4(__uint_as_float(rr[4]), __uint_as_float(rr[5]), __uint_as_float(rr[6]), __uint_as_float(rr[7]));
@@ -938,26 +1109,35 @@ __global__ void __launch_bounds__(kBqThreads, 1) tc_bwd_query_kernel(const __gri
 //   dk1, dk2, dk3 from G_j and the key features                              (ALUs)
 // =======================================================================================
 constexpr int kBkThreads = 320;   // warp 0: TMA loads, warp 1: MMA, warps 2..9: two worker groups of 128 threads
-template <int DV> struct BkCfg {
+template <int DV, int F> struct BkCfg {
     static constexpr int kVBytes = 2 * kBlk;                              // V stage (two 64-column blocks; d = 64 uses one)
+    static constexpr int kABytes = MT<F>::kBlocks * kBlk;                 // one folded key tile
     static constexpr int kOffV = 0;                                       // 2 stages
     static constexpr int kOffA = 2 * kVBytes;                             // 2 folded key tiles (one per group)
-    static constexpr int kOffB3 = kOffA + 2 * kBlk;                       // dCsym operand [d+16][64]
-    static constexpr int kB3Bytes = (DV + 16) * 128;
-    static constexpr int kOffBq = kOffB3 + ((kB3Bytes + 1023) / 1024) * 1024;   // dCsym operand [64][d]
-    static constexpr int kOffO = kOffBq + kBlk;                           // 2 dV staging tiles (one per group)
+    static constexpr int kOffB3 = kOffA + 2 * kABytes;                    // dCsym operand [d+16][kPad], one block per 64 monomials
+    static constexpr int kB3Block = (((DV + 16) * 128 + 1023) / 1024) * 1024;
+    static constexpr int kB3Bytes = MT<F>::kBlocks * (DV + 16) * 128;
+    static constexpr int kBqBlock = MT<F>::kPad * 128;                    // dCsym operand [kPad][d], one block per 64 value channels
+    static constexpr int kOffBq = kOffB3 + MT<F>::kBlocks * kB3Block;
+    // dV staging tiles (one per group) for a TMA store; with the wider tiles of F = 2 they do not fit and dV leaves
+    // straight from registers (32-byte stores)
+    static constexpr bool kStagedOut = F == 3;
+    static constexpr int kOffO = kOffBq + ((2 * kBqBlock + 1023) / 1024) * 1024;
     static constexpr int kOBytes = kTileTokens * DV * 2;
-    static constexpr int kOffBars = kOffO + 2 * kOBytes;
+    static constexpr int kOffBars = kOffO + (kStagedOut ? 2 * kOBytes : 0);
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
+    static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
+    static constexpr int kColD4 = 256, kD4Stride = F == 3 ? 64 : 96;      // TMEM: D3[grp] at 128 grp, D4[grp] at 256 + stride grp
 };
 
-template <int DV>
+template <int DV, int F>
 __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapB3,
                                                                    const __grid_constant__ CUtensorMap mapBq, const __grid_constant__ CUtensorMap mapdV,
                                                                    const float* __restrict__ kf, const float* __restrict__ dstate,
-                                                                   float* __restrict__ dkf, int N, int BH, int ld, int* status) {
-    using Cfg = BkCfg<DV>;
+                                                                   float* __restrict__ dkf, __nv_bfloat16* __restrict__ dV, int N, int BH, int ld, int* status) {
+    using Cfg = BkCfg<DV, F>;
+    using M = MT<F>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
@@ -1002,7 +1182,7 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_slot;     // D3[grp] at columns 128*grp, D4[grp] at columns 256 + 64*grp
+    const uint32_t tmem = *tmem_slot;     // D3[grp] at columns 128*grp, D4[grp] at columns 256 + kD4Stride*grp
     grid_dependency_wait();
     bool ok = true;
 
@@ -1019,7 +1199,7 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc4 = idesc_bf16(128, kMonoPad, false, false);   // G  = V (K-major over g) * dCsym (K-major over g)
+            const uint32_t idesc4 = idesc_bf16(128, M::kPad, false, false);    // G  = V (K-major over g) * dCsym (K-major over g)
             const uint32_t idesc3 = idesc_bf16(128, DV, false, false);         // dV = Tsym_k (K-major over m) * dCsym^T (K-major over m)
             const uint32_t b3a = smem_u32(smem + Cfg::kOffB3), bqa = smem_u32(smem + Cfg::kOffBq);
             int cur_bh = -1, nload = 0;
@@ -1031,9 +1211,9 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                         umma_commit(op_free);
                         if (!mbar_wait(op_free, (nload - 1) & 1)) { report_timeout(status, 402); break; }
                     }
-                    mbar_arrive_expect_tx(op_full, Cfg::kB3Bytes + kMonoPad * DV * 2);
-                    tma_load_2d(smem + Cfg::kOffB3, &mapB3, op_full, 0, bh * (DV + 16));
-                    for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + Cfg::kOffBq + b * (kBlk / 2), &mapBq, op_full, b * 64, bh * kMonoPad);
+                    mbar_arrive_expect_tx(op_full, Cfg::kB3Bytes + M::kPad * DV * 2);
+                    for (int b = 0; b < M::kBlocks; ++b) tma_load_2d(smem + Cfg::kOffB3 + b * Cfg::kB3Block, &mapB3, op_full, b * 64, bh * (DV + 16));
+                    for (int b = 0; b < DV / 64; ++b) tma_load_2d(smem + Cfg::kOffBq + b * Cfg::kBqBlock, &mapBq, op_full, b * 64, bh * M::kPad);
                     if (!mbar_wait(op_full, nload & 1)) { report_timeout(status, 403); break; }
                     ++nload;
                     cur_bh = bh;
@@ -1043,17 +1223,17 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                 const uint32_t va = smem_u32(smem + Cfg::kOffV + st * Cfg::kVBytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16(tmem + 256 + 64 * grp, smem_desc_sw128(va + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(bqa + (ks >> 2) * (kBlk / 2) + (ks & 3) * 32, 16, 1024), idesc4, ks > 0 ? 1u : 0u);
+                    umma_bf16(tmem + Cfg::kColD4 + Cfg::kD4Stride * grp, smem_desc_sw128(va + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                              smem_desc_sw128(bqa + (ks >> 2) * Cfg::kBqBlock + (ks & 3) * 32, 16, 1024), idesc4, ks > 0 ? 1u : 0u);
                 umma_commit(&d4_full[grp]);
                 umma_commit(&empty_v[st]);
                 if (!mbar_wait(&a_full[grp], u & 1)) { report_timeout(status, 405); break; }
                 tc_fence_after();
-                const uint32_t aa = smem_u32(smem + Cfg::kOffA + grp * kBlk);
+                const uint32_t aa = smem_u32(smem + Cfg::kOffA + grp * Cfg::kABytes);
 #pragma unroll
-                for (int ks = 0; ks < kMonoPad / 16; ++ks)
-                    umma_bf16(tmem + 128 * grp, smem_desc_sw128(aa + ks * 32, 16, 1024), smem_desc_sw128(b3a + ks * 32, 16, 1024), idesc3,
-                              ks > 0 ? 1u : 0u);
+                for (int ks = 0; ks < M::kPad / 16; ++ks)
+                    umma_bf16(tmem + 128 * grp, smem_desc_sw128(aa + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
+                              smem_desc_sw128(b3a + (ks >> 2) * Cfg::kB3Block + (ks & 3) * 32, 16, 1024), idesc3, ks > 0 ? 1u : 0u);
                 umma_commit(&d3_full[grp]);
             }
         }
@@ -1061,26 +1241,26 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const bool leader = (warp - 2) == 4 * grp && lane == 0;
-        float kn[18];     // key features of the group's next tile, loaded one tile ahead (row index clamped)
+        float kn[M::kKf];     // key features of the group's next tile, loaded one tile ahead (row index clamped)
         auto prefetch = [&](int it) {
             const int work = w0 + it, bh = work / tiles_per_head, tok = min((work % tiles_per_head) * kTileTokens + row, N - 1);
 #pragma unroll
-            for (int f = 0; f < 3; ++f) load6(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+            for (int f = 0; f < F; ++f) load_feat<M::kDphi>(kn + M::kDphi * f, kf + (((size_t)bh * F + f) * N + tok) * M::kDphi);
         };
         if (grp < nwork) prefetch(grp);
         for (int it = grp; it < nwork; it += 2) {
             const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
             const int u = it >> 1;
             const int tok = tile * kTileTokens + row;
-            float k[18];
+            float k[M::kKf];
 #pragma unroll
-            for (int i = 0; i < 18; ++i) k[i] = tok < N ? kn[i] : 0.f;
+            for (int i = 0; i < M::kKf; ++i) k[i] = tok < N ? kn[i] : 0.f;
             if (it + 2 < nwork) prefetch(it + 2);
             {
-                float ts[kMono];
-                key_folded(k, ts);
+                float ts[M::kN];
+                key_folded_t<F>(k, ts);
                 // the folded key tile of this group is free: its last reader (the dV MMA two tiles ago) was waited for below
-                store_mono_row(smem_u32(smem + Cfg::kOffA + grp * kBlk), row, ts, 1.f);
+                store_mono_row_t<F>(smem_u32(smem + Cfg::kOffA + grp * Cfg::kABytes), row, ts, 1.f);
                 fence_proxy_async();
                 mbar_arrive(&a_full[grp]);
             }
@@ -1089,60 +1269,80 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                float G[kMono];
-                const uint32_t ta = tmem + 256 + 64 * grp + ((uint32_t)(quarter * 32) << 16);
-                const float* dz = dstate + (size_t)bh * kMono * ld + DV;
+                float G[M::kN];
+                const uint32_t ta = tmem + Cfg::kColD4 + Cfg::kD4Stride * grp + ((uint32_t)(quarter * 32) << 16);
+                const float* dz = dstate + (size_t)bh * M::kN * ld + DV;
 #pragma unroll
-                for (int c = 0; c < kMono / 8; ++c) {
+                for (int c = 0; c < (M::kN + 7) / 8; ++c) {
                     uint32_t rr[8];
                     tmem_ld8(ta + 8 * c, rr);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) G[8 * c + e] = __uint_as_float(rr[e]) + __ldg(dz + (size_t)(8 * c + e) * ld);
+                    for (int e = 0; e < 8; ++e)
+                        if (8 * c + e < M::kN) G[8 * c + e] = __uint_as_float(rr[e]) + __ldg(dz + (size_t)(8 * c + e) * ld);
                 }
-                float dk[18];
-                key_folded_grad(k, G, dk);
+                float dk[M::kKf];
+                key_folded_grad_t<F>(k, G, dk);
                 if (tok < N) {
 #pragma unroll
-                    for (int f = 0; f < 3; ++f) store6(dkf + (((size_t)bh * 3 + f) * N + tok) * 6, dk + 6 * f);
+                    for (int f = 0; f < F; ++f) store_feat<M::kDphi>(dkf + (((size_t)bh * F + f) * N + tok) * M::kDphi, dk + M::kDphi * f);
                 }
             }
             // ---- dV
             if (ok && !mbar_wait(&d3_full[grp], u & 1)) { ok = false; report_timeout(status, 407); }
             ok = __all_sync(0xffffffffu, ok);
-            if (leader) tma_store_wait_read0();          // this group's staging tile has been read by its previous store
-            named_barrier(1 + grp, 128);
-            if (ok) {
-                tc_fence_after();
-                const uint32_t ta = tmem + 128 * grp + ((uint32_t)(quarter * 32) << 16);
-                const uint32_t os = smem_u32(smem + Cfg::kOffO + grp * Cfg::kOBytes);
+            if constexpr (Cfg::kStagedOut) {
+                if (leader) tma_store_wait_read0();          // this group's staging tile has been read by its previous store
+                named_barrier(1 + grp, 128);
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t ta = tmem + 128 * grp + ((uint32_t)(quarter * 32) << 16);
+                    const uint32_t os = smem_u32(smem + Cfg::kOffO + grp * Cfg::kOBytes);
 #pragma unroll
-                for (int h = 0; h < DV / 64; ++h) {      // 64 columns per batch of TMEM loads
-                    uint32_t r[64];
+                    for (int h = 0; h < DV / 64; ++h) {      // 64 columns per batch of TMEM loads
+                        uint32_t r[64];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) tmem_ld16(ta + 64 * h + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
-                    tmem_ld_wait();
+                        for (int c = 0; c < 4; ++c) tmem_ld16(ta + 64 * h + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t w[8];
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t w[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1]));
-                        const uint32_t blk = os + h * kBlk;
-                        st_shared_v4(blk + sw128_off(row, 2 * c), w[0], w[1], w[2], w[3]);
-                        st_shared_v4(blk + sw128_off(row, 2 * c + 1), w[4], w[5], w[6], w[7]);
+                            for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[16 * c + 2 * e]), __uint_as_float(r[16 * c + 2 * e + 1]));
+                            const uint32_t blk = os + h * kBlk;
+                            st_shared_v4(blk + sw128_off(row, 2 * c), w[0], w[1], w[2], w[3]);
+                            st_shared_v4(blk + sw128_off(row, 2 * c + 1), w[4], w[5], w[6], w[7]);
+                        }
                     }
+                    tc_fence_before();
+                    mbar_arrive(&acc_empty[grp]);
+                    fence_proxy_async();
                 }
-                tc_fence_before();
-                mbar_arrive(&acc_empty[grp]);
-                fence_proxy_async();
-            }
-            named_barrier(1 + grp, 128);
-            if (ok && leader) {
-                for (int b = 0; b < DV / 64; ++b) tma_store_3d(&mapdV, smem + Cfg::kOffO + grp * Cfg::kOBytes + b * kBlk, b * 64, tile * kTileTokens, bh);
-                tma_store_commit();
+                named_barrier(1 + grp, 128);
+                if (ok && leader) {
+                    for (int b = 0; b < DV / 64; ++b) tma_store_3d(&mapdV, smem + Cfg::kOffO + grp * Cfg::kOBytes + b * kBlk, b * 64, tile * kTileTokens, bh);
+                    tma_store_commit();
+                }
+            } else {
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t ta = tmem + 128 * grp + ((uint32_t)(quarter * 32) << 16);
+                    __nv_bfloat16* dst = dV + ((size_t)bh * N + (tok < N ? tok : 0)) * DV;
+#pragma unroll 2
+                    for (int c = 0; c < DV / 16; ++c) {
+                        uint32_t r[16], w[8];
+                        tmem_ld16(ta + 16 * c, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                        if (tok < N) st_global_v8(dst + 16 * c, w);      // one full 32-byte sector per store
+                    }
+                    tc_fence_before();
+                    mbar_arrive(&acc_empty[grp]);
+                }
             }
         }
-        if (leader) tma_store_wait_all0();
+        if (Cfg::kStagedOut && leader) tma_store_wait_all0();
     }
     tc_fence_before();
     __syncthreads();
@@ -1174,93 +1374,109 @@ inline bool set_smem(K kernel, int bytes) {
     return true;
 }
 
-template <int DV>
+template <int DV, int F>
 inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
                                       const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec, bool readout) {
+    constexpr int kPad = MT<F>::kPad;
     CUtensorMap mapV, mapO, mapB3;
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
     __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
     if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens) ||
-        !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), kMonoPad, DV + 16))
+        !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), kPad, DV + 16))
         return HLA_ERR_CUDA;
     int* status = reinterpret_cast<int*>(ws + L.status);
     float* part = reinterpret_cast<float*>(ws + off_part);
     float* state = reinterpret_cast<float*>(ws + L.state);
     float* eta = reinterpret_cast<float*>(ws + L.eta);
-    if (!set_smem(tc_state_build_kernel<DV>, kSbSmem) || !set_smem(tc_readout_kernel<DV>, RoCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_state_build_kernel<DV, F>, SbCfg<F>::kSmem) || !set_smem(tc_readout_kernel<DV, F>, RoCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
     rec.begin("tc_state_build");
-    launch_pdl(tc_state_build_kernel<DV>, dim3(D.S, BH), dim3(kSbThreads), kSbSmem, st, mapV, kf, part, D.N, D.S, D.ld, status);
+    launch_pdl(tc_state_build_kernel<DV, F>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<F>::kSmem, st, mapV, kf, part, D.N, D.S, D.ld, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, state, b3, bq, D.S, D.ld, 0, 0);
+    launch_pdl(tc_reduce_emit_kernel<DV, F>, dim3(kPad / 8, BH), dim3(256), 0, st, part, state, b3, bq, D.S, D.ld, 0, 0);
     if (!rec.end()) return HLA_ERR_CUDA;
     if (!readout) return HLA_OK;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_readout");
-    launch_pdl(tc_readout_kernel<DV>, grid, dim3(kRoThreads), RoCfg<DV>::kSmem, st, mapB3, mapO, qf, eta, D.N, BH, D.eps, status);
+    launch_pdl(tc_readout_kernel<DV, F>, grid, dim3(kRoThreads), RoCfg<DV, F>::kSmem, st, mapB3, mapO, qf, eta, D.N, BH, D.eps, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
 // Reduction of the pieces the fused key-side kernel (G CTAs over heads x T tiles, at most `smax` pieces per head) left.
-inline hla_status reduce_pieces(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec) {
+template <int F>
+inline hla_status reduce_pieces_f(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec) {
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
     __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
     float* part = reinterpret_cast<float*>(ws + off_part);
     float* state = reinterpret_cast<float*>(ws + L.state);
     const int T = (D.N + kTileTokens - 1) / kTileTokens;
     rec.begin("tc_reduce_emit");
-    if (D.d == 128) launch_pdl(tc_reduce_emit_kernel<128>, dim3(8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
-    else launch_pdl(tc_reduce_emit_kernel<64>, dim3(8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
+    if (D.d == 128) launch_pdl(tc_reduce_emit_kernel<128, F>, dim3(MT<F>::kPad / 8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
+    else launch_pdl(tc_reduce_emit_kernel<64, F>, dim3(MT<F>::kPad / 8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+inline hla_status reduce_pieces(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec) {
+    return D.F == 3 ? reduce_pieces_f<3>(P, D, BH, ws, L, off_part, smax, G, rec) : reduce_pieces_f<2>(P, D, BH, ws, L, off_part, smax, G, rec);
 }
 
 // readout = false stops after the state has been built and reduced (the fused query-side kernel reads it out).
 inline hla_status core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
                                const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec, bool readout = true) {
-    if (D.d == 128) return launch_core_forward<128>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
-    return launch_core_forward<64>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
+    if (D.F == 3) {
+        if (D.d == 128) return launch_core_forward<128, 3>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
+        return launch_core_forward<64, 3>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
+    }
+    if (D.d == 128) return launch_core_forward<128, 2>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
+    return launch_core_forward<64, 2>(P, D, BH, qf, kf, V, O, ws, L, off_part, sm_count, rec, readout);
 }
 
-template <int DV>
+template <int DV, int F>
 inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, const void* dO,
                                        float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count,
                                        LaunchRec& rec) {
+    constexpr int kPad = MT<F>::kPad;
     CUtensorMap mapV, mapdO, mapdV, mapBq, mapBd3, mapBdq;
     __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
     __nv_bfloat16* bd3 = reinterpret_cast<__nv_bfloat16*>(ws + P.bd3);
     __nv_bfloat16* bdq = reinterpret_cast<__nv_bfloat16*>(ws + P.bdq);
     if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapdO, dO, BH, D.N, DV, kTileTokens) ||
-        !make_map_bhnd(&mapdV, dV, BH, D.N, DV, kTileTokens) || !make_map_2d(&mapBq, bq, (size_t)BH * kMonoPad, DV, kMonoPad) ||
-        !make_map_2d(&mapBd3, bd3, (size_t)BH * (DV + 16), kMonoPad, DV + 16) || !make_map_2d(&mapBdq, bdq, (size_t)BH * kMonoPad, DV, kMonoPad))
+        !make_map_bhnd(&mapdV, dV, BH, D.N, DV, kTileTokens) || !make_map_2d(&mapBq, bq, (size_t)BH * kPad, DV, kPad) ||
+        !make_map_2d(&mapBd3, bd3, (size_t)BH * (DV + 16), kPad, DV + 16) || !make_map_2d(&mapBdq, bdq, (size_t)BH * kPad, DV, kPad))
         return HLA_ERR_CUDA;
     int* status = reinterpret_cast<int*>(ws + L.status);
     float* part = reinterpret_cast<float*>(ws + off_part);
     const float* state = reinterpret_cast<const float*>(ws + L.state);
     float* dstate = reinterpret_cast<float*>(ws + L.dstate);
     const float* eta = reinterpret_cast<const float*>(ws + L.eta);
-    if (!set_smem(tc_bwd_query_kernel<DV>, kBqSmem) || !set_smem(tc_bwd_key_kernel<DV>, BkCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_bwd_query_kernel<DV, F>, BqCfg<F>::kSmem) || !set_smem(tc_bwd_key_kernel<DV, F>, BkCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
     rec.begin("tc_bwd_query");
-    launch_pdl(tc_bwd_query_kernel<DV>, dim3(D.S, BH), dim3(kBqThreads), kBqSmem, st, mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps, status);
+    launch_pdl(tc_bwd_query_kernel<DV, F>, dim3(D.S, BH), dim3(kBqThreads), BqCfg<F>::kSmem, st, mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps,
+               status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
-    launch_pdl(tc_reduce_emit_kernel<DV>, dim3(8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld, 0, 0);
+    launch_pdl(tc_reduce_emit_kernel<DV, F>, dim3(kPad / 8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld, 0, 0);
     if (!rec.end()) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_bwd_key");
-    launch_pdl(tc_bwd_key_kernel<DV>, grid, dim3(kBkThreads), BkCfg<DV>::kSmem, st, mapV, mapBd3, mapBdq, mapdV, kf, dstate, dkf, D.N, BH, D.ld, status);
+    launch_pdl(tc_bwd_key_kernel<DV, F>, grid, dim3(kBkThreads), BkCfg<DV, F>::kSmem, st, mapV, mapBd3, mapBdq, mapdV, kf, dstate, dkf,
+               static_cast<__nv_bfloat16*>(dV), D.N, BH, D.ld, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
 inline hla_status core_backward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, const void* dO,
                                 float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
-    if (D.d == 128) return launch_core_backward<128>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
-    return launch_core_backward<64>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+    if (D.F == 3) {
+        if (D.d == 128) return launch_core_backward<128, 3>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+        return launch_core_backward<64, 3>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+    }
+    if (D.d == 128) return launch_core_backward<128, 2>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+    return launch_core_backward<64, 2>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
 }
 
 }  // namespace tc

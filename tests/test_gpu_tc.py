@@ -37,6 +37,38 @@ def test_core_forward_bf16_features(d, N, B, H, splits):
     assert run.op.launches() == 3
 
 
+@pytest.mark.parametrize("d,N,B,H,splits", [(128, 1000, 1, 2, 0), (64, 1500, 2, 2, 5), (128, 77, 1, 3, 0), (128, 4096 + 40, 1, 2, 7), (64, 129, 1, 1, 4)])
+def test_core_forward_and_backward_two_factors(d, N, B, H, splits):
+    """The paper's 2-factor variant (d_phi = 12: 78 monomials q_a q_b, a <= b, in two operand blocks) at the feature level:
+    state (folded over the symmetry of q (x) q), normaliser, output and all three gradients against the oracle."""
+    s = synth.HlaShape("t", B, H, N, d, "bf16", "inv_sqrt_d", False, 2, 12)
+    _, _, V = synth.make_qkv(s)
+    V = synth.bf16_round(V * np.float32(np.sqrt(d)))
+    qf, kf = synth.make_features(s)
+    dO = synth.make_dO(s)
+    run = DeviceRun(s, "none", EPS, splits)
+    assert run.op.layout.tensor_core == 1 and run.op.layout.state_rows == 78
+    O = run.forward(qf, kf, V)
+    assert run.op.launches() == 3
+    f64 = lambda a: a.astype(np.float64)
+    Oq, eta = orc.hla_core_forward(f64(qf), f64(kf), f64(V), EPS, "quadratic" if N <= 1500 else "factored")
+    C, z = run.state()
+    Co, zo = oracle_state(f64(kf), f64(V))
+    Co, zo = fold_symmetric(Co, 12, 2), fold_symmetric(zo[..., None], 12, 2)[..., 0]
+    assert relerr(z, zo) < 1e-5
+    assert relerr(C, Co) < TOL["bf16"] / 4
+    assert relerr(run.eta(), eta) < TOL["bf16"] / 4
+    assert relerr(O, Oq) < TOL["bf16"], relerr(O, Oq)
+    dq, dk, dv = run.backward(dO)
+    assert run.op.launches() == 3
+    rq, rk, rv = orc.hla_core_backward(f64(qf), f64(kf), f64(V), f64(dO), EPS, "quadratic" if N <= 1000 else "factored")
+    assert relerr(dv, rv) < TOL["bf16"], relerr(dv, rv)
+    assert relerr(dq, rq) < TOL["bf16"], relerr(dq, rq)
+    assert relerr(dk, rk) < TOL["bf16"], relerr(dk, rk)
+    again = run.forward(qf, kf, V)
+    assert np.array_equal(O, again)
+
+
 def test_config2_small_bf16_forward_stagewise():
     """B=2,H=12,N=4096,d=64 bf16 with the phi maps: features against the oracle's,
     then the core against the oracle core run on the features the GPU produced,
