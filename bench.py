@@ -600,7 +600,7 @@ def main():
         del w, op
         torch.cuda.empty_cache()
         extra = {}
-        for name in ("long_bf16", "dit_bf16", "small_bf16", "paper_r1_bf16", "paper_r2_bf16"):
+        for name in ("long_bf16", "dit_bf16", "small_bf16", "paper_r1_bf16", "paper_r2_bf16", "train_bf16_2f"):
             if name != shape.name:
                 extra[name] = extra_leg(name, rank, dev, peaks, local)
 

@@ -261,7 +261,6 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     D.ld = c.d + 4;
     D.eps = c.eps;
     x->tc = tc::supported(c.dtype == HLA_BF16, c.d, c.F, c.d_phi) && (long long)c.B * c.H * c.N < (1ll << 31);   // the tensor-core kernels index tokens in 32 bits
-    if (c.F == 2 && c.phi == HLA_PHI_MLP) x->tc = false;      // the 2-factor geometry runs on the tensor cores at the feature level only
     const int tile = x->tc ? tc::kTileTokens : simt::kTok;
     const int tiles = (c.N + tile - 1) / tile;
     int S = c.n_splits;

@@ -21,37 +21,41 @@ namespace tc {
 constexpr int kFqThreads = 28 * 32;
 constexpr int kFqGeluWarp0 = 3, kFqFeatWarp0 = 19, kFqOutWarp0 = 23, kFqReadoutMmaWarp = 27;
 
-template <int DV> struct FqCfg {
+template <int DV, int F> struct FqCfg {
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
     static constexpr int kW2Bytes = (DV / 64) * 2048;            // [16 rows][DV] bf16, K-major
     static constexpr int kNmma = DV + 16;                        // readout product: d value channels, then the normaliser column
-    static constexpr int kB3Bytes = kNmma * 128;
+    static constexpr int kB3Block = ((kNmma * 128 + 1023) / 1024) * 1024;   // one 64-monomial block of the state operand
+    static constexpr int kB3Bytes = MT<F>::kBlocks * kNmma * 128;           // bytes its TMA loads deliver
     static constexpr int kOffX = 0;                              // 2 Q tiles (the load of a tile takes longer than a tile's arithmetic)
     static constexpr int kOffW1 = 2 * kXBytes;                   // (the GELU tile lives in TMEM)
     static constexpr int kOffW2 = kOffW1 + kW1Bytes;
     static constexpr int kOffB3 = kOffW2 + ((kW2Bytes + 1023) / 1024) * 1024;      // state operand of the current head
-    static constexpr int kOffA = kOffB3 + ((kB3Bytes + 1023) / 1024) * 1024;        // monomial tile
-    static constexpr int kOffO = kOffA + kBlk;                   // O staging tile
+    static constexpr int kOffA = kOffB3 + MT<F>::kBlocks * kB3Block;               // monomial tile
+    static constexpr int kOffO = kOffA + MT<F>::kBlocks * kBlk;  // O staging tile
     // b1 is added on the tensor cores by a ninth K step of the first-layer product: A = a constant tile whose K column
     // 0 is 1, B = a tile whose K row 0 is b1 (both zero elsewhere)
     static constexpr int kOffOnes = kOffO + kXBytes;             // [128 rows][64 K] bf16, K-major (16 K columns used)
     static constexpr int kB1Bytes = (DV / 64) * 2048;            // [16 K rows][DV] bf16, MN-major
     static constexpr int kOffB1 = kOffOnes + kBlk;
-    static constexpr int kOffBias = kOffB1 + kB1Bytes;           // b1[DV] (unused by the kernel), b2[8] floats
-    static constexpr int kOffBars = kOffBias + (DV + 8) * 4;
+    static constexpr int kOffBias = kOffB1 + kB1Bytes;           // b1[DV] (unused by the kernel), b2[16] floats
+    static constexpr int kOffBars = kOffBias + (DV + 16) * 4;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
+    static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
 
 // Q [BH][N][DV] bf16 (3-D map, rows past N read as zero), O the same (stores are clipped at N).
-template <int DV>
+template <int DV, int F>
 __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapW1,
                                                                         const __grid_constant__ CUtensorMap mapB3, const __grid_constant__ CUtensorMap mapO,
                                                                         const __nv_bfloat16* __restrict__ b1g, const __nv_bfloat16* __restrict__ W2g,
                                                                         const __nv_bfloat16* __restrict__ b2g, float* __restrict__ qf_out,
                                                                         float* __restrict__ eta_out, int N, int BH, float eps, int* status) {
-    using Cfg = FqCfg<DV>;
+    using Cfg = FqCfg<DV, F>;
+    using M = MT<F>;
+    constexpr int DP = M::kDphi;
     constexpr int HC = DV / 4;          // hidden units per GELU thread
     extern __shared__ uint8_t smem_raw[];
     grid_launch_dependents();
@@ -85,10 +89,10 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     // second-layer weights as a K-major MMA operand [16 rows (outputs, 6 used)][DV], and the biases
     for (int i = tid; i < Cfg::kW2Bytes / 16; i += kFqThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffW2)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
-    for (int i = tid; i < DV * 6; i += kFqThreads) {
-        const int j = i / 6, o = i % 6;
+    for (int i = tid; i < DV * DP; i += kFqThreads) {
+        const int j = i / DP, o = i % DP;
         uint8_t* base = smem + Cfg::kOffW2 + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = half_bf16(W2g[j * 6 + o]);
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(o, (j & 63) >> 3) + (j & 7) * 2) = half_bf16(W2g[j * DP + o]);
     }
     for (int i = tid; i < (kBlk + Cfg::kB1Bytes) / 16; i += kFqThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffOnes)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
@@ -96,7 +100,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
         *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffOnes + sw128_off(i, 0)) = __float2bfloat16_rn(1.f);
     for (int j = tid; j < DV; j += kFqThreads)      // K row 0 of the MN-major tile: 64-column block j / 64, no swizzle in row 0
         *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffB1 + (j >> 6) * 2048 + (j & 63) * 2) = b1g[j];
-    for (int j = tid; j < DV + 8; j += kFqThreads) bias[j] = j < DV ? __bfloat162float(b1g[j]) : (j - DV < 6 ? __bfloat162float(b2g[j - DV]) : 0.f);
+    for (int j = tid; j < DV + 16; j += kFqThreads) bias[j] = j < DV ? __bfloat162float(b1g[j]) : (j - DV < DP ? __bfloat162float(b2g[j - DV]) : 0.f);
     fence_proxy_async();
     if (tid == 0) {
         mbar_init(x_full, 1);
@@ -194,6 +198,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             const uint32_t idesc3 = idesc_bf16(128, Cfg::kNmma, false, false);   // monomial tile K-major, state operand K-major over the monomials
             const uint64_t ad = smem_desc_sw128(smem_u32(smem + Cfg::kOffA), 16, 1024);
             const uint64_t bd = smem_desc_sw128(smem_u32(smem + Cfg::kOffB3), 16, 1024);
+            static_assert(Cfg::kB3Block % 16 == 0, "descriptor advance");
             int cur_bh = -1, nload = 0;
             bool good = true;
             for (int it = 0; it < nwork && good; ++it) {
@@ -204,7 +209,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
                         if (!mbar_wait(b3_free, (nload - 1) & 1)) { good = false; break; }
                     }
                     mbar_arrive_expect_tx(b3_full, Cfg::kB3Bytes);
-                    tma_load_2d(smem + Cfg::kOffB3, &mapB3, b3_full, 0, bh * Cfg::kNmma);
+                    for (int b = 0; b < M::kBlocks; ++b) tma_load_2d(smem + Cfg::kOffB3 + b * Cfg::kB3Block, &mapB3, b3_full, b * 64, bh * Cfg::kNmma);
                     if (!mbar_wait(b3_full, nload & 1)) { good = false; break; }
                     ++nload;
                     cur_bh = bh;
@@ -212,8 +217,9 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
                 if (!(mbar_wait(a_full, it & 1) && mbar_wait(acc_empty, (it & 1) ^ 1))) { good = false; break; }
                 tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < kMonoPad / 16; ++ks)
-                    umma_bf16(tmem + 320, desc_advance(ad, ks * 32), desc_advance(bd, ks * 32), idesc3, ks > 0 ? 1u : 0u);
+                for (int ks = 0; ks < M::kPad / 16; ++ks)
+                    umma_bf16(tmem + 320, desc_advance(ad, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(bd, (ks >> 2) * Cfg::kB3Block + (ks & 3) * 32), idesc3,
+                              ks > 0 ? 1u : 0u);
                 umma_commit(a_empty);
                 umma_commit(acc_full);
             }
@@ -276,22 +282,23 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            uint32_t r[8];
-            tmem_ld8(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), r);
+            uint32_t r[16];
+            if constexpr (DP <= 8) tmem_ld8(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), *reinterpret_cast<uint32_t(*)[8]>(r));
+            else tmem_ld16(tmem + 256 + 32 * b + ((uint32_t)(quarter * 32) << 16), r);
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(&d2_empty[b]);
             const int tok = tile * kTileTokens + row;
-            float q[6];
+            float q[DP];
 #pragma unroll
-            for (int o = 0; o < 6; ++o) q[o] = tok < N ? fmaxf(__uint_as_float(r[o]) + b2s[o], 0.f) : 0.f;
-            if (tok < N) store6(qf_out + ((size_t)bh * N + tok) * 6, q);
-            float mono[kMono];
-            query_monomials(q, mono);
+            for (int o = 0; o < DP; ++o) q[o] = tok < N ? fmaxf(__uint_as_float(r[o]) + b2s[o], 0.f) : 0.f;
+            if (tok < N) store_feat<DP>(qf_out + ((size_t)bh * N + tok) * DP, q);
+            float mono[M::kN];
+            query_monomials_t<F>(q, mono);
             if (!mbar_wait(a_empty, (it & 1) ^ 1)) { ok = false; report_timeout(status, 706); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            store_mono_row(smem_u32(smem + Cfg::kOffA), row, mono, 1.f);
+            store_mono_row_t<F>(smem_u32(smem + Cfg::kOffA), row, mono, 1.f);
             fence_proxy_async();
             mbar_arrive(a_full);
         }
@@ -333,20 +340,20 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-template <int DV>
+template <int DV, int F>
 inline hla_status launch_phiq_readout(const Plan& P, const Dims& D, int BH, const hla_mlp* phi_q, const void* Q, void* O, char* ws,
                                       const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
     CUtensorMap mapQ, mapW1, mapB3, mapO;
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
     if (!make_map_bhnd(&mapQ, Q, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens) ||
-        !make_map_2d(&mapW1, phi_q->W1, DV, DV, DV) || !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), kMonoPad, DV + 16))
+        !make_map_2d(&mapW1, phi_q->W1, DV, DV, DV) || !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), MT<F>::kPad, DV + 16))
         return HLA_ERR_CUDA;
-    if (!set_smem(tc_phiq_readout_kernel<DV>, FqCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_phiq_readout_kernel<DV, F>, FqCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
     rec.begin("tc_phiq_readout");
-    launch_pdl(tc_phiq_readout_kernel<DV>, grid, dim3(kFqThreads), FqCfg<DV>::kSmem, rec.st, 
+    launch_pdl(tc_phiq_readout_kernel<DV, F>, grid, dim3(kFqThreads), FqCfg<DV, F>::kSmem, rec.st,
         mapQ, mapW1, mapB3, mapO, static_cast<const __nv_bfloat16*>(phi_q->b1), static_cast<const __nv_bfloat16*>(phi_q->W2),
         static_cast<const __nv_bfloat16*>(phi_q->b2), reinterpret_cast<float*>(ws + L.qf), reinterpret_cast<float*>(ws + L.eta), D.N, BH, D.eps,
         reinterpret_cast<int*>(ws + L.status));
@@ -355,8 +362,12 @@ inline hla_status launch_phiq_readout(const Plan& P, const Dims& D, int BH, cons
 
 inline hla_status phiq_readout(const Plan& P, const Dims& D, int BH, const hla_mlp* phi_q, const void* Q, void* O, char* ws, const hla_ws_layout& L,
                                int sm_count, LaunchRec& rec) {
-    if (D.d == 128) return launch_phiq_readout<128>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
-    return launch_phiq_readout<64>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+    if (D.F == 3) {
+        if (D.d == 128) return launch_phiq_readout<128, 3>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+        return launch_phiq_readout<64, 3>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+    }
+    if (D.d == 128) return launch_phiq_readout<128, 2>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+    return launch_phiq_readout<64, 2>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
 }
 
 }  // namespace tc

@@ -30,23 +30,28 @@ constexpr int kFkThreads = 25 * 32;
 constexpr int kFkGeluWarp0 = 3, kFkFeatWarp0 = 19, kFkStateWarp = 23, kFkZWarp = 24;
 constexpr int kFkB1Row = 12;        // K row of the staged W2 tiles that carries b1 (rows 6..15 are padding of the second layer)
 
-// TMEM columns
-constexpr int kFkColD2 = 256;       // D2[b] at 256 + 32 b (16 columns used)
-constexpr int kFkColOnes = 272;     // 8 columns: the constant A operand of the bias step (K column kFkB1Row is 1)
-constexpr int kFkColG = 320;        // G[b] (bf16 pairs) at 320 + 64 b
-constexpr int kFkColC = 448;        // Csym^T accumulator, 64 columns, lane = value channel
+// TMEM columns (D1[b] at 128 b).  F = 3: D2[b] at 256 + 32 b (16 used), the constant A operand of the bias step (8 columns, K column
+// kFkB1Row is 1) at 272, G[b] (bf16 pairs) at 320 + 64 b, the Csym^T accumulator (64 columns, lane = value channel) at 448.
+// F = 2 needs 80 accumulator columns: G[b] at 256 + 64 b, D2[b] at 384 + 16 b, the constant operand at 416, Csym^T at 432.
+template <int F> struct FkCols {
+    static constexpr int kD2 = F == 3 ? 256 : 384, kD2Stride = F == 3 ? 32 : 16;
+    static constexpr int kOnes = F == 3 ? 272 : 416;
+    static constexpr int kG = F == 3 ? 320 : 256;
+    static constexpr int kC = F == 3 ? 448 : 432;
+};
 
-template <int DV> struct FkCfg {
+template <int DV, int F> struct FkCfg {
+    static constexpr int NM = MT<F>::kMaps;
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
     static constexpr int kW2Bytes = (DV / 64) * 2048;            // [16 rows][DV] bf16 per map
     static constexpr int kOffX = 0;                              // 2 K tiles
     static constexpr int kOffW1 = 2 * kXBytes;
-    static constexpr int kOffW2 = kOffW1 + 3 * kW1Bytes;
-    static constexpr int kOffV = ((kOffW2 + 3 * kW2Bytes + 1023) / 1024) * 1024;   // V tile: two 64-column blocks (the second stays zero for d = 64)
+    static constexpr int kOffW2 = kOffW1 + NM * kW1Bytes;
+    static constexpr int kOffV = ((kOffW2 + NM * kW2Bytes + 1023) / 1024) * 1024;   // V tile: two 64-column blocks (the second stays zero for d = 64)
     static constexpr int kOffF = kOffV + 2 * kBlk;               // folded key tile
-    static constexpr int kOffB2 = kOffF + kBlk;                  // b2: 3 x 8 floats
-    static constexpr int kOffBars = kOffB2 + 128;
+    static constexpr int kOffB2 = kOffF + MT<F>::kBlocks * kBlk; // b2: NM x 16 floats
+    static constexpr int kOffBars = kOffB2 + 256;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
     static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
@@ -88,11 +93,44 @@ __device__ __forceinline__ void folded_row_store(uint32_t blk, uint32_t row, con
     (folded_chunk_store<C>(blk, row, s12, k3, std::make_integer_sequence<int, 8>{}), ...);
 }
 
-template <int DV>
+// The same for the 2-factor geometry: monomial M = (a <= b) of 12 features, value k1[a] k2[b] + k1[b] k2[a] (a < b), k1[a] k2[a] (a == b).
+__host__ __device__ constexpr int mono_ab2(int m) {
+    int idx = 0;
+    for (int a = 0; a < 12; ++a)
+        for (int b = a; b < 12; ++b) {
+            if (idx == m) return 12 * a + b;
+            ++idx;
+        }
+    return 0;
+}
+template <int M>
+__device__ __forceinline__ float folded_value2(const float (&k1)[12], const float (&k2)[12]) {
+    if constexpr (M >= MT<2>::kN) {
+        return 0.f;
+    } else {
+        constexpr int ab = mono_ab2(M), a = ab / 12, b = ab % 12;
+        if constexpr (a == b) return k1[a] * k2[a];
+        else return fmaf(k1[a], k2[b], k1[b] * k2[a]);
+    }
+}
+template <int C, int... E>
+__device__ __forceinline__ void folded_chunk_store2(uint32_t tile, uint32_t row, const float (&k1)[12], const float (&k2)[12], std::integer_sequence<int, E...>) {
+    const float v[8] = {folded_value2<8 * C + E>(k1, k2)...};
+    st_shared_v4(tile + (C >> 3) * kBlk + sw128_off(row, C & 7), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+template <int... C>
+__device__ __forceinline__ void folded_row_store2(uint32_t tile, uint32_t row, const float (&k1)[12], const float (&k2)[12], std::integer_sequence<int, C...>) {
+    (folded_chunk_store2<C>(tile, row, k1, k2, std::make_integer_sequence<int, 8>{}), ...);
+}
+
+template <int DV, int F>
 __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ PhiMaps maps,
                                                                       const __grid_constant__ CUtensorMap mapV, PhiPtrs P, float* __restrict__ kf_out,
                                                                       float* __restrict__ part, int N, int BH, int ld, int smax, int* status) {
-    using Cfg = FkCfg<DV>;
+    using Cfg = FkCfg<DV, F>;
+    using M = MT<F>;
+    using Col = FkCols<F>;
+    constexpr int NM = M::kMaps, DP = M::kDphi;
     constexpr int HC = DV / 4;          // hidden units per GELU thread
     extern __shared__ uint8_t smem_raw[];
     grid_launch_dependents();
@@ -128,17 +166,17 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
     // second-layer weights as a K-major MMA operand [16 rows (outputs, 6 used)][DV] per map, halved (the GELU warps
     // form 2 GELU); row kFkB1Row of the same tile holds b1: read as an MN-major operand [16 K rows][DV] it is the B
     // operand of the bias step of the first layer
-    for (int i = tid; i < 3 * Cfg::kW2Bytes / 16; i += kFkThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffW2)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < NM * Cfg::kW2Bytes / 16; i += kFkThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffW2)[i] = make_uint4(0, 0, 0, 0);
     if (DV == 64)
         for (int i = tid; i < kBlk / 16; i += kFkThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffV + kBlk)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
-    for (int i = tid; i < 3 * DV * 7; i += kFkThreads) {
-        const int m = i / (DV * 7), j = (i / 7) % DV, o = i % 7;
+    for (int i = tid; i < NM * DV * (DP + 1); i += kFkThreads) {
+        const int m = i / (DV * (DP + 1)), j = (i / (DP + 1)) % DV, o = i % (DP + 1);
         uint8_t* base = smem + Cfg::kOffW2 + m * Cfg::kW2Bytes + (j >> 6) * 2048;
-        const int r = o < 6 ? o : kFkB1Row;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(r, (j & 63) >> 3) + (j & 7) * 2) = o < 6 ? half_bf16(P.W2[m][j * 6 + o]) : P.b1[m][j];
+        const int r = o < DP ? o : kFkB1Row;
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(r, (j & 63) >> 3) + (j & 7) * 2) = o < DP ? half_bf16(P.W2[m][j * DP + o]) : P.b1[m][j];
     }
-    for (int i = tid; i < 3 * 8; i += kFkThreads) b2s[i] = (i & 7) < 6 ? __bfloat162float(P.b2[i >> 3][i & 7]) : 0.f;
+    for (int i = tid; i < NM * 16; i += kFkThreads) b2s[i] = (i & 15) < DP ? __bfloat162float(P.b2[i >> 4][i & 15]) : 0.f;
     fence_proxy_async();
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -176,7 +214,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         uint32_t c[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) c[i] = i == kFkB1Row / 2 ? one : 0u;
-        tmem_st8(tmem + kFkColOnes + ((uint32_t)((warp & 3) * 32) << 16), c[0], c[1], c[2], c[3], c[4], c[5], c[6], c[7]);
+        tmem_st8(tmem + Col::kOnes + ((uint32_t)((warp & 3) * 32) << 16), c[0], c[1], c[2], c[3], c[4], c[5], c[6], c[7]);
         tmem_st_wait();
     }
     tc_fence_before();
@@ -187,8 +225,8 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(w_full, 3 * Cfg::kW1Bytes);
-            for (int m = 0; m < 3; ++m)
+            mbar_arrive_expect_tx(w_full, NM * Cfg::kW1Bytes);
+            for (int m = 0; m < NM; ++m)
                 for (int b = 0; b < DV / 64; ++b)
                     tma_load_2d(smem + Cfg::kOffW1 + m * Cfg::kW1Bytes + b * (DV * 128), &maps.w1[m], w_full, b * 64, 0);
             for (int it = 0; it < nwork; ++it) {
@@ -207,8 +245,8 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
             const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 2048, 1024);
             bool good = mbar_wait(w_full, 0);
-            for (int unit = 0; unit < 3 * nwork && good; ++unit) {
-                const int it = unit / 3, m = unit - 3 * it, st = it & 1, b = unit & 1;
+            for (int unit = 0; unit < NM * nwork && good; ++unit) {
+                const int it = unit / NM, m = unit - NM * it, st = it & 1, b = unit & 1;
                 if (m == 0 && !mbar_wait(&x_full[st], (it >> 1) & 1)) { good = false; break; }
                 if (!mbar_wait(&d1_empty[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
                 tc_fence_after();
@@ -216,9 +254,9 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
-                umma_bf16_ta(tmem + 128 * b, tmem + kFkColOnes, desc_advance(bd0, m * Cfg::kW2Bytes), idesc1, 1u);
+                umma_bf16_ta(tmem + 128 * b, tmem + Col::kOnes, desc_advance(bd0, m * Cfg::kW2Bytes), idesc1, 1u);
                 umma_commit(&d1_full[b]);
-                if (m == 2) umma_commit(&x_empty[st]);
+                if (m == NM - 1) umma_commit(&x_empty[st]);
             }
             if (!good) report_timeout(status, 802);
         }
@@ -227,14 +265,14 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
             const uint32_t idesc2 = idesc_bf16(128, 16, false, false);  // G from TMEM, W2 operand K-major
             const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2), 16, 1024);
             bool good = true;
-            for (int unit = 0; unit < 3 * nwork && good; ++unit) {
-                const int m = unit % 3, b = unit & 1, par = (unit >> 1) & 1;
+            for (int unit = 0; unit < NM * nwork && good; ++unit) {
+                const int m = unit % NM, b = unit & 1, par = (unit >> 1) & 1;
                 if (!(mbar_wait(&g_full[b], par) && mbar_wait(&d2_empty[b], par ^ 1))) { good = false; break; }
                 tc_fence_after();
                 const uint64_t vd = desc_advance(vd0, m * Cfg::kW2Bytes);
 #pragma unroll
                 for (int ks = 0; ks < DV / 16; ++ks)
-                    umma_bf16_ta(tmem + kFkColD2 + 32 * b, tmem + kFkColG + 64 * b + 8 * ks, desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32), idesc2,
+                    umma_bf16_ta(tmem + Col::kD2 + Col::kD2Stride * b, tmem + Col::kG + 64 * b + 8 * ks, desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32), idesc2,
                                  ks > 0 ? 1u : 0u);
                 umma_commit(&g_free[b]);
                 umma_commit(&d2_full[b]);
@@ -243,7 +281,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         }
     } else if (warp == kFkStateWarp) {
         if (lane == 0) {      // Csym^T += V tile^T (MN-major, M = value channels) * folded key tile (MN-major, N = 64), K = 128 tokens
-            const uint32_t idesc = idesc_bf16(128, kMonoPad, true, true);
+            const uint32_t idesc = idesc_bf16(128, M::kPad, true, true);
             const uint32_t va = smem_u32(smem + Cfg::kOffV), fa = smem_u32(smem + Cfg::kOffF);
             auto load_v = [&](int it) {
                 const int work = w0 + it, bh = work / T, tile = work - bh * T;
@@ -261,7 +299,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < kTileTokens / 16; ++ks)
-                    umma_bf16(tmem + kFkColC, smem_desc_sw128(va + ks * 2048, kBlk, 1024), smem_desc_sw128(fa + ks * 2048, kBlk, 1024), idesc,
+                    umma_bf16(tmem + Col::kC, smem_desc_sw128(va + ks * 2048, kBlk, 1024), smem_desc_sw128(fa + ks * 2048, kBlk, 1024), idesc,
                               (!first || ks > 0) ? 1u : 0u);
                 umma_commit(v_empty);
                 umma_commit(f_empty);
@@ -281,36 +319,48 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         // zsym: column sums of the folded key tile as the state product sees it (bf16 values, fp32 sums); lane l owns
         // the monomials 2 l and 2 l + 1
         const uint32_t fa = smem_u32(smem + Cfg::kOffF);
-        float za = 0.f, zb = 0.f;
+        // (block 0: lane l owns the monomials 2 l, 2 l + 1; the 16 columns of a second block belong to lanes 0..7)
+        float za = 0.f, zb = 0.f, zc = 0.f, zd = 0.f;
         for (int it = 0; it < nwork; ++it) {
             if (ok && !mbar_wait(f_full, it & 1)) { ok = false; report_timeout(status, 805); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f};
+            float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f}, tc_[4] = {0.f, 0.f, 0.f, 0.f}, td[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
             for (int r = 0; r < kTileTokens; ++r) {
                 uint32_t wv;
                 asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(fa + sw128_off(r, lane >> 2) + (lane & 3) * 4) : "memory");
                 ta[r & 3] += __uint_as_float(wv << 16);
                 tb[r & 3] += __uint_as_float(wv & 0xffff0000u);
+                if (M::kBlocks == 2 && lane < 8) {
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(fa + kBlk + sw128_off(r, lane >> 2) + (lane & 3) * 4) : "memory");
+                    tc_[r & 3] += __uint_as_float(wv << 16);
+                    td[r & 3] += __uint_as_float(wv & 0xffff0000u);
+                }
             }
             za += (ta[0] + ta[1]) + (ta[2] + ta[3]);
             zb += (tb[0] + tb[1]) + (tb[2] + tb[3]);
+            zc += (tc_[0] + tc_[1]) + (tc_[2] + tc_[3]);
+            zd += (td[0] + td[1]) + (td[2] + td[3]);
             __syncwarp();
             if (lane == 0) mbar_arrive(f_empty);
             if (piece_ends(it)) {
                 const int bh = head_of(it);
                 const int piece = blockIdx.x - owner_of_work((long long)bh * T, total, G);
-                float* out = part + ((size_t)bh * smax + piece) * kMono * ld;
-                if (2 * lane < kMono) {
-                    out[(size_t)(2 * lane) * ld + DV] = za;
-                    out[(size_t)(2 * lane + 1) * ld + DV] = zb;
-                    for (int c = DV + 1; c < ld; ++c) {
-                        out[(size_t)(2 * lane) * ld + c] = 0.f;
-                        out[(size_t)(2 * lane + 1) * ld + c] = 0.f;
+                float* out = part + ((size_t)bh * smax + piece) * M::kN * ld;
+                auto put = [&](int m, float v) {
+                    if (m < M::kN) {
+                        out[(size_t)m * ld + DV] = v;
+                        for (int c = DV + 1; c < ld; ++c) out[(size_t)m * ld + c] = 0.f;
                     }
+                };
+                put(2 * lane, za);
+                put(2 * lane + 1, zb);
+                if (M::kBlocks == 2 && lane < 8) {
+                    put(64 + 2 * lane, zc);
+                    put(64 + 2 * lane + 1, zd);
                 }
-                za = zb = 0.f;
+                za = zb = zc = zd = 0.f;
             }
         }
     } else if (warp >= kFkFeatWarp0) {
@@ -323,36 +373,40 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         for (int it = 0; it < nwork && ok; ++it) {
             const int work = w0 + it, bh = work / T, tile = work - bh * T;
             const int tok = tile * kTileTokens + row;
-            float k1[6], s12[6][6];
+            float k1[DP], s12[6][6];
 #pragma unroll
-            for (int m = 0; m < 3; ++m) {
-                const int unit = 3 * it + m, b = unit & 1;
+            for (int m = 0; m < NM; ++m) {
+                const int unit = NM * it + m, b = unit & 1;
                 if (!mbar_wait(&d2_full[b], (unit >> 1) & 1)) { ok = false; report_timeout(status, 806); }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t r[8];
-                tmem_ld8(tmem + kFkColD2 + 32 * b + lane_base, r);
+                uint32_t r[16];
+                if constexpr (DP <= 8) tmem_ld8(tmem + Col::kD2 + Col::kD2Stride * b + lane_base, *reinterpret_cast<uint32_t(*)[8]>(r));
+                else tmem_ld16(tmem + Col::kD2 + Col::kD2Stride * b + lane_base, r);
                 tmem_ld_wait();
                 tc_fence_before();
                 mbar_arrive(&d2_empty[b]);
-                float f[6];
+                float f[DP];
 #pragma unroll
-                for (int o = 0; o < 6; ++o) f[o] = tok < N ? fmaxf(__uint_as_float(r[o]) + b2s[8 * m + o], 0.f) : 0.f;
-                if (tok < N) store6(kf_out + ((size_t)(bh * 3 + m) * N + tok) * 6, f);
+                for (int o = 0; o < DP; ++o) f[o] = tok < N ? fmaxf(__uint_as_float(r[o]) + b2s[16 * m + o], 0.f) : 0.f;
+                if (tok < N) store_feat<DP>(kf_out + ((size_t)(bh * NM + m) * N + tok) * DP, f);
                 if (m == 0) {
 #pragma unroll
-                    for (int o = 0; o < 6; ++o) k1[o] = f[o];
-                } else if (m == 1) {
+                    for (int o = 0; o < DP; ++o) k1[o] = f[o];
+                } else if (F == 3 && m == 1) {
+                    if constexpr (F == 3) {
 #pragma unroll
-                    for (int x = 0; x < 6; ++x)
+                        for (int x = 0; x < 6; ++x)
 #pragma unroll
-                        for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k1[x] * f[x] : fmaf(k1[x], f[y], k1[y] * f[x]);
+                            for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k1[x] * f[x] : fmaf(k1[x], f[y], k1[y] * f[x]);
+                    }
                 } else {
                     if (!mbar_wait(f_empty, (it & 1) ^ 1)) { ok = false; report_timeout(status, 807); }
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    folded_row_store(fblk, row, s12, f, std::make_integer_sequence<int, 8>{});
+                    if constexpr (F == 3) folded_row_store(fblk, row, s12, f, std::make_integer_sequence<int, 8>{});
+                    else folded_row_store2(fblk, row, k1, f, std::make_integer_sequence<int, 10>{});
                     fence_proxy_async();
                     mbar_arrive(f_full);
                 }
@@ -363,16 +417,17 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
                 if (!ok) break;
                 tc_fence_after();
                 const int piece = blockIdx.x - owner_of_work((long long)bh * T, total, G);
-                float* out = part + ((size_t)bh * smax + piece) * kMono * ld;
+                float* out = part + ((size_t)bh * smax + piece) * M::kN * ld;
                 const int g = quarter * 32 + lane;       // TMEM lane = value channel
                 if (quarter * 32 < DV) {
 #pragma unroll
-                    for (int c = 0; c < kMono / 8; ++c) {
+                    for (int c = 0; c < (M::kN + 7) / 8; ++c) {
                         uint32_t rr[8];
-                        tmem_ld8(tmem + kFkColC + lane_base + 8 * c, rr);
+                        tmem_ld8(tmem + Col::kC + lane_base + 8 * c, rr);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) out[(size_t)(8 * c + e) * ld + g] = __uint_as_float(rr[e]);
+                        for (int e = 0; e < 8; ++e)
+                            if (8 * c + e < M::kN) out[(size_t)(8 * c + e) * ld + g] = __uint_as_float(rr[e]);
                     }
                 }
                 tc_fence_before();
@@ -383,7 +438,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
     } else {
         // GELU: thread = token row x quarter of the hidden units
         const int quarter = warp & 3, prt = (warp - kFkGeluWarp0) >> 2;
-        for (int unit = 0; unit < 3 * nwork; ++unit) {
+        for (int unit = 0; unit < NM * nwork; ++unit) {
             const int b = unit & 1, par = (unit >> 1) & 1;
             if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 809); }
             if (ok && !mbar_wait(&g_free[b], par ^ 1)) { ok = false; report_timeout(status, 810); }
@@ -391,7 +446,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
             if (!ok) break;
             tc_fence_after();
             const uint32_t ta = tmem + 128 * b + ((uint32_t)(quarter * 32) << 16) + prt * HC;
-            const uint32_t tg = tmem + kFkColG + 64 * b + ((uint32_t)(quarter * 32) << 16) + prt * (HC / 2);
+            const uint32_t tg = tmem + Col::kG + 64 * b + ((uint32_t)(quarter * 32) << 16) + prt * (HC / 2);
             uint32_t r[HC];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) tmem_ld16(ta + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
@@ -433,32 +488,37 @@ inline int fused_key_grid(int BH, int N, int sm_count) {
     return (int)(total < sm_count ? total : sm_count);
 }
 
-template <int DV>
+template <int DV, int F>
 inline hla_status launch_phik_state(const Dims& D, int BH, const hla_mlp* phi_k, const void* K, const void* V, char* ws, const hla_ws_layout& L,
                                     size_t off_part, int smax, int sm_count, LaunchRec& rec) {
     CUtensorMap mapK, mapV;
     PhiMaps mk;
     PhiPtrs pk{};
     if (!make_map_bhnd(&mapK, K, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens)) return HLA_ERR_CUDA;
-    for (int f = 0; f < 3; ++f) {
+    for (int f = 0; f < MT<F>::kMaps; ++f) {
         if (!make_map_2d(&mk.w1[f], phi_k[f].W1, DV, DV, DV)) return HLA_ERR_CUDA;
         pk.b1[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b1);
         pk.W2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].W2);
         pk.b2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b2);
     }
-    if (!set_smem(tc_phik_state_kernel<DV>, FkCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    for (int f = MT<F>::kMaps; f < 3; ++f) mk.w1[f] = mk.w1[0];
+    if (!set_smem(tc_phik_state_kernel<DV, F>, FkCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     const int grid = fused_key_grid(BH, D.N, sm_count);
     rec.begin("tc_phik_state");
     // first kernel of hla_forward, and it stages the weights before its dependency wait: no overlap with what precedes it
-    launch_serial(tc_phik_state_kernel<DV>, grid, dim3(kFkThreads), FkCfg<DV>::kSmem, rec.st, mapK, mk, mapV, pk, reinterpret_cast<float*>(ws + L.kf),
+    launch_serial(tc_phik_state_kernel<DV, F>, grid, dim3(kFkThreads), FkCfg<DV, F>::kSmem, rec.st, mapK, mk, mapV, pk, reinterpret_cast<float*>(ws + L.kf),
                   reinterpret_cast<float*>(ws + off_part), D.N, BH, D.ld, smax, reinterpret_cast<int*>(ws + L.status));
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
 inline hla_status phik_state(const Dims& D, int BH, const hla_mlp* phi_k, const void* K, const void* V, char* ws, const hla_ws_layout& L,
                              size_t off_part, int smax, int sm_count, LaunchRec& rec) {
-    if (D.d == 128) return launch_phik_state<128>(D, BH, phi_k, K, V, ws, L, off_part, smax, sm_count, rec);
-    return launch_phik_state<64>(D, BH, phi_k, K, V, ws, L, off_part, smax, sm_count, rec);
+    if (D.F == 3) {
+        if (D.d == 128) return launch_phik_state<128, 3>(D, BH, phi_k, K, V, ws, L, off_part, smax, sm_count, rec);
+        return launch_phik_state<64, 3>(D, BH, phi_k, K, V, ws, L, off_part, smax, sm_count, rec);
+    }
+    if (D.d == 128) return launch_phik_state<128, 2>(D, BH, phi_k, K, V, ws, L, off_part, smax, sm_count, rec);
+    return launch_phik_state<64, 2>(D, BH, phi_k, K, V, ws, L, off_part, smax, sm_count, rec);
 }
 
 }  // namespace tc

@@ -79,18 +79,23 @@ struct PhiBwdPtrs {
 constexpr int kPbThreads = 608;
 constexpr int kPbEpiWarp0 = 3;
 
-template <int DV, int NMAPS> struct PbCfg {
+// DP = d_phi: 6 (F = 3) or 12 (F = 2).  The dp tile of a unit is [dp_hi | dp_lo] = 2 DP K columns: one K = 16 step for DP = 6 (two
+// tiles share one swizzled block at K columns 0..15 and 16..31), two steps for DP = 12 (one block per tile, K columns 0..23).
+template <int DV, int NMAPS, int DP> struct PbCfg {
     static constexpr int kXStages = 2;
     static constexpr int kXBytes = kTileTokens * DV * 2;
     static constexpr int kW1Bytes = DV * DV * 2;
-    static constexpr int kW2tBytes = (DV / 64) * 2048;           // per map: [16 K rows][DV] bf16, MN-major B operand of the dg product
+    static constexpr int kDgSteps = DP == 6 ? 1 : 2;             // K = 16 steps of the dg product
+    static constexpr int kW2tBlock = kDgSteps * 2048;            // [16 kDgSteps K rows][64 hidden] bf16
+    static constexpr int kW2tBytes = (DV / 64) * kW2tBlock;      // per map: MN-major B operand of the dg product
+    static constexpr int kDpBlocks = DP == 6 ? 1 : 2;
     static constexpr int kOffX = 0;
     static constexpr int kOffW1 = kXStages * kXBytes;            // (the dh tiles live in TMEM)
-    static constexpr int kOffDp = kOffW1 + NMAPS * kW1Bytes;     // one swizzled block = 4 dp tiles [128 tok][16] (K slices 0..3)
-    static constexpr int kOffW2t = kOffDp + kBlk;
-    // b1 is added on the tensor cores by a ninth K step of the h product: A = K columns 32..47 of the dp block (column
-    // 44 is a constant 1, never written again; the dp tiles use columns 0..31), B = the map's W2^T tile, whose K row 12
-    // holds b1 (rows 12..15 meet the zero columns 12..15 of the dp tiles in the dg product, so they are free there)
+    static constexpr int kOffDp = kOffW1 + NMAPS * kW1Bytes;     // dp tiles (see above)
+    static constexpr int kOffW2t = kOffDp + kDpBlocks * kBlk;
+    // b1 is added on the tensor cores by a ninth K step of the h product: A = K columns 32..47 of the first dp block (column
+    // 44 is a constant 1, never written again; the dp tiles use lower columns), B = the last K step of the map's W2^T
+    // tile, whose row 12 holds b1 (the rows from 2 DP on meet zero columns of the dp tiles in the dg product, so they are free there)
     static constexpr int kB1Row = 12;
     // dX staging tile (128 x DV) for a TMA store: query side and d = 64.  On the key side at d = 128 (a drain every
     // third unit) the two block-wide barriers of the staged drain cost more than the direct stores they replace
@@ -112,12 +117,12 @@ template <int DV, int NMAPS> struct PbCfg {
 // h and the dh tile are double-buffered; dg is taken into registers at the start of a unit so that the next unit's dg
 // product overlaps this unit's arithmetic; the dX accumulator of a tile is drained one unit late, straight from
 // registers to global memory.  The epilogue threads also write the dp tiles (one feature pair each, one unit ahead).
-template <int DV, int NMAPS, bool KSIDE>
+template <int DV, int NMAPS, bool KSIDE, int DP>
 __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
                                                                         const __grid_constant__ CUtensorMap mapdX, PhiBwdPtrs P,
                                                                         const float* __restrict__ feat, const float* __restrict__ dfeat,
                                                                         __nv_bfloat16* __restrict__ dX, long long rows, int N, int* status) {
-    using Cfg = PbCfg<DV, NMAPS>;
+    using Cfg = PbCfg<DV, NMAPS, DP>;
     constexpr int HC = DV / 4;
     constexpr int XST = Cfg::kXStages;
     extern __shared__ uint8_t smem_raw[];
@@ -145,13 +150,15 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     const int ntiles = (int)(t1 - t0);
     const int nunits = ntiles * NMAPS;
 
-    // W2^T stacked twice (rows 0..5 meet dp_hi, rows 6..11 meet dp_lo, rows 12..15 are zero), as an MN-major operand
-    for (int i = tid; i < NMAPS * 16 * DV; i += kPbThreads) {
-        const int m = i / (16 * DV), k = (i / DV) & 15, j = i % DV;
-        uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * 2048;
-        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) = k < 12 ? half_bf16(P.W2[m][j * 6 + (k % 6)]) : (k == Cfg::kB1Row ? P.b1[m][j] : __float2bfloat16_rn(0.f));
+    // W2^T stacked twice (rows 0..DP-1 meet dp_hi, rows DP..2DP-1 meet dp_lo, the rest is zero but for b1), as an MN-major operand
+    constexpr int kRows = 16 * Cfg::kDgSteps, kB1Abs = kRows - 16 + Cfg::kB1Row;
+    for (int i = tid; i < NMAPS * kRows * DV; i += kPbThreads) {
+        const int m = i / (kRows * DV), k = (i / DV) % kRows, j = i % DV;
+        uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * Cfg::kW2tBlock;
+        *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) =
+            k < 2 * DP ? half_bf16(P.W2[m][j * DP + (k % DP)]) : (k == kB1Abs ? P.b1[m][j] : __float2bfloat16_rn(0.f));
     }
-    for (int i = tid; i < kBlk / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < Cfg::kDpBlocks * kBlk / 16; i += kPbThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     for (int i = tid; i < kTileTokens; i += kPbThreads)      // K column 32 + kB1Row of the dp block
         *reinterpret_cast<__nv_bfloat16*>(smem + Cfg::kOffDp + sw128_off(i, 4 + Cfg::kB1Row / 8) + (Cfg::kB1Row & 7) * 2) = __float2bfloat16_rn(1.f);
@@ -207,7 +214,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
             const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp) + 64, 16, 1024);
-            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
+            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t) + (Cfg::kDgSteps - 1) * 2048, Cfg::kW2tBlock, 1024);      // the K step with the b1 row
             bool good = mbar_wait(w_full, 0);
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int it = unit / NMAPS, m = unit % NMAPS, st = it % XST, b = unit & 1;
@@ -231,7 +238,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             const uint32_t idesc_dg = idesc_bf16(128, DV, false, true);  // dg = dp (K-major) * W2^T (MN-major)
             const uint32_t idesc2 = idesc_bf16(128, DV, false, false);   // dX = dh (TMEM) * W1 as [in][hidden] (K-major)
             const uint64_t pd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp), 16, 1024);
-            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
+            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), Cfg::kW2tBlock, 1024);
             const uint64_t wd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), 16, 1024);
             bool good = mbar_wait(w_full, 0);
             // dg of `unit`; the epilogue of unit - 1 must have taken its dg into registers
@@ -240,7 +247,10 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 if (unit > 0 && !mbar_wait(dg_empty, (unit - 1) & 1)) return false;
                 if (!mbar_wait(&dp_full[slot], (unit >> 1) & 1)) return false;
                 tc_fence_after();
-                umma_bf16(tmem + 256, desc_advance(pd0, slot * 32), desc_advance(vd0, m * Cfg::kW2tBytes), idesc_dg, 0u);
+#pragma unroll
+                for (int ks = 0; ks < Cfg::kDgSteps; ++ks)      // the slot's K columns: 16 slot.. (DP = 6, one block), or block `slot` (DP = 12)
+                    umma_bf16(tmem + 256, desc_advance(pd0, (DP == 6 ? slot * 32 : slot * kBlk) + ks * 32), desc_advance(vd0, m * Cfg::kW2tBytes + ks * 2048), idesc_dg,
+                              ks > 0 ? 1u : 0u);
                 umma_commit(dg_full);
                 return true;
             };
@@ -337,7 +347,10 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         // Slot (u + 1) & 1 is free then: its last reader, the dg product of unit u - 1, completed before unit u - 1's
         // dg was read.
         const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
-        float2 fpre = make_float2(0.f, 0.f), gpre = make_float2(0.f, 0.f);
+        constexpr int NP = DP / 6;          // feature pairs per thread of parts 0..2: features 2 NP part .. 2 NP part + 2 NP - 1
+        float fpre[2 * NP], gpre[2 * NP];
+#pragma unroll
+        for (int i = 0; i < 2 * NP; ++i) fpre[i] = gpre[i] = 0.f;
         bool live_pre = false;
         int off_it = -1;          // tile whose row offset is cached in off_tile (the offset of map 0)
         size_t off_tile = 0;
@@ -350,24 +363,35 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 grow = live_pre ? grow : rows - 1;
                 if (KSIDE) {
                     const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
-                    off_tile = ((size_t)bh * NMAPS * N + n) * 6;
+                    off_tile = ((size_t)bh * NMAPS * N + n) * DP;
                 } else {
-                    off_tile = (size_t)grow * 6;
+                    off_tile = (size_t)grow * DP;
                 }
                 off_it = it;
             }
-            const size_t off = off_tile + (KSIDE ? (size_t)m * N * 6 : 0);
-            fpre = __ldg(reinterpret_cast<const float2*>(feat + off) + part);
-            gpre = __ldg(reinterpret_cast<const float2*>(dfeat + off) + part);
+            const size_t off = off_tile + (KSIDE ? (size_t)m * N * DP : 0);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 f = __ldg(reinterpret_cast<const float2*>(feat + off) + NP * part + i);
+                const float2 g = __ldg(reinterpret_cast<const float2*>(dfeat + off) + NP * part + i);
+                fpre[2 * i] = f.x; fpre[2 * i + 1] = f.y;
+                gpre[2 * i] = g.x; gpre[2 * i + 1] = g.y;
+            }
         };
-        auto dp_store = [&](int unit) {      // the pair loaded by the last dp_load goes into the tile of `unit`
+        auto dp_store = [&](int unit) {      // the pairs loaded by the last dp_load go into the tile of `unit`
             if (unit >= nunits) return;
             if (part < 3) {
-                const float d0 = (live_pre && fpre.x > 0.f) ? gpre.x : 0.f, d1 = (live_pre && fpre.y > 0.f) ? gpre.y : 0.f;
-                const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
-                const uint32_t slot = unit & 1, khi = 2 * part, klo = 6 + 2 * part;      // K indices of the pair: hi half, lo half
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(dpblk + sw128_off(row, 2 * slot + (khi >> 3)) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(dpblk + sw128_off(row, 2 * slot + (klo >> 3)) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
+                const uint32_t slot = unit & 1;
+                // DP = 6: both tiles in one block, K columns 16 slot ..; DP = 12: one block per tile
+                const uint32_t blk = dpblk + (DP == 6 ? 0u : slot * kBlk), col0 = DP == 6 ? 16 * slot : 0;
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    const float d0 = (live_pre && fpre[2 * i] > 0.f) ? gpre[2 * i] : 0.f, d1 = (live_pre && fpre[2 * i + 1] > 0.f) ? gpre[2 * i + 1] : 0.f;
+                    const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
+                    const uint32_t khi = col0 + 2 * (NP * part + i), klo = khi + DP;      // K columns of the pair: hi half, lo half
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, khi >> 3) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, klo >> 3) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
+                }
             }
             fence_proxy_async();
             mbar_arrive(&dp_full[unit & 1]);
@@ -425,9 +449,10 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-template <int DV>
+template <int DV, int F>
 inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, void* dQ,
                                       void* dK, char* ws, const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
+    constexpr int NM = MT<F>::kMaps, DP = MT<F>::kDphi;
     const long long rows = (long long)BH * D.N;
     CUtensorMap mapQ, mapK, mapdQ, mapdK;
     PhiMaps mq, mk;
@@ -439,31 +464,36 @@ inline hla_status launch_phi_backward(const Dims& D, int BH, const hla_mlp* phi_
     mq.w1[2] = mq.w1[0];
     pq.b1[0] = static_cast<const __nv_bfloat16*>(phi_q->b1);
     pq.W2[0] = static_cast<const __nv_bfloat16*>(phi_q->W2);
-    for (int f = 0; f < 3; ++f) {
+    for (int f = 0; f < NM; ++f) {
         if (!make_map_2d(&mk.w1[f], phi_k[f].W1, DV, DV, DV)) return HLA_ERR_CUDA;
         pk.b1[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b1);
         pk.W2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].W2);
     }
+    for (int f = NM; f < 3; ++f) mk.w1[f] = mk.w1[0];
     int* status = reinterpret_cast<int*>(ws + L.status);
-    if (!set_smem(tc_phi_backward_kernel<DV, 1, false>, PbCfg<DV, 1>::kSmem) || !set_smem(tc_phi_backward_kernel<DV, 3, true>, PbCfg<DV, 3>::kSmem))
+    if (!set_smem(tc_phi_backward_kernel<DV, 1, false, DP>, PbCfg<DV, 1, DP>::kSmem) || !set_smem(tc_phi_backward_kernel<DV, NM, true, DP>, PbCfg<DV, NM, DP>::kSmem))
         return HLA_ERR_CUDA;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     cudaStream_t st = rec.st;
     rec.begin("tc_phi_backward_q");
-    launch_pdl(tc_phi_backward_kernel<DV, 1, false>, grid, dim3(kPbThreads), PbCfg<DV, 1>::kSmem, st, 
+    launch_pdl(tc_phi_backward_kernel<DV, 1, false, DP>, grid, dim3(kPbThreads), PbCfg<DV, 1, DP>::kSmem, st,
         mapQ, mq, mapdQ, pq, reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), static_cast<__nv_bfloat16*>(dQ), rows, D.N, status);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_phi_backward_k");
-    launch_pdl(tc_phi_backward_kernel<DV, 3, true>, grid, dim3(kPbThreads), PbCfg<DV, 3>::kSmem, st, 
+    launch_pdl(tc_phi_backward_kernel<DV, NM, true, DP>, grid, dim3(kPbThreads), PbCfg<DV, NM, DP>::kSmem, st,
         mapK, mk, mapdK, pk, reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), static_cast<__nv_bfloat16*>(dK), rows, D.N, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
 inline hla_status phi_backward(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K, void* dQ, void* dK,
                                char* ws, const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
-    if (D.d == 128) return launch_phi_backward<128>(D, BH, phi_q, phi_k, Q, K, dQ, dK, ws, L, sm_count, rec);
-    return launch_phi_backward<64>(D, BH, phi_q, phi_k, Q, K, dQ, dK, ws, L, sm_count, rec);
+    if (D.F == 3) {
+        if (D.d == 128) return launch_phi_backward<128, 3>(D, BH, phi_q, phi_k, Q, K, dQ, dK, ws, L, sm_count, rec);
+        return launch_phi_backward<64, 3>(D, BH, phi_q, phi_k, Q, K, dQ, dK, ws, L, sm_count, rec);
+    }
+    if (D.d == 128) return launch_phi_backward<128, 2>(D, BH, phi_q, phi_k, Q, K, dQ, dK, ws, L, sm_count, rec);
+    return launch_phi_backward<64, 2>(D, BH, phi_q, phi_k, Q, K, dQ, dK, ws, L, sm_count, rec);
 }
 
 }  // namespace tc

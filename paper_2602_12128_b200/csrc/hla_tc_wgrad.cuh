@@ -24,10 +24,12 @@ constexpr int kWgThreads = 21 * 32;
 constexpr int kWgEpiWarp0 = 3, kWgSumWarp0 = 19;
 constexpr int kWgColDg = 128, kWgColW1 = 256, kWgColW2 = 384;      // TMEM columns (h at 0)
 
-template <int DV, int NMAPS> struct WgCfg {
+template <int DV, int NMAPS, int DP> struct WgCfg {
     static constexpr int kXBytes = 2 * kBlk;                     // two 64-column blocks per stage (the second stays zero for d = 64)
     static constexpr int kW1Bytes = DV * DV * 2;
-    static constexpr int kW2tBytes = (DV / 64) * 2048;           // per map: [16 K rows][DV] bf16 (rows 0..11: W2^T twice, halved; row 12: b1)
+    static constexpr int kDgSteps = DP == 6 ? 1 : 2;             // K = 16 steps of the dg product: [dp_hi | dp_lo] is 2 DP columns wide
+    static constexpr int kW2tBlock = kDgSteps * 2048;
+    static constexpr int kW2tBytes = (DV / 64) * kW2tBlock;      // per map: [16 kDgSteps K rows][DV] bf16 (W2^T twice, halved; row 12 of the last step: b1)
     static constexpr int kOffX = 0;                              // 2 stages
     static constexpr int kOffW1 = 2 * kXBytes;                   // the current map's W1
     static constexpr int kOffDp = kOffW1 + kW1Bytes;             // 3 dp blocks [128 tok][64]: K columns 0..5 dp_hi, 6..11 dp_lo; column 44 of block 0 is 1
@@ -39,16 +41,17 @@ template <int DV, int NMAPS> struct WgCfg {
     static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
     static constexpr int kB1Row = 12;
-    // one partial per (CTA, map), in floats: dW1 [DV][DV], dW2ext [DV][16], db1 [DV], db2 [4 token quarters][8]
-    static constexpr int kPartW2 = DV * DV, kPartB1 = kPartW2 + DV * 16, kPartB2 = kPartB1 + DV, kPartFloats = kPartB2 + 32;
+    // one partial per (CTA, map), in floats: dW1 [DV][DV], dW2ext [DV][kW2Cols], db1 [DV], db2 [4 token quarters][16]
+    static constexpr int kW2Cols = 16 * kDgSteps;
+    static constexpr int kPartW2 = DV * DV, kPartB1 = kPartW2 + DV * kW2Cols, kPartB2 = kPartB1 + DV, kPartFloats = kPartB2 + 64;
 };
 
 // X [rows][DV] bf16.  KSIDE: feat / dfeat are [bh][NMAPS][N][6], else [rows][6].  wpart: [gridDim.x][NMAPS][kPartFloats].
-template <int DV, int NMAPS, bool KSIDE>
+template <int DV, int NMAPS, bool KSIDE, int DP>
 __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ PhiMaps maps,
                                                                      PhiBwdPtrs P, const float* __restrict__ feat, const float* __restrict__ dfeat,
                                                                      float* __restrict__ wpart, long long rows, int N, int* status) {
-    using Cfg = WgCfg<DV, NMAPS>;
+    using Cfg = WgCfg<DV, NMAPS, DP>;
     constexpr int HC = DV / 4;
     extern __shared__ uint8_t smem_raw[];
     grid_launch_dependents();
@@ -76,11 +79,12 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
     const int nunits = ntiles * NMAPS;      // unit u = map (u / ntiles), tile (u % ntiles)
     float* out_cta = wpart + (size_t)blockIdx.x * NMAPS * Cfg::kPartFloats;
 
-    for (int i = tid; i < NMAPS * 16 * DV; i += kWgThreads) {
-        const int m = i / (16 * DV), k = (i / DV) & 15, j = i % DV;
-        uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * 2048;
+    constexpr int kRows = 16 * Cfg::kDgSteps, kB1Abs = kRows - 16 + Cfg::kB1Row;
+    for (int i = tid; i < NMAPS * kRows * DV; i += kWgThreads) {
+        const int m = i / (kRows * DV), k = (i / DV) % kRows, j = i % DV;
+        uint8_t* base = smem + Cfg::kOffW2t + m * Cfg::kW2tBytes + (j >> 6) * Cfg::kW2tBlock;
         *reinterpret_cast<__nv_bfloat16*>(base + sw128_off(k, (j & 63) >> 3) + (j & 7) * 2) =
-            k < 12 ? half_bf16(P.W2[m][j * 6 + (k % 6)]) : (k == Cfg::kB1Row ? P.b1[m][j] : __float2bfloat16_rn(0.f));
+            k < 2 * DP ? half_bf16(P.W2[m][j * DP + (k % DP)]) : (k == kB1Abs ? P.b1[m][j] : __float2bfloat16_rn(0.f));
     }
     for (int i = tid; i < 3 * kBlk / 16; i += kWgThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffDp)[i] = make_uint4(0, 0, 0, 0);
     for (int i = tid; i < 2 * Cfg::kXBytes / 16; i += kWgThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffX)[i] = make_uint4(0, 0, 0, 0);
@@ -140,7 +144,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             const uint64_t xd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffX), 16, 1024);
             const uint64_t wd = smem_desc_sw128(smem_u32(smem + Cfg::kOffW1), DV * 128, 1024);
             const uint64_t od = smem_desc_sw128(smem_u32(smem + Cfg::kOffDp) + 64, 16, 1024);
-            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
+            const uint64_t bd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t) + (Cfg::kDgSteps - 1) * 2048, Cfg::kW2tBlock, 1024);      // the K step with the b1 row
             bool good = true;
             for (int unit = 0; unit < nunits && good; ++unit) {
                 const int m = unit / ntiles, it = unit - m * ntiles, st = unit & 1;
@@ -163,14 +167,17 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             const uint32_t idesc_w2 = idesc_bf16(128, 64, true, true);    // dW2ext = G^T (MN-major, M = hidden) * dp block (MN-major, N = 64)
             const uint32_t dpa = smem_u32(smem + Cfg::kOffDp), xa = smem_u32(smem + Cfg::kOffX);
             const uint32_t ga = smem_u32(smem + Cfg::kOffG), da = smem_u32(smem + Cfg::kOffDh);
-            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), 2048, 1024);
+            const uint64_t vd0 = smem_desc_sw128(smem_u32(smem + Cfg::kOffW2t), Cfg::kW2tBlock, 1024);
             bool good = true;
             auto issue_dg = [&](int unit) -> bool {      // the arithmetic warps of unit - 1 must have taken their dg into registers
                 const int m = unit / ntiles;
                 if (unit > 0 && !mbar_wait(dg_empty, (unit - 1) & 1)) return false;
                 if (!mbar_wait(&dp_full[unit % 3], (unit / 3) & 1)) return false;
                 tc_fence_after();
-                umma_bf16(tmem + kWgColDg, smem_desc_sw128(dpa + (unit % 3) * kBlk, 16, 1024), desc_advance(vd0, m * Cfg::kW2tBytes), idesc_dg, 0u);
+#pragma unroll
+                for (int ks = 0; ks < Cfg::kDgSteps; ++ks)
+                    umma_bf16(tmem + kWgColDg, smem_desc_sw128(dpa + (unit % 3) * kBlk + ks * 32, 16, 1024), desc_advance(vd0, m * Cfg::kW2tBytes + ks * 2048), idesc_dg,
+                              ks > 0 ? 1u : 0u);
                 umma_commit(dg_full);
                 return true;
             };
@@ -240,9 +247,11 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
         // dp = dfeat (.) 1[feat > 0] as [dp_hi | dp_lo] (two bf16 halves, so dg is exact to ~2^-17): every thread of parts 0..2
         // owns one pair of features of its row, loads it two units ahead and writes the tile of unit u + 1 at the start of
         // unit u.  Block (u + 1) % 3 is free then: its last readers, the products of unit u - 2, were waited for in unit u - 1.
-        float2 fpre = make_float2(0.f, 0.f), gpre = make_float2(0.f, 0.f);
+        constexpr int NP = DP / 6;          // feature pairs per thread of parts 0..2
+        float fpre[2 * NP], gpre[2 * NP], b2s[2 * NP];      // b2s: db2 of this thread's features, summed over its tokens of the current map
+#pragma unroll
+        for (int i = 0; i < 2 * NP; ++i) fpre[i] = gpre[i] = b2s[i] = 0.f;
         bool live_pre = false;
-        float b2a = 0.f, b2b = 0.f;      // db2: this thread's pair, summed over its tokens of the current map
         auto dp_load = [&](int unit) {
             if (part == 3 || unit >= nunits) return;
             const int m = unit / ntiles, it = unit - m * ntiles;
@@ -252,39 +261,51 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             size_t off;
             if (KSIDE) {
                 const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
-                off = (((size_t)bh * NMAPS + m) * N + n) * 6;
+                off = (((size_t)bh * NMAPS + m) * N + n) * DP;
             } else {
-                off = (size_t)grow * 6;
+                off = (size_t)grow * DP;
             }
-            fpre = __ldg(reinterpret_cast<const float2*>(feat + off) + part);
-            gpre = __ldg(reinterpret_cast<const float2*>(dfeat + off) + part);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float2 f = __ldg(reinterpret_cast<const float2*>(feat + off) + NP * part + i);
+                const float2 g = __ldg(reinterpret_cast<const float2*>(dfeat + off) + NP * part + i);
+                fpre[2 * i] = f.x; fpre[2 * i + 1] = f.y;
+                gpre[2 * i] = g.x; gpre[2 * i + 1] = g.y;
+            }
         };
-        auto dp_store = [&](int unit) {      // the pair loaded by the last dp_load goes into the tile of `unit`
+        auto dp_store = [&](int unit) {      // the pairs loaded by the last dp_load go into the tile of `unit`
             if (unit >= nunits) return;
             if (part < 3) {
-                const float d0 = (live_pre && fpre.x > 0.f) ? gpre.x : 0.f, d1 = (live_pre && fpre.y > 0.f) ? gpre.y : 0.f;
-                const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
-                const uint32_t blk = dpblk + (unit % 3) * kBlk, khi = 2 * part, klo = 6 + 2 * part;      // K indices of the pair: hi half, lo half
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, khi >> 3) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, klo >> 3) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
-                if (unit % ntiles == 0) b2a = b2b = 0.f;
-                b2a += d0;
-                b2b += d1;
+                const uint32_t blk = dpblk + (unit % 3) * kBlk;
+                if (unit % ntiles == 0) {
+#pragma unroll
+                    for (int i = 0; i < 2 * NP; ++i) b2s[i] = 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    const float d0 = (live_pre && fpre[2 * i] > 0.f) ? gpre[2 * i] : 0.f, d1 = (live_pre && fpre[2 * i + 1] > 0.f) ? gpre[2 * i + 1] : 0.f;
+                    const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
+                    const uint32_t khi = 2 * (NP * part + i), klo = khi + DP;      // K columns of the pair: hi half, lo half
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, khi >> 3) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, klo >> 3) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
+                    b2s[2 * i] += d0;
+                    b2s[2 * i + 1] += d1;
+                }
             }
             fence_proxy_async();
             mbar_arrive(&dp_full[unit % 3]);
         };
         // db2 partial of map m: this warp's 32 tokens summed by shuffles, one partial per token quarter
         auto flush_db2 = [&](int m) {
+            float* o = out_cta + (size_t)m * Cfg::kPartFloats + Cfg::kPartB2 + quarter * 16;
             if (part < 3) {
-                const float a = warp_sum(b2a), b = warp_sum(b2b);
-                if (lane == 0) {
-                    float* o = out_cta + (size_t)m * Cfg::kPartFloats + Cfg::kPartB2 + quarter * 8 + 2 * part;
-                    o[0] = a;
-                    o[1] = b;
+#pragma unroll
+                for (int i = 0; i < 2 * NP; ++i) {
+                    const float a = warp_sum(b2s[i]);
+                    if (lane == 0) o[2 * NP * part + i] = a;
                 }
-            } else if (lane < 2) {
-                out_cta[(size_t)m * Cfg::kPartFloats + Cfg::kPartB2 + quarter * 8 + 6 + lane] = 0.f;
+            } else if (lane < 16 - 6 * NP) {
+                o[6 * NP + lane] = 0.f;
             }
         };
         dp_load(0);
@@ -358,13 +379,16 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
                             dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
                     }
                     if (part == 0) {
-                        uint32_t r[16];
-                        tmem_ld16(tmem + kWgColW2 + lane_base, r);
-                        tmem_ld_wait();
-                        float4* dst = reinterpret_cast<float4*>(o + Cfg::kPartW2 + (size_t)row * 16);
 #pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                        for (int c = 0; c < Cfg::kW2Cols / 16; ++c) {
+                            uint32_t r[16];
+                            tmem_ld16(tmem + kWgColW2 + lane_base + 16 * c, r);
+                            tmem_ld_wait();
+                            float4* dst = reinterpret_cast<float4*>(o + Cfg::kPartW2 + (size_t)row * Cfg::kW2Cols + 16 * c);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)
+                                dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                        }
                     }
                 }
                 tc_fence_before();
@@ -385,13 +409,14 @@ struct WgradOut {
     float* dW2[4];
     float* db2[4];
 };
-template <int DV>
+template <int DV, int DP>
 __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __restrict__ wpart, WgradOut out, int nmaps_in_part, int map0, int nctas) {
-    constexpr int PF = WgCfg<DV, 1>::kPartFloats, oW2 = WgCfg<DV, 1>::kPartW2, oB1 = WgCfg<DV, 1>::kPartB1, oB2 = WgCfg<DV, 1>::kPartB2;
+    using C1 = WgCfg<DV, 1, DP>;
+    constexpr int PF = C1::kPartFloats, oW2 = C1::kPartW2, oB1 = C1::kPartB1, oB2 = C1::kPartB2, W2C = C1::kW2Cols;
     grid_launch_dependents();
     grid_dependency_wait();
-    const int m = blockIdx.y;                      // map of this launch
-    const int total = DV * DV + DV * 6 + DV + 6;   // outputs of one map
+    const int m = blockIdx.y;                        // map of this launch
+    const int total = DV * DV + DV * DP + DV + DP;   // outputs of one map
     for (int i = blockIdx.x * 256 + threadIdx.x; i < total; i += gridDim.x * 256) {
         const float* src = wpart + (size_t)m * PF;
         const size_t stride = (size_t)nmaps_in_part * PF;
@@ -399,18 +424,18 @@ __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __res
         if (i < DV * DV) {
             for (int c = 0; c < nctas; ++c) a += src[c * stride + i];
             out.dW1[map0 + m][i] = a;
-        } else if (i < DV * DV + DV * 6) {
-            const int j = (i - DV * DV) / 6, o = (i - DV * DV) % 6;
-            for (int c = 0; c < nctas; ++c) a += src[c * stride + oW2 + j * 16 + o] + src[c * stride + oW2 + j * 16 + 6 + o];
-            out.dW2[map0 + m][j * 6 + o] = 0.5f * a;      // the G tile held 2 GELU(h)
-        } else if (i < DV * DV + DV * 6 + DV) {
-            const int j = i - DV * DV - DV * 6;
+        } else if (i < DV * DV + DV * DP) {
+            const int j = (i - DV * DV) / DP, o = (i - DV * DV) % DP;
+            for (int c = 0; c < nctas; ++c) a += src[c * stride + oW2 + j * W2C + o] + src[c * stride + oW2 + j * W2C + DP + o];
+            out.dW2[map0 + m][j * DP + o] = 0.5f * a;      // the G tile held 2 GELU(h)
+        } else if (i < DV * DV + DV * DP + DV) {
+            const int j = i - DV * DV - DV * DP;
             for (int c = 0; c < nctas; ++c) a += src[c * stride + oB1 + j];
             out.db1[map0 + m][j] = a;
         } else {
-            const int o = i - DV * DV - DV * 6 - DV;
+            const int o = i - DV * DV - DV * DP - DV;
             for (int c = 0; c < nctas; ++c)
-                for (int q = 0; q < 4; ++q) a += src[c * stride + oB2 + q * 8 + o];
+                for (int q = 0; q < 4; ++q) a += src[c * stride + oB2 + q * 16 + o];
             out.db2[map0 + m][o] = a;
         }
     }
@@ -419,15 +444,16 @@ __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __res
 inline size_t wgrad_part_bytes(int d, long long rows, int sm_count) {
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    const size_t pf = d == 128 ? WgCfg<128, 1>::kPartFloats : WgCfg<64, 1>::kPartFloats;
-    return (size_t)grid * 3 * pf * 4;      // the key side's three maps share one launch; the query side reuses the region
+    const size_t pf = d == 128 ? WgCfg<128, 1, 12>::kPartFloats : WgCfg<64, 1, 12>::kPartFloats;      // the larger of the two geometries
+    return (size_t)grid * 3 * pf * 4;      // the key side's maps share one launch; the query side reuses the region
 }
 
-// dphi_q / dphi_k: fp32 device outputs with the shapes of the weights (dphi_k points to three entries); either may be null.
-template <int DV>
+// dphi_q / dphi_k: fp32 device outputs with the shapes of the weights (dphi_k points to one entry per key map); either may be null.
+template <int DV, int F>
 inline hla_status launch_phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K,
                                    const hla_mlp_grad* dphi_q, const hla_mlp_grad* dphi_k, char* ws, const hla_ws_layout& L, size_t off_wpart,
                                    int sm_count, LaunchRec& rec) {
+    constexpr int NM = MT<F>::kMaps, DP = MT<F>::kDphi;
     const long long rows = (long long)BH * D.N;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
@@ -443,16 +469,16 @@ inline hla_status launch_phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, 
         mq.w1[2] = mq.w1[0];
         pq.b1[0] = static_cast<const __nv_bfloat16*>(phi_q->b1);
         pq.W2[0] = static_cast<const __nv_bfloat16*>(phi_q->W2);
-        if (!set_smem(tc_phi_wgrad_kernel<DV, 1, false>, WgCfg<DV, 1>::kSmem)) return HLA_ERR_CUDA;
+        if (!set_smem(tc_phi_wgrad_kernel<DV, 1, false, DP>, WgCfg<DV, 1, DP>::kSmem)) return HLA_ERR_CUDA;
         rec.begin("tc_phi_wgrad_q");
-        launch_serial(tc_phi_wgrad_kernel<DV, 1, false>, grid, dim3(kWgThreads), WgCfg<DV, 1>::kSmem, st, mapQ, mq, pq,
+        launch_serial(tc_phi_wgrad_kernel<DV, 1, false, DP>, grid, dim3(kWgThreads), WgCfg<DV, 1, DP>::kSmem, st, mapQ, mq, pq,
                       reinterpret_cast<const float*>(ws + L.qf), reinterpret_cast<const float*>(ws + L.dqf), wpart, rows, D.N, status);
         if (!rec.end()) return HLA_ERR_CUDA;
         WgradOut o{};
         o.dW1[0] = static_cast<float*>(dphi_q->dW1); o.db1[0] = static_cast<float*>(dphi_q->db1);
         o.dW2[0] = static_cast<float*>(dphi_q->dW2); o.db2[0] = static_cast<float*>(dphi_q->db2);
         rec.begin("tc_wgrad_reduce");
-        launch_pdl(tc_wgrad_reduce_kernel<DV>, dim3(32, 1), dim3(256), 0, st, (const float*)wpart, o, 1, 0, grid);
+        launch_pdl(tc_wgrad_reduce_kernel<DV, DP>, dim3(32, 1), dim3(256), 0, st, (const float*)wpart, o, 1, 0, grid);
         if (!rec.end()) return HLA_ERR_CUDA;
     }
     if (dphi_k) {
@@ -461,22 +487,23 @@ inline hla_status launch_phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, 
         PhiBwdPtrs pk{};
         if (!make_map_2d(&mapK, K, (size_t)rows, DV, kTileTokens)) return HLA_ERR_CUDA;
         WgradOut o{};
-        for (int f = 0; f < 3; ++f) {
+        for (int f = 0; f < NM; ++f) {
             if (!make_map_2d(&mk.w1[f], phi_k[f].W1, DV, DV, DV)) return HLA_ERR_CUDA;
             pk.b1[f] = static_cast<const __nv_bfloat16*>(phi_k[f].b1);
             pk.W2[f] = static_cast<const __nv_bfloat16*>(phi_k[f].W2);
             o.dW1[f] = static_cast<float*>(dphi_k[f].dW1); o.db1[f] = static_cast<float*>(dphi_k[f].db1);
             o.dW2[f] = static_cast<float*>(dphi_k[f].dW2); o.db2[f] = static_cast<float*>(dphi_k[f].db2);
         }
-        if (!set_smem(tc_phi_wgrad_kernel<DV, 3, true>, WgCfg<DV, 3>::kSmem)) return HLA_ERR_CUDA;
+        for (int f = NM; f < 3; ++f) mk.w1[f] = mk.w1[0];
+        if (!set_smem(tc_phi_wgrad_kernel<DV, NM, true, DP>, WgCfg<DV, NM, DP>::kSmem)) return HLA_ERR_CUDA;
         rec.begin("tc_phi_wgrad_k");
         // it stages caller-provided weights before its dependency wait, and the reduction before it still reads the
         // partial region: no overlap with what precedes it
-        launch_serial(tc_phi_wgrad_kernel<DV, 3, true>, grid, dim3(kWgThreads), WgCfg<DV, 3>::kSmem, st, mapK, mk, pk,
+        launch_serial(tc_phi_wgrad_kernel<DV, NM, true, DP>, grid, dim3(kWgThreads), WgCfg<DV, NM, DP>::kSmem, st, mapK, mk, pk,
                       reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), wpart, rows, D.N, status);
         if (!rec.end()) return HLA_ERR_CUDA;
         rec.begin("tc_wgrad_reduce");
-        launch_pdl(tc_wgrad_reduce_kernel<DV>, dim3(32, 3), dim3(256), 0, st, (const float*)wpart, o, 3, 0, grid);
+        launch_pdl(tc_wgrad_reduce_kernel<DV, DP>, dim3(32, NM), dim3(256), 0, st, (const float*)wpart, o, NM, 0, grid);
         if (!rec.end()) return HLA_ERR_CUDA;
     }
     return HLA_OK;
@@ -485,8 +512,12 @@ inline hla_status launch_phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, 
 inline hla_status phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, const hla_mlp* phi_k, const void* Q, const void* K,
                             const hla_mlp_grad* dphi_q, const hla_mlp_grad* dphi_k, char* ws, const hla_ws_layout& L, size_t off_wpart, int sm_count,
                             LaunchRec& rec) {
-    if (D.d == 128) return launch_phi_wgrad<128>(D, BH, phi_q, phi_k, Q, K, dphi_q, dphi_k, ws, L, off_wpart, sm_count, rec);
-    return launch_phi_wgrad<64>(D, BH, phi_q, phi_k, Q, K, dphi_q, dphi_k, ws, L, off_wpart, sm_count, rec);
+    if (D.F == 3) {
+        if (D.d == 128) return launch_phi_wgrad<128, 3>(D, BH, phi_q, phi_k, Q, K, dphi_q, dphi_k, ws, L, off_wpart, sm_count, rec);
+        return launch_phi_wgrad<64, 3>(D, BH, phi_q, phi_k, Q, K, dphi_q, dphi_k, ws, L, off_wpart, sm_count, rec);
+    }
+    if (D.d == 128) return launch_phi_wgrad<128, 2>(D, BH, phi_q, phi_k, Q, K, dphi_q, dphi_k, ws, L, off_wpart, sm_count, rec);
+    return launch_phi_wgrad<64, 2>(D, BH, phi_q, phi_k, Q, K, dphi_q, dphi_k, ws, L, off_wpart, sm_count, rec);
 }
 
 }  // namespace tc

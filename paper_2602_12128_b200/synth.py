@@ -48,6 +48,10 @@ CONFIGS["paper_r1_bf16"] = HlaShape("paper_r1_bf16", 1, 12, 32760, 128, "bf16", 
 CONFIGS["paper_r2_bf16"] = HlaShape("paper_r2_bf16", 1, 12, 12600, 128, "bf16", "rms_qk", backward=True)
 
 
+# The paper's 2-factor variant (appendix "Defining phi": 12 feature channels for 2 factors; Table 2 row HLA-2F-R1-21) at the training-step shape.
+CONFIGS["train_bf16_2f"] = HlaShape("train_bf16_2f", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=True, F=2, d_phi=12)
+
+
 def bf16_round(x: np.ndarray) -> np.ndarray:
     """Round float32 values to the nearest bfloat16 (ties to even); result stays float32."""
     x = np.ascontiguousarray(x, dtype=np.float32)

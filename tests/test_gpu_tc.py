@@ -187,6 +187,58 @@ def test_full_backward_bf16_mlp_stagewise():
     assert run.op.launches() == 5
 
 
+@pytest.mark.parametrize("d,N,B,H", [(128, 1500, 2, 2), (64, 700, 1, 3), (128, 100, 1, 1)])
+def test_two_factor_variant_with_the_phi_maps_stagewise(d, N, B, H):
+    """The paper's 2-factor variant (two key maps, d_phi = 12) on the tensor-core kernels with the phi maps: every stage of
+    the forward, the backward and the weight gradients against the oracle run on that stage's actual inputs."""
+    s = synth.HlaShape("t", B, H, N, d, "bf16", "rms_qk", True, 2, 12)
+    Q, K, V = synth.make_qkv(s)
+    dO = synth.make_dO(s)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    assert len(pk) == 2 and pq[2].shape == (d, 12)
+    run = DeviceRun(s, "mlp", EPS)
+    assert run.op.layout.tensor_core == 1 and run.op.layout.state_rows == 78
+    run.set_weights(pq, pk)
+    O = run.forward(Q, K, V)
+    assert run.op.launches() == 3
+    f64 = lambda a: a.astype(np.float64)
+    gq, gk = run.features()
+    _, _, qf, kf = orc.hla_forward(f64(Q), f64(K), f64(V), pq, pk, EPS, "factored")
+    assert relerr(gq, qf) < TOL["bf16"] and relerr(gk, kf) < TOL["bf16"]
+    Oc, eta = orc.hla_core_forward(gq, gk, f64(V), EPS, "quadratic" if N <= 1500 else "factored")
+    assert relerr(O, Oc) < TOL["bf16"], relerr(O, Oc)
+    assert relerr(run.eta(), eta) < TOL["bf16"] / 4
+    dQ, dK, dV = run.backward(dO)
+    assert run.op.launches() == 5
+    nq = s.B * s.H * s.N * s.d_phi
+    dqf = run.region("dqf", nq, (s.B, s.H, s.N, s.d_phi))
+    dkf = run.region("dkf", nq * s.F, (s.B, s.H, s.F, s.N, s.d_phi))
+    rq, rk, rv = orc.hla_core_backward(gq, gk, f64(V), f64(dO), EPS, "factored")
+    assert relerr(dV, rv) < TOL["bf16"] and relerr(dqf, rq) < TOL["bf16"] and relerr(dkf, rk) < TOL["bf16"]
+    rQ = orc.phi_mlp_backward(f64(Q).reshape(-1, d), *pq, dqf.reshape(-1, s.d_phi)).reshape(Q.shape)
+    rK = sum(orc.phi_mlp_backward(f64(K).reshape(-1, d), *pk[f], dkf[:, :, f].reshape(-1, s.d_phi)).reshape(K.shape) for f in range(s.F))
+    pre_q = orc.phi_mlp(f64(Q).reshape(-1, d), *pq, relu=False).reshape(gq.shape)
+    pre_k = np.stack([orc.phi_mlp(f64(K).reshape(-1, d), *w, relu=False).reshape(gq.shape) for w in pk], axis=2)
+    flip_q, flip_k = (gq > 0) != (pre_q > 0), (gk > 0) != (pre_k > 0)
+    assert flip_q.mean() < 5e-3 and flip_k.mean() < 5e-3
+    same_q, same_k = ~flip_q.any(axis=-1), ~flip_k.any(axis=(2, 4))
+    assert relerr(dQ[same_q], rQ[same_q]) < TOL["bf16"], relerr(dQ[same_q], rQ[same_q])
+    assert relerr(dK[same_k], rK[same_k]) < TOL["bf16"], relerr(dK[same_k], rK[same_k])
+    # weight gradients of the three maps at the masked feature gradients the GPU used
+    wq, wk = run.op.backward_weights(run.Q, run.K)
+    torch.cuda.synchronize()
+    assert run.op.device_status() == binding.HLA_OK
+    sides = [(Q, pq, gq, dqf, wq)] + [(K, pk[f], gk[:, :, f], dkf[:, :, f], wk[f]) for f in range(s.F)]
+    for X, w, feat, dfeat, got in sides:
+        acc = None
+        for b in range(B):
+            for h in range(H):
+                g = orc.phi_mlp_backward_weights(f64(X[b, h]), *w, f64(dfeat[b, h]) * (feat[b, h] > 0), relu=False)
+                acc = g if acc is None else tuple(a + c for a, c in zip(acc, g))
+        for t, ref in zip(got, acc):
+            assert relerr(t.float().cpu().numpy(), ref) < TOL["bf16"]
+
+
 def test_bounded_wait_reports_timeout_and_context_stays_usable():
     """Failure detection without a fault: a wait that nothing satisfies runs out after its limit, the kernel returns,
     the host reads HLA_ERR_DEVICE_TIMEOUT, and the same context computes a correct forward afterwards."""
