@@ -65,9 +65,9 @@ typedef enum {
  * Problem statement.  V, O, dO, dV (and Q, K, dQ, dK in HLA_PHI_MLP mode) are
  * [B,H,N,d] in `dtype`.  Features (HLA_PHI_NONE inputs and their gradients) are
  * always fp32.  Supported set: F in {1,2,3,4}, d_phi^F <= 256, d <= 128 and
- * d % 4 == 0, causal == 0.  dtype bf16 with d in {64,128}, F = 3, d_phi = 6 and
- * B*H*N < 2^31 runs on the tensor-core kernels; everything else in the
- * supported set (F = 2 with d_phi = 12 included) runs on the fp32 SIMT kernels.
+ * d % 4 == 0, causal == 0.  dtype bf16 with d in {64,128}, (F, d_phi) = (3, 6) or
+ * (2, 12) - the paper's two variants - and B*H*N < 2^31 runs on the tensor-core
+ * kernels; everything else in the supported set runs on the fp32 SIMT kernels.
  */
 typedef struct {
     int32_t B, H, N, d;
