@@ -23,8 +23,9 @@ Two independent forms of the same operator are implemented:
     per-token outer-product tensors T_k, T_q, the context tensor C = T_k (x)_1 V,
     the key-side sum z, eta = T_q . z, and the readout T_q (x) C;
 
-plus the sequential-update recurrence (Eq. "seq.updates") for the state, analytic
-gradients in both forms, and the feature networks phi of the appendix
+plus the sequential-update recurrence (Eq. "seq.updates") for the state, causal HLA
+(Section 4.4) as the masked quadratic definition and as the sequential recurrence
+with one output per token, analytic gradients in every form, and the feature networks phi of the appendix
 ("Defining phi": Linear - GELU - Linear - optional ReLU).
 
 Readings of points the paper leaves open (the same readings the CUDA library
@@ -38,6 +39,10 @@ takes):
   * In the theorem's proof the summed token index is the key/value index j.
   * The P = d_phi**F features of a token are flattened with the FIRST factor's
     index slowest (the listings' `bhsdef -> view(dp**3)`).
+  * Causal HLA (Section 4.4): the text speaks of multiplying an n x n {0,1} matrix M "to the keys"; the sequential
+    form it then gives (C^i holds tokens 1..i and is read by T_q^i) fixes the meaning: A_ij is kept for j <= i, the
+    diagonal included, and the normaliser sums the kept entries.  Decay factors (a non-binary M) are cited, not
+    defined, and are not implemented.
   * Value modulation (Section 4.5; appendix "Defining phi"): the text fixes T + phi_v1(T) (.) phi_v2(V), two
     Linear layers of width d with a GELU in between, no final activation, and says only that phi_v1, phi_v2 "use a
     LayerNorm".  Reading taken here: the LayerNorm acts on the input of each map (over the d channels of a
@@ -287,10 +292,133 @@ def hla_factored_backward(q, ks, v, do, eps):
 
 
 # --------------------------------------------------------------------------- #
+# Causal HLA (Section 4.4 "Causal Attention, Decay Factors and Sequential
+# Updates", Eq. "seq.updates")
+# --------------------------------------------------------------------------- #
+def causal_mask(n):
+    """M in {0,1}^{n x n}: token i sees tokens j <= i (itself included)."""
+    return np.tril(np.ones((n, n), F64))
+
+
+def hla_quadratic_causal(q, ks, v, eps):
+    """The definition with the {0,1} mask applied to the Hadamard product:
+    A_ij = M_ij prod_f s^f_ij,  o_i = (sum_j A_ij v_j) / (sum_j A_ij + eps).  Returns (o, eta)."""
+    A = attention_matrix(q, ks) * causal_mask(np.asarray(q).shape[0])
+    eta = A.sum(axis=1)
+    num = A @ np.asarray(v, F64)
+    return num / (eta + eps)[:, None], eta
+
+
+def hla_streaming(q, ks, v, eps):
+    """Sequential updates: at token i the context tensor takes C^i = C^{i-1} + T_{k_i} (x) v_i (and the key-side sum
+    z^i = z^{i-1} + T_{k_i}), and the output of that token is the product of T_q^i with C^i, normalised by
+    T_q^i . z^i + eps.  Returns (o, eta)."""
+    Fn = len(ks)
+    Tk = outer_features(ks)
+    Tq = outer_features([q] * Fn)
+    v = np.asarray(v, F64)
+    n = Tk.shape[0]
+    C = np.zeros((Tk.shape[1], v.shape[1]), F64)
+    z = np.zeros(Tk.shape[1], F64)
+    o = np.empty((n, v.shape[1]), F64)
+    eta = np.empty(n, F64)
+    for i in range(n):
+        C = C + np.multiply.outer(Tk[i], v[i])
+        z = z + Tk[i]
+        eta[i] = Tq[i] @ z
+        o[i] = (Tq[i] @ C) / (eta[i] + eps)
+    return o, eta
+
+
+def hla_quadratic_causal_backward(q, ks, v, do, eps):
+    """Gradients of L = sum(do * o) through the masked quadratic form.  Returns (dq, dks, dv)."""
+    q = np.asarray(q, F64)
+    ks = [np.asarray(k, F64) for k in ks]
+    v = np.asarray(v, F64)
+    do = np.asarray(do, F64)
+    M = causal_mask(q.shape[0])
+    s = similarity_matrices(q, ks)
+    A = attention_matrix(q, ks) * M
+    eta = A.sum(axis=1)
+    r = 1.0 / (eta + eps)
+    o = (A @ v) * r[:, None]
+    # dL/dA_ij = r_i * do_i . (v_j - o_i) where the mask lets A_ij vary, 0 elsewhere
+    dA = M * (r[:, None] * (do @ v.T - np.sum(do * o, axis=1)[:, None]))
+    dv = (A * r[:, None]).T @ do
+    dq = np.zeros_like(q)
+    dks = []
+    for f in range(len(ks)):
+        others = np.ones_like(A)
+        for f2 in range(len(ks)):
+            if f2 != f:
+                others = others * s[f2]
+        ds = dA * others
+        dq += ds @ ks[f]
+        dks.append(ds.T @ q)
+    return dq, dks, dv
+
+
+def hla_streaming_backward(q, ks, v, do, eps):
+    """Gradients of L = sum(do * o) through the sequential form: a forward sweep that carries C^i, z^i for the
+    query-side gradients, and a reverse sweep that carries the gradient of the state (token j's key tensor enters
+    every C^i with i >= j, so it collects dC^j = sum_{i >= j} T_q^i (x) dnum_i).  Returns (dq, dks, dv)."""
+    q = np.asarray(q, F64)
+    ks = [np.asarray(k, F64) for k in ks]
+    v = np.asarray(v, F64)
+    do = np.asarray(do, F64)
+    Fn = len(ks)
+    Tk = outer_features(ks)
+    Tq = outer_features([q] * Fn)
+    n, P = Tk.shape
+    C = np.zeros((P, v.shape[1]), F64)
+    z = np.zeros(P, F64)
+    dTq = np.empty((n, P), F64)
+    dnum = np.empty_like(v)
+    deta = np.empty(n, F64)
+    for i in range(n):
+        C = C + np.multiply.outer(Tk[i], v[i])
+        z = z + Tk[i]
+        r = 1.0 / (Tq[i] @ z + eps)
+        o = (Tq[i] @ C) * r
+        dnum[i] = do[i] * r
+        deta[i] = -r * (do[i] @ o)
+        dTq[i] = C @ dnum[i] + deta[i] * z
+    dC = np.zeros_like(C)
+    dz = np.zeros(P, F64)
+    dTk = np.empty((n, P), F64)
+    dv = np.empty_like(v)
+    for i in range(n - 1, -1, -1):
+        dC = dC + np.multiply.outer(Tq[i], dnum[i])
+        dz = dz + deta[i] * Tq[i]
+        dv[i] = Tk[i] @ dC
+        dTk[i] = dC @ v[i] + dz
+    dq = np.zeros_like(q)
+    for slot in range(Fn):
+        dq += _slot_contract(dTq, [q] * Fn, slot)
+    dks = [_slot_contract(dTk, ks, f) for f in range(Fn)]
+    return dq, dks, dv
+
+
+_FORWARD_FORMS = {
+    "quadratic": lambda q, ks, v, eps: hla_quadratic(q, ks, v, eps),
+    "factored": lambda q, ks, v, eps: hla_factored(q, ks, v, eps)[:2],
+    "causal_quadratic": lambda q, ks, v, eps: hla_quadratic_causal(q, ks, v, eps),
+    "causal_streaming": lambda q, ks, v, eps: hla_streaming(q, ks, v, eps),
+}
+
+
+def _backward_form(form):
+    return {"quadratic": hla_quadratic_backward, "factored": hla_factored_backward,
+            "causal_quadratic": hla_quadratic_causal_backward,
+            "causal_streaming": hla_streaming_backward}[form]
+
+
+# --------------------------------------------------------------------------- #
 # Whole-operator wrappers over [B, H, N, *] tensors (Algorithm 1 steps 4-5)
 # --------------------------------------------------------------------------- #
 def hla_core_forward(qf, kf, V, eps, form="factored"):
-    """qf [B,H,N,d_phi], kf [B,H,F,N,d_phi], V [B,H,N,d] -> (O [B,H,N,d], eta [B,H,N])."""
+    """qf [B,H,N,d_phi], kf [B,H,F,N,d_phi], V [B,H,N,d] -> (O [B,H,N,d], eta [B,H,N]).
+    form: "factored" | "quadratic" (all tokens see all tokens), "causal_quadratic" | "causal_streaming"."""
     B, H, N, _ = qf.shape
     Fn = kf.shape[2]
     O = np.empty(V.shape, F64)
@@ -298,10 +426,7 @@ def hla_core_forward(qf, kf, V, eps, form="factored"):
     for b in range(B):
         for h in range(H):
             ks = [kf[b, h, f] for f in range(Fn)]
-            if form == "quadratic":
-                o, eta = hla_quadratic(qf[b, h], ks, V[b, h], eps)
-            else:
-                o, eta, _, _ = hla_factored(qf[b, h], ks, V[b, h], eps)
+            o, eta = _FORWARD_FORMS[form](qf[b, h], ks, V[b, h], eps)
             O[b, h] = o
             ETA[b, h] = eta
     return O, ETA
@@ -314,7 +439,7 @@ def hla_core_backward(qf, kf, V, dO, eps, form="factored"):
     dqf = np.empty(qf.shape, F64)
     dkf = np.empty(kf.shape, F64)
     dV = np.empty(V.shape, F64)
-    fn = hla_quadratic_backward if form == "quadratic" else hla_factored_backward
+    fn = _backward_form(form)
     for b in range(B):
         for h in range(H):
             ks = [kf[b, h, f] for f in range(Fn)]

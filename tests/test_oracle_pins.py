@@ -233,6 +233,145 @@ def test_backward_forms_agree_and_scale_identities():
     np.testing.assert_allclose(g1[2].sum(axis=0), do.sum(axis=0), rtol=1e-10)
 
 
+# ---- causal HLA (Section 4.4, Eq. "seq.updates") -------------------------------------------
+def brute_force_causal(q, ks, v, eps):
+    """Token i averages the values of tokens 0..i with weights prod_f (q_i . k^f_j): plain loops."""
+    n, d = len(v), len(v[0])
+    out = [[0.0] * d for _ in range(n)]
+    etas = [0.0] * n
+    for i in range(n):
+        w = []
+        for j in range(i + 1):
+            a = 1.0
+            for k in ks:
+                a *= sum(q[i][t] * k[j][t] for t in range(len(q[i])))
+            w.append(a)
+        etas[i] = sum(w)
+        for g in range(d):
+            out[i][g] = sum(w[j] * v[j][g] for j in range(i + 1)) / (etas[i] + eps)
+    return np.array(out), np.array(etas)
+
+
+@pytest.mark.parametrize("F,dphi", [(1, 5), (2, 4), (3, 3), (2, 12), (3, 6)])
+def test_causal_quadratic_equals_streaming_equals_brute_force(F, dphi):
+    n, d = 11, 5
+    rng = np.random.default_rng(100 + F)
+    q, ks = feats(n, dphi, F, rng)
+    v = rng.standard_normal((n, d))
+    want_o, want_eta = brute_force_causal(q.tolist(), [k.tolist() for k in ks], v.tolist(), 1e-3)
+    oq, eq = orc.hla_quadratic_causal(q, ks, v, 1e-3)
+    os_, es = orc.hla_streaming(q, ks, v, 1e-3)
+    np.testing.assert_allclose(oq, want_o, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(eq, want_eta, rtol=1e-12)
+    np.testing.assert_allclose(os_, want_o, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(es, want_eta, rtol=1e-11)
+
+
+def test_causal_special_cases():
+    """What the mask fixes without any arithmetic of the oracle's own: the first token returns its own value,
+    the last token's output is the unmasked operator's last row, a prefix of the sequence gives a prefix of the
+    output (no token sees the future), and F = 1 is causal normalised linear attention by cumulative sums."""
+    n, dphi, d, F = 17, 4, 6, 3
+    rng = np.random.default_rng(5)
+    q, ks = feats(n, dphi, F, rng)
+    v = rng.standard_normal((n, d))
+    for fn in (orc.hla_quadratic_causal, orc.hla_streaming):
+        o, eta = fn(q, ks, v, 0.0)
+        np.testing.assert_allclose(o[0], v[0], rtol=1e-12)
+        np.testing.assert_allclose(o[-1], orc.hla_quadratic(q, ks, v, 0.0)[0][-1], rtol=1e-11)
+        o_pre, eta_pre = fn(q[:9], [k[:9] for k in ks], v[:9], 0.0)
+        np.testing.assert_allclose(o[:9], o_pre, rtol=1e-12)
+        np.testing.assert_allclose(eta[:9], eta_pre, rtol=1e-12)
+        # changing a later token leaves earlier outputs alone
+        v2 = v.copy(); v2[12] += 3.0
+        k2 = [k.copy() for k in ks]; k2[1][12] *= 2.0
+        o2, _ = fn(q, k2, v2, 0.0)
+        np.testing.assert_array_equal(o2[:12], o[:12])
+        assert np.abs(o2[12:] - o[12:]).max() > 1e-3
+    # F = 1: o_i = q_i . cumsum_j (k_j v_j^T) / q_i . cumsum_j k_j
+    S = np.cumsum(ks[0][:, :, None] * v[:, None, :], axis=0)
+    zc = np.cumsum(ks[0], axis=0)
+    want = np.einsum("np,npg->ng", q, S) / np.einsum("np,np->n", q, zc)[:, None]
+    np.testing.assert_allclose(orc.hla_quadratic_causal(q, ks[:1], v, 0.0)[0], want, rtol=1e-11)
+    np.testing.assert_allclose(orc.hla_streaming(q, ks[:1], v, 0.0)[0], want, rtol=1e-11)
+    # constant values: every (causal) convex combination returns the constant
+    vc = np.tile(rng.standard_normal(d), (n, 1))
+    np.testing.assert_allclose(orc.hla_streaming(q, ks, vc, 0.0)[0], vc, rtol=1e-11)
+
+
+@pytest.mark.parametrize("F,dphi", [(1, 4), (2, 3), (3, 3)])
+@pytest.mark.parametrize("form", ["causal_quadratic", "causal_streaming"])
+def test_causal_gradients_finite_differences(F, dphi, form):
+    n, d = 8, 3
+    rng = np.random.default_rng(11)
+    q = np.abs(rng.standard_normal((n, dphi))) + 0.1
+    ks = [np.abs(rng.standard_normal((n, dphi))) + 0.1 for _ in range(F)]
+    v = rng.standard_normal((n, d))
+    do = rng.standard_normal((n, d))
+    eps = 1e-2
+    bw = orc.hla_quadratic_causal_backward if form == "causal_quadratic" else orc.hla_streaming_backward
+    dq, dks, dv = bw(q, ks, v, do, eps)
+
+    def loss(q_=q, ks_=ks, v_=v):
+        # the loss is evaluated by the pure-Python loops, not by the function under test
+        o, _ = brute_force_causal(q_.tolist(), [k.tolist() for k in ks_], v_.tolist(), eps)
+        return float(np.sum(do * o))
+
+    np.testing.assert_allclose(dq, fd_grad(lambda x: loss(q_=x), q), rtol=1e-6, atol=1e-8)
+    np.testing.assert_allclose(dv, fd_grad(lambda x: loss(v_=x), v), rtol=1e-6, atol=1e-8)
+    for f in range(F):
+        def lf(x, f=f):
+            kk = list(ks); kk[f] = x
+            return loss(ks_=kk)
+        np.testing.assert_allclose(dks[f], fd_grad(lf, ks[f]), rtol=1e-6, atol=1e-8)
+
+
+def test_causal_backward_forms_agree_and_identities():
+    n, dphi, d, F = 37, 6, 8, 3
+    rng = np.random.default_rng(12)
+    q, ks = feats(n, dphi, F, rng)
+    v = rng.standard_normal((n, d))
+    do = rng.standard_normal((n, d))
+    g1 = orc.hla_quadratic_causal_backward(q, ks, v, do, 0.0)
+    g2 = orc.hla_streaming_backward(q, ks, v, do, 0.0)
+    np.testing.assert_allclose(g2[0], g1[0], rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(g2[2], g1[2], rtol=1e-9, atol=1e-12)
+    for f in range(F):
+        np.testing.assert_allclose(g2[1][f], g1[1][f], rtol=1e-9, atol=1e-12)
+    # scale invariance of every row (eps = 0) and rows summing to one, as without the mask
+    np.testing.assert_allclose(np.sum(q * g1[0], axis=1), 0.0, atol=1e-10)
+    for f in range(F):
+        assert abs(np.sum(ks[f] * g1[1][f])) < 1e-9
+    np.testing.assert_allclose(g1[2].sum(axis=0), do.sum(axis=0), rtol=1e-10)
+    # the last token is seen only by itself: dv_last = do_last (its own weight is 1 after normalisation
+    # only if it were alone; in general dv_last = A_nn / eta_n * do_n)
+    A = orc.attention_matrix(q, ks)
+    np.testing.assert_allclose(g1[2][-1], A[-1, -1] / np.tril(A)[-1].sum() * do[-1], rtol=1e-10)
+    # the first query sees one token: o_0 = v_0 whatever q_0 is -> dq_0 = 0
+    np.testing.assert_allclose(g1[0][0], 0.0, atol=1e-12)
+
+
+def test_causal_wrappers_dispatch_per_head():
+    rng = np.random.default_rng(13)
+    B, H, N, dphi, d, F = 2, 2, 7, 3, 4, 3
+    qf = np.abs(rng.standard_normal((B, H, N, dphi)))
+    kf = np.abs(rng.standard_normal((B, H, F, N, dphi)))
+    V = rng.standard_normal((B, H, N, d))
+    dO = rng.standard_normal((B, H, N, d))
+    O, eta = orc.hla_core_forward(qf, kf, V, 1e-3, "causal_streaming")
+    dq, dk, dV = orc.hla_core_backward(qf, kf, V, dO, 1e-3, "causal_quadratic")
+    for b in range(B):
+        for h in range(H):
+            ks = [kf[b, h, f] for f in range(F)]
+            want, weta = brute_force_causal(qf[b, h].tolist(), [k.tolist() for k in ks], V[b, h].tolist(), 1e-3)
+            np.testing.assert_allclose(O[b, h], want, rtol=1e-11)
+            np.testing.assert_allclose(eta[b, h], weta, rtol=1e-11)
+            g = orc.hla_streaming_backward(qf[b, h], ks, V[b, h], dO[b, h], 1e-3)
+            np.testing.assert_allclose(dq[b, h], g[0], rtol=1e-9, atol=1e-12)
+            np.testing.assert_allclose(dV[b, h], g[2], rtol=1e-9, atol=1e-12)
+            for f in range(F):
+                np.testing.assert_allclose(dk[b, h, f], g[1][f], rtol=1e-9, atol=1e-12)
+
 # ---- phi networks ------------------------------------------------------------------------
 def test_gelu_against_math_erf_and_known_values():
     xs = np.linspace(-6, 6, 97)
