@@ -266,9 +266,9 @@ def hla_destroy(ctx: int) -> None:
 class Hla:
     """Owns a context and its workspace tensor.  All compute happens in hla_forward / hla_backward."""
 
-    def __init__(self, B, H, N, d, dtype="bf16", phi="mlp", F=0, d_phi=0, eps=0.0, n_splits=0, device="cuda", value_mod=False):
+    def __init__(self, B, H, N, d, dtype="bf16", phi="mlp", F=0, d_phi=0, eps=0.0, n_splits=0, device="cuda", value_mod=False, causal=False):
         self.cfg = HlaConfig(B, H, N, d, F, d_phi, HLA_PHI_MLP if phi == "mlp" else HLA_PHI_NONE,
-                             HLA_BF16 if dtype == "bf16" else HLA_F32, eps, n_splits, 0, 1 if value_mod else 0)
+                             HLA_BF16 if dtype == "bf16" else HLA_F32, eps, n_splits, 1 if causal else 0, 1 if value_mod else 0)
         self.torch_dtype = torch.bfloat16 if dtype == "bf16" else torch.float32
         self.ctx = hla_create(self.cfg)
         self.layout = hla_workspace_layout(self.ctx)

@@ -14,6 +14,7 @@
 #include "hla_tc_fused_k.cuh"
 #include "hla_tc_wgrad.cuh"
 #include "hla_tc_vmod.cuh"
+#include "hla_tc_causal.cuh"
 
 using namespace hla;
 
@@ -233,7 +234,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
         else return HLA_ERR_INVALID_ARG;
     }
     if (!(c.eps > 0.f)) c.eps = 1e-6f;
-    if (c.causal != 0) return HLA_ERR_UNSUPPORTED;
+    if (c.causal != 0 && c.causal != 1) return HLA_ERR_INVALID_ARG;
     if (c.value_mod != 0 && c.value_mod != 1) return HLA_ERR_INVALID_ARG;
     if (c.value_mod && !(c.dtype == HLA_BF16 && (c.d == 64 || c.d == 128) && (long long)c.B * c.H * c.N < (1ll << 31))) return HLA_ERR_UNSUPPORTED;
     if (c.F > kMaxF) return HLA_ERR_UNSUPPORTED;
@@ -261,6 +262,10 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     D.ld = c.d + 4;
     D.eps = c.eps;
     x->tc = tc::supported(c.dtype == HLA_BF16, c.d, c.F, c.d_phi) && (long long)c.B * c.H * c.N < (1ll << 31);   // the tensor-core kernels index tokens in 32 bits
+    if (c.causal && !(x->tc && c.F == 3)) {      // the causal sweep exists for the 3-factor tensor-core set only
+        delete x;
+        return HLA_ERR_UNSUPPORTED;
+    }
     const int tile = x->tc ? tc::kTileTokens : simt::kTok;
     const int tiles = (c.N + tile - 1) / tile;
     int S = c.n_splits;
@@ -367,11 +372,17 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
             s = tc::reduce_pieces(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, ctx->off_part, ctx->k_pieces,
                                   tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec);
             if (s != HLA_OK) return s;
-            return tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
+            s = tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
+            if (s != HLA_OK || !ctx->cfg.causal) return s;
+            // causal: the pass above left the features of both sides in the workspace (its O is overwritten now); the
+            // pieces of the key-side kernel become the pieces of the sweep
+            return tc::causal_sweep(ctx->D, ctx->BH, reinterpret_cast<const float*>(ws + ctx->L.qf), reinterpret_cast<const float*>(ws + ctx->L.kf), V, O,
+                                    ws, ctx->L, ctx->off_part, ctx->k_pieces, tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec);
         } else {
             qf = static_cast<const float*>(Q);
             kf = static_cast<const float*>(K);
         }
+        if (ctx->cfg.causal) return tc::causal_forward(ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->rec);
         return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
     }
     if (ctx->cfg.dtype == HLA_F32) return forward_simt<float>(ctx, Q, K, V, O, ws, st);
@@ -389,6 +400,7 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     (void)cudaGetLastError();
     follow_device(ctx);
     tc::HostCacheScope scope(&ctx->hc);
+    if (ctx->cfg.causal) return HLA_ERR_UNSUPPORTED;
     if (ctx->tc) {
         const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
         // the phi backward writes rows of dQ, dK with 32-byte stores; so does the 2-factor key pass with dV

@@ -1,0 +1,455 @@
+// Causal HLA (Section 4.4 "Causal Attention, Decay Factors and Sequential Updates", Eq. "seq.updates") on the tensor
+// cores, F = 3 factors with d_phi = 6, at the level of the folded monomial features.
+//
+// Token i sees the tokens j <= i.  With the context tensor carried along the sequence (C^i = C^{i-1} + T_{k_i} (x) v_i),
+// the output of a 128-token tile splits into what the tokens before the tile contribute and what the tile's own tokens do:
+//     [num | eta]_i = mono_i . [Csym | zsym](tokens before the tile)  +  sum_{j in tile, j <= i} (mono_i . Tsym_j) [v_j | 1]
+// The first term is the readout of the non-causal path against the state *before* the tile; the second is a 128 x 128
+// block of the masked attention matrix times the value tile.  The sequence of a head is cut into pieces (one per CTA that
+// touches the head); a first pass builds the state of every piece, a fixed-order exclusive scan over the pieces of a head
+// gives each piece its initial state, and the kernel below sweeps a piece tile by tile:
+//
+//     P      = mono tile * Tsym tile^T                    (MMA, K = 64)      P[i][j] = prod_f (q_i . k^f_j)
+//     acc    = mono tile * [Csym | zsym]                  (MMA, K = 64)      state before the tile, bf16 image in shared memory
+//     state += Tsym tile^T * [V | 1]                      (MMA, K = 128 tokens, 64 rows)   fp32 in tensor memory
+//     Pm     = bf16(P) where j <= i, else 0               (threads; written back to tensor memory as the next A operand)
+//     acc   += Pm * [V | 1]                               (MMA, K = 128 tokens)
+//     o_i    = acc_i[0..d) / (acc_i[d] + eps)             (threads; TMA store)
+//     state -> bf16 image for the next tile               (threads)
+//
+// Operand rows are shifted by 8 columns, as in the query pass of the backward: a row of the folded key tile is
+// [1, 0 x 7, Tsym_0..55] and a row of the monomial tile is [0 x 8, mono_0..55].  Read as the block that follows the
+// value blocks, the key tile therefore supplies the "ones" column d of [V | 1], so the normaliser and the key-side sum
+// zsym come out of the same products as the numerator and the state (column d), and no product of their own is needed.
+// State row 8 + m holds [Csym[m][0..d), zsym[m], 0 ...]; rows 0..7 are kept zero in the bf16 image.
+//
+// Warp roles: 0 TMA (value tiles), 1 MMA issue, 2..5 operand rows (monomials of q, folded keys), 6..9 mask,
+// 10..13 state image, 14..17 epilogue.
+#pragma once
+#include "hla_tc.cuh"
+
+namespace hla {
+namespace tc {
+
+constexpr int kCaThreads = 18 * 32;
+constexpr int kCaGenWarp0 = 2, kCaMaskWarp0 = 6, kCaConvWarp0 = 10, kCaEpiWarp0 = 14;
+constexpr int kCaRowPad = 8;      // operand column / state row of monomial 0
+
+template <int DV> struct CaCfg {
+    static constexpr int kVB = DV / 64;                     // 64-column blocks of a value tile
+    static constexpr int kStages = 2;
+    static constexpr int kOffT = kVB * kBlk;                // folded key tile: directly after the value blocks
+    static constexpr int kOffM = kOffT + kBlk;              // query monomial tile
+    static constexpr int kStageBytes = kOffM + kBlk;
+    static constexpr int kB3Block = 64 * 128;               // 64 state rows x 64 columns
+    static constexpr int kOffB3 = kStages * kStageBytes;    // bf16 image of the state: kVB + 1 blocks
+    static constexpr int kOffO = kOffB3 + (kVB + 1) * kB3Block;
+    static constexpr int kOffBars = kOffO + kVB * kBlk;
+    static constexpr int kSmem = 1024 + kOffBars + 256;
+    static constexpr int kNAcc = DV + 16, kNState = DV + 8;
+    static constexpr int kColAcc = 0, kColState = DV + 16, kColP = 2 * DV + 32;      // tensor-memory columns
+    static_assert(kColP + 128 <= 512, "tensor memory");
+    static_assert(kSmem <= 227 * 1024, "shared memory");
+};
+
+// Work items are (head, tile), w = bh * T + tile.  G == 0: grid (S, heads), CTA (s, bh) owns the tiles
+// [s * ceil(T / S), (s + 1) * ceil(T / S)) of its head and piece slot (bh, s).  G > 0: G CTAs own contiguous runs of
+// work items, CTA c the items [total c / G, total (c + 1) / G); a run inside one head is piece c - (first CTA of the head).
+struct CaWork {
+    int w0, w1;
+};
+__device__ __forceinline__ CaWork causal_work(int T, int BH, int S, int G) {
+    CaWork w;
+    if (G == 0) {
+        const int tiles_per = (T + S - 1) / S;
+        const int bh = blockIdx.y, s = blockIdx.x;
+        w.w0 = bh * T + min(T, s * tiles_per);
+        w.w1 = bh * T + min(T, (s + 1) * tiles_per);
+    } else {
+        const long long total = (long long)BH * T;
+        w.w0 = (int)(total * blockIdx.x / G);
+        w.w1 = (int)(total * (blockIdx.x + 1) / G);
+    }
+    return w;
+}
+__device__ __forceinline__ int causal_slot(int bh, int T, int BH, int S, int G) {
+    if (G == 0) return bh * S + blockIdx.x;
+    return bh * S + ((int)blockIdx.x - owner_of_work((long long)bh * T, (long long)BH * T, G));
+}
+
+// [first, 0 x 7, v_0..55] as one 128-byte operand row
+__device__ __forceinline__ void store_shifted_row(uint32_t blk, uint32_t row, float first, const float (&v)[kMono]) {
+    st_shared_v4(blk + sw128_off(row, 0), pack_bf16(first, 0.f), 0u, 0u, 0u);
+#pragma unroll
+    for (int c = 1; c < 8; ++c)
+        st_shared_v4(blk + sw128_off(row, c), pack_bf16(v[8 * c - 8], v[8 * c - 7]), pack_bf16(v[8 * c - 6], v[8 * c - 5]),
+                     pack_bf16(v[8 * c - 4], v[8 * c - 3]), pack_bf16(v[8 * c - 2], v[8 * c - 1]));
+}
+
+// In-place exclusive scan of the piece states of every head, in piece order (bit-reproducible); the sum of all pieces,
+// i.e. the state after the last token, goes to `state`.
+template <int F>
+__global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__ part, float* __restrict__ state, int S, int ld, int G, int T) {
+    constexpr int kN = MT<F>::kN;
+    const int bh = blockIdx.y;
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const size_t n_per = (size_t)kN * ld;
+    int count = S;
+    if (G > 0) {
+        const long long total = (long long)gridDim.y * T;
+        count = owner_of_work((long long)bh * T + T - 1, total, G) - owner_of_work((long long)bh * T, total, G) + 1;
+    }
+    const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (e >= n_per) return;
+    float* p = part + (size_t)bh * S * n_per + e;
+    float run = 0.f;
+    for (int s = 0; s < count; ++s) {
+        const float t = p[(size_t)s * n_per];
+        p[(size_t)s * n_per] = run;
+        run += t;
+    }
+    state[(size_t)bh * n_per + e] = run;
+}
+
+template <int DV>
+__global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
+                                                                          const float* __restrict__ qf, const float* __restrict__ kf,
+                                                                          const float* __restrict__ init, float* __restrict__ eta_out, int N, int BH,
+                                                                          int S, int ld, int G, float eps, int* status) {
+    using Cfg = CaCfg<DV>;
+    constexpr int kStageBytes = Cfg::kStageBytes;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
+    uint64_t* v_full = bars;              // [2] TMA
+    uint64_t* gen_full = bars + 2;        // [2] 128 arrivals: both operand-row tiles of the stage are written
+    uint64_t* stage_free = bars + 4;      // [2] MMA commit: every product that reads the stage has finished
+    uint64_t* p_full = bars + 6;          // MMA commit
+    uint64_t* pm_ready = bars + 7;        // 128 arrivals: masked bf16 block is in tensor memory
+    uint64_t* b3_ready = bars + 8;        // 128 arrivals: state image (and, at the start of a piece, the state) is in place
+    uint64_t* state_full = bars + 9;      // MMA commit
+    uint64_t* acc_full = bars + 10;       // MMA commit
+    uint64_t* acc_free = bars + 11;       // 128 arrivals
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 13);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int T = (N + kTileTokens - 1) / kTileTokens;
+    const CaWork cw = causal_work(T, BH, S, G);
+    const int w0 = cw.w0, nwork = cw.w1 - cw.w0;
+    grid_launch_dependents();
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&v_full[i], 1);
+            mbar_init(&gen_full[i], 128);
+            mbar_init(&stage_free[i], 1);
+        }
+        mbar_init(p_full, 1);
+        mbar_init(pm_ready, 128);
+        mbar_init(b3_ready, 128);
+        mbar_init(state_full, 1);
+        mbar_init(acc_full, 1);
+        mbar_init(acc_free, 128);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&mapV);
+        prefetch_tmap(&mapO);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    grid_dependency_wait();
+    bool ok = true;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int it = 0; it < nwork; ++it) {
+                const int st = it & 1, u = it >> 1, work = w0 + it;
+                if (!mbar_wait(&stage_free[st], (u & 1) ^ 1)) { report_timeout(status, 901); break; }
+                mbar_arrive_expect_tx(&v_full[st], DV * kTileTokens * 2);
+                for (int b = 0; b < Cfg::kVB; ++b) tma_load_3d(smem + st * kStageBytes + b * kBlk, &mapV, &v_full[st], b * 64, (work % T) * kTileTokens, work / T);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t id_p = idesc_bf16(128, 128, false, false);
+            const uint32_t id_r = idesc_bf16(128, Cfg::kNAcc, false, true);
+            const uint32_t id_s = idesc_bf16(64, Cfg::kNState, true, true);
+            const uint32_t b3a = smem_u32(smem + Cfg::kOffB3);
+            for (int it = 0; it < nwork; ++it) {
+                const int st = it & 1, u = it >> 1;
+                const uint32_t sa = smem_u32(smem + st * kStageBytes), ta = sa + Cfg::kOffT, ma = sa + Cfg::kOffM;
+                if (!mbar_wait(&gen_full[st], u & 1)) { report_timeout(status, 902); break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)      // P = mono * Tsym^T
+                    umma_bf16(tmem + Cfg::kColP, smem_desc_sw128(ma + ks * 32, 16, 1024), smem_desc_sw128(ta + ks * 32, 16, 1024), id_p, ks > 0 ? 1u : 0u);
+                umma_commit(p_full);
+                if (!(mbar_wait(b3_ready, it & 1) && mbar_wait(acc_free, (it & 1) ^ 1))) { report_timeout(status, 903); break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)      // acc = mono * [Csym | zsym] of the tokens before the tile
+                    umma_bf16(tmem + Cfg::kColAcc, smem_desc_sw128(ma + ks * 32, 16, 1024), smem_desc_sw128(b3a + ks * 2048, Cfg::kB3Block, 1024), id_r,
+                              ks > 0 ? 1u : 0u);
+                if (!mbar_wait(&v_full[st], u & 1)) { report_timeout(status, 904); break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kTileTokens / 16; ++ks)      // state += Tsym^T * [V | 1]
+                    umma_bf16(tmem + Cfg::kColState, smem_desc_sw128(ta + ks * 2048, kBlk, 1024), smem_desc_sw128(sa + ks * 2048, kBlk, 1024), id_s, 1u);
+                umma_commit(state_full);
+                if (!mbar_wait(pm_ready, it & 1)) { report_timeout(status, 905); break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < kTileTokens / 16; ++ks)      // acc += Pm * [V | 1]
+                    umma_bf16_ta(tmem + Cfg::kColAcc, tmem + Cfg::kColP + 8 * ks, smem_desc_sw128(sa + ks * 2048, kBlk, 1024), id_r, 1u);
+                umma_commit(acc_full);
+                umma_commit(&stage_free[st]);
+            }
+        }
+    } else if (warp < kCaMaskWarp0) {
+        // operand rows: thread = token row of the tile
+        const int row = tid - kCaGenWarp0 * 32;
+        float qn[6], kn[18];
+        auto prefetch = [&](int it) {
+            const int work = w0 + it, bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
+            load_feat<6>(qn, qf + ((size_t)bh * N + tok) * 6);
+#pragma unroll
+            for (int f = 0; f < 3; ++f) load_feat<6>(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+        };
+        if (nwork > 0) prefetch(0);
+        for (int it = 0; it < nwork; ++it) {
+            const int st = it & 1, u = it >> 1, work = w0 + it;
+            const bool valid = (work % T) * kTileTokens + row < N;
+            float q[6], k[18];
+#pragma unroll
+            for (int i = 0; i < 6; ++i) q[i] = valid ? qn[i] : 0.f;
+#pragma unroll
+            for (int i = 0; i < 18; ++i) k[i] = valid ? kn[i] : 0.f;
+            if (it + 1 < nwork) prefetch(it + 1);
+            if (ok && !mbar_wait(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 906); }
+            if (!ok) continue;
+            const uint32_t sa = smem_u32(smem + st * kStageBytes);
+            {
+                float mono[kMono];
+                query_monomials_t<3>(q, mono);
+                store_shifted_row(sa + Cfg::kOffM, row, 0.f, mono);
+            }
+            {
+                float ts[kMono];
+                key_folded_t<3>(k, ts);
+                store_shifted_row(sa + Cfg::kOffT, row, valid ? 1.f : 0.f, ts);
+            }
+            fence_proxy_async();
+            mbar_arrive(&gen_full[st]);
+        }
+    } else if (warp < kCaConvWarp0) {
+        // mask: thread = query row i of the block; keeps the columns j <= i, rounds to bf16, writes the block back in place
+        const int qt = warp & 3, row = qt * 32 + lane;
+        const uint32_t pa = tmem + Cfg::kColP + ((uint32_t)(qt * 32) << 16);
+        for (int it = 0; it < nwork; ++it) {
+            if (ok && !mbar_wait(p_full, it & 1)) { ok = false; report_timeout(status, 907); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                uint32_t w[16];
+                if (b <= qt) {      // columns 32 b .. 32 b + 31; a warp's rows are 32 qt .. 32 qt + 31
+                    uint32_t r[32];
+                    tmem_ld16(pa + 32 * b, *reinterpret_cast<uint32_t(*)[16]>(r));
+                    tmem_ld16(pa + 32 * b + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int j = 32 * b + 2 * e;
+                        w[e] = pack_bf16(j <= row ? __uint_as_float(r[2 * e]) : 0.f, j + 1 <= row ? __uint_as_float(r[2 * e + 1]) : 0.f);
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) w[e] = 0u;
+                }
+                tmem_st8(pa + 16 * b, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                tmem_st8(pa + 16 * b + 8, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(pm_ready);
+        }
+    } else if (warp < kCaEpiWarp0) {
+        // state image.  A 64-row accumulator keeps row R in lane 32 (R / 16) + R % 16: lanes 0..15 of each warp's quarter.
+        const int qt = warp & 3, R = qt * 16 + lane, m = R - kCaRowPad;
+        const bool active = lane < 16, mine = active && m >= 0 && m < kMono;
+        const uint32_t sa = tmem + Cfg::kColState + ((uint32_t)(qt * 32) << 16);
+        const uint32_t b3a = smem_u32(smem + Cfg::kOffB3);
+        constexpr int kChunks = Cfg::kNAcc / 8;      // 16-byte chunks of an image row
+        auto store_chunk = [&](int c, const float (&v)[8]) {
+            if (active)
+                st_shared_v4(b3a + (c >> 3) * Cfg::kB3Block + sw128_off(R, c & 7), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
+                             pack_bf16(v[6], v[7]));
+        };
+        for (int it = 0; it < nwork; ++it) {
+            const int work = w0 + it, bh = work / T;
+            if (it == 0 || work % T == 0) {
+                // a piece begins: its initial state goes to tensor memory (fp32) and to the image (bf16)
+                const float* src = init + ((size_t)causal_slot(bh, T, BH, S, G) * kMono + (mine ? m : 0)) * ld;
+#pragma unroll 1
+                for (int c = 0; c < kChunks; ++c) {
+                    float v[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[e] = 0.f;
+                    if (mine && 8 * c < ld) {
+                        const float4 a = *reinterpret_cast<const float4*>(src + 8 * c);
+                        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+                        if (8 * c + 4 < ld) {
+                            const float4 b = *reinterpret_cast<const float4*>(src + 8 * c + 4);
+                            v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+                        }
+                    }
+                    if (8 * c < Cfg::kNState)
+                        tmem_st8(sa + 8 * c, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]), __float_as_uint(v[4]),
+                                 __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
+                    store_chunk(c, v);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                fence_proxy_async();
+                mbar_arrive(b3_ready);
+            }
+            if (ok && !mbar_wait(state_full, it & 1)) { ok = false; report_timeout(status, 908); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (it + 1 < nwork && (work + 1) % T != 0) {
+                tc_fence_after();
+#pragma unroll 1
+                for (int c = 0; c < kChunks; ++c) {
+                    float v[8];
+                    if (8 * c < Cfg::kNState) {
+                        uint32_t r[8];
+                        tmem_ld8(sa + 8 * c, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) v[e] = mine && (8 * c + e <= DV) ? __uint_as_float(r[e]) : 0.f;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) v[e] = 0.f;
+                    }
+                    store_chunk(c, v);
+                }
+                tc_fence_before();
+                fence_proxy_async();
+                mbar_arrive(b3_ready);
+            }
+        }
+    } else {
+        // epilogue: thread = token row
+        const int qt = warp & 3, row = qt * 32 + lane, etid = tid - kCaEpiWarp0 * 32;
+        const uint32_t aa = tmem + Cfg::kColAcc + ((uint32_t)(qt * 32) << 16);
+        const uint32_t os = smem_u32(smem + Cfg::kOffO);
+        for (int it = 0; it < nwork; ++it) {
+            const int work = w0 + it, bh = work / T, tile = work % T;
+            if (!mbar_wait(acc_full, it & 1)) {
+                report_timeout(status, 909);
+                *abort_flag = 1;
+            }
+            if (etid == 0) tma_store_wait_read0();      // the staging tile has been read by the previous store
+            named_barrier(1, 128);
+            if (*abort_flag) break;
+            tc_fence_after();
+            uint32_t re[8];
+            tmem_ld8(aa + DV, re);
+            tmem_ld_wait();
+            const float eta = __uint_as_float(re[0]);
+            const float rinv = 1.f / (eta + eps);
+#pragma unroll
+            for (int h = 0; h < Cfg::kVB; ++h) {
+                uint32_t r[64];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld16(aa + 64 * h + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
+                tmem_ld_wait();
+                if (h == Cfg::kVB - 1) {
+                    tc_fence_before();
+                    mbar_arrive(acc_free);
+                }
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    st_shared_v4(os + h * kBlk + sw128_off(row, c), pack_bf16(__uint_as_float(r[8 * c]) * rinv, __uint_as_float(r[8 * c + 1]) * rinv),
+                                 pack_bf16(__uint_as_float(r[8 * c + 2]) * rinv, __uint_as_float(r[8 * c + 3]) * rinv),
+                                 pack_bf16(__uint_as_float(r[8 * c + 4]) * rinv, __uint_as_float(r[8 * c + 5]) * rinv),
+                                 pack_bf16(__uint_as_float(r[8 * c + 6]) * rinv, __uint_as_float(r[8 * c + 7]) * rinv));
+            }
+            fence_proxy_async();
+            named_barrier(1, 128);
+            if (etid == 0) {
+                for (int b = 0; b < Cfg::kVB; ++b) tma_store_3d(&mapO, smem + Cfg::kOffO + b * kBlk, b * 64, tile * kTileTokens, bh);
+                tma_store_commit();
+            }
+            const int tok = tile * kTileTokens + row;
+            if (tok < N) eta_out[(size_t)bh * N + tok] = eta;
+        }
+        if (etid == 0) tma_store_wait_all0();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// Exclusive scan of the piece states, then the causal sweep.  The pieces are those of the kernel that built them:
+// G == 0: S pieces per head from a (S, heads) grid; G > 0: the pieces of a persistent kernel of G CTAs (at most S per head).
+template <int DV>
+inline hla_status launch_causal_sweep(const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws, const hla_ws_layout& L,
+                                      size_t off_part, int S, int G, LaunchRec& rec) {
+    CUtensorMap mapV, mapO;
+    if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens)) return HLA_ERR_CUDA;
+    int* status = reinterpret_cast<int*>(ws + L.status);
+    float* part = reinterpret_cast<float*>(ws + off_part);
+    float* state = reinterpret_cast<float*>(ws + L.state);
+    float* eta = reinterpret_cast<float*>(ws + L.eta);
+    if (!set_smem(tc_causal_forward_kernel<DV>, CaCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    const int T = (D.N + kTileTokens - 1) / kTileTokens;
+    rec.begin("tc_scan_pieces");
+    launch_pdl(tc_scan_pieces_kernel<3>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, state, S, D.ld, G, T);
+    if (!rec.end()) return HLA_ERR_CUDA;
+    rec.begin("tc_causal_forward");
+    launch_pdl(tc_causal_forward_kernel<DV>, G > 0 ? dim3(G) : dim3(S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapV, mapO, qf, kf, part, eta, D.N, BH, S,
+               D.ld, G, D.eps, status);
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+
+inline hla_status causal_sweep(const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws, const hla_ws_layout& L,
+                               size_t off_part, int S, int G, LaunchRec& rec) {
+    if (D.F != 3) return HLA_ERR_UNSUPPORTED;
+    if (D.d == 128) return launch_causal_sweep<128>(D, BH, qf, kf, V, O, ws, L, off_part, S, G, rec);
+    return launch_causal_sweep<64>(D, BH, qf, kf, V, O, ws, L, off_part, S, G, rec);
+}
+
+// Feature-level causal forward: state of every piece (the non-causal state build, one piece per split) -> scan -> sweep.
+template <int DV>
+inline hla_status launch_causal_state_build(const Dims& D, int BH, const float* kf, const void* V, char* ws, const hla_ws_layout& L, size_t off_part,
+                                            LaunchRec& rec) {
+    CUtensorMap mapV;
+    if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_state_build_kernel<DV, 3>, SbCfg<3>::kSmem)) return HLA_ERR_CUDA;
+    rec.begin("tc_state_build");
+    launch_pdl(tc_state_build_kernel<DV, 3>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<3>::kSmem, rec.st, mapV, kf, reinterpret_cast<float*>(ws + off_part), D.N, D.S,
+               D.ld, reinterpret_cast<int*>(ws + L.status));
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+
+inline hla_status causal_forward(const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws, const hla_ws_layout& L,
+                                 size_t off_part, LaunchRec& rec) {
+    if (D.F != 3) return HLA_ERR_UNSUPPORTED;
+    const hla_status s = D.d == 128 ? launch_causal_state_build<128>(D, BH, kf, V, ws, L, off_part, rec)
+                                    : launch_causal_state_build<64>(D, BH, kf, V, ws, L, off_part, rec);
+    if (s != HLA_OK) return s;
+    return causal_sweep(D, BH, qf, kf, V, O, ws, L, off_part, D.S, 0, rec);
+}
+
+}  // namespace tc
+}  // namespace hla

@@ -55,11 +55,11 @@ def dev_weights(phi_q, phi_k, dtype):
 class DeviceRun:
     """One library context fed from numpy inputs; keeps device tensors for reuse."""
 
-    def __init__(self, shape: synth.HlaShape, phi="mlp", eps=0.0, n_splits=0):
+    def __init__(self, shape: synth.HlaShape, phi="mlp", eps=0.0, n_splits=0, causal=False):
         self.shape = shape
         self.phi = phi
         self.op = binding.Hla(shape.B, shape.H, shape.N, shape.d, dtype=shape.dtype, phi=phi, F=shape.F, d_phi=shape.d_phi,
-                              eps=eps, n_splits=n_splits)
+                              eps=eps, n_splits=n_splits, causal=causal)
 
     def set_weights(self, phi_q, phi_k):
         self.op.set_phi(*dev_weights(phi_q, phi_k, self.shape.dtype))

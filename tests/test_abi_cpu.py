@@ -69,7 +69,9 @@ def test_feature_level_entry_has_no_feature_regions():
     (dict(phi=7), binding.HLA_ERR_INVALID_ARG),
     (dict(dtype=3), binding.HLA_ERR_INVALID_ARG),
     (dict(F=1), binding.HLA_ERR_INVALID_ARG),            # no default d_phi for F = 1
-    (dict(causal=1), binding.HLA_ERR_UNSUPPORTED),
+    (dict(causal=2), binding.HLA_ERR_INVALID_ARG),
+    (dict(causal=1, F=2), binding.HLA_ERR_UNSUPPORTED),                 # the causal sweep: 3 factors, bf16, d in {64, 128}
+    (dict(causal=1, dtype=binding.HLA_F32, d=16), binding.HLA_ERR_UNSUPPORTED),
     (dict(F=3, d_phi=7), binding.HLA_ERR_UNSUPPORTED),   # 343 features > 256
     (dict(F=5, d_phi=2), binding.HLA_ERR_UNSUPPORTED),
     (dict(d=256), binding.HLA_ERR_UNSUPPORTED),
