@@ -21,18 +21,22 @@
 // [1, 0 x 7, Tsym_0..55] and a row of the monomial tile is [0 x 8, mono_0..55].  Read as the block that follows the
 // value blocks, the key tile therefore supplies the "ones" column d of [V | 1], so the normaliser and the key-side sum
 // zsym come out of the same products as the numerator and the state (column d), and no product of their own is needed.
-// State row 8 + m holds [Csym[m][0..d), zsym[m], 0 ...]; rows 0..7 are kept zero in the bf16 image.
+// State row 8 + m holds [Csym[m][0..d), zsym[m], 0 ...]; rows 0..7 are kept zero in the bf16 image.  The image is
+// double-buffered: the image for tile t + 1 is written while the products of tile t still read theirs.
 //
-// Warp roles: 0 TMA (value tiles), 1 MMA issue, 2..5 operand rows (monomials of q, folded keys), 6..9 mask,
-// 10..13 state image, 14..17 epilogue.
+// Warp roles: 0 TMA (value tiles), 1 MMA issue, 2..5 monomial rows of q, 6..9 folded key rows, 10..17 mask (two warps
+// per 32 rows, 64 columns each), 18..21 state image, 22..25 epilogue.  A role is one warp per scheduler running a
+// straight instruction stream per tile, so what bounds a tile is the longest of these streams: they are kept short
+// (selects only where the mask cuts a 32 x 32 block, conversions 32 columns at a time, out-of-line waits, rolled loops).
 #pragma once
 #include "hla_tc.cuh"
+#include "hla_tc_fused_k.cuh"
 
 namespace hla {
 namespace tc {
 
-constexpr int kCaThreads = 18 * 32;
-constexpr int kCaGenWarp0 = 2, kCaMaskWarp0 = 6, kCaConvWarp0 = 10, kCaEpiWarp0 = 14;
+constexpr int kCaThreads = 26 * 32;
+constexpr int kCaGenQWarp0 = 2, kCaGenKWarp0 = 6, kCaMaskWarp0 = 10, kCaConvWarp0 = 18, kCaEpiWarp0 = 22;
 constexpr int kCaRowPad = 8;      // operand column / state row of monomial 0
 
 template <int DV> struct CaCfg {
@@ -42,8 +46,9 @@ template <int DV> struct CaCfg {
     static constexpr int kOffM = kOffT + kBlk;              // query monomial tile
     static constexpr int kStageBytes = kOffM + kBlk;
     static constexpr int kB3Block = 64 * 128;               // 64 state rows x 64 columns
-    static constexpr int kOffB3 = kStages * kStageBytes;    // bf16 image of the state: kVB + 1 blocks
-    static constexpr int kOffO = kOffB3 + (kVB + 1) * kB3Block;
+    static constexpr int kB3Bytes = (kVB + 1) * kB3Block;   // one bf16 image of the state
+    static constexpr int kOffB3 = kStages * kStageBytes;    // two images: the sweep writes the next one while the current one is read
+    static constexpr int kOffO = kOffB3 + 2 * kB3Bytes;
     static constexpr int kOffBars = kOffO + kVB * kBlk;
     static constexpr int kSmem = 1024 + kOffBars + 256;
     static constexpr int kNAcc = DV + 16, kNState = DV + 8;
@@ -86,6 +91,34 @@ __device__ __forceinline__ void store_shifted_row(uint32_t blk, uint32_t row, fl
                      pack_bf16(v[8 * c - 4], v[8 * c - 3]), pack_bf16(v[8 * c - 2], v[8 * c - 1]));
 }
 
+// The same rows formed 16 bytes at a time, so that only a few values are live at once.  Chunk C (1..7) holds the
+// monomials 8 C - 8 .. 8 C - 1.
+template <int M> __device__ __forceinline__ float mono_value(const float (&q)[6]) {
+    constexpr int abc = mono_abc(M), a = abc / 36, b = (abc / 6) % 6, c = abc % 6;
+    return q[a] * q[b] * q[c];
+}
+template <int C, int... E>
+__device__ __forceinline__ void shifted_mono_chunk(uint32_t blk, uint32_t row, const float (&q)[6], std::integer_sequence<int, E...>) {
+    const float v[8] = {mono_value<8 * (C - 1) + E>(q)...};
+    st_shared_v4(blk + sw128_off(row, C), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+template <int... C>
+__device__ __forceinline__ void shifted_mono_row(uint32_t blk, uint32_t row, const float (&q)[6], std::integer_sequence<int, C...>) {
+    st_shared_v4(blk + sw128_off(row, 0), 0u, 0u, 0u, 0u);
+    (shifted_mono_chunk<C + 1>(blk, row, q, std::make_integer_sequence<int, 8>{}), ...);
+}
+template <int C, int... E>
+__device__ __forceinline__ void shifted_key_chunk(uint32_t blk, uint32_t row, const float (&s12)[6][6], const float (&k3)[6], std::integer_sequence<int, E...>) {
+    const float v[8] = {folded_value<8 * (C - 1) + E>(s12, k3)...};
+    st_shared_v4(blk + sw128_off(row, C), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+template <int... C>
+__device__ __forceinline__ void shifted_key_row(uint32_t blk, uint32_t row, float first, const float (&s12)[6][6], const float (&k3)[6],
+                                                std::integer_sequence<int, C...>) {
+    st_shared_v4(blk + sw128_off(row, 0), pack_bf16(first, 0.f), 0u, 0u, 0u);
+    (shifted_key_chunk<C + 1>(blk, row, s12, k3, std::make_integer_sequence<int, 8>{}), ...);
+}
+
 // In-place exclusive scan of the piece states of every head, in piece order (bit-reproducible); the sum of all pieces,
 // i.e. the state after the last token, goes to `state`.
 template <int F>
@@ -123,16 +156,17 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* v_full = bars;              // [2] TMA
-    uint64_t* gen_full = bars + 2;        // [2] 128 arrivals: both operand-row tiles of the stage are written
+    uint64_t* gen_full = bars + 2;        // [2] 256 arrivals: both operand-row tiles of the stage are written
     uint64_t* stage_free = bars + 4;      // [2] MMA commit: every product that reads the stage has finished
     uint64_t* p_full = bars + 6;          // MMA commit
-    uint64_t* pm_ready = bars + 7;        // 128 arrivals: masked bf16 block is in tensor memory
+    uint64_t* pm_ready = bars + 7;        // 256 arrivals: masked bf16 block is in tensor memory
     uint64_t* b3_ready = bars + 8;        // 128 arrivals: state image (and, at the start of a piece, the state) is in place
     uint64_t* state_full = bars + 9;      // MMA commit
     uint64_t* acc_full = bars + 10;       // MMA commit
     uint64_t* acc_free = bars + 11;       // 128 arrivals
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 13);
+    uint64_t* state_read = bars + 12;     // 128 arrivals: the state after a tile has been read out of tensor memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 14);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int T = (N + kTileTokens - 1) / kTileTokens;
@@ -143,15 +177,16 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(&v_full[i], 1);
-            mbar_init(&gen_full[i], 128);
+            mbar_init(&gen_full[i], 256);
             mbar_init(&stage_free[i], 1);
         }
         mbar_init(p_full, 1);
-        mbar_init(pm_ready, 128);
+        mbar_init(pm_ready, 256);
         mbar_init(b3_ready, 128);
         mbar_init(state_full, 1);
         mbar_init(acc_full, 1);
         mbar_init(acc_free, 128);
+        mbar_init(state_read, 128);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&mapV);
@@ -161,6 +196,9 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
+    // rows 0..7 of the state images (and their padding columns) are never written again: zero both images once
+    for (int i = tid; i < 2 * Cfg::kB3Bytes / 16; i += kCaThreads) reinterpret_cast<uint4*>(smem + Cfg::kOffB3)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -172,7 +210,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
         if (lane == 0) {
             for (int it = 0; it < nwork; ++it) {
                 const int st = it & 1, u = it >> 1, work = w0 + it;
-                if (!mbar_wait(&stage_free[st], (u & 1) ^ 1)) { report_timeout(status, 901); break; }
+                if (!mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { report_timeout(status, 901); break; }
                 mbar_arrive_expect_tx(&v_full[st], DV * kTileTokens * 2);
                 for (int b = 0; b < Cfg::kVB; ++b) tma_load_3d(smem + st * kStageBytes + b * kBlk, &mapV, &v_full[st], b * 64, (work % T) * kTileTokens, work / T);
             }
@@ -182,44 +220,77 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             const uint32_t id_p = idesc_bf16(128, 128, false, false);
             const uint32_t id_r = idesc_bf16(128, Cfg::kNAcc, false, true);
             const uint32_t id_s = idesc_bf16(64, Cfg::kNState, true, true);
-            const uint32_t b3a = smem_u32(smem + Cfg::kOffB3);
+            const uint32_t b3base = smem_u32(smem + Cfg::kOffB3);
             for (int it = 0; it < nwork; ++it) {
                 const int st = it & 1, u = it >> 1;
                 const uint32_t sa = smem_u32(smem + st * kStageBytes), ta = sa + Cfg::kOffT, ma = sa + Cfg::kOffM;
-                if (!mbar_wait(&gen_full[st], u & 1)) { report_timeout(status, 902); break; }
+                if (!mbar_wait_c(&gen_full[st], u & 1)) { report_timeout(status, 902); break; }
                 tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)      // P = mono * Tsym^T
-                    umma_bf16(tmem + Cfg::kColP, smem_desc_sw128(ma + ks * 32, 16, 1024), smem_desc_sw128(ta + ks * 32, 16, 1024), id_p, ks > 0 ? 1u : 0u);
+                {      // P = mono * Tsym^T
+                    uint64_t da = smem_desc_sw128(ma, 16, 1024), db = smem_desc_sw128(ta, 16, 1024);
+#pragma unroll 1
+                    for (int ks = 0; ks < 4; ++ks, da += 2, db += 2) umma_bf16(tmem + Cfg::kColP, da, db, id_p, ks > 0 ? 1u : 0u);
+                }
                 umma_commit(p_full);
-                if (!(mbar_wait(b3_ready, it & 1) && mbar_wait(acc_free, (it & 1) ^ 1))) { report_timeout(status, 903); break; }
+                // the state product waits until the state after the previous tile has been read out of tensor memory, not
+                // until its image is written; the first tile of a piece waits for the initial state
+                if (it > 0 && !mbar_wait_c(state_read, (it - 1) & 1)) { report_timeout(status, 911); break; }
+                if ((it == 0 || (w0 + it) % T == 0) && !mbar_wait_c(b3_ready, it & 1)) { report_timeout(status, 903); break; }
+                if (!mbar_wait_c(&v_full[st], u & 1)) { report_timeout(status, 904); break; }
                 tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)      // acc = mono * [Csym | zsym] of the tokens before the tile
-                    umma_bf16(tmem + Cfg::kColAcc, smem_desc_sw128(ma + ks * 32, 16, 1024), smem_desc_sw128(b3a + ks * 2048, Cfg::kB3Block, 1024), id_r,
-                              ks > 0 ? 1u : 0u);
-                if (!mbar_wait(&v_full[st], u & 1)) { report_timeout(status, 904); break; }
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < kTileTokens / 16; ++ks)      // state += Tsym^T * [V | 1]
-                    umma_bf16(tmem + Cfg::kColState, smem_desc_sw128(ta + ks * 2048, kBlk, 1024), smem_desc_sw128(sa + ks * 2048, kBlk, 1024), id_s, 1u);
+                {      // state += Tsym^T * [V | 1]
+                    uint64_t da = smem_desc_sw128(ta, kBlk, 1024), db = smem_desc_sw128(sa, kBlk, 1024);
+#pragma unroll 1
+                    for (int ks = 0; ks < kTileTokens / 16; ++ks, da += 128, db += 128) umma_bf16(tmem + Cfg::kColState, da, db, id_s, 1u);
+                }
                 umma_commit(state_full);
-                if (!mbar_wait(pm_ready, it & 1)) { report_timeout(status, 905); break; }
+                if (!(mbar_wait_c(b3_ready, it & 1) && mbar_wait_c(acc_free, (it & 1) ^ 1))) { report_timeout(status, 903); break; }
                 tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < kTileTokens / 16; ++ks)      // acc += Pm * [V | 1]
-                    umma_bf16_ta(tmem + Cfg::kColAcc, tmem + Cfg::kColP + 8 * ks, smem_desc_sw128(sa + ks * 2048, kBlk, 1024), id_r, 1u);
+                const uint32_t b3a = b3base + (it & 1) * Cfg::kB3Bytes;
+                {      // acc = mono * [Csym | zsym] of the tokens before the tile
+                    uint64_t da = smem_desc_sw128(ma, 16, 1024), db = smem_desc_sw128(b3a, Cfg::kB3Block, 1024);
+#pragma unroll 1
+                    for (int ks = 0; ks < 4; ++ks, da += 2, db += 128) umma_bf16(tmem + Cfg::kColAcc, da, db, id_r, ks > 0 ? 1u : 0u);
+                }
+                if (!mbar_wait_c(pm_ready, it & 1)) { report_timeout(status, 905); break; }
+                tc_fence_after();
+                {      // acc += Pm * [V | 1]
+                    uint64_t db = smem_desc_sw128(sa, kBlk, 1024);
+#pragma unroll 1
+                    for (int ks = 0; ks < kTileTokens / 16; ++ks, db += 128) umma_bf16_ta(tmem + Cfg::kColAcc, tmem + Cfg::kColP + 8 * ks + (ks >= 4 ? 32 : 0), db, id_r, 1u);
+                }
                 umma_commit(acc_full);
                 umma_commit(&stage_free[st]);
             }
         }
-    } else if (warp < kCaMaskWarp0) {
-        // operand rows: thread = token row of the tile
-        const int row = tid - kCaGenWarp0 * 32;
-        float qn[6], kn[18];
+    } else if (warp < kCaGenKWarp0) {
+        // monomial rows of the queries: thread = token row of the tile
+        const int row = tid - kCaGenQWarp0 * 32;
+        float qn[6];
         auto prefetch = [&](int it) {
             const int work = w0 + it, bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
             load_feat<6>(qn, qf + ((size_t)bh * N + tok) * 6);
+        };
+        if (nwork > 0) prefetch(0);
+        for (int it = 0; it < nwork; ++it) {
+            const int st = it & 1, u = it >> 1, work = w0 + it;
+            const bool valid = (work % T) * kTileTokens + row < N;
+            float q[6];
+#pragma unroll
+            for (int i = 0; i < 6; ++i) q[i] = valid ? qn[i] : 0.f;
+            if (ok && !mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 906); }
+            if (!ok) continue;
+            shifted_mono_row(smem_u32(smem + st * kStageBytes) + Cfg::kOffM, row, q, std::make_integer_sequence<int, 7>{});
+            fence_proxy_async();
+            mbar_arrive(&gen_full[st]);
+            if (it + 1 < nwork) prefetch(it + 1);      // after the fence: a fence waits for the loads in flight
+        }
+    } else if (warp < kCaMaskWarp0) {
+        // folded key rows
+        const int row = tid - kCaGenKWarp0 * 32;
+        float kn[18];
+        auto prefetch = [&](int it) {
+            const int work = w0 + it, bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
 #pragma unroll
             for (int f = 0; f < 3; ++f) load_feat<6>(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
         };
@@ -227,56 +298,57 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
         for (int it = 0; it < nwork; ++it) {
             const int st = it & 1, u = it >> 1, work = w0 + it;
             const bool valid = (work % T) * kTileTokens + row < N;
-            float q[6], k[18];
-#pragma unroll
-            for (int i = 0; i < 6; ++i) q[i] = valid ? qn[i] : 0.f;
+            float k[18];
 #pragma unroll
             for (int i = 0; i < 18; ++i) k[i] = valid ? kn[i] : 0.f;
-            if (it + 1 < nwork) prefetch(it + 1);
-            if (ok && !mbar_wait(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 906); }
+            if (ok && !mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 910); }
             if (!ok) continue;
-            const uint32_t sa = smem_u32(smem + st * kStageBytes);
-            {
-                float mono[kMono];
-                query_monomials_t<3>(q, mono);
-                store_shifted_row(sa + Cfg::kOffM, row, 0.f, mono);
+            float s12[6][6], k3[6];      // [x][y], x < y: k1[x] k2[y] + k1[y] k2[x];  [x][x]: k1[x] k2[x]
+#pragma unroll
+            for (int x = 0; x < 6; ++x) {
+                k3[x] = k[12 + x];
+#pragma unroll
+                for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k[x] * k[6 + x] : fmaf(k[x], k[6 + y], k[y] * k[6 + x]);
             }
-            {
-                float ts[kMono];
-                key_folded_t<3>(k, ts);
-                store_shifted_row(sa + Cfg::kOffT, row, valid ? 1.f : 0.f, ts);
-            }
+            shifted_key_row(smem_u32(smem + st * kStageBytes) + Cfg::kOffT, row, valid ? 1.f : 0.f, s12, k3, std::make_integer_sequence<int, 7>{});
             fence_proxy_async();
             mbar_arrive(&gen_full[st]);
+            if (it + 1 < nwork) prefetch(it + 1);
         }
     } else if (warp < kCaConvWarp0) {
-        // mask: thread = query row i of the block; keeps the columns j <= i, rounds to bf16, writes the block back in place
-        const int qt = warp & 3, row = qt * 32 + lane;
-        const uint32_t pa = tmem + Cfg::kColP + ((uint32_t)(qt * 32) << 16);
+        // mask: thread = query row i of the block, two warps per 32 rows: warp (qt, half) owns the columns 64 half .. 64 half
+        // + 63 of the rows 32 qt .. 32 qt + 31.  A 32 x 32 sub-block left of the diagonal is kept whole, right of it dropped;
+        // only the diagonal one is cut element by element.  Each warp packs its 64 columns over the first 32 of them.
+        const int qt = warp & 3, half = (warp - kCaMaskWarp0) >> 2;
+        const uint32_t pa = tmem + Cfg::kColP + 64 * half + ((uint32_t)(qt * 32) << 16);
         for (int it = 0; it < nwork; ++it) {
-            if (ok && !mbar_wait(p_full, it & 1)) { ok = false; report_timeout(status, 907); }
+            if (ok && !mbar_wait_c(p_full, it & 1)) { ok = false; report_timeout(status, 907); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
+#pragma unroll 1
+            for (int bb = 0; bb < 2; ++bb) {      // sub-block column 2 half + bb against sub-block row qt
+                const int b = 2 * half + bb;
                 uint32_t w[16];
-                if (b <= qt) {      // columns 32 b .. 32 b + 31; a warp's rows are 32 qt .. 32 qt + 31
+                if (b <= qt) {
                     uint32_t r[32];
-                    tmem_ld16(pa + 32 * b, *reinterpret_cast<uint32_t(*)[16]>(r));
-                    tmem_ld16(pa + 32 * b + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
+                    tmem_ld16(pa + 32 * bb, *reinterpret_cast<uint32_t(*)[16]>(r));
+                    tmem_ld16(pa + 32 * bb + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
                     tmem_ld_wait();
+                    if (b < qt) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int j = 32 * b + 2 * e;
-                        w[e] = pack_bf16(j <= row ? __uint_as_float(r[2 * e]) : 0.f, j + 1 <= row ? __uint_as_float(r[2 * e + 1]) : 0.f);
+                        for (int e = 0; e < 16; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            w[e] = pack_bf16(2 * e <= lane ? __uint_as_float(r[2 * e]) : 0.f, 2 * e + 1 <= lane ? __uint_as_float(r[2 * e + 1]) : 0.f);
                     }
                 } else {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) w[e] = 0u;
                 }
-                tmem_st8(pa + 16 * b, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
-                tmem_st8(pa + 16 * b + 8, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+                tmem_st8(pa + 16 * bb, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                tmem_st8(pa + 16 * bb + 8, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
             }
             tmem_st_wait();
             tc_fence_before();
@@ -287,12 +359,12 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
         const int qt = warp & 3, R = qt * 16 + lane, m = R - kCaRowPad;
         const bool active = lane < 16, mine = active && m >= 0 && m < kMono;
         const uint32_t sa = tmem + Cfg::kColState + ((uint32_t)(qt * 32) << 16);
-        const uint32_t b3a = smem_u32(smem + Cfg::kOffB3);
+        const uint32_t b3base = smem_u32(smem + Cfg::kOffB3);
         constexpr int kChunks = Cfg::kNAcc / 8;      // 16-byte chunks of an image row
-        auto store_chunk = [&](int c, const float (&v)[8]) {
+        auto store_chunk = [&](int img, int c, const float (&v)[8]) {      // image `img` is the one item `img` (mod 2) reads
             if (active)
-                st_shared_v4(b3a + (c >> 3) * Cfg::kB3Block + sw128_off(R, c & 7), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
-                             pack_bf16(v[6], v[7]));
+                st_shared_v4(b3base + (img & 1) * Cfg::kB3Bytes + (c >> 3) * Cfg::kB3Block + sw128_off(R, c & 7), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]),
+                             pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
         };
         for (int it = 0; it < nwork; ++it) {
             const int work = w0 + it, bh = work / T;
@@ -315,36 +387,50 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                     if (8 * c < Cfg::kNState)
                         tmem_st8(sa + 8 * c, __float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]), __float_as_uint(v[4]),
                                  __float_as_uint(v[5]), __float_as_uint(v[6]), __float_as_uint(v[7]));
-                    store_chunk(c, v);
+                    store_chunk(it, c, v);
                 }
                 tmem_st_wait();
                 tc_fence_before();
                 fence_proxy_async();
                 mbar_arrive(b3_ready);
             }
-            if (ok && !mbar_wait(state_full, it & 1)) { ok = false; report_timeout(status, 908); }
+            if (ok && !mbar_wait_c(state_full, it & 1)) { ok = false; report_timeout(status, 908); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (it + 1 < nwork && (work + 1) % T != 0) {
                 tc_fence_after();
+                // 32 columns per batch of loads; column d (zsym) rides with the last batch.  The state product of the next tile
+                // may run as soon as the last load has completed.  Rows that hold no monomial stay zero.
+                const uint32_t img = b3base + ((it + 1) & 1) * Cfg::kB3Bytes;
 #pragma unroll 1
-                for (int c = 0; c < kChunks; ++c) {
-                    float v[8];
-                    if (8 * c < Cfg::kNState) {
-                        uint32_t r[8];
-                        tmem_ld8(sa + 8 * c, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) v[e] = mine && (8 * c + e <= DV) ? __uint_as_float(r[e]) : 0.f;
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) v[e] = 0.f;
+                for (int h = 0; h < DV / 32; ++h) {
+                    uint32_t r[32], rz[8];
+                    tmem_ld16(sa + 32 * h, *reinterpret_cast<uint32_t(*)[16]>(r));
+                    tmem_ld16(sa + 32 * h + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
+                    if (h == DV / 32 - 1) tmem_ld8(sa + DV, rz);
+                    tmem_ld_wait();
+                    if (h == DV / 32 - 1) {
+                        tc_fence_before();
+                        mbar_arrive(state_read);
                     }
-                    store_chunk(c, v);
+                    if (mine) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int cc = 4 * h + c;      // 16-byte chunk of the image row
+                            st_shared_v4(img + (cc >> 3) * Cfg::kB3Block + sw128_off(R, cc & 7), pack_bf16(__uint_as_float(r[8 * c]), __uint_as_float(r[8 * c + 1])),
+                                         pack_bf16(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3])),
+                                         pack_bf16(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5])),
+                                         pack_bf16(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7])));
+                        }
+                        if (h == DV / 32 - 1)
+                            st_shared_v4(img + (DV / 64) * Cfg::kB3Block + sw128_off(R, 0), pack_bf16(__uint_as_float(rz[0]), 0.f), 0u, 0u, 0u);
+                    }
                 }
                 tc_fence_before();
                 fence_proxy_async();
                 mbar_arrive(b3_ready);
+            } else {
+                mbar_arrive(state_read);      // nothing is read: the next tile (if any) starts a piece with a state of its own
             }
         }
     } else {
@@ -354,7 +440,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
         const uint32_t os = smem_u32(smem + Cfg::kOffO);
         for (int it = 0; it < nwork; ++it) {
             const int work = w0 + it, bh = work / T, tile = work % T;
-            if (!mbar_wait(acc_full, it & 1)) {
+            if (!mbar_wait_c(acc_full, it & 1)) {
                 report_timeout(status, 909);
                 *abort_flag = 1;
             }
@@ -367,19 +453,19 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             tmem_ld_wait();
             const float eta = __uint_as_float(re[0]);
             const float rinv = 1.f / (eta + eps);
-#pragma unroll
-            for (int h = 0; h < Cfg::kVB; ++h) {
-                uint32_t r[64];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld16(aa + 64 * h + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(r + 16 * c));
+#pragma unroll 1
+            for (int h = 0; h < DV / 32; ++h) {
+                uint32_t r[32];
+                tmem_ld16(aa + 32 * h, *reinterpret_cast<uint32_t(*)[16]>(r));
+                tmem_ld16(aa + 32 * h + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
                 tmem_ld_wait();
-                if (h == Cfg::kVB - 1) {
+                if (h == DV / 32 - 1) {
                     tc_fence_before();
                     mbar_arrive(acc_free);
                 }
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    st_shared_v4(os + h * kBlk + sw128_off(row, c), pack_bf16(__uint_as_float(r[8 * c]) * rinv, __uint_as_float(r[8 * c + 1]) * rinv),
+                for (int c = 0; c < 4; ++c)
+                    st_shared_v4(os + (h >> 1) * kBlk + sw128_off(row, 4 * (h & 1) + c), pack_bf16(__uint_as_float(r[8 * c]) * rinv, __uint_as_float(r[8 * c + 1]) * rinv),
                                  pack_bf16(__uint_as_float(r[8 * c + 2]) * rinv, __uint_as_float(r[8 * c + 3]) * rinv),
                                  pack_bf16(__uint_as_float(r[8 * c + 4]) * rinv, __uint_as_float(r[8 * c + 5]) * rinv),
                                  pack_bf16(__uint_as_float(r[8 * c + 6]) * rinv, __uint_as_float(r[8 * c + 7]) * rinv));

@@ -68,6 +68,27 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
         if (global_timer_ns() - t0 > limit_ns) return false;
     return true;
 }
+// The same wait with its polling loop out of line: a kernel with many wait sites and many warp roles keeps its
+// instruction footprint (and with it the misses of the per-SM instruction cache) small this way.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity) {
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar_addr), "r"(parity), "r"(kWaitHintNs)
+            : "memory");
+        if (ok) return true;
+        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+__device__ __forceinline__ bool mbar_wait_c(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(smem_u32(bar), parity);
+}
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05.mma operand reads)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
