@@ -24,7 +24,7 @@
 // State row 8 + m holds [Csym[m][0..d), zsym[m], 0 ...]; rows 0..7 are kept zero in the bf16 image.  The image is
 // double-buffered: the image for tile t + 1 is written while the products of tile t still read theirs.
 //
-// Warp roles: 0 TMA (value tiles), 1 MMA issue, 2..5 monomial rows of q, 6..9 folded key rows, 10..17 mask (two warps
+// Warp roles: 0 TMA (value tiles), 1 MMA issue (P, readout, Pm * V), 26 MMA issue (state), 2..5 monomial rows of q, 6..9 folded key rows, 10..17 mask (two warps
 // per 32 rows, 64 columns each), 18..21 state image, 22..25 epilogue.  A role is one warp per scheduler running a
 // straight instruction stream per tile, so what bounds a tile is the longest of these streams: they are kept short
 // (selects only where the mask cuts a 32 x 32 block, conversions 32 columns at a time, out-of-line waits, rolled loops).
@@ -35,7 +35,8 @@
 namespace hla {
 namespace tc {
 
-constexpr int kCaThreads = 26 * 32;
+constexpr int kCaThreads = 27 * 32;
+constexpr int kCaStateMmaWarp = 26;
 constexpr int kCaGenQWarp0 = 2, kCaGenKWarp0 = 6, kCaMaskWarp0 = 10, kCaConvWarp0 = 18, kCaEpiWarp0 = 22;
 constexpr int kCaRowPad = 8;      // operand column / state row of monomial 0
 
@@ -155,18 +156,21 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
-    uint64_t* v_full = bars;              // [2] TMA
-    uint64_t* gen_full = bars + 2;        // [2] 256 arrivals: both operand-row tiles of the stage are written
-    uint64_t* stage_free = bars + 4;      // [2] MMA commit: every product that reads the stage has finished
-    uint64_t* p_full = bars + 6;          // MMA commit
-    uint64_t* pm_ready = bars + 7;        // 256 arrivals: masked bf16 block is in tensor memory
-    uint64_t* b3_ready = bars + 8;        // 128 arrivals: state image (and, at the start of a piece, the state) is in place
-    uint64_t* state_full = bars + 9;      // MMA commit
-    uint64_t* acc_full = bars + 10;       // MMA commit
-    uint64_t* acc_free = bars + 11;       // 128 arrivals
-    uint64_t* state_read = bars + 12;     // 128 arrivals: the state after a tile has been read out of tensor memory
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 14);
+    uint64_t* stage_ready = bars;         // [2] 256 arrivals + the TMA transaction: operand-row tiles written, value tile landed
+    uint64_t* stage_free = bars + 2;      // [2] 2 MMA commits (one per issuing thread): every product that reads the stage has finished
+    uint64_t* p_full = bars + 4;          // MMA commit
+    uint64_t* pm_ready = bars + 5;        // 256 arrivals: masked bf16 block is in tensor memory
+    uint64_t* b3_ready = bars + 15;       // [2] 128 arrivals, barrier it & 1: state image of tile it (at the start of a piece also the
+                                          // state) is in place; two barriers because the image of tile it + 1 can be ready before
+                                          // the readout of tile it has waited
+    uint64_t* acc_free = bars + 12;       // 128 arrivals: the accumulator has been drained
+    uint64_t* rd_done = bars + 13;        // [2] MMA commit after the readout of tile it, on barrier it & 1 (a waiter may lag two
+                                          // tiles behind the issuing thread, which one barrier's phase parity cannot tell apart)
+    uint64_t* state_full = bars + 7;      // MMA commit
+    uint64_t* acc_full = bars + 8;        // MMA commit
+    uint64_t* state_read = bars + 9;      // 128 arrivals: the state after a tile has been read out of tensor memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 11);      // (bars + 12: acc_free)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int T = (N + kTileTokens - 1) / kTileTokens;
@@ -176,16 +180,18 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
 
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&v_full[i], 1);
-            mbar_init(&gen_full[i], 256);
-            mbar_init(&stage_free[i], 1);
+            mbar_init(&stage_ready[i], 257);
+            mbar_init(&stage_free[i], 2);
         }
         mbar_init(p_full, 1);
         mbar_init(pm_ready, 256);
-        mbar_init(b3_ready, 128);
+        mbar_init(&b3_ready[0], 128);
+        mbar_init(&b3_ready[1], 128);
+        mbar_init(acc_free, 128);
+        mbar_init(&rd_done[0], 1);
+        mbar_init(&rd_done[1], 1);
         mbar_init(state_full, 1);
         mbar_init(acc_full, 1);
-        mbar_init(acc_free, 128);
         mbar_init(state_read, 128);
         *abort_flag = 0;
         fence_mbar_init();
@@ -211,20 +217,19 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             for (int it = 0; it < nwork; ++it) {
                 const int st = it & 1, u = it >> 1, work = w0 + it;
                 if (!mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { report_timeout(status, 901); break; }
-                mbar_arrive_expect_tx(&v_full[st], DV * kTileTokens * 2);
-                for (int b = 0; b < Cfg::kVB; ++b) tma_load_3d(smem + st * kStageBytes + b * kBlk, &mapV, &v_full[st], b * 64, (work % T) * kTileTokens, work / T);
+                mbar_arrive_expect_tx(&stage_ready[st], DV * kTileTokens * 2);
+                for (int b = 0; b < Cfg::kVB; ++b) tma_load_3d(smem + st * kStageBytes + b * kBlk, &mapV, &stage_ready[st], b * 64, (work % T) * kTileTokens, work / T);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t id_p = idesc_bf16(128, 128, false, false);
             const uint32_t id_r = idesc_bf16(128, Cfg::kNAcc, false, true);
-            const uint32_t id_s = idesc_bf16(64, Cfg::kNState, true, true);
             const uint32_t b3base = smem_u32(smem + Cfg::kOffB3);
             for (int it = 0; it < nwork; ++it) {
                 const int st = it & 1, u = it >> 1;
                 const uint32_t sa = smem_u32(smem + st * kStageBytes), ta = sa + Cfg::kOffT, ma = sa + Cfg::kOffM;
-                if (!mbar_wait_c(&gen_full[st], u & 1)) { report_timeout(status, 902); break; }
+                if (!mbar_wait_c(&stage_ready[st], u & 1)) { report_timeout(status, 902); break; }
                 tc_fence_after();
                 {      // P = mono * Tsym^T
                     uint64_t da = smem_desc_sw128(ma, 16, 1024), db = smem_desc_sw128(ta, 16, 1024);
@@ -232,19 +237,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                     for (int ks = 0; ks < 4; ++ks, da += 2, db += 2) umma_bf16(tmem + Cfg::kColP, da, db, id_p, ks > 0 ? 1u : 0u);
                 }
                 umma_commit(p_full);
-                // the state product waits until the state after the previous tile has been read out of tensor memory, not
-                // until its image is written; the first tile of a piece waits for the initial state
-                if (it > 0 && !mbar_wait_c(state_read, (it - 1) & 1)) { report_timeout(status, 911); break; }
-                if ((it == 0 || (w0 + it) % T == 0) && !mbar_wait_c(b3_ready, it & 1)) { report_timeout(status, 903); break; }
-                if (!mbar_wait_c(&v_full[st], u & 1)) { report_timeout(status, 904); break; }
-                tc_fence_after();
-                {      // state += Tsym^T * [V | 1]
-                    uint64_t da = smem_desc_sw128(ta, kBlk, 1024), db = smem_desc_sw128(sa, kBlk, 1024);
-#pragma unroll 1
-                    for (int ks = 0; ks < kTileTokens / 16; ++ks, da += 128, db += 128) umma_bf16(tmem + Cfg::kColState, da, db, id_s, 1u);
-                }
-                umma_commit(state_full);
-                if (!(mbar_wait_c(b3_ready, it & 1) && mbar_wait_c(acc_free, (it & 1) ^ 1))) { report_timeout(status, 903); break; }
+                if (!(mbar_wait_c(&b3_ready[it & 1], (it >> 1) & 1) && mbar_wait_c(acc_free, (it & 1) ^ 1))) { report_timeout(status, 903); break; }
                 tc_fence_after();
                 const uint32_t b3a = b3base + (it & 1) * Cfg::kB3Bytes;
                 {      // acc = mono * [Csym | zsym] of the tokens before the tile
@@ -252,14 +245,38 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
 #pragma unroll 1
                     for (int ks = 0; ks < 4; ++ks, da += 2, db += 128) umma_bf16(tmem + Cfg::kColAcc, da, db, id_r, ks > 0 ? 1u : 0u);
                 }
+                umma_commit(&rd_done[it & 1]);
                 if (!mbar_wait_c(pm_ready, it & 1)) { report_timeout(status, 905); break; }
                 tc_fence_after();
-                {      // acc += Pm * [V | 1]
+                {      // acc += Pm * [V | 1]; the two packed halves of Pm sit at columns 0..31 and 64..95 of the block
                     uint64_t db = smem_desc_sw128(sa, kBlk, 1024);
 #pragma unroll 1
                     for (int ks = 0; ks < kTileTokens / 16; ++ks, db += 128) umma_bf16_ta(tmem + Cfg::kColAcc, tmem + Cfg::kColP + 8 * ks + (ks >= 4 ? 32 : 0), db, id_r, 1u);
                 }
                 umma_commit(acc_full);
+                umma_commit(&stage_free[st]);
+            }
+        }
+    } else if (warp == kCaStateMmaWarp) {
+        // The state products are issued by a thread of their own: they depend on nothing the other products make, and the
+        // chain state -> image -> readout of consecutive tiles is the long one.
+        if (lane == 0) {
+            const uint32_t id_s = idesc_bf16(64, Cfg::kNState, true, true);
+            for (int it = 0; it < nwork; ++it) {
+                const int st = it & 1, u = it >> 1;
+                const uint32_t sa = smem_u32(smem + st * kStageBytes), ta = sa + Cfg::kOffT;
+                // the state after the previous tile must have been read out of tensor memory; the first tile of a piece
+                // waits for the initial state
+                if (it > 0 && !mbar_wait_c(state_read, (it - 1) & 1)) { report_timeout(status, 911); break; }
+                if ((it == 0 || (w0 + it) % T == 0) && !mbar_wait_c(&b3_ready[it & 1], (it >> 1) & 1)) { report_timeout(status, 912); break; }
+                if (!mbar_wait_c(&stage_ready[st], u & 1)) { report_timeout(status, 904); break; }
+                tc_fence_after();
+                {      // state += Tsym^T * [V | 1]
+                    uint64_t da = smem_desc_sw128(ta, kBlk, 1024), db = smem_desc_sw128(sa, kBlk, 1024);
+#pragma unroll 1
+                    for (int ks = 0; ks < kTileTokens / 16; ++ks, da += 128, db += 128) umma_bf16(tmem + Cfg::kColState, da, db, id_s, 1u);
+                }
+                umma_commit(state_full);
                 umma_commit(&stage_free[st]);
             }
         }
@@ -282,7 +299,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             if (!ok) continue;
             shifted_mono_row(smem_u32(smem + st * kStageBytes) + Cfg::kOffM, row, q, std::make_integer_sequence<int, 7>{});
             fence_proxy_async();
-            mbar_arrive(&gen_full[st]);
+            mbar_arrive(&stage_ready[st]);
             if (it + 1 < nwork) prefetch(it + 1);      // after the fence: a fence waits for the loads in flight
         }
     } else if (warp < kCaMaskWarp0) {
@@ -312,7 +329,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             }
             shifted_key_row(smem_u32(smem + st * kStageBytes) + Cfg::kOffT, row, valid ? 1.f : 0.f, s12, k3, std::make_integer_sequence<int, 7>{});
             fence_proxy_async();
-            mbar_arrive(&gen_full[st]);
+            mbar_arrive(&stage_ready[st]);
             if (it + 1 < nwork) prefetch(it + 1);
         }
     } else if (warp < kCaConvWarp0) {
@@ -392,12 +409,16 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                 tmem_st_wait();
                 tc_fence_before();
                 fence_proxy_async();
-                mbar_arrive(b3_ready);
+                mbar_arrive(&b3_ready[it & 1]);
             }
             if (ok && !mbar_wait_c(state_full, it & 1)) { ok = false; report_timeout(status, 908); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (it + 1 < nwork && (work + 1) % T != 0) {
+                // the image written now was last read by the readout of the previous tile (issued by the other thread)
+                if (it > 0 && ok && !mbar_wait_c(&rd_done[(it - 1) & 1], ((it - 1) >> 1) & 1)) { ok = false; report_timeout(status, 913); }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
                 tc_fence_after();
                 // 32 columns per batch of loads; column d (zsym) rides with the last batch.  The state product of the next tile
                 // may run as soon as the last load has completed.  Rows that hold no monomial stay zero.
@@ -428,7 +449,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                 }
                 tc_fence_before();
                 fence_proxy_async();
-                mbar_arrive(b3_ready);
+                mbar_arrive(&b3_ready[(it + 1) & 1]);
             } else {
                 mbar_arrive(state_read);      // nothing is read: the next tile (if any) starts a piece with a state of its own
             }
