@@ -244,7 +244,8 @@ class Workload:
         del Q, K, V
         pq, pk = synth.make_phi_weights(shape.d, shape.d_phi, shape.F, shape.dtype)
         to_dev = lambda a: torch.from_numpy(a).to(tdt).to(dev)
-        self.op = binding.Hla(shape.B, shape.H, shape.N, shape.d, dtype=shape.dtype, phi="mlp", F=shape.F, d_phi=shape.d_phi, eps=1e-6, device=dev)
+        self.op = binding.Hla(shape.B, shape.H, shape.N, shape.d, dtype=shape.dtype, phi="mlp", F=shape.F, d_phi=shape.d_phi, eps=1e-6, device=dev,
+                              causal=shape.causal)
         self.op.set_phi(tuple(to_dev(a) for a in pq), [tuple(to_dev(a) for a in w) for w in pk])
         self.O = torch.empty_like(self.V)
         self.dQ, self.dK, self.dV = (torch.empty_like(self.V) for _ in range(3)) if shape.backward else (None, None, None)
@@ -294,8 +295,9 @@ class Workload:
         return kt
 
 
-def value_mod_leg(shape, w, dev):
-    """hla_value_mod_forward (+ backward for workloads with a backward) on the workload's O and V, sustained like the rest."""
+def value_mod_leg(shape, w, dev, short=False):
+    """hla_value_mod_forward (+ backward for workloads with a backward) on the workload's O and V, sustained like the rest
+    (short: three calls only, for a profiler capture)."""
     import torch
     from paper_2602_12128_b200 import binding
     tdt = torch.bfloat16
@@ -325,6 +327,8 @@ def value_mod_leg(shape, w, dev):
     torch.cuda.synchronize()
     if op.device_status() != binding.HLA_OK:
         raise SystemExit("device-side wait timed out (value modulation)")
+    if short:
+        return None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(5):
@@ -371,7 +375,7 @@ def extra_leg(name, rank, dev, peaks, local):
     fl, _ = work_model(shape)
     roof = roofline_of(shape, ms, 1, peaks)
     roof.pop("peaks")
-    out = {"config": {"B": shape.B, "H": shape.H, "N": shape.N, "d": shape.d, "pass": "fwd+bwd" if shape.backward else "fwd"},
+    out = {"config": {"B": shape.B, "H": shape.H, "N": shape.N, "d": shape.d, "pass": "fwd+bwd" if shape.backward else "fwd", "causal": bool(shape.causal)},
            "ms_per_step": ms, "steps": n, "tflops": fl / (ms * 1e-3) / 1e12, "tokens_per_s": shape.B * shape.N / (ms * 1e-3),
            "gpu_launches_per_step": w.launches, "step_roofline": roof,
            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_min_mhz", "power_w", "reasons", "samples_under_load")}}
@@ -396,6 +400,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations (the `extra` object of the line)")
     ap.add_argument("--profile", action="store_true", help="only warm-up and the timed steps: no sustained phase, no extra legs (for ncu)")
+    ap.add_argument("--also", default="", help="with --profile: comma list of side calls to run three times after the steps "
+                    "(weights = hla_backward_weights, vmod = hla_value_mod_forward/backward), so that a capture can name their kernels")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.profile:
@@ -587,6 +593,16 @@ def main():
                  "products per map (the recomputed hidden layer is not counted)"}
         del gq, gk
 
+    if args.profile and world == 1:
+        also = [a for a in args.also.split(",") if a]
+        if "weights" in also and shape.backward:
+            gq, gk = op.backward_weights(w.Q, w.K)
+            for _ in range(2):
+                binding.hla_backward_weights(op.ctx, w.Q, w.K, gq, gk, op.workspace)
+            torch.cuda.synchronize()
+        if "vmod" in also:
+            value_mod_leg(shape, w, dev, short=True)
+
     # ---- value modulation of the attention result (Section 4.5; separate calls, not part of `value`) --------------------
     vmod = None
     if not args.profile and world == 1 and shape.dtype == "bf16" and shape.d in (64, 128):
@@ -600,7 +616,7 @@ def main():
         del w, op
         torch.cuda.empty_cache()
         extra = {}
-        for name in ("long_bf16", "dit_bf16", "small_bf16", "paper_r1_bf16", "paper_r2_bf16", "train_bf16_2f"):
+        for name in ("long_bf16", "dit_bf16", "small_bf16", "paper_r1_bf16", "paper_r2_bf16", "train_bf16_2f", "train_bf16_causal"):
             if name != shape.name:
                 extra[name] = extra_leg(name, rank, dev, peaks, local)
 

@@ -31,6 +31,7 @@ class HlaShape:
     backward: bool = False
     F: int = 3
     d_phi: int = 6
+    causal: bool = False
 
 
 # The five configurations of the benchmark definition.
@@ -50,6 +51,9 @@ CONFIGS["paper_r2_bf16"] = HlaShape("paper_r2_bf16", 1, 12, 12600, 128, "bf16", 
 
 # The paper's 2-factor variant (appendix "Defining phi": 12 feature channels for 2 factors; Table 2 row HLA-2F-R1-21) at the training-step shape.
 CONFIGS["train_bf16_2f"] = HlaShape("train_bf16_2f", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=True, F=2, d_phi=12)
+
+# Causal HLA (Section 4.4: token i sees the tokens j <= i) at the training-step shape.
+CONFIGS["train_bf16_causal"] = HlaShape("train_bf16_causal", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=False, causal=True)
 
 
 def bf16_round(x: np.ndarray) -> np.ndarray:
