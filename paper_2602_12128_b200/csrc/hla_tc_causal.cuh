@@ -138,10 +138,16 @@ __global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__
     if (e >= n_per) return;
     float* p = part + (size_t)bh * S * n_per + e;
     float run = 0.f;
-    for (int s = 0; s < count; ++s) {
-        const float t = p[(size_t)s * n_per];
-        p[(size_t)s * n_per] = run;
-        run += t;
+    for (int s0 = 0; s0 < count; s0 += 8) {      // eight independent loads in flight, then the scan in piece order
+        float t[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) t[k] = s0 + k < count ? p[(size_t)(s0 + k) * n_per] : 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (s0 + k < count) {
+                p[(size_t)(s0 + k) * n_per] = run;
+                run += t[k];
+            }
     }
     state[(size_t)bh * n_per + e] = run;
 }

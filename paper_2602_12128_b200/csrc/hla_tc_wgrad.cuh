@@ -409,35 +409,57 @@ struct WgradOut {
     float* dW2[4];
     float* db2[4];
 };
+// Sum of the per-CTA partials in a fixed order (bit-reproducible): a block owns 32 consecutive outputs, warp w adds the
+// partials of the CTAs w, w + 8, ... (coalesced 128-byte reads, a dozen and a half independent loads per thread), and
+// the eight warp sums are added in warp order.
 template <int DV, int DP>
 __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __restrict__ wpart, WgradOut out, int nmaps_in_part, int map0, int nctas) {
     using C1 = WgCfg<DV, 1, DP>;
     constexpr int PF = C1::kPartFloats, oW2 = C1::kPartW2, oB1 = C1::kPartB1, oB2 = C1::kPartB2, W2C = C1::kW2Cols;
+    __shared__ float red[8][32];
     grid_launch_dependents();
     grid_dependency_wait();
     const int m = blockIdx.y;                        // map of this launch
     const int total = DV * DV + DV * DP + DV + DP;   // outputs of one map
-    for (int i = blockIdx.x * 256 + threadIdx.x; i < total; i += gridDim.x * 256) {
-        const float* src = wpart + (size_t)m * PF;
-        const size_t stride = (size_t)nmaps_in_part * PF;
-        float a = 0.f;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float* src = wpart + (size_t)m * PF;
+    const size_t stride = (size_t)nmaps_in_part * PF;
+    for (int base = blockIdx.x * 32; base < total; base += gridDim.x * 32) {
+        const int i = base + lane;
+        // an output is the sum over the CTAs of `nterm` partial entries `step` floats apart, starting at `off`
+        int off = 0, nterm = 0, step = 0;
+        float scale = 1.f;
         if (i < DV * DV) {
-            for (int c = 0; c < nctas; ++c) a += src[c * stride + i];
-            out.dW1[map0 + m][i] = a;
+            off = i; nterm = 1;
         } else if (i < DV * DV + DV * DP) {
             const int j = (i - DV * DV) / DP, o = (i - DV * DV) % DP;
-            for (int c = 0; c < nctas; ++c) a += src[c * stride + oW2 + j * W2C + o] + src[c * stride + oW2 + j * W2C + DP + o];
-            out.dW2[map0 + m][j * DP + o] = 0.5f * a;      // the G tile held 2 GELU(h)
+            off = oW2 + j * W2C + o; nterm = 2; step = DP; scale = 0.5f;      // the G tile held 2 GELU(h)
         } else if (i < DV * DV + DV * DP + DV) {
-            const int j = i - DV * DV - DV * DP;
-            for (int c = 0; c < nctas; ++c) a += src[c * stride + oB1 + j];
-            out.db1[map0 + m][j] = a;
-        } else {
-            const int o = i - DV * DV - DV * DP - DV;
-            for (int c = 0; c < nctas; ++c)
-                for (int q = 0; q < 4; ++q) a += src[c * stride + oB2 + q * 16 + o];
-            out.db2[map0 + m][o] = a;
+            off = oB1 + (i - DV * DV - DV * DP); nterm = 1;
+        } else if (i < total) {
+            off = oB2 + (i - DV * DV - DV * DP - DV); nterm = 4; step = 16;
         }
+        float a = 0.f;
+        if (nterm == 1) {
+#pragma unroll 4
+            for (int c = warp; c < nctas; c += 8) a += src[c * stride + off];
+        } else {
+            for (int c = warp; c < nctas; c += 8)
+                for (int q = 0; q < nterm; ++q) a += src[c * stride + off + q * step];
+        }
+        red[warp][lane] = a;
+        __syncthreads();
+        if (warp == 0 && i < total) {
+            float t = red[0][lane];
+#pragma unroll
+            for (int w = 1; w < 8; ++w) t += red[w][lane];
+            t *= scale;
+            if (i < DV * DV) out.dW1[map0 + m][i] = t;
+            else if (i < DV * DV + DV * DP) out.dW2[map0 + m][i - DV * DV] = t;
+            else if (i < DV * DV + DV * DP + DV) out.db1[map0 + m][i - DV * DV - DV * DP] = t;
+            else out.db2[map0 + m][i - DV * DV - DV * DP - DV] = t;
+        }
+        __syncthreads();
     }
 }
 
@@ -478,7 +500,7 @@ inline hla_status launch_phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, 
         o.dW1[0] = static_cast<float*>(dphi_q->dW1); o.db1[0] = static_cast<float*>(dphi_q->db1);
         o.dW2[0] = static_cast<float*>(dphi_q->dW2); o.db2[0] = static_cast<float*>(dphi_q->db2);
         rec.begin("tc_wgrad_reduce");
-        launch_pdl(tc_wgrad_reduce_kernel<DV, DP>, dim3(32, 1), dim3(256), 0, st, (const float*)wpart, o, 1, 0, grid);
+        launch_pdl(tc_wgrad_reduce_kernel<DV, DP>, dim3((DV * DV + DV * DP + DV + DP + 31) / 32, 1), dim3(256), 0, st, (const float*)wpart, o, 1, 0, grid);
         if (!rec.end()) return HLA_ERR_CUDA;
     }
     if (dphi_k) {
@@ -503,7 +525,7 @@ inline hla_status launch_phi_wgrad(const Dims& D, int BH, const hla_mlp* phi_q, 
                       reinterpret_cast<const float*>(ws + L.kf), reinterpret_cast<const float*>(ws + L.dkf), wpart, rows, D.N, status);
         if (!rec.end()) return HLA_ERR_CUDA;
         rec.begin("tc_wgrad_reduce");
-        launch_pdl(tc_wgrad_reduce_kernel<DV, DP>, dim3(32, NM), dim3(256), 0, st, (const float*)wpart, o, NM, 0, grid);
+        launch_pdl(tc_wgrad_reduce_kernel<DV, DP>, dim3((DV * DV + DV * DP + DV + DP + 31) / 32, NM), dim3(256), 0, st, (const float*)wpart, o, NM, 0, grid);
         if (!rec.end()) return HLA_ERR_CUDA;
     }
     return HLA_OK;
