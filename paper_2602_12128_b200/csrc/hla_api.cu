@@ -32,6 +32,7 @@ struct hla_ctx {
     bool vmod, phi_v_set;   // value modulation enabled at creation; its weights given
     hla_vmlp phi_v[2];
     tc::VmodPlan vmp;   // scratch of the value modulation inside the workspace
+    size_t off_delta;   // dO . o per token (scratch of the causal backward)
     size_t off_wpart;   // per-CTA partials of the weight gradients (scratch; tensor-core path with the phi maps)
     tc::Plan tcp;       // tensor-core operand buffers inside the workspace
     size_t ws_bytes;
@@ -316,6 +317,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     x->off_part = cv.take(part_bytes);
     x->off_wpart = (x->tc && mlp) ? cv.take(tc::wgrad_part_bytes(c.d, (long long)x->BH * c.N, x->sm_count)) : kNone;
     if (x->tc) cv.off = tc::plan(x->tcp, D, x->BH, cv.off);
+    x->off_delta = c.causal ? cv.take(tok * 4) : kNone;      // dO . o per token (causal backward)
     x->vmod = c.value_mod != 0;
     x->phi_v_set = false;
     if (x->vmod) cv.off = tc::vmod_plan(x->vmp, c.d, (long long)x->BH * c.N, cv.off);
@@ -400,7 +402,6 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     (void)cudaGetLastError();
     follow_device(ctx);
     tc::HostCacheScope scope(&ctx->hc);
-    if (ctx->cfg.causal) return HLA_ERR_UNSUPPORTED;
     if (ctx->tc) {
         const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
         // the phi backward writes rows of dQ, dK with 32-byte stores; so does the 2-factor key pass with dV
@@ -410,7 +411,13 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
         const float* kf = mlp ? reinterpret_cast<const float*>(ws + ctx->L.kf) : static_cast<const float*>(K);
         float* dqf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dqf) : static_cast<float*>(dQ);
         float* dkf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dkf) : static_cast<float*>(dK);
-        s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
+        if (ctx->cfg.causal) {
+            s = tc::causal_backward_values(ctx->D, ctx->BH, qf, kf, O, dO, dV, ws, ctx->L, ctx->off_part, ctx->off_delta, ctx->rec);
+            if (s != HLA_OK) return s;
+            return HLA_ERR_UNSUPPORTED;      // (feature gradients: next)
+        } else {
+            s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
+        }
         if (s != HLA_OK || !mlp) return s;
         return tc::phi_backward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, dQ, dK, ws, ctx->L, ctx->sm_count, ctx->rec);
     }

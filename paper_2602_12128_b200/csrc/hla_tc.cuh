@@ -397,9 +397,15 @@ template <int F> struct SbCfg {
     static constexpr int kTmemCols = F == 3 ? 64 : 128;
 };
 
-template <int DV, int F>
+// GRAD = false: the state of Theorem 4.2, rows = folded key features of `kf`, values = V.
+// GRAD = true (3 factors only): the gradient of that state when every token sees only the tokens up to itself,
+// [dCsym | dzsym] = sum_i r_i mono_i (x) [dO_i | -delta_i]: `kf` points to the query features, the value map to dO,
+// r_i = 1 / (eta_i + eps) and delta_i = dO_i . o_i come from `eta` and `delta`.
+template <int DV, int F, bool GRAD = false>
 __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __grid_constant__ CUtensorMap mapV, const float* __restrict__ kf,
-                                                                       float* __restrict__ part, int N, int S, int ld, int* status) {
+                                                                       float* __restrict__ part, int N, int S, int ld, int* status,
+                                                                       const float* __restrict__ eta = nullptr, const float* __restrict__ delta = nullptr,
+                                                                       float eps = 0.f) {
     using M = MT<F>;
     using Cfg = SbCfg<F>;
     constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
@@ -489,23 +495,42 @@ __global__ void __launch_bounds__(kSbThreads, 1) tc_state_build_kernel(const __g
         for (int i = 0; i < M::kN; ++i) zacc[i] = 0.f;
         // The key features of the group's next tile are loaded while the current one is processed (row index clamped:
         // the loads are unconditional, out-of-range rows are zeroed when used).
-        float k[M::kKf], kn[M::kKf];
+        float k[M::kKf], kn[M::kKf], en = 0.f, dn = 0.f;
         auto prefetch = [&](int it) {
             const int tok = min((tile0 + it) * kTileTokens + row, N - 1);
+            if constexpr (GRAD) {
+                load_feat<M::kDphi>(kn, kf + ((size_t)bh * N + tok) * M::kDphi);
+                en = __ldg(eta + (size_t)bh * N + tok);
+                dn = __ldg(delta + (size_t)bh * N + tok);
+            } else {
 #pragma unroll
-            for (int f = 0; f < F; ++f) load_feat<M::kDphi>(kn + M::kDphi * f, kf + (((size_t)bh * F + f) * N + tok) * M::kDphi);
+                for (int f = 0; f < F; ++f) load_feat<M::kDphi>(kn + M::kDphi * f, kf + (((size_t)bh * F + f) * N + tok) * M::kDphi);
+            }
         };
         if (grp < ntiles) prefetch(grp);
         for (int it = grp; it < ntiles; it += 2) {
             const int st = it % kStages, u = it / kStages;
             const int tok = (tile0 + it) * kTileTokens + row;
 #pragma unroll
-            for (int i = 0; i < M::kKf; ++i) k[i] = tok < N ? kn[i] : 0.f;
+            for (int i = 0; i < (GRAD ? M::kDphi : M::kKf); ++i) k[i] = tok < N ? kn[i] : 0.f;
+            const float rr = GRAD && tok < N ? 1.f / (en + eps) : 0.f, nd = -dn;
             if (it + 2 < ntiles) prefetch(it + 2);
             float ts[M::kN];
-            key_folded_t<F>(k, ts);
+            if constexpr (GRAD) {
+                float q[M::kDphi];
 #pragma unroll
-            for (int i = 0; i < M::kN; ++i) zacc[i] += ts[i];
+                for (int i = 0; i < M::kDphi; ++i) q[i] = k[i];
+                query_monomials_t<F>(q, ts);
+#pragma unroll
+                for (int i = 0; i < M::kN; ++i) {
+                    ts[i] *= rr;
+                    zacc[i] = fmaf(nd, ts[i], zacc[i]);
+                }
+            } else {
+                key_folded_t<F>(k, ts);
+#pragma unroll
+                for (int i = 0; i < M::kN; ++i) zacc[i] += ts[i];
+            }
             if (ok && !mbar_wait(&empty[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 103); }
             if (ok) {
                 store_mono_row_t<F>(smem_u32(smem + st * kStageBytes + 2 * kBlk), row, ts, 1.f);
@@ -1391,7 +1416,7 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
     if (!set_smem(tc_state_build_kernel<DV, F>, SbCfg<F>::kSmem) || !set_smem(tc_readout_kernel<DV, F>, RoCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
     rec.begin("tc_state_build");
-    launch_pdl(tc_state_build_kernel<DV, F>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<F>::kSmem, st, mapV, kf, part, D.N, D.S, D.ld, status);
+    launch_pdl(tc_state_build_kernel<DV, F>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<F>::kSmem, st, mapV, kf, part, D.N, D.S, D.ld, status, (const float*)nullptr, (const float*)nullptr, 0.f);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_reduce_emit");
     launch_pdl(tc_reduce_emit_kernel<DV, F>, dim3(kPad / 8, BH), dim3(256), 0, st, part, state, b3, bq, D.S, D.ld, 0, 0);

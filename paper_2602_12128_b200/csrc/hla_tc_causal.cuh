@@ -94,19 +94,21 @@ __device__ __forceinline__ void store_shifted_row(uint32_t blk, uint32_t row, fl
 
 // The same rows formed 16 bytes at a time, so that only a few values are live at once.  Chunk C (1..7) holds the
 // monomials 8 C - 8 .. 8 C - 1.
-template <int M> __device__ __forceinline__ float mono_value(const float (&q)[6]) {
+template <int M> __device__ __forceinline__ float mono_value(const float (&qs)[6], const float (&q)[6]) {
     constexpr int abc = mono_abc(M), a = abc / 36, b = (abc / 6) % 6, c = abc % 6;
-    return q[a] * q[b] * q[c];
+    return qs[a] * q[b] * q[c];
 }
 template <int C, int... E>
-__device__ __forceinline__ void shifted_mono_chunk(uint32_t blk, uint32_t row, const float (&q)[6], std::integer_sequence<int, E...>) {
-    const float v[8] = {mono_value<8 * (C - 1) + E>(q)...};
+__device__ __forceinline__ void shifted_mono_chunk(uint32_t blk, uint32_t row, const float (&qs)[6], const float (&q)[6], std::integer_sequence<int, E...>) {
+    const float v[8] = {mono_value<8 * (C - 1) + E>(qs, q)...};
     st_shared_v4(blk + sw128_off(row, C), pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
 }
+// [first, 0 x 7, qs_a q_b q_c ...]: qs = q gives the monomials, qs = r q the monomials scaled by r
 template <int... C>
-__device__ __forceinline__ void shifted_mono_row(uint32_t blk, uint32_t row, const float (&q)[6], std::integer_sequence<int, C...>) {
-    st_shared_v4(blk + sw128_off(row, 0), 0u, 0u, 0u, 0u);
-    (shifted_mono_chunk<C + 1>(blk, row, q, std::make_integer_sequence<int, 8>{}), ...);
+__device__ __forceinline__ void shifted_mono_row(uint32_t blk, uint32_t row, float first, const float (&qs)[6], const float (&q)[6],
+                                                 std::integer_sequence<int, C...>) {
+    st_shared_v4(blk + sw128_off(row, 0), pack_bf16(first, 0.f), 0u, 0u, 0u);
+    (shifted_mono_chunk<C + 1>(blk, row, qs, q, std::make_integer_sequence<int, 8>{}), ...);
 }
 template <int C, int... E>
 __device__ __forceinline__ void shifted_key_chunk(uint32_t blk, uint32_t row, const float (&s12)[6][6], const float (&k3)[6], std::integer_sequence<int, E...>) {
@@ -121,8 +123,9 @@ __device__ __forceinline__ void shifted_key_row(uint32_t blk, uint32_t row, floa
 }
 
 // In-place exclusive scan of the piece states of every head, in piece order (bit-reproducible); the sum of all pieces,
-// i.e. the state after the last token, goes to `state`.
-template <int F>
+// i.e. the state after the last token, goes to `state`.  REVERSE: the scan runs from the last piece to the first (every
+// piece gets the sum of the pieces after it).
+template <int F, bool REVERSE = false>
 __global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__ part, float* __restrict__ state, int S, int ld, int G, int T) {
     constexpr int kN = MT<F>::kN;
     const int bh = blockIdx.y;
@@ -141,21 +144,28 @@ __global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__
     for (int s0 = 0; s0 < count; s0 += 8) {      // eight independent loads in flight, then the scan in piece order
         float t[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) t[k] = s0 + k < count ? p[(size_t)(s0 + k) * n_per] : 0.f;
+        for (int k = 0; k < 8; ++k) t[k] = s0 + k < count ? p[(size_t)(REVERSE ? count - 1 - s0 - k : s0 + k) * n_per] : 0.f;
 #pragma unroll
         for (int k = 0; k < 8; ++k)
             if (s0 + k < count) {
-                p[(size_t)(s0 + k) * n_per] = run;
+                p[(size_t)(REVERSE ? count - 1 - s0 - k : s0 + k) * n_per] = run;
                 run += t[k];
             }
     }
     state[(size_t)bh * n_per + e] = run;
 }
 
-template <int DV>
+// MODE 0: the forward sweep described above.
+// MODE 1: the same sweep run backwards over the tokens with the two operand-row tiles exchanged, for the gradient of the
+// values: dV_j = sum_{i >= j} (Tsym_j . r_i mono_i) dO_i.  The "query" rows are the folded keys, the "key" rows are the
+// scaled monomials [-delta_i, 0 x 7, r_i mono_i] (delta_i = dO_i . o_i, so the carried state is [dCsym | dzsym]), the value
+// tile is dO, a CTA walks its piece from the last tile to the first (grid (S, heads) only), the mask keeps i >= j, and
+// the result leaves without a normaliser.
+template <int DV, int MODE>
 __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
                                                                           const float* __restrict__ qf, const float* __restrict__ kf,
-                                                                          const float* __restrict__ init, float* __restrict__ eta_out, int N, int BH,
+                                                                          const float* __restrict__ init, float* __restrict__ eta_out,
+                                                                          const float* __restrict__ eta_in, const float* __restrict__ delta, int N, int BH,
                                                                           int S, int ld, int G, float eps, int* status) {
     using Cfg = CaCfg<DV>;
     constexpr int kStageBytes = Cfg::kStageBytes;
@@ -182,6 +192,8 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
     const int T = (N + kTileTokens - 1) / kTileTokens;
     const CaWork cw = causal_work(T, BH, S, G);
     const int w0 = cw.w0, nwork = cw.w1 - cw.w0;
+    auto work_of = [&](int it) { return MODE == 0 ? w0 + it : w0 + nwork - 1 - it; };                 // (head, tile) of the CTA's it-th item
+    auto starts = [&](int it) { return it == 0 || (MODE == 0 && (w0 + it) % T == 0); };          // a piece begins with this item
     grid_launch_dependents();
 
     if (tid == 0) {
@@ -221,7 +233,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
     if (warp == 0) {
         if (lane == 0) {
             for (int it = 0; it < nwork; ++it) {
-                const int st = it & 1, u = it >> 1, work = w0 + it;
+                const int st = it & 1, u = it >> 1, work = work_of(it);
                 if (!mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { report_timeout(status, 901); break; }
                 mbar_arrive_expect_tx(&stage_ready[st], DV * kTileTokens * 2);
                 for (int b = 0; b < Cfg::kVB; ++b) tma_load_3d(smem + st * kStageBytes + b * kBlk, &mapV, &stage_ready[st], b * 64, (work % T) * kTileTokens, work / T);
@@ -274,7 +286,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                 // the state after the previous tile must have been read out of tensor memory; the first tile of a piece
                 // waits for the initial state
                 if (it > 0 && !mbar_wait_c(state_read, (it - 1) & 1)) { report_timeout(status, 911); break; }
-                if ((it == 0 || (w0 + it) % T == 0) && !mbar_wait_c(&b3_ready[it & 1], (it >> 1) & 1)) { report_timeout(status, 912); break; }
+                if (starts(it) && !mbar_wait_c(&b3_ready[it & 1], (it >> 1) & 1)) { report_timeout(status, 912); break; }
                 if (!mbar_wait_c(&stage_ready[st], u & 1)) { report_timeout(status, 904); break; }
                 tc_fence_after();
                 {      // state += Tsym^T * [V | 1]
@@ -286,57 +298,75 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                 umma_commit(&stage_free[st]);
             }
         }
-    } else if (warp < kCaGenKWarp0) {
-        // monomial rows of the queries: thread = token row of the tile
-        const int row = tid - kCaGenQWarp0 * 32;
-        float qn[6];
-        auto prefetch = [&](int it) {
-            const int work = w0 + it, bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
-            load_feat<6>(qn, qf + ((size_t)bh * N + tok) * 6);
-        };
-        if (nwork > 0) prefetch(0);
-        for (int it = 0; it < nwork; ++it) {
-            const int st = it & 1, u = it >> 1, work = w0 + it;
-            const bool valid = (work % T) * kTileTokens + row < N;
-            float q[6];
-#pragma unroll
-            for (int i = 0; i < 6; ++i) q[i] = valid ? qn[i] : 0.f;
-            if (ok && !mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 906); }
-            if (!ok) continue;
-            shifted_mono_row(smem_u32(smem + st * kStageBytes) + Cfg::kOffM, row, q, std::make_integer_sequence<int, 7>{});
-            fence_proxy_async();
-            mbar_arrive(&stage_ready[st]);
-            if (it + 1 < nwork) prefetch(it + 1);      // after the fence: a fence waits for the loads in flight
-        }
     } else if (warp < kCaMaskWarp0) {
-        // folded key rows
-        const int row = tid - kCaGenKWarp0 * 32;
-        float kn[18];
-        auto prefetch = [&](int it) {
-            const int work = w0 + it, bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
+        // operand rows: thread = token row of the tile.  Warps 2..5 write the tile the attention block and the readout take as
+        // their A operand (MODE 0: monomials of q; MODE 1: folded keys), warps 6..9 the tile that sits behind the value blocks
+        // (MODE 0: folded keys with the ones column; MODE 1: scaled monomials with -delta in that column).
+        const bool first_group = warp < kCaGenKWarp0;
+        const int row = (tid - kCaGenQWarp0 * 32) & 127;
+        const bool from_q = first_group == (MODE == 0);
+        const int dst_off = first_group ? Cfg::kOffM : Cfg::kOffT;
+        if (from_q) {
+            float qn[6], en = 0.f, dn = 0.f;
+            auto prefetch = [&](int it) {
+                const int work = work_of(it), bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
+                load_feat<6>(qn, qf + ((size_t)bh * N + tok) * 6);
+                if (MODE == 1) {
+                    en = __ldg(eta_in + (size_t)bh * N + tok);
+                    dn = __ldg(delta + (size_t)bh * N + tok);
+                }
+            };
+            if (nwork > 0) prefetch(0);
+            for (int it = 0; it < nwork; ++it) {
+                const int st = it & 1, u = it >> 1, work = work_of(it);
+                const bool valid = (work % T) * kTileTokens + row < N;
+                float q[6], qs[6], first = 0.f;
 #pragma unroll
-            for (int f = 0; f < 3; ++f) load_feat<6>(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
-        };
-        if (nwork > 0) prefetch(0);
-        for (int it = 0; it < nwork; ++it) {
-            const int st = it & 1, u = it >> 1, work = w0 + it;
-            const bool valid = (work % T) * kTileTokens + row < N;
-            float k[18];
+                for (int i = 0; i < 6; ++i) q[i] = valid ? qn[i] : 0.f;
+                if (MODE == 1) {
+                    const float r = valid ? 1.f / (en + eps) : 0.f;
 #pragma unroll
-            for (int i = 0; i < 18; ++i) k[i] = valid ? kn[i] : 0.f;
-            if (ok && !mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 910); }
-            if (!ok) continue;
-            float s12[6][6], k3[6];      // [x][y], x < y: k1[x] k2[y] + k1[y] k2[x];  [x][x]: k1[x] k2[x]
+                    for (int i = 0; i < 6; ++i) qs[i] = r * q[i];
+                    first = valid ? -dn : 0.f;
+                } else {
 #pragma unroll
-            for (int x = 0; x < 6; ++x) {
-                k3[x] = k[12 + x];
-#pragma unroll
-                for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k[x] * k[6 + x] : fmaf(k[x], k[6 + y], k[y] * k[6 + x]);
+                    for (int i = 0; i < 6; ++i) qs[i] = q[i];
+                }
+                if (ok && !mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 906); }
+                if (!ok) continue;
+                shifted_mono_row(smem_u32(smem + st * kStageBytes) + dst_off, row, first, qs, q, std::make_integer_sequence<int, 7>{});
+                fence_proxy_async();
+                mbar_arrive(&stage_ready[st]);
+                if (it + 1 < nwork) prefetch(it + 1);      // after the fence: a fence waits for the loads in flight
             }
-            shifted_key_row(smem_u32(smem + st * kStageBytes) + Cfg::kOffT, row, valid ? 1.f : 0.f, s12, k3, std::make_integer_sequence<int, 7>{});
-            fence_proxy_async();
-            mbar_arrive(&stage_ready[st]);
-            if (it + 1 < nwork) prefetch(it + 1);
+        } else {
+            float kn[18];
+            auto prefetch = [&](int it) {
+                const int work = work_of(it), bh = work / T, tok = min((work % T) * kTileTokens + row, N - 1);
+#pragma unroll
+                for (int f = 0; f < 3; ++f) load_feat<6>(kn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
+            };
+            if (nwork > 0) prefetch(0);
+            for (int it = 0; it < nwork; ++it) {
+                const int st = it & 1, u = it >> 1, work = work_of(it);
+                const bool valid = (work % T) * kTileTokens + row < N;
+                float k[18];
+#pragma unroll
+                for (int i = 0; i < 18; ++i) k[i] = valid ? kn[i] : 0.f;
+                if (ok && !mbar_wait_c(&stage_free[st], (u & 1) ^ 1)) { ok = false; report_timeout(status, 910); }
+                if (!ok) continue;
+                float s12[6][6], k3[6];      // [x][y], x < y: k1[x] k2[y] + k1[y] k2[x];  [x][x]: k1[x] k2[x]
+#pragma unroll
+                for (int x = 0; x < 6; ++x) {
+                    k3[x] = k[12 + x];
+#pragma unroll
+                    for (int y = x; y < 6; ++y) s12[x][y] = (x == y) ? k[x] * k[6 + x] : fmaf(k[x], k[6 + y], k[y] * k[6 + x]);
+                }
+                shifted_key_row(smem_u32(smem + st * kStageBytes) + dst_off, row, (MODE == 0 && valid) ? 1.f : 0.f, s12, k3, std::make_integer_sequence<int, 7>{});
+                fence_proxy_async();
+                mbar_arrive(&stage_ready[st]);
+                if (it + 1 < nwork) prefetch(it + 1);
+            }
         }
     } else if (warp < kCaConvWarp0) {
         // mask: thread = query row i of the block, two warps per 32 rows: warp (qt, half) owns the columns 64 half .. 64 half
@@ -353,18 +383,23 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             for (int bb = 0; bb < 2; ++bb) {      // sub-block column 2 half + bb against sub-block row qt
                 const int b = 2 * half + bb;
                 uint32_t w[16];
-                if (b <= qt) {
+                const bool whole = MODE == 0 ? b < qt : b > qt;      // sub-block entirely on the kept side of the diagonal
+                if (whole || b == qt) {
                     uint32_t r[32];
                     tmem_ld16(pa + 32 * bb, *reinterpret_cast<uint32_t(*)[16]>(r));
                     tmem_ld16(pa + 32 * bb + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
                     tmem_ld_wait();
-                    if (b < qt) {
+                    if (whole) {
 #pragma unroll
                         for (int e = 0; e < 16; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                    } else {
+                    } else if (MODE == 0) {
 #pragma unroll
                         for (int e = 0; e < 16; ++e)
                             w[e] = pack_bf16(2 * e <= lane ? __uint_as_float(r[2 * e]) : 0.f, 2 * e + 1 <= lane ? __uint_as_float(r[2 * e + 1]) : 0.f);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            w[e] = pack_bf16(2 * e >= lane ? __uint_as_float(r[2 * e]) : 0.f, 2 * e + 1 >= lane ? __uint_as_float(r[2 * e + 1]) : 0.f);
                     }
                 } else {
 #pragma unroll
@@ -390,8 +425,8 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                              pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
         };
         for (int it = 0; it < nwork; ++it) {
-            const int work = w0 + it, bh = work / T;
-            if (it == 0 || work % T == 0) {
+            const int work = work_of(it), bh = work / T;
+            if (starts(it)) {
                 // a piece begins: its initial state goes to tensor memory (fp32) and to the image (bf16)
                 const float* src = init + ((size_t)causal_slot(bh, T, BH, S, G) * kMono + (mine ? m : 0)) * ld;
 #pragma unroll 1
@@ -420,7 +455,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             if (ok && !mbar_wait_c(state_full, it & 1)) { ok = false; report_timeout(status, 908); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (it + 1 < nwork && (work + 1) % T != 0) {
+            if (it + 1 < nwork && !starts(it + 1)) {
                 // the image written now was last read by the readout of the previous tile (issued by the other thread)
                 if (it > 0 && ok && !mbar_wait_c(&rd_done[(it - 1) & 1], ((it - 1) >> 1) & 1)) { ok = false; report_timeout(status, 913); }
                 ok = __all_sync(0xffffffffu, ok);
@@ -466,7 +501,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
         const uint32_t aa = tmem + Cfg::kColAcc + ((uint32_t)(qt * 32) << 16);
         const uint32_t os = smem_u32(smem + Cfg::kOffO);
         for (int it = 0; it < nwork; ++it) {
-            const int work = w0 + it, bh = work / T, tile = work % T;
+            const int work = work_of(it), bh = work / T, tile = work % T;
             if (!mbar_wait_c(acc_full, it & 1)) {
                 report_timeout(status, 909);
                 *abort_flag = 1;
@@ -479,7 +514,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
             tmem_ld8(aa + DV, re);
             tmem_ld_wait();
             const float eta = __uint_as_float(re[0]);
-            const float rinv = 1.f / (eta + eps);
+            const float rinv = MODE == 0 ? 1.f / (eta + eps) : 1.f;
 #pragma unroll 1
             for (int h = 0; h < DV / 32; ++h) {
                 uint32_t r[32];
@@ -504,7 +539,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
                 tma_store_commit();
             }
             const int tok = tile * kTileTokens + row;
-            if (tok < N) eta_out[(size_t)bh * N + tok] = eta;
+            if (MODE == 0 && tok < N) eta_out[(size_t)bh * N + tok] = eta;
         }
         if (etid == 0) tma_store_wait_all0();
     }
@@ -524,14 +559,14 @@ inline hla_status launch_causal_sweep(const Dims& D, int BH, const float* qf, co
     float* part = reinterpret_cast<float*>(ws + off_part);
     float* state = reinterpret_cast<float*>(ws + L.state);
     float* eta = reinterpret_cast<float*>(ws + L.eta);
-    if (!set_smem(tc_causal_forward_kernel<DV>, CaCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_causal_forward_kernel<DV, 0>, CaCfg<DV>::kSmem)) return HLA_ERR_CUDA;
     const int T = (D.N + kTileTokens - 1) / kTileTokens;
     rec.begin("tc_scan_pieces");
     launch_pdl(tc_scan_pieces_kernel<3>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, state, S, D.ld, G, T);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_causal_forward");
-    launch_pdl(tc_causal_forward_kernel<DV>, G > 0 ? dim3(G) : dim3(S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapV, mapO, qf, kf, part, eta, D.N, BH, S,
-               D.ld, G, D.eps, status);
+    launch_pdl(tc_causal_forward_kernel<DV, 0>, G > 0 ? dim3(G) : dim3(S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapV, mapO, qf, kf,
+               (const float*)part, eta, (const float*)nullptr, (const float*)nullptr, D.N, BH, S, D.ld, G, D.eps, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
@@ -551,7 +586,7 @@ inline hla_status launch_causal_state_build(const Dims& D, int BH, const float* 
     if (!set_smem(tc_state_build_kernel<DV, 3>, SbCfg<3>::kSmem)) return HLA_ERR_CUDA;
     rec.begin("tc_state_build");
     launch_pdl(tc_state_build_kernel<DV, 3>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<3>::kSmem, rec.st, mapV, kf, reinterpret_cast<float*>(ws + off_part), D.N, D.S,
-               D.ld, reinterpret_cast<int*>(ws + L.status));
+               D.ld, reinterpret_cast<int*>(ws + L.status), (const float*)nullptr, (const float*)nullptr, 0.f);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
 
@@ -562,6 +597,71 @@ inline hla_status causal_forward(const Dims& D, int BH, const float* qf, const f
                                     : launch_causal_state_build<64>(D, BH, kf, V, ws, L, off_part, rec);
     if (s != HLA_OK) return s;
     return causal_sweep(D, BH, qf, kf, V, O, ws, L, off_part, D.S, 0, rec);
+}
+
+// delta_i = dO_i . o_i for every token row (bf16 rows of d values, fp32 sum): d / 8 lanes per row, 16 bytes per lane.
+template <int DV>
+__global__ void __launch_bounds__(256) tc_delta_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO, float* __restrict__ delta,
+                                                       long long rows) {
+    constexpr int LPR = DV / 8;                 // lanes per row
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const long long t = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long row = t / LPR;
+    const int part = (int)(t % LPR);
+    float a = 0.f;
+    if (row < rows) {
+        const uint4 x = *reinterpret_cast<const uint4*>(O + row * DV + 8 * part);
+        const uint4 y = *reinterpret_cast<const uint4*>(dO + row * DV + 8 * part);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            a = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), a);
+            a = fmaf(__uint_as_float(xs[e] & 0xffff0000u), __uint_as_float(ys[e] & 0xffff0000u), a);
+        }
+    }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (row < rows && part == 0) delta[row] = a;
+}
+
+// Backward of the causal operator at the feature level, part 1: delta, the gradient state of every piece, its suffix scan,
+// and the sweep that gives dV.
+template <int DV>
+inline hla_status launch_causal_backward_values(const Dims& D, int BH, const float* qf, const float* kf, const void* O, const void* dO, void* dV, char* ws,
+                                                const hla_ws_layout& L, size_t off_part, size_t off_delta, LaunchRec& rec) {
+    CUtensorMap mapdO, mapdV;
+    if (!make_map_bhnd(&mapdO, dO, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapdV, dV, BH, D.N, DV, kTileTokens)) return HLA_ERR_CUDA;
+    int* status = reinterpret_cast<int*>(ws + L.status);
+    float* part = reinterpret_cast<float*>(ws + off_part);
+    float* dstate = reinterpret_cast<float*>(ws + L.dstate);
+    float* eta = reinterpret_cast<float*>(ws + L.eta);
+    float* delta = reinterpret_cast<float*>(ws + off_delta);
+    if (!set_smem(tc_state_build_kernel<DV, 3, true>, SbCfg<3>::kSmem) || !set_smem(tc_causal_forward_kernel<DV, 1>, CaCfg<DV>::kSmem)) return HLA_ERR_CUDA;
+    const int T = (D.N + kTileTokens - 1) / kTileTokens;
+    const long long rows = (long long)BH * D.N;
+    rec.begin("tc_delta");
+    launch_pdl(tc_delta_kernel<DV>, dim3((unsigned)((rows * (DV / 8) + 255) / 256)), dim3(256), 0, rec.st, static_cast<const __nv_bfloat16*>(O),
+               static_cast<const __nv_bfloat16*>(dO), delta, rows);
+    if (!rec.end()) return HLA_ERR_CUDA;
+    rec.begin("tc_dstate_build");
+    launch_pdl(tc_state_build_kernel<DV, 3, true>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<3>::kSmem, rec.st, mapdO, qf, part, D.N, D.S, D.ld, status,
+               (const float*)eta, (const float*)delta, D.eps);
+    if (!rec.end()) return HLA_ERR_CUDA;
+    rec.begin("tc_scan_pieces");
+    launch_pdl(tc_scan_pieces_kernel<3, true>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, dstate, D.S, D.ld, 0, T);
+    if (!rec.end()) return HLA_ERR_CUDA;
+    rec.begin("tc_causal_dv");
+    launch_pdl(tc_causal_forward_kernel<DV, 1>, dim3(D.S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapdO, mapdV, qf, kf, (const float*)part,
+               (float*)nullptr, (const float*)eta, (const float*)delta, D.N, BH, D.S, D.ld, 0, D.eps, status);
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+
+inline hla_status causal_backward_values(const Dims& D, int BH, const float* qf, const float* kf, const void* O, const void* dO, void* dV, char* ws,
+                                         const hla_ws_layout& L, size_t off_part, size_t off_delta, LaunchRec& rec) {
+    if (D.F != 3) return HLA_ERR_UNSUPPORTED;
+    if (D.d == 128) return launch_causal_backward_values<128>(D, BH, qf, kf, O, dO, dV, ws, L, off_part, off_delta, rec);
+    return launch_causal_backward_values<64>(D, BH, qf, kf, O, dO, dV, ws, L, off_part, off_delta, rec);
 }
 
 }  // namespace tc
