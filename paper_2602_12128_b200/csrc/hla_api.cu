@@ -15,6 +15,7 @@
 #include "hla_tc_wgrad.cuh"
 #include "hla_tc_vmod.cuh"
 #include "hla_tc_causal.cuh"
+#include "hla_tc_causal_grad.cuh"
 
 using namespace hla;
 
@@ -412,9 +413,7 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
         float* dqf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dqf) : static_cast<float*>(dQ);
         float* dkf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dkf) : static_cast<float*>(dK);
         if (ctx->cfg.causal) {
-            s = tc::causal_backward_values(ctx->D, ctx->BH, qf, kf, O, dO, dV, ws, ctx->L, ctx->off_part, ctx->off_delta, ctx->rec);
-            if (s != HLA_OK) return s;
-            return HLA_ERR_UNSUPPORTED;      // (feature gradients: next)
+            s = tc::causal_backward(ctx->D, ctx->BH, qf, kf, V, O, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->off_delta, ctx->rec);
         } else {
             s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
         }

@@ -625,10 +625,19 @@ __global__ void __launch_bounds__(256) tc_delta_kernel(const __nv_bfloat16* __re
     if (row < rows && part == 0) delta[row] = a;
 }
 
-// Backward of the causal operator at the feature level, part 1: delta, the gradient state of every piece, its suffix scan,
-// and the sweep that gives dV.
 template <int DV>
-inline hla_status launch_causal_backward_values(const Dims& D, int BH, const float* qf, const float* kf, const void* O, const void* dO, void* dV, char* ws,
+inline hla_status launch_causal_delta(const Dims& D, int BH, const void* O, const void* dO, char* ws, size_t off_delta, LaunchRec& rec) {
+    const long long rows = (long long)BH * D.N;
+    rec.begin("tc_delta");
+    launch_pdl(tc_delta_kernel<DV>, dim3((unsigned)((rows * (DV / 8) + 255) / 256)), dim3(256), 0, rec.st, static_cast<const __nv_bfloat16*>(O),
+               static_cast<const __nv_bfloat16*>(dO), reinterpret_cast<float*>(ws + off_delta), rows);
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+
+// Backward of the causal operator at the feature level, value side: the gradient state of every piece, its suffix scan,
+// and the sweep that gives dV (delta must have been computed).
+template <int DV>
+inline hla_status launch_causal_backward_values(const Dims& D, int BH, const float* qf, const float* kf, const void* dO, void* dV, char* ws,
                                                 const hla_ws_layout& L, size_t off_part, size_t off_delta, LaunchRec& rec) {
     CUtensorMap mapdO, mapdV;
     if (!make_map_bhnd(&mapdO, dO, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapdV, dV, BH, D.N, DV, kTileTokens)) return HLA_ERR_CUDA;
@@ -639,11 +648,6 @@ inline hla_status launch_causal_backward_values(const Dims& D, int BH, const flo
     float* delta = reinterpret_cast<float*>(ws + off_delta);
     if (!set_smem(tc_state_build_kernel<DV, 3, true>, SbCfg<3>::kSmem) || !set_smem(tc_causal_forward_kernel<DV, 1>, CaCfg<DV>::kSmem)) return HLA_ERR_CUDA;
     const int T = (D.N + kTileTokens - 1) / kTileTokens;
-    const long long rows = (long long)BH * D.N;
-    rec.begin("tc_delta");
-    launch_pdl(tc_delta_kernel<DV>, dim3((unsigned)((rows * (DV / 8) + 255) / 256)), dim3(256), 0, rec.st, static_cast<const __nv_bfloat16*>(O),
-               static_cast<const __nv_bfloat16*>(dO), delta, rows);
-    if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_dstate_build");
     launch_pdl(tc_state_build_kernel<DV, 3, true>, dim3(D.S, BH), dim3(kSbThreads), SbCfg<3>::kSmem, rec.st, mapdO, qf, part, D.N, D.S, D.ld, status,
                (const float*)eta, (const float*)delta, D.eps);
@@ -655,13 +659,6 @@ inline hla_status launch_causal_backward_values(const Dims& D, int BH, const flo
     launch_pdl(tc_causal_forward_kernel<DV, 1>, dim3(D.S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapdO, mapdV, qf, kf, (const float*)part,
                (float*)nullptr, (const float*)eta, (const float*)delta, D.N, BH, D.S, D.ld, 0, D.eps, status);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
-}
-
-inline hla_status causal_backward_values(const Dims& D, int BH, const float* qf, const float* kf, const void* O, const void* dO, void* dV, char* ws,
-                                         const hla_ws_layout& L, size_t off_part, size_t off_delta, LaunchRec& rec) {
-    if (D.F != 3) return HLA_ERR_UNSUPPORTED;
-    if (D.d == 128) return launch_causal_backward_values<128>(D, BH, qf, kf, O, dO, dV, ws, L, off_part, off_delta, rec);
-    return launch_causal_backward_values<64>(D, BH, qf, kf, O, dO, dV, ws, L, off_part, off_delta, rec);
 }
 
 }  // namespace tc
