@@ -20,7 +20,7 @@
 // the two MMA-issuing threads and the barrier protocol are those of the forward sweep.
 //
 // Warp roles: 0 TMA (X and Y tiles), 1 MMA issue (Sc, readout, Sm * W), 26 MMA issue (state), 2..5 operand rows W,
-// 10..17 mask, 18..21 state image, 22..25 epilogue; warps 6..9 idle.
+// 10..17 mask, 18..21 state image, 22..25 and 6..9 epilogue (two groups, alternate tiles).
 #pragma once
 #include "hla_tc_causal.cuh"
 
@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
     uint64_t* p_full = bars + 4;          // MMA commit: Sc is complete
     uint64_t* pm_ready = bars + 5;        // 256 arrivals: Sm is in tensor memory
     uint64_t* state_full = bars + 7;      // MMA commit
-    uint64_t* acc_full = bars + 8;        // MMA commit
+    uint64_t* acc_full = bars + 19;       // [2] MMA commit, barrier it & 1 (each epilogue group waits on its own)
     uint64_t* state_read = bars + 9;      // 128 arrivals
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
     uint64_t* acc_free = bars + 17;       // [2] 128 arrivals, barrier it & 1: accumulator and state-column vector of tile it have been read
@@ -83,11 +83,11 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
             mbar_init(&stage_free[i], 2);
             mbar_init(&b3_ready[i], 128);
             mbar_init(&acc_free[i], 128);
+            mbar_init(&acc_full[i], 1);
         }
         mbar_init(p_full, 1);
         mbar_init(pm_ready, 256);
         mbar_init(state_full, 1);
-        mbar_init(acc_full, 1);
         mbar_init(state_read, 128);
         fence_mbar_init();
         prefetch_tmap(&mapX);
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
 #pragma unroll 1
                     for (int ks = 0; ks < kTileTokens / 16; ++ks, db += 128) umma_bf16_ta(tmem + Cfg::kColAcc, tmem + Cfg::kColS + 8 * ks + (ks >= 4 ? 32 : 0), db, id_w, 1u);
                 }
-                umma_commit(acc_full);
+                umma_commit(&acc_full[it & 1]);
                 umma_commit(&stage_free[st]);
             }
         }
@@ -234,9 +234,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
                 if (it + 1 < nwork) prefetch(it + 1);
             }
         }
-    } else if (warp < kCaMaskWarp0) {
-        // idle
-    } else if (warp < kCaConvWarp0) {
+    } else if (warp >= kCaMaskWarp0 && warp < kCaConvWarp0) {
         // mask: thread = row x of Sc (DIR 0: query token i; DIR 1: key token j), two warps per 32 rows, 64 columns each.
         // DIR 0 keeps the columns y <= x and subtracts the row's own delta; DIR 1 keeps y >= x and subtracts the delta of
         // the column's token.
@@ -292,7 +290,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
             tc_fence_before();
             mbar_arrive(pm_ready);
         }
-    } else if (warp < kCaEpiWarp0) {
+    } else if (warp >= kCaConvWarp0 && warp < kCaEpiWarp0) {
         // state image (rows as in the forward sweep) and, beside it, column d of the state in fp32
         const int qt = warp & 3, R = qt * 16 + lane, m = R - kCaRowPad;
         const bool active = lane < 16, mine = active && m >= 0 && m < kMono;
@@ -370,9 +368,11 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
                 mbar_arrive(state_read);
             }
         }
-    } else if (warp < kCaStateMmaWarp) {
-        // epilogue: thread = row x of the accumulator (DIR 0: query token, DIR 1: key token)
-        const int qt = warp & 3, row = qt * 32 + lane;
+    } else {
+        // epilogue: thread = row x of the accumulator (DIR 0: query token, DIR 1: key token).  Two groups (warps 22..25 and
+        // 6..9) take the tiles in turn: a group releases the accumulator as soon as it has read it and then has two tile
+        // times for the gradient arithmetic of its rows.
+        const int qt = warp & 3, row = qt * 32 + lane, grp = warp < kCaMaskWarp0 ? 1 : 0;
         const uint32_t aa = tmem + Cfg::kColAcc + ((uint32_t)(qt * 32) << 16);
         float fn[DIR == 0 ? 6 : 18], en = 0.f, dn = 0.f;
         auto prefetch = [&](int it) {
@@ -386,15 +386,15 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
                 for (int f = 0; f < 3; ++f) load_feat<6>(fn + 6 * f, kf + (((size_t)bh * 3 + f) * N + tok) * 6);
             }
         };
-        if (nwork > 0) prefetch(0);
-        for (int it = 0; it < nwork; ++it) {
+        if (nwork > grp) prefetch(grp);
+        for (int it = grp; it < nwork; it += 2) {
             const int tok = tile_of(it) * kTileTokens + row;
             float f[DIR == 0 ? 6 : 18];
 #pragma unroll
             for (int i = 0; i < (DIR == 0 ? 6 : 18); ++i) f[i] = fn[i];
             const float r = 1.f / (en + eps), dl = dn;
-            if (it + 1 < nwork) prefetch(it + 1);
-            if (ok && !mbar_wait_c(acc_full, it & 1)) { ok = false; report_timeout(status, 934); }
+            if (it + 2 < nwork) prefetch(it + 2);
+            if (ok && !mbar_wait_c(&acc_full[grp], (it >> 1) & 1)) { ok = false; report_timeout(status, 934); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();

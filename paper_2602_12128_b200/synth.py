@@ -53,7 +53,7 @@ CONFIGS["paper_r2_bf16"] = HlaShape("paper_r2_bf16", 1, 12, 12600, 128, "bf16", 
 CONFIGS["train_bf16_2f"] = HlaShape("train_bf16_2f", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=True, F=2, d_phi=12)
 
 # Causal HLA (Section 4.4: token i sees the tokens j <= i) at the training-step shape.
-CONFIGS["train_bf16_causal"] = HlaShape("train_bf16_causal", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=False, causal=True)
+CONFIGS["train_bf16_causal"] = HlaShape("train_bf16_causal", 2, 24, 32760, 128, "bf16", "inv_sqrt_d", backward=True, causal=True)
 
 
 def bf16_round(x: np.ndarray) -> np.ndarray:
