@@ -65,9 +65,16 @@ typedef enum {
  * Problem statement.  V, O, dO, dV (and Q, K, dQ, dK in HLA_PHI_MLP mode) are
  * [B,H,N,d] in `dtype`.  Features (HLA_PHI_NONE inputs and their gradients) are
  * always fp32.  Supported set: F in {1,2,3,4}, d_phi^F <= 256, d <= 128 and
- * d % 4 == 0, causal == 0.  dtype bf16 with d in {64,128}, (F, d_phi) = (3, 6) or
+ * d % 4 == 0.  dtype bf16 with d in {64,128}, (F, d_phi) = (3, 6) or
  * (2, 12) - the paper's two variants - and B*H*N < 2^31 runs on the tensor-core
  * kernels; everything else in the supported set runs on the fp32 SIMT kernels.
+ * causal = 1 (Section 4.4 "Causal Attention, Decay Factors and Sequential
+ * Updates": token i sees the tokens j <= i, itself included, and the normaliser
+ * sums the same entries, o_i = sum_{j<=i} A_ij v_j / (sum_{j<=i} A_ij + eps))
+ * is supported for the 3-factor tensor-core set only (bf16, d in {64,128},
+ * F = 3, d_phi = 6), forward and backward; any other combination with
+ * causal = 1 is HLA_ERR_UNSUPPORTED.  Decay factors (a non-binary mask) are
+ * not defined by the paper and not supported.
  */
 typedef struct {
     int32_t B, H, N, d;
@@ -77,7 +84,7 @@ typedef struct {
     int32_t dtype;    /* hla_dtype                                                             */
     float eps;        /* added to the normaliser, o = num / (eta + eps); <= 0 -> 1e-6          */
     int32_t n_splits; /* token splits of the state build per head; 0 -> chosen from the SM count */
-    int32_t causal;   /* must be 0: the causal / decayed variant (Section 4.4) is not built    */
+    int32_t causal;   /* 0: every token sees every token; 1: token i sees tokens j <= i          */
     int32_t value_mod; /* 1: the workspace also holds the scratch of hla_value_mod_forward / _backward (bf16 with
                           d in {64,128} only; HLA_ERR_UNSUPPORTED otherwise); 0: those calls are refused            */
 } hla_config;
@@ -148,7 +155,9 @@ hla_status hla_workspace_layout(const hla_ctx *ctx, hla_ws_layout *out);
 
 /*
  * Forward: O = HLA(Q, K, V).  Leaves the features, the state (C, z) and eta in
- * the workspace for a later hla_backward.  The workspace must be 256-byte
+ * the workspace for a later hla_backward.  With causal = 1 the state left in the
+ * workspace is the one after the last token (Eq. "seq.updates": C^N) and eta_i
+ * is the masked row sum.  The workspace must be 256-byte
  * aligned and at least hla_workspace_bytes() long.
  */
 hla_status hla_forward(hla_ctx *ctx, const void *Q, const void *K, const void *V, void *O,
@@ -162,6 +171,9 @@ hla_status hla_forward(hla_ctx *ctx, const void *Q, const void *K, const void *V
  * (their rows leave the kernel as 32-byte stores); anything else is refused with
  * HLA_ERR_INVALID_ARG before a launch.
  * Gradients with respect to the phi weights are not computed by this call.
+ * With causal = 1, O must be the output of that forward (the call reads it for
+ * dO_i . o_i; without the mask it is not read) and V, O, dO, dV must be 16-byte
+ * aligned like every tensor.
  */
 hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *V, const void *O,
                         const void *dO, void *dQ, void *dK, void *dV,
