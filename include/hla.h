@@ -164,6 +164,17 @@ hla_status hla_forward(hla_ctx *ctx, const void *Q, const void *K, const void *V
                        void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Sequential updates (Section 4.4, Eq. "seq.updates": C^i = C^{i-1} + T_{k_i} (x) v_i; the context tensor is the state of
+ * the sequence).  Contexts created with causal = 1 only.  With carry = 1 every following hla_forward on a workspace
+ * starts from the state (C, z) that the previous hla_forward left in that workspace instead of from zero, and leaves
+ * the updated state there: a sequence handed over in chunks of N tokens per call gives the outputs of one causal pass
+ * over the concatenation (the state is carried in fp32).  The first chunk of a sequence is run with carry = 0 (or on a
+ * workspace whose state region the caller has zeroed; hla_workspace_layout gives its offset and size).  hla_backward is
+ * HLA_ERR_UNSUPPORTED while carry = 1.  HLA_ERR_INVALID_ARG for a context without the mask or a value other than 0, 1.
+ */
+hla_status hla_set_carry(hla_ctx *ctx, int carry);
+
+/*
  * Backward of the forward that last wrote `workspace` (same Q, K, V, O; the
  * workspace untouched in between): dQ, dK, dV = d sum(dO * O) / d(Q, K, V).
  * In HLA_PHI_NONE mode dQ, dK are fp32 feature gradients with the shapes of Q, K.

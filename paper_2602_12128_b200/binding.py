@@ -17,7 +17,7 @@ HLA_BF16, HLA_F32 = 0, 1
 HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
-    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_backward_weights", "hla_set_phi_v", "hla_value_mod_forward", "hla_value_mod_backward", "hla_forward_static",
+    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_backward_weights", "hla_set_phi_v", "hla_set_carry", "hla_value_mod_forward", "hla_value_mod_backward", "hla_forward_static",
     "hla_last_device_status", "hla_selftest_bounded_wait", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
     "hla_destroy", "hla_status_string",
 ]
@@ -82,6 +82,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_backward.restype = c_int32
     lib.hla_backward_weights.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(HlaMlpGrad), POINTER(HlaMlpGrad), c_void_p, c_size_t, c_void_p]
     lib.hla_backward_weights.restype = c_int32
+    lib.hla_set_carry.argtypes = [c_void_p, c_int32]
+    lib.hla_set_carry.restype = c_int32
     lib.hla_set_phi_v.argtypes = [c_void_p, POINTER(HlaVmlp), POINTER(HlaVmlp)]
     lib.hla_set_phi_v.restype = c_int32
     lib.hla_value_mod_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
@@ -183,6 +185,12 @@ def hla_backward_weights(ctx: int, Q, K, dphi_q, dphi_k, workspace, stream=None,
     st = load_library().hla_backward_weights(ctx, _ptr(Q), _ptr(K), q, ks, _ptr(workspace), nbytes, _stream(stream))
     if st != HLA_OK:
         raise HlaError(st, "hla_backward_weights")
+
+
+def hla_set_carry(ctx: int, carry: bool) -> None:
+    st = load_library().hla_set_carry(ctx, 1 if carry else 0)
+    if st != HLA_OK:
+        raise HlaError(st, "hla_set_carry")
 
 
 def hla_set_phi_v(ctx: int, v1, v2) -> None:
@@ -292,6 +300,9 @@ class Hla:
         dV = torch.empty_like(V) if dV is None else dV
         hla_backward(self.ctx, Q, K, V, O, dO, dQ, dK, dV, self.workspace, stream)
         return dQ, dK, dV
+
+    def set_carry(self, carry: bool):
+        hla_set_carry(self.ctx, carry)
 
     def set_phi_v(self, v1, v2):
         self._vweights = (v1, v2)           # keep the tensors alive: the library only borrows pointers

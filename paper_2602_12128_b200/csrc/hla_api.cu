@@ -34,6 +34,7 @@ struct hla_ctx {
     hla_vmlp phi_v[2];
     tc::VmodPlan vmp;   // scratch of the value modulation inside the workspace
     size_t off_delta;   // dO . o per token (scratch of the causal backward)
+    bool carry;         // causal forward starts from the state the previous call left in the workspace
     size_t off_wpart;   // per-CTA partials of the weight gradients (scratch; tensor-core path with the phi maps)
     tc::Plan tcp;       // tensor-core operand buffers inside the workspace
     size_t ws_bytes;
@@ -319,6 +320,7 @@ hla_status hla_create(const hla_config* cfg, hla_ctx** out) {
     x->off_wpart = (x->tc && mlp) ? cv.take(tc::wgrad_part_bytes(c.d, (long long)x->BH * c.N, x->sm_count)) : kNone;
     if (x->tc) cv.off = tc::plan(x->tcp, D, x->BH, cv.off);
     x->off_delta = c.causal ? cv.take(tok * 4) : kNone;      // dO . o per token (causal backward)
+    x->carry = false;
     x->vmod = c.value_mod != 0;
     x->phi_v_set = false;
     if (x->vmod) cv.off = tc::vmod_plan(x->vmp, c.d, (long long)x->BH * c.N, cv.off);
@@ -342,6 +344,13 @@ hla_status hla_set_phi(hla_ctx* ctx, const hla_mlp* phi_q, const hla_mlp* phi_k)
     ctx->phi_q = *phi_q;
     for (int f = 0; f < ctx->D.F; ++f) ctx->phi_k[f] = phi_k[f];
     ctx->phi_set = true;
+    return HLA_OK;
+}
+
+hla_status hla_set_carry(hla_ctx* ctx, int carry) {
+    if (!ctx || (carry != 0 && carry != 1)) return HLA_ERR_INVALID_ARG;
+    if (!ctx->cfg.causal) return HLA_ERR_INVALID_ARG;
+    ctx->carry = carry != 0;
     return HLA_OK;
 }
 
@@ -373,19 +382,19 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
             s = tc::phik_state(ctx->D, ctx->BH, ctx->phi_k, K, V, ws, ctx->L, ctx->off_part, ctx->k_pieces, ctx->sm_count, ctx->rec);
             if (s != HLA_OK) return s;
             s = tc::reduce_pieces(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, ctx->off_part, ctx->k_pieces,
-                                  tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec);
+                                  tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec, ctx->cfg.causal != 0);
             if (s != HLA_OK) return s;
             s = tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
             if (s != HLA_OK || !ctx->cfg.causal) return s;
             // causal: the pass above left the features of both sides in the workspace (its O is overwritten now); the
             // pieces of the key-side kernel become the pieces of the sweep
             return tc::causal_sweep(ctx->D, ctx->BH, reinterpret_cast<const float*>(ws + ctx->L.qf), reinterpret_cast<const float*>(ws + ctx->L.kf), V, O,
-                                    ws, ctx->L, ctx->off_part, ctx->k_pieces, tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec);
+                                    ws, ctx->L, ctx->off_part, ctx->k_pieces, tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->carry, ctx->rec);
         } else {
             qf = static_cast<const float*>(Q);
             kf = static_cast<const float*>(K);
         }
-        if (ctx->cfg.causal) return tc::causal_forward(ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->rec);
+        if (ctx->cfg.causal) return tc::causal_forward(ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->carry, ctx->rec);
         return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
     }
     if (ctx->cfg.dtype == HLA_F32) return forward_simt<float>(ctx, Q, K, V, O, ws, st);
@@ -413,6 +422,7 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
         float* dqf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dqf) : static_cast<float*>(dQ);
         float* dkf = mlp ? reinterpret_cast<float*>(ws + ctx->L.dkf) : static_cast<float*>(dK);
         if (ctx->cfg.causal) {
+            if (ctx->carry) return HLA_ERR_UNSUPPORTED;      // a chunk that started from a carried state has no backward here
             s = tc::causal_backward(ctx->D, ctx->BH, qf, kf, V, O, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->off_delta, ctx->rec);
         } else {
             s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);

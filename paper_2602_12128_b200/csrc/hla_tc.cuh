@@ -1431,20 +1431,25 @@ inline hla_status launch_core_forward(const Plan& P, const Dims& D, int BH, cons
 }
 
 // Reduction of the pieces the fused key-side kernel (G CTAs over heads x T tiles, at most `smax` pieces per head) left.
+// scratch_state: the fp32 sum goes to the gradient-state region instead of the state region (the causal forward keeps
+// the state region for the state it carries from call to call).
 template <int F>
-inline hla_status reduce_pieces_f(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec) {
+inline hla_status reduce_pieces_f(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec,
+                                  bool scratch_state) {
     __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
     __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
     float* part = reinterpret_cast<float*>(ws + off_part);
-    float* state = reinterpret_cast<float*>(ws + L.state);
+    float* state = reinterpret_cast<float*>(ws + (scratch_state ? L.dstate : L.state));
     const int T = (D.N + kTileTokens - 1) / kTileTokens;
     rec.begin("tc_reduce_emit");
     if (D.d == 128) launch_pdl(tc_reduce_emit_kernel<128, F>, dim3(MT<F>::kPad / 8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
     else launch_pdl(tc_reduce_emit_kernel<64, F>, dim3(MT<F>::kPad / 8, BH), dim3(256), 0, rec.st, part, state, b3, bq, smax, D.ld, G, T);
     return rec.end() ? HLA_OK : HLA_ERR_CUDA;
 }
-inline hla_status reduce_pieces(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec) {
-    return D.F == 3 ? reduce_pieces_f<3>(P, D, BH, ws, L, off_part, smax, G, rec) : reduce_pieces_f<2>(P, D, BH, ws, L, off_part, smax, G, rec);
+inline hla_status reduce_pieces(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, size_t off_part, int smax, int G, LaunchRec& rec,
+                                bool scratch_state = false) {
+    return D.F == 3 ? reduce_pieces_f<3>(P, D, BH, ws, L, off_part, smax, G, rec, scratch_state)
+                    : reduce_pieces_f<2>(P, D, BH, ws, L, off_part, smax, G, rec, scratch_state);
 }
 
 // readout = false stops after the state has been built and reduced (the fused query-side kernel reads it out).

@@ -124,9 +124,10 @@ __device__ __forceinline__ void shifted_key_row(uint32_t blk, uint32_t row, floa
 
 // In-place exclusive scan of the piece states of every head, in piece order (bit-reproducible); the sum of all pieces,
 // i.e. the state after the last token, goes to `state`.  REVERSE: the scan runs from the last piece to the first (every
-// piece gets the sum of the pieces after it).
+// piece gets the sum of the pieces after it).  carry != 0: the scan starts from what `state` holds (the state an earlier
+// call left there: Eq. "seq.updates" continued across calls) instead of zero.
 template <int F, bool REVERSE = false>
-__global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__ part, float* __restrict__ state, int S, int ld, int G, int T) {
+__global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__ part, float* __restrict__ state, int S, int ld, int G, int T, int carry) {
     constexpr int kN = MT<F>::kN;
     const int bh = blockIdx.y;
     grid_launch_dependents();
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(256) tc_scan_pieces_kernel(float* __restrict__
     const size_t e = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (e >= n_per) return;
     float* p = part + (size_t)bh * S * n_per + e;
-    float run = 0.f;
+    float run = carry ? state[(size_t)bh * n_per + e] : 0.f;
     for (int s0 = 0; s0 < count; s0 += 8) {      // eight independent loads in flight, then the scan in piece order
         float t[8];
 #pragma unroll
@@ -552,7 +553,7 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_forward_kernel(const 
 // G == 0: S pieces per head from a (S, heads) grid; G > 0: the pieces of a persistent kernel of G CTAs (at most S per head).
 template <int DV>
 inline hla_status launch_causal_sweep(const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws, const hla_ws_layout& L,
-                                      size_t off_part, int S, int G, LaunchRec& rec) {
+                                      size_t off_part, int S, int G, bool carry, LaunchRec& rec) {
     CUtensorMap mapV, mapO;
     if (!make_map_bhnd(&mapV, V, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens)) return HLA_ERR_CUDA;
     int* status = reinterpret_cast<int*>(ws + L.status);
@@ -562,7 +563,7 @@ inline hla_status launch_causal_sweep(const Dims& D, int BH, const float* qf, co
     if (!set_smem(tc_causal_forward_kernel<DV, 0>, CaCfg<DV>::kSmem)) return HLA_ERR_CUDA;
     const int T = (D.N + kTileTokens - 1) / kTileTokens;
     rec.begin("tc_scan_pieces");
-    launch_pdl(tc_scan_pieces_kernel<3>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, state, S, D.ld, G, T);
+    launch_pdl(tc_scan_pieces_kernel<3>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, state, S, D.ld, G, T, carry ? 1 : 0);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_causal_forward");
     launch_pdl(tc_causal_forward_kernel<DV, 0>, G > 0 ? dim3(G) : dim3(S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapV, mapO, qf, kf,
@@ -571,10 +572,10 @@ inline hla_status launch_causal_sweep(const Dims& D, int BH, const float* qf, co
 }
 
 inline hla_status causal_sweep(const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws, const hla_ws_layout& L,
-                               size_t off_part, int S, int G, LaunchRec& rec) {
+                               size_t off_part, int S, int G, bool carry, LaunchRec& rec) {
     if (D.F != 3) return HLA_ERR_UNSUPPORTED;
-    if (D.d == 128) return launch_causal_sweep<128>(D, BH, qf, kf, V, O, ws, L, off_part, S, G, rec);
-    return launch_causal_sweep<64>(D, BH, qf, kf, V, O, ws, L, off_part, S, G, rec);
+    if (D.d == 128) return launch_causal_sweep<128>(D, BH, qf, kf, V, O, ws, L, off_part, S, G, carry, rec);
+    return launch_causal_sweep<64>(D, BH, qf, kf, V, O, ws, L, off_part, S, G, carry, rec);
 }
 
 // Feature-level causal forward: state of every piece (the non-causal state build, one piece per split) -> scan -> sweep.
@@ -591,12 +592,12 @@ inline hla_status launch_causal_state_build(const Dims& D, int BH, const float* 
 }
 
 inline hla_status causal_forward(const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws, const hla_ws_layout& L,
-                                 size_t off_part, LaunchRec& rec) {
+                                 size_t off_part, bool carry, LaunchRec& rec) {
     if (D.F != 3) return HLA_ERR_UNSUPPORTED;
     const hla_status s = D.d == 128 ? launch_causal_state_build<128>(D, BH, kf, V, ws, L, off_part, rec)
                                     : launch_causal_state_build<64>(D, BH, kf, V, ws, L, off_part, rec);
     if (s != HLA_OK) return s;
-    return causal_sweep(D, BH, qf, kf, V, O, ws, L, off_part, D.S, 0, rec);
+    return causal_sweep(D, BH, qf, kf, V, O, ws, L, off_part, D.S, 0, carry, rec);
 }
 
 // delta_i = dO_i . o_i for every token row (bf16 rows of d values, fp32 sum): d / 8 lanes per row, 16 bytes per lane.
@@ -653,7 +654,7 @@ inline hla_status launch_causal_backward_values(const Dims& D, int BH, const flo
                (const float*)eta, (const float*)delta, D.eps);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_scan_pieces");
-    launch_pdl(tc_scan_pieces_kernel<3, true>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, dstate, D.S, D.ld, 0, T);
+    launch_pdl(tc_scan_pieces_kernel<3, true>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, dstate, D.S, D.ld, 0, T, 0);
     if (!rec.end()) return HLA_ERR_CUDA;
     rec.begin("tc_causal_dv");
     launch_pdl(tc_causal_forward_kernel<DV, 1>, dim3(D.S, BH), dim3(kCaThreads), CaCfg<DV>::kSmem, rec.st, mapdO, mapdV, qf, kf, (const float*)part,

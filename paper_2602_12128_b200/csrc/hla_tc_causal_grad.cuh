@@ -456,7 +456,7 @@ inline hla_status launch_causal_backward_features(const Dims& D, int BH, const f
                    (const float*)nullptr, (const float*)nullptr, 0.f);
         if (!rec.end()) return HLA_ERR_CUDA;
         rec.begin("tc_scan_pieces");
-        launch_pdl(tc_scan_pieces_kernel<3>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, state, D.S, D.ld, 0, T);
+        launch_pdl(tc_scan_pieces_kernel<3>, dim3((kMono * D.ld + 255) / 256, BH), dim3(256), 0, rec.st, part, state, D.S, D.ld, 0, T, 0);
         if (!rec.end()) return HLA_ERR_CUDA;
         rec.begin("tc_causal_dq");
         launch_pdl(tc_causal_grad_kernel<DV, 0>, dim3(D.S, BH), dim3(kCaThreads), CgCfg<DV>::kSmem, rec.st, mapdO, mapV, qf, kf, eta, delta, (const float*)part, dqf,

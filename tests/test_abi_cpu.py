@@ -132,3 +132,19 @@ def test_calls_validate_before_launching():
     binding.hla_destroy(ctx)
     assert binding.status_string(binding.HLA_ERR_DEVICE_TIMEOUT) == "device-side wait timed out"
     assert binding.hla_workspace_bytes(None) == 0
+
+
+def test_set_carry_validation():
+    """Sequential updates across calls exist for contexts with the mask only; the flag is 0 or 1."""
+    lib = binding.load_library()
+    st, ctx = create(causal=1)
+    assert st == binding.HLA_OK
+    assert lib.hla_set_carry(ctx, 1) == binding.HLA_OK
+    assert lib.hla_set_carry(ctx, 0) == binding.HLA_OK
+    assert lib.hla_set_carry(ctx, 2) == binding.HLA_ERR_INVALID_ARG
+    assert lib.hla_set_carry(None, 1) == binding.HLA_ERR_INVALID_ARG
+    binding.hla_destroy(ctx)
+    st, ctx = create()
+    assert st == binding.HLA_OK
+    assert lib.hla_set_carry(ctx, 1) == binding.HLA_ERR_INVALID_ARG
+    binding.hla_destroy(ctx)

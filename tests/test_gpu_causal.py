@@ -215,3 +215,57 @@ def test_causal_backward_full_size_sampled():
     gq, _, _ = orc.hla_quadratic_causal_backward(f64(qf[0, h, :300]), [k[:300] for k in ks_all], f64(V[0, h, :300]), f64(dO[0, h, :300]), 1e-12)
     assert relerr(dq[0, h, :300], gq) < TOL["bf16"]
     report("causal backward full size", dq_head=relerr(dq[0, h, :300], gq), dv_sum=np.abs(dv.sum(axis=2) - f64(dO).sum(axis=2)).max() / scale)
+
+
+@pytest.mark.parametrize("d,N,chunks,splits", [(128, 700, 3, 0), (64, 1000, 2, 3), (128, 128, 4, 1)])
+def test_sequential_updates_across_calls(d, N, chunks, splits):
+    """Eq. "seq.updates" across calls: a sequence handed over in chunks of N tokens, each call starting from the state the
+    previous one left in the workspace, gives the outputs of one causal pass over the concatenation; the state left after
+    the last chunk is the state of the whole sequence; a backward on a carried chunk is refused."""
+    s = synth.HlaShape("t", 1, 2, N * chunks, d, "bf16", "inv_sqrt_d")
+    _, _, V = synth.make_qkv(s)
+    V = synth.bf16_round(V * np.float32(np.sqrt(d)))
+    qf, kf = synth.make_features(s)
+    Oq, eta = orc.hla_core_forward(f64(qf), f64(kf), f64(V), EPS, "causal_streaming")
+    sc = synth.HlaShape("t", 1, 2, N, d, "bf16", "inv_sqrt_d")
+    run = DeviceRun(sc, "none", EPS, splits, causal=True)
+    outs, etas = [], []
+    for c in range(chunks):
+        run.op.set_carry(c > 0)
+        sl = slice(c * N, (c + 1) * N)
+        outs.append(run.forward(np.ascontiguousarray(qf[:, :, sl]), np.ascontiguousarray(kf[:, :, :, sl]), np.ascontiguousarray(V[:, :, sl])))
+        etas.append(run.eta())
+    O = np.concatenate(outs, axis=2)
+    assert relerr(O, Oq) < TOL["bf16"], relerr(O, Oq)
+    assert relerr(np.concatenate(etas, axis=2), eta) < TOL["bf16"] / 4
+    C, z = run.state()
+    Co, zo = oracle_state(f64(kf), f64(V))
+    Co, zo = fold_symmetric(Co), fold_symmetric(zo[..., None])[..., 0]
+    assert relerr(z, zo) < 1e-5 and relerr(C, Co) < TOL["bf16"] / 4
+    with pytest.raises(binding.HlaError) as e:
+        run.backward(synth.make_dO(sc))
+    assert e.value.status == binding.HLA_ERR_UNSUPPORTED
+    report("sequential updates across calls", d=d, N=N, chunks=chunks, maxnorm=relerr(O, Oq))
+
+
+def test_sequential_updates_with_phi_maps():
+    """The same with the phi maps in front (the pieces of the fused key-side kernel are scanned from the carried state)."""
+    d, N, chunks = 128, 900, 3
+    s = synth.HlaShape("t", 1, 2, N * chunks, d, "bf16", "inv_sqrt_d")
+    Q, K, V = synth.make_qkv(s)
+    pq, pk = synth.make_phi_weights(d, 6, 3, "bf16")
+    sc = synth.HlaShape("t", 1, 2, N, d, "bf16", "inv_sqrt_d")
+    run = DeviceRun(sc, "mlp", EPS, causal=True)
+    run.set_weights(pq, pk)
+    outs, gqs, gks = [], [], []
+    for c in range(chunks):
+        run.op.set_carry(c > 0)
+        sl = slice(c * N, (c + 1) * N)
+        outs.append(run.forward(np.ascontiguousarray(Q[:, :, sl]), np.ascontiguousarray(K[:, :, sl]), np.ascontiguousarray(V[:, :, sl])))
+        gq, gk = run.features()
+        gqs.append(gq)
+        gks.append(gk)
+    O = np.concatenate(outs, axis=2)
+    gq, gk = np.concatenate(gqs, axis=2), np.concatenate(gks, axis=3)
+    Oc, _ = orc.hla_core_forward(gq, gk, f64(V), EPS, "causal_streaming")      # the core on the features the GPU produced
+    assert relerr(O, Oc) < TOL["bf16"], relerr(O, Oc)
