@@ -130,10 +130,14 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
                 const uint32_t ya = smem_u32(smem + st * kStageBytes), wa = ya + Cfg::kOffW, xa = ya + Cfg::kOffX;
                 if (!mbar_wait_c(&stage_ready[st], u & 1)) { report_timeout(status, 922); break; }
                 tc_fence_after();
+                {      // Sc = X Y^T: four K steps per 64-column block, 32 bytes apart inside a 128-byte row
+                    uint64_t da = smem_desc_sw128(xa, 16, 1024), db = smem_desc_sw128(ya, 16, 1024);
+                    uint32_t acc = 0u;
 #pragma unroll 1
-                for (int ks = 0; ks < DV / 16; ++ks)      // Sc = X Y^T
-                    umma_bf16(tmem + Cfg::kColS, smem_desc_sw128(xa + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(ya + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024), id_s, ks > 0 ? 1u : 0u);
+                    for (int blk = 0; blk < Cfg::kVB; ++blk, da += (kBlk >> 4) - 8, db += (kBlk >> 4) - 8)
+#pragma unroll 1
+                        for (int k = 0; k < 4; ++k, da += 2, db += 2, acc = 1u) umma_bf16(tmem + Cfg::kColS, da, db, id_s, acc);
+                }
                 umma_commit(p_full);
                 if (!(mbar_wait_c(&b3_ready[it & 1], (it >> 1) & 1) && (it == 0 || mbar_wait_c(&acc_free[(it - 1) & 1], ((it - 1) >> 1) & 1)))) {
                     report_timeout(status, 923);
@@ -141,10 +145,14 @@ __global__ void __launch_bounds__(kCaThreads, 1) tc_causal_grad_kernel(const __g
                 }
                 tc_fence_after();
                 const uint32_t b3a = b3base + (it & 1) * Cfg::kB3Bytes;
+                {      // acc = X * image^T: one column per state row, value channels as K
+                    uint64_t da = smem_desc_sw128(xa, 16, 1024), db = smem_desc_sw128(b3a, 16, 1024);
+                    uint32_t acc = 0u;
 #pragma unroll 1
-                for (int ks = 0; ks < DV / 16; ++ks)      // acc = X * image^T: one column per state row, value channels as K
-                    umma_bf16(tmem + Cfg::kColAcc, smem_desc_sw128(xa + (ks >> 2) * kBlk + (ks & 3) * 32, 16, 1024),
-                              smem_desc_sw128(b3a + (ks >> 2) * Cfg::kB3Block + (ks & 3) * 32, 16, 1024), id_r, ks > 0 ? 1u : 0u);
+                    for (int blk = 0; blk < Cfg::kVB; ++blk, da += (kBlk >> 4) - 8, db += (Cfg::kB3Block >> 4) - 8)
+#pragma unroll 1
+                        for (int k = 0; k < 4; ++k, da += 2, db += 2, acc = 1u) umma_bf16(tmem + Cfg::kColAcc, da, db, id_r, acc);
+                }
                 if (!mbar_wait_c(pm_ready, it & 1)) { report_timeout(status, 925); break; }
                 tc_fence_after();
                 {      // acc += Sm * W; the two packed halves of Sm sit at columns 0..31 and 64..95 of the block
