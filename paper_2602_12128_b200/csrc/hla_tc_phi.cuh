@@ -75,9 +75,12 @@ struct PhiBwdPtrs {
     const __nv_bfloat16* W2[3];
 };
 
-// warp 0: TMA loads, warp 1: dg and dX MMAs, warp 2: h MMAs, warps 3..18: epilogue (thread = token row x quarter of the columns)
-constexpr int kPbThreads = 608;
-constexpr int kPbEpiWarp0 = 3;
+// warp 0: TMA loads, warp 1: dg and dX MMAs, warp 2: h MMAs, warps 3..18: epilogue (thread = token row x quarter of the columns),
+// warps 19..22: dp tiles (thread = token row).  The dp tiles were written by the epilogue threads at first; per unit that
+// cost each of the sixteen epilogue warps, whose instruction stream is what bounds the kernel, 600 of its 2850 cycles
+// (two loads, the split into two bf16 halves, two 4-byte stores, and above all one proxy fence per thread).
+constexpr int kPbThreads = 736;
+constexpr int kPbEpiWarp0 = 3, kPbDpWarp0 = 19;
 
 // DP = d_phi: 6 (F = 3) or 12 (F = 2).  The dp tile of a unit is [dp_hi | dp_lo] = 2 DP K columns: one K = 16 step for DP = 6 (two
 // tiles share one swizzled block at K columns 0..15 and 16..31), two steps for DP = 12 (one block per tile, K columns 0..23).
@@ -134,7 +137,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* h_full = bars + 4;       // [2] MMA commit
     uint64_t* dh_full = bars + 8;      // [2] 512 arrivals
     uint64_t* dh_free = bars + 10;     // [2] MMA commit
-    uint64_t* dp_full = bars + 12;     // [2] 512 arrivals
+    uint64_t* dp_full = bars + 12;     // [2] 128 arrivals
+    uint64_t* dp_free = bars + 28;     // [2] MMA commit: the dg product that read the slot has completed
     uint64_t* dg_full = bars + 20;     // MMA commit
     uint64_t* dg_empty = bars + 21;    // 512 arrivals
     uint64_t* dx_full = bars + 22;     // MMA commit
@@ -171,7 +175,10 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             mbar_init(&dh_full[i], 512);
             mbar_init(&dh_free[i], 1);
         }
-        for (int i = 0; i < 2; ++i) mbar_init(&dp_full[i], 512);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&dp_full[i], 128);
+            mbar_init(&dp_free[i], 1);
+        }
         mbar_init(dg_full, 1);
         mbar_init(dg_empty, 512);
         mbar_init(dx_full, 1);
@@ -252,6 +259,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                     umma_bf16(tmem + 256, desc_advance(pd0, (DP == 6 ? slot * 32 : slot * kBlk) + ks * 32), desc_advance(vd0, m * Cfg::kW2tBytes + ks * 2048), idesc_dg,
                               ks > 0 ? 1u : 0u);
                 umma_commit(dg_full);
+                umma_commit(&dp_free[slot]);
                 return true;
             };
             if (good && nunits > 0) good = issue_dg(0);
@@ -272,6 +280,52 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 if (m == NMAPS - 1) umma_commit(dx_full);
             }
             if (!good) report_timeout(status, 603);
+        }
+    } else if (warp >= kPbDpWarp0) {
+        // dp = dfeat (.) 1[feat > 0] of one token row as the A operand [dp_hi | dp_lo] of the dg product: the two bf16 halves
+        // of every value, so that dg is exact to ~2^-17.  DP = 6: the two slots share one block (K columns 16 slot ..);
+        // DP = 12: one block per slot.  The producer runs up to two units ahead of the dg products.
+        const int row = tid - kPbDpWarp0 * 32;
+        const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
+        for (int unit = 0; unit < nunits; ++unit) {
+            const int it = unit / NMAPS, m = unit % NMAPS, slot = unit & 1;
+            long long grow = (t0 + it) * kTileTokens + row;
+            const bool live = grow < rows;
+            grow = live ? grow : rows - 1;
+            size_t off;
+            if (KSIDE) {
+                const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
+                off = (((size_t)bh * NMAPS + m) * N + n) * DP;
+            } else {
+                off = (size_t)grow * DP;
+            }
+            float d[DP];
+#pragma unroll
+            for (int i = 0; i < DP / 2; ++i) {
+                const float2 f = __ldg(reinterpret_cast<const float2*>(feat + off) + i);
+                const float2 g = __ldg(reinterpret_cast<const float2*>(dfeat + off) + i);
+                d[2 * i] = (live && f.x > 0.f) ? g.x : 0.f;
+                d[2 * i + 1] = (live && f.y > 0.f) ? g.y : 0.f;
+            }
+            uint32_t w[DP];      // [hi pairs | lo pairs]
+#pragma unroll
+            for (int i = 0; i < DP / 2; ++i) {
+                const float l0 = d[2 * i] - __bfloat162float(__float2bfloat16_rn(d[2 * i])), l1 = d[2 * i + 1] - __bfloat162float(__float2bfloat16_rn(d[2 * i + 1]));
+                w[i] = pack_bf16(d[2 * i], d[2 * i + 1]);
+                w[DP / 2 + i] = pack_bf16(l0, l1);
+            }
+            if (ok && !mbar_wait(&dp_free[slot], ((unit >> 1) & 1) ^ 1)) { ok = false; report_timeout(status, 611); }
+            if (!ok) break;
+            if constexpr (DP == 6) {
+                st_shared_v4(dpblk + sw128_off(row, 2 * slot), w[0], w[1], w[2], w[3]);
+                st_shared_v4(dpblk + sw128_off(row, 2 * slot + 1), w[4], w[5], 0u, 0u);
+            } else {
+                const uint32_t blk = dpblk + slot * kBlk;
+#pragma unroll
+                for (int c = 0; c < 3; ++c) st_shared_v4(blk + sw128_off(row, c), w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+            }
+            fence_proxy_async();
+            mbar_arrive(&dp_full[slot]);
         }
     } else {
         const int quarter = warp & 3, part = (warp - kPbEpiWarp0) >> 2;
@@ -341,68 +395,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 mbar_arrive(dx_empty);
             }
         };
-        // dp = dfeat (.) 1[feat > 0] as the A operand [dp_hi | dp_lo] of the dg product.  Every epilogue thread of parts
-        // 0..2 owns one pair of features of its row: it loads them two units ahead (row index clamped, the loads are
-        // unconditional) and writes the tile of unit u + 1 at the start of unit u, so no single warp carries this work.
-        // Slot (u + 1) & 1 is free then: its last reader, the dg product of unit u - 1, completed before unit u - 1's
-        // dg was read.
-        const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
-        constexpr int NP = DP / 6;          // feature pairs per thread of parts 0..2: features 2 NP part .. 2 NP part + 2 NP - 1
-        float fpre[2 * NP], gpre[2 * NP];
-#pragma unroll
-        for (int i = 0; i < 2 * NP; ++i) fpre[i] = gpre[i] = 0.f;
-        bool live_pre = false;
-        int off_it = -1;          // tile whose row offset is cached in off_tile (the offset of map 0)
-        size_t off_tile = 0;
-        auto dp_load = [&](int unit) {
-            if (part == 3 || unit >= nunits) return;
-            const int it = unit / NMAPS, m = unit % NMAPS;
-            if (it != off_it) {
-                long long grow = (t0 + it) * kTileTokens + row;
-                live_pre = grow < rows;
-                grow = live_pre ? grow : rows - 1;
-                if (KSIDE) {
-                    const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
-                    off_tile = ((size_t)bh * NMAPS * N + n) * DP;
-                } else {
-                    off_tile = (size_t)grow * DP;
-                }
-                off_it = it;
-            }
-            const size_t off = off_tile + (KSIDE ? (size_t)m * N * DP : 0);
-#pragma unroll
-            for (int i = 0; i < NP; ++i) {
-                const float2 f = __ldg(reinterpret_cast<const float2*>(feat + off) + NP * part + i);
-                const float2 g = __ldg(reinterpret_cast<const float2*>(dfeat + off) + NP * part + i);
-                fpre[2 * i] = f.x; fpre[2 * i + 1] = f.y;
-                gpre[2 * i] = g.x; gpre[2 * i + 1] = g.y;
-            }
-        };
-        auto dp_store = [&](int unit) {      // the pairs loaded by the last dp_load go into the tile of `unit`
-            if (unit >= nunits) return;
-            if (part < 3) {
-                const uint32_t slot = unit & 1;
-                // DP = 6: both tiles in one block, K columns 16 slot ..; DP = 12: one block per tile
-                const uint32_t blk = dpblk + (DP == 6 ? 0u : slot * kBlk), col0 = DP == 6 ? 16 * slot : 0;
-#pragma unroll
-                for (int i = 0; i < NP; ++i) {
-                    const float d0 = (live_pre && fpre[2 * i] > 0.f) ? gpre[2 * i] : 0.f, d1 = (live_pre && fpre[2 * i + 1] > 0.f) ? gpre[2 * i + 1] : 0.f;
-                    const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
-                    const uint32_t khi = col0 + 2 * (NP * part + i), klo = khi + DP;      // K columns of the pair: hi half, lo half
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, khi >> 3) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, klo >> 3) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
-                }
-            }
-            fence_proxy_async();
-            mbar_arrive(&dp_full[unit & 1]);
-        };
-        dp_load(0);
-        dp_store(0);
-        dp_load(1);
         for (int unit = 0; unit < nunits && ok; ++unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
-            dp_store(unit + 1);
-            dp_load(unit + 2);
             if (!mbar_wait(dg_full, unit & 1)) { ok = false; report_timeout(status, 608); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
