@@ -79,8 +79,10 @@ struct PhiBwdPtrs {
 // warps 19..22: dp tiles (thread = token row).  The dp tiles were written by the epilogue threads at first; per unit that
 // cost each of the sixteen epilogue warps, whose instruction stream is what bounds the kernel, 600 of its 2850 cycles
 // (two loads, the split into two bf16 halves, two 4-byte stores, and above all one proxy fence per thread).
-constexpr int kPbThreads = 736;
-constexpr int kPbEpiWarp0 = 3, kPbDpWarp0 = 19;
+// Warps 23..26: drain of the dX accumulator (thread = token row): TMEM -> bf16 -> swizzled staging tile -> TMA store.  It
+// ran on the epilogue warps at first (557 of their cycles per unit on the key side, a third of a unit on the query side).
+constexpr int kPbThreads = 864;
+constexpr int kPbEpiWarp0 = 3, kPbDpWarp0 = 19, kPbDrainWarp0 = 23;
 
 // DP = d_phi: 6 (F = 3) or 12 (F = 2).  The dp tile of a unit is [dp_hi | dp_lo] = 2 DP K columns: one K = 16 step for DP = 6 (two
 // tiles share one swizzled block at K columns 0..15 and 16..31), two steps for DP = 12 (one block per tile, K columns 0..23).
@@ -100,11 +102,8 @@ template <int DV, int NMAPS, int DP> struct PbCfg {
     // 44 is a constant 1, never written again; the dp tiles use lower columns), B = the last K step of the map's W2^T
     // tile, whose row 12 holds b1 (the rows from 2 DP on meet zero columns of the dp tiles in the dg product, so they are free there)
     static constexpr int kB1Row = 12;
-    // dX staging tile (128 x DV) for a TMA store: query side and d = 64.  On the key side at d = 128 (a drain every
-    // third unit) the two block-wide barriers of the staged drain cost more than the direct stores they replace
-    // (measured, also as a drain in two halves).
-    static constexpr bool kStagedDrain = NMAPS == 1 || DV == 64;
-    static constexpr int kStageBlocks = kStagedDrain ? DV / 64 : 0;
+    // dX staging tile (128 x DV) for the TMA store of the drain
+    static constexpr int kStageBlocks = DV / 64;
     static constexpr int kOffStage = kOffW2t + NMAPS * kW2tBytes;
     static constexpr int kOffBars = kOffStage + kStageBlocks * kBlk;
     static constexpr int kSmemUsed = 1024 + kOffBars + 256;
@@ -142,11 +141,11 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
     uint64_t* dg_full = bars + 20;     // MMA commit
     uint64_t* dg_empty = bars + 21;    // 512 arrivals
     uint64_t* dx_full = bars + 22;     // MMA commit
-    uint64_t* dx_empty = bars + 23;    // 512 arrivals
+    uint64_t* dx_empty = bars + 23;    // 128 arrivals
     uint64_t* w_full = bars + 24;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
     uint64_t* stage_free = bars + 26;  // 1 arrival: the previous TMA store has read the dX staging tile
-    uint64_t* stage_full = bars + 27;  // 512 arrivals: the staging tile of this drain is written
+    uint64_t* stage_full = bars + 27;  // 128 arrivals: the staging tile of this drain is written
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -182,10 +181,10 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         mbar_init(dg_full, 1);
         mbar_init(dg_empty, 512);
         mbar_init(dx_full, 1);
-        mbar_init(dx_empty, 512);
+        mbar_init(dx_empty, 128);
         mbar_init(w_full, 1);
         mbar_init(stage_free, 1);
-        mbar_init(stage_full, 512);
+        mbar_init(stage_full, 128);
         fence_mbar_init();
         prefetch_tmap(&mapX);
         prefetch_tmap(&mapdX);
@@ -281,6 +280,60 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             }
             if (!good) report_timeout(status, 603);
         }
+    } else if (warp >= kPbDrainWarp0) {
+        // dX of a tile: TMEM -> bf16 -> swizzled staging tile -> TMA store (rows past the end are clipped by the store).
+        // The two hand-overs around the staging tile go through mbarriers with bounded waits, so a warp that has given up
+        // elsewhere cannot leave the others waiting for ever.
+        const int quarter = warp & 3, row = quarter * 32 + lane;
+        const uint32_t tx = tmem + 384 + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t sbase = smem_u32(smem + Cfg::kOffStage);
+        const bool leader = tid == kPbDrainWarp0 * 32;
+        for (int it = 0; it < ntiles; ++it) {
+            if (ok && !mbar_wait(dx_full, it & 1)) { ok = false; report_timeout(status, 606); }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            if (leader) {
+                tma_store_wait_read0();      // the previous tile's store has read the staging tile
+                mbar_arrive(stage_free);
+            }
+#pragma unroll 1
+            for (int h = 0; h < DV / 32; ++h) {
+                uint32_t r[32];
+                tmem_ld16(tx + 32 * h, *reinterpret_cast<uint32_t(*)[16]>(r));
+                tmem_ld16(tx + 32 * h + 16, *reinterpret_cast<uint32_t(*)[16]>(r + 16));
+                tmem_ld_wait();
+                if (h == DV / 32 - 1) {
+                    tc_fence_before();
+                    mbar_arrive(dx_empty);          // the accumulator has been read
+                }
+                if (h == 0) {
+                    if (!mbar_wait(stage_free, it & 1)) { ok = false; report_timeout(status, 609); }
+                    ok = __all_sync(0xffffffffu, ok);
+                }
+                if (ok) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        st_shared_v4(sbase + (h >> 1) * kBlk + sw128_off(row, 4 * (h & 1) + c), pack_bf16(__uint_as_float(r[8 * c]), __uint_as_float(r[8 * c + 1])),
+                                     pack_bf16(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3])),
+                                     pack_bf16(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5])),
+                                     pack_bf16(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7])));
+                }
+            }
+            if (!ok) break;
+            fence_proxy_async();
+            mbar_arrive(stage_full);
+            if (leader) {
+                if (mbar_wait(stage_full, it & 1)) {
+                    for (int blk = 0; blk < Cfg::kStageBlocks; ++blk)
+                        tma_store_2d(&mapdX, smem + Cfg::kOffStage + blk * kBlk, blk * 64, (int)((t0 + it) * kTileTokens));
+                    tma_store_commit();
+                } else {
+                    report_timeout(status, 610);
+                }
+            }
+        }
+        if (leader) tma_store_wait_all0();
     } else if (warp >= kPbDpWarp0) {
         // dp = dfeat (.) 1[feat > 0] of one token row as the A operand [dp_hi | dp_lo] of the dg product: the two bf16 halves
         // of every value, so that dg is exact to ~2^-17.  DP = 6: the two slots share one block (K columns 16 slot ..);
@@ -331,70 +384,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         const int quarter = warp & 3, part = (warp - kPbEpiWarp0) >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        // dX of tile `it`: TMEM -> bf16 -> global memory.  Staged: through a swizzled tile in shared memory and a TMA store
-        // (direct 32-byte stores put 32 separate sectors into every store instruction and hold the 16 warps for ~1000
-        // cycles per tile).  Otherwise each thread stores its HC contiguous columns directly, one sector per store.
-        auto drain_dx = [&](int it) {
-            if (ok && !mbar_wait(dx_full, it & 1)) { ok = false; report_timeout(status, 606); }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) return;
-            tc_fence_after();
-            const uint32_t tx = tmem + 384 + lane_base + part * HC;
-            if constexpr (Cfg::kStagedDrain) {
-                uint32_t w[HC / 2];
-#pragma unroll
-                for (int c = 0; c < HC / 16; ++c) {
-                    uint32_t r[16];
-                    tmem_ld16(tx + 16 * c, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) w[8 * c + e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                }
-                tc_fence_before();
-                mbar_arrive(dx_empty);          // the accumulator is in registers
-                const int col0 = part * HC;     // first column of this thread
-                const uint32_t sblk = smem_u32(smem + Cfg::kOffStage) + (col0 / 64) * kBlk;
-                // The two hand-overs around the staging tile go through mbarriers with bounded waits (not bar.sync), so a
-                // warp that has given up elsewhere cannot leave the others waiting for ever.
-                const bool leader = tid == kPbEpiWarp0 * 32;
-                if (leader) {
-                    tma_store_wait_read0();      // the previous tile's store has read the staging tile
-                    mbar_arrive(stage_free);
-                }
-                if (!mbar_wait(stage_free, it & 1)) { ok = false; report_timeout(status, 609); }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return;
-#pragma unroll
-                for (int j = 0; j < HC / 8; ++j)
-                    st_shared_v4(sblk + sw128_off(row, (col0 & 63) / 8 + j), w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-                fence_proxy_async();
-                mbar_arrive(stage_full);
-                if (leader) {
-                    if (mbar_wait(stage_full, it & 1)) {
-                        for (int blk = 0; blk < Cfg::kStageBlocks; ++blk)
-                            tma_store_2d(&mapdX, smem + Cfg::kOffStage + blk * kBlk, blk * 64, (int)((t0 + it) * kTileTokens));
-                        tma_store_commit();
-                    } else {
-                        report_timeout(status, 610);
-                    }
-                }
-            } else {
-                const long long grow = (t0 + it) * kTileTokens + row;
-                uint4* dst = reinterpret_cast<uint4*>(dX + (size_t)grow * DV + part * HC);
-#pragma unroll
-                for (int c = 0; c < HC / 16; ++c) {
-                    uint32_t r[16];
-                    tmem_ld16(tx + 16 * c, r);
-                    tmem_ld_wait();
-                    uint32_t w[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                    if (grow < rows) st_global_v8(dst + 2 * c, w);      // one full 32-byte sector per store
-                }
-                tc_fence_before();
-                mbar_arrive(dx_empty);
-            }
-        };
         for (int unit = 0; unit < nunits && ok; ++unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
             if (!mbar_wait(dg_full, unit & 1)) { ok = false; report_timeout(status, 608); }
@@ -433,10 +422,7 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(&dh_full[b]);
-            if (m == 0 && it > 0) drain_dx(it - 1);
         }
-        if (ok && ntiles > 0) drain_dx(ntiles - 1);
-        if (Cfg::kStagedDrain && tid == kPbEpiWarp0 * 32) tma_store_wait_all0();
     }
     tc_fence_before();
     __syncthreads();
