@@ -228,6 +228,9 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
                 // h[b] also holds the dh operand of unit - 2 (written over the h columns that were read): it is free when
                 // that unit's dX product has completed
                 if (!mbar_wait(&dh_free[b], ((unit >> 1) & 1) ^ 1)) { good = false; break; }
+                // dg of this unit must be complete too, so that h_full tells the epilogue warps both (one wait per unit on
+                // their instruction stream instead of two); dg(unit) was issued a unit ago
+                if (!mbar_wait(dg_full, unit & 1)) { good = false; break; }
                 tc_fence_after();
                 const uint64_t xd = desc_advance(xd0, st * Cfg::kXBytes), wd = desc_advance(wd0, m * Cfg::kW1Bytes);
 #pragma unroll
@@ -386,7 +389,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         for (int unit = 0; unit < nunits && ok; ++unit) {
             const int it = unit / NMAPS, m = unit % NMAPS, b = unit & 1, par = (unit >> 1) & 1;
-            if (!mbar_wait(dg_full, unit & 1)) { ok = false; report_timeout(status, 608); }
+            // h_full(unit) also says that dg(unit) is complete (the thread that issues the h products waits for it first)
+            if (!mbar_wait(&h_full[b], par)) { ok = false; report_timeout(status, 604); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -396,12 +400,8 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(dg_empty);
-            // (dg(u) complete also means the dX product of unit u - 2 has completed - same issuing thread, issued earlier,
-            // and a commit covers everything before it - so the dh tile of this parity is free without a wait of its own.)
-            if (!mbar_wait(&h_full[b], par)) { ok = false; report_timeout(status, 604); }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
+            // (the h products of this unit were issued after the dX product of unit - 2 had completed, so the dh tile of this
+            // parity is free)
             const uint32_t ta = tmem + 128 * b + lane_base + part * HC;
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) {
