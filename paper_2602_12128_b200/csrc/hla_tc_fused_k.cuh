@@ -139,10 +139,12 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* x_full = bars;           // [2] TMA
     uint64_t* x_empty = bars + 2;      // [2] MMA commit
-    uint64_t* d1_full = bars + 4;      // [2] MMA commit
+    uint64_t* d1_full = bars + 4;      // [2] two MMA commits: the first-layer product of the unit, and the second-layer product of
+                                       // unit - 2 (the G tile of this parity has been read: the GELU warps may write it again), so
+                                       // that the GELU warps wait once per unit; the first phase gets the second arrival at set-up
     uint64_t* d1_empty = bars + 6;     // [2] 512 arrivals
     uint64_t* g_full = bars + 8;       // [2] 512 arrivals
-    uint64_t* g_free = bars + 10;      // [2] MMA commit
+    uint64_t* g_free = bars + 10;      // (unused: see d1_full)
     uint64_t* d2_full = bars + 12;     // [2] MMA commit
     uint64_t* d2_empty = bars + 14;    // [2] 128 arrivals
     uint64_t* w_full = bars + 16;      // TMA
@@ -182,7 +184,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         for (int i = 0; i < 2; ++i) {
             mbar_init(&x_full[i], 1);
             mbar_init(&x_empty[i], 1);
-            mbar_init(&d1_full[i], 1);
+            mbar_init(&d1_full[i], 2);
             mbar_init(&d1_empty[i], 512);
             mbar_init(&g_full[i], 512);
             mbar_init(&g_free[i], 1);
@@ -197,6 +199,8 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         mbar_init(acc_done, 1);
         mbar_init(acc_free, 128);
         fence_mbar_init();
+        mbar_arrive(&d1_full[0]);      // no second-layer product precedes the first two units
+        mbar_arrive(&d1_full[1]);
         prefetch_tmap(&mapK);
         prefetch_tmap(&mapV);
     }
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
                 for (int ks = 0; ks < DV / 16; ++ks)
                     umma_bf16_ta(tmem + Col::kD2 + Col::kD2Stride * b, tmem + Col::kG + 64 * b + 8 * ks, desc_advance(vd, (ks >> 2) * 2048 + (ks & 3) * 32), idesc2,
                                  ks > 0 ? 1u : 0u);
-                umma_commit(&g_free[b]);
+                umma_commit(&d1_full[b]);      // G[b] is free again: second arrival of the phase of unit + 2
                 umma_commit(&d2_full[b]);
             }
             if (!good) report_timeout(status, 803);
@@ -441,7 +445,6 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         for (int unit = 0; unit < NM * nwork; ++unit) {
             const int b = unit & 1, par = (unit >> 1) & 1;
             if (!mbar_wait(&d1_full[b], par)) { ok = false; report_timeout(status, 809); }
-            if (ok && !mbar_wait(&g_free[b], par ^ 1)) { ok = false; report_timeout(status, 810); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
