@@ -397,9 +397,6 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             uint32_t dgr[HC];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) tmem_ld16(tmem + 256 + lane_base + part * HC + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(dgr + 16 * c));
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(dg_empty);
             // (the h products of this unit were issued after the dX product of unit - 2 had completed, so the dh tile of this
             // parity is free)
             const uint32_t ta = tmem + 128 * b + lane_base + part * HC;
@@ -407,7 +404,11 @@ __global__ void __launch_bounds__(kPbThreads, 1) tc_phi_backward_kernel(const __
             for (int c = 0; c < HC / 16; ++c) {
                 uint32_t r[16];
                 tmem_ld16(ta + 16 * c, r);
-                tmem_ld_wait();
+                tmem_ld_wait();           // first round: dg and the first h columns in one batch of loads
+                if (c == 0) {
+                    tc_fence_before();
+                    mbar_arrive(dg_empty);
+                }
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
