@@ -191,6 +191,32 @@ hla_status hla_backward(hla_ctx *ctx, const void *Q, const void *K, const void *
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * The two passes in two halves, for a sequence whose N tokens are split over several devices (one context per device,
+ * each created with its own share of N).  Theorem 4.2's state C = sum_j T_k[j] v_j^T and the key-side sum z are sums
+ * over the tokens, so the shards' states add: between the two halves of a pass the caller adds the state region of the
+ * workspaces of all shards (fp32; hla_workspace_layout gives `state` / `dstate`, state_rows and state_ld; one all-reduce
+ * of B*H*state_rows*state_ld floats) and leaves the sum in every workspace.
+ *   forward:   hla_forward_keys (feature maps of K, state of the shard)  ->  sum of `state` over the shards  ->
+ *              hla_forward_queries (feature map of Q, readout against the summed state, O of the shard's tokens)
+ *   backward:  hla_backward_queries (query pass: dQ-side gradients, gradient state of the shard)  ->  sum of `dstate`
+ *              over the shards  ->  hla_backward_keys (key pass on the summed gradient state, then the phi backward:
+ *              dQ, dK, dV of the shard's tokens)
+ * Each half takes the arguments of the whole call and uses those it needs (the key half of the forward K and V, the
+ * query half Q and O; both halves of the backward the full list).  With a single shard and no sum in between the two
+ * halves give the results of hla_forward / hla_backward bit for bit.  Tensor-core set without the mask only:
+ * HLA_ERR_UNSUPPORTED on the fp32 SIMT path and for causal = 1 (a causal pass would need an exclusive scan of the
+ * shards' states instead of their sum).  The library itself never communicates between devices.
+ */
+hla_status hla_forward_keys(hla_ctx *ctx, const void *K, const void *V, void *workspace, size_t workspace_bytes, void *cuda_stream);
+hla_status hla_forward_queries(hla_ctx *ctx, const void *Q, void *O, void *workspace, size_t workspace_bytes, void *cuda_stream);
+hla_status hla_backward_queries(hla_ctx *ctx, const void *Q, const void *K, const void *V, const void *O,
+                                const void *dO, void *dQ, void *dK, void *dV,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+hla_status hla_backward_keys(hla_ctx *ctx, const void *Q, const void *K, const void *V, const void *O,
+                             const void *dO, void *dQ, void *dK, void *dV,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Gradients of sum(dO * O) with respect to the weights of the feature networks (Section 5, "Training Details": the
  * paper trains the phi maps with the rest of the model; Algorithm 1 step 4 defines where they act).  HLA_PHI_MLP
  * contexts on the tensor-core kernels only (HLA_ERR_UNSUPPORTED otherwise).  Call it after hla_backward with the

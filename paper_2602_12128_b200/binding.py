@@ -17,7 +17,7 @@ HLA_BF16, HLA_F32 = 0, 1
 HLA_PHI_MLP, HLA_PHI_NONE = 0, 1
 
 EXPORTS = [
-    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_backward_weights", "hla_set_phi_v", "hla_set_carry", "hla_value_mod_forward", "hla_value_mod_backward", "hla_forward_static",
+    "hla_create", "hla_set_phi", "hla_workspace_bytes", "hla_workspace_layout", "hla_forward", "hla_backward", "hla_forward_keys", "hla_forward_queries", "hla_backward_queries", "hla_backward_keys", "hla_backward_weights", "hla_set_phi_v", "hla_set_carry", "hla_value_mod_forward", "hla_value_mod_backward", "hla_forward_static",
     "hla_last_device_status", "hla_selftest_bounded_wait", "hla_last_launch_count", "hla_timing_enable", "hla_timing_collect", "hla_timing_get",
     "hla_destroy", "hla_status_string",
 ]
@@ -80,6 +80,13 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.hla_forward.restype = c_int32
     lib.hla_backward.argtypes = [c_void_p] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
     lib.hla_backward.restype = c_int32
+    lib.hla_forward_keys.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.hla_forward_keys.restype = c_int32
+    lib.hla_forward_queries.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.hla_forward_queries.restype = c_int32
+    for name in ("hla_backward_queries", "hla_backward_keys"):
+        getattr(lib, name).argtypes = [c_void_p] + [c_void_p] * 8 + [c_void_p, c_size_t, c_void_p]
+        getattr(lib, name).restype = c_int32
     lib.hla_backward_weights.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(HlaMlpGrad), POINTER(HlaMlpGrad), c_void_p, c_size_t, c_void_p]
     lib.hla_backward_weights.restype = c_int32
     lib.hla_set_carry.argtypes = [c_void_p, c_int32]
@@ -175,6 +182,33 @@ def hla_backward(ctx: int, Q, K, V, O, dO, dQ, dK, dV, workspace, stream=None, w
                                      _ptr(workspace), nbytes, _stream(stream))
     if st != HLA_OK:
         raise HlaError(st, "hla_backward")
+
+
+def hla_forward_keys(ctx: int, K, V, workspace, stream=None) -> None:
+    st = load_library().hla_forward_keys(ctx, _ptr(K), _ptr(V), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_forward_keys")
+
+
+def hla_forward_queries(ctx: int, Q, O, workspace, stream=None) -> None:
+    st = load_library().hla_forward_queries(ctx, _ptr(Q), _ptr(O), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, "hla_forward_queries")
+
+
+def _backward_half(name, ctx, Q, K, V, O, dO, dQ, dK, dV, workspace, stream):
+    st = getattr(load_library(), name)(ctx, _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream))
+    if st != HLA_OK:
+        raise HlaError(st, name)
+
+
+def hla_backward_queries(ctx: int, Q, K, V, O, dO, dQ, dK, dV, workspace, stream=None) -> None:
+    _backward_half("hla_backward_queries", ctx, Q, K, V, O, dO, dQ, dK, dV, workspace, stream)
+
+
+def hla_backward_keys(ctx: int, Q, K, V, O, dO, dQ, dK, dV, workspace, stream=None) -> None:
+    _backward_half("hla_backward_keys", ctx, Q, K, V, O, dO, dQ, dK, dV, workspace, stream)
 
 
 def hla_backward_weights(ctx: int, Q, K, dphi_q, dphi_k, workspace, stream=None, workspace_bytes=None) -> None:
@@ -300,6 +334,11 @@ class Hla:
         dV = torch.empty_like(V) if dV is None else dV
         hla_backward(self.ctx, Q, K, V, O, dO, dQ, dK, dV, self.workspace, stream)
         return dQ, dK, dV
+
+    def state_region(self, gradient=False):
+        """The fp32 state (or gradient state) of the last pass as a flat view of the workspace: what shards of a sequence add."""
+        n = self.cfg.B * self.cfg.H * self.layout.state_rows * self.layout.state_ld
+        return self.region("dstate" if gradient else "state")[:n]
 
     def set_carry(self, carry: bool):
         hla_set_carry(self.ctx, carry)

@@ -362,16 +362,30 @@ hla_status hla_workspace_layout(const hla_ctx* ctx, hla_ws_layout* out) {
     return HLA_OK;
 }
 
-hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V, void* O, void* workspace,
-                       size_t workspace_bytes, void* cuda_stream) {
-    const void* ptrs[4] = {Q, K, V, O};
-    hla_status s = check_call(ctx, ptrs, 4, workspace, workspace_bytes);
+}  // extern "C"
+
+namespace {
+// phase 0: the whole forward; 1: key side only (state left in the workspace); 2: query side only, on the state in the workspace
+hla_status forward_impl(hla_ctx* ctx, const void* Q, const void* K, const void* V, void* O, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                        int phase) {
+    hla_status s;
+    if (phase == 1) {
+        const void* ptrs[2] = {K, V};
+        s = check_call(ctx, ptrs, 2, workspace, workspace_bytes);
+    } else if (phase == 2) {
+        const void* ptrs[2] = {Q, O};
+        s = check_call(ctx, ptrs, 2, workspace, workspace_bytes);
+    } else {
+        const void* ptrs[4] = {Q, K, V, O};
+        s = check_call(ctx, ptrs, 4, workspace, workspace_bytes);
+    }
     if (s != HLA_OK) return s;
+    if (phase != 0 && (!ctx->tc || ctx->cfg.causal)) return HLA_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
     ctx->rec.start_call(st);
     (void)cudaGetLastError();
-    if (cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
+    if (phase != 2 && cudaMemsetAsync(ws + ctx->L.status, 0, 64, st) != cudaSuccess) return HLA_ERR_CUDA;
     follow_device(ctx);
     tc::HostCacheScope scope(&ctx->hc);
     if (ctx->tc) {
@@ -379,11 +393,16 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
         if (ctx->cfg.phi == HLA_PHI_MLP) {
             // one kernel for the key maps and the state build -> reduction of its pieces -> one kernel for phi_q, readout
             // and normaliser
-            s = tc::phik_state(ctx->D, ctx->BH, ctx->phi_k, K, V, ws, ctx->L, ctx->off_part, ctx->k_pieces, ctx->sm_count, ctx->rec);
-            if (s != HLA_OK) return s;
-            s = tc::reduce_pieces(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, ctx->off_part, ctx->k_pieces,
-                                  tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec, ctx->cfg.causal != 0);
-            if (s != HLA_OK) return s;
+            if (phase != 2) {
+                s = tc::phik_state(ctx->D, ctx->BH, ctx->phi_k, K, V, ws, ctx->L, ctx->off_part, ctx->k_pieces, ctx->sm_count, ctx->rec);
+                if (s != HLA_OK) return s;
+                s = tc::reduce_pieces(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, ctx->off_part, ctx->k_pieces,
+                                      tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->rec, ctx->cfg.causal != 0);
+                if (s != HLA_OK || phase == 1) return s;
+            } else {
+                s = tc::emit_from_state(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, false, ctx->rec);
+                if (s != HLA_OK) return s;
+            }
             s = tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
             if (s != HLA_OK || !ctx->cfg.causal) return s;
             // causal: the pass above left the features of both sides in the workspace (its O is overwritten now); the
@@ -395,14 +414,35 @@ hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V
             kf = static_cast<const float*>(K);
         }
         if (ctx->cfg.causal) return tc::causal_forward(ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->carry, ctx->rec);
-        return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
+        if (phase == 2) {
+            s = tc::emit_from_state(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, false, ctx->rec);
+            if (s != HLA_OK) return s;
+            return tc::readout_only(ctx->tcp, ctx->D, ctx->BH, qf, O, ws, ctx->L, ctx->sm_count, ctx->rec);
+        }
+        return tc::core_forward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, O, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec, phase == 0);
     }
     if (ctx->cfg.dtype == HLA_F32) return forward_simt<float>(ctx, Q, K, V, O, ws, st);
     return forward_simt<__nv_bfloat16>(ctx, Q, K, V, O, ws, st);
 }
+}  // namespace
 
-hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ,
-                        void* dK, void* dV, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+extern "C" {
+
+hla_status hla_forward(hla_ctx* ctx, const void* Q, const void* K, const void* V, void* O, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return forward_impl(ctx, Q, K, V, O, workspace, workspace_bytes, cuda_stream, 0);
+}
+hla_status hla_forward_keys(hla_ctx* ctx, const void* K, const void* V, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return forward_impl(ctx, nullptr, K, V, nullptr, workspace, workspace_bytes, cuda_stream, 1);
+}
+hla_status hla_forward_queries(hla_ctx* ctx, const void* Q, void* O, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return forward_impl(ctx, Q, nullptr, nullptr, O, workspace, workspace_bytes, cuda_stream, 2);
+}
+
+}  // extern "C"
+
+namespace {
+hla_status backward_impl(hla_ctx* ctx, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ, void* dK, void* dV,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream, int phase) {
     const void* ptrs[8] = {Q, K, V, O, dO, dQ, dK, dV};
     hla_status s = check_call(ctx, ptrs, 8, workspace, workspace_bytes);
     if (s != HLA_OK) return s;
@@ -412,6 +452,7 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
     (void)cudaGetLastError();
     follow_device(ctx);
     tc::HostCacheScope scope(&ctx->hc);
+    if (phase != 0 && (!ctx->tc || ctx->cfg.causal)) return HLA_ERR_UNSUPPORTED;
     if (ctx->tc) {
         const bool mlp = ctx->cfg.phi == HLA_PHI_MLP;
         // the phi backward writes rows of dQ, dK with 32-byte stores; so does the 2-factor key pass with dV
@@ -425,13 +466,29 @@ hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* 
             if (ctx->carry) return HLA_ERR_UNSUPPORTED;      // a chunk that started from a carried state has no backward here
             s = tc::causal_backward(ctx->D, ctx->BH, qf, kf, V, O, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->off_delta, ctx->rec);
         } else {
-            s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec);
+            s = tc::core_backward(ctx->tcp, ctx->D, ctx->BH, qf, kf, V, dO, dqf, dkf, dV, ws, ctx->L, ctx->off_part, ctx->sm_count, ctx->rec, phase);
         }
-        if (s != HLA_OK || !mlp) return s;
+        if (s != HLA_OK || !mlp || phase == 1) return s;
         return tc::phi_backward(ctx->D, ctx->BH, &ctx->phi_q, ctx->phi_k, Q, K, dQ, dK, ws, ctx->L, ctx->sm_count, ctx->rec);
     }
     if (ctx->cfg.dtype == HLA_F32) return backward_simt<float>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
     return backward_simt<__nv_bfloat16>(ctx, Q, K, V, O, dO, dQ, dK, dV, ws, st);
+}
+}  // namespace
+
+extern "C" {
+
+hla_status hla_backward(hla_ctx* ctx, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ, void* dK, void* dV,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return backward_impl(ctx, Q, K, V, O, dO, dQ, dK, dV, workspace, workspace_bytes, cuda_stream, 0);
+}
+hla_status hla_backward_queries(hla_ctx* ctx, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ, void* dK, void* dV,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return backward_impl(ctx, Q, K, V, O, dO, dQ, dK, dV, workspace, workspace_bytes, cuda_stream, 1);
+}
+hla_status hla_backward_keys(hla_ctx* ctx, const void* Q, const void* K, const void* V, const void* O, const void* dO, void* dQ, void* dK, void* dV,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return backward_impl(ctx, Q, K, V, O, dO, dQ, dK, dV, workspace, workspace_bytes, cuda_stream, 2);
 }
 
 hla_status hla_backward_weights(hla_ctx* ctx, const void* Q, const void* K, const hla_mlp_grad* dphi_q, const hla_mlp_grad* dphi_k, void* workspace,

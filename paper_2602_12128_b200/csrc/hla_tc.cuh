@@ -1452,6 +1452,44 @@ inline hla_status reduce_pieces(const Plan& P, const Dims& D, int BH, char* ws, 
                     : reduce_pieces_f<2>(P, D, BH, ws, L, off_part, smax, G, rec, scratch_state);
 }
 
+// The two bf16 operand images of a state that already sits, summed, in the workspace (the state region, or with
+// gradient = true the gradient-state region): what the reduction emits, from one "piece" that is the state itself.  Used
+// when the caller has added the states of several sequence shards between the key side and the query side of a pass.
+template <int DV, int F>
+inline hla_status launch_emit_from_state(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, bool gradient, LaunchRec& rec) {
+    float* st = reinterpret_cast<float*>(ws + (gradient ? L.dstate : L.state));
+    __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + (gradient ? P.bd3 : P.b3));
+    __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + (gradient ? P.bdq : P.bq));
+    rec.begin("tc_reduce_emit");
+    launch_pdl(tc_reduce_emit_kernel<DV, F>, dim3(MT<F>::kPad / 8, BH), dim3(256), 0, rec.st, (const float*)st, st, b3, bq, 1, D.ld, 0, 0);
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+inline hla_status emit_from_state(const Plan& P, const Dims& D, int BH, char* ws, const hla_ws_layout& L, bool gradient, LaunchRec& rec) {
+    if (D.F == 3) return D.d == 128 ? launch_emit_from_state<128, 3>(P, D, BH, ws, L, gradient, rec) : launch_emit_from_state<64, 3>(P, D, BH, ws, L, gradient, rec);
+    return D.d == 128 ? launch_emit_from_state<128, 2>(P, D, BH, ws, L, gradient, rec) : launch_emit_from_state<64, 2>(P, D, BH, ws, L, gradient, rec);
+}
+
+// The readout alone (feature-level entry), on the operand image in the workspace.
+template <int DV, int F>
+inline hla_status launch_readout_only(const Plan& P, const Dims& D, int BH, const float* qf, void* O, char* ws, const hla_ws_layout& L, int sm_count,
+                                      LaunchRec& rec) {
+    CUtensorMap mapO, mapB3;
+    __nv_bfloat16* b3 = reinterpret_cast<__nv_bfloat16*>(ws + P.b3);
+    if (!make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens) || !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), MT<F>::kPad, DV + 16)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_readout_kernel<DV, F>, RoCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
+    const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
+    const long long total = (long long)BH * tiles;
+    const int grid = (int)(total < sm_count ? total : sm_count);
+    rec.begin("tc_readout");
+    launch_pdl(tc_readout_kernel<DV, F>, grid, dim3(kRoThreads), RoCfg<DV, F>::kSmem, rec.st, mapB3, mapO, qf, reinterpret_cast<float*>(ws + L.eta), D.N, BH,
+               D.eps, reinterpret_cast<int*>(ws + L.status));
+    return rec.end() ? HLA_OK : HLA_ERR_CUDA;
+}
+inline hla_status readout_only(const Plan& P, const Dims& D, int BH, const float* qf, void* O, char* ws, const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
+    if (D.F == 3) return D.d == 128 ? launch_readout_only<128, 3>(P, D, BH, qf, O, ws, L, sm_count, rec) : launch_readout_only<64, 3>(P, D, BH, qf, O, ws, L, sm_count, rec);
+    return D.d == 128 ? launch_readout_only<128, 2>(P, D, BH, qf, O, ws, L, sm_count, rec) : launch_readout_only<64, 2>(P, D, BH, qf, O, ws, L, sm_count, rec);
+}
+
 // readout = false stops after the state has been built and reduced (the fused query-side kernel reads it out).
 inline hla_status core_forward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, void* O, char* ws,
                                const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec, bool readout = true) {
@@ -1466,7 +1504,9 @@ inline hla_status core_forward(const Plan& P, const Dims& D, int BH, const float
 template <int DV, int F>
 inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, const void* dO,
                                        float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count,
-                                       LaunchRec& rec) {
+                                       LaunchRec& rec, int phase) {
+    // phase 0: the whole backward; 1: query pass and reduction only (leaves the gradient state in the workspace);
+    // 2: key pass only, on the gradient state in the workspace (its operand images are formed first)
     constexpr int kPad = MT<F>::kPad;
     CUtensorMap mapV, mapdO, mapdV, mapBq, mapBd3, mapBdq;
     __nv_bfloat16* bq = reinterpret_cast<__nv_bfloat16*>(ws + P.bq);
@@ -1483,13 +1523,19 @@ inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, con
     const float* eta = reinterpret_cast<const float*>(ws + L.eta);
     if (!set_smem(tc_bwd_query_kernel<DV, F>, BqCfg<F>::kSmem) || !set_smem(tc_bwd_key_kernel<DV, F>, BkCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     cudaStream_t st = rec.st;
-    rec.begin("tc_bwd_query");
-    launch_pdl(tc_bwd_query_kernel<DV, F>, dim3(D.S, BH), dim3(kBqThreads), BqCfg<F>::kSmem, st, mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps,
-               status);
-    if (!rec.end()) return HLA_ERR_CUDA;
-    rec.begin("tc_reduce_emit");
-    launch_pdl(tc_reduce_emit_kernel<DV, F>, dim3(kPad / 8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld, 0, 0);
-    if (!rec.end()) return HLA_ERR_CUDA;
+    if (phase != 2) {
+        rec.begin("tc_bwd_query");
+        launch_pdl(tc_bwd_query_kernel<DV, F>, dim3(D.S, BH), dim3(kBqThreads), BqCfg<F>::kSmem, st, mapdO, mapBq, qf, eta, state, dqf, part, D.N, D.S, D.ld, D.eps,
+                   status);
+        if (!rec.end()) return HLA_ERR_CUDA;
+        rec.begin("tc_reduce_emit");
+        launch_pdl(tc_reduce_emit_kernel<DV, F>, dim3(kPad / 8, BH), dim3(256), 0, st, part, dstate, bd3, bdq, D.S, D.ld, 0, 0);
+        if (!rec.end()) return HLA_ERR_CUDA;
+        if (phase == 1) return HLA_OK;
+    } else {
+        const hla_status e = launch_emit_from_state<DV, F>(P, D, BH, ws, L, true, rec);
+        if (e != HLA_OK) return e;
+    }
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
@@ -1500,13 +1546,14 @@ inline hla_status launch_core_backward(const Plan& P, const Dims& D, int BH, con
 }
 
 inline hla_status core_backward(const Plan& P, const Dims& D, int BH, const float* qf, const float* kf, const void* V, const void* dO,
-                                float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec) {
+                                float* dqf, float* dkf, void* dV, char* ws, const hla_ws_layout& L, size_t off_part, int sm_count, LaunchRec& rec,
+                                int phase = 0) {
     if (D.F == 3) {
-        if (D.d == 128) return launch_core_backward<128, 3>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
-        return launch_core_backward<64, 3>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+        if (D.d == 128) return launch_core_backward<128, 3>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec, phase);
+        return launch_core_backward<64, 3>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec, phase);
     }
-    if (D.d == 128) return launch_core_backward<128, 2>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
-    return launch_core_backward<64, 2>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec);
+    if (D.d == 128) return launch_core_backward<128, 2>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec, phase);
+    return launch_core_backward<64, 2>(P, D, BH, qf, kf, V, dO, dqf, dkf, dV, ws, L, off_part, sm_count, rec, phase);
 }
 
 }  // namespace tc

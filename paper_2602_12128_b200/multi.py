@@ -1,8 +1,15 @@
-"""Host-side logic of the multi-GPU benchmark: one process per GPU, each running the
-whole operator on its own seeded batch.  Heads and batches are independent in every
-equation of the operator, so the data path has no collective; the only exchange is the
-maximum over ranks of the measured device time.  Works on any torch.distributed backend
-(NCCL on GPUs, gloo in the CPU tests)."""
+"""Host-side logic of the multi-GPU modes.
+
+Replicas (the benchmark): one process per GPU, each running the whole operator on its own seeded batch.  Heads and
+batches are independent in every equation of the operator, so the data path has no collective; the only exchange is the
+maximum over ranks of the measured device time.
+
+Sequence sharding (optional): the N tokens of every head are split over the ranks.  The state of Theorem 4.2 is a sum
+over tokens, so each pass needs one all-reduce (sum) of the fp32 state between its key half and its query half
+(`sharded_forward`, `sharded_backward`: the library's half-pass entry points with `all_reduce_sum` in between; the
+library itself never communicates).
+
+Works on any torch.distributed backend (NCCL on GPUs, gloo in the CPU tests)."""
 from __future__ import annotations
 
 import torch
@@ -25,3 +32,36 @@ def max_over_ranks(ms: float, dist=None, device="cpu") -> float:
 def whole_job_rate(units_per_rank: float, world: int, ms: float) -> float:
     """Units per second of the whole job: every rank processed `units_per_rank` in `ms` (the slowest rank's time)."""
     return world * units_per_rank / (ms * 1e-3)
+
+
+def shard_bounds(n_tokens: int, world: int, rank: int):
+    """[first, last) token of a rank's contiguous share of a sequence: shares differ by at most one token."""
+    base, extra = divmod(n_tokens, world)
+    first = rank * base + min(rank, extra)
+    return first, first + base + (1 if rank < extra else 0)
+
+
+def all_reduce_sum(t, dist=None):
+    """Sum of a tensor over the ranks, in place (a no-op for one process)."""
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return t
+
+
+def sharded_forward(op, Q, K, V, O, dist=None, stream=None):
+    """Forward of one rank's shard of the tokens: key half, sum of the state over the ranks, query half.  `op` is a
+    binding.Hla created with the shard's own N."""
+    from . import binding
+    binding.hla_forward_keys(op.ctx, K, V, op.workspace, stream)
+    all_reduce_sum(op.state_region(), dist)
+    binding.hla_forward_queries(op.ctx, Q, O, op.workspace, stream)
+    return O
+
+
+def sharded_backward(op, Q, K, V, O, dO, dQ, dK, dV, dist=None, stream=None):
+    """Backward of one rank's shard: query half, sum of the gradient state over the ranks, key half."""
+    from . import binding
+    binding.hla_backward_queries(op.ctx, Q, K, V, O, dO, dQ, dK, dV, op.workspace, stream)
+    all_reduce_sum(op.state_region(gradient=True), dist)
+    binding.hla_backward_keys(op.ctx, Q, K, V, O, dO, dQ, dK, dV, op.workspace, stream)
+    return dQ, dK, dV

@@ -53,3 +53,73 @@ def test_single_process_needs_no_group():
     from paper_2602_12128_b200 import multi
     assert multi.max_over_ranks(3.5) == 3.5
     assert multi.whole_job_rate(10.0, 1, 1000.0) == 10.0
+
+
+def _shard_worker(rank, world, port, out):
+    """Sequence sharding on the oracle: each rank builds the state of its own tokens, the ranks add them with the
+    library's host helper, and every rank reads out its own tokens against the sum."""
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import hla_oracle as orc
+    from paper_2602_12128_b200 import multi
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(5)                      # the same full problem on every rank
+    n, dphi, d, F = 37, 3, 4, 3
+    q = np.abs(rng.standard_normal((n, dphi)))
+    ks = [np.abs(rng.standard_normal((n, dphi))) for _ in range(F)]
+    v = rng.standard_normal((n, d))
+    do = rng.standard_normal((n, d))
+    lo, hi = multi.shard_bounds(n, world, rank)
+    C, z = orc.context_state([k[lo:hi] for k in ks], v[lo:hi])
+    state = torch.from_numpy(np.concatenate([C, z[:, None]], axis=1))
+    multi.all_reduce_sum(state, dist)
+    Cs, zs = state.numpy()[:, :d], state.numpy()[:, d]
+    o, eta = orc.readout(q[lo:hi], F, Cs, zs, 1e-3)
+    o_full, eta_full = orc.hla_quadratic(q, ks, v, 1e-3)
+    ok_fwd = bool(np.allclose(o, o_full[lo:hi], rtol=1e-10, atol=1e-12) and np.allclose(eta, eta_full[lo:hi], rtol=1e-10))
+    # backward: the gradient state is a sum over the query tokens
+    Tq = orc.outer_features([q[lo:hi]] * F)
+    r = 1.0 / (eta + 1e-3)
+    dnum = do[lo:hi] * r[:, None]
+    deta = -r * np.sum(do[lo:hi] * o, axis=1)
+    dstate = torch.from_numpy(np.concatenate([Tq.T @ dnum, (Tq.T @ deta)[:, None]], axis=1))
+    multi.all_reduce_sum(dstate, dist)
+    dC, dz = dstate.numpy()[:, :d], dstate.numpy()[:, d]
+    Tk = orc.outer_features([k[lo:hi] for k in ks])
+    dv = Tk @ dC
+    _, _, dv_full = orc.hla_quadratic_backward(q, ks, v, do, 1e-3)
+    ok_bwd = bool(np.allclose(dv, dv_full[lo:hi], rtol=1e-9, atol=1e-12)) and dz.shape == (dphi ** F,)
+    out.put((rank, lo, hi, ok_fwd, ok_bwd))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sequence_sharding_state_sum_two_ranks():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [(r[1], r[2]) for r in res] == [(0, 19), (19, 37)]       # 37 tokens over two ranks: 19 + 18
+    assert all(r[3] and r[4] for r in res)
+
+
+def test_shard_bounds_cover_the_sequence():
+    sys.path.insert(0, ROOT)
+    from paper_2602_12128_b200 import multi
+    for n in (1, 7, 128, 32760):
+        for world in (1, 2, 3, 8):
+            b = [multi.shard_bounds(n, world, r) for r in range(world)]
+            assert b[0][0] == 0 and b[-1][1] == n
+            assert all(b[i][1] == b[i + 1][0] for i in range(world - 1))
+            sizes = [hi - lo for lo, hi in b]
+            assert max(sizes) - min(sizes) <= 1
