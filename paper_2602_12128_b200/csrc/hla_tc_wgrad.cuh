@@ -13,15 +13,16 @@
 // CTA order, so the result is bit-reproducible.
 //
 // warp 0: TMA loads, warp 1: dg, dW1 and dW2 MMAs, warp 2: h MMAs, warps 3..18: arithmetic (thread = token row x quarter
-// of the hidden units), warps 19..20: column sums of the dh tile (db1).
+// of the hidden units), warps 19..20: column sums of the dh tile (db1), warps 21..24: dp tiles and db2 (thread = token row;
+// off the arithmetic warps' instruction stream, which is what bounds the kernel).
 #pragma once
 #include "hla_tc_phi.cuh"
 
 namespace hla {
 namespace tc {
 
-constexpr int kWgThreads = 21 * 32;
-constexpr int kWgEpiWarp0 = 3, kWgSumWarp0 = 19;
+constexpr int kWgThreads = 25 * 32;
+constexpr int kWgEpiWarp0 = 3, kWgSumWarp0 = 19, kWgDpWarp0 = 21;
 constexpr int kWgColDg = 128, kWgColW1 = 256, kWgColW2 = 384;      // TMEM columns (h at 0)
 
 template <int DV, int NMAPS, int DP> struct WgCfg {
@@ -63,7 +64,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
     uint64_t* w_empty = bars + 5;      // MMA commit after the map's last product
     uint64_t* h_full = bars + 6;       // MMA commit
     uint64_t* h_empty = bars + 7;      // 512 arrivals
-    uint64_t* dp_full = bars + 8;      // [3] 512 arrivals
+    uint64_t* dp_full = bars + 8;      // [3] 128 arrivals
+    uint64_t* dp_free = bars + 18;     // [3] MMA commit: the unit's products have read the block
     uint64_t* dg_full = bars + 11;     // MMA commit
     uint64_t* dg_empty = bars + 12;    // 512 arrivals
     uint64_t* gd_full = bars + 13;     // 512 arrivals: G and dh tiles written
@@ -102,7 +104,10 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
         mbar_init(w_empty, 1);
         mbar_init(h_full, 1);
         mbar_init(h_empty, 512);
-        for (int i = 0; i < 3; ++i) mbar_init(&dp_full[i], 512);
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(&dp_full[i], 128);
+            mbar_init(&dp_free[i], 1);
+        }
         mbar_init(dg_full, 1);
         mbar_init(dg_empty, 512);
         mbar_init(gd_full, 512);
@@ -150,6 +155,8 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
                 const int m = unit / ntiles, it = unit - m * ntiles, st = unit & 1;
                 if (it == 0 && !mbar_wait(w_full, m & 1)) { good = false; break; }
                 if (!(mbar_wait(&x_full[st], (unit >> 1) & 1) && mbar_wait(h_empty, (unit & 1) ^ 1))) { good = false; break; }
+                // the unit's dg product must be complete too, so that h_full tells the arithmetic warps both
+                if (!mbar_wait(dg_full, unit & 1)) { good = false; break; }
                 tc_fence_after();
                 const uint64_t xd = desc_advance(xd0, st * Cfg::kXBytes);
 #pragma unroll
@@ -199,6 +206,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
                     umma_bf16(tmem + kWgColW2, smem_desc_sw128(ga + ks * 2048, kBlk, 1024), smem_desc_sw128(dps + ks * 2048, kBlk, 1024), idesc_w2,
                               (it > 0 || ks > 0) ? 1u : 0u);
                 umma_commit(gd_empty);
+                umma_commit(&dp_free[unit % 3]);
                 umma_commit(&x_empty[st]);
                 if (it == ntiles - 1) {
                     umma_commit(acc_full);
@@ -207,7 +215,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             }
             if (!good) report_timeout(status, 1004);
         }
-    } else if (warp >= kWgSumWarp0) {
+    } else if (warp >= kWgSumWarp0 && warp < kWgDpWarp0) {
         // db1: column sums of the dh tile as the dW1 product sees it (bf16 values, fp32 sums); warp w owns the 64-column
         // block w, lane l its columns 2 l and 2 l + 1
         const int blk = warp - kWgSumWarp0;
@@ -239,25 +247,19 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
                 }
             }
         }
-    } else {
-        const int quarter = warp & 3, part = (warp - kWgEpiWarp0) >> 2;
-        const int row = quarter * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    } else if (warp >= kWgDpWarp0) {
+        // dp = dfeat (.) 1[feat > 0] of one token row as [dp_hi | dp_lo] (two bf16 halves, so dg is exact to ~2^-17) into
+        // block unit % 3, and db2 = sum over the tokens of dp (this warp's 32 tokens by shuffles: one partial per token quarter)
+        const int quarter = warp - kWgDpWarp0, row = quarter * 32 + lane;
         const uint32_t dpblk = smem_u32(smem + Cfg::kOffDp);
-        // dp = dfeat (.) 1[feat > 0] as [dp_hi | dp_lo] (two bf16 halves, so dg is exact to ~2^-17): every thread of parts 0..2
-        // owns one pair of features of its row, loads it two units ahead and writes the tile of unit u + 1 at the start of
-        // unit u.  Block (u + 1) % 3 is free then: its last readers, the products of unit u - 2, were waited for in unit u - 1.
-        constexpr int NP = DP / 6;          // feature pairs per thread of parts 0..2
-        float fpre[2 * NP], gpre[2 * NP], b2s[2 * NP];      // b2s: db2 of this thread's features, summed over its tokens of the current map
+        float b2s[DP];
 #pragma unroll
-        for (int i = 0; i < 2 * NP; ++i) fpre[i] = gpre[i] = b2s[i] = 0.f;
-        bool live_pre = false;
-        auto dp_load = [&](int unit) {
-            if (part == 3 || unit >= nunits) return;
+        for (int i = 0; i < DP; ++i) b2s[i] = 0.f;
+        for (int unit = 0; unit < nunits; ++unit) {
             const int m = unit / ntiles, it = unit - m * ntiles;
             long long grow = (t0 + it) * kTileTokens + row;
-            live_pre = grow < rows;
-            grow = live_pre ? grow : rows - 1;
+            const bool live = grow < rows;
+            grow = live ? grow : rows - 1;
             size_t off;
             if (KSIDE) {
                 const uint32_t bh = (uint32_t)grow / (uint32_t)N, n = (uint32_t)grow - bh * (uint32_t)N;   // rows < 2^31 (checked on the host)
@@ -265,77 +267,61 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             } else {
                 off = (size_t)grow * DP;
             }
+            uint32_t w[DP];      // [hi pairs | lo pairs]
 #pragma unroll
-            for (int i = 0; i < NP; ++i) {
-                const float2 f = __ldg(reinterpret_cast<const float2*>(feat + off) + NP * part + i);
-                const float2 g = __ldg(reinterpret_cast<const float2*>(dfeat + off) + NP * part + i);
-                fpre[2 * i] = f.x; fpre[2 * i + 1] = f.y;
-                gpre[2 * i] = g.x; gpre[2 * i + 1] = g.y;
+            for (int i = 0; i < DP / 2; ++i) {
+                const float2 f = __ldg(reinterpret_cast<const float2*>(feat + off) + i);
+                const float2 g = __ldg(reinterpret_cast<const float2*>(dfeat + off) + i);
+                const float d0 = (live && f.x > 0.f) ? g.x : 0.f, d1 = (live && f.y > 0.f) ? g.y : 0.f;
+                const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
+                w[i] = pack_bf16(d0, d1);
+                w[DP / 2 + i] = pack_bf16(l0, l1);
+                b2s[2 * i] += d0;
+                b2s[2 * i + 1] += d1;
             }
-        };
-        auto dp_store = [&](int unit) {      // the pairs loaded by the last dp_load go into the tile of `unit`
-            if (unit >= nunits) return;
-            if (part < 3) {
-                const uint32_t blk = dpblk + (unit % 3) * kBlk;
-                if (unit % ntiles == 0) {
+            if (ok && !mbar_wait(&dp_free[unit % 3], ((unit / 3) & 1) ^ 1)) { ok = false; report_timeout(status, 1010); }
+            if (!ok) break;
+            const uint32_t blk = dpblk + (unit % 3) * kBlk;
+            if constexpr (DP == 6) {
+                st_shared_v4(blk + sw128_off(row, 0), w[0], w[1], w[2], w[3]);
+                asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(blk + sw128_off(row, 1)), "r"(w[4]), "r"(w[5]) : "memory");
+            } else {
 #pragma unroll
-                    for (int i = 0; i < 2 * NP; ++i) b2s[i] = 0.f;
-                }
-#pragma unroll
-                for (int i = 0; i < NP; ++i) {
-                    const float d0 = (live_pre && fpre[2 * i] > 0.f) ? gpre[2 * i] : 0.f, d1 = (live_pre && fpre[2 * i + 1] > 0.f) ? gpre[2 * i + 1] : 0.f;
-                    const float l0 = d0 - __bfloat162float(__float2bfloat16_rn(d0)), l1 = d1 - __bfloat162float(__float2bfloat16_rn(d1));
-                    const uint32_t khi = 2 * (NP * part + i), klo = khi + DP;      // K columns of the pair: hi half, lo half
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, khi >> 3) + (khi & 7) * 2), "r"(pack_bf16(d0, d1)) : "memory");
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(blk + sw128_off(row, klo >> 3) + (klo & 7) * 2), "r"(pack_bf16(l0, l1)) : "memory");
-                    b2s[2 * i] += d0;
-                    b2s[2 * i + 1] += d1;
-                }
+                for (int c = 0; c < 3; ++c) st_shared_v4(blk + sw128_off(row, c), w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
             }
             fence_proxy_async();
             mbar_arrive(&dp_full[unit % 3]);
-        };
-        // db2 partial of map m: this warp's 32 tokens summed by shuffles, one partial per token quarter
-        auto flush_db2 = [&](int m) {
-            float* o = out_cta + (size_t)m * Cfg::kPartFloats + Cfg::kPartB2 + quarter * 16;
-            if (part < 3) {
+            if (it == ntiles - 1) {      // the map is complete: its db2 partial of this token quarter
+                float* o = out_cta + (size_t)m * Cfg::kPartFloats + Cfg::kPartB2 + quarter * 16;
 #pragma unroll
-                for (int i = 0; i < 2 * NP; ++i) {
+                for (int i = 0; i < DP; ++i) {
                     const float a = warp_sum(b2s[i]);
-                    if (lane == 0) o[2 * NP * part + i] = a;
+                    if (lane == 0) o[i] = a;
+                    b2s[i] = 0.f;
                 }
-            } else if (lane < 16 - 6 * NP) {
-                o[6 * NP + lane] = 0.f;
+                if (lane < 16 - DP) o[DP + lane] = 0.f;
             }
-        };
-        dp_load(0);
-        dp_store(0);
-        dp_load(1);
+        }
+    } else {
+        const int quarter = warp & 3, part = (warp - kWgEpiWarp0) >> 2;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         for (int unit = 0; unit < nunits && ok; ++unit) {
             const int m = unit / ntiles, it = unit - m * ntiles;
-            // the pair of unit + 1 belongs to the next map when this is the map's last tile: its db2 sum is flushed first
-            if (it == ntiles - 1) flush_db2(m);
-            dp_store(unit + 1);
-            dp_load(unit + 2);
-            if (!mbar_wait(dg_full, unit & 1)) { ok = false; report_timeout(status, 1006); }
+            // h_full(unit) also says that dg(unit) is complete (the thread that issues the h products waits for it first)
+            if (!mbar_wait(h_full, unit & 1)) { ok = false; report_timeout(status, 1007); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             uint32_t dgr[HC];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) tmem_ld16(tmem + kWgColDg + lane_base + part * HC + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(dgr + 16 * c));
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(dg_empty);
-            if (!mbar_wait(h_full, unit & 1)) { ok = false; report_timeout(status, 1007); }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
             uint32_t hr[HC];
 #pragma unroll
             for (int c = 0; c < HC / 16; ++c) tmem_ld16(tmem + lane_base + part * HC + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(hr + 16 * c));
             tmem_ld_wait();
             tc_fence_before();
+            mbar_arrive(dg_empty);
             mbar_arrive(h_empty);
             uint32_t gw[HC / 2], dw[HC / 2];
 #pragma unroll
