@@ -9,6 +9,9 @@ Backward: GELU'(x) = Phi(x) + x pdf(x) through the same kind of tanh:
 (r y = (1 - th^2) / 4: the derivative of the tanh form with its inner derivative a free polynomial); fit_tanh_grad()
 fits a, b, C0, C1 against the exact GELU' on |x| <= 8.
 
+Weight gradients need GELU and GELU' of the same element; fit_tanh_grad_shared() keeps the forward's a, b (so that one
+tanh serves both) and fits only C0, C1 of the derivative form (max error 5.2e-4 instead of 1.5e-4).
+
 Run:  python fit_gelu_tanh.py   -> prints both sets of constants and their maximum absolute errors; the constants in
 hla_tc_phi.cuh are this script's output."""
 import numpy as np
@@ -48,8 +51,18 @@ def fit_tanh_grad():
     return c, np.abs(gelu_grad_tanh(x, c) - ref).max()
 
 
+def fit_tanh_grad_shared(a, b):
+    from scipy.optimize import least_squares
+    x = np.linspace(-8, 8, 32001)
+    ref = gelu_grad_exact(x)
+    c = least_squares(lambda c: gelu_grad_tanh(x, (a, b, c[0], c[1])) - ref, np.array([1.6, 0.2])).x
+    return c, np.abs(gelu_grad_tanh(x, (a, b, c[0], c[1])) - ref).max()
+
+
 if __name__ == "__main__":
     c, err = fit_tanh_grad()
     print("tanh form of GELU': a = %.8ff, b = %.8ff, C0 = %.8ff, C1 = %.8ff, max |error| = %.3e" % (*c, err))
     (a, b), err = fit_tanh()
     print("tanh form: a = %.8ff, b = %.8ff, max |Phi error| = %.3e" % (a, b, err))
+    c, err = fit_tanh_grad_shared(a, b)
+    print("GELU' on the forward's tanh: C0 = %.8ff, C1 = %.8ff, max |error| = %.3e" % (*c, err))

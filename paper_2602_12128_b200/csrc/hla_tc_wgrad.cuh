@@ -328,8 +328,9 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             for (int e = 0; e < HC / 2; ++e) {
                 const float2 h = make_float2(__uint_as_float(hr[2 * e]), __uint_as_float(hr[2 * e + 1]));
                 const float2 dg = make_float2(__uint_as_float(dgr[2 * e]), __uint_as_float(dgr[2 * e + 1]));
-                const float2 g = gelu2_twice(h);                                 // 2 GELU(h); the factor 1/2 is applied when the partial is reduced
-                const float2 dh = __fmul2_rn(dg, gelu_grad2_twice(h));           // dg holds dg / 2 (halved W2^T)
+                float2 g, gr;
+                gelu_both2_twice(h, g, gr);                                      // 2 GELU(h) (the factor 1/2 is applied when the partial is reduced) and 2 GELU'(h)
+                const float2 dh = __fmul2_rn(dg, gr);                            // dg holds dg / 2 (halved W2^T)
                 gw[e] = pack_bf16(g.x, g.y);
                 dw[e] = pack_bf16(dh.x, dh.y);
             }
