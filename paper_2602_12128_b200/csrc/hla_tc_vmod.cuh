@@ -63,29 +63,31 @@ __global__ void __launch_bounds__(256) vmod_fold_kernel(VmlpPtrs a, VmlpPtrs b, 
 }
 
 // Row statistics of a 128-token bf16 tile in shared memory (two 64-column swizzled blocks): mean and 1 / sqrt(var + eps).
+// One pass over the row: sums of (x - shift) and (x - shift)^2 with shift = the mean of the row's first eight elements, which
+// is within a few standard deviations of the row mean, so the difference of the two moments loses no more than a few bits.
 template <int DV>
 __device__ __forceinline__ void tile_row_stats(uint32_t tile, int row, float& mu, float& rstd) {
-    float s = 0.f;
+    float2 shift = make_float2(0.f, 0.f), s = shift, q = shift;      // shift holds minus the shift
 #pragma unroll 4
     for (int c = 0; c < DV / 8; ++c) {
         uint32_t w[4];
         asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(tile + (c >> 3) * kBlk + sw128_off(row, c & 7)) : "memory");
+        if (c == 0) {
+            float t = 0.f;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) s += __uint_as_float(w[e] << 16) + __uint_as_float(w[e] & 0xffff0000u);
-    }
-    mu = s * (1.f / DV);
-    float v = 0.f;
-#pragma unroll 4
-    for (int c = 0; c < DV / 8; ++c) {
-        uint32_t w[4];
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(tile + (c >> 3) * kBlk + sw128_off(row, c & 7)) : "memory");
+            for (int e = 0; e < 4; ++e) t += __uint_as_float(w[e] << 16) + __uint_as_float(w[e] & 0xffff0000u);
+            shift = splat2(-0.125f * t);
+        }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const float a = __uint_as_float(w[e] << 16) - mu, b = __uint_as_float(w[e] & 0xffff0000u) - mu;
-            v = fmaf(a, a, fmaf(b, b, v));
+            const float2 dlt = __fadd2_rn(make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u)), shift);
+            s = __fadd2_rn(s, dlt);
+            q = __ffma2_rn(dlt, dlt, q);
         }
     }
-    rstd = rsqrtf(v * (1.f / DV) + kLnEps);
+    const float m = (s.x + s.y) * (1.f / DV);
+    mu = m - shift.x;
+    rstd = rsqrtf(fmaxf((q.x + q.y) * (1.f / DV) - m * m, 0.f) + kLnEps);
 }
 // The A operand of the extra K step, 8 TMEM columns of one row: K0, K1 = -mu_hi; K2 = -mu_lo; K3, K4 = sigma_hi; K5 = sigma_lo.
 __device__ __forceinline__ void store_aug_row(uint32_t taddr, float mu, float rstd) {
@@ -104,6 +106,13 @@ __device__ __forceinline__ void lds_row16(uint32_t tile, int row, int c, uint32_
 __device__ __forceinline__ void sts_row16(uint32_t tile, int row, int c, const uint32_t (&w)[8]) {
     st_shared_v4(tile + (c >> 2) * kBlk + sw128_off(row, (2 * c) & 7), w[0], w[1], w[2], w[3]);
     st_shared_v4(tile + (c >> 2) * kBlk + sw128_off(row, (2 * c + 1) & 7), w[4], w[5], w[6], w[7]);
+}
+// Products of two pairs of bf16, each rounded once to bf16 (the same value as an fp32 product rounded to bf16: the
+// product of two 8-bit significands is exact in fp32).
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
 }
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
@@ -381,23 +390,28 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
 }
 
 // ---- backward of one map (input gradient) ---------------------------------------------------------------------------
-// warp 0: TMA (weights, X tiles), warp 1: dg and dxhat MMAs, warp 2: h MMAs, warps 3..18: GELU' (thread = token row x quarter of
-// the hidden units), warps 19..22: dy = dOut (.) Yother and row statistics, warps 23..26: LayerNorm backward and output.
-// Shared-memory tiles: X (two stages, kept until the tile's output is formed: the LayerNorm backward needs xhat), dOut (one
-// stage: read by the dy warps, then overwritten by the result tile and stored - or added to dX - by TMA), Yother (one stage:
-// multiplied in place into dy, the A operand of the dg product).
+// warp 0: TMA (lane 0: weights and X tiles, lane 1: dOut and Yother tiles), warp 1: dg and dxhat MMAs, warp 2: h MMAs, warps
+// 3..18: GELU' (thread = token row x quarter of the hidden units), warps 19..22: dy = dOut (.) Yother, row statistics and the residual, warps 23..26: LayerNorm backward,
+// warp 27: TMA stores.
+// Shared-memory tiles: X (two stages, kept until the tile's output is formed: the LayerNorm backward needs xhat; the result
+// is written over the X tile row by row and stored - or added to dX - by TMA from there), dOut and Yother (one stage each,
+// free again as soon as dy is formed and the dg product has read it, so the next tile's pair is in flight while this
+// tile runs through GELU', the dxhat product and the LayerNorm backward).  Yother is multiplied in place into dy, the A
+// operand of the dg product.
+// RESIDUAL: the dy warps copy the rows of dOut into tensor memory, where the output warps find them at the end of the tile.
 // The two row means of the LayerNorm backward come from the hidden layer, where the GELU' warps already hold the numbers:
 //     sum_i dxhat_i = sum_j dh_j c_j,     sum_i dxhat_i xhat_i = sum_j dh_j (h_j - b1'_j)       (dxhat = dh W1'^T, h = xhat W1' + b1')
-constexpr int kVbThreads = 27 * 32;
-constexpr int kVbGeluWarp0 = 3, kVbProdWarp0 = 19, kVbOutWarp0 = 23;
-constexpr int kVbColDg = 128, kVbColDx = 256, kVbColAug = 384;      // TMEM columns (h at 0, aug[b] at 384 + 8 b)
+constexpr int kVbThreads = 28 * 32;
+constexpr int kVbGeluWarp0 = 3, kVbProdWarp0 = 19, kVbOutWarp0 = 23, kVbStoreWarp = 27;
+constexpr int kVbAhead = 3;                                         // tiles between the L2 prefetch and the load
+constexpr int kVbColDg = 128, kVbColDx = 256, kVbColAug = 384, kVbColRes = 400;   // TMEM columns (h at 0, aug[b] at 384 + 8 b, dOut rows: 64)
 
 template <int DV> struct VbCfg {
     static constexpr int kXBytes = 2 * kBlk;
     static constexpr int kWBytes = DV * DV * 2;
     static constexpr int kAuxBytes = (DV / 64) * 2048;
     static constexpr int kOffX = 0;                              // 2 stages
-    static constexpr int kOffDo = 2 * kXBytes;                   // dOut tile -> result tile
+    static constexpr int kOffDo = 2 * kXBytes;                   // dOut tile
     static constexpr int kOffDy = kOffDo + kXBytes;              // Yother tile -> dy tile
     static constexpr int kOffW1 = kOffDy + kXBytes;
     static constexpr int kOffW2 = kOffW1 + kWBytes;
@@ -429,12 +443,12 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
     float* cb = reinterpret_cast<float*>(smem + Cfg::kOffCb);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBars);
     uint64_t* x_full = bars;           // [2] TMA
-    uint64_t* x_empty = bars + 2;      // [2] 128 arrivals (output warps)
+    uint64_t* x_empty = bars + 2;      // [2] 1 arrival: the result tile written over the X tile has been read by its store
     uint64_t* st_full = bars + 4;      // [2] 128 arrivals
     uint64_t* in_full = bars + 6;      // TMA: the dOut and Yother tiles have landed
     uint64_t* dy_full = bars + 7;      // 128 arrivals
     uint64_t* dy_empty = bars + 8;     // MMA commit
-    uint64_t* do_free = bars + 9;      // 1 arrival: the result tile has been read by its store
+    uint64_t* do_free = bars + 9;      // 128 arrivals: the dy warps are done with the dOut tile
     uint64_t* h_full = bars + 10;      // MMA commit
     uint64_t* dh_full = bars + 11;     // 512 arrivals
     uint64_t* dh_free = bars + 12;     // MMA commit (the dxhat product has read dh: the h columns are free)
@@ -443,8 +457,9 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
     uint64_t* dx_full = bars + 15;     // MMA commit
     uint64_t* dx_empty = bars + 16;    // [2] 128 arrivals, by tile parity
     uint64_t* w_full = bars + 18;      // TMA
-    uint64_t* o_full = bars + 19;      // 128 arrivals: the result tile is written
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+    uint64_t* o_full = bars + 19;      // [2] 128 arrivals, by tile parity: the result tile is written
+    uint64_t* res_full = bars + 21;    // 128 arrivals (RESIDUAL): the tile's dOut rows are in tensor memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -454,14 +469,16 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(&x_full[i], 1);
-            mbar_init(&x_empty[i], 128);
+            mbar_init(&x_empty[i], 1);
             mbar_init(&st_full[i], 128);
             mbar_init(&dx_empty[i], 128);
+            mbar_init(&o_full[i], 128);
         }
         mbar_init(in_full, 1);
         mbar_init(dy_full, 128);
         mbar_init(dy_empty, 1);
-        mbar_init(do_free, 1);
+        mbar_init(do_free, 128);
+        mbar_init(res_full, 128);
         mbar_init(h_full, 1);
         mbar_init(dh_full, 512);
         mbar_init(dh_free, 1);
@@ -469,7 +486,6 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
         mbar_init(dg_empty, 512);
         mbar_init(dx_full, 1);
         mbar_init(w_full, 1);
-        mbar_init(o_full, 128);
         fence_mbar_init();
         prefetch_tmap(&mapX);
         prefetch_tmap(&mapW1);
@@ -504,12 +520,34 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                 tma_load_2d(smem + Cfg::kOffW2 + b * (DV * 128), &mapW2, w_full, b * 64, 0);
                 tma_load_2d(smem + Cfg::kOffAux + b * 2048, &mapAux, w_full, b * 64, 0);
             }
+            // The shared-memory stages cover little of the latency of DRAM, so the three input tiles of a step are
+            // brought into L2 kVbAhead steps before their loads are issued.
+            auto prefetch = [&](int j) {
+                if (j >= ntiles) return;
+                for (int b = 0; b < DV / 64; ++b) {
+                    tma_prefetch_2d(&mapX, b * 64, (int)((t0 + j) * kTileTokens));
+                    tma_prefetch_2d(&mapdO, b * 64, (int)((t0 + j) * kTileTokens));
+                    tma_prefetch_2d(&mapY, b * 64, (int)((t0 + j) * kTileTokens));
+                }
+            };
+            for (int j = 1; j < kVbAhead; ++j) prefetch(j);
             for (int it = 0; it < ntiles; ++it) {
                 const int st = it & 1, u = it >> 1;
+                prefetch(it + kVbAhead);
                 if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 1201); break; }
                 mbar_arrive_expect_tx(&x_full[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b)
                     tma_load_2d(smem + Cfg::kOffX + st * Cfg::kXBytes + b * kBlk, &mapX, &x_full[st], b * 64, (int)((t0 + it) * kTileTokens));
+            }
+        } else if (lane == 1) {
+            // dOut and Yother tiles: free once the dg product of the previous tile has read dy and the dy warps are done with dOut
+            for (int it = 0; it < ntiles; ++it) {
+                if (it > 0 && !(mbar_wait(dy_empty, (it - 1) & 1) && mbar_wait(do_free, (it - 1) & 1))) { report_timeout(status, 1205); break; }
+                mbar_arrive_expect_tx(in_full, 2 * DV * kTileTokens * 2);
+                for (int b = 0; b < DV / 64; ++b) {
+                    tma_load_2d(smem + Cfg::kOffDo + b * kBlk, &mapdO, in_full, b * 64, (int)((t0 + it) * kTileTokens));
+                    tma_load_2d(smem + Cfg::kOffDy + b * kBlk, &mapY, in_full, b * 64, (int)((t0 + it) * kTileTokens));
+                }
             }
         }
     } else if (warp == 2) {
@@ -567,13 +605,28 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
             }
             if (!good) report_timeout(status, 1203);
         }
+    } else if (warp == kVbStoreWarp) {
+        // the result tile leaves through TMA; its X stage is free for the next load once the store has read it
+        if (lane == 0) {
+            for (int it = 0; it < ntiles; ++it) {
+                const int st = it & 1;
+                if (!mbar_wait(&o_full[st], (it >> 1) & 1)) { report_timeout(status, 1210); break; }
+                const uint8_t* src = smem + Cfg::kOffX + st * Cfg::kXBytes;
+                for (int b = 0; b < DV / 64; ++b) {
+                    if (accumulate) tma_reduce_add_2d(&mapdX, src + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
+                    else tma_store_2d(&mapdX, src + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
+                }
+                tma_store_commit();
+                tma_store_wait_read0();
+                mbar_arrive(&x_empty[st]);
+            }
+            tma_store_wait_all0();
+        }
     } else if (warp >= kVbOutWarp0) {
         // LayerNorm backward: dx = rstd (dxhat - mean(dxhat) - xhat mean(dxhat xhat)) (+ dOut); thread = token row.  The result
-        // replaces the dOut tile and leaves through TMA.
+        // replaces the row of the X tile it was computed from.
         const int quarter = warp & 3, row = quarter * 32 + lane;
-        const bool leader = warp == kVbOutWarp0 && lane == 0;
         const uint32_t ta = tmem + kVbColDx + ((uint32_t)(quarter * 32) << 16);
-        const uint32_t dot = smem_u32(smem + Cfg::kOffDo);
         for (int it = 0; it < ntiles; ++it) {
             const int st = it & 1;
             if (ok && !mbar_wait(dx_full, it & 1)) { ok = false; report_timeout(status, 1204); }
@@ -590,67 +643,47 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                 s2 += v.y;
             }
             const float m1 = s1 * (1.f / DV), m2 = s2 * (1.f / DV);
+            // dx = rs acc - rs m1' - rs rstd m2' (x - mu) = rs acc + (k3 x + k4), with rs = rstd / 2: the GELU' warps leave out the
+            // factor 1/2 of GELU', so acc, m1' and m2' are twice dxhat and its two means
+            const float rs = 0.5f * rstd, k3 = -rs * rstd * m2, k4 = -rs * m1 - k3 * mu;
             const uint32_t xt = smem_u32(smem + Cfg::kOffX + st * Cfg::kXBytes);
+            if (RESIDUAL) {
+                if (ok && !mbar_wait(res_full, it & 1)) { ok = false; report_timeout(status, 1213); }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+            }
 #pragma unroll 2
             for (int c = 0; c < DV / 16; ++c) {
                 uint32_t r[16], xw[8], dw[8], w[8];
                 tmem_ld16(ta + 16 * c, r);
+                if (RESIDUAL) tmem_ld8(tmem + kVbColRes + ((uint32_t)(quarter * 32) << 16) + 8 * c, dw);
                 lds_row16(xt, row, c, xw);
-                if (RESIDUAL) lds_row16(dot, row, c, dw);
                 tmem_ld_wait();
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float xa = (bf_lo(xw[e]) - mu) * rstd, xb = (bf_hi(xw[e]) - mu) * rstd;
-                    float a = rstd * (__uint_as_float(r[2 * e]) - m1 - xa * m2), b = rstd * (__uint_as_float(r[2 * e + 1]) - m1 - xb * m2);
-                    if (RESIDUAL) {
-                        a += bf_lo(dw[e]);
-                        b += bf_hi(dw[e]);
-                    }
-                    w[e] = pack_bf16(a, b);
+                    const float2 lin = __ffma2_rn(make_float2(bf_lo(xw[e]), bf_hi(xw[e])), splat2(k3), splat2(k4));
+                    float2 v = __ffma2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), splat2(rs), lin);
+                    if (RESIDUAL) v = __fadd2_rn(v, make_float2(bf_lo(dw[e]), bf_hi(dw[e])));
+                    w[e] = pack_bf16(v.x, v.y);
                 }
-                sts_row16(dot, row, c, w);
+                sts_row16(xt, row, c, w);
             }
             tc_fence_before();
             mbar_arrive(&dx_empty[st]);
-            mbar_arrive(&x_empty[st]);
             fence_proxy_async();
-            mbar_arrive(o_full);
-            if (leader) {
-                if (mbar_wait(o_full, it & 1)) {
-                    for (int b = 0; b < DV / 64; ++b) {
-                        if (accumulate) tma_reduce_add_2d(&mapdX, smem + Cfg::kOffDo + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
-                        else tma_store_2d(&mapdX, smem + Cfg::kOffDo + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
-                    }
-                    tma_store_commit();
-                    tma_store_wait_read0();
-                    mbar_arrive(do_free);
-                } else {
-                    report_timeout(status, 1210);
-                }
-            }
+            mbar_arrive(&o_full[st]);
         }
-        if (leader) tma_store_wait_all0();
     } else if (warp >= kVbProdWarp0) {
-        // dy = dOut (.) Yother in place over the Yother tile -> A operand of the dg product; then the row statistics of the X tile
+        // dy = dOut (.) Yother in place over the Yother tile -> A operand of the dg product (the pair of tiles is ahead of the X
+        // tile), then the row statistics of the X tile
         const int t = tid - kVbProdWarp0 * 32;      // 0..127
         const int quarter = warp & 3, row = quarter * 32 + lane;
         constexpr int CPR = DV / 8;                 // 16-byte chunks per row
         const uint32_t dot = smem_u32(smem + Cfg::kOffDo), dyt = smem_u32(smem + Cfg::kOffDy);
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         for (int it = 0; it < ntiles; ++it) {
             const int st = it & 1, par = (it >> 1) & 1;
-            if (t == 0) {
-                // both tiles are free: the dg product of the previous tile has read dy, its result tile has been stored
-                bool free_ = it == 0 || (mbar_wait(dy_empty, (it - 1) & 1) && mbar_wait(do_free, (it - 1) & 1));
-                if (free_) {
-                    mbar_arrive_expect_tx(in_full, 2 * DV * kTileTokens * 2);
-                    for (int b = 0; b < DV / 64; ++b) {
-                        tma_load_2d(smem + Cfg::kOffDo + b * kBlk, &mapdO, in_full, b * 64, (int)((t0 + it) * kTileTokens));
-                        tma_load_2d(smem + Cfg::kOffDy + b * kBlk, &mapY, in_full, b * 64, (int)((t0 + it) * kTileTokens));
-                    }
-                } else {
-                    report_timeout(status, 1205);
-                }
-            }
             if (ok && !mbar_wait(in_full, it & 1)) { ok = false; report_timeout(status, 1211); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -661,13 +694,11 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                 uint32_t a[4], b[4];
                 asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(dot + off) : "memory");
                 asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]) : "r"(dyt + off) : "memory");
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) w[e] = pack_bf16(bf_lo(a[e]) * bf_lo(b[e]), bf_hi(a[e]) * bf_hi(b[e]));
-                st_shared_v4(dyt + off, w[0], w[1], w[2], w[3]);
+                st_shared_v4(dyt + off, mul_bf16x2(a[0], b[0]), mul_bf16x2(a[1], b[1]), mul_bf16x2(a[2], b[2]), mul_bf16x2(a[3], b[3]));
             }
             fence_proxy_async();
             mbar_arrive(dy_full);
+            if (!RESIDUAL) mbar_arrive(do_free);
             // statistics: buffer st was last read by the output warps of tile it - 2
             if (ok && !mbar_wait(&x_full[st], par)) { ok = false; report_timeout(status, 1206); }
             if (ok && it >= 2 && !mbar_wait(&dx_empty[st], par ^ 1)) { ok = false; report_timeout(status, 1207); }
@@ -675,11 +706,29 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
             if (!ok) break;
             float mu, rstd;
             tile_row_stats<DV>(smem_u32(smem + Cfg::kOffX + st * Cfg::kXBytes), row, mu, rstd);
-            store_aug_row(tmem + kVbColAug + 8 * st + ((uint32_t)(quarter * 32) << 16), mu, rstd);
+            store_aug_row(tmem + kVbColAug + 8 * st + lane_base, mu, rstd);
             stat[st * kTileTokens + row] = make_float2(mu, rstd);
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(&st_full[st]);
+            if (RESIDUAL) {
+                // the rows of dOut, as they are, into tensor memory for the output warps (one buffer: free once they have
+                // finished the previous tile), so that the dOut tile does not have to stay until the end of this one
+                if (ok && it > 0 && !mbar_wait(&dx_empty[(it - 1) & 1], ((it - 1) >> 1) & 1)) { ok = false; report_timeout(status, 1212); }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll 2
+                for (int c = 0; c < DV / 16; ++c) {
+                    uint32_t dw[8];
+                    lds_row16(dot, row, c, dw);
+                    tmem_st8(tmem + kVbColRes + lane_base + 8 * c, dw[0], dw[1], dw[2], dw[3], dw[4], dw[5], dw[6], dw[7]);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(res_full);
+                mbar_arrive(do_free);
+            }
         }
     } else {
         // dh = dg (.) GELU'(h), h = rstd acc: thread = token row x quarter of the hidden units; dh goes back into the h columns
@@ -715,7 +764,7 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                     const int j = part * HC + 16 * c + 2 * e;
                     const float2 h = __fmul2_rn(make_float2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), splat2(rstd));
                     const float2 dg = make_float2(__uint_as_float(dgr[16 * c + 2 * e]), __uint_as_float(dgr[16 * c + 2 * e + 1]));
-                    const float2 dh = __fmul2_rn(__fmul2_rn(dg, splat2(0.5f)), gelu_grad2_twice(h));
+                    const float2 dh = __fmul2_rn(dg, gelu_grad2_twice(h));      // twice dh: the output warps halve
                     w[e] = pack_bf16(dh.x, dh.y);
                     const float2 dr = make_float2(bf_lo(w[e]), bf_hi(w[e]));      // dh as the dxhat product sees it
                     const float2 cj = *reinterpret_cast<const float2*>(cb + j), bj = *reinterpret_cast<const float2*>(cb + DV + j);
