@@ -403,7 +403,6 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
 //     sum_i dxhat_i = sum_j dh_j c_j,     sum_i dxhat_i xhat_i = sum_j dh_j (h_j - b1'_j)       (dxhat = dh W1'^T, h = xhat W1' + b1')
 constexpr int kVbThreads = 28 * 32;
 constexpr int kVbGeluWarp0 = 3, kVbProdWarp0 = 19, kVbOutWarp0 = 23, kVbStoreWarp = 27;
-constexpr int kVbAhead = 3;                                         // tiles between the L2 prefetch and the load
 constexpr int kVbColDg = 128, kVbColDx = 256, kVbColAug = 384, kVbColRes = 400;   // TMEM columns (h at 0, aug[b] at 384 + 8 b, dOut rows: 64)
 
 template <int DV> struct VbCfg {
@@ -520,20 +519,8 @@ __global__ void __launch_bounds__(kVbThreads, 1) tc_vmlp_backward_kernel(const _
                 tma_load_2d(smem + Cfg::kOffW2 + b * (DV * 128), &mapW2, w_full, b * 64, 0);
                 tma_load_2d(smem + Cfg::kOffAux + b * 2048, &mapAux, w_full, b * 64, 0);
             }
-            // The shared-memory stages cover little of the latency of DRAM, so the three input tiles of a step are
-            // brought into L2 kVbAhead steps before their loads are issued.
-            auto prefetch = [&](int j) {
-                if (j >= ntiles) return;
-                for (int b = 0; b < DV / 64; ++b) {
-                    tma_prefetch_2d(&mapX, b * 64, (int)((t0 + j) * kTileTokens));
-                    tma_prefetch_2d(&mapdO, b * 64, (int)((t0 + j) * kTileTokens));
-                    tma_prefetch_2d(&mapY, b * 64, (int)((t0 + j) * kTileTokens));
-                }
-            };
-            for (int j = 1; j < kVbAhead; ++j) prefetch(j);
             for (int it = 0; it < ntiles; ++it) {
                 const int st = it & 1, u = it >> 1;
-                prefetch(it + kVbAhead);
                 if (!mbar_wait(&x_empty[st], (u & 1) ^ 1)) { report_timeout(status, 1201); break; }
                 mbar_arrive_expect_tx(&x_full[st], DV * kTileTokens * 2);
                 for (int b = 0; b < DV / 64; ++b)
