@@ -24,6 +24,12 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ---- registers per thread ------------------------------------------------------------
+// Registers per thread of the calling group of four warps (all four execute it; a multiple of 8): a group that needs few
+// gives some back to the pool of the SM, a group that needs many takes them (and waits until they are there).
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // ---- programmatic dependent launch --------------------------------------------------
 // Every tensor-core kernel is launched with the programmatic-stream-serialization attribute: its blocks may be
 // scheduled while the previous kernel of the stream is still draining, run their set-up (barriers, TMEM, weight
