@@ -99,6 +99,73 @@ def test_two_shards_one_after_the_other(phi, N, cut):
         assert l2(dq2, dq) < 1e-2 and l2(dk2, dk) < 1e-2, (l2(dq2, dq), l2(dk2, dk))
 
 
+class _TwoRanks:
+    """Stands in for torch.distributed with two ranks on one device: `states` holds what each rank's all_gather would
+    deliver (the shards run one after the other, so both states exist before the helper is called)."""
+
+    def __init__(self, rank, states):
+        self.rank, self.states = rank, states
+
+    def is_initialized(self):
+        return True
+
+    def get_world_size(self):
+        return len(self.states)
+
+    def get_rank(self):
+        return self.rank
+
+    def all_gather(self, parts, local):
+        assert torch.equal(local, self.states[self.rank])
+        for dst, src in zip(parts, self.states):
+            dst.copy_(src)
+
+
+@pytest.mark.parametrize("phi,N,cut", [("none", 1000, 437), ("mlp", 1500, 640), ("none", 300, 128)])
+def test_causal_two_shards_one_after_the_other(phi, N, cut):
+    """Causal forward of a sequence cut into two shards: each shard's pass starts from the state of the tokens before
+    it (multi.sharded_causal_forward with the exclusive prefix over the ranks) and gives its slice of the unsharded
+    causal result."""
+    s, Q, K, V, _ = make(phi, N)
+    pq, pk = synth.make_phi_weights(s.d, s.d_phi, s.F, s.dtype)
+    whole = DeviceRun(s, phi, EPS, causal=True)
+    if phi == "mlp":
+        whole.set_weights(pq, pk)
+    O = whole.forward(Q, K, V)
+    io = "bf16" if phi == "mlp" else "f32"
+    shards = []
+    for lo, hi in ((0, cut), (cut, N)):
+        ops = [binding.Hla(1, s.H, hi - lo, s.d, dtype="bf16", phi=phi, eps=EPS, causal=c) for c in (False, True)]
+        if phi == "mlp":
+            for op in ops:
+                op.set_phi(*dev_weights(pq, pk, "bf16"))
+        q = to_dev(np.ascontiguousarray(Q[:, :, lo:hi]), io)
+        k = to_dev(np.ascontiguousarray(K[:, :, lo:hi] if phi == "mlp" else K[:, :, :, lo:hi]), io)
+        v = to_dev(np.ascontiguousarray(V[:, :, lo:hi]), "bf16")
+        shards.append(dict(plain=ops[0], causal=ops[1], q=q, k=k, v=v, o=torch.empty_like(v)))
+    states = []
+    for sh in shards:      # what every rank holds before the all_gather
+        binding.hla_forward_keys(sh["plain"].ctx, sh["k"], sh["v"], sh["plain"].workspace)
+        states.append(sh["plain"].state_region().clone())
+    for r, sh in enumerate(shards):
+        multi.sharded_causal_forward(sh["causal"], sh["plain"], sh["q"], sh["k"], sh["v"], sh["o"], dist=_TwoRanks(r, states))
+    torch.cuda.synchronize()
+    for sh in shards:
+        assert sh["causal"].device_status() == binding.HLA_OK and sh["plain"].device_status() == binding.HLA_OK
+    O2 = np.concatenate([to_np(sh["o"]) for sh in shards], axis=2)
+    assert relerr(O2, O) < 5e-3, relerr(O2, O)
+    if phi == "none":
+        rO, _ = orc.hla_core_forward(f64(Q), f64(K), f64(V), EPS, "causal_quadratic")
+        assert relerr(O2, rO) < TOL["bf16"], relerr(O2, rO)
+    # the first shard starts from nothing: its slice is the causal result of its own tokens, bit for bit
+    first = binding.Hla(1, s.H, cut, s.d, dtype="bf16", phi=phi, eps=EPS, causal=True)
+    if phi == "mlp":
+        first.set_phi(*dev_weights(pq, pk, "bf16"))
+    o1 = first.forward(shards[0]["q"], shards[0]["k"], shards[0]["v"])
+    torch.cuda.synchronize()
+    assert np.array_equal(to_np(o1), to_np(shards[0]["o"]))
+
+
 def test_halves_are_refused_where_they_do_not_exist():
     s, Q, K, V, dO = make("none", 300)
     run = DeviceRun(s, "none", EPS, causal=True)

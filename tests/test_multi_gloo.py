@@ -113,6 +113,60 @@ def test_sequence_sharding_state_sum_two_ranks():
     assert all(r[3] and r[4] for r in res)
 
 
+def _causal_shard_worker(rank, world, port, out):
+    """Causal sequence sharding on the oracle: each rank builds the state of its own tokens, the library's host helper
+    gives it the state of the tokens before its shard (an exclusive prefix over the ranks), and the rank's causal
+    outputs follow from its own sequential pass plus that state (the pass is linear in the state it starts from)."""
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import hla_oracle as orc
+    from paper_2602_12128_b200 import multi
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(11)                     # the same full problem on every rank
+    n, dphi, d, F, eps = 41, 3, 4, 3, 1e-3
+    q = np.abs(rng.standard_normal((n, dphi)))
+    ks = [np.abs(rng.standard_normal((n, dphi))) for _ in range(F)]
+    v = rng.standard_normal((n, d))
+    lo, hi = multi.shard_bounds(n, world, rank)
+    C, z = orc.context_state([k[lo:hi] for k in ks], v[lo:hi])
+    local = torch.from_numpy(np.concatenate([C, z[:, None]], axis=1))
+    before = multi.exclusive_prefix_state(local, dist).numpy()
+    if lo > 0:
+        Cb, zb = orc.context_state([k[:lo] for k in ks], v[:lo])
+    else:
+        Cb, zb = np.zeros_like(C), np.zeros_like(z)
+    ok_prefix = bool(np.allclose(before[:, :d], Cb, rtol=1e-12, atol=1e-12) and np.allclose(before[:, d], zb, rtol=1e-12, atol=1e-12))
+    o_loc, eta_loc = orc.hla_streaming(q[lo:hi], [k[lo:hi] for k in ks], v[lo:hi], eps)
+    Tq = orc.outer_features([q[lo:hi]] * F)
+    eta = eta_loc + Tq @ before[:, d]
+    o = (o_loc * (eta_loc + eps)[:, None] + Tq @ before[:, :d]) / (eta + eps)[:, None]
+    o_full, eta_full = orc.hla_quadratic_causal(q, ks, v, eps)
+    ok_out = bool(np.allclose(o, o_full[lo:hi], rtol=1e-9, atol=1e-12) and np.allclose(eta, eta_full[lo:hi], rtol=1e-10))
+    out.put((rank, lo, hi, ok_prefix, ok_out))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_causal_sequence_sharding_exclusive_prefix(world):
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_causal_shard_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res[0][1] == 0 and res[-1][2] == 41 and all(res[i][2] == res[i + 1][1] for i in range(world - 1))
+    assert all(r[3] and r[4] for r in res)
+
+
 def test_shard_bounds_cover_the_sequence():
     sys.path.insert(0, ROOT)
     from paper_2602_12128_b200 import multi
