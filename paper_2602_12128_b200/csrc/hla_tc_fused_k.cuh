@@ -320,32 +320,33 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
             if (!good) report_timeout(status, 804);
         }
     } else if (warp == kFkZWarp) {
-        // zsym: column sums of the folded key tile as the state product sees it (bf16 values, fp32 sums); lane l owns
-        // the monomials 2 l and 2 l + 1
+        // zsym: column sums of the folded key tile as the state product sees it (bf16 values, fp32 sums).  One 16-byte load
+        // per lane and step: lane l adds the eight monomials of chunk l & 7 over the rows l >> 3, l >> 3 + 4, ... (a second
+        // block of 16 columns: chunk l & 1, rows l >> 1, l >> 1 + 16, ...) and keeps its partial sums for the whole piece;
+        // the lanes' sums meet at the end of the piece, in a fixed order.
         const uint32_t fa = smem_u32(smem + Cfg::kOffF);
-        // (block 0: lane l owns the monomials 2 l, 2 l + 1; the 16 columns of a second block belong to lanes 0..7)
-        float za = 0.f, zb = 0.f, zc = 0.f, zd = 0.f;
+        float z0[8], z1[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z0[e] = z1[e] = 0.f;
+        auto add_chunk = [](float (&z)[8], uint32_t addr) {
+            uint32_t w[4];
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr) : "memory");
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                z[2 * e] += __uint_as_float(w[e] << 16);
+                z[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+            }
+        };
         for (int it = 0; it < nwork; ++it) {
             if (ok && !mbar_wait(f_full, it & 1)) { ok = false; report_timeout(status, 805); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f}, tc_[4] = {0.f, 0.f, 0.f, 0.f}, td[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
-            for (int r = 0; r < kTileTokens; ++r) {
-                uint32_t wv;
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(fa + sw128_off(r, lane >> 2) + (lane & 3) * 4) : "memory");
-                ta[r & 3] += __uint_as_float(wv << 16);
-                tb[r & 3] += __uint_as_float(wv & 0xffff0000u);
-                if (M::kBlocks == 2 && lane < 8) {
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(fa + kBlk + sw128_off(r, lane >> 2) + (lane & 3) * 4) : "memory");
-                    tc_[r & 3] += __uint_as_float(wv << 16);
-                    td[r & 3] += __uint_as_float(wv & 0xffff0000u);
-                }
+            for (int j = 0; j < kTileTokens / 4; ++j) add_chunk(z0, fa + sw128_off((lane >> 3) + 4 * j, lane & 7));
+            if (M::kBlocks == 2) {
+#pragma unroll
+                for (int j = 0; j < kTileTokens / 16; ++j) add_chunk(z1, fa + kBlk + sw128_off((lane >> 1) + 16 * j, lane & 1));
             }
-            za += (ta[0] + ta[1]) + (ta[2] + ta[3]);
-            zb += (tb[0] + tb[1]) + (tb[2] + tb[3]);
-            zc += (tc_[0] + tc_[1]) + (tc_[2] + tc_[3]);
-            zd += (td[0] + td[1]) + (td[2] + td[3]);
             __syncwarp();
             if (lane == 0) mbar_arrive(f_empty);
             if (piece_ends(it)) {
@@ -358,13 +359,24 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
                         for (int c = DV + 1; c < ld; ++c) out[(size_t)m * ld + c] = 0.f;
                     }
                 };
-                put(2 * lane, za);
-                put(2 * lane + 1, zb);
-                if (M::kBlocks == 2 && lane < 8) {
-                    put(64 + 2 * lane, zc);
-                    put(64 + 2 * lane + 1, zd);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float v = z0[e];
+                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                    if (lane < 8) put(8 * lane + e, v);
+                    z0[e] = 0.f;
                 }
-                za = zb = zc = zd = 0.f;
+                if (M::kBlocks == 2) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        float v = z1[e];
+#pragma unroll
+                        for (int o = 2; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (lane < 2) put(64 + 8 * lane + e, v);
+                        z1[e] = 0.f;
+                    }
+                }
             }
         }
     } else if (warp >= kFkFeatWarp0) {
