@@ -17,7 +17,7 @@
 //   warps 3..18   GELU: thread = token row x quarter of the hidden units
 //   warps 19..22  features: ReLU, store k^m, folded key row -> B operand of the state product; drain of a finished piece
 //   warp 23       state product Csym^T += V^T Tsym_k, and the TMA loads of V
-//   warp 24       zsym: column sums of the folded key tile
+//   warps 24..27  zsym: column sums of the folded key tile (16 columns per warp)
 #pragma once
 #include <utility>
 
@@ -26,8 +26,8 @@
 namespace hla {
 namespace tc {
 
-constexpr int kFkThreads = 25 * 32;
-constexpr int kFkGeluWarp0 = 3, kFkFeatWarp0 = 19, kFkStateWarp = 23, kFkZWarp = 24;
+constexpr int kFkThreads = 28 * 32;
+constexpr int kFkGeluWarp0 = 3, kFkFeatWarp0 = 19, kFkStateWarp = 23, kFkZWarp0 = 24, kFkZWarps = 4;
 constexpr int kFkB1Row = 12;        // K row of the staged W2 tiles that carries b1 (rows 6..15 are padding of the second layer)
 
 // TMEM columns (D1[b] at 128 b).  F = 3: D2[b] at 256 + 32 b (16 used), the constant A operand of the bias step (8 columns, K column
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
         mbar_init(v_full, 1);
         mbar_init(v_empty, 1);
         mbar_init(f_full, 128);
-        mbar_init(f_empty, 2);
+        mbar_init(f_empty, 1 + kFkZWarps);
         mbar_init(acc_done, 1);
         mbar_init(acc_free, 128);
         fence_mbar_init();
@@ -319,11 +319,14 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
             }
             if (!good) report_timeout(status, 804);
         }
-    } else if (warp == kFkZWarp) {
-        // zsym: column sums of the folded key tile as the state product sees it (bf16 values, fp32 sums).  One 16-byte load
-        // per lane and step: lane l adds the eight monomials of chunk l & 7 over the rows l >> 3, l >> 3 + 4, ... (a second
-        // block of 16 columns: chunk l & 1, rows l >> 1, l >> 1 + 16, ...) and keeps its partial sums for the whole piece;
-        // the lanes' sums meet at the end of the piece, in a fixed order.
+    } else if (warp >= kFkZWarp0) {
+        // zsym: column sums of the folded key tile as the state product sees it (bf16 values, fp32 sums).  One warp summed
+        // them at first and needed 4500 (three factors) to 10600 (two factors) cycles per tile, as long as the rest of the
+        // tile: a lone warp issues an instruction every five cycles or so.  Now four warps take 16 columns each: one
+        // 16-byte load per lane and step, lane l adds the eight monomials of chunk 2 w + (l & 1) over the rows l >> 1,
+        // l >> 1 + 16, ...; with a second block of 16 columns its two chunks go to warps 0 and 1 (rows l, l + 32, ...).
+        // The lanes keep their partial sums for the whole piece and add them up at its end, in a fixed order.
+        const int zw = warp - kFkZWarp0;
         const uint32_t fa = smem_u32(smem + Cfg::kOffF);
         float z0[8], z1[8];
 #pragma unroll
@@ -337,15 +340,16 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
                 z[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
             }
         };
+        const bool second = M::kBlocks == 2 && zw < 2;
         for (int it = 0; it < nwork; ++it) {
             if (ok && !mbar_wait(f_full, it & 1)) { ok = false; report_timeout(status, 805); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-#pragma unroll 8
-            for (int j = 0; j < kTileTokens / 4; ++j) add_chunk(z0, fa + sw128_off((lane >> 3) + 4 * j, lane & 7));
-            if (M::kBlocks == 2) {
 #pragma unroll
-                for (int j = 0; j < kTileTokens / 16; ++j) add_chunk(z1, fa + kBlk + sw128_off((lane >> 1) + 16 * j, lane & 1));
+            for (int j = 0; j < kTileTokens / 16; ++j) add_chunk(z0, fa + sw128_off((lane >> 1) + 16 * j, 2 * zw + (lane & 1)));
+            if (second) {
+#pragma unroll
+                for (int j = 0; j < kTileTokens / 32; ++j) add_chunk(z1, fa + kBlk + sw128_off(lane + 32 * j, zw));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(f_empty);
@@ -362,18 +366,18 @@ __global__ void __launch_bounds__(kFkThreads, 1) tc_phik_state_kernel(const __gr
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     float v = z0[e];
-                    v += __shfl_xor_sync(0xffffffffu, v, 8);
-                    v += __shfl_xor_sync(0xffffffffu, v, 16);
-                    if (lane < 8) put(8 * lane + e, v);
+#pragma unroll
+                    for (int o = 2; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (lane < 2) put(8 * (2 * zw + lane) + e, v);
                     z0[e] = 0.f;
                 }
-                if (M::kBlocks == 2) {
+                if (M::kBlocks == 2) {      // (every warp runs the shuffles; warps 2 and 3 hold zeros)
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         float v = z1[e];
 #pragma unroll
-                        for (int o = 2; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                        if (lane < 2) put(64 + 8 * lane + e, v);
+                        for (int o = 1; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (second && lane == 0) put(64 + 8 * zw + e, v);
                         z1[e] = 0.f;
                     }
                 }
