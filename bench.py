@@ -82,10 +82,8 @@ def kernel_models(shape):
 
 # DRAM traffic per token-head of a launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # scaled by token-heads; see profiles/).  None = not captured yet.
-NCU_TRAFFIC_PER_TOKEN_HEAD = {
-    "tc_phik_state": 584.9, "tc_state_build": 333.0, "tc_phiq_readout": 475.5, "tc_bwd_query": 303.4, "tc_bwd_key": 593.7,
-    "tc_phi_backward_q": 500.5, "tc_phi_backward_k": 616.2,
-}
+NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_phik_state": 586.7, "tc_state_build": 333.0, "tc_phiq_readout": 476.9, "tc_bwd_query": 304.3, "tc_bwd_key": 594.4,
+                              "tc_phi_backward_q": 499.6, "tc_phi_backward_k": 616.1}
 
 
 class ClockSampler:
