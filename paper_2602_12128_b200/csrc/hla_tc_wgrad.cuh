@@ -13,7 +13,7 @@
 // CTA order, so the result is bit-reproducible.
 //
 // warp 0: TMA loads, warp 1: dg, dW1 and dW2 MMAs, warp 2: h MMAs, warps 3..18: arithmetic (thread = token row x quarter
-// of the hidden units), warps 19..20: column sums of the dh tile (db1), warps 21..24: dp tiles and db2 (thread = token row;
+// of the hidden units), warps 19..22: column sums of the dh tile (db1), warps 23..26: dp tiles and db2 (thread = token row;
 // off the arithmetic warps' instruction stream, which is what bounds the kernel).
 #pragma once
 #include "hla_tc_phi.cuh"
@@ -21,8 +21,8 @@
 namespace hla {
 namespace tc {
 
-constexpr int kWgThreads = 25 * 32;
-constexpr int kWgEpiWarp0 = 3, kWgSumWarp0 = 19, kWgDpWarp0 = 21;
+constexpr int kWgThreads = 27 * 32;
+constexpr int kWgEpiWarp0 = 3, kWgSumWarp0 = 19, kWgDpWarp0 = 23;
 constexpr int kWgColDg = 128, kWgColW1 = 256, kWgColW2 = 384;      // TMEM columns (h at 0)
 
 template <int DV, int NMAPS, int DP> struct WgCfg {
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
         mbar_init(dg_full, 1);
         mbar_init(dg_empty, 512);
         mbar_init(gd_full, 512);
-        mbar_init(gd_empty, 1 + DV / 64);
+        mbar_init(gd_empty, 1 + DV / 32);
         mbar_init(acc_full, 1);
         mbar_init(acc_empty, 512);
         fence_mbar_init();
@@ -216,34 +216,45 @@ __global__ void __launch_bounds__(kWgThreads, 1) tc_phi_wgrad_kernel(const __gri
             if (!good) report_timeout(status, 1004);
         }
     } else if (warp >= kWgSumWarp0 && warp < kWgDpWarp0) {
-        // db1: column sums of the dh tile as the dW1 product sees it (bf16 values, fp32 sums); warp w owns the 64-column
-        // block w, lane l its columns 2 l and 2 l + 1
-        const int blk = warp - kWgSumWarp0;
-        if (blk < DV / 64) {
-            const uint32_t da = smem_u32(smem + Cfg::kOffDh) + blk * kBlk;
-            float sa = 0.f, sb = 0.f;
+        // db1: column sums of the dh tile as the dW1 product sees it (bf16 values, fp32 sums).  Warp w owns the 32 hidden
+        // units 32 w ..: one 16-byte load per lane and step, lane l adds the eight columns of chunk 4 w + (l & 3) over the
+        // rows l >> 2, l >> 2 + 8, ... and keeps its partial sums for the whole map; the lanes' sums meet after the map's last
+        // tile, in a fixed order.  (Two warps with one 4-byte load per row took as long as a whole unit: a lone warp issues
+        // an instruction every five cycles or so.)
+        const int sw = warp - kWgSumWarp0;
+        if (sw < DV / 32) {
+            const uint32_t da = smem_u32(smem + Cfg::kOffDh) + (sw >> 1) * kBlk;
+            const int chunk = 4 * (sw & 1) + (lane & 3);
+            float sm[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sm[e] = 0.f;
             for (int unit = 0; unit < nunits; ++unit) {
                 const int m = unit / ntiles, it = unit - m * ntiles;
                 if (ok && !mbar_wait(gd_full, unit & 1)) { ok = false; report_timeout(status, 1005); }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
-                for (int r = 0; r < kTileTokens; ++r) {
-                    uint32_t wv;
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wv) : "r"(da + sw128_off(r, lane >> 2) + (lane & 3) * 4) : "memory");
-                    ta[r & 3] += __uint_as_float(wv << 16);
-                    tb[r & 3] += __uint_as_float(wv & 0xffff0000u);
+                for (int j = 0; j < kTileTokens / 8; ++j) {
+                    uint32_t w[4];
+                    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(da + sw128_off((lane >> 2) + 8 * j, chunk)) : "memory");
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        sm[2 * e] += __uint_as_float(w[e] << 16);
+                        sm[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                    }
                 }
-                sa += (ta[0] + ta[1]) + (ta[2] + ta[3]);
-                sb += (tb[0] + tb[1]) + (tb[2] + tb[3]);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(gd_empty);
                 if (it == ntiles - 1) {
-                    float* o = out_cta + (size_t)m * Cfg::kPartFloats + Cfg::kPartB1 + blk * 64 + 2 * lane;
-                    o[0] = sa;
-                    o[1] = sb;
-                    sa = sb = 0.f;
+                    float* o = out_cta + (size_t)m * Cfg::kPartFloats + Cfg::kPartB1 + (sw >> 1) * 64 + 8 * chunk;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        float v = sm[e];
+#pragma unroll
+                        for (int x = 4; x < 32; x <<= 1) v += __shfl_xor_sync(0xffffffffu, v, x);
+                        if (lane < 4) o[e] = v;
+                        sm[e] = 0.f;
+                    }
                 }
             }
         }
