@@ -1150,7 +1150,8 @@ template <int DV, int F> struct BkCfg {
     static constexpr int kOffO = kOffBq + ((2 * kBqBlock + 1023) / 1024) * 1024;
     static constexpr int kOBytes = kTileTokens * DV * 2;
     static constexpr int kOffBars = kOffO + (kStagedOut ? 2 * kOBytes : 0);
-    static constexpr int kSmemUsed = 1024 + kOffBars + 256;
+    static constexpr int kOffDz = kOffBars + 256;                         // float [2 groups][128]: dzsym of the group's current head
+    static constexpr int kSmemUsed = 1024 + kOffDz + 1024;
     static_assert(kSmemUsed <= 227 * 1024, "shared memory");
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;
     static constexpr int kColD4 = 256, kD4Stride = F == 3 ? 64 : 96;      // TMEM: D3[grp] at 128 grp, D4[grp] at 256 + stride grp
@@ -1273,10 +1274,18 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
             for (int f = 0; f < F; ++f) load_feat<M::kDphi>(kn + M::kDphi * f, kf + (((size_t)bh * F + f) * N + tok) * M::kDphi);
         };
         if (grp < nwork) prefetch(grp);
+        float* dzs = reinterpret_cast<float*>(smem + Cfg::kOffDz) + grp * 128;
+        int cur_bh = -1;
         for (int it = grp; it < nwork; it += 2) {
             const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
             const int u = it >> 1;
             const int tok = tile * kTileTokens + row;
+            if (bh != cur_bh) {      // dzsym of the head, once per head and group instead of 56 global loads per thread and tile
+                named_barrier(1 + grp, 128);
+                if (row < M::kN) dzs[row] = __ldg(dstate + (size_t)bh * M::kN * ld + DV + (size_t)row * ld);
+                named_barrier(1 + grp, 128);
+                cur_bh = bh;
+            }
             float k[M::kKf];
 #pragma unroll
             for (int i = 0; i < M::kKf; ++i) k[i] = tok < N ? kn[i] : 0.f;
@@ -1296,7 +1305,6 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                 tc_fence_after();
                 float G[M::kN];
                 const uint32_t ta = tmem + Cfg::kColD4 + Cfg::kD4Stride * grp + ((uint32_t)(quarter * 32) << 16);
-                const float* dz = dstate + (size_t)bh * M::kN * ld + DV;
 #pragma unroll
                 for (int c = 0; c < (M::kN + 7) / 8; ++c) {
                     uint32_t rr[8];
@@ -1304,7 +1312,7 @@ __global__ void __launch_bounds__(kBkThreads, 1) tc_bwd_key_kernel(const __grid_
                     tmem_ld_wait();
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
-                        if (8 * c + e < M::kN) G[8 * c + e] = __uint_as_float(rr[e]) + __ldg(dz + (size_t)(8 * c + e) * ld);
+                        if (8 * c + e < M::kN) G[8 * c + e] = __uint_as_float(rr[e]) + dzs[8 * c + e];
                 }
                 float dk[M::kKf];
                 key_folded_grad_t<F>(k, G, dk);
