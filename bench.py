@@ -82,7 +82,7 @@ def kernel_models(shape):
 
 # DRAM traffic per token-head of a launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # scaled by token-heads; see profiles/).  None = not captured yet.
-NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_phik_state": 586.7, "tc_state_build": 333.0, "tc_phiq_readout": 476.9, "tc_bwd_query": 304.3, "tc_bwd_key": 594.4,
+NCU_TRAFFIC_PER_TOKEN_HEAD = {"tc_phik_state": 586.7, "tc_state_build": 333.0, "tc_phiq_readout": 476.9, "tc_bwd_query": 304.3, "tc_bwd_key": 594.3,
                               "tc_phi_backward_q": 499.6, "tc_phi_backward_k": 616.1}
 
 
