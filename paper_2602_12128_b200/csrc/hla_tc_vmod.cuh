@@ -132,7 +132,7 @@ template <int DV, bool COMBINE> struct VfCfg {
     static constexpr int kWBytes = DV * DV * 2;
     static constexpr int kAuxBytes = (DV / 64) * 2048;           // [16 K rows][DV] bf16
     static constexpr int kOffX = 0;
-    static constexpr int kOffE = kXStages * kXBytes;             // COMBINE: [T tile | Y2 tile -> Out tile]; else the Out tile
+    static constexpr int kOffE = kXStages * kXBytes;             // COMBINE: two Y2 tiles (-> Out tiles), by tile parity; else the Out tile
     static constexpr int kEBytes = (COMBINE ? 2 : 1) * kXBytes;
     static constexpr int kOffW1 = kOffE + kEBytes;
     static constexpr int kOffW2 = kOffW1 + kWBytes;
@@ -167,9 +167,9 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
     uint64_t* d2_full = bars + 14;     // MMA commit
     uint64_t* d2_empty = bars + 15;    // 128 arrivals
     uint64_t* w_full = bars + 16;      // TMA
-    uint64_t* e_ready = bars + 17;     // the output tile may be used: TMA (COMBINE: its two input tiles have landed) or one arrival
+    uint64_t* e_ready = bars + 19;     // [2] COMBINE: the Y2 tile of that parity has landed (TMA); else [0]: one arrival, the output tile may be used
     uint64_t* o_full = bars + 18;      // 128 arrivals: the output tile is written
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 21);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long tiles = (rows + kTileTokens - 1) / kTileTokens;
@@ -179,9 +179,10 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
     if (tid == 0) {
         for (int i = 0; i < 3; ++i) {
             mbar_init(&x_full[i], 1);
-            mbar_init(&x_empty[i], 1);
+            mbar_init(&x_empty[i], COMBINE ? 128 : 1);      // COMBINE: the output warps read T from the X tile
         }
         for (int i = 0; i < 2; ++i) {
+            mbar_init(&e_ready[i], 1);
             mbar_init(&st_full[i], 128);
             mbar_init(&d1_full[i], 1);
             mbar_init(&g_full[i], 512);
@@ -190,7 +191,6 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
         mbar_init(d2_full, 1);
         mbar_init(d2_empty, 128);
         mbar_init(w_full, 1);
-        mbar_init(e_ready, 1);
         mbar_init(o_full, 128);
         fence_mbar_init();
         prefetch_tmap(&mapX);
@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
                     umma_bf16(tmem + 128 * b, desc_advance(xd, (ks >> 2) * kBlk + (ks & 3) * 32), desc_advance(wd, ks * 2048), idesc1, ks > 0 ? 1u : 0u);
                 umma_bf16_ta(tmem + 128 * b, tmem + kVfColAug + 8 * b, ad, idesc1, 1u);
                 umma_commit(&d1_full[b]);
-                umma_commit(&x_empty[st]);
+                if (!COMBINE) umma_commit(&x_empty[st]);
             }
             if (!good) report_timeout(status, 1102);
         }
@@ -276,36 +276,41 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
             if (!good) report_timeout(status, 1103);
         }
     } else if (warp >= kVfOutWarp0) {
-        // Out = y (or T + y (.) Y2): thread = token row; the result tile is formed in shared memory and stored by TMA
+        // Out = y (or T + y (.) Y2): thread = token row; the result tile is formed in shared memory and stored by TMA.
+        // COMBINE: T is read from the X tile the map was computed from (the tile stays until this pass is done with it), Y2
+        // comes by TMA into one of two tiles (by tile parity) a whole tile ahead, and the result is written over it.
         const int quarter = warp & 3, row = quarter * 32 + lane;
         const bool leader = warp == kVfOutWarp0 && lane == 0;
         const uint32_t ta = tmem + kVfColD2 + ((uint32_t)(quarter * 32) << 16);
-        const uint32_t et = smem_u32(smem + Cfg::kOffE);                        // COMBINE: T tile
-        const uint32_t ot = et + (COMBINE ? Cfg::kXBytes : 0);                  // COMBINE: Y2 tile, overwritten by the result
-        auto open_tile = [&](int it) {      // leader only: the output tile is free; COMBINE fetches its two input tiles
+        auto open_tile = [&](int it) {      // leader only: the tile of that parity is free; COMBINE fetches Y2 into it
             if (COMBINE) {
-                mbar_arrive_expect_tx(e_ready, 2 * DV * kTileTokens * 2);
-                for (int b = 0; b < DV / 64; ++b) {
-                    tma_load_2d(smem + Cfg::kOffE + b * kBlk, &mapX, e_ready, b * 64, (int)((t0 + it) * kTileTokens));
-                    tma_load_2d(smem + Cfg::kOffE + Cfg::kXBytes + b * kBlk, &mapY2, e_ready, b * 64, (int)((t0 + it) * kTileTokens));
-                }
+                mbar_arrive_expect_tx(&e_ready[it & 1], DV * kTileTokens * 2);
+                for (int b = 0; b < DV / 64; ++b)
+                    tma_load_2d(smem + Cfg::kOffE + (it & 1) * Cfg::kXBytes + b * kBlk, &mapY2, &e_ready[it & 1], b * 64, (int)((t0 + it) * kTileTokens));
             } else {
-                mbar_arrive(e_ready);
+                mbar_arrive(&e_ready[0]);
             }
         };
         if (leader && ntiles > 0) open_tile(0);
         for (int it = 0; it < ntiles; ++it) {
+            const int eb = COMBINE ? (it & 1) : 0, epar = COMBINE ? ((it >> 1) & 1) : (it & 1);
+            if (COMBINE && leader && it + 1 < ntiles) {
+                tma_store_wait_read0();      // the store of tile it - 1 has read the tile of the other parity
+                open_tile(it + 1);
+            }
             if (ok && !mbar_wait(d2_full, it & 1)) { ok = false; report_timeout(status, 1104); }
-            if (ok && !mbar_wait(e_ready, it & 1)) { ok = false; report_timeout(status, 1108); }
+            if (ok && !mbar_wait(&e_ready[eb], epar)) { ok = false; report_timeout(status, 1108); }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            const uint32_t xt = smem_u32(smem + Cfg::kOffX + (it % XST) * Cfg::kXBytes);      // COMBINE: T tile
+            const uint32_t ot = smem_u32(smem + Cfg::kOffE + eb * Cfg::kXBytes);              // Y2 tile, overwritten by the result
 #pragma unroll 2
             for (int c = 0; c < DV / 16; ++c) {
                 uint32_t r[16], xw[8], yw[8], w[8];
                 tmem_ld16(ta + 16 * c, r);
                 if (COMBINE) {
-                    lds_row16(et, row, c, xw);
+                    lds_row16(xt, row, c, xw);
                     lds_row16(ot, row, c, yw);
                 }
                 tmem_ld_wait();
@@ -322,14 +327,17 @@ __global__ void __launch_bounds__(kVfThreads, 1) tc_vmlp_forward_kernel(const __
             }
             tc_fence_before();
             mbar_arrive(d2_empty);
+            if (COMBINE) mbar_arrive(&x_empty[it % XST]);
             fence_proxy_async();
             mbar_arrive(o_full);
             if (leader) {
                 if (mbar_wait(o_full, it & 1)) {
-                    for (int b = 0; b < DV / 64; ++b) tma_store_2d(&mapOut, smem + Cfg::kOffE + (COMBINE ? Cfg::kXBytes : 0) + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
+                    for (int b = 0; b < DV / 64; ++b) tma_store_2d(&mapOut, smem + Cfg::kOffE + eb * Cfg::kXBytes + b * kBlk, b * 64, (int)((t0 + it) * kTileTokens));
                     tma_store_commit();
-                    tma_store_wait_read0();
-                    if (it + 1 < ntiles) open_tile(it + 1);
+                    if (!COMBINE) {
+                        tma_store_wait_read0();
+                        if (it + 1 < ntiles) open_tile(it + 1);
+                    }
                 } else {
                     report_timeout(status, 1109);
                 }
