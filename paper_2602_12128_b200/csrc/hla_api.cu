@@ -403,10 +403,10 @@ hla_status forward_impl(hla_ctx* ctx, const void* Q, const void* K, const void* 
                 s = tc::emit_from_state(ctx->tcp, ctx->D, ctx->BH, ws, ctx->L, false, ctx->rec);
                 if (s != HLA_OK) return s;
             }
-            s = tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec);
+            // causal: only the feature map of the query side runs (no readout), which leaves the features of both sides in the
+            // workspace; the pieces of the key-side kernel become the pieces of the sweep
+            s = tc::phiq_readout(ctx->tcp, ctx->D, ctx->BH, &ctx->phi_q, Q, O, ws, ctx->L, ctx->sm_count, ctx->rec, !ctx->cfg.causal);
             if (s != HLA_OK || !ctx->cfg.causal) return s;
-            // causal: the pass above left the features of both sides in the workspace (its O is overwritten now); the
-            // pieces of the key-side kernel become the pieces of the sweep
             return tc::causal_sweep(ctx->D, ctx->BH, reinterpret_cast<const float*>(ws + ctx->L.qf), reinterpret_cast<const float*>(ws + ctx->L.kf), V, O,
                                     ws, ctx->L, ctx->off_part, ctx->k_pieces, tc::fused_key_grid(ctx->BH, ctx->D.N, ctx->sm_count), ctx->carry, ctx->rec);
         } else {

@@ -46,8 +46,10 @@ template <int DV, int F> struct FqCfg {
     static constexpr int kSmem = kSmemUsed > 120 * 1024 ? kSmemUsed : 120 * 1024;   // one CTA per SM (512 TMEM columns)
 };
 
-// Q [BH][N][DV] bf16 (3-D map, rows past N read as zero), O the same (stores are clipped at N).
-template <int DV, int F>
+// Q [BH][N][DV] bf16 (3-D map, rows past N read as zero), O the same (stores are clipped at N).  READOUT = false: the feature
+// map only (the causal operator reads its states tile by tile in a sweep of its own and needs just the query features):
+// the readout product, its epilogue and the monomial tile are left out, O and eta are not written.
+template <int DV, int F, bool READOUT = true>
 __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapW1,
                                                                         const __grid_constant__ CUtensorMap mapB3, const __grid_constant__ CUtensorMap mapO,
                                                                         const __nv_bfloat16* __restrict__ b1g, const __nv_bfloat16* __restrict__ W2g,
@@ -194,7 +196,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             if (!good) report_timeout(status, 703);
         }
     } else if (warp == kFqReadoutMmaWarp) {
-        if (lane == 0 && nwork > 0) {      // [num | eta] = monomial tile * state operand of the tile's head
+        if (READOUT && lane == 0 && nwork > 0) {      // [num | eta] = monomial tile * state operand of the tile's head
             const uint32_t idesc3 = idesc_bf16(128, Cfg::kNmma, false, false);   // monomial tile K-major, state operand K-major over the monomials
             const uint64_t ad = smem_desc_sw128(smem_u32(smem + Cfg::kOffA), 16, 1024);
             const uint64_t bd = smem_desc_sw128(smem_u32(smem + Cfg::kOffB3), 16, 1024);
@@ -231,7 +233,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
         const bool leader = warp == kFqOutWarp0 && lane == 0;
         const uint32_t ta = tmem + 320 + ((uint32_t)(quarter * 32) << 16);
         const uint32_t os = smem_u32(smem + Cfg::kOffO);
-        for (int it = 0; it < nwork; ++it) {
+        for (int it = 0; READOUT && it < nwork; ++it) {
             const int work = w0 + it, bh = work / tiles_per_head, tile = work % tiles_per_head;
             if (ok && !mbar_wait(acc_full, it & 1)) { ok = false; report_timeout(status, 704); }
             ok = __all_sync(0xffffffffu, ok);
@@ -271,7 +273,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
             const int tok = tile * kTileTokens + row;
             if (ok && tok < N) eta_out[(size_t)bh * N + tok] = eta;
         }
-        if (leader) tma_store_wait_all0();
+        if (READOUT && leader) tma_store_wait_all0();
     } else if (warp >= kFqFeatWarp0) {
         // q = ReLU(D2 + b2) -> global memory (kept for the backward); monomial row -> A operand of the readout product
         const int quarter = warp & 3, row = quarter * 32 + lane;
@@ -293,6 +295,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
 #pragma unroll
             for (int o = 0; o < DP; ++o) q[o] = tok < N ? fmaxf(__uint_as_float(r[o]) + b2s[o], 0.f) : 0.f;
             if (tok < N) store_feat<DP>(qf_out + ((size_t)bh * N + tok) * DP, q);
+            if (!READOUT) continue;
             float mono[M::kN];
             query_monomials_t<F>(q, mono);
             if (!mbar_wait(a_empty, (it & 1) ^ 1)) { ok = false; report_timeout(status, 706); }
@@ -340,7 +343,7 @@ __global__ void __launch_bounds__(kFqThreads, 1) tc_phiq_readout_kernel(const __
     if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-template <int DV, int F>
+template <int DV, int F, bool READOUT>
 inline hla_status launch_phiq_readout(const Plan& P, const Dims& D, int BH, const hla_mlp* phi_q, const void* Q, void* O, char* ws,
                                       const hla_ws_layout& L, int sm_count, LaunchRec& rec) {
     CUtensorMap mapQ, mapW1, mapB3, mapO;
@@ -348,12 +351,12 @@ inline hla_status launch_phiq_readout(const Plan& P, const Dims& D, int BH, cons
     if (!make_map_bhnd(&mapQ, Q, BH, D.N, DV, kTileTokens) || !make_map_bhnd(&mapO, O, BH, D.N, DV, kTileTokens) ||
         !make_map_2d(&mapW1, phi_q->W1, DV, DV, DV) || !make_map_2d(&mapB3, b3, (size_t)BH * (DV + 16), MT<F>::kPad, DV + 16))
         return HLA_ERR_CUDA;
-    if (!set_smem(tc_phiq_readout_kernel<DV, F>, FqCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
+    if (!set_smem(tc_phiq_readout_kernel<DV, F, READOUT>, FqCfg<DV, F>::kSmem)) return HLA_ERR_CUDA;
     const int tiles = (D.N + kTileTokens - 1) / kTileTokens;
     const long long total = (long long)BH * tiles;
     const int grid = (int)(total < sm_count ? total : sm_count);
-    rec.begin("tc_phiq_readout");
-    launch_pdl(tc_phiq_readout_kernel<DV, F>, grid, dim3(kFqThreads), FqCfg<DV, F>::kSmem, rec.st,
+    rec.begin(READOUT ? "tc_phiq_readout" : "tc_phiq");
+    launch_pdl(tc_phiq_readout_kernel<DV, F, READOUT>, grid, dim3(kFqThreads), FqCfg<DV, F>::kSmem, rec.st,
         mapQ, mapW1, mapB3, mapO, static_cast<const __nv_bfloat16*>(phi_q->b1), static_cast<const __nv_bfloat16*>(phi_q->W2),
         static_cast<const __nv_bfloat16*>(phi_q->b2), reinterpret_cast<float*>(ws + L.qf), reinterpret_cast<float*>(ws + L.eta), D.N, BH, D.eps,
         reinterpret_cast<int*>(ws + L.status));
@@ -361,13 +364,18 @@ inline hla_status launch_phiq_readout(const Plan& P, const Dims& D, int BH, cons
 }
 
 inline hla_status phiq_readout(const Plan& P, const Dims& D, int BH, const hla_mlp* phi_q, const void* Q, void* O, char* ws, const hla_ws_layout& L,
-                               int sm_count, LaunchRec& rec) {
+                               int sm_count, LaunchRec& rec, bool readout = true) {
     if (D.F == 3) {
-        if (D.d == 128) return launch_phiq_readout<128, 3>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
-        return launch_phiq_readout<64, 3>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+        if (!readout) {
+            if (D.d == 128) return launch_phiq_readout<128, 3, false>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+            return launch_phiq_readout<64, 3, false>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+        }
+        if (D.d == 128) return launch_phiq_readout<128, 3, true>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+        return launch_phiq_readout<64, 3, true>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
     }
-    if (D.d == 128) return launch_phiq_readout<128, 2>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
-    return launch_phiq_readout<64, 2>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+    if (!readout) return HLA_ERR_UNSUPPORTED;
+    if (D.d == 128) return launch_phiq_readout<128, 2, true>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
+    return launch_phiq_readout<64, 2, true>(P, D, BH, phi_q, Q, O, ws, L, sm_count, rec);
 }
 
 }  // namespace tc
